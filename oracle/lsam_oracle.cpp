@@ -1,0 +1,513 @@
+// lsam_oracle.cpp -- CPU oracle (TEST INFRASTRUCTURE ONLY; see lsam_oracle.h).
+//
+// Written from the paper's statement of the method:
+//   * SAM perturbation  x~ = x + rho * grad f(x; xi) / (||grad f(x; xi)|| + gamma)      (Eq. 3, look-back map)
+//   * SAM gradient      g  = grad f(x~; xi), the SAME minibatch xi in both passes        (Theorems 3 and 4)
+//   * worker score      G  = g + lambda (x - y)                                          (Algorithm 1, first update)
+//   * sampler           Nesterov-momentum step on G                                      (Section 4.3)
+//   * centre update     g' = (1/(n tau)) sum_i sum_s x_s^(i) - y ;  g = g' + beta (g' - g'_prev) ;
+//                       y <- y + eta' g ; counters reset                                 (Algorithm 2, sync branch)
+// All arithmetic is double.  Loops are written in the order of the definitions; the only
+// parallelism is OpenMP over the independent replicas.
+#include "lsam_oracle.h"
+
+#include <cmath>
+#include <cstring>
+#include <vector>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+namespace {
+
+// ---- schedule hash: splitmix64 finaliser (Steele, Lea, Flood 2014), chained over (seed^tag, t, k*2^20+j)
+inline uint64_t mix64(uint64_t z) {
+  z = (z ^ (z >> 30)) * 0xbf58476d1ce4e5b9ULL;
+  z = (z ^ (z >> 27)) * 0x94d049bb133111ebULL;
+  return z ^ (z >> 31);
+}
+const uint64_t TAG_IDX = 0x6c73616d5f696478ULL;    // ASCII "lsam_idx"
+const uint64_t TAG_STALE = 0x6c73616d5f73746cULL;  // ASCII "lsam_stl"
+inline uint64_t hash5(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j) {
+  return mix64(mix64(mix64(seed ^ tag) + t) + ((k << 20) + j));
+}
+
+// ---- bf16 round-to-nearest-even of an fp32 value (published format: 1-8-7, top half of binary32)
+inline float bf16_round(float v) {
+  uint32_t u;
+  std::memcpy(&u, &v, 4);
+  if ((u & 0x7f800000u) == 0x7f800000u) return v;  // inf / nan unchanged
+  uint32_t lsb = (u >> 16) & 1u;
+  u += 0x7fffu + lsb;
+  u &= 0xffff0000u;
+  float r;
+  std::memcpy(&r, &u, 4);
+  return r;
+}
+
+struct Layer {
+  int in, out;
+  int64_t w_off, b_off;  // offsets in the unpadded parameter vector; b_off = -1: no bias
+  bool residual;         // h_next = h + relu(W h + b)
+};
+
+struct Net {
+  int model = 0;
+  bool bf16 = false;
+  std::vector<Layer> layers;
+  int64_t d = 0;
+  int in0 = 0;
+
+  double q(double v) const { return bf16 ? (double)bf16_round((float)v) : v; }
+};
+
+bool build_net(const oracle_config& c, Net& net) {
+  net.model = c.model;
+  net.bf16 = (c.gemm_dtype == ORACLE_GEMM_BF16);
+  net.layers.clear();
+  if (c.K < 1) return false;
+  if (c.model == ORACLE_MODEL_FLAT) {
+    if (c.flat_d < 1) return false;
+    net.d = c.flat_d;
+    return true;
+  }
+  if (c.batch < 1 || c.n_samples < 1) return false;
+  if (c.model == ORACLE_MODEL_LSQ) {
+    if (c.widths[0] < 1) return false;
+    net.in0 = c.widths[0];
+    net.layers.push_back({c.widths[0], 1, 0, -1, false});
+    net.d = c.widths[0];
+    return true;
+  }
+  if (c.model != ORACLE_MODEL_MLP && c.model != ORACLE_MODEL_RESMLP) return false;
+  if (c.n_layers < 1 || c.n_layers > 8) return false;
+  int64_t off = 0;
+  for (int l = 0; l < c.n_layers; ++l) {
+    Layer L;
+    L.in = c.widths[l];
+    L.out = c.widths[l + 1];
+    if (L.in < 1 || L.out < 1) return false;
+    L.w_off = off;
+    off += (int64_t)L.in * L.out;
+    L.b_off = off;
+    off += L.out;
+    // residual MLP: every hidden layer whose input and output widths agree carries a skip connection
+    L.residual = (c.model == ORACLE_MODEL_RESMLP) && (l < c.n_layers - 1) && (L.in == L.out);
+    net.layers.push_back(L);
+  }
+  net.d = off;
+  net.in0 = c.widths[0];
+  return true;
+}
+
+// Mean loss over the minibatch and its gradient.  a0: [B, in0] inputs (already rounded in bf16 mode).
+// If logits_out != nullptr only the forward pass is run and the head outputs are returned.
+double net_loss_grad(const Net& net, const double* params, const std::vector<double>& a0, int B,
+                     const float* y_f, const int32_t* y_i, const int32_t* idx, double* grad, double* logits_out) {
+  const int L = (int)net.layers.size();
+  if (net.model == ORACLE_MODEL_LSQ) {
+    // f = (1/(2B)) sum_b (a_b . w - y_b)^2 ;  grad = (1/B) sum_b (a_b . w - y_b) a_b
+    const int n = net.in0;
+    std::vector<double> r(B);
+    double loss = 0.0;
+    for (int b = 0; b < B; ++b) {
+      double p = 0.0;
+      for (int i = 0; i < n; ++i) p += a0[(size_t)b * n + i] * params[i];
+      if (logits_out) logits_out[b] = p;
+      r[b] = logits_out ? 0.0 : p - (double)y_f[idx[b]];
+      loss += r[b] * r[b];
+    }
+    if (logits_out) return 0.0;
+    loss /= (2.0 * B);
+    for (int i = 0; i < n; ++i) {
+      double s = 0.0;
+      for (int b = 0; b < B; ++b) s += r[b] * a0[(size_t)b * n + i];
+      grad[i] = s / B;
+    }
+    return loss;
+  }
+
+  // operand copy of the parameters (bf16 mode: every weight and bias rounded once; fp32 mode: unchanged)
+  std::vector<double> pq((size_t)net.d);
+  for (int64_t e = 0; e < net.d; ++e) pq[(size_t)e] = net.q(params[e]);
+
+  // ---- forward
+  std::vector<std::vector<double>> h(L + 1);       // h[l]: input of layer l, [B, in_l]
+  std::vector<std::vector<unsigned char>> mask(L);  // mask[l][b*out+o] = (pre-activation > 0), hidden layers
+  h[0] = a0;
+  std::vector<double> logits;
+  for (int l = 0; l < L; ++l) {
+    const Layer& ly = net.layers[l];
+    const bool head = (l == L - 1);
+    std::vector<double> z((size_t)B * ly.out);
+    for (int b = 0; b < B; ++b)
+      for (int o = 0; o < ly.out; ++o) {
+        const double* w = pq.data() + ly.w_off + (int64_t)o * ly.in;
+        const double* a = h[l].data() + (size_t)b * ly.in;
+        double s = 0.0;
+        for (int i = 0; i < ly.in; ++i) s += w[i] * a[i];
+        z[(size_t)b * ly.out + o] = s + pq[(size_t)(ly.b_off + o)];
+      }
+    if (head) {
+      logits.swap(z);
+    } else {
+      mask[l].resize((size_t)B * ly.out);
+      h[l + 1].resize((size_t)B * ly.out);
+      for (size_t e = 0; e < z.size(); ++e) {
+        const double r = z[e] > 0.0 ? z[e] : 0.0;
+        mask[l][e] = z[e] > 0.0;
+        const double skip = ly.residual ? h[l][e] : 0.0;  // in == out for residual layers
+        h[l + 1][e] = net.q(skip + r);                     // stored activation (bf16 mode: rounded)
+      }
+    }
+  }
+  const int C = net.layers[L - 1].out;
+  if (logits_out) {
+    std::memcpy(logits_out, logits.data(), sizeof(double) * (size_t)B * C);
+    return 0.0;
+  }
+
+  // ---- softmax cross-entropy, mean over the batch
+  double loss = 0.0;
+  std::vector<double> dz((size_t)B * C);
+  for (int b = 0; b < B; ++b) {
+    const double* lg = logits.data() + (size_t)b * C;
+    double m = lg[0];
+    for (int c = 1; c < C; ++c) m = lg[c] > m ? lg[c] : m;
+    double se = 0.0;
+    for (int c = 0; c < C; ++c) se += std::exp(lg[c] - m);
+    const int y = y_i[idx[b]];
+    loss += (m + std::log(se)) - lg[y];
+    for (int c = 0; c < C; ++c) {
+      const double p = std::exp(lg[c] - m) / se;
+      dz[(size_t)b * C + c] = net.q((p - (c == y ? 1.0 : 0.0)) / B);
+    }
+  }
+  loss /= B;
+
+  // ---- backward: dz = gradient w.r.t. the pre-activation of layer l; dh = gradient w.r.t. its input
+  std::vector<double> dh_next;  // gradient w.r.t. h[l+1] (needed by residual layers)
+  for (int l = L - 1; l >= 0; --l) {
+    const Layer& ly = net.layers[l];
+    for (int o = 0; o < ly.out; ++o) {
+      double sb = 0.0;
+      for (int b = 0; b < B; ++b) sb += dz[(size_t)b * ly.out + o];
+      grad[ly.b_off + o] = sb;
+      // dW[o][i] = sum_b dz[b][o] h[b][i], samples added in ascending order
+      double* gw = grad + ly.w_off + (int64_t)o * ly.in;
+      for (int i = 0; i < ly.in; ++i) gw[i] = 0.0;
+      for (int b = 0; b < B; ++b) {
+        const double dzbo = dz[(size_t)b * ly.out + o];
+        const double* a = h[l].data() + (size_t)b * ly.in;
+        for (int i = 0; i < ly.in; ++i) gw[i] += dzbo * a[i];
+      }
+    }
+    if (l == 0) break;
+    std::vector<double> dh((size_t)B * ly.in);
+    for (int b = 0; b < B; ++b) {
+      // dh[b][i] = sum_o dz[b][o] W[o][i]  (+ the skip path of a residual layer), output units in ascending order
+      double* dhb = dh.data() + (size_t)b * ly.in;
+      for (int i = 0; i < ly.in; ++i) dhb[i] = 0.0;
+      for (int o = 0; o < ly.out; ++o) {
+        const double dzbo = dz[(size_t)b * ly.out + o];
+        const double* w = pq.data() + ly.w_off + (int64_t)o * ly.in;
+        for (int i = 0; i < ly.in; ++i) dhb[i] += dzbo * w[i];
+      }
+      for (int i = 0; i < ly.in; ++i) {
+        const double skip = ly.residual ? dh_next[(size_t)b * ly.in + i] : 0.0;
+        dhb[i] = net.q(dhb[i] + skip);
+      }
+    }
+    // pre-activation gradient of layer l-1 (always a hidden layer here)
+    const Layer& lp = net.layers[l - 1];
+    std::vector<double> dzp((size_t)B * lp.out);
+    for (size_t e = 0; e < dzp.size(); ++e) dzp[e] = mask[l - 1][e] ? dh[e] : 0.0;
+    dz.swap(dzp);
+    dh_next.swap(dh);
+  }
+  return loss;
+}
+
+void gather_inputs(const Net& net, const float* X, const int32_t* idx, int B, std::vector<double>& a0) {
+  const int n = net.in0;
+  a0.resize((size_t)B * n);
+  for (int b = 0; b < B; ++b)
+    for (int i = 0; i < n; ++i) a0[(size_t)b * n + i] = net.q((double)X[(int64_t)idx[b] * n + i]);
+}
+
+}  // namespace
+
+struct oracle_ctx {
+  oracle_config cfg;
+  Net net;
+  const float* X = nullptr;
+  const float* Yf = nullptr;
+  const int32_t* Yi = nullptr;
+  std::vector<int32_t> rid;
+  int64_t d = 0;
+  std::vector<double> x, v, acc, g1, g2, xp;  // [K, d]
+  std::vector<std::vector<double>> y_hist;    // centre versions; y_hist[t_y] is current
+  std::vector<double> gprev;
+  bool have_prev = false;
+  int64_t t = 0, t_y = 0;
+  std::vector<int64_t> t_x;
+  std::vector<int64_t> ver_at_step;  // ver_at_step[s] = centre version that was current when step s started
+  std::vector<double> loss, gn1, gn2;
+  const float* eg1 = nullptr;
+  const float* eg2 = nullptr;
+};
+
+extern "C" {
+
+uint64_t oracle_mix64(uint64_t z) { return mix64(z); }
+uint64_t oracle_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j) { return hash5(seed, tag, t, k, j); }
+uint64_t oracle_tag_idx(void) { return TAG_IDX; }
+uint64_t oracle_tag_stale(void) { return TAG_STALE; }
+float oracle_bf16_round(float v) { return bf16_round(v); }
+int oracle_num_threads(void) {
+#ifdef _OPENMP
+  return omp_get_max_threads();
+#else
+  return 1;
+#endif
+}
+
+int64_t oracle_param_count(const oracle_config* cfg) {
+  Net net;
+  if (!cfg || !build_net(*cfg, net)) return -1;
+  return net.d;
+}
+
+oracle_ctx* oracle_create(const oracle_config* cfg, const float* X, const void* Y, const double* x0,
+                          const double* y0, const int32_t* replica_ids) {
+  if (!cfg || !x0 || !y0) return nullptr;
+  oracle_ctx* o = new oracle_ctx();
+  o->cfg = *cfg;
+  if (!build_net(*cfg, o->net) || cfg->tau < 1 || cfg->stale_max < 0) {
+    delete o;
+    return nullptr;
+  }
+  if (cfg->model != ORACLE_MODEL_FLAT && (!X || !Y)) {
+    delete o;
+    return nullptr;
+  }
+  o->X = X;
+  if (cfg->model == ORACLE_MODEL_LSQ) o->Yf = (const float*)Y;
+  else o->Yi = (const int32_t*)Y;
+  const int K = cfg->K;
+  o->d = o->net.d;
+  const size_t n = (size_t)K * o->d;
+  o->rid.resize(K);
+  for (int k = 0; k < K; ++k) o->rid[k] = replica_ids ? replica_ids[k] : k;
+  o->x.assign(x0, x0 + n);
+  o->v.assign(n, 0.0);
+  o->acc.assign(n, 0.0);
+  o->g1.assign(n, 0.0);
+  o->g2.assign(n, 0.0);
+  o->xp.assign(n, 0.0);
+  o->y_hist.emplace_back(y0, y0 + o->d);
+  o->gprev.assign(o->d, 0.0);
+  o->t_x.assign(K, 0);
+  o->loss.assign(K, 0.0);
+  o->gn1.assign(K, 0.0);
+  o->gn2.assign(K, 0.0);
+  return o;
+}
+
+void oracle_destroy(oracle_ctx* o) { delete o; }
+
+static void schedule_of(const oracle_ctx* o, int64_t t, int k, int32_t* idx, int32_t* stale, int32_t* ver) {
+  const oracle_config& c = o->cfg;
+  const uint64_t kid = (uint64_t)o->rid[k];
+  if (idx && c.model != ORACLE_MODEL_FLAT)
+    for (int j = 0; j < c.batch; ++j)
+      idx[j] = (int32_t)(hash5(c.seed, TAG_IDX, (uint64_t)t, kid, (uint64_t)j) % (uint64_t)c.n_samples);
+  const int64_t s = (int64_t)(hash5(c.seed, TAG_STALE, (uint64_t)t, kid, 0) % (uint64_t)(c.stale_max + 1));
+  if (stale) *stale = (int32_t)s;
+  if (ver) {
+    const int64_t ts = t - s > 0 ? t - s : 0;
+    *ver = (ts < (int64_t)o->ver_at_step.size()) ? (int32_t)o->ver_at_step[ts] : -1;
+  }
+}
+
+int oracle_step(oracle_ctx* o, double eta, double rho) {
+  if (!o) return 1;
+  const oracle_config& c = o->cfg;
+  const int K = c.K;
+  const int64_t d = o->d;
+  if (c.model == ORACLE_MODEL_FLAT && (!o->eg1 || !o->eg2)) return 2;
+  o->ver_at_step.push_back(o->t_y);  // centre version current when this tick starts
+  const int64_t t = o->t;
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int k = 0; k < K; ++k) {
+    double* x = o->x.data() + (size_t)k * d;
+    double* v = o->v.data() + (size_t)k * d;
+    double* acc = o->acc.data() + (size_t)k * d;
+    double* g1 = o->g1.data() + (size_t)k * d;
+    double* g2 = o->g2.data() + (size_t)k * d;
+    double* xp = o->xp.data() + (size_t)k * d;
+    std::vector<int32_t> idx(c.model == ORACLE_MODEL_FLAT ? 0 : c.batch);
+    int32_t s, ver;
+    schedule_of(o, t, k, idx.data(), &s, &ver);
+    const double* yk = o->y_hist[ver].data();  // possibly stale centre seen by this worker
+    std::vector<double> a0;
+    // ascent gradient g1 = grad of the minibatch loss at x_k
+    if (c.model == ORACLE_MODEL_FLAT) {
+      for (int64_t j = 0; j < d; ++j) g1[j] = (double)o->eg1[(size_t)k * d + j];
+      o->loss[k] = 0.0;
+    } else {
+      gather_inputs(o->net, o->X, idx.data(), c.batch, a0);
+      o->loss[k] = net_loss_grad(o->net, x, a0, c.batch, o->Yf, o->Yi, idx.data(), g1, nullptr);
+    }
+    double ss = 0.0;
+    for (int64_t j = 0; j < d; ++j) ss += g1[j] * g1[j];
+    const double n1 = std::sqrt(ss);
+    o->gn1[k] = n1;
+    // look-back map: x~ = x + rho g1 / (||g1|| + gamma)
+    for (int64_t j = 0; j < d; ++j) xp[j] = x[j] + rho * g1[j] / (n1 + c.gamma);
+    // descent gradient at x~ on the same minibatch
+    if (c.model == ORACLE_MODEL_FLAT) {
+      for (int64_t j = 0; j < d; ++j) g2[j] = (double)o->eg2[(size_t)k * d + j];
+    } else {
+      net_loss_grad(o->net, xp, a0, c.batch, o->Yf, o->Yi, idx.data(), g2, nullptr);
+    }
+    double ss2 = 0.0;
+    for (int64_t j = 0; j < d; ++j) ss2 += g2[j] * g2[j];
+    o->gn2[k] = std::sqrt(ss2);
+    // sampler: momentum step on G = g2 + lambda (x - y); the pull is evaluated at x_k, not at x~
+    for (int64_t j = 0; j < d; ++j) {
+      const double G = g2[j] + c.lambda * (x[j] - yk[j]);
+      v[j] = c.mu * v[j] + G;
+      x[j] = c.nesterov ? x[j] - eta * (G + c.mu * v[j]) : x[j] - eta * v[j];
+      acc[j] += x[j];  // running sum of post-update iterates since the last sync
+    }
+    o->t_x[k] += 1;
+  }
+  o->t += 1;
+  return 0;
+}
+
+int oracle_should_couple(const oracle_ctx* o) {
+  if (!o) return 0;
+  int64_t s = 0;
+  for (int64_t c : o->t_x) s += c;
+  return (s > 0 && s % ((int64_t)o->cfg.K * o->cfg.tau) == 0) ? 1 : 0;
+}
+
+int oracle_couple(oracle_ctx* o) {
+  if (!o) return 1;
+  if (!oracle_should_couple(o)) return 3;
+  const oracle_config& c = o->cfg;
+  const int64_t d = o->d;
+  const std::vector<double>& y = o->y_hist.back();
+  std::vector<double> yn(d);
+  const double ntau = (double)c.K * (double)c.tau;
+  for (int64_t j = 0; j < d; ++j) {
+    double s = 0.0;
+    for (int k = 0; k < c.K; ++k) s += o->acc[(size_t)k * d + j];
+    const double gp = s / ntau - y[j];                                        // g'
+    const double g = o->have_prev ? gp + c.beta * (gp - o->gprev[j]) : gp;    // look-ahead direction
+    yn[j] = y[j] + c.eta_prime * g;                                           // ascent on log pi_LSAM
+    o->gprev[j] = gp;
+  }
+  o->y_hist.push_back(std::move(yn));
+  o->have_prev = true;
+  std::fill(o->acc.begin(), o->acc.end(), 0.0);
+  std::fill(o->t_x.begin(), o->t_x.end(), 0);
+  o->t_y += 1;
+  return 0;
+}
+
+int oracle_read_params(const oracle_ctx* o, int which, double* dst) {
+  if (!o || !dst || which < -1 || which >= o->cfg.K) return 1;
+  const double* src = which < 0 ? o->y_hist.back().data() : o->x.data() + (size_t)which * o->d;
+  std::memcpy(dst, src, sizeof(double) * (size_t)o->d);
+  return 0;
+}
+
+int oracle_read_state(const oracle_ctx* o, double* x, double* v, double* y, double* acc, double* gprev) {
+  if (!o) return 1;
+  const size_t n = (size_t)o->cfg.K * o->d;
+  if (x) std::memcpy(x, o->x.data(), sizeof(double) * n);
+  if (v) std::memcpy(v, o->v.data(), sizeof(double) * n);
+  if (acc) std::memcpy(acc, o->acc.data(), sizeof(double) * n);
+  if (y) std::memcpy(y, o->y_hist.back().data(), sizeof(double) * (size_t)o->d);
+  if (gprev) std::memcpy(gprev, o->gprev.data(), sizeof(double) * (size_t)o->d);
+  return 0;
+}
+
+int oracle_write_state(oracle_ctx* o, const double* x, const double* v, const double* y) {
+  if (!o) return 1;
+  const size_t n = (size_t)o->cfg.K * o->d;
+  if (x) o->x.assign(x, x + n);
+  if (v) o->v.assign(v, v + n);
+  if (y) o->y_hist.back().assign(y, y + o->d);
+  return 0;
+}
+
+int oracle_read_schedule(const oracle_ctx* o, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver) {
+  if (!o || t < 0) return 1;
+  for (int k = 0; k < o->cfg.K; ++k)
+    schedule_of(o, t, k, idx ? idx + (size_t)k * o->cfg.batch : nullptr, stale ? stale + k : nullptr,
+                ver ? ver + k : nullptr);
+  return 0;
+}
+
+int oracle_read_step_info(const oracle_ctx* o, double* loss, double* gnorm1, double* gnorm2) {
+  if (!o) return 1;
+  const size_t n = sizeof(double) * (size_t)o->cfg.K;
+  if (loss) std::memcpy(loss, o->loss.data(), n);
+  if (gnorm1) std::memcpy(gnorm1, o->gn1.data(), n);
+  if (gnorm2) std::memcpy(gnorm2, o->gn2.data(), n);
+  return 0;
+}
+
+int oracle_read_grads(const oracle_ctx* o, double* g1, double* g2, double* x_pert) {
+  if (!o) return 1;
+  const size_t n = sizeof(double) * (size_t)o->cfg.K * o->d;
+  if (g1) std::memcpy(g1, o->g1.data(), n);
+  if (g2) std::memcpy(g2, o->g2.data(), n);
+  if (x_pert) std::memcpy(x_pert, o->xp.data(), n);
+  return 0;
+}
+
+int oracle_set_external_grads(oracle_ctx* o, const float* g1, const float* g2) {
+  if (!o || o->cfg.model != ORACLE_MODEL_FLAT) return 1;
+  o->eg1 = g1;
+  o->eg2 = g2;
+  return 0;
+}
+
+int oracle_read_counters(const oracle_ctx* o, int64_t* t, int64_t* t_y, int64_t* t_x) {
+  if (!o) return 1;
+  if (t) *t = o->t;
+  if (t_y) *t_y = o->t_y;
+  if (t_x) std::memcpy(t_x, o->t_x.data(), sizeof(int64_t) * (size_t)o->cfg.K);
+  return 0;
+}
+
+int oracle_loss_grad(const oracle_config* cfg, const float* X, const void* Y, const double* params,
+                     const int32_t* idx, int32_t n_idx, double* loss, double* grad) {
+  Net net;
+  if (!cfg || !build_net(*cfg, net) || cfg->model == ORACLE_MODEL_FLAT) return 1;
+  std::vector<double> a0;
+  gather_inputs(net, X, idx, n_idx, a0);
+  const float* yf = cfg->model == ORACLE_MODEL_LSQ ? (const float*)Y : nullptr;
+  const int32_t* yi = cfg->model == ORACLE_MODEL_LSQ ? nullptr : (const int32_t*)Y;
+  const double l = net_loss_grad(net, params, a0, n_idx, yf, yi, idx, grad, nullptr);
+  if (loss) *loss = l;
+  return 0;
+}
+
+int oracle_forward(const oracle_config* cfg, const float* X, const double* params, const int32_t* idx,
+                   int32_t n_idx, double* out) {
+  Net net;
+  if (!cfg || !build_net(*cfg, net) || cfg->model == ORACLE_MODEL_FLAT || !out) return 1;
+  std::vector<double> a0;
+  gather_inputs(net, X, idx, n_idx, a0);
+  std::vector<double> dummy;
+  net_loss_grad(net, params, a0, n_idx, nullptr, nullptr, idx, nullptr, out);
+  return 0;
+}
+
+}  // extern "C"

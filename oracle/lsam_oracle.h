@@ -1,0 +1,109 @@
+/*
+ * lsam_oracle.h -- CPU oracle for the per-worker LSAM step and the worker/centre coupling.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, double-precision restatement of
+ * Algorithm 2 (asynchronous distributed LSAM) with the SAM perturbation of Eq. 3 and the
+ * Gaussian-kernel pull of Algorithm 1 (first update line).  It shares no code with the CUDA
+ * library and must never be reached from the product path: only the test-suite, the smoke
+ * check and the benchmark's CPU-baseline leg may load it.
+ *
+ * Every function takes HOST pointers.  Parameters and optimiser state are double.
+ * The parameter vector of one replica is the unpadded concatenation, layer by layer, of
+ * W_l stored [out, in] row-major followed by b_l ([out]).  The least-squares model has a
+ * single weight vector w [in] and no bias.  The FLAT model has no data: both gradients of a
+ * step are supplied by the caller.
+ *
+ * Parity status of the pieces (what pins them independently of this file is listed in the
+ * test-suite): schedule hash, gradients, perturbation, worker update, centre update are
+ * pinned; free-running trajectories and the default hyper-parameters are "parity unpinned"
+ * (the paper prints no worked numerical example).
+ */
+#ifndef LSAM_ORACLE_H
+#define LSAM_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { ORACLE_MODEL_LSQ = 0, ORACLE_MODEL_MLP = 1, ORACLE_MODEL_RESMLP = 2, ORACLE_MODEL_FLAT = 3 };
+enum { ORACLE_GEMM_FP32 = 0, ORACLE_GEMM_BF16 = 1 };
+
+typedef struct {
+  int32_t model;        /* ORACLE_MODEL_*                                                    */
+  int32_t n_layers;     /* number of weight matrices (LSQ: 1; FLAT: 0)                       */
+  int32_t widths[9];    /* in, hidden..., out : n_layers + 1 entries (LSQ: widths[0] = in)   */
+  int32_t K;            /* number of worker replicas (the paper's n)                         */
+  int32_t batch;        /* per-worker minibatch size                                         */
+  int32_t gemm_dtype;   /* ORACLE_GEMM_*: BF16 rounds matmul operands, accumulates in double */
+  int32_t nesterov;     /* 1: x <- x - eta (G + mu v); 0: x <- x - eta v                     */
+  int32_t tau;          /* sync period of Algorithm 2                                        */
+  int32_t stale_max;    /* staleness drawn uniformly from [0, stale_max]                     */
+  int32_t reserved;
+  int64_t n_samples;    /* rows of X                                                         */
+  int64_t flat_d;       /* FLAT model only: length of a replica's vector                     */
+  uint64_t seed;
+  double mu;            /* worker momentum                                                   */
+  double gamma;         /* stabiliser of Eq. 3                                               */
+  double lambda;        /* pull strength of the Gaussian kernel                              */
+  double beta;          /* centre look-ahead factor                                          */
+  double eta_prime;     /* centre step size                                                  */
+} oracle_config;
+
+typedef struct oracle_ctx oracle_ctx;
+
+/* Number of parameters of one replica (unpadded), or -1 for an invalid configuration. */
+int64_t oracle_param_count(const oracle_config* cfg);
+
+/* X [n_samples, widths[0]] fp32 row-major; Y: float targets [n_samples] for LSQ, int32 labels
+ * for MLP/RESMLP, NULL for FLAT.  X and Y are borrowed.  x0 [K, d], y0 [d] are copied.
+ * replica_ids (nullable, [K]): global worker ids fed to the schedule hash, so that a small
+ * oracle can replay selected workers of a larger run; NULL means 0..K-1.                   */
+oracle_ctx* oracle_create(const oracle_config* cfg, const float* X, const void* Y,
+                          const double* x0, const double* y0, const int32_t* replica_ids);
+void oracle_destroy(oracle_ctx*);
+
+/* One tick of the sampling loop of Algorithm 2 for every replica (eta, rho per call). */
+int oracle_step(oracle_ctx*, double eta, double rho);
+/* 1 when the sync condition of Algorithm 2 holds (and at least one iterate was collected). */
+int oracle_should_couple(const oracle_ctx*);
+/* The centre update of Algorithm 2; returns non-zero and does nothing if the trigger is false. */
+int oracle_couple(oracle_ctx*);
+
+/* which in [0,K): replica; which = -1: current centre. dst [d]. */
+int oracle_read_params(const oracle_ctx*, int which, double* dst);
+/* Any of the pointers may be NULL.  x, v, acc: [K, d]; y, gprev: [d].  acc is the per-replica
+ * running sum of post-update iterates since the last sync.                                  */
+int oracle_read_state(const oracle_ctx*, double* x, double* v, double* y, double* acc, double* gprev);
+/* Overwrite worker iterates, momentum buffers and the CURRENT centre (any pointer may be NULL). */
+int oracle_write_state(oracle_ctx*, const double* x, const double* v, const double* y);
+/* Schedule of step t (any t >= 0 for idx and stale; ver needs t <= number of steps taken). */
+int oracle_read_schedule(const oracle_ctx*, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver);
+/* Quantities of the LAST step: loss at x_k, ||g1_k||, ||g2_k||  ([K] each, nullable). */
+int oracle_read_step_info(const oracle_ctx*, double* loss, double* gnorm1, double* gnorm2);
+/* Gradients and perturbed point of the LAST step, [K, d] each, nullable. */
+int oracle_read_grads(const oracle_ctx*, double* g1, double* g2, double* x_pert);
+/* FLAT model: gradients used by the next steps, [K, d] fp32, borrowed. */
+int oracle_set_external_grads(oracle_ctx*, const float* g1, const float* g2);
+/* Counters: t (steps), t_y (centre version), t_x [K]. */
+int oracle_read_counters(const oracle_ctx*, int64_t* t, int64_t* t_y, int64_t* t_x);
+
+/* Stand-alone pieces, exposed so that they can be pinned one by one. */
+/* Mean loss and its gradient at `params` on the minibatch idx[0..n_idx).  grad [d]. */
+int oracle_loss_grad(const oracle_config* cfg, const float* X, const void* Y, const double* params,
+                     const int32_t* idx, int32_t n_idx, double* loss, double* grad);
+/* Logits (MLP/RESMLP: [n_idx, classes]) or predictions (LSQ: [n_idx]) at `params`. */
+int oracle_forward(const oracle_config* cfg, const float* X, const double* params,
+                   const int32_t* idx, int32_t n_idx, double* out);
+uint64_t oracle_mix64(uint64_t z);
+uint64_t oracle_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j);
+uint64_t oracle_tag_idx(void);
+uint64_t oracle_tag_stale(void);
+float oracle_bf16_round(float v);
+int oracle_num_threads(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif
