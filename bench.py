@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the LSAM worker step on B200: worker-samples/s, roofline of the dominant kernel, CPU-oracle baseline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c1|c2|c3|c4|c5] [--impl reference]
+
+A step is one pass of the whole hot path (schedule, gather, ascent gradient, norm, perturbation, descent gradient,
+fused update) for all K replicas, plus the centre update whenever the sync trigger fires (every tau steps).
+With more than one GPU every rank runs an independent copy of the workload (replicas only: the path has no
+exchange step on one GPU and the cross-GPU accumulator all-reduce is not built), so scaling is weak.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+LSQ, MLP, RESMLP, FLAT = 0, 1, 2, 3
+
+# The five workloads (shapes, replica counts, batch sizes and radii as configured; eta, tau, lambda0 filled with the
+# paper's Appendix-D ranges where a workload leaves them open).
+WORKLOADS = {
+    "c1": dict(model=LSQ, widths=(256,), K=4, B=32, n=4096, classes=0, bf16=False, rho=0.05, eta=0.01, tau=4, stale_max=0,
+               name="least squares 4096x256, K=4, B=32"),
+    "c2": dict(model=MLP, widths=(784, 1024, 10), K=8, B=128, n=60000, classes=10, bf16=False, rho=0.05, eta=0.05, tau=4,
+               stale_max=0, name="MLP 784-1024-10 fp32, K=8, B=128"),
+    "c3": dict(model=MLP, widths=(3072, 2048, 2048, 2048, 100), K=16, B=128, n=50000, classes=100, bf16=True, rho=0.1,
+               eta=0.05, tau=4, stale_max=0, name="MLP 3072-2048x3-100 bf16 GEMM, K=16, B=128"),
+    "c4": dict(model=RESMLP, widths=(3072, 4096, 4096, 4096, 4096, 1000), K=32, B=256, n=200000, classes=1000, bf16=True,
+               rho=0.1, eta=0.05, tau=4, stale_max=3, name="residual MLP 3072-4096x4-1000 bf16 GEMM, K=32, B=256, staleness [0,3]"),
+    "c5": dict(model=FLAT, widths=(), K=8, B=0, n=0, classes=0, bf16=False, rho=0.1, eta=0.05, tau=4, stale_max=0, d=256_000_000,
+               name="optimiser-only sweep point d=256M, K=8"),
+}
+LAMBDA0, MU, BETA, ETA_PRIME, GAMMA = 0.5, 0.9, 0.9, 1.0, 1e-12
+NOMINAL_HBM_GBS, FALLBACK_HBM_GBS, FALLBACK_BF16_TF = 8000.0, 6650.0, 1590.0
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x max SM clock
+
+
+def param_count(w):
+    if w["model"] == FLAT:
+        return w["d"]
+    if w["model"] == LSQ:
+        return w["widths"][0]
+    ws = w["widths"]
+    return sum(ws[i] * ws[i + 1] + ws[i + 1] for i in range(len(ws) - 1))
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return dict(hbm=float(j["hbm_gbs"]), bf16=float(j["bf16_tflops"]), bf16_sustained=float(j.get("bf16_tflops_sustained", j["bf16_tflops"])), src="measured")
+    return dict(hbm=FALLBACK_HBM_GBS, bf16=FALLBACK_BF16_TF, bf16_sustained=1400.0, src="fallback")
+
+
+# ---------------------------------------------------------------------------------------------- algorithmic work per step
+def work_model(w, tc):
+    """Algorithmic bytes / flops per STEP of each kernel class (what the method must move or compute)."""
+    K, B, d = w["K"], w["B"], param_count(w)
+    op = 2 if w["bf16"] else 4
+    out = {}
+    out["norm"] = dict(bytes=4.0 * K * d)                                    # read g1
+    out["perturb"] = dict(bytes=(4.0 + 4.0 + op) * K * d)                    # read x, g1; write x~
+    out["update"] = dict(bytes=(4.0 + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2, x rw, v rw, operand copy; y, acc rw
+    if w["model"] in (MLP, RESMLP):
+        ws = w["widths"]
+        f_fwd = f_dg = f_wg = 0.0
+        b_fwd = b_dg = b_wg = 0.0
+        for l in range(len(ws) - 1):
+            i, o = ws[l], ws[l + 1]
+            f_fwd += 2.0 * B * i * o
+            b_fwd += op * (i * o + B * i + B * o)
+            f_wg += 2.0 * B * i * o
+            b_wg += 4.0 * i * o + op * B * (i + o)
+            if l > 0:
+                f_dg += 2.0 * B * i * o
+                b_dg += op * (i * o + B * i + B * o)
+        for name, f, b in (("gemm_fwd", f_fwd, b_fwd), ("gemm_dgrad", f_dg, b_dg), ("gemm_wgrad", f_wg, b_wg)):
+            out[name] = dict(flops=2.0 * K * f, bytes=2.0 * K * b)          # two gradient passes per step
+    return out
+
+
+# ---------------------------------------------------------------------------------------------- clocks
+class ClockSampler:
+    Q = "clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap"
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None, reasons=sorted(reasons), samples=len(sm))
+
+
+# ---------------------------------------------------------------------------------------------- inputs (device, seeded)
+def make_inputs(w, dev, seed=0):
+    import torch
+
+    g = torch.Generator(device=dev).manual_seed(seed)
+    K = w["K"]
+    if w["model"] == FLAT:
+        d = w["d"]
+        x0 = torch.randn(K, d, device=dev, generator=g)
+        g1 = torch.randn(K, d, device=dev, generator=g) * 0.1
+        g2 = torch.randn(K, d, device=dev, generator=g) * 0.1
+        return dict(X=None, Y=None, x0=x0, y0=x0.mean(0), g1=g1, g2=g2)
+    n, fin = w["n"], w["widths"][0]
+    if w["model"] == LSQ:
+        X = torch.randn(n, fin, device=dev, generator=g)
+        wstar = torch.randn(fin, device=dev, generator=g)
+        Y = X @ wstar + 0.01 * torch.randn(n, device=dev, generator=g)
+        w0 = torch.randn(fin, device=dev, generator=g)
+    else:
+        C = w["classes"]
+        means = torch.randn(C, fin, device=dev, generator=g)
+        Y = (torch.arange(n, device=dev) % C).to(torch.int32)
+        X = torch.randn(n, fin, device=dev, generator=g)
+        X += means[Y.long()]
+        parts = []
+        ws = w["widths"]
+        for l in range(len(ws) - 1):
+            parts.append((torch.randn(ws[l + 1], ws[l], device=dev, generator=g) * (2.0 / ws[l]) ** 0.5).reshape(-1))
+            parts.append(torch.zeros(ws[l + 1], device=dev))
+        w0 = torch.cat(parts)
+    x0 = w0.unsqueeze(0).expand(K, -1).contiguous()
+    return dict(X=X, Y=Y, x0=x0, y0=w0)
+
+
+def make_cfg(G, w, flags=0):
+    lam = LAMBDA0 / (w["eta"] * w["tau"])
+    return G.make_config(w["model"], widths=w["widths"], K=w["K"], batch=max(w["B"], 1) if w["model"] != FLAT else 0,
+                         gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
+                         beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
+                         flat_d=w.get("d", 0), flags=flags)
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_baseline(w, X, Y, x0_row, budget_s=20.0):
+    """Time the oracle, as it stands, on a bounded sample of the workload: a subset of replicas and of each minibatch."""
+    import oracle as O
+
+    cores = O.num_threads()
+    d = param_count(w)
+    lam = LAMBDA0 / (w["eta"] * w["tau"])
+    if w["model"] == FLAT:
+        Ks, ds = w["K"], min(d, 4_000_000)
+        cfg = O.make_config(O.MODEL_FLAT, K=Ks, flat_d=ds, mu=MU, gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME)
+        rng = np.random.default_rng(0)
+        x0 = rng.standard_normal((Ks, ds))
+        g1 = (0.1 * rng.standard_normal((Ks, ds))).astype(np.float32)
+        o = O.Oracle(cfg, None, None, x0, x0.mean(0))
+        o.set_external_grads(g1, g1)
+        o.step(w["eta"], w["rho"])
+        t0 = time.perf_counter()
+        steps = 3
+        for _ in range(steps):
+            o.step(w["eta"], w["rho"])
+        dt = (time.perf_counter() - t0) / steps
+        return dict(value=36.0 * Ks * ds / dt / 1e9, unit="GB/s (36 B per element-replica)", cores=min(cores, Ks), kind="oracle",
+                    sample=f"K={Ks} replicas, d={ds} of {d} elements, {steps} steps"), dt
+    # flops per worker-sample (12 per weight: two passes of fwd + dgrad + wgrad) and a measured-free guess of 1.5 GFLOP/s/core
+    flop_ws = 12.0 * d
+    Ks = min(w["K"], cores)
+    Bs = int(max(1, min(w["B"], budget_s * 1.5e9 / flop_ws)))
+    cfg = O.make_config(w["model"], widths=w["widths"], K=Ks, batch=Bs, gemm_dtype=O.GEMM_BF16 if w["bf16"] else O.GEMM_FP32, mu=MU,
+                        gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=w["n"])
+    x0 = np.repeat(x0_row[None, :].astype(np.float64), Ks, axis=0)
+    o = O.Oracle(cfg, X, Y, x0, x0_row.astype(np.float64))
+    steps = 1 if flop_ws * Bs > 2e9 else 5
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        o.step(w["eta"], w["rho"])
+    dt = (time.perf_counter() - t0) / steps
+    o.close()
+    return dict(value=Ks * Bs / dt, unit="worker-samples/s", cores=min(cores, Ks), kind="oracle",
+                sample=f"{Ks} of {w['K']} replicas x {Bs} of {w['B']} samples per minibatch, full model, {steps} step(s)"), dt
+
+
+def run_reference(args, w, metric, unit):
+    """--impl reference: the CPU oracle timed on bounded samples of the same workload (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import torch
+
+    inp = make_inputs(w, torch.device("cpu"), seed=0)
+    X = None if inp["X"] is None else inp["X"].numpy()
+    Y = None if inp["Y"] is None else inp["Y"].numpy()
+    x0_row = inp["y0"].numpy()
+    vals, dts = [], []
+    per = max(2.0, min(20.0, 120.0 / max(args.steps + args.warmup, 1)))
+    for i in range(args.warmup + args.steps):
+        cb, dt = oracle_baseline(w, X, Y, x0_row, budget_s=per)
+        if i >= args.warmup:
+            vals.append(cb["value"])
+            dts.append(dt)
+    v = float(np.mean(vals))
+    cb["value"] = v
+    line = dict(impl="reference", metric=metric, value=v, unit=unit, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=float(np.mean(dts) * 1e3), higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
+                data="synthetic", config=dict(workload=w["name"]), cpu_baseline=cb,
+                e2e=dict(value=v, unit=unit, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--flat-d", type=int, default=None, help="c5 only: vector length of the sweep point")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    w = dict(WORKLOADS[args.workload])
+    if args.flat_d and w["model"] == FLAT:
+        w["d"] = args.flat_d
+        w["name"] = f"optimiser-only sweep point d={args.flat_d}, K=8"
+    flat = w["model"] == FLAT
+    metric = "fused_update_hbm_gbs" if flat else "lsam_worker_samples_per_s"
+    unit = "GB/s" if flat else "worker-samples/s"
+    if args.impl == "reference":
+        return run_reference(args, w, metric, unit)
+
+    import torch
+    import torch.distributed as dist
+
+    from paper_2509_03110_b200 import binding as G
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    warm = max(args.warmup, 3)
+
+    inp = make_inputs(w, dev, seed=rank)
+    cfg = make_cfg(G, w)
+    ctx = G.Lsam(cfg, inp["X"], inp["Y"], inp["x0"], inp["y0"])
+    d = ctx.d
+    inp["x0"] = None
+    torch.cuda.empty_cache()
+    if flat:
+        ctx.set_external_grads(inp["g1"], inp["g2"])
+    stream = ctx.stream
+    eta, rho = w["eta"], w["rho"]
+
+    def one_step():
+        ctx.step(eta, rho)
+        if ctx.should_couple():
+            ctx.couple()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    # ---- device-resident timing (value), with per-kernel-class events for the roofline
+    for _ in range(warm):
+        one_step()
+    ctx.profile_enable(True)
+    ctx.profile_read()
+    launches0 = ctx.launch_count()
+    clocks = ClockSampler(local)
+    barrier()
+    clocks.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        one_step()
+    e1.record(stream)
+    barrier()
+    clk = clocks.stop()
+    ms = e0.elapsed_time(e1)
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    launches = ctx.launch_count() - launches0
+    if ctx.status() != 0:
+        raise SystemExit("device status word is not clean after the timed region")
+    if world > 1:
+        tmax = torch.tensor([ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    ms_step = ms / args.steps
+    units_step = (36.0 * w["K"] * d / 1e9) if flat else float(w["K"] * w["B"])
+    value = world * units_step / (ms_step * 1e-3)
+
+    # ---- end to end through the C ABI with host buffers (minibatch H2D and loss D2H inside the timed region)
+    e2e = None
+    if not flat:
+        nst = min(args.steps, 8)
+        nb = min(nst, 4)
+        fin = w["widths"][0]
+        t_now = ctx.counters()[0]
+        xbs, ybs = [], []
+        for i in range(nb):
+            idx, _, _ = ctx.read_schedule(t_now + i, want_ver=False)
+            ii = torch.from_numpy(idx.reshape(-1).astype(np.int64)).to(dev)
+            xbs.append(inp["X"][ii].reshape(w["K"], w["B"], fin).cpu().pin_memory())
+            ybs.append(inp["Y"][ii].reshape(w["K"], w["B"]).cpu().pin_memory())
+        loss = np.zeros(w["K"], np.float32)
+        ctx.step_batch(eta, rho, xbs[0], ybs[0], loss)
+        barrier()
+        e0.record(stream)
+        for i in range(nst):
+            ctx.step_batch(eta, rho, xbs[i % nb], ybs[i % nb], loss)
+            if ctx.should_couple():
+                ctx.couple()
+        e1.record(stream)
+        barrier()
+        ems = e0.elapsed_time(e1)
+        if world > 1:
+            tmax = torch.tensor([ems], device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            ems = float(tmax.item())
+        e2e = dict(value=world * w["K"] * w["B"] / (ems / nst * 1e-3), unit=unit, h2d_bytes_per_step=int(xbs[0].numel() * 4 + ybs[0].numel() * 4),
+                   d2h_bytes_per_step=int(4 * w["K"]), steps=nst)
+    else:
+        # optimiser-only: the gradients are the step's inputs; copy them from pinned host memory every step
+        K = w["K"]
+        hg = torch.empty(2, K, d, dtype=torch.float32).pin_memory() if d <= 64_000_000 else None
+        if hg is not None:
+            hg[0].copy_(inp["g1"].cpu())
+            hg[1].copy_(inp["g2"].cpu())
+            out = np.zeros(d, np.float32)
+            barrier()
+            nst = min(args.steps, 5)
+            e0.record(stream)
+            for _ in range(nst):
+                inp["g1"].copy_(hg[0], non_blocking=True)
+                inp["g2"].copy_(hg[1], non_blocking=True)
+                one_step()
+                ctx.read_step_info()
+            e1.record(stream)
+            barrier()
+            ems = e0.elapsed_time(e1)
+            e2e = dict(value=world * units_step / (ems / nst * 1e-3), unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K), steps=nst)
+        else:
+            e2e = dict(value=None, unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K),
+                       note="gradient buffers of this sweep point exceed the pinned-memory budget; run --flat-d <= 64000000")
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel class
+    pk = peaks()
+    work = work_model(w, ctx.uses_tcgen05())
+    tot_ms = sum(v[0] for v in prof.values())
+    top = max(prof, key=lambda k: prof[k][0])
+    tms, tn = prof[top]
+    per_launch_s = tms / max(tn, 1) * 1e-3
+    shares = {k: round(v[0] / tot_ms, 4) for k, v in prof.items() if v[1] > 0}
+    wk = work.get(top, {})
+    launches_per_step = tn / args.steps
+    roof = dict(kernel=top, share_of_kernel_time=shares.get(top), traffic=None, kernel_time_shares=shares)
+    if top in ("gemm_fwd", "gemm_dgrad") and ctx.uses_tcgen05():
+        ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
+        roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_sustained"], peak_source=f"{pk['src']} (sustained bf16)")
+    elif top.startswith("gemm") and not ctx.uses_tcgen05() and not w["bf16"]:
+        ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
+        roof.update(bound="alu", achieved=ach, peak=FP32_ALU_TFLOPS, unit="TFLOP/s", frac=ach / FP32_ALU_TFLOPS, peak_source="148 SMs x 128 FMA lanes x 2 x 1.965 GHz")
+    elif "bytes" in wk:
+        ach = wk["bytes"] / launches_per_step / per_launch_s / 1e9
+        roof.update(bound="hbm", achieved=ach, peak=pk["hbm"], unit="GB/s", frac=ach / pk["hbm"], peak_source=f"{pk['src']} copy bandwidth",
+                    frac_of_nominal_8TBs=ach / NOMINAL_HBM_GBS)
+        if "flops" in wk:
+            roof["tflops"] = wk["flops"] / launches_per_step / per_launch_s / 1e12
+    else:
+        roof.update(bound="latency", achieved=None, peak=None, unit=None, frac=None)
+    # the three streaming kernels of the fused update path, always reported
+    stream_gbs = {}
+    for k in ("norm", "perturb", "update"):
+        if prof[k][1] > 0:
+            n_main = prof[k][1] / (2 if k == "norm" else 1)  # the norm class counts its tiny finalize launch too
+            stream_gbs[k] = round(work[k]["bytes"] * args.steps / (prof[k][0] * 1e-3) / 1e9, 1)
+    roof["streaming_kernels_gbs"] = stream_gbs
+
+    cpu = None
+    if not args.no_cpu_baseline:
+        X = None if inp["X"] is None else inp["X"].cpu().numpy()
+        Y = None if inp["Y"] is None else inp["Y"].cpu().numpy()
+        cpu, _ = oracle_baseline(w, X, Y, inp["y0"].cpu().numpy())
+
+    line = dict(metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=warm, ms_per_step=ms_step,
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if w["bf16"] else "f32", data="synthetic",
+                config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt",
+                            l2="working set larger than L2" if 4.0 * w["K"] * d > 126e6 else "L2-resident state (latency-bound workload)",
+                            parallelism="replicas only" if world > 1 else "1 GPU"),
+                clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)
+    print(json.dumps(line))
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

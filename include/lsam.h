@@ -1,0 +1,176 @@
+/*
+ * lsam.h -- C ABI of the B200 (sm_100a) LSAM worker-step library.
+ *
+ * What it computes.  K worker replicas of a model are held as stacked parameter tensors on one GPU.
+ * One lsam_step() is one tick of the sampling loop of Algorithm 2 ("Asynchronous Distributed LSAM")
+ * for every replica k:
+ *     g1_k = grad f(x_k; xi_k)                          minibatch gradient (ascent pass)
+ *     x~_k = x_k + rho g1_k / (||g1_k|| + gamma)        look-back map, Eq. 3
+ *     g2_k = grad f(x~_k; xi_k)                         same minibatch (Theorems 3 and 4)
+ *     G    = g2_k + lambda (x_k - y_ver(k))             worker score, Gaussian kernel (Algorithm 1, first update)
+ *     v_k <- mu v_k + G ;  x_k <- x_k - eta (G + mu v_k)  Nesterov momentum sampler (Section 4.3)
+ *     Acc += x_k ;  t_x[k] += 1                         running sum of post-update iterates (Algorithm 2, sync branch)
+ * and lsam_couple() is the sync branch of Algorithm 2:
+ *     g' = Acc / (K tau) - y ;  g = g' + beta (g' - g'_prev) ;  y <- y + eta' g ;  Acc <- 0 ; t_x <- 0 ; t_y += 1.
+ * The asynchrony of Algorithm 2 is replayed deterministically: replica k reads the centre version that was
+ * current s_k steps ago, s_k drawn uniformly from [0, stale_max] by an integer hash of (seed, t, k); the
+ * minibatch indices come from the same hash.
+ *
+ * Conventions.
+ *  - Every entry point returns an int status (LSAM_OK = 0); nothing throws or aborts.  lsam_last_error()
+ *    gives a message for the last failure of a context.
+ *  - Pointers named d_* are DEVICE pointers, h_* are HOST pointers; others say which in their comment.
+ *  - The caller owns all device memory (data, workspace) and the CUDA stream; the library owns only the
+ *    host-side context.  All work is enqueued on the stream given to lsam_init(); calls are asynchronous
+ *    unless they copy to host memory or say that they synchronise.
+ *  - Parameter vector of one replica (what x0, y0, lsam_read_params use): the UNPADDED concatenation, layer by
+ *    layer, of W_l stored [out, in] row-major then b_l [out].  LSQ: the weight vector w [in] only.  FLAT: flat_d
+ *    values.  Inside the workspace each segment start is padded to a multiple of 64 elements.
+ */
+#ifndef LSAM_H
+#define LSAM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct lsam_ctx lsam_ctx;
+
+enum {
+  LSAM_OK = 0,
+  LSAM_ERR_INVALID = 1,   /* bad argument or configuration                                          */
+  LSAM_ERR_WORKSPACE = 2, /* workspace too small or misaligned                                      */
+  LSAM_ERR_STATE = 3,     /* call not allowed in this state (e.g. lsam_couple while the trigger is false) */
+  LSAM_ERR_CUDA = 4,      /* a CUDA runtime / driver call failed                                    */
+  LSAM_ERR_NONFINITE = 5, /* a gradient norm was NaN or infinite (reported by lsam_status)          */
+  LSAM_ERR_TIMEOUT = 6    /* a bounded device-side wait expired (reported by lsam_status)           */
+};
+
+enum { LSAM_MODEL_LSQ = 0, LSAM_MODEL_MLP = 1, LSAM_MODEL_RESMLP = 2, LSAM_MODEL_FLAT = 3 };
+enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
+enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2 };
+enum {
+  LSAM_FLAG_KEEP_G1 = 1,   /* keep copies of the ascent gradient and (BF16 mode) of x~ for lsam_read_grads  */
+  LSAM_FLAG_STEP_INFO = 2  /* also reduce ||g2_k|| every step (one extra read of the gradient buffer)      */
+};
+
+/* Models.
+ *  LSQ    f = (1/(2B)) sum_j (a_j . w - y_j)^2, widths[0] = number of features, no bias, fp32 only.
+ *  MLP    h_{l+1} = relu(W_l h_l + b_l), linear head, softmax cross-entropy averaged over the minibatch.
+ *  RESMLP as MLP, but every hidden layer with equal input and output width is h_{l+1} = h_l + relu(W_l h_l + b_l).
+ *  FLAT   no model: the two gradients of a step are buffers supplied with lsam_set_external_grads().
+ * gemm_dtype BF16: matmul operands (weights, biases, inputs, stored activations and backward signals) are
+ * rounded to bf16, products accumulate in fp32, gradients and all optimiser state stay fp32.            */
+typedef struct {
+  int32_t model;      /* LSAM_MODEL_*                                                               */
+  int32_t n_layers;   /* weight matrices (MLP/RESMLP: 1..8; LSQ: 1; FLAT: 0)                        */
+  int32_t widths[9];  /* in, hidden..., out: n_layers + 1 entries                                   */
+  int32_t K;          /* worker replicas, the paper's n (Algorithm 2 inputs)                        */
+  int32_t batch;      /* per-worker minibatch size B                                                */
+  int32_t gemm_dtype; /* LSAM_GEMM_*                                                                */
+  int32_t gemm_impl;  /* LSAM_IMPL_*: AUTO picks tcgen05 for bf16 shapes it supports, else SIMT       */
+  int32_t nesterov;   /* 1: Nesterov form (Section 4.3); 0: heavy-ball x <- x - eta v               */
+  int32_t tau;        /* sync period tau                                                            */
+  int32_t stale_max;  /* staleness uniform in [0, stale_max], 0 = every worker reads the current centre; <= 15 */
+  int32_t flags;      /* LSAM_FLAG_*                                                                */
+  int64_t n_samples;  /* rows of the dataset                                                        */
+  int64_t flat_d;     /* FLAT only: vector length                                                   */
+  uint64_t seed;      /* schedule seed: indices and staleness are pure functions of (seed, t, k, j) */
+  float mu;           /* worker momentum                                                            */
+  float gamma;        /* stabiliser gamma > 0 of Eq. 3                                              */
+  float lambda;       /* pull strength lambda (the rule lambda0/(eta tau) of Appendix D is the caller's) */
+  float beta;         /* centre look-ahead factor beta (Section 4.2)                                */
+  float eta_prime;    /* centre step size eta'                                                      */
+  float reserved;
+} lsam_config;
+
+/* Unpadded parameter count d of one replica, or -1 if the configuration is invalid. */
+int64_t lsam_param_count(const lsam_config* cfg);
+
+/* Bytes of device workspace lsam_init() needs for this configuration (0 if invalid).  Host-only call. */
+size_t lsam_workspace_bytes(const lsam_config* cfg);
+
+/* Create a context (Algorithm 2, initialisation line: workers x0, centre y0, counters zero).
+ *  d_X  [n_samples, widths[0]] fp32 row-major, device, BORROWED until lsam_destroy (NULL for FLAT).
+ *  d_Y  device, borrowed: fp32 targets [n_samples] (LSQ) or int32 labels (MLP/RESMLP); NULL for FLAT.
+ *  d_x0 [K, d] fp32 device, d_y0 [d] fp32 device: copied into the workspace.
+ *  d_workspace: >= lsam_workspace_bytes() bytes, 256-byte aligned, owned by the caller, must outlive the context.
+ *  cuda_stream: a cudaStream_t (NULL = default stream).
+ * Errors: LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE, LSAM_ERR_CUDA; *out is NULL on failure. */
+int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const void* d_Y, const float* d_x0,
+              const float* d_y0, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
+
+/* One worker tick for all K replicas (sampling loop of Algorithm 2; Eq. 3; Algorithm 1, first update), with
+ * the minibatch drawn by the seeded schedule.  eta and rho are per call, so any schedule (eta0/sqrt(t+1),
+ * rho0/sqrt(t+1), step decay) is the caller's.  Asynchronous on the context's stream. */
+int lsam_step(lsam_ctx* ctx, float eta, float rho);
+
+/* Same tick, but the minibatch is supplied by the caller instead of gathered from the resident dataset:
+ *  xb [K, B, widths[0]] fp32, yb [K, B] (fp32 targets or int32 labels); both on the host (on_host = 1, copied
+ *  with cudaMemcpyAsync on the stream; use pinned memory) or on the device (on_host = 0).
+ *  h_loss (nullable, host [K]): receives the minibatch loss at x_k; if given, the call synchronises the stream.
+ * The staleness part of the schedule is unchanged.  Not available for FLAT. */
+int lsam_step_batch(lsam_ctx* ctx, float eta, float rho, const float* xb, const void* yb, int on_host, float* h_loss);
+
+/* Sync branch of Algorithm 2 (centre update with look-ahead, counters reset).  Returns LSAM_ERR_STATE and does
+ * nothing when the trigger (sum_k t_x[k] > 0 and sum_k t_x[k] mod K tau == 0) is false. */
+int lsam_couple(lsam_ctx* ctx);
+/* 1 if the trigger of the sync branch holds, else 0.  Host-only. */
+int lsam_should_couple(const lsam_ctx* ctx);
+
+/* Copy the unpadded parameters of replica `which` (0..K-1) or of the current centre (which = -1) to dst [n >= d].
+ * dst_on_device = 0: dst is host memory and the call synchronises the stream; 1: device memory, stream-ordered. */
+int lsam_read_params(lsam_ctx* ctx, int which, float* dst, int64_t n, int dst_on_device);
+
+/* ---- helpers (tests, checkpointing, measurement) ---- */
+/* Schedule of step t: h_idx [K, B] minibatch rows, h_stale [K], h_ver [K] centre version read (any may be NULL).
+ * idx and stale are defined for every t >= 0; ver only for steps already taken (else LSAM_ERR_STATE).
+ * Computed by the device kernel the step itself uses; synchronises. */
+int lsam_read_schedule(lsam_ctx* ctx, int64_t t, int32_t* h_idx, int32_t* h_stale, int32_t* h_ver);
+/* Of the last step: minibatch loss at x_k, ||g1_k||, ||g2_k|| (host [K] each, nullable; ||g2|| needs
+ * LSAM_FLAG_STEP_INFO, else it reads 0).  Synchronises. */
+int lsam_read_step_info(lsam_ctx* ctx, float* h_loss, float* h_gnorm1, float* h_gnorm2);
+/* Of the last step: pass = 1 ascent gradient (needs LSAM_FLAG_KEEP_G1), 2 descent gradient, 3 perturbed point x~
+ * (as stored: rounded to bf16 in BF16 mode, where it also needs LSAM_FLAG_KEEP_G1 because the operand buffer
+ * is reused by the update).  h_dst [K, d] unpadded, host.  Synchronises. */
+int lsam_read_grads(lsam_ctx* ctx, int pass, float* h_dst);
+/* FLAT only: device buffers [K, d] fp32 (row stride d) holding g1 and g2 for the following steps; borrowed. */
+int lsam_set_external_grads(lsam_ctx* ctx, const float* d_g1, const float* d_g2);
+/* Overwrite worker iterates x [K, d], momentum v [K, d] and the CURRENT centre y [d] (device pointers, any may be
+ * NULL) -- teacher forcing and resume.  Counters and the centre history are left as they are. */
+int lsam_write_state(lsam_ctx* ctx, const float* d_x, const float* d_v, const float* d_y);
+/* Read back momentum buffers and accumulator for checkpointing: h_v [K, d], h_acc [d], h_gprev [d] (nullable). Synchronises. */
+int lsam_read_state(lsam_ctx* ctx, float* h_v, float* h_acc, float* h_gprev);
+/* Counters: steps taken t, centre version t_y, per-worker t_x [K] (host, nullable). */
+int lsam_read_counters(const lsam_ctx* ctx, int64_t* t, int64_t* t_y, int64_t* h_t_x);
+/* Synchronise the stream and map the device status word to LSAM_OK / LSAM_ERR_NONFINITE / LSAM_ERR_TIMEOUT. */
+int lsam_status(lsam_ctx* ctx);
+/* Per-kernel-class device timing.  enable != 0: every launch of the following steps is bracketed by CUDA events
+ * on the context's stream.  lsam_profile_read synchronises, adds the elapsed times to ms[c] and the launch counts
+ * to launches[c] for c < LSAM_PROF_CLASSES (host arrays), and clears the record. */
+enum {
+  LSAM_PROF_SCHEDULE = 0, LSAM_PROF_GATHER, LSAM_PROF_GEMM_FWD, LSAM_PROF_GEMM_DGRAD, LSAM_PROF_GEMM_WGRAD,
+  LSAM_PROF_LOSS, LSAM_PROF_BIAS_GRAD, LSAM_PROF_LSQ_GRAD, LSAM_PROF_NORM, LSAM_PROF_PERTURB, LSAM_PROF_UPDATE,
+  LSAM_PROF_COUPLE, LSAM_PROF_COPY, LSAM_PROF_CLASSES
+};
+int lsam_profile_enable(lsam_ctx* ctx, int enable);
+int lsam_profile_read(lsam_ctx* ctx, double* h_ms, int64_t* h_launches);
+/* Kernels launched by this context since it was created. */
+int64_t lsam_launch_count(const lsam_ctx* ctx);
+/* 1 if the model GEMMs of this context run on the tcgen05 tensor-core path, 0 if on the SIMT path. */
+int lsam_uses_tcgen05(const lsam_ctx* ctx);
+const char* lsam_last_error(const lsam_ctx* ctx);
+/* Frees the host context only; the caller frees the workspace. */
+void lsam_destroy(lsam_ctx* ctx);
+
+/* Host-side statement of the schedule hash, H(seed, tag, t, k, j) = mix(mix(mix(seed ^ tag) + t) + (k 2^20 + j))
+ * with mix the SplitMix64 finaliser; tag 0 = minibatch index stream, 1 = staleness stream. */
+uint64_t lsam_schedule_hash(uint64_t seed, int tag, uint64_t t, uint64_t k, uint64_t j);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

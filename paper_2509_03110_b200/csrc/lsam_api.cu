@@ -1,0 +1,706 @@
+// lsam_api.cu -- host side of the C ABI declared in include/lsam.h: configuration checks, workspace layout,
+// and the launch sequence of one worker tick (schedule -> gather -> ascent gradient -> norm -> perturb ->
+// descent gradient -> fused update) and of the centre update.  No device memory is allocated here: every
+// buffer is carved from the caller's workspace.
+#include "lsam.h"
+
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+#include "model_kernels.cuh"
+#include "stream_kernels.cuh"
+#include "gemm_tcgen05.cuh"
+
+using namespace lsam;
+
+namespace {
+
+struct LayerInfo {
+  int in, out;
+  int64_t w_unp, b_unp;  // offsets in the unpadded vector
+  int64_t w_pad, b_pad;  // offsets in the padded row
+  bool residual;
+};
+
+struct Layout {
+  bool ok = false;
+  int64_t d = 0, ld = 0;
+  std::vector<LayerInfo> layers;
+  SegMap seg{};
+  int ring = 2;
+  int64_t nchunks = 0;
+  bool vec4 = true;
+  // byte offsets into the workspace
+  size_t x, v, g, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status;
+  size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage;
+  size_t total = 0;
+};
+
+constexpr int64_t kSegAlign = 64;
+
+bool plan(const lsam_config& c, Layout& L) {
+  L = Layout();
+  if (c.K < 1 || c.K > 4096 || c.tau < 1 || c.stale_max < 0 || c.stale_max > 15) return false;
+  if (c.gemm_dtype != LSAM_GEMM_FP32 && c.gemm_dtype != LSAM_GEMM_BF16) return false;
+  if (c.gemm_impl < LSAM_IMPL_AUTO || c.gemm_impl > LSAM_IMPL_TCGEN05) return false;
+  if (!(c.gamma > 0.f)) return false;
+  const bool bf = c.gemm_dtype == LSAM_GEMM_BF16;
+  L.seg.n = 0;
+  if (c.model == LSAM_MODEL_FLAT) {
+    if (c.flat_d < 1 || bf) return false;
+    L.d = c.flat_d;
+    L.ld = round_up(L.d, 4);
+    L.vec4 = (L.d % 4 == 0);
+    L.seg.n = 1;
+    L.seg.src[0] = 0; L.seg.dst[0] = 0; L.seg.len[0] = L.d;
+  } else if (c.model == LSAM_MODEL_LSQ) {
+    if (c.widths[0] < 1 || c.batch < 1 || c.n_samples < 1 || bf) return false;
+    L.d = c.widths[0];
+    L.ld = round_up(L.d, kSegAlign);
+    L.layers.push_back({c.widths[0], 1, 0, -1, 0, -1, false});
+    L.seg.n = 1;
+    L.seg.src[0] = 0; L.seg.dst[0] = 0; L.seg.len[0] = L.d;
+  } else if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {
+    if (c.n_layers < 1 || c.n_layers > 8 || c.batch < 1 || c.n_samples < 1) return false;
+    int64_t unp = 0, pad = 0;
+    for (int l = 0; l < c.n_layers; ++l) {
+      LayerInfo li;
+      li.in = c.widths[l];
+      li.out = c.widths[l + 1];
+      if (li.in < 1 || li.out < 1) return false;
+      li.w_unp = unp; unp += (int64_t)li.in * li.out;
+      li.b_unp = unp; unp += li.out;
+      li.w_pad = pad; pad = round_up(pad + (int64_t)li.in * li.out, kSegAlign);
+      li.b_pad = pad; pad = round_up(pad + li.out, kSegAlign);
+      li.residual = (c.model == LSAM_MODEL_RESMLP) && (l < c.n_layers - 1) && (li.in == li.out);
+      L.layers.push_back(li);
+      L.seg.src[L.seg.n] = li.w_unp; L.seg.dst[L.seg.n] = li.w_pad; L.seg.len[L.seg.n] = (int64_t)li.in * li.out; ++L.seg.n;
+      L.seg.src[L.seg.n] = li.b_unp; L.seg.dst[L.seg.n] = li.b_pad; L.seg.len[L.seg.n] = li.out; ++L.seg.n;
+    }
+    L.d = unp;
+    L.ld = pad;
+  } else {
+    return false;
+  }
+  L.ring = c.stale_max + 2;
+  // partial-sum slots per replica; FLAT may fall back to scalar chunks when the caller's gradient buffers are misaligned
+  L.nchunks = ceil_div(L.ld, (c.model == LSAM_MODEL_FLAT) ? norm_chunk<1>() : norm_chunk<4>());
+
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 256); return o; };
+  const size_t K = c.K, ld = L.ld, B = c.batch > 0 ? c.batch : 1;
+  const size_t esz = bf ? 2 : 4;
+  const bool flat = c.model == LSAM_MODEL_FLAT;
+  L.status = take(256);
+  L.scalars = take(sizeof(float) * 8 * K);  // norm1, norm2, scale, loss (4 x [K], padded)
+  L.x = take(4 * K * ld);
+  L.v = take(4 * K * ld);
+  L.g = flat ? 0 : take(4 * K * ld);
+  L.g1keep = (!flat && (c.flags & LSAM_FLAG_KEEP_G1)) ? take(4 * K * ld) : 0;
+  L.xpkeep = (!flat && bf && (c.flags & LSAM_FLAG_KEEP_G1)) ? take(esz * K * ld) : 0;  // x~ survives the update
+  L.xop = take(esz * K * ld);  // fp32: perturbed point x~;  bf16: operand copy of x, overwritten by x~
+  L.acc = take(4 * ld);
+  L.yring = take(4 * (size_t)L.ring * ld);
+  L.gprev = take(4 * ld);
+  L.tmp = take(4 * ld);
+  L.idx = take(4 * K * B * 2);     // step indices + scratch for lsam_read_schedule
+  L.sched = take(4 * K * 8);       // stale, ver, slot + scratch copies
+  L.partial = take(4 * K * (size_t)L.nchunks);
+  L.ylab = take(4 * K * B);
+  for (int i = 0; i < 9; ++i) L.act[i] = L.mask[i] = 0;
+  L.logits = L.rowloss = L.dz[0] = L.dz[1] = L.dh[0] = L.dh[1] = L.xstage = L.ystage = 0;
+  if (!flat) {
+    const size_t in0 = c.widths[0];
+    L.act[0] = take((c.model == LSAM_MODEL_LSQ ? 4 : esz) * K * B * in0);
+    L.xstage = take(4 * K * B * in0);
+    L.ystage = take(4 * K * B);
+    if (c.model != LSAM_MODEL_LSQ) {
+      size_t maxw = 0;
+      for (size_t l = 0; l < L.layers.size(); ++l) {
+        const size_t w = L.layers[l].out;
+        maxw = w > maxw ? w : maxw;
+        if (l + 1 < L.layers.size()) {
+          L.act[l + 1] = take(esz * K * B * w);
+          L.mask[l] = take(K * B * w);
+        }
+      }
+      L.logits = take(4 * K * B * (size_t)L.layers.back().out);
+      L.rowloss = take(4 * K * B);
+      for (int i = 0; i < 2; ++i) L.dz[i] = take(esz * K * B * maxw);
+      for (int i = 0; i < 2; ++i) L.dh[i] = take(esz * K * B * maxw);
+    }
+  }
+  L.total = off;
+  L.ok = true;
+  return true;
+}
+
+struct Profiler {
+  bool on = false;
+  std::vector<cudaEvent_t> pool;
+  std::vector<int> cls;  // class of record i (events 2i, 2i+1)
+  size_t used = 0;
+};
+
+}  // namespace
+
+struct lsam_ctx {
+  lsam_config cfg;
+  Layout L;
+  char* ws = nullptr;
+  cudaStream_t stream = nullptr;
+  const float* X = nullptr;
+  const uint32_t* Y = nullptr;
+  const float* eg1 = nullptr;
+  const float* eg2 = nullptr;
+  bool ext_vec4 = true;
+  int64_t t = 0, t_y = 0;
+  std::vector<int64_t> t_x;
+  std::vector<int> ver_at_step;
+  bool have_prev = false;
+  bool use_tc = false;
+  int64_t launches = 0;
+  Profiler prof;
+  std::string err;
+  TcPlan tc;
+
+  template <typename T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+  float* x() const { return at<float>(L.x); }
+  float* v() const { return at<float>(L.v); }
+  float* g() const { return at<float>(L.g); }
+  float* norm1() const { return at<float>(L.scalars); }
+  float* norm2() const { return at<float>(L.scalars) + cfg.K; }
+  float* scale() const { return at<float>(L.scalars) + 2 * cfg.K; }
+  float* loss() const { return at<float>(L.scalars) + 3 * cfg.K; }
+  int* status() const { return at<int>(L.status); }
+  int32_t* idx() const { return at<int32_t>(L.idx); }
+  int32_t* idx_scratch() const { return at<int32_t>(L.idx) + (size_t)cfg.K * (cfg.batch > 0 ? cfg.batch : 1); }
+  int32_t* stale() const { return at<int32_t>(L.sched); }
+  int32_t* ver() const { return at<int32_t>(L.sched) + cfg.K; }
+  int32_t* slot() const { return at<int32_t>(L.sched) + 2 * cfg.K; }
+  int32_t* sched_scratch() const { return at<int32_t>(L.sched) + 4 * cfg.K; }
+  float* yslot(int64_t version) const { return at<float>(L.yring) + (size_t)(version % L.ring) * L.ld; }
+
+  int fail(int code, const std::string& m) { err = m; return code; }
+};
+
+namespace {
+
+#define LSAM_CUDA(ctx, call)                                                                          \
+  do {                                                                                                \
+    cudaError_t e__ = (call);                                                                         \
+    if (e__ != cudaSuccess)                                                                           \
+      return (ctx)->fail(LSAM_ERR_CUDA, std::string(#call) + ": " + cudaGetErrorString(e__));         \
+  } while (0)
+
+int prof_begin(lsam_ctx* c, int cls) {
+  c->launches += 1;
+  if (!c->prof.on) return LSAM_OK;
+  Profiler& p = c->prof;
+  while (p.pool.size() < 2 * (p.used + 1)) {
+    cudaEvent_t e;
+    LSAM_CUDA(c, cudaEventCreate(&e));
+    p.pool.push_back(e);
+  }
+  if (p.cls.size() <= p.used) p.cls.resize(p.used + 1);
+  p.cls[p.used] = cls;
+  LSAM_CUDA(c, cudaEventRecord(p.pool[2 * p.used], c->stream));
+  return LSAM_OK;
+}
+int prof_end(lsam_ctx* c) {
+  LSAM_CUDA(c, cudaPeekAtLastError());
+  if (!c->prof.on) return LSAM_OK;
+  Profiler& p = c->prof;
+  LSAM_CUDA(c, cudaEventRecord(p.pool[2 * p.used + 1], c->stream));
+  p.used += 1;
+  return LSAM_OK;
+}
+// LAUNCH(ctx, class, kernel<<<...>>>(...));
+#define LAUNCH(ctx, cls, ...)                                  \
+  do {                                                         \
+    int rc__ = prof_begin((ctx), (cls));                       \
+    if (rc__ != LSAM_OK) return rc__;                          \
+    __VA_ARGS__;                                               \
+    rc__ = prof_end((ctx));                                    \
+    if (rc__ != LSAM_OK) return rc__;                          \
+  } while (0)
+
+// ---- norm of [K, n] rows -> norm_out[K] (and scale[K] = rho / (norm + gamma) if scale_out)
+int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float rho, float* norm_out, float* scale_out) {
+  float* partial = c->at<float>(c->L.partial);
+  const int64_t nch = c->L.nchunks;
+  dim3 grid((unsigned)ceil_div(n, vec4 ? norm_chunk<4>() : norm_chunk<1>()), c->cfg.K);
+  if ((int64_t)grid.x > nch) return c->fail(LSAM_ERR_WORKSPACE, "norm: partial-sum buffer too small");
+  if (vec4) LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<4><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch));
+  else LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<1><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch));
+  LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)grid.x, rho, c->cfg.gamma, norm_out, scale_out, c->status()));
+  return LSAM_OK;
+}
+
+template <typename TP>
+int launch_perturb(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4) {
+  TP* xt = c->at<TP>(c->L.xop);
+  const int64_t per = (int64_t)kPertThreads * kPertIter * (vec4 ? 4 : 1);
+  dim3 grid((unsigned)ceil_div(n, per), c->cfg.K);
+  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld));
+  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld));
+  return LSAM_OK;
+}
+
+int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float eta) {
+  UpdateArgs a;
+  a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
+  a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
+  a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
+  const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16;
+  const bool nes = c->cfg.nesterov != 0;
+  const unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
+#define LSAM_UPD_LAUNCH(V, N, T, W) LAUNCH(c, LSAM_PROF_UPDATE, update_kernel<V, N, T, W><<<grid, kUpdThreads, 0, c->stream>>>(a))
+  if (vec4) {
+    if (bf) { if (nes) LSAM_UPD_LAUNCH(4, true, bf16, true); else LSAM_UPD_LAUNCH(4, false, bf16, true); }
+    else    { if (nes) LSAM_UPD_LAUNCH(4, true, float, false); else LSAM_UPD_LAUNCH(4, false, float, false); }
+  } else {
+    if (bf) { if (nes) LSAM_UPD_LAUNCH(1, true, bf16, true); else LSAM_UPD_LAUNCH(1, false, bf16, true); }
+    else    { if (nes) LSAM_UPD_LAUNCH(1, true, float, false); else LSAM_UPD_LAUNCH(1, false, float, false); }
+  }
+#undef LSAM_UPD_LAUNCH
+  return LSAM_OK;
+}
+
+int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot) {
+  VerHist h;
+  for (int s = 0; s < 16; ++s) {
+    const int64_t ts = t - s > 0 ? t - s : 0;
+    h.v[s] = ts < (int64_t)c->ver_at_step.size() ? c->ver_at_step[(size_t)ts] : -1;
+  }
+  const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
+  LAUNCH(c, LSAM_PROF_SCHEDULE,
+         schedule_kernel<<<c->cfg.K, 128, 0, c->stream>>>(c->cfg.seed, (uint64_t)t, flat ? 1 : c->cfg.n_samples, flat ? 0 : c->cfg.batch,
+                                                           c->cfg.stale_max, h, c->L.ring, flat ? nullptr : idx, stale, ver, slot));
+  return LSAM_OK;
+}
+
+// ---- SIMT GEMM launches in logical coordinates
+template <typename TA, typename TB, class Epi>
+int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N, int Kd, const Epi& epi) {
+  dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), c->cfg.K);
+  LAUNCH(c, cls, gemm_simt_kernel<TA, TB, Epi><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi));
+  return LSAM_OK;
+}
+
+// One gradient pass of the classifier at the parameters P ([K, ld], type T); gradient -> g, loss -> loss_out (nullable).
+template <typename T>
+int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
+  const Layout& L = c->L;
+  const int K = c->cfg.K, B = c->cfg.batch;
+  const int nl = (int)L.layers.size();
+  const int64_t ld = L.ld;
+  int rc;
+  // forward
+  for (int l = 0; l < nl; ++l) {
+    const LayerInfo& li = L.layers[l];
+    const T* a_in = c->at<T>(L.act[l]);
+    const bool head = (l == nl - 1);
+    if (c->use_tc) {
+      rc = tc_forward(c->tc, l, c->stream);
+      if (rc != 0) return c->fail(LSAM_ERR_CUDA, "tcgen05 forward launch failed");
+      continue;
+    }
+    GemmOperand A{a_in, (int64_t)B * li.in, li.in, 1};      // (z, b, i)
+    GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, o, i)
+    if (head) {
+      EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), B, li.out};
+      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
+    } else {
+      EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.act[l + 1]), li.residual ? a_in : nullptr, c->at<uint8_t>(L.mask[l]), B, li.out};
+      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
+    }
+    if (rc != LSAM_OK) return rc;
+  }
+  // loss and its gradient w.r.t. the logits
+  const int C = L.layers[nl - 1].out;
+  const int64_t rows = (int64_t)K * B;
+  int cur = 0;
+  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<(unsigned)ceil_div(rows, 8), 256, 0, c->stream>>>(
+      c->at<float>(L.logits), c->at<int32_t>(L.ylab), rows, C, B, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status()));
+  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out));
+  // backward
+  for (int l = nl - 1; l >= 0; --l) {
+    const LayerInfo& li = L.layers[l];
+    const T* dz = c->at<T>(L.dz[cur]);
+    const T* a_in = c->at<T>(L.act[l]);
+    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 256), K), 256, 0, c->stream>>>(dz, B, li.out, c->g(), ld, li.b_pad));
+    if (c->use_tc) {
+      rc = tc_backward(c->tc, l, cur, c->stream);
+      if (rc != 0) return c->fail(LSAM_ERR_CUDA, "tcgen05 backward launch failed");
+      cur ^= 1;
+      continue;
+    }
+    {
+      GemmOperand A{dz, (int64_t)B * li.out, 1, li.out};     // (z, o, b)
+      GemmOperand Bm{a_in, (int64_t)B * li.in, 1, li.in};    // (z, i, b)
+      EpiWgrad e{c->g(), ld, li.w_pad, li.in};
+      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.out, li.in, B, e);
+      if (rc != LSAM_OK) return rc;
+    }
+    if (l > 0) {
+      GemmOperand A{dz, (int64_t)B * li.out, li.out, 1};     // (z, b, o)
+      GemmOperand W{P + li.w_pad, ld, 1, li.in};             // (z, i, o)
+      EpiDgrad<T> e{li.residual ? c->at<T>(L.dh[(l + 1) & 1]) : nullptr,
+                    L.layers[l - 1].residual ? c->at<T>(L.dh[l & 1]) : nullptr,
+                    c->at<T>(L.dz[cur ^ 1]), c->at<uint8_t>(L.mask[l - 1]), B, li.in};
+      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_DGRAD, A, W, B, li.in, li.out, e);
+      if (rc != LSAM_OK) return rc;
+    }
+    cur ^= 1;
+  }
+  return LSAM_OK;
+}
+
+// Gradient of the minibatch loss at the parameters held in `params` (x master, or the operand buffer).
+int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out) {
+  const lsam_config& cfg = c->cfg;
+  if (cfg.model == LSAM_MODEL_LSQ) {
+    const float* P = perturbed ? c->at<float>(c->L.xop) : c->x();
+    LAUNCH(c, LSAM_PROF_LSQ_GRAD, lsq_grad_kernel<<<cfg.K, 256, sizeof(float) * cfg.batch, c->stream>>>(
+        c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, cfg.widths[0], c->g(), c->L.ld, loss_out));
+    return LSAM_OK;
+  }
+  if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out);
+  return mlp_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out);
+}
+
+int refresh_operand_copy(lsam_ctx* c) {
+  if (c->cfg.gemm_dtype != LSAM_GEMM_BF16) return LSAM_OK;
+  dim3 grid((unsigned)ceil_div(c->L.ld, 256), c->cfg.K);
+  LAUNCH(c, LSAM_PROF_COPY, cast_rows_kernel<bf16><<<grid, 256, 0, c->stream>>>(c->x(), c->L.ld, c->at<bf16>(c->L.xop), c->L.ld, c->L.ld));
+  return LSAM_OK;
+}
+
+template <bool TO_PADDED>
+int seg_copy(lsam_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd, int rows) {
+  int64_t maxlen = 0;
+  for (int i = 0; i < c->L.seg.n; ++i) maxlen = c->L.seg.len[i] > maxlen ? c->L.seg.len[i] : maxlen;
+  dim3 grid((unsigned)ceil_div(maxlen, 256), c->L.seg.n, rows);
+  LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<TO_PADDED, float, float><<<grid, 256, 0, c->stream>>>(src, lds, dst, ldd, c->L.seg));
+  return LSAM_OK;
+}
+
+int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
+  const lsam_config& cfg = c->cfg;
+  const Layout& L = c->L;
+  const bool flat = cfg.model == LSAM_MODEL_FLAT;
+  if (flat && (!c->eg1 || !c->eg2)) return c->fail(LSAM_ERR_STATE, "FLAT model: call lsam_set_external_grads first");
+  int rc;
+  c->ver_at_step.push_back((int)c->t_y);  // centre version current when this tick starts
+  if ((rc = launch_schedule(c, c->t, c->idx(), c->stale(), c->ver(), c->slot())) != LSAM_OK) return rc;
+  const int64_t rows = (int64_t)cfg.K * cfg.batch;
+  if (!flat && gather) {
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16)
+      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<bf16><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+    else
+      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+  }
+  const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
+  const int64_t n = flat ? L.d : L.ld;
+  const int64_t ldg = flat ? L.d : L.ld;
+  // ascent gradient, its norm, perturbation
+  const float* g1 = flat ? c->eg1 : c->g();
+  if (!flat && (rc = grad_pass(c, false, c->loss())) != LSAM_OK) return rc;
+  if (!flat && L.g1keep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
+  if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
+  if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16>(c, g1, ldg, n, vec4);
+  else rc = launch_perturb<float>(c, g1, ldg, n, vec4);
+  if (rc != LSAM_OK) return rc;
+  if (L.xpkeep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.xpkeep), c->at<bf16>(L.xop), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
+  // descent gradient at the perturbed point, same minibatch
+  const float* g2 = flat ? c->eg2 : c->g();
+  if (!flat && (rc = grad_pass(c, true, nullptr)) != LSAM_OK) return rc;
+  if (cfg.flags & LSAM_FLAG_STEP_INFO)
+    if ((rc = launch_norm(c, g2, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
+  // fused worker update
+  if ((rc = launch_update(c, g2, ldg, n, vec4, eta)) != LSAM_OK) return rc;
+  for (auto& tx : c->t_x) tx += 1;
+  c->t += 1;
+  return LSAM_OK;
+}
+
+}  // namespace
+
+// =================================================================================================== C ABI
+extern "C" {
+
+uint64_t lsam_schedule_hash(uint64_t seed, int tag, uint64_t t, uint64_t k, uint64_t j) {
+  return schedule_hash(seed, tag == 0 ? kTagIdx : kTagStale, t, k, j);
+}
+
+int64_t lsam_param_count(const lsam_config* cfg) {
+  Layout L;
+  if (!cfg || !plan(*cfg, L)) return -1;
+  return L.d;
+}
+
+size_t lsam_workspace_bytes(const lsam_config* cfg) {
+  Layout L;
+  if (!cfg || !plan(*cfg, L)) return 0;
+  return L.total;
+}
+
+int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const void* d_Y, const float* d_x0,
+              const float* d_y0, void* d_workspace, size_t workspace_bytes, void* cuda_stream) {
+  if (!out) return LSAM_ERR_INVALID;
+  *out = nullptr;
+  if (!cfg || !d_x0 || !d_y0 || !d_workspace) return LSAM_ERR_INVALID;
+  Layout L;
+  if (!plan(*cfg, L)) return LSAM_ERR_INVALID;
+  if (cfg->model != LSAM_MODEL_FLAT && (!d_X || !d_Y)) return LSAM_ERR_INVALID;
+  if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(d_workspace) & 255) != 0) return LSAM_ERR_WORKSPACE;
+  lsam_ctx* c = new lsam_ctx();
+  c->cfg = *cfg;
+  c->L = L;
+  c->ws = reinterpret_cast<char*>(d_workspace);
+  c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  c->X = reinterpret_cast<const float*>(d_X);
+  c->Y = reinterpret_cast<const uint32_t*>(d_Y);
+  c->t_x.assign(cfg->K, 0);
+  auto bail = [&](int code) { delete c; return code; };
+  // tensor-core path: decided once per context
+  const bool mlp = cfg->model == LSAM_MODEL_MLP || cfg->model == LSAM_MODEL_RESMLP;
+  bool tc_ok = false;
+  if (mlp && cfg->gemm_dtype == LSAM_GEMM_BF16 && cfg->gemm_impl != LSAM_IMPL_SIMT) tc_ok = tc_supported(*cfg);
+  if (cfg->gemm_impl == LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
+  c->use_tc = tc_ok;
+  if (cudaMemsetAsync(c->ws, 0, L.total, c->stream) != cudaSuccess) return bail(LSAM_ERR_CUDA);
+  int rc;
+  if ((rc = seg_copy<true>(c, d_x0, L.d, c->x(), L.ld, cfg->K)) != LSAM_OK) return bail(rc);
+  if ((rc = seg_copy<true>(c, d_y0, L.d, c->yslot(0), L.ld, 1)) != LSAM_OK) return bail(rc);
+  if ((rc = refresh_operand_copy(c)) != LSAM_OK) return bail(rc);
+  if (c->use_tc) {
+    TcBuffers b;
+    b.xop = c->at<bf16>(L.xop); b.g = c->g(); b.ld = L.ld;
+    for (int i = 0; i < 9; ++i) { b.act[i] = c->at<bf16>(L.act[i]); b.mask[i] = c->at<uint8_t>(L.mask[i]); }
+    b.logits = c->at<float>(L.logits);
+    for (int i = 0; i < 2; ++i) { b.dz[i] = c->at<bf16>(L.dz[i]); b.dh[i] = c->at<bf16>(L.dh[i]); }
+    b.status = c->status();
+    std::vector<TcLayer> tl;
+    for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
+    std::string why;
+    if (tc_plan(c->tc, *cfg, tl, b, &c->launches, why) != 0) { delete c; return LSAM_ERR_CUDA; }
+  }
+  *out = c;
+  return LSAM_OK;
+}
+
+int lsam_step(lsam_ctx* c, float eta, float rho) {
+  if (!c) return LSAM_ERR_INVALID;
+  return step_common(c, eta, rho, true);
+}
+
+int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const void* yb, int on_host, float* h_loss) {
+  if (!c || !xb || !yb) return LSAM_ERR_INVALID;
+  const lsam_config& cfg = c->cfg;
+  if (cfg.model == LSAM_MODEL_FLAT) return c->fail(LSAM_ERR_INVALID, "lsam_step_batch: not available for FLAT");
+  const int64_t rows = (int64_t)cfg.K * cfg.batch;
+  const int64_t nx = rows * cfg.widths[0];
+  const cudaMemcpyKind kind = on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+  const bool conv = cfg.gemm_dtype == LSAM_GEMM_BF16;
+  float* xdst = conv ? c->at<float>(c->L.xstage) : c->at<float>(c->L.act[0]);
+  c->launches += 2;
+  LSAM_CUDA(c, cudaMemcpyAsync(xdst, xb, sizeof(float) * nx, kind, c->stream));
+  LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(c->L.ylab), yb, 4 * rows, kind, c->stream));
+  if (conv)
+    LAUNCH(c, LSAM_PROF_GATHER, convert_batch_kernel<bf16><<<(unsigned)ceil_div(nx, 256), 256, 0, c->stream>>>(xdst, c->at<bf16>(c->L.act[0]), nx));
+  int rc = step_common(c, eta, rho, false);
+  if (rc != LSAM_OK) return rc;
+  if (h_loss) {
+    LSAM_CUDA(c, cudaMemcpyAsync(h_loss, c->loss(), sizeof(float) * cfg.K, cudaMemcpyDeviceToHost, c->stream));
+    LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  }
+  return LSAM_OK;
+}
+
+int lsam_should_couple(const lsam_ctx* c) {
+  if (!c) return 0;
+  int64_t s = 0;
+  for (int64_t v : c->t_x) s += v;
+  return (s > 0 && s % ((int64_t)c->cfg.K * c->cfg.tau) == 0) ? 1 : 0;
+}
+
+int lsam_couple(lsam_ctx* c) {
+  if (!c) return LSAM_ERR_INVALID;
+  if (!lsam_should_couple(c)) return c->fail(LSAM_ERR_STATE, "lsam_couple: sync trigger is false");
+  const Layout& L = c->L;
+  const float inv = 1.0f / ((float)c->cfg.K * (float)c->cfg.tau);
+  LAUNCH(c, LSAM_PROF_COUPLE, couple_kernel<<<(unsigned)ceil_div(L.ld, 256), 256, 0, c->stream>>>(
+      c->at<float>(L.acc), c->yslot(c->t_y), c->yslot(c->t_y + 1), c->at<float>(L.gprev), L.ld, inv, c->cfg.beta, c->cfg.eta_prime, c->have_prev ? 1 : 0));
+  c->have_prev = true;
+  c->t_y += 1;
+  for (auto& tx : c->t_x) tx = 0;
+  return LSAM_OK;
+}
+
+int lsam_read_params(lsam_ctx* c, int which, float* dst, int64_t n, int dst_on_device) {
+  if (!c || !dst || which < -1 || which >= c->cfg.K) return LSAM_ERR_INVALID;
+  if (n < c->L.d) return c->fail(LSAM_ERR_INVALID, "lsam_read_params: destination too small");
+  const float* src = which < 0 ? c->yslot(c->t_y) : c->x() + (size_t)which * c->L.ld;
+  int rc;
+  if (dst_on_device) return seg_copy<false>(c, src, c->L.ld, dst, c->L.d, 1);
+  float* tmp = c->at<float>(c->L.tmp);
+  if ((rc = seg_copy<false>(c, src, c->L.ld, tmp, c->L.d, 1)) != LSAM_OK) return rc;
+  LSAM_CUDA(c, cudaMemcpyAsync(dst, tmp, sizeof(float) * c->L.d, cudaMemcpyDeviceToHost, c->stream));
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LSAM_OK;
+}
+
+int lsam_read_schedule(lsam_ctx* c, int64_t t, int32_t* h_idx, int32_t* h_stale, int32_t* h_ver) {
+  if (!c || t < 0) return LSAM_ERR_INVALID;
+  if (h_ver && t >= (int64_t)c->ver_at_step.size()) return c->fail(LSAM_ERR_STATE, "lsam_read_schedule: centre version of a future step");
+  const int K = c->cfg.K;
+  int32_t* s = c->sched_scratch();
+  int rc = launch_schedule(c, t, c->idx_scratch(), s, s + K, s + 2 * K);
+  if (rc != LSAM_OK) return rc;
+  if (h_idx && c->cfg.model != LSAM_MODEL_FLAT)
+    LSAM_CUDA(c, cudaMemcpyAsync(h_idx, c->idx_scratch(), 4 * (size_t)K * c->cfg.batch, cudaMemcpyDeviceToHost, c->stream));
+  if (h_stale) LSAM_CUDA(c, cudaMemcpyAsync(h_stale, s, 4 * K, cudaMemcpyDeviceToHost, c->stream));
+  if (h_ver) LSAM_CUDA(c, cudaMemcpyAsync(h_ver, s + K, 4 * K, cudaMemcpyDeviceToHost, c->stream));
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LSAM_OK;
+}
+
+int lsam_read_step_info(lsam_ctx* c, float* h_loss, float* h_gnorm1, float* h_gnorm2) {
+  if (!c) return LSAM_ERR_INVALID;
+  const size_t n = sizeof(float) * c->cfg.K;
+  if (h_loss) LSAM_CUDA(c, cudaMemcpyAsync(h_loss, c->loss(), n, cudaMemcpyDeviceToHost, c->stream));
+  if (h_gnorm1) LSAM_CUDA(c, cudaMemcpyAsync(h_gnorm1, c->norm1(), n, cudaMemcpyDeviceToHost, c->stream));
+  if (h_gnorm2) LSAM_CUDA(c, cudaMemcpyAsync(h_gnorm2, c->norm2(), n, cudaMemcpyDeviceToHost, c->stream));
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LSAM_OK;
+}
+
+int lsam_read_grads(lsam_ctx* c, int pass, float* h_dst) {
+  if (!c || !h_dst || pass < 1 || pass > 3) return LSAM_ERR_INVALID;
+  const Layout& L = c->L;
+  const int K = c->cfg.K;
+  const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
+  float* tmp = c->at<float>(L.tmp);
+  for (int k = 0; k < K; ++k) {
+    int rc = LSAM_OK;
+    if (pass == 3) {
+      if (c->cfg.gemm_dtype == LSAM_GEMM_BF16) {
+        if (!L.xpkeep) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(3) in BF16 mode needs LSAM_FLAG_KEEP_G1");
+        int64_t maxlen = 0;
+        for (int i = 0; i < L.seg.n; ++i) maxlen = L.seg.len[i] > maxlen ? L.seg.len[i] : maxlen;
+        dim3 grid((unsigned)ceil_div(maxlen, 256), L.seg.n, 1);
+        LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(c->at<bf16>(L.xpkeep) + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
+      } else {
+        rc = seg_copy<false>(c, c->at<float>(L.xop) + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
+      }
+    } else if (flat) {
+      const float* src = pass == 1 ? c->eg1 : c->eg2;
+      if (!src) return c->fail(LSAM_ERR_STATE, "no external gradients set");
+      LSAM_CUDA(c, cudaMemcpyAsync(tmp, src + (size_t)k * L.d, sizeof(float) * L.d, cudaMemcpyDeviceToDevice, c->stream));
+    } else {
+      if (pass == 1 && !L.g1keep) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(1) needs LSAM_FLAG_KEEP_G1");
+      const float* src = pass == 1 ? c->at<float>(L.g1keep) : c->g();
+      rc = seg_copy<false>(c, src + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
+    }
+    if (rc != LSAM_OK) return rc;
+    LSAM_CUDA(c, cudaMemcpyAsync(h_dst + (size_t)k * L.d, tmp, sizeof(float) * L.d, cudaMemcpyDeviceToHost, c->stream));
+    LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  }
+  return LSAM_OK;
+}
+
+int lsam_set_external_grads(lsam_ctx* c, const float* d_g1, const float* d_g2) {
+  if (!c || !d_g1 || !d_g2) return LSAM_ERR_INVALID;
+  if (c->cfg.model != LSAM_MODEL_FLAT) return c->fail(LSAM_ERR_INVALID, "external gradients are for the FLAT model only");
+  c->eg1 = d_g1;
+  c->eg2 = d_g2;
+  c->ext_vec4 = ((reinterpret_cast<uintptr_t>(d_g1) | reinterpret_cast<uintptr_t>(d_g2)) & 15) == 0;
+  return LSAM_OK;
+}
+
+int lsam_write_state(lsam_ctx* c, const float* d_x, const float* d_v, const float* d_y) {
+  if (!c) return LSAM_ERR_INVALID;
+  int rc;
+  if (d_x && (rc = seg_copy<true>(c, d_x, c->L.d, c->x(), c->L.ld, c->cfg.K)) != LSAM_OK) return rc;
+  if (d_v && (rc = seg_copy<true>(c, d_v, c->L.d, c->v(), c->L.ld, c->cfg.K)) != LSAM_OK) return rc;
+  if (d_y && (rc = seg_copy<true>(c, d_y, c->L.d, c->yslot(c->t_y), c->L.ld, 1)) != LSAM_OK) return rc;
+  if (d_x) return refresh_operand_copy(c);
+  return LSAM_OK;
+}
+
+int lsam_read_state(lsam_ctx* c, float* h_v, float* h_acc, float* h_gprev) {
+  if (!c) return LSAM_ERR_INVALID;
+  const Layout& L = c->L;
+  float* tmp = c->at<float>(L.tmp);
+  auto one = [&](const float* src, float* dst) -> int {
+    int rc = seg_copy<false>(c, src, L.ld, tmp, L.d, 1);
+    if (rc != LSAM_OK) return rc;
+    LSAM_CUDA(c, cudaMemcpyAsync(dst, tmp, sizeof(float) * L.d, cudaMemcpyDeviceToHost, c->stream));
+    LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+    return LSAM_OK;
+  };
+  int rc;
+  if (h_v)
+    for (int k = 0; k < c->cfg.K; ++k)
+      if ((rc = one(c->v() + (size_t)k * L.ld, h_v + (size_t)k * L.d)) != LSAM_OK) return rc;
+  if (h_acc && (rc = one(c->at<float>(L.acc), h_acc)) != LSAM_OK) return rc;
+  if (h_gprev && (rc = one(c->at<float>(L.gprev), h_gprev)) != LSAM_OK) return rc;
+  return LSAM_OK;
+}
+
+int lsam_read_counters(const lsam_ctx* c, int64_t* t, int64_t* t_y, int64_t* h_t_x) {
+  if (!c) return LSAM_ERR_INVALID;
+  if (t) *t = c->t;
+  if (t_y) *t_y = c->t_y;
+  if (h_t_x) std::memcpy(h_t_x, c->t_x.data(), sizeof(int64_t) * c->t_x.size());
+  return LSAM_OK;
+}
+
+int lsam_status(lsam_ctx* c) {
+  if (!c) return LSAM_ERR_INVALID;
+  int h = 0;
+  LSAM_CUDA(c, cudaMemcpyAsync(&h, c->status(), sizeof(int), cudaMemcpyDeviceToHost, c->stream));
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (h & STATUS_TIMEOUT) return c->fail(LSAM_ERR_TIMEOUT, "a bounded device-side wait expired");
+  if (h & STATUS_NONFINITE) return c->fail(LSAM_ERR_NONFINITE, "a gradient norm was not finite");
+  if (h & STATUS_BAD_INDEX) return c->fail(LSAM_ERR_INVALID, "a sample index or label was out of range");
+  return LSAM_OK;
+}
+
+int lsam_profile_enable(lsam_ctx* c, int enable) {
+  if (!c) return LSAM_ERR_INVALID;
+  c->prof.on = enable != 0;
+  return LSAM_OK;
+}
+
+int lsam_profile_read(lsam_ctx* c, double* h_ms, int64_t* h_launches) {
+  if (!c) return LSAM_ERR_INVALID;
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  Profiler& p = c->prof;
+  for (size_t i = 0; i < p.used; ++i) {
+    float ms = 0.f;
+    LSAM_CUDA(c, cudaEventElapsedTime(&ms, p.pool[2 * i], p.pool[2 * i + 1]));
+    const int cl = p.cls[i];
+    if (h_ms) h_ms[cl] += (double)ms;
+    if (h_launches) h_launches[cl] += 1;
+  }
+  p.used = 0;
+  return LSAM_OK;
+}
+
+int64_t lsam_launch_count(const lsam_ctx* c) { return c ? c->launches : 0; }
+int lsam_uses_tcgen05(const lsam_ctx* c) { return (c && c->use_tc) ? 1 : 0; }
+const char* lsam_last_error(const lsam_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+void lsam_destroy(lsam_ctx* c) {
+  if (!c) return;
+  for (cudaEvent_t e : c->prof.pool) cudaEventDestroy(e);
+  delete c;
+}
+
+}  // extern "C"

@@ -1,0 +1,243 @@
+// model_kernels.cuh -- minibatch gather, GEMM epilogues, softmax cross-entropy, bias gradient, least squares,
+// and the SIMT batched GEMM used for fp32 models and for shapes the tensor-core path does not cover.
+#pragma once
+
+#include "common.cuh"
+
+namespace lsam {
+
+// ------------------------------------------------------------------------------------------------ S1 gather
+// xb[k][b][:] = TA(X[idx[k][b]][:]);  yb[k][b] = Y[idx[k][b]] (4-byte elements).  grid (K*B), block 128.
+template <typename TA>
+__global__ void __launch_bounds__(128)
+gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx,
+              int64_t n_samples, int in, TA* __restrict__ xb, uint32_t* __restrict__ yb, int* __restrict__ status) {
+  const int64_t r = blockIdx.x;
+  int64_t s = idx[r];
+  if (s < 0 || s >= n_samples) {
+    if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_INDEX);
+    s = 0;
+  }
+  const float* src = X + s * in;
+  TA* dst = xb + r * in;
+  for (int i = threadIdx.x; i < in; i += blockDim.x) dst[i] = from_float<TA>(src[i]);
+  if (threadIdx.x == 0 && yb != nullptr) yb[r] = Y[s];
+}
+
+// Caller-supplied minibatch: convert [rows, in] fp32 to the activation type.
+template <typename TA>
+__global__ void __launch_bounds__(256)
+convert_batch_kernel(const float* __restrict__ src, TA* __restrict__ dst, int64_t n) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j < n) dst[j] = from_float<TA>(src[j]);
+}
+
+// ------------------------------------------------------------------------------------------------ epilogues
+// Every GEMM hands its accumulator to one of these functors in LOGICAL coordinates:
+//   z = replica, b = sample in the minibatch, f = feature (output unit for forward, input unit for dgrad),
+//   or (z, o, i) = (replica, output unit, input unit) for the weight gradient.
+// TP = parameter operand type, TA = activation storage type.
+
+// hidden layer: v = acc + bias[f]; r = relu(v); mask = v > 0; out = TA(skip + r)
+template <typename TP, typename TA>
+struct EpiFwdHidden {
+  const TP* bias;  int64_t ld_p;           // bias[z * ld_p + f]
+  TA* out;  const TA* skip;  uint8_t* mask;  // [K, B, width]
+  int B, width;
+  __device__ inline void operator()(int z, int b, int f, float acc) const {
+    const float v = acc + to_float(bias[(int64_t)z * ld_p + f]);
+    const int64_t e = ((int64_t)z * B + b) * width + f;
+    const float r = v > 0.f ? v : 0.f;
+    mask[e] = v > 0.f;
+    const float sk = skip ? to_float(skip[e]) : 0.f;
+    out[e] = from_float<TA>(sk + r);
+  }
+};
+
+// head: logits = acc + bias[f]  (fp32, not rounded)
+template <typename TP>
+struct EpiFwdHead {
+  const TP* bias;  int64_t ld_p;
+  float* logits;  // [K, B, C]
+  int B, width;
+  __device__ inline void operator()(int z, int b, int f, float acc) const {
+    logits[((int64_t)z * B + b) * width + f] = acc + to_float(bias[(int64_t)z * ld_p + f]);
+  }
+};
+
+// dgrad of layer l: dh = TA(acc + skip_grad);  dz_prev = mask_prev ? dh : 0;  optionally keep dh (residual nets)
+template <typename TA>
+struct EpiDgrad {
+  const TA* dh_next;      // gradient w.r.t. the output of a residual layer (nullptr otherwise) [K, B, width]
+  TA* dh_out;             // nullable
+  TA* dz_prev;            // [K, B, width]
+  const uint8_t* mask_prev;
+  int B, width;
+  __device__ inline void operator()(int z, int b, int f, float acc) const {
+    const int64_t e = ((int64_t)z * B + b) * width + f;
+    const float s = dh_next ? acc + to_float(dh_next[e]) : acc;
+    const TA q = from_float<TA>(s);
+    if (dh_out) dh_out[e] = q;
+    dz_prev[e] = mask_prev[e] ? q : from_float<TA>(0.f);
+  }
+};
+
+// wgrad: g[z][w_off + o * in + i] = acc
+struct EpiWgrad {
+  float* g;  int64_t ld_g, w_off;  int in;
+  __device__ inline void operator()(int z, int o, int i, float acc) const {
+    g[(int64_t)z * ld_g + w_off + (int64_t)o * in + i] = acc;
+  }
+};
+
+// ------------------------------------------------------------------------------------------------ SIMT batched GEMM
+// C(z, m, n) = sum_kk A(z, m, kk) * B(z, n, kk), accumulated in fp32 in ascending kk; arbitrary element strides.
+// 64 x 64 tile, 16-deep slices, 256 threads, 4 x 4 outputs per thread.  SWAP_MN hands (z, n, m) to the epilogue.
+struct GemmOperand { const void* p; int64_t sz, sr, sk; };  // element (z, r, kk) at p[z*sz + r*sr + kk*sk]
+
+template <typename TA_, typename TB_, class Epi>
+__global__ void __launch_bounds__(256)
+gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi) {
+  constexpr int BM = 64, BN = 64, BK = 16;
+  __shared__ float As[BK][BM + 4];
+  __shared__ float Bs[BK][BN + 4];
+  const int z = blockIdx.z;
+  const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+  const TA_* Ap = reinterpret_cast<const TA_*>(A.p) + (int64_t)z * A.sz;
+  const TB_* Bp = reinterpret_cast<const TB_*>(Bo.p) + (int64_t)z * Bo.sz;
+  const int tid = threadIdx.x;
+  const int tx = tid & 15, ty = tid >> 4;
+  // loader mapping: along the contiguous direction of each operand
+  const bool a_kc = (A.sk == 1), b_kc = (Bo.sk == 1);
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  for (int k0 = 0; k0 < Kd; k0 += BK) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int lin = e * 256 + tid;
+      int r, kk;
+      if (a_kc) { kk = lin & 15; r = lin >> 4; } else { r = lin & 63; kk = lin >> 6; }
+      const int gm = m0 + r, gk = k0 + kk;
+      As[kk][r] = (gm < M && gk < Kd) ? to_float(Ap[(int64_t)gm * A.sr + (int64_t)gk * A.sk]) : 0.f;
+      if (b_kc) { kk = lin & 15; r = lin >> 4; } else { r = lin & 63; kk = lin >> 6; }
+      const int gn = n0 + r;
+      const int gk2 = k0 + kk;
+      Bs[kk][r] = (gn < N && gk2 < Kd) ? to_float(Bp[(int64_t)gn * Bo.sr + (int64_t)gk2 * Bo.sk]) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int kk = 0; kk < BK; ++kk) {
+      const float4 av = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
+      const float a_[4] = {av.x, av.y, av.z, av.w};
+      const float b_[4] = {bv.x, bv.y, bv.z, bv.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a_[i], b_[j], acc[i][j]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int gm = m0 + ty * 4 + i;
+    if (gm >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int gn = n0 + tx * 4 + j;
+      if (gn < N) epi(z, gm, gn, acc[i][j]);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ softmax cross-entropy
+// One warp per sample row.  rowloss[r] = logsumexp(l) - l[y];  dz[r][c] = TA((softmax(l)[c] - [c == y]) / B).
+template <typename TA>
+__global__ void __launch_bounds__(256)
+softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int64_t rows, int C, int B,
+                  TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status) {
+  const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const int lane = threadIdx.x & 31;
+  const float* lg = logits + r * C;
+  float m = -INFINITY;
+  for (int c = lane; c < C; c += 32) m = fmaxf(m, lg[c]);
+  m = warp_max(m);
+  float se = 0.f;
+  for (int c = lane; c < C; c += 32) se += expf(lg[c] - m);
+  se = warp_sum(se);
+  int y = labels[r];
+  if (y < 0 || y >= C) {
+    if (lane == 0) atomicOr(status, STATUS_BAD_INDEX);
+    y = 0;
+  }
+  if (lane == 0) rowloss[r] = (m + logf(se)) - lg[y];
+  const float inv = 1.f / se, invB = 1.f / (float)B;
+  TA* out = dz + r * C;
+  for (int c = lane; c < C; c += 32) {
+    const float p = expf(lg[c] - m) * inv;
+    out[c] = from_float<TA>((p - (c == y ? 1.f : 0.f)) * invB);
+  }
+}
+
+// loss[k] = mean over the minibatch of rowloss[k][b], samples added in ascending order.  grid K, block 32.
+__global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float* __restrict__ loss) {
+  const int k = blockIdx.x;
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int b = 0; b < B; ++b) s += (double)rowloss[(int64_t)k * B + b];
+    loss[k] = (float)(s / B);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ bias gradient
+// g[z][b_off + o] = sum_b dz[z][b][o], samples in ascending order.  grid (ceil(out / 256), K).
+template <typename TA>
+__global__ void __launch_bounds__(256)
+bias_grad_kernel(const TA* __restrict__ dz, int B, int out, float* __restrict__ g, int64_t ld_g, int64_t b_off) {
+  const int o = blockIdx.x * blockDim.x + threadIdx.x;
+  if (o >= out) return;
+  const int z = blockIdx.y;
+  const TA* p = dz + (int64_t)z * B * out + o;
+  float s = 0.f;
+  for (int b = 0; b < B; ++b) s += to_float(p[(int64_t)b * out]);
+  g[(int64_t)z * ld_g + b_off + o] = s;
+}
+
+// ------------------------------------------------------------------------------------------------ least squares
+// One CTA per replica: r_b = a_b . w - y_b (one warp per sample), loss = sum r_b^2 / (2B),
+// g[i] = (1/B) sum_b r_b a_b[i] (one thread per feature, samples in ascending order).
+// xb [K, B, in] gathered minibatch, yb [K, B] targets, w = params (row stride ld_p).  Dynamic smem: B floats.
+__global__ void __launch_bounds__(256)
+lsq_grad_kernel(const float* __restrict__ xb, const float* __restrict__ yb, const float* __restrict__ params,
+                int64_t ld_p, int B, int in, float* __restrict__ g, int64_t ld_g, float* __restrict__ loss) {
+  extern __shared__ float res[];
+  const int k = blockIdx.x;
+  const float* w = params + (int64_t)k * ld_p;
+  const float* a = xb + (int64_t)k * B * in;
+  const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+  for (int b = wid; b < B; b += nw) {
+    float p = 0.f;
+    for (int i = lane; i < in; i += 32) p = fmaf(a[(int64_t)b * in + i], w[i], p);
+    p = warp_sum(p);
+    if (lane == 0) res[b] = p - yb[(int64_t)k * B + b];
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && loss != nullptr) {
+    double s = 0.0;
+    for (int b = 0; b < B; ++b) s += (double)res[b] * (double)res[b];
+    loss[k] = (float)(s / (2.0 * B));
+  }
+  const float invB = 1.f / (float)B;
+  for (int i = threadIdx.x; i < in; i += blockDim.x) {
+    float s = 0.f;
+    for (int b = 0; b < B; ++b) s = fmaf(res[b], a[(int64_t)b * in + i], s);
+    g[(int64_t)k * ld_g + i] = s * invB;
+  }
+}
+
+}  // namespace lsam

@@ -1,0 +1,259 @@
+// stream_kernels.cuh -- schedule, per-replica norm, perturbation, fused worker update, centre update.
+// All of these are HBM-streaming kernels over the stacked [K, ld] state (ld = padded row length).
+#pragma once
+
+#include "common.cuh"
+
+namespace lsam {
+
+// ------------------------------------------------------------------------------------------------ S0 schedule
+// hist.v[s] = centre version that was current when step t - s started (s = 0..15), clamped at step 0.
+struct VerHist { int v[16]; };
+
+// grid K, any block size.  idx [K, B]; stale, ver, slot [K].  slot = ring slot holding the version read.
+__global__ void schedule_kernel(uint64_t seed, uint64_t t, int64_t n_samples, int B, int stale_max, VerHist hist,
+                                int ring, int32_t* __restrict__ idx, int32_t* __restrict__ stale,
+                                int32_t* __restrict__ ver, int32_t* __restrict__ slot) {
+  const uint64_t k = blockIdx.x;
+  if (idx != nullptr)
+    for (int j = threadIdx.x; j < B; j += blockDim.x)
+      idx[k * B + j] = (int32_t)(schedule_hash(seed, kTagIdx, t, k, (uint64_t)j) % (uint64_t)n_samples);
+  if (threadIdx.x == 0) {
+    const int s = (int)(schedule_hash(seed, kTagStale, t, k, 0) % (uint64_t)(stale_max + 1));
+    const int u = hist.v[s];
+    if (stale) stale[k] = s;
+    if (ver) ver[k] = u;
+    if (slot) slot[k] = u >= 0 ? u % ring : 0;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ S3 norm
+// Pass 1: partial[k][chunk] = sum of squares of one fixed chunk of g_k, in a fixed order:
+// per thread ITER vectors in ascending address order, xor-shuffle tree, warps in ascending order.
+constexpr int kNormThreads = 256;
+constexpr int kNormIter = 8;
+template <int VEC>
+__host__ __device__ constexpr int64_t norm_chunk() { return (int64_t)kNormThreads * VEC * kNormIter; }
+
+template <int VEC>
+__global__ void __launch_bounds__(kNormThreads)
+sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float* __restrict__ partial, int64_t nchunks) {
+  __shared__ float red[kNormThreads / 32];
+  const int k = blockIdx.y;
+  const int64_t base = (int64_t)blockIdx.x * norm_chunk<VEC>();
+  const float* row = g + (int64_t)k * ldg;
+  float s = 0.f;
+  if (VEC == 4) {
+    float4 r[kNormIter];
+#pragma unroll
+    for (int i = 0; i < kNormIter; ++i) {
+      const int64_t j = base + ((int64_t)i * kNormThreads + threadIdx.x) * 4;
+      r[i] = (j < n) ? __ldcs(reinterpret_cast<const float4*>(row + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int i = 0; i < kNormIter; ++i) s += (r[i].x * r[i].x + r[i].y * r[i].y) + (r[i].z * r[i].z + r[i].w * r[i].w);
+  } else {
+#pragma unroll
+    for (int i = 0; i < kNormIter; ++i) {
+      const int64_t j = base + (int64_t)i * kNormThreads + threadIdx.x;
+      const float a = (j < n) ? row[j] : 0.f;
+      s += a * a;
+    }
+  }
+  const float tot = block_sum<float>(s, red);
+  if (threadIdx.x == 0) partial[(int64_t)k * nchunks + blockIdx.x] = tot;
+}
+
+// Pass 2: norm[k] = sqrt(sum of partials) accumulated in double in a fixed order; scale[k] = rho / (norm + gamma).
+// grid K, block 256; partial has row stride nchunks, of which the first nused are summed.  A non-finite norm raises STATUS_NONFINITE and leaves scale = 0 (no perturbation).
+__global__ void __launch_bounds__(256)
+norm_finalize_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t nused, float rho, float gamma,
+                     float* __restrict__ norm_out, float* __restrict__ scale_out, int* __restrict__ status) {
+  __shared__ double red[8];
+  const int k = blockIdx.x;
+  double s = 0.0;
+  for (int64_t c = threadIdx.x; c < nused; c += blockDim.x) s += (double)partial[(int64_t)k * nchunks + c];
+  const double tot = block_sum<double>(s, red);
+  if (threadIdx.x == 0) {
+    const float nrm = (float)sqrt(tot);
+    norm_out[k] = nrm;
+    if (scale_out) {
+      if (isfinite(nrm)) {
+        scale_out[k] = rho / (nrm + gamma);
+      } else {
+        scale_out[k] = 0.f;
+        atomicOr(status, STATUS_NONFINITE);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ S4 perturb
+// xt[k][j] = x[k][j] + scale[k] * g[k][j]  (Eq. 3 with scale = rho / (||g|| + gamma)); the master x is not modified.
+// TP = float (fp32 operand) or bf16 (tensor-core operand copy).  grid (chunks, K).
+constexpr int kPertThreads = 256;
+constexpr int kPertIter = 4;
+
+template <int VEC, typename TP>
+__global__ void __launch_bounds__(kPertThreads)
+perturb_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ g, int64_t ldg, int64_t n,
+               const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt) {
+  const int k = blockIdx.y;
+  const float sc = scale[k];
+  const int64_t base = (int64_t)blockIdx.x * ((int64_t)kPertThreads * VEC * kPertIter);
+  const float* xr = x + (int64_t)k * ldx;
+  const float* gr = g + (int64_t)k * ldg;
+  TP* tr = xt + (int64_t)k * ldt;
+  if (VEC == 4) {
+    float4 xv[kPertIter], gv[kPertIter];
+#pragma unroll
+    for (int i = 0; i < kPertIter; ++i) {
+      const int64_t j = base + ((int64_t)i * kPertThreads + threadIdx.x) * 4;
+      if (j < n) {
+        xv[i] = *reinterpret_cast<const float4*>(xr + j);
+        gv[i] = __ldcs(reinterpret_cast<const float4*>(gr + j));
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < kPertIter; ++i) {
+      const int64_t j = base + ((int64_t)i * kPertThreads + threadIdx.x) * 4;
+      if (j < n) {
+        const float a = fmaf(sc, gv[i].x, xv[i].x), b = fmaf(sc, gv[i].y, xv[i].y);
+        const float c = fmaf(sc, gv[i].z, xv[i].z), d = fmaf(sc, gv[i].w, xv[i].w);
+        if (sizeof(TP) == 4) {
+          *reinterpret_cast<float4*>(reinterpret_cast<float*>(tr) + j) = make_float4(a, b, c, d);
+        } else {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+          uint2 pk;
+          pk.x = *reinterpret_cast<uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(tr) + j) = pk;
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < kPertIter; ++i) {
+      const int64_t j = base + (int64_t)i * kPertThreads + threadIdx.x;
+      if (j < n) tr[j] = from_float<TP>(fmaf(sc, gr[j], xr[j]));
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ S6 fused update
+// One thread owns VEC consecutive columns for ALL replicas (k ascending), so that the centre versions are
+// re-read from cache and the iterate accumulator is read and written once per column:
+//   G = g2 + lambda (x - y_slot[k]);  v <- mu v + G;  x <- x - eta (G + mu v)  [Nesterov]  or  x - eta v;
+//   acc += sum_k x_new;  optional operand copy xop = TP(x_new).
+struct UpdateArgs {
+  float* x;            // [K, ld]
+  float* v;            // [K, ld]
+  const float* g;      // [K, ldg]
+  const float* yring;  // [ring, ld]
+  const int32_t* slot; // [K] ring slot of the centre version read by replica k
+  float* acc;          // [ld]
+  void* xop;           // [K, ld] operand copy (or nullptr)
+  int64_t ld, ldg, n;
+  int K;
+  float eta, mu, lambda;
+};
+
+constexpr int kUpdThreads = 256;
+
+template <int VEC, bool NESTEROV, typename TP, bool WRITE_OP>
+__global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a) {
+  const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * VEC;
+  if (j >= a.n) return;
+  if (VEC == 4) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 2
+    for (int k = 0; k < a.K; ++k) {
+      const int64_t o = (int64_t)k * a.ld + j;
+      const float4 gv = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)k * a.ldg + j));
+      float4 xv = *reinterpret_cast<const float4*>(a.x + o);
+      float4 vv = *reinterpret_cast<const float4*>(a.v + o);
+      const float4 yv = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[k] * a.ld + j));
+      float G;
+#define LSAM_UPD(c)                                                         \
+  G = fmaf(a.lambda, xv.c - yv.c, gv.c);                                    \
+  vv.c = fmaf(a.mu, vv.c, G);                                               \
+  xv.c = NESTEROV ? xv.c - a.eta * fmaf(a.mu, vv.c, G) : xv.c - a.eta * vv.c; \
+  s.c += xv.c;
+      LSAM_UPD(x) LSAM_UPD(y) LSAM_UPD(z) LSAM_UPD(w)
+#undef LSAM_UPD
+      *reinterpret_cast<float4*>(a.x + o) = xv;
+      __stcs(reinterpret_cast<float4*>(a.v + o), vv);
+      if (WRITE_OP) {
+        if (sizeof(TP) == 2) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(xv.x, xv.y), hi = __floats2bfloat162_rn(xv.z, xv.w);
+          uint2 pk;
+          pk.x = *reinterpret_cast<uint32_t*>(&lo);
+          pk.y = *reinterpret_cast<uint32_t*>(&hi);
+          *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(a.xop) + o) = pk;
+        }
+      }
+    }
+    float4 av = *reinterpret_cast<const float4*>(a.acc + j);
+    av.x += s.x; av.y += s.y; av.z += s.z; av.w += s.w;
+    *reinterpret_cast<float4*>(a.acc + j) = av;
+  } else {
+    float s = 0.f;
+    for (int k = 0; k < a.K; ++k) {
+      const int64_t o = (int64_t)k * a.ld + j;
+      const float gv = a.g[(int64_t)k * a.ldg + j];
+      float xv = a.x[o], vv = a.v[o];
+      const float yv = a.yring[(int64_t)a.slot[k] * a.ld + j];
+      const float G = fmaf(a.lambda, xv - yv, gv);
+      vv = fmaf(a.mu, vv, G);
+      xv = NESTEROV ? xv - a.eta * fmaf(a.mu, vv, G) : xv - a.eta * vv;
+      s += xv;
+      a.x[o] = xv;
+      a.v[o] = vv;
+      if (WRITE_OP) reinterpret_cast<TP*>(a.xop)[o] = from_float<TP>(xv);
+    }
+    a.acc[j] += s;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ S7 centre update
+//   g' = acc / (K tau) - y;  g = have_prev ? g' + beta (g' - g'_prev) : g';  y_new = y + eta' g;
+//   g'_prev <- g';  acc <- 0.       (sync branch of Algorithm 2 with the look-ahead of Section 4.2)
+__global__ void __launch_bounds__(256)
+couple_kernel(float* __restrict__ acc, const float* __restrict__ y_cur, float* __restrict__ y_new,
+              float* __restrict__ gprev, int64_t n, float inv_ktau, float beta, float eta_prime, int have_prev) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  const float y = y_cur[j];
+  const float gp = fmaf(acc[j], inv_ktau, -y);
+  const float g = have_prev ? fmaf(beta, gp - gprev[j], gp) : gp;
+  y_new[j] = fmaf(eta_prime, g, y);
+  gprev[j] = gp;
+  acc[j] = 0.f;
+}
+
+// ------------------------------------------------------------------------------------------------ small utilities
+// dst[k][j] = TP(src[k][j]) over [K, n] with row strides.
+template <typename TP>
+__global__ void __launch_bounds__(256)
+cast_rows_kernel(const float* __restrict__ src, int64_t lds, TP* __restrict__ dst, int64_t ldd, int64_t n) {
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= n) return;
+  const int k = blockIdx.y;
+  dst[(int64_t)k * ldd + j] = from_float<TP>(src[(int64_t)k * lds + j]);
+}
+
+// Copy between an unpadded vector and its padded layout.  seg[i] = {unpadded offset, padded offset, length}.
+struct SegMap { int n; int64_t src[18], dst[18], len[18]; };
+
+template <bool TO_PADDED, typename TS, typename TD>
+__global__ void __launch_bounds__(256)
+seg_copy_kernel(const TS* __restrict__ src, int64_t lds, TD* __restrict__ dst, int64_t ldd, SegMap m) {
+  const int k = blockIdx.z, sgi = blockIdx.y;
+  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (sgi >= m.n || j >= m.len[sgi]) return;
+  const int64_t so = TO_PADDED ? m.src[sgi] : m.dst[sgi];
+  const int64_t dof = TO_PADDED ? m.dst[sgi] : m.src[sgi];
+  dst[(int64_t)k * ldd + dof + j] = from_float<TD>(to_float(src[(int64_t)k * lds + so + j]));
+}
+
+}  // namespace lsam

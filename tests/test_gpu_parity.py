@@ -1,0 +1,291 @@
+"""Parity of the CUDA library (through its C ABI) against the CPU oracle on identical seeded inputs.
+
+Tolerances (relative L2, worst replica): fp32 per step 1e-5, fp32 20-step trajectory 1e-3,
+bf16-GEMM per step 2e-3 (operand roundings are mirrored by the oracle; what is left are rare one-ulp
+rounding flips of stored bf16 values), bf16-GEMM 20-step trajectory 2e-2.  Integers are bit-exact.
+"""
+import numpy as np
+import pytest
+
+import oracle as O
+from harness import Pair, max_rel_rows, rel_l2
+from paper_2509_03110_b200 import binding as G
+from paper_2509_03110_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_STEP_FP32 = 1e-5
+TOL_TRAJ_FP32 = 1e-3
+TOL_STEP_BF16 = 2e-3
+TOL_TRAJ_BF16 = 2e-2
+
+
+def _assert_all(errs, tol, what=""):
+    for k, v in errs.items():
+        assert v <= tol, f"{what} {k}: {v:.3e} > {tol:.1e}"
+
+
+# ------------------------------------------------------------------------------------------------ schedule (integers)
+def test_schedule_bit_exact_with_staleness():
+    X, y, _ = synth.least_squares_data(500, 16, seed=0)
+    rng = np.random.default_rng(1)
+    x0 = rng.standard_normal((5, 16)).astype(np.float32)
+    p = Pair(G.MODEL_LSQ, widths=(16,), K=5, batch=37, X=X, Y=y, x0=x0, y0=x0.mean(0), tau=2, stale_max=3, seed=1234, lam=0.1)
+    for t in range(12):
+        p.step(0.01, 0.05)
+        oi, os_, ov = p.oracle.read_schedule(t)
+        gi, gs, gv = p.gpu.read_schedule(t)
+        np.testing.assert_array_equal(gi, oi)
+        np.testing.assert_array_equal(gs, os_)
+        np.testing.assert_array_equal(gv, ov)
+        p.couple_if_due()
+    # a step in the future: indices and staleness are pure functions of (seed, t, k, j)
+    oi, os_, _ = p.oracle.read_schedule(10**6)
+    gi, gs, _ = p.gpu.read_schedule(10**6, want_ver=False)
+    np.testing.assert_array_equal(gi, oi)
+    np.testing.assert_array_equal(gs, os_)
+    ot, oty, otx = p.oracle.counters()
+    gt, gty, gtx = p.gpu.counters()
+    assert (ot, oty) == (gt, gty) and (otx == gtx).all()
+    # host statement of the hash agrees with the oracle's
+    for (t, k, j) in [(0, 0, 0), (7, 3, 11), (10**6, 4, 36)]:
+        assert G.lsam_schedule_hash(1234, 0, t, k, j) == O.hash5(1234, O.lib().oracle_tag_idx(), t, k, j)
+        assert G.lsam_schedule_hash(1234, 1, t, k, 0) == O.hash5(1234, O.lib().oracle_tag_stale(), t, k, 0)
+    assert p.gpu.status() == 0
+    p.close()
+
+
+# ------------------------------------------------------------------------------------------------ optimiser-only (FLAT)
+@pytest.mark.parametrize("K,d", [(1, 1), (8, 3), (1, 1000), (8, 1000), (3, 8191), (8, 1_000_000), (2, 1_048_577)])
+@pytest.mark.parametrize("nesterov", [1, 0])
+def test_flat_streaming_kernels(K, d, nesterov):
+    if nesterov == 0 and d > 10000:
+        pytest.skip("heavy-ball form is covered at the small sizes")
+    x0, y0, g1, g2 = synth.flat_problem(K, d, seed=d % 97)
+    p = Pair(G.MODEL_FLAT, K=K, flat_d=d, x0=x0, y0=y0, tau=3, stale_max=2, seed=5, lam=0.3, beta=0.9, eta_prime=1.0, nesterov=nesterov)
+    p.set_external_grads(g1, g2)
+    for t in range(20):
+        p.step(0.05, 0.1)
+        if t == 0:
+            e = p.grad_errors()
+            _assert_all(e, TOL_STEP_FP32, f"FLAT K={K} d={d} step0")
+            _, n1, _ = p.oracle.read_step_info()
+            _, gn1, _ = p.gpu.read_step_info()
+            np.testing.assert_allclose(gn1, n1, rtol=TOL_STEP_FP32)
+            _assert_all(p.errors(), TOL_STEP_FP32, f"FLAT K={K} d={d} step0")
+        p.couple_if_due()
+    _assert_all(p.errors(), TOL_TRAJ_FP32, f"FLAT K={K} d={d} 20 steps")
+    assert p.gpu.counters()[1] == 6
+    assert p.gpu.status() == 0
+    p.close()
+
+
+def test_flat_invariants_at_sweep_size():
+    # properties that hold at any size, checked on the device output of a full-size sweep point (d = 25.6M, K = 8):
+    # ||x~ - x|| = rho n / (n + gamma),  g1 . (x~ - x) = rho n^2 / (n + gamma)  (proof of Proposition 7)
+    import torch
+
+    K, d = 8, 25_600_000
+    gen = torch.Generator(device="cuda").manual_seed(0)
+    x0 = torch.randn(K, d, device="cuda", generator=gen)
+    g1 = torch.randn(K, d, device="cuda", generator=gen) * 0.1
+    g2 = torch.randn(K, d, device="cuda", generator=gen) * 0.1
+    y0 = x0.mean(0)
+    cfg = G.make_config(G.MODEL_FLAT, K=K, flat_d=d, tau=4, lam=0.5, mu=0.9)
+    gpu = G.Lsam(cfg, None, None, x0, y0)
+    gpu.set_external_grads(g1, g2)
+    rho, eta = 0.1, 0.05
+    gpu.step(eta, rho)
+    _, n1, _ = gpu.read_step_info()
+    xt = torch.empty(d, device="cuda")
+    for k in (0, 7):
+        n = torch.linalg.vector_norm(g1[k].double()).item()
+        assert abs(n1[k] - n) <= 1e-6 * n
+        # sampled elements of the update against the definition, one by one
+        sel = torch.randint(0, d, (1000,), device="cuda", generator=gen)
+        xk = gpu.read_params(k, out=xt)
+        G_ = g2[k, sel].double() + float(np.float32(0.5)) * (x0[k, sel].double() - y0[sel].double())
+        want = x0[k, sel].double() - float(np.float32(eta)) * (G_ + float(np.float32(0.9)) * G_)
+        assert torch.allclose(xk[sel].double(), want, rtol=1e-5, atol=1e-6)
+    xp = torch.from_numpy(gpu.read_grads(3)[0]).cuda().double()
+    delta = xp - x0[0].double()
+    n = torch.linalg.vector_norm(g1[0].double()).item()
+    assert abs(torch.linalg.vector_norm(delta).item() - rho * n / (n + 1e-12)) <= 1e-5 * rho
+    assert abs((g1[0].double() @ delta).item() - rho * n) <= 1e-5 * rho * n
+    assert gpu.status() == 0
+    gpu.close()
+
+
+# ------------------------------------------------------------------------------------------------ least squares (config 1)
+def test_config1_least_squares_100_steps():
+    X, y, _ = synth.least_squares_data(4096, 256, noise=0.01, seed=0)
+    rng = np.random.default_rng(0)
+    w0 = rng.standard_normal(256).astype(np.float32)
+    x0 = synth.replicate(w0, 4)
+    eta, tau = 0.01, 4
+    lam = 0.5 / (eta * tau)
+    p = Pair(G.MODEL_LSQ, widths=(256,), K=4, batch=32, X=X, Y=y, x0=x0, y0=w0, tau=tau, seed=0, lam=lam, mu=0.9,
+             flags=G.FLAG_KEEP_G1 | G.FLAG_STEP_INFO)
+    for t in range(100):
+        p.step(eta, 0.05)
+        if t == 0:
+            _assert_all(p.grad_errors(), TOL_STEP_FP32, "C1 step0")
+            ol, on1, on2 = p.oracle.read_step_info()
+            gl, gn1, gn2 = p.gpu.read_step_info()
+            np.testing.assert_allclose(gl, ol, rtol=TOL_STEP_FP32)
+            np.testing.assert_allclose(gn1, on1, rtol=TOL_STEP_FP32)
+            np.testing.assert_allclose(gn2, on2, rtol=TOL_STEP_FP32)
+        p.couple_if_due()
+        if t == 19:
+            _assert_all(p.errors(), TOL_TRAJ_FP32, "C1 20 steps")
+    _assert_all(p.errors(), 5e-3, "C1 100 steps")
+    assert p.gpu.counters()[1] == 25 and p.gpu.status() == 0
+    p.close()
+
+
+# ------------------------------------------------------------------------------------------------ classifiers
+def _mlp_pair(model, widths, K, B, n, dtype, impl=G.IMPL_AUTO, seed=0, jitter=0.0, **hp):
+    X, labels = synth.gaussian_mixture(n, widths[0], widths[-1], seed=seed)
+    w0 = synth.mlp_init(widths, seed=seed)
+    x0 = synth.replicate(w0, K, jitter=jitter, seed=seed)
+    return Pair(model, widths=widths, K=K, batch=B, X=X, Y=labels, x0=x0, y0=w0, gemm_dtype=dtype, gemm_impl=impl,
+                flags=G.FLAG_KEEP_G1 | G.FLAG_STEP_INFO, **hp)
+
+
+def _per_step_then_trajectory(p, eta, rho, tol_step, tol_traj, steps=20, forced=3, what=""):
+    # teacher-forced steps: both sides start each step from the oracle's state
+    for t in range(forced):
+        p.teacher_force()
+        p.step(eta, rho)
+        _assert_all(p.grad_errors(), tol_step, f"{what} forced step {t}")
+        e = p.errors()
+        e.pop("acc")
+        _assert_all(e, tol_step, f"{what} forced step {t}")
+        ol, on1, on2 = p.oracle.read_step_info()
+        gl, gn1, gn2 = p.gpu.read_step_info()
+        np.testing.assert_allclose(gl, ol, rtol=max(tol_step, 1e-5))
+        np.testing.assert_allclose(gn1, on1, rtol=tol_step)
+        np.testing.assert_allclose(gn2, on2, rtol=tol_step)
+        p.couple_if_due()
+    p.teacher_force()
+    for t in range(forced, forced + steps):
+        p.step(eta, rho)
+        p.couple_if_due()
+    e = p.errors()
+    e.pop("acc")
+    # the trajectory tolerance is stated for the parameters (workers and centre).  The momentum buffer is
+    # dominated by lambda (x - y), a difference of nearly equal fp32 numbers, so its noise floor relative
+    # to ||v|| is an order of magnitude higher than that of x itself.
+    ev = e.pop("v")
+    assert ev <= 10 * tol_traj, f"{what} free-running {steps} steps v: {ev:.3e}"
+    _assert_all(e, tol_traj, f"{what} free-running {steps} steps")
+    assert p.gpu.status() == 0
+
+
+@pytest.mark.parametrize("model,widths,K,B", [
+    (G.MODEL_MLP, (20, 33, 7), 3, 10),            # ragged everything
+    (G.MODEL_MLP, (64, 128, 96, 10), 4, 64),      # several tiles
+    (G.MODEL_RESMLP, (48, 80, 80, 80, 12), 2, 32),
+    (G.MODEL_MLP, (30, 5), 2, 9),                 # linear softmax model
+])
+def test_classifier_fp32_small(model, widths, K, B):
+    p = _mlp_pair(model, widths, K, B, n=300, dtype=G.GEMM_FP32, tau=4, lam=0.4, seed=3, jitter=0.01)
+    _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, what=f"fp32 {widths}")
+    p.close()
+
+
+@pytest.mark.parametrize("model,widths,K,B", [
+    (G.MODEL_MLP, (20, 33, 7), 3, 10),
+    (G.MODEL_MLP, (64, 128, 96, 10), 4, 64),
+    (G.MODEL_RESMLP, (48, 80, 80, 80, 12), 2, 32),
+])
+def test_classifier_bf16_simt_small(model, widths, K, B):
+    p = _mlp_pair(model, widths, K, B, n=300, dtype=G.GEMM_BF16, impl=G.IMPL_SIMT, tau=4, lam=0.4, seed=4, jitter=0.01)
+    assert not p.gpu.uses_tcgen05()
+    _per_step_then_trajectory(p, 0.05, 0.1, TOL_STEP_BF16, TOL_TRAJ_BF16, what=f"bf16 simt {widths}")
+    p.close()
+
+
+def test_config2_mlp_784_1024_10_full_shape():
+    widths = (784, 1024, 10)
+    p = _mlp_pair(G.MODEL_MLP, widths, K=8, B=128, n=60000, dtype=G.GEMM_FP32, tau=4, lam=0.5 / (0.05 * 4), seed=0)
+    _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, steps=20, forced=2, what="C2")
+    p.close()
+
+
+def test_step_batch_matches_gathered_step():
+    # the caller-supplied minibatch path (host buffers) must reproduce the resident-dataset path exactly
+    import torch
+
+    widths = (32, 40, 6)
+    X, labels = synth.gaussian_mixture(200, 32, 6, seed=1)
+    w0 = synth.mlp_init(widths, seed=1)
+    x0 = synth.replicate(w0, 3)
+    kw = dict(widths=widths, K=3, batch=16, n_samples=200, tau=2, lam=0.3, seed=9)
+    dX, dY = torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda()
+    a = G.Lsam(G.make_config(G.MODEL_MLP, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+    b = G.Lsam(G.make_config(G.MODEL_MLP, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+    loss = np.zeros(3, np.float32)
+    for t in range(5):
+        a.step(0.05, 0.05)
+        idx, _, _ = b.read_schedule(t, want_ver=False)
+        xb = torch.from_numpy(X[idx.ravel()].reshape(3, 16, 32)).pin_memory()
+        yb = torch.from_numpy(labels[idx.ravel()].reshape(3, 16)).pin_memory()
+        b.step_batch(0.05, 0.05, xb, yb, loss)
+        np.testing.assert_array_equal(loss, a.read_step_info()[0])
+        if a.should_couple():
+            assert a.couple() == 0 and b.couple() == 0
+    np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
+    np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
+    a.close()
+    b.close()
+
+
+def test_deterministic_repeat():
+    # same seed, same inputs: two runs agree bit for bit (fixed reduction orders, no float atomics)
+    outs = []
+    for _ in range(2):
+        p = _mlp_pair(G.MODEL_MLP, (64, 128, 96, 10), 4, 64, n=300, dtype=G.GEMM_FP32, tau=2, lam=0.4, seed=3, stale_max=2)
+        for t in range(6):
+            p.gpu.step(0.05, 0.05)
+            if p.gpu.should_couple():
+                p.gpu.couple()
+        outs.append((p.gpu.read_all_params(), p.gpu.read_params(-1)))
+        p.close()
+    np.testing.assert_array_equal(outs[0][0], outs[1][0])
+    np.testing.assert_array_equal(outs[0][1], outs[1][1])
+
+
+# ------------------------------------------------------------------------------------------------ errors (host-side only)
+def test_error_paths():
+    import torch
+
+    assert G.lsam_param_count(G.make_config(G.MODEL_FLAT, K=1, flat_d=0)) == -1
+    assert G.lsam_workspace_bytes(G.make_config(G.MODEL_MLP, widths=(4, 0, 2), K=1, batch=1)) == 0
+    assert G.lsam_workspace_bytes(G.make_config(G.MODEL_FLAT, K=1, flat_d=8, gamma=0.0)) == 0
+    cfg = G.make_config(G.MODEL_FLAT, K=2, flat_d=8, tau=2)
+    x0 = torch.zeros(2, 8, device="cuda")
+    y0 = torch.zeros(8, device="cuda")
+    # workspace too small
+    h = G.C.c_void_p()
+    ws = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    rc = G.lib().lsam_init(G.C.byref(h), G.C.byref(cfg), None, None, G.C.c_void_p(x0.data_ptr()), G.C.c_void_p(y0.data_ptr()),
+                           G.C.c_void_p((ws.data_ptr() + 255) // 256 * 256), 512, None)
+    assert rc == G.LSAM_ERR_WORKSPACE and not h.value
+    # null pointers
+    rc = G.lib().lsam_init(G.C.byref(h), G.C.byref(cfg), None, None, None, None, None, 0, None)
+    assert rc == G.LSAM_ERR_INVALID
+    gpu = G.Lsam(cfg, None, None, x0, y0)
+    with pytest.raises(G.LsamError) as ei:
+        gpu.step(0.1, 0.1)  # no external gradients yet
+    assert ei.value.code == G.LSAM_ERR_STATE
+    assert gpu.couple() == G.LSAM_ERR_STATE  # trigger false
+    g = torch.ones(2, 8, device="cuda")
+    gbad = g.clone()
+    gbad[1, 3] = float("nan")  # injected on the host side: the norm kernel reports it, nothing traps
+    gpu.set_external_grads(gbad, g)
+    gpu.step(0.1, 0.1)
+    assert gpu.status() == G.LSAM_ERR_NONFINITE
+    x = gpu.read_all_params()
+    assert np.isfinite(x).all()  # scale = 0 for the bad replica, the update itself used the finite g2
+    gpu.close()
