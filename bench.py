@@ -23,21 +23,23 @@ sys.path.insert(0, ROOT)
 
 LSQ, MLP, RESMLP, FLAT = 0, 1, 2, 3
 
-# The five workloads (shapes, replica counts, batch sizes and radii as configured; eta, tau, lambda0 filled with the
-# paper's Appendix-D ranges where a workload leaves them open).
+# The five workloads (shapes, replica counts, batch sizes and radii as configured).  Where a workload leaves them open:
+# tau = 16 as in the paper's experiments, lambda = lambda0 / (eta tau) with lambda0 = 0.9 from the grid of Appendix D,
+# beta = 0.9, eta' = 1.  (With the look-ahead beta = 0.9 and worker momentum 0.9 the worker/centre recursion alone is
+# linearly unstable for short sync periods and weak pulls; tau = 16 with lambda0 = 0.9 is in its stable region.)
 WORKLOADS = {
-    "c1": dict(model=LSQ, widths=(256,), K=4, B=32, n=4096, classes=0, bf16=False, rho=0.05, eta=0.01, tau=4, stale_max=0,
+    "c1": dict(model=LSQ, widths=(256,), K=4, B=32, n=4096, classes=0, bf16=False, rho=0.05, eta=0.01, tau=4, stale_max=0, lambda0=0.5,
                name="least squares 4096x256, K=4, B=32"),
-    "c2": dict(model=MLP, widths=(784, 1024, 10), K=8, B=128, n=60000, classes=10, bf16=False, rho=0.05, eta=0.05, tau=4,
+    "c2": dict(model=MLP, widths=(784, 1024, 10), K=8, B=128, n=60000, classes=10, bf16=False, rho=0.05, eta=0.05, tau=16,
                stale_max=0, name="MLP 784-1024-10 fp32, K=8, B=128"),
     "c3": dict(model=MLP, widths=(3072, 2048, 2048, 2048, 100), K=16, B=128, n=50000, classes=100, bf16=True, rho=0.1,
-               eta=0.05, tau=4, stale_max=0, name="MLP 3072-2048x3-100 bf16 GEMM, K=16, B=128"),
+               eta=0.01, tau=16, stale_max=0, name="MLP 3072-2048x3-100 bf16 GEMM, K=16, B=128"),
     "c4": dict(model=RESMLP, widths=(3072, 4096, 4096, 4096, 4096, 1000), K=32, B=256, n=200000, classes=1000, bf16=True,
-               rho=0.1, eta=0.05, tau=4, stale_max=3, name="residual MLP 3072-4096x4-1000 bf16 GEMM, K=32, B=256, staleness [0,3]"),
-    "c5": dict(model=FLAT, widths=(), K=8, B=0, n=0, classes=0, bf16=False, rho=0.1, eta=0.05, tau=4, stale_max=0, d=256_000_000,
+               rho=0.1, eta=0.002, tau=16, stale_max=3, head_scale=0.1, res_scale=0.25, name="residual MLP 3072-4096x4-1000 bf16 GEMM, K=32, B=256, staleness [0,3]"),
+    "c5": dict(model=FLAT, widths=(), K=8, B=0, n=0, classes=0, bf16=False, rho=0.1, eta=0.05, tau=16, stale_max=0, d=256_000_000,
                name="optimiser-only sweep point d=256M, K=8"),
 }
-LAMBDA0, MU, BETA, ETA_PRIME, GAMMA = 0.5, 0.9, 0.9, 1.0, 1e-12
+LAMBDA0, MU, BETA, ETA_PRIME, GAMMA = 0.9, 0.9, 0.9, 1.0, 1e-12
 NOMINAL_HBM_GBS, FALLBACK_HBM_GBS, FALLBACK_BF16_TF = 8000.0, 6650.0, 1590.0
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x max SM clock
 
@@ -154,7 +156,12 @@ def make_inputs(w, dev, seed=0):
         parts = []
         ws = w["widths"]
         for l in range(len(ws) - 1):
-            parts.append((torch.randn(ws[l + 1], ws[l], device=dev, generator=g) * (2.0 / ws[l]) ** 0.5).reshape(-1))
+            scale = (2.0 / ws[l]) ** 0.5
+            if l == len(ws) - 2:
+                scale *= w.get("head_scale", 1.0)       # small head: the initial loss starts near log(classes)
+            elif w["model"] == RESMLP and ws[l] == ws[l + 1]:
+                scale *= w.get("res_scale", 1.0)        # damped residual branches: no normalisation layers here
+            parts.append((torch.randn(ws[l + 1], ws[l], device=dev, generator=g) * scale).reshape(-1))
             parts.append(torch.zeros(ws[l + 1], device=dev))
         w0 = torch.cat(parts)
     x0 = w0.unsqueeze(0).expand(K, -1).contiguous()
@@ -162,7 +169,7 @@ def make_inputs(w, dev, seed=0):
 
 
 def make_cfg(G, w, flags=0):
-    lam = LAMBDA0 / (w["eta"] * w["tau"])
+    lam = w.get("lambda0", LAMBDA0) / (w["eta"] * w["tau"])
     return G.make_config(w["model"], widths=w["widths"], K=w["K"], batch=max(w["B"], 1) if w["model"] != FLAT else 0,
                          gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
                          beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
@@ -176,7 +183,7 @@ def oracle_baseline(w, X, Y, x0_row, budget_s=20.0):
 
     cores = O.num_threads()
     d = param_count(w)
-    lam = LAMBDA0 / (w["eta"] * w["tau"])
+    lam = w.get("lambda0", LAMBDA0) / (w["eta"] * w["tau"])
     if w["model"] == FLAT:
         Ks, ds = w["K"], min(d, 4_000_000)
         cfg = O.make_config(O.MODEL_FLAT, K=Ks, flat_d=ds, mu=MU, gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME)
