@@ -170,6 +170,29 @@ void lsam_destroy(lsam_ctx* ctx);
  * with mix the SplitMix64 finaliser; tag 0 = minibatch index stream, 1 = staleness stream. */
 uint64_t lsam_schedule_hash(uint64_t seed, int tag, uint64_t t, uint64_t k, uint64_t j);
 
+/* Row norms without any allocation.  (The paper has no counterpart: this is a convenience of the library.)
+ * For callers that must not allocate device memory -- code running inside a memory pool that has already handed
+ * out the whole GPU, plug-ins that are only given their input and output buffers, latency-critical loops where a
+ * cudaMalloc would synchronise the device -- this computes norm[k] = sqrt(sum_{j<n} g[k*ld + j]^2) for k < K with
+ * the same two-pass, fixed-order reduction that lsam_step() uses for ||g1_k||, but keeps the per-chunk partial sums
+ * in an array that is part of the library image instead of a caller workspace.
+ *  d_g    device, [K, ld] fp32 rows of which the first n elements are reduced (ld >= n).
+ *  d_norm device, [K] fp32 output.
+ *  cuda_stream  a cudaStream_t (NULL = default stream); the call is asynchronous on it.
+ *  h_err  nullable host buffer of h_err_len bytes that receives a message when the call fails.
+ * Limit: K * ceil(n / C) <= LSAM_STATIC_NORM_MAX_PARTIALS, with C = 8192 elements when d_g is 16-byte aligned and
+ * ld is a multiple of 4, else C = 2048.  Larger problems are refused with LSAM_ERR_WORKSPACE and nothing is launched.
+ * The array (LSAM_STATIC_NORM_MAX_PARTIALS floats = 1 MiB) is held by every GPU that loads the library until the
+ * process exits.  All calls on one GPU share it and it keeps the previous call's contents; every slot a call reads
+ * it has written itself first, so nothing needs clearing, but two calls that overlap on the GPU (different streams,
+ * or different host threads) race on it: serialise them.  The first call on each device looks up the array's device
+ * address (with that device current); make that first call outside any stream capture.
+ * No cudaMalloc, cudaFree or other allocating routine is called.  Errors: LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE,
+ * LSAM_ERR_CUDA. */
+#define LSAM_STATIC_NORM_MAX_PARTIALS 262144
+int lsam_row_norms_static(const float* d_g, int64_t ld, int64_t n, int32_t K, float* d_norm, void* cuda_stream,
+                          char* h_err, size_t h_err_len);
+
 #ifdef __cplusplus
 }
 #endif

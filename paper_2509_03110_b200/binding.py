@@ -24,7 +24,7 @@ EXPORTS = [
     "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads",
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
-    "lsam_destroy", "lsam_schedule_hash",
+    "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static",
 ]
 
 
@@ -90,6 +90,7 @@ def lib():
     L.lsam_destroy.argtypes = [vp]
     L.lsam_schedule_hash.restype = C.c_uint64
     L.lsam_schedule_hash.argtypes = [C.c_uint64, C.c_int, C.c_uint64, C.c_uint64, C.c_uint64]
+    L.lsam_row_norms_static.argtypes = [vp, C.c_int64, C.c_int64, C.c_int32, vp, vp, C.c_char_p, C.c_size_t]
     _lib = L
     return L
 
@@ -118,6 +119,23 @@ def lsam_workspace_bytes(cfg):
 
 def lsam_schedule_hash(seed, tag, t, k, j):
     return int(lib().lsam_schedule_hash(seed, tag, t, k, j))
+
+
+STATIC_NORM_MAX_PARTIALS = 262144
+
+
+def lsam_row_norms_static(g, n, out, stream=None):
+    """Row norms of the CUDA tensor g [K, ld] (first n columns) into the CUDA tensor out [K], with no allocation.
+
+    For callers that may not allocate device memory (see include/lsam.h): the partial sums live in an array inside
+    the library.  Returns (status, message).  Calls that overlap on one GPU race on that array; the first call on a
+    device should be made outside stream capture.
+    """
+    K, ld = g.shape
+    err = C.create_string_buffer(256)
+    s = C.c_void_p(stream.cuda_stream) if stream is not None else None
+    rc = lib().lsam_row_norms_static(C.c_void_p(g.data_ptr()), ld, int(n), K, C.c_void_p(out.data_ptr()), s, err, 256)
+    return int(rc), err.value.decode()
 
 
 def _np_ptr(a):

@@ -6,6 +6,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -704,3 +705,70 @@ void lsam_destroy(lsam_ctx* c) {
 }
 
 }  // extern "C"
+
+// =================================================================================================== no-allocation entry point
+// Scratch for lsam_row_norms_static(): per-chunk partial sums of squares.  It lives in the library image, so every
+// GPU that loads the library carries this 1 MiB until the process exits, and all calls on a GPU share it.
+// In host code this name is only a handle for cudaGetSymbolAddress(); it is NOT a device pointer.
+static __device__ __align__(256) float lsam_static_norm_partials[LSAM_STATIC_NORM_MAX_PARTIALS];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+float* g_static_partials_addr[kMaxDevices] = {};  // device address of the array, looked up once per device
+
+int static_fail(int code, const char* msg, char* h_err, size_t h_err_len) {
+  if (h_err && h_err_len > 0) std::snprintf(h_err, h_err_len, "%s", msg);
+  return code;
+}
+}  // namespace
+
+extern "C" int lsam_row_norms_static(const float* d_g, int64_t ld, int64_t n, int32_t K, float* d_norm, void* cuda_stream,
+                                     char* h_err, size_t h_err_len) {
+  if (h_err && h_err_len > 0) h_err[0] = 0;
+  if (!d_g || !d_norm || K < 1 || n < 1 || ld < n)
+    return static_fail(LSAM_ERR_INVALID, "lsam_row_norms_static: need d_g, d_norm, K >= 1, n >= 1, ld >= n", h_err, h_err_len);
+  const bool vec4 = (reinterpret_cast<uintptr_t>(d_g) & 15) == 0 && (ld % 4) == 0;
+  const int64_t chunk = vec4 ? norm_chunk<4>() : norm_chunk<1>();
+  const int64_t nch = ceil_div(n, chunk);
+  if (nch > LSAM_STATIC_NORM_MAX_PARTIALS || (int64_t)K * nch > LSAM_STATIC_NORM_MAX_PARTIALS || K > 65535) {
+    char msg[256];
+    std::snprintf(msg, sizeof msg,
+                  "lsam_row_norms_static: K * ceil(n / %lld) = %lld partial sums exceed the built-in scratch of %d (use lsam_step with a workspace)",
+                  (long long)chunk, (long long)K * (long long)nch, LSAM_STATIC_NORM_MAX_PARTIALS);
+    return static_fail(LSAM_ERR_WORKSPACE, msg, h_err, h_err_len);
+  }
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices)
+    return static_fail(LSAM_ERR_CUDA, "lsam_row_norms_static: cudaGetDevice failed", h_err, h_err_len);
+  float* partial = nullptr;
+  {
+    // set-up, once per device and with that device current: resolve the array's device address
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_partials_addr[dev]) {
+      void* p = nullptr;
+      const cudaError_t e = cudaGetSymbolAddress(&p, lsam_static_norm_partials);
+      if (e != cudaSuccess || !p) {
+        char msg[256];
+        std::snprintf(msg, sizeof msg, "lsam_row_norms_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        return static_fail(LSAM_ERR_CUDA, msg, h_err, h_err_len);
+      }
+      g_static_partials_addr[dev] = static_cast<float*>(p);
+    }
+    partial = g_static_partials_addr[dev];
+  }
+  cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  // Every slot the second pass reads (k * nch + c, c < nch) is written by the first pass of this same call,
+  // so the previous call's contents never need clearing.
+  dim3 grid((unsigned)nch, (unsigned)K);
+  if (vec4) sumsq_partial_kernel<4><<<grid, kNormThreads, 0, stream>>>(d_g, ld, n, partial, nch);
+  else sumsq_partial_kernel<1><<<grid, kNormThreads, 0, stream>>>(d_g, ld, n, partial, nch);
+  norm_finalize_kernel<<<K, 256, 0, stream>>>(partial, nch, nch, 0.f, 1.f, d_norm, nullptr, nullptr);
+  const cudaError_t e = cudaPeekAtLastError();
+  if (e != cudaSuccess) {
+    char msg[256];
+    std::snprintf(msg, sizeof msg, "lsam_row_norms_static: launch failed: %s", cudaGetErrorString(e));
+    return static_fail(LSAM_ERR_CUDA, msg, h_err, h_err_len);
+  }
+  return LSAM_OK;
+}
