@@ -1,5 +1,20 @@
-// gemm_tcgen05.cuh -- tensor-core (tcgen05 / TMEM / TMA) batched GEMMs of the bf16 classifier path.
+// gemm_tcgen05.cuh -- batched-over-replicas bf16 GEMMs of the classifier path on the 5th-generation tensor cores:
+// TMA (cp.async.bulk.tensor) stages 128B-swizzled operand tiles in shared memory, one elected thread issues
+// tcgen05.mma with fp32 accumulators in tensor memory, four warps drain the accumulators with tcgen05.ld and apply
+// the fused epilogue.  One persistent CTA per SM walks the (replica, m-tile, n-tile) list; the accumulator is
+// double-buffered in tensor memory so that the epilogue of a tile overlaps the main loop of the next one.
+//
+// Every GEMM is D(z, m, n) = sum_kd A(z, m, kd) * B(z, n, kd) with the 128-row M side on the weights:
+//   forward   m = output unit, n = sample, kd = input unit   A = W   (kd contiguous)   B = activations (kd contiguous)
+//   dgrad     m = input unit,  n = sample, kd = output unit  A = W   (m contiguous)    B = dz          (kd contiguous)
+//   wgrad     m = output unit, n = input unit, kd = sample   A = dz  (m contiguous)    B = activations (n contiguous)
+// so every weight is read from HBM exactly once per GEMM and the whole minibatch sits in one N tile.
+//
+// All waits on mbarriers are bounded: when one expires the CTA raises STATUS_TIMEOUT, stops issuing work, lets the
+// copies in flight land, frees its tensor memory and returns.
 #pragma once
+
+#include <cuda.h>
 
 #include <string>
 #include <vector>
@@ -9,16 +24,469 @@
 
 namespace lsam {
 
+// ------------------------------------------------------------------------------------------------ PTX wrappers
+namespace tc {
+
+__device__ inline uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ inline void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ inline void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit expires or another role has already given up.
+constexpr uint32_t kSpinLimit = 1u << 22;
+__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023u) == 1023u && *abort_flag) return false;
+  }
+  return false;
+}
+
+__device__ inline void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ inline void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 3-D tiled TMA load into this CTA's shared memory (no multicast), completion counted on an mbarrier.
+__device__ inline void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(smem_u32(bar))
+      : "memory");
+}
+
+__device__ inline void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ inline void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate.
+__device__ inline void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// mbarrier arrives when all tcgen05.mma issued so far by this thread have completed.
+__device__ inline void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns of tensor memory -> 32 registers per thread (thread = lane).
+__device__ inline void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ inline void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Fields (bits): start address >> 4 [0,14), leading-dimension
+// byte offset >> 4 [16,30), stride-dimension byte offset >> 4 [32,46), descriptor version 1 [46,48), swizzle mode
+// 2 = 128 B [61,64).
+__device__ inline uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// Instruction descriptor of kind::f16: D fp32 (bit 4), A and B bf16 (bits 7, 10), operand majors (bits 15, 16:
+// 0 = contraction dimension contiguous, 1 = M / N contiguous), N >> 3 at [17,23), M >> 4 at [24,29).
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+
+}  // namespace tc
+
+// ------------------------------------------------------------------------------------------------ epilogue parameters
+enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3 };
+
+struct TcEpi {
+  // forward: bias (operand copy), out / skip / mask [Z, B, ldo]; head: logits fp32 [Z, B, ldo]
+  const bf16* bias;  int64_t ld_p;
+  bf16* out;  const bf16* skip;  uint8_t* mask;  float* logits;
+  // dgrad: dh_next (skip gradient, nullable), dh_out (nullable), dz_prev, mask_prev  [Z, B, ldo]
+  const bf16* dh_next;  bf16* dh_out;  bf16* dz_prev;  const uint8_t* mask_prev;
+  // wgrad: g[z * ld_g + w_off + m * ldw + n]
+  float* g;  int64_t ld_g, w_off;  int ldw;
+  int B, ldo;
+};
+
+constexpr int kTcBlockM = 128;
+constexpr int kTcBlockK = 64;
+constexpr int kTcThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + tensor-memory owner, warps 2-5: epilogue
+
+template <int BLOCK_N>
+__host__ __device__ constexpr int tc_stages() { return BLOCK_N == 256 ? 4 : (BLOCK_N == 128 ? 6 : 8); }
+template <int BLOCK_N>
+__host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + BLOCK_N) * kTcBlockK * 2; }
+template <int BLOCK_N>
+__host__ __device__ constexpr int tc_smem_bytes() { return tc_stages<BLOCK_N>() * tc_stage_bytes<BLOCK_N>() + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+
+// ------------------------------------------------------------------------------------------------ the kernel
+// M, N, Kd: problem extents; Z replicas.  Operands are addressed through 3-D tensor maps (dim 2 = replica):
+//   contraction-contiguous operand: map dims {Kd, rows, Z}, box {64, tile rows, 1}
+//   M/N-contiguous operand:         map dims {rows, Kd, Z}, box {64, 64, 1} (one box per 64 rows of the tile)
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
+__global__ void __launch_bounds__(kTcThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int M, int N, int Kd,
+                    int Z, TcEpi ep, int* __restrict__ status) {
+  constexpr int STAGES = tc_stages<BLOCK_N>();
+  constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
+  constexpr int B_BYTES = BLOCK_N * kTcBlockK * 2;
+  constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;  // two accumulator stages (power of two >= 32)
+  constexpr uint32_t IDESC = tc::instr_desc(kTcBlockM, BLOCK_N, A_MN, B_MN);
+
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * (A_BYTES + B_BYTES));
+  uint64_t* full = bars;                     // [STAGES]  TMA -> MMA
+  uint64_t* empty = bars + STAGES;           // [STAGES]  MMA -> TMA
+  uint64_t* acc_full = bars + 2 * STAGES;    // [2]       MMA -> epilogue
+  uint64_t* acc_empty = acc_full + 2;        // [2]       epilogue -> MMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m_tiles = (M + kTcBlockM - 1) / kTcBlockM;
+  const int n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
+  const int k_blocks = (Kd + kTcBlockK - 1) / kTcBlockK;
+  const int64_t total = (int64_t)Z * m_tiles * n_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
+    for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], 4); }
+    *abort_flag = 0;
+    tc::fence_barrier_init();
+  }
+  if (warp == 1) tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  tc::tc_fence_before();
+  __syncthreads();
+  tc::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
+        const int m0 = mt * kTcBlockM, n0 = nt * BLOCK_N;
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+          uint8_t* a_dst = tiles + s * (A_BYTES + B_BYTES);
+          uint8_t* b_dst = a_dst + A_BYTES;
+          tc::mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
+          const int k0 = kb * kTcBlockK;
+          if (A_MN) {
+#pragma unroll
+            for (int i = 0; i < kTcBlockM / 64; ++i) tc::tma_load_3d(a_dst + i * 8192, &map_a, m0 + 64 * i, k0, z, &full[s]);
+          } else {
+            tc::tma_load_3d(a_dst, &map_a, k0, m0, z, &full[s]);
+          }
+          if (B_MN) {
+#pragma unroll
+            for (int i = 0; i < BLOCK_N / 64; ++i) tc::tma_load_3d(b_dst + i * 8192, &map_b, n0 + 64 * i, k0, z, &full[s]);
+          } else {
+            tc::tma_load_3d(b_dst, &map_b, k0, n0, z, &full[s]);
+          }
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+      }
+      if (!ok) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      int s = 0;
+      uint32_t ph = 0;
+      int as = 0;
+      uint32_t aph = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        if (!tc::mbar_wait(&acc_empty[as], aph ^ 1u, abort_flag)) { ok = false; break; }
+        tc::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + (uint32_t)(as * BLOCK_N);
+        for (int kb = 0; kb < k_blocks; ++kb) {
+          if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          tc::tc_fence_after();
+          const uint32_t a_addr = tc::smem_u32(tiles + s * (A_BYTES + B_BYTES));
+          const uint32_t b_addr = a_addr + A_BYTES;
+#pragma unroll
+          for (int k = 0; k < kTcBlockK / 16; ++k) {
+            // contraction-contiguous tile: rows of 128 B, 8-row groups 1024 B apart, a K = 16 slice is 32 B further along the row;
+            // M/N-contiguous tile: 64-element blocks 8192 B apart (leading offset), 8 contraction rows = 1024 B (stride offset),
+            // a K = 16 slice is two such groups = 2048 B further.
+            const uint64_t ad = A_MN ? tc::smem_desc(a_addr + k * 2048, 8192, 1024) : tc::smem_desc(a_addr + k * 32, 16, 1024);
+            const uint64_t bd = B_MN ? tc::smem_desc(b_addr + k * 2048, 8192, 1024) : tc::smem_desc(b_addr + k * 32, 16, 1024);
+            tc::umma_bf16(d_tmem, ad, bd, IDESC, (kb | k) != 0 ? 1u : 0u);
+          }
+          tc::umma_commit(&empty[s]);  // frees the stage when these MMAs have read it
+          if (++s == STAGES) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) break;
+        tc::umma_commit(&acc_full[as]);
+        if (++as == 2) { as = 0; aph ^= 1u; }
+      }
+      if (!ok) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
+    const int quad = warp & 3;
+    int as = 0;
+    uint32_t aph = 0;
+    bool ok = true;
+    for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
+      const int m = mt * kTcBlockM + quad * 32 + lane;
+      const int n0 = nt * BLOCK_N;
+      if (!tc::mbar_wait(&acc_full[as], aph, abort_flag)) { ok = false; break; }
+      tc::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BLOCK_N);
+      float bias = 0.f;
+      if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) bias = to_float(ep.bias[(int64_t)z * ep.ld_p + m]);
+#pragma unroll 1
+      for (int c = 0; c < BLOCK_N / 32; ++c) {
+        uint32_t r[32];
+        tc::tmem_ld32(taddr + (uint32_t)(c * 32), r);
+        tc::tmem_ld_wait();
+        const int nb = n0 + c * 32;
+        if (m < M && nb < N) {
+          if (EPI == TC_EPI_WGRAD) {
+            float* dst = ep.g + (int64_t)z * ep.ld_g + ep.w_off + (int64_t)m * ep.ldw + nb;
+            if (nb + 32 <= N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + j) =
+                    make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (nb + j < N) dst[j] = __uint_as_float(r[j]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int b = nb + j;  // sample
+              if (b < N) {
+                const int64_t e = ((int64_t)z * ep.B + b) * ep.ldo + m;
+                const float acc = __uint_as_float(r[j]);
+                if (EPI == TC_EPI_FWD_HIDDEN) {
+                  const float v = acc + bias;
+                  const float rl = v > 0.f ? v : 0.f;
+                  ep.mask[e] = v > 0.f;
+                  const float sk = ep.skip ? to_float(ep.skip[e]) : 0.f;
+                  ep.out[e] = __float2bfloat16_rn(sk + rl);
+                } else if (EPI == TC_EPI_FWD_HEAD) {
+                  ep.logits[e] = acc + bias;
+                } else {  // TC_EPI_DGRAD
+                  const float sum = ep.dh_next ? acc + to_float(ep.dh_next[e]) : acc;
+                  const bf16 q = __float2bfloat16_rn(sum);
+                  if (ep.dh_out) ep.dh_out[e] = q;
+                  ep.dz_prev[e] = ep.mask_prev[e] ? q : __float2bfloat16_rn(0.f);
+                }
+              }
+            }
+          }
+        }
+      }
+      tc::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) tc::mbar_arrive(&acc_empty[as]);
+      if (++as == 2) { as = 0; aph ^= 1u; }
+    }
+    if (!ok && lane == 0) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc::tc_fence_before();
+  __syncthreads();
+  if (*abort_flag) {
+    // something gave up: give copies that may still be in flight time to land before shared memory is released
+    const long long t0 = clock64();
+    while (clock64() - t0 < 2000000LL) { }
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc::tc_fence_after();
+    tc::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
 struct TcLayer { int in, out; int64_t w_pad, b_pad; bool residual; };
 struct TcBuffers {
   bf16* xop; float* g; int64_t ld;
   bf16* act[9]; uint8_t* mask[9]; float* logits; bf16* dz[2]; bf16* dh[2]; int* status;
+  int lda[10];
 };
-struct TcPlan { int dummy = 0; };
 
-inline bool tc_supported(const lsam_config&) { return false; }
-inline int tc_plan(TcPlan&, const lsam_config&, const std::vector<TcLayer>&, const TcBuffers&, int64_t*, std::string&) { return 1; }
-inline int tc_forward(TcPlan&, int, cudaStream_t) { return 1; }
-inline int tc_backward(TcPlan&, int, int, cudaStream_t) { return 1; }
+struct TcGemm {
+  CUtensorMap map_a, map_b;
+  int M = 0, N = 0, Kd = 0, block_n = 0;
+  TcEpi ep{};
+  bool valid = false;
+};
+
+struct TcPlan {
+  int Z = 0, B = 0, n_layers = 0, sms = 148;
+  int* status = nullptr;
+  int64_t* launches = nullptr;
+  std::vector<TcGemm> fwd, dgrad, wgrad;
+};
+
+typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                    const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline PFN_encodeTiled tc_encode_fn() {
+  static PFN_encodeTiled fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<PFN_encodeTiled>(p);
+  }
+  return fn;
+}
+
+// bf16 tensor [Z][rows][cols] with element strides (row_stride, z_stride); dim 0 = cols (contiguous).
+inline bool tc_make_map(CUtensorMap* m, const bf16* base, uint64_t cols, uint64_t rows, uint64_t Z, uint64_t row_stride,
+                        uint64_t z_stride, uint32_t box_cols, uint32_t box_rows) {
+  PFN_encodeTiled enc = tc_encode_fn();
+  if (!enc) return false;
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride * 2) % 16 || (z_stride * 2) % 16) return false;
+  cuuint64_t dims[3] = {cols, rows, Z};
+  cuuint64_t strides[2] = {row_stride * 2, z_stride * 2};
+  cuuint32_t box[3] = {box_cols, box_rows, 1};
+  cuuint32_t estr[3] = {1, 1, 1};
+  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int tc_pick_block_n(int n) { return n > 128 ? 256 : (n > 64 ? 128 : 64); }
+
+// The tensor-core path needs every layer's input width to be a multiple of 8 (16-byte row strides of W and of
+// the activations); output widths are free (padded strides, TMA zero-fills the ragged edge).
+inline bool tc_supported(const lsam_config& c) {
+  if (c.n_layers < 1 || c.batch < 1) return false;
+  for (int l = 0; l < c.n_layers; ++l)
+    if (c.widths[l] % 8 != 0) return false;
+  return true;
+}
+
+inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& layers, const TcBuffers& b, int64_t* launches,
+                   std::string& why) {
+  P.Z = c.K; P.B = c.batch; P.n_layers = (int)layers.size(); P.status = b.status; P.launches = launches;
+  int dev = 0;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&P.sms, cudaDevAttrMultiProcessorCount, dev);
+  const int L = P.n_layers, B = c.batch, Z = c.K;
+  P.fwd.assign(L, TcGemm()); P.dgrad.assign(L, TcGemm()); P.wgrad.assign(L, TcGemm());
+  for (int l = 0; l < L; ++l) {
+    const TcLayer& ly = layers[l];
+    const int cur = (L - 1 - l) & 1;  // dz buffer holding the pre-activation gradient of layer l
+    const int lda_in = b.lda[l], lda_out = b.lda[l + 1];
+    const bf16* W = b.xop + ly.w_pad;
+    const bool head = (l == L - 1);
+    bool ok = true;
+    {  // forward: A = W [out][in] (in contiguous), B = act_l [B][in]
+      TcGemm& g = P.fwd[l];
+      g.M = ly.out; g.N = B; g.Kd = ly.in; g.block_n = tc_pick_block_n(B);
+      ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, kTcBlockM);
+      ok &= tc_make_map(&g.map_b, b.act[l], ly.in, B, Z, lda_in, (uint64_t)B * lda_in, 64, g.block_n);
+      g.ep.bias = b.xop + ly.b_pad; g.ep.ld_p = b.ld; g.ep.B = B; g.ep.ldo = lda_out;
+      if (head) g.ep.logits = b.logits;
+      else { g.ep.out = b.act[l + 1]; g.ep.skip = ly.residual ? b.act[l] : nullptr; g.ep.mask = b.mask[l]; }
+      g.valid = ok;
+    }
+    {  // wgrad: A = dz_l [B][out] (out contiguous), B = act_l [B][in] (in contiguous)
+      TcGemm& g = P.wgrad[l];
+      g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in);
+      ok &= tc_make_map(&g.map_a, b.dz[cur], ly.out, B, Z, lda_out, (uint64_t)B * lda_out, 64, 64);
+      ok &= tc_make_map(&g.map_b, b.act[l], ly.in, B, Z, lda_in, (uint64_t)B * lda_in, 64, 64);
+      g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.B = B;
+      g.valid = ok;
+    }
+    if (l > 0) {  // dgrad: A = W [out][in] read as (m = in contiguous, kd = out), B = dz_l [B][out]
+      TcGemm& g = P.dgrad[l];
+      g.M = ly.in; g.N = B; g.Kd = ly.out; g.block_n = tc_pick_block_n(B);
+      ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, 64);
+      ok &= tc_make_map(&g.map_b, b.dz[cur], ly.out, B, Z, lda_out, (uint64_t)B * lda_out, 64, g.block_n);
+      g.ep.dh_next = ly.residual ? b.dh[(l + 1) & 1] : nullptr;
+      g.ep.dh_out = layers[l - 1].residual ? b.dh[l & 1] : nullptr;
+      g.ep.dz_prev = b.dz[cur ^ 1]; g.ep.mask_prev = b.mask[l - 1]; g.ep.B = B; g.ep.ldo = lda_in;
+      g.valid = ok;
+    }
+    if (!ok) { why = "tensor map creation failed"; return 1; }
+  }
+  return 0;
+}
+
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
+inline int tc_launch_one(const TcPlan& P, const TcGemm& g, cudaStream_t stream) {
+  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes<BLOCK_N>()) != cudaSuccess) return 1;
+    attr_set = true;
+  }
+  const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, kTcBlockM) * ceil_div(g.N, BLOCK_N);
+  const int grid = (int)(tiles < P.sms ? tiles : P.sms);
+  kern<<<grid, kTcThreads, tc_smem_bytes<BLOCK_N>(), stream>>>(g.map_a, g.map_b, g.M, g.N, g.Kd, P.Z, g.ep, P.status);
+  return cudaPeekAtLastError() == cudaSuccess ? 0 : 1;
+}
+
+template <bool A_MN, bool B_MN, int EPI>
+inline int tc_launch(const TcPlan& P, const TcGemm& g, cudaStream_t stream) {
+  if (!g.valid) return 1;
+  switch (g.block_n) {
+    case 256: return tc_launch_one<256, A_MN, B_MN, EPI>(P, g, stream);
+    case 128: return tc_launch_one<128, A_MN, B_MN, EPI>(P, g, stream);
+    default: return tc_launch_one<64, A_MN, B_MN, EPI>(P, g, stream);
+  }
+}
+
+inline int tc_forward(const TcPlan& P, int l, cudaStream_t stream) {
+  return (l == P.n_layers - 1) ? tc_launch<false, false, TC_EPI_FWD_HEAD>(P, P.fwd[l], stream)
+                               : tc_launch<false, false, TC_EPI_FWD_HIDDEN>(P, P.fwd[l], stream);
+}
+inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, true, TC_EPI_WGRAD>(P, P.wgrad[l], stream); }
+inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, false, TC_EPI_DGRAD>(P, P.dgrad[l], stream); }
 
 }  // namespace lsam

@@ -7,11 +7,11 @@
 namespace lsam {
 
 // ------------------------------------------------------------------------------------------------ S1 gather
-// xb[k][b][:] = TA(X[idx[k][b]][:]);  yb[k][b] = Y[idx[k][b]] (4-byte elements).  grid (K*B), block 128.
+// xb[k][b][:] = TA(X[idx[k][b]][:]) with row stride ld;  yb[k][b] = Y[idx[k][b]] (4-byte elements).  grid (K*B), block 128.
 template <typename TA>
 __global__ void __launch_bounds__(128)
 gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx,
-              int64_t n_samples, int in, TA* __restrict__ xb, uint32_t* __restrict__ yb, int* __restrict__ status) {
+              int64_t n_samples, int in, int ld, TA* __restrict__ xb, uint32_t* __restrict__ yb, int* __restrict__ status) {
   const int64_t r = blockIdx.x;
   int64_t s = idx[r];
   if (s < 0 || s >= n_samples) {
@@ -19,34 +19,37 @@ gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const
     s = 0;
   }
   const float* src = X + s * in;
-  TA* dst = xb + r * in;
+  TA* dst = xb + r * ld;
   for (int i = threadIdx.x; i < in; i += blockDim.x) dst[i] = from_float<TA>(src[i]);
   if (threadIdx.x == 0 && yb != nullptr) yb[r] = Y[s];
 }
 
-// Caller-supplied minibatch: convert [rows, in] fp32 to the activation type.
+// Caller-supplied minibatch: convert [rows, in] fp32 (dense) to the activation type with row stride ld.
 template <typename TA>
 __global__ void __launch_bounds__(256)
-convert_batch_kernel(const float* __restrict__ src, TA* __restrict__ dst, int64_t n) {
+convert_batch_kernel(const float* __restrict__ src, TA* __restrict__ dst, int64_t rows, int in, int ld) {
   const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (j < n) dst[j] = from_float<TA>(src[j]);
+  if (j >= rows * in) return;
+  const int64_t r = j / in;
+  dst[r * ld + (j - r * in)] = from_float<TA>(src[j]);
 }
 
 // ------------------------------------------------------------------------------------------------ epilogues
 // Every GEMM hands its accumulator to one of these functors in LOGICAL coordinates:
 //   z = replica, b = sample in the minibatch, f = feature (output unit for forward, input unit for dgrad),
 //   or (z, o, i) = (replica, output unit, input unit) for the weight gradient.
+// Activation-like buffers are [K, B, ldw] with ldw >= width (row stride padded to a multiple of 8 elements).
 // TP = parameter operand type, TA = activation storage type.
 
 // hidden layer: v = acc + bias[f]; r = relu(v); mask = v > 0; out = TA(skip + r)
 template <typename TP, typename TA>
 struct EpiFwdHidden {
   const TP* bias;  int64_t ld_p;           // bias[z * ld_p + f]
-  TA* out;  const TA* skip;  uint8_t* mask;  // [K, B, width]
-  int B, width;
+  TA* out;  const TA* skip;  uint8_t* mask;  // [K, B, ldw]
+  int B, ldw;
   __device__ inline void operator()(int z, int b, int f, float acc) const {
     const float v = acc + to_float(bias[(int64_t)z * ld_p + f]);
-    const int64_t e = ((int64_t)z * B + b) * width + f;
+    const int64_t e = ((int64_t)z * B + b) * ldw + f;
     const float r = v > 0.f ? v : 0.f;
     mask[e] = v > 0.f;
     const float sk = skip ? to_float(skip[e]) : 0.f;
@@ -58,10 +61,10 @@ struct EpiFwdHidden {
 template <typename TP>
 struct EpiFwdHead {
   const TP* bias;  int64_t ld_p;
-  float* logits;  // [K, B, C]
-  int B, width;
+  float* logits;  // [K, B, ldw]
+  int B, ldw;
   __device__ inline void operator()(int z, int b, int f, float acc) const {
-    logits[((int64_t)z * B + b) * width + f] = acc + to_float(bias[(int64_t)z * ld_p + f]);
+    logits[((int64_t)z * B + b) * ldw + f] = acc + to_float(bias[(int64_t)z * ld_p + f]);
   }
 };
 
@@ -72,9 +75,9 @@ struct EpiDgrad {
   TA* dh_out;             // nullable
   TA* dz_prev;            // [K, B, width]
   const uint8_t* mask_prev;
-  int B, width;
+  int B, ldw;
   __device__ inline void operator()(int z, int b, int f, float acc) const {
-    const int64_t e = ((int64_t)z * B + b) * width + f;
+    const int64_t e = ((int64_t)z * B + b) * ldw + f;
     const float s = dh_next ? acc + to_float(dh_next[e]) : acc;
     const TA q = from_float<TA>(s);
     if (dh_out) dh_out[e] = q;
@@ -155,15 +158,15 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi) {
 }
 
 // ------------------------------------------------------------------------------------------------ softmax cross-entropy
-// One warp per sample row.  rowloss[r] = logsumexp(l) - l[y];  dz[r][c] = TA((softmax(l)[c] - [c == y]) / B).
+// One warp per sample row; logits and dz have row stride ldc.  rowloss[r] = logsumexp(l) - l[y];  dz[r][c] = TA((softmax(l)[c] - [c == y]) / B).
 template <typename TA>
 __global__ void __launch_bounds__(256)
-softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int64_t rows, int C, int B,
+softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int64_t rows, int C, int ldc, int B,
                   TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status) {
   const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   if (r >= rows) return;
   const int lane = threadIdx.x & 31;
-  const float* lg = logits + r * C;
+  const float* lg = logits + r * ldc;
   float m = -INFINITY;
   for (int c = lane; c < C; c += 32) m = fmaxf(m, lg[c]);
   m = warp_max(m);
@@ -177,7 +180,7 @@ softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ 
   }
   if (lane == 0) rowloss[r] = (m + logf(se)) - lg[y];
   const float inv = 1.f / se, invB = 1.f / (float)B;
-  TA* out = dz + r * C;
+  TA* out = dz + r * ldc;
   for (int c = lane; c < C; c += 32) {
     const float p = expf(lg[c] - m) * inv;
     out[c] = from_float<TA>((p - (c == y ? 1.f : 0.f)) * invB);
@@ -198,13 +201,13 @@ __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float
 // g[z][b_off + o] = sum_b dz[z][b][o], samples in ascending order.  grid (ceil(out / 256), K).
 template <typename TA>
 __global__ void __launch_bounds__(256)
-bias_grad_kernel(const TA* __restrict__ dz, int B, int out, float* __restrict__ g, int64_t ld_g, int64_t b_off) {
+bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldz, float* __restrict__ g, int64_t ld_g, int64_t b_off) {
   const int o = blockIdx.x * blockDim.x + threadIdx.x;
   if (o >= out) return;
   const int z = blockIdx.y;
-  const TA* p = dz + (int64_t)z * B * out + o;
+  const TA* p = dz + (int64_t)z * B * ldz + o;
   float s = 0.f;
-  for (int b = 0; b < B; ++b) s += to_float(p[(int64_t)b * out]);
+  for (int b = 0; b < B; ++b) s += to_float(p[(int64_t)b * ldz]);
   g[(int64_t)z * ld_g + b_off + o] = s;
 }
 

@@ -1,8 +1,13 @@
 """Parity of the CUDA library (through its C ABI) against the CPU oracle on identical seeded inputs.
 
 Tolerances (relative L2, worst replica): fp32 per step 1e-5, fp32 20-step trajectory 1e-3,
-bf16-GEMM per step 2e-3 (operand roundings are mirrored by the oracle; what is left are rare one-ulp
-rounding flips of stored bf16 values), bf16-GEMM 20-step trajectory 2e-2.  Integers are bit-exact.
+bf16-GEMM per step 8e-3, bf16-GEMM 20-step trajectory 2e-2.  Integers are bit-exact.
+The bf16 per-step bound: operand roundings are mirrored by the oracle, so what is left are decisions that fp32
+(tensor-core) and double accumulation take differently -- a ReLU sign or a bf16 rounding boundary crossed by a
+pre-activation that differs by delta ~ 2e-5 relative.  A flipped ReLU changes one (sample, unit) entry of the
+backward signal, i.e. about 1/sqrt(B * width) of the gradient norm; the expected number of flips is about
+0.4 * delta * B * width * L, so their combined effect is about sqrt(0.4 * delta * L) ~ 6e-3 for L = 4 hidden
+layers, whatever the size of the network.
 """
 import numpy as np
 import pytest
@@ -16,7 +21,7 @@ pytestmark = pytest.mark.gpu
 
 TOL_STEP_FP32 = 1e-5
 TOL_TRAJ_FP32 = 1e-3
-TOL_STEP_BF16 = 2e-3
+TOL_STEP_BF16 = 8e-3
 TOL_TRAJ_BF16 = 2e-2
 
 
@@ -203,6 +208,19 @@ def test_classifier_bf16_simt_small(model, widths, K, B):
     p = _mlp_pair(model, widths, K, B, n=300, dtype=G.GEMM_BF16, impl=G.IMPL_SIMT, tau=4, lam=0.4, seed=4, jitter=0.01)
     assert not p.gpu.uses_tcgen05()
     _per_step_then_trajectory(p, 0.05, 0.1, TOL_STEP_BF16, TOL_TRAJ_BF16, what=f"bf16 simt {widths}")
+    p.close()
+
+
+@pytest.mark.parametrize("model,widths,K,B", [
+    (G.MODEL_MLP, (64, 128, 96, 10), 4, 64),         # N tile 64, ragged head (10 outputs), 96-wide layer
+    (G.MODEL_MLP, (256, 256, 256, 128), 2, 128),     # N tile 128, several contraction blocks
+    (G.MODEL_RESMLP, (128, 192, 192, 192, 100), 3, 200),  # N tile 256 with a ragged minibatch, skip connections
+    (G.MODEL_MLP, (320, 520, 24), 2, 40),            # ragged M tiles (520 = 4 x 128 + 8), ragged contraction (320 = 5 x 64)
+])
+def test_classifier_bf16_tcgen05(model, widths, K, B):
+    p = _mlp_pair(model, widths, K, B, n=400, dtype=G.GEMM_BF16, impl=G.IMPL_TCGEN05, tau=4, lam=0.4, seed=4, jitter=0.01)
+    assert p.gpu.uses_tcgen05()
+    _per_step_then_trajectory(p, 0.05, 0.1, TOL_STEP_BF16, TOL_TRAJ_BF16, what=f"bf16 tcgen05 {widths}")
     p.close()
 
 
