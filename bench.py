@@ -254,11 +254,15 @@ def main():
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
     ap.add_argument("--flat-d", type=int, default=None, help="c5 only: vector length of the sweep point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
     if args.flat_d and w["model"] == FLAT:
         w["d"] = args.flat_d
         w["name"] = f"optimiser-only sweep point d={args.flat_d}, K=8"
+    if args.replicas:
+        w["K"] = args.replicas
+        w["name"] += f" [K overridden to {args.replicas}]"
     flat = w["model"] == FLAT
     metric = "fused_update_hbm_gbs" if flat else "lsam_worker_samples_per_s"
     unit = "GB/s" if flat else "worker-samples/s"

@@ -5,10 +5,13 @@
 // double-buffered in tensor memory so that the epilogue of a tile overlaps the main loop of the next one.
 //
 // Every GEMM is D(z, m, n) = sum_kd A(z, m, kd) * B(z, n, kd) with the 128-row M side on the weights:
-//   forward   m = output unit, n = sample, kd = input unit   A = W   (kd contiguous)   B = activations (kd contiguous)
-//   dgrad     m = input unit,  n = sample, kd = output unit  A = W   (m contiguous)    B = dz          (kd contiguous)
-//   wgrad     m = output unit, n = input unit, kd = sample   A = dz  (m contiguous)    B = activations (n contiguous)
-// so every weight is read from HBM exactly once per GEMM and the whole minibatch sits in one N tile.
+//   forward   m = output unit, n = sample, kd = input unit   A = W   (kd contiguous)   B = activations (n contiguous)
+//   dgrad     m = input unit,  n = sample, kd = output unit  A = W   (m contiguous)    B = dz          (n contiguous)
+//   wgrad     m = output unit, n = input unit, kd = sample   A = dz  (kd contiguous)   B = activations (kd contiguous)
+// so every weight is read from HBM exactly once per GEMM and the whole minibatch sits in one N tile.  Activations,
+// masks, logits and backward signals are feature-major [Z, width, ldb] (sample index contiguous): the accumulator
+// row a thread drains from tensor memory is then one feature x 32 consecutive samples, i.e. contiguous 16-byte
+// vectors in every buffer the epilogue touches.
 //
 // All waits on mbarriers are bounded: when one expires the CTA raises STATUS_TIMEOUT, stops issuing work, lets the
 // copies in flight land, frees its tensor memory and returns.
@@ -135,14 +138,14 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool a_mn, bool 
 enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3 };
 
 struct TcEpi {
-  // forward: bias (operand copy), out / skip / mask [Z, B, ldo]; head: logits fp32 [Z, B, ldo]
+  // forward: bias (operand copy), out / skip / mask [Z, M, ldb]; head: logits fp32 [Z, M, ldb]
   const bf16* bias;  int64_t ld_p;
   bf16* out;  const bf16* skip;  uint8_t* mask;  float* logits;
-  // dgrad: dh_next (skip gradient, nullable), dh_out (nullable), dz_prev, mask_prev  [Z, B, ldo]
+  // dgrad: dh_next (skip gradient, nullable), dh_out (nullable), dz_prev, mask_prev  [Z, M, ldb]
   const bf16* dh_next;  bf16* dh_out;  bf16* dz_prev;  const uint8_t* mask_prev;
   // wgrad: g[z * ld_g + w_off + m * ldw + n]
   float* g;  int64_t ld_g, w_off;  int ldw;
-  int B, ldo;
+  int ldb;  // sample stride of the feature-major buffers (multiple of 16)
 };
 
 constexpr int kTcBlockM = 128;
@@ -153,8 +156,11 @@ template <int BLOCK_N>
 __host__ __device__ constexpr int tc_stages() { return BLOCK_N == 256 ? 4 : (BLOCK_N == 128 ? 6 : 8); }
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + BLOCK_N) * kTcBlockK * 2; }
+constexpr int kTcStageOutBytes = 4 * 32 * 33 * 4;  // epilogue staging: one 32 x 33 fp32 block per epilogue warp
 template <int BLOCK_N>
-__host__ __device__ constexpr int tc_smem_bytes() { return tc_stages<BLOCK_N>() * tc_stage_bytes<BLOCK_N>() + 1024 /*alignment slack*/ + 256 /*barriers*/; }
+__host__ __device__ constexpr int tc_smem_bytes() {
+  return tc_stages<BLOCK_N>() * tc_stage_bytes<BLOCK_N>() + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTcStageOutBytes;
+}
 
 // ------------------------------------------------------------------------------------------------ the kernel
 // M, N, Kd: problem extents; Z replicas.  Operands are addressed through 3-D tensor maps (dim 2 = replica):
@@ -179,6 +185,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   uint64_t* acc_empty = acc_full + 2;        // [2]       epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  float* stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (M + kTcBlockM - 1) / kTcBlockM;
@@ -286,41 +293,116 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         tc::tmem_ld32(taddr + (uint32_t)(c * 32), r);
         tc::tmem_ld_wait();
         const int nb = n0 + c * 32;
-        if (m < M && nb < N) {
-          if (EPI == TC_EPI_WGRAD) {
-            float* dst = ep.g + (int64_t)z * ep.ld_g + ep.w_off + (int64_t)m * ep.ldw + nb;
-            if (nb + 32 <= N) {
+        if (EPI == TC_EPI_WGRAD) {
+          // Stage the warp's 32 x 32 block through shared memory (row stride 33: conflict-free both ways) so that
+          // every store instruction of the warp writes one full 128-byte line of a gradient row.
+          float* st = stage + (warp - 2) * (32 * 33);
 #pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + j) =
-                    make_float4(__uint_as_float(r[j]), __uint_as_float(r[j + 1]), __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+          for (int j = 0; j < 32; ++j) st[lane * 33 + j] = __uint_as_float(r[j]);
+          __syncwarp();
+          const int mrow0 = mt * kTcBlockM + quad * 32;
+          const int col = nb + lane;
+          if (col < N) {
+            float* dst = ep.g + (int64_t)z * ep.ld_g + ep.w_off + (int64_t)mrow0 * ep.ldw + col;
+            const int rows = M - mrow0 < 32 ? M - mrow0 : 32;
+#pragma unroll 8
+            for (int i = 0; i < rows; ++i) dst[(int64_t)i * ep.ldw] = st[i * 33 + lane];
+          }
+          __syncwarp();
+        } else if (m < M && nb < N) {
+          // element (unit m, sample nb + j) of the feature-major buffers: 32 consecutive samples per thread
+          const int64_t t0 = ((int64_t)z * M + m) * ep.ldb + nb;
+          const bool full = nb + 32 <= N;
+          const int nvalid = full ? 32 : N - nb;
+          if (EPI == TC_EPI_FWD_HIDDEN) {
+            uint4 skv[4], ov[4], mv[2];
+            bf16* skb = reinterpret_cast<bf16*>(skv);
+            bf16* ob = reinterpret_cast<bf16*>(ov);
+            uint8_t* mb = reinterpret_cast<uint8_t*>(mv);
+            if (ep.skip != nullptr) {
+              if (full) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) skv[q] = *reinterpret_cast<const uint4*>(ep.skip + t0 + q * 8);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) skb[j] = j < nvalid ? ep.skip[t0 + j] : __float2bfloat16_rn(0.f);
+              }
+            } else {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) skv[q] = make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const float v = __uint_as_float(r[j]) + bias;
+              mb[j] = v > 0.f ? 1 : 0;
+              ob[j] = __float2bfloat16_rn(to_float(skb[j]) + (v > 0.f ? v : 0.f));
+            }
+            if (full) {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(ep.out + t0 + q * 8) = ov[q];
+#pragma unroll
+              for (int q = 0; q < 2; ++q) *reinterpret_cast<uint4*>(ep.mask + t0 + q * 16) = mv[q];
             } else {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (nb + j < N) dst[j] = __uint_as_float(r[j]);
+                if (j < nvalid) { ep.out[t0 + j] = ob[j]; ep.mask[t0 + j] = mb[j]; }
             }
-          } else {
+          } else if (EPI == TC_EPI_FWD_HEAD) {
+            if (full) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(ep.logits + t0 + j) = make_float4(__uint_as_float(r[j]) + bias, __uint_as_float(r[j + 1]) + bias,
+                                                                             __uint_as_float(r[j + 2]) + bias, __uint_as_float(r[j + 3]) + bias);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < nvalid) ep.logits[t0 + j] = __uint_as_float(r[j]) + bias;
+            }
+          } else {  // TC_EPI_DGRAD
+            uint4 skv[4], qv[4], zv[4], mv[2];
+            bf16* skb = reinterpret_cast<bf16*>(skv);
+            bf16* qb = reinterpret_cast<bf16*>(qv);
+            bf16* zb = reinterpret_cast<bf16*>(zv);
+            uint8_t* mb = reinterpret_cast<uint8_t*>(mv);
+            if (full) {
+#pragma unroll
+              for (int q = 0; q < 2; ++q) mv[q] = *reinterpret_cast<const uint4*>(ep.mask_prev + t0 + q * 16);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) mb[j] = j < nvalid ? ep.mask_prev[t0 + j] : 0;
+            }
+            if (ep.dh_next != nullptr) {
+              if (full) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) skv[q] = *reinterpret_cast<const uint4*>(ep.dh_next + t0 + q * 8);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) skb[j] = j < nvalid ? ep.dh_next[t0 + j] : __float2bfloat16_rn(0.f);
+              }
+            } else {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) skv[q] = make_uint4(0u, 0u, 0u, 0u);
+            }
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
-              const int b = nb + j;  // sample
-              if (b < N) {
-                const int64_t e = ((int64_t)z * ep.B + b) * ep.ldo + m;
-                const float acc = __uint_as_float(r[j]);
-                if (EPI == TC_EPI_FWD_HIDDEN) {
-                  const float v = acc + bias;
-                  const float rl = v > 0.f ? v : 0.f;
-                  ep.mask[e] = v > 0.f;
-                  const float sk = ep.skip ? to_float(ep.skip[e]) : 0.f;
-                  ep.out[e] = __float2bfloat16_rn(sk + rl);
-                } else if (EPI == TC_EPI_FWD_HEAD) {
-                  ep.logits[e] = acc + bias;
-                } else {  // TC_EPI_DGRAD
-                  const float sum = ep.dh_next ? acc + to_float(ep.dh_next[e]) : acc;
-                  const bf16 q = __float2bfloat16_rn(sum);
-                  if (ep.dh_out) ep.dh_out[e] = q;
-                  ep.dz_prev[e] = ep.mask_prev[e] ? q : __float2bfloat16_rn(0.f);
-                }
+              const bf16 qq = __float2bfloat16_rn(__uint_as_float(r[j]) + to_float(skb[j]));
+              qb[j] = qq;
+              zb[j] = mb[j] ? qq : __float2bfloat16_rn(0.f);
+            }
+            if (full) {
+              if (ep.dh_out != nullptr) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(ep.dh_out + t0 + q * 8) = qv[q];
               }
+#pragma unroll
+              for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(ep.dz_prev + t0 + q * 8) = zv[q];
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (j < nvalid) {
+                  if (ep.dh_out != nullptr) ep.dh_out[t0 + j] = qb[j];
+                  ep.dz_prev[t0 + j] = zb[j];
+                }
             }
           }
         }
@@ -353,7 +435,7 @@ struct TcLayer { int in, out; int64_t w_pad, b_pad; bool residual; };
 struct TcBuffers {
   bf16* xop; float* g; int64_t ld;
   bf16* act[9]; uint8_t* mask[9]; float* logits; bf16* dz[2]; bf16* dh[2]; int* status;
-  int lda[10];
+  int ldb;
 };
 
 struct TcGemm {
@@ -418,39 +500,39 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   cudaDeviceGetAttribute(&P.sms, cudaDevAttrMultiProcessorCount, dev);
   const int L = P.n_layers, B = c.batch, Z = c.K;
   P.fwd.assign(L, TcGemm()); P.dgrad.assign(L, TcGemm()); P.wgrad.assign(L, TcGemm());
+  const uint64_t ldb = (uint64_t)b.ldb;
   for (int l = 0; l < L; ++l) {
     const TcLayer& ly = layers[l];
     const int cur = (L - 1 - l) & 1;  // dz buffer holding the pre-activation gradient of layer l
-    const int lda_in = b.lda[l], lda_out = b.lda[l + 1];
     const bf16* W = b.xop + ly.w_pad;
     const bool head = (l == L - 1);
     bool ok = true;
-    {  // forward: A = W [out][in] (in contiguous), B = act_l [B][in]
+    {  // forward: A = W [out][in] (in contiguous), B = act_l [in][B] (samples contiguous)
       TcGemm& g = P.fwd[l];
       g.M = ly.out; g.N = B; g.Kd = ly.in; g.block_n = tc_pick_block_n(B);
       ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, kTcBlockM);
-      ok &= tc_make_map(&g.map_b, b.act[l], ly.in, B, Z, lda_in, (uint64_t)B * lda_in, 64, g.block_n);
-      g.ep.bias = b.xop + ly.b_pad; g.ep.ld_p = b.ld; g.ep.B = B; g.ep.ldo = lda_out;
+      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, 64);
+      g.ep.bias = b.xop + ly.b_pad; g.ep.ld_p = b.ld; g.ep.ldb = b.ldb;
       if (head) g.ep.logits = b.logits;
       else { g.ep.out = b.act[l + 1]; g.ep.skip = ly.residual ? b.act[l] : nullptr; g.ep.mask = b.mask[l]; }
       g.valid = ok;
     }
-    {  // wgrad: A = dz_l [B][out] (out contiguous), B = act_l [B][in] (in contiguous)
+    {  // wgrad: A = dz_l [out][B] (samples contiguous = contraction), B = act_l [in][B]
       TcGemm& g = P.wgrad[l];
       g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in);
-      ok &= tc_make_map(&g.map_a, b.dz[cur], ly.out, B, Z, lda_out, (uint64_t)B * lda_out, 64, 64);
-      ok &= tc_make_map(&g.map_b, b.act[l], ly.in, B, Z, lda_in, (uint64_t)B * lda_in, 64, 64);
-      g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.B = B;
+      ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
+      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.block_n);
+      g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.valid = ok;
     }
-    if (l > 0) {  // dgrad: A = W [out][in] read as (m = in contiguous, kd = out), B = dz_l [B][out]
+    if (l > 0) {  // dgrad: A = W [out][in] read as (m = in contiguous, kd = out), B = dz_l [out][B] (samples contiguous)
       TcGemm& g = P.dgrad[l];
       g.M = ly.in; g.N = B; g.Kd = ly.out; g.block_n = tc_pick_block_n(B);
       ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, 64);
-      ok &= tc_make_map(&g.map_b, b.dz[cur], ly.out, B, Z, lda_out, (uint64_t)B * lda_out, 64, g.block_n);
+      ok &= tc_make_map(&g.map_b, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, 64);
       g.ep.dh_next = ly.residual ? b.dh[(l + 1) & 1] : nullptr;
       g.ep.dh_out = layers[l - 1].residual ? b.dh[l & 1] : nullptr;
-      g.ep.dz_prev = b.dz[cur ^ 1]; g.ep.mask_prev = b.mask[l - 1]; g.ep.B = B; g.ep.ldo = lda_in;
+      g.ep.dz_prev = b.dz[cur ^ 1]; g.ep.mask_prev = b.mask[l - 1]; g.ep.ldb = b.ldb;
       g.valid = ok;
     }
     if (!ok) { why = "tensor map creation failed"; return 1; }
@@ -483,10 +565,10 @@ inline int tc_launch(const TcPlan& P, const TcGemm& g, cudaStream_t stream) {
 }
 
 inline int tc_forward(const TcPlan& P, int l, cudaStream_t stream) {
-  return (l == P.n_layers - 1) ? tc_launch<false, false, TC_EPI_FWD_HEAD>(P, P.fwd[l], stream)
-                               : tc_launch<false, false, TC_EPI_FWD_HIDDEN>(P, P.fwd[l], stream);
+  return (l == P.n_layers - 1) ? tc_launch<false, true, TC_EPI_FWD_HEAD>(P, P.fwd[l], stream)
+                               : tc_launch<false, true, TC_EPI_FWD_HIDDEN>(P, P.fwd[l], stream);
 }
-inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, true, TC_EPI_WGRAD>(P, P.wgrad[l], stream); }
-inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, false, TC_EPI_DGRAD>(P, P.dgrad[l], stream); }
+inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<false, false, TC_EPI_WGRAD>(P, P.wgrad[l], stream); }
+inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, true, TC_EPI_DGRAD>(P, P.dgrad[l], stream); }
 
 }  // namespace lsam

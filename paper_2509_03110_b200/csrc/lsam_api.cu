@@ -30,7 +30,7 @@ struct Layout {
   bool ok = false;
   int64_t d = 0, ld = 0;
   std::vector<LayerInfo> layers;
-  std::vector<int> lda;  // row stride of the activation-like buffers of width widths[l] (multiple of 8 elements)
+  int ldb = 0;  // sample stride of the feature-major activation-like buffers [K, width, ldb] (multiple of 16)
   SegMap seg{};
   int ring = 2;
   int64_t nchunks = 0;
@@ -63,7 +63,6 @@ bool plan(const lsam_config& c, Layout& L) {
     L.d = c.widths[0];
     L.ld = round_up(L.d, kSegAlign);
     L.layers.push_back({c.widths[0], 1, 0, -1, 0, -1, false});
-    L.lda.push_back(c.widths[0]);
     L.seg.n = 1;
     L.seg.src[0] = 0; L.seg.dst[0] = 0; L.seg.len[0] = L.d;
   } else if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {
@@ -83,7 +82,7 @@ bool plan(const lsam_config& c, Layout& L) {
       L.seg.src[L.seg.n] = li.w_unp; L.seg.dst[L.seg.n] = li.w_pad; L.seg.len[L.seg.n] = (int64_t)li.in * li.out; ++L.seg.n;
       L.seg.src[L.seg.n] = li.b_unp; L.seg.dst[L.seg.n] = li.b_pad; L.seg.len[L.seg.n] = li.out; ++L.seg.n;
     }
-    for (int l = 0; l <= c.n_layers; ++l) L.lda.push_back((int)round_up(c.widths[l], 8));
+    L.ldb = (int)round_up(c.batch, 16);
     L.d = unp;
     L.ld = pad;
   } else {
@@ -117,24 +116,26 @@ bool plan(const lsam_config& c, Layout& L) {
   for (int i = 0; i < 9; ++i) L.act[i] = L.mask[i] = 0;
   L.logits = L.rowloss = L.dz[0] = L.dz[1] = L.dh[0] = L.dh[1] = L.xstage = L.ystage = 0;
   if (!flat) {
-    const size_t in0 = L.lda[0];
-    L.act[0] = take((c.model == LSAM_MODEL_LSQ ? 4 : esz) * K * B * in0);
-    L.xstage = take(4 * K * B * (size_t)c.widths[0]);
+    const size_t in0 = c.widths[0];
+    const size_t ldb = L.ldb;
+    // least squares keeps its minibatch sample-major [K, B, in]; the classifiers store everything feature-major [K, width, ldb]
+    L.act[0] = (c.model == LSAM_MODEL_LSQ) ? take(4 * K * B * in0) : take(esz * K * in0 * ldb);
+    L.xstage = take(4 * K * B * in0);
     L.ystage = take(4 * K * B);
     if (c.model != LSAM_MODEL_LSQ) {
       size_t maxw = 0;
       for (size_t l = 0; l < L.layers.size(); ++l) {
-        const size_t w = L.lda[l + 1];
+        const size_t w = L.layers[l].out;
         maxw = w > maxw ? w : maxw;
         if (l + 1 < L.layers.size()) {
-          L.act[l + 1] = take(esz * K * B * w);
-          L.mask[l] = take(K * B * w);
+          L.act[l + 1] = take(esz * K * w * ldb);
+          L.mask[l] = take(K * w * ldb);
         }
       }
-      L.logits = take(4 * K * B * (size_t)L.lda.back());
+      L.logits = take(4 * K * (size_t)L.layers.back().out * ldb);
       L.rowloss = take(4 * K * B);
-      for (int i = 0; i < 2; ++i) L.dz[i] = take(esz * K * B * maxw);
-      for (int i = 0; i < 2; ++i) L.dh[i] = take(esz * K * B * maxw);
+      for (int i = 0; i < 2; ++i) L.dz[i] = take(esz * K * maxw * ldb);
+      for (int i = 0; i < 2; ++i) L.dh[i] = take(esz * K * maxw * ldb);
     }
   }
   L.total = off;
@@ -302,6 +303,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
   const int K = c->cfg.K, B = c->cfg.batch;
   const int nl = (int)L.layers.size();
   const int64_t ld = L.ld;
+  const int ldb = L.ldb;
   int rc;
   // forward
   for (int l = 0; l < nl; ++l) {
@@ -314,30 +316,29 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
       if (trc != 0) return c->fail(LSAM_ERR_CUDA, "tcgen05 forward launch failed");
       continue;
     }
-    GemmOperand A{a_in, (int64_t)B * L.lda[l], L.lda[l], 1};  // (z, b, i)
+    GemmOperand A{a_in, (int64_t)li.in * ldb, 1, ldb};       // (z, b, i) in the feature-major buffer [z][i][b]
     GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, o, i)
     if (head) {
-      EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), B, L.lda[l + 1]};
+      EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), li.out, ldb};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
     } else {
-      EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.act[l + 1]), li.residual ? a_in : nullptr, c->at<uint8_t>(L.mask[l]), B, L.lda[l + 1]};
+      EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.act[l + 1]), li.residual ? a_in : nullptr, c->at<uint8_t>(L.mask[l]), li.out, ldb};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
     }
     if (rc != LSAM_OK) return rc;
   }
   // loss and its gradient w.r.t. the logits
   const int C = L.layers[nl - 1].out;
-  const int64_t rows = (int64_t)K * B;
   int cur = 0;
-  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<(unsigned)ceil_div(rows, 8), 256, 0, c->stream>>>(
-      c->at<float>(L.logits), c->at<int32_t>(L.ylab), rows, C, L.lda[nl], B, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status()));
+  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 128), K), 128, 0, c->stream>>>(
+      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status()));
   if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out));
   // backward
   for (int l = nl - 1; l >= 0; --l) {
     const LayerInfo& li = L.layers[l];
     const T* dz = c->at<T>(L.dz[cur]);
     const T* a_in = c->at<T>(L.act[l]);
-    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 256), K), 256, 0, c->stream>>>(dz, B, li.out, L.lda[l + 1], c->g(), ld, li.b_pad));
+    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad));
     if (c->use_tc) {
       int trc = 0;
       LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream));
@@ -347,18 +348,18 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
       continue;
     }
     {
-      GemmOperand A{dz, (int64_t)B * L.lda[l + 1], 1, L.lda[l + 1]};  // (z, o, b)
-      GemmOperand Bm{a_in, (int64_t)B * L.lda[l], 1, L.lda[l]};       // (z, i, b)
+      GemmOperand A{dz, (int64_t)li.out * ldb, ldb, 1};      // (z, o, b)
+      GemmOperand Bm{a_in, (int64_t)li.in * ldb, ldb, 1};    // (z, i, b)
       EpiWgrad e{c->g(), ld, li.w_pad, li.in};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.out, li.in, B, e);
       if (rc != LSAM_OK) return rc;
     }
     if (l > 0) {
-      GemmOperand A{dz, (int64_t)B * L.lda[l + 1], L.lda[l + 1], 1};  // (z, b, o)
+      GemmOperand A{dz, (int64_t)li.out * ldb, 1, ldb};      // (z, b, o)
       GemmOperand W{P + li.w_pad, ld, 1, li.in};             // (z, i, o)
       EpiDgrad<T> e{li.residual ? c->at<T>(L.dh[(l + 1) & 1]) : nullptr,
                     L.layers[l - 1].residual ? c->at<T>(L.dh[l & 1]) : nullptr,
-                    c->at<T>(L.dz[cur ^ 1]), c->at<uint8_t>(L.mask[l - 1]), B, L.lda[l]};
+                    c->at<T>(L.dz[cur ^ 1]), c->at<uint8_t>(L.mask[l - 1]), li.in, ldb};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_DGRAD, A, W, B, li.in, li.out, e);
       if (rc != LSAM_OK) return rc;
     }
@@ -406,10 +407,15 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
   if ((rc = launch_schedule(c, c->t, c->idx(), c->stale(), c->ver(), c->slot())) != LSAM_OK) return rc;
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   if (!flat && gather) {
-    if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<bf16><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], L.lda[0], c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
-    else
-      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], L.lda[0], c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+    if (cfg.model == LSAM_MODEL_LSQ) {
+      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], cfg.widths[0], c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+    } else {
+      dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
+      if (cfg.gemm_dtype == LSAM_GEMM_BF16)
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+      else
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+    }
   }
   const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
   const int64_t n = flat ? L.d : L.ld;
@@ -492,7 +498,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     b.logits = c->at<float>(L.logits);
     for (int i = 0; i < 2; ++i) { b.dz[i] = c->at<bf16>(L.dz[i]); b.dh[i] = c->at<bf16>(L.dh[i]); }
     b.status = c->status();
-    for (size_t i = 0; i < L.lda.size() && i < 10; ++i) b.lda[i] = L.lda[i];
+    b.ldb = L.ldb;
     std::vector<TcLayer> tl;
     for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
     std::string why;
@@ -514,16 +520,18 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   const int64_t nx = rows * cfg.widths[0];
   const cudaMemcpyKind kind = on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
-  const bool bf = cfg.gemm_dtype == LSAM_GEMM_BF16;
-  const bool conv = bf || c->L.lda[0] != cfg.widths[0];  // staged when the type or the row stride differs
-  float* xdst = conv ? c->at<float>(c->L.xstage) : c->at<float>(c->L.act[0]);
+  const bool lsq = cfg.model == LSAM_MODEL_LSQ;
+  float* xdst = lsq ? c->at<float>(c->L.act[0]) : c->at<float>(c->L.xstage);  // classifiers: staged, then stored feature-major
   c->launches += 2;
   LSAM_CUDA(c, cudaMemcpyAsync(xdst, xb, sizeof(float) * nx, kind, c->stream));
   LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(c->L.ylab), yb, 4 * rows, kind, c->stream));
-  if (conv && bf)
-    LAUNCH(c, LSAM_PROF_GATHER, convert_batch_kernel<bf16><<<(unsigned)ceil_div(nx, 256), 256, 0, c->stream>>>(xdst, c->at<bf16>(c->L.act[0]), rows, cfg.widths[0], c->L.lda[0]));
-  else if (conv)
-    LAUNCH(c, LSAM_PROF_GATHER, convert_batch_kernel<float><<<(unsigned)ceil_div(nx, 256), 256, 0, c->stream>>>(xdst, c->at<float>(c->L.act[0]), rows, cfg.widths[0], c->L.lda[0]));
+  if (!lsq) {
+    dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16)
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status()));
+    else
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status()));
+  }
   int rc = step_common(c, eta, rho, false);
   if (rc != LSAM_OK) return rc;
   if (h_loss) {

@@ -24,32 +24,55 @@ gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const
   if (threadIdx.x == 0 && yb != nullptr) yb[r] = Y[s];
 }
 
-// Caller-supplied minibatch: convert [rows, in] fp32 (dense) to the activation type with row stride ld.
+// Classifier inputs are stored FEATURE-MAJOR: xt[k][i][b] = TA(X[idx[k][b]][i]) with row stride ldb, so that the
+// sample index is the contiguous one (see the layout note above the epilogues).  32 x 32 tiles go through shared
+// memory: reads run along the features of a sample, writes along the samples of a feature.
+// grid (ceil(in / 32), ceil(B / 32), K), block (32, 8).  idx == nullptr: rows come from the dense minibatch src [K, B, in].
 template <typename TA>
 __global__ void __launch_bounds__(256)
-convert_batch_kernel(const float* __restrict__ src, TA* __restrict__ dst, int64_t rows, int in, int ld) {
-  const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= rows * in) return;
-  const int64_t r = j / in;
-  dst[r * ld + (j - r * in)] = from_float<TA>(src[j]);
+gather_t_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx, int64_t n_samples,
+                int B, int in, int ldb, TA* __restrict__ xt, uint32_t* __restrict__ yb, int* __restrict__ status) {
+  __shared__ float tile[32][33];
+  const int k = blockIdx.z, i0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
+  for (int r = threadIdx.y; r < 32; r += 8) {
+    const int b = b0 + r, i = i0 + threadIdx.x;
+    float v = 0.f;
+    if (b < B) {
+      int64_t s = idx ? (int64_t)idx[(int64_t)k * B + b] : (int64_t)k * B + b;
+      if (idx && (s < 0 || s >= n_samples)) {
+        if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_INDEX);
+        s = 0;
+      }
+      if (i < in) v = X[s * in + i];
+      if (idx && blockIdx.x == 0 && threadIdx.x == 0 && yb != nullptr) yb[(int64_t)k * B + b] = Y[s];
+    }
+    tile[r][threadIdx.x] = v;
+  }
+  __syncthreads();
+  for (int r = threadIdx.y; r < 32; r += 8) {
+    const int i = i0 + r, b = b0 + threadIdx.x;
+    if (i < in && b < B) xt[((int64_t)k * in + i) * ldb + b] = from_float<TA>(tile[threadIdx.x][r]);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------ epilogues
 // Every GEMM hands its accumulator to one of these functors in LOGICAL coordinates:
 //   z = replica, b = sample in the minibatch, f = feature (output unit for forward, input unit for dgrad),
 //   or (z, o, i) = (replica, output unit, input unit) for the weight gradient.
-// Activation-like buffers are [K, B, ldw] with ldw >= width (row stride padded to a multiple of 8 elements).
+// Activation-like buffers (activations, ReLU masks, logits, backward signals) are FEATURE-MAJOR: [K, width, ldb]
+// with the sample index contiguous (ldb >= B, a multiple of 16).  In the tensor-core epilogue a thread owns one
+// feature and 32 consecutive samples, so this layout makes its accesses contiguous 16-byte vectors.
 // TP = parameter operand type, TA = activation storage type.
 
 // hidden layer: v = acc + bias[f]; r = relu(v); mask = v > 0; out = TA(skip + r)
 template <typename TP, typename TA>
 struct EpiFwdHidden {
   const TP* bias;  int64_t ld_p;           // bias[z * ld_p + f]
-  TA* out;  const TA* skip;  uint8_t* mask;  // [K, B, ldw]
-  int B, ldw;
+  TA* out;  const TA* skip;  uint8_t* mask;  // [K, width, ldb]
+  int width, ldb;
   __device__ inline void operator()(int z, int b, int f, float acc) const {
     const float v = acc + to_float(bias[(int64_t)z * ld_p + f]);
-    const int64_t e = ((int64_t)z * B + b) * ldw + f;
+    const int64_t e = ((int64_t)z * width + f) * ldb + b;
     const float r = v > 0.f ? v : 0.f;
     mask[e] = v > 0.f;
     const float sk = skip ? to_float(skip[e]) : 0.f;
@@ -61,23 +84,23 @@ struct EpiFwdHidden {
 template <typename TP>
 struct EpiFwdHead {
   const TP* bias;  int64_t ld_p;
-  float* logits;  // [K, B, ldw]
-  int B, ldw;
+  float* logits;  // [K, width, ldb]
+  int width, ldb;
   __device__ inline void operator()(int z, int b, int f, float acc) const {
-    logits[((int64_t)z * B + b) * ldw + f] = acc + to_float(bias[(int64_t)z * ld_p + f]);
+    logits[((int64_t)z * width + f) * ldb + b] = acc + to_float(bias[(int64_t)z * ld_p + f]);
   }
 };
 
 // dgrad of layer l: dh = TA(acc + skip_grad);  dz_prev = mask_prev ? dh : 0;  optionally keep dh (residual nets)
 template <typename TA>
 struct EpiDgrad {
-  const TA* dh_next;      // gradient w.r.t. the output of a residual layer (nullptr otherwise) [K, B, width]
+  const TA* dh_next;      // gradient w.r.t. the output of a residual layer (nullptr otherwise) [K, width, ldb]
   TA* dh_out;             // nullable
-  TA* dz_prev;            // [K, B, width]
+  TA* dz_prev;            // [K, width, ldb]
   const uint8_t* mask_prev;
-  int B, ldw;
+  int width, ldb;
   __device__ inline void operator()(int z, int b, int f, float acc) const {
-    const int64_t e = ((int64_t)z * B + b) * ldw + f;
+    const int64_t e = ((int64_t)z * width + f) * ldb + b;
     const float s = dh_next ? acc + to_float(dh_next[e]) : acc;
     const TA q = from_float<TA>(s);
     if (dh_out) dh_out[e] = q;
@@ -158,32 +181,32 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi) {
 }
 
 // ------------------------------------------------------------------------------------------------ softmax cross-entropy
-// One warp per sample row; logits and dz have row stride ldc.  rowloss[r] = logsumexp(l) - l[y];  dz[r][c] = TA((softmax(l)[c] - [c == y]) / B).
+// One thread per sample (consecutive threads = consecutive samples, so every access is coalesced); logits and dz are
+// feature-major [K, C, ldb].  rowloss[k][b] = logsumexp(l) - l[y];  dz[k][c][b] = TA((softmax(l)[c] - [c == y]) / B).
+// grid (ceil(B / 128), K), block 128.
 template <typename TA>
-__global__ void __launch_bounds__(256)
-softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int64_t rows, int C, int ldc, int B,
+__global__ void __launch_bounds__(128)
+softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int B, int C, int ldb,
                   TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status) {
-  const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  if (r >= rows) return;
-  const int lane = threadIdx.x & 31;
-  const float* lg = logits + r * ldc;
+  const int b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= B) return;
+  const int k = blockIdx.y;
+  const float* lg = logits + (int64_t)k * C * ldb + b;
   float m = -INFINITY;
-  for (int c = lane; c < C; c += 32) m = fmaxf(m, lg[c]);
-  m = warp_max(m);
+  for (int c = 0; c < C; ++c) m = fmaxf(m, lg[(int64_t)c * ldb]);
   float se = 0.f;
-  for (int c = lane; c < C; c += 32) se += expf(lg[c] - m);
-  se = warp_sum(se);
-  int y = labels[r];
+  for (int c = 0; c < C; ++c) se += expf(lg[(int64_t)c * ldb] - m);
+  int y = labels[(int64_t)k * B + b];
   if (y < 0 || y >= C) {
-    if (lane == 0) atomicOr(status, STATUS_BAD_INDEX);
+    atomicOr(status, STATUS_BAD_INDEX);
     y = 0;
   }
-  if (lane == 0) rowloss[r] = (m + logf(se)) - lg[y];
+  rowloss[(int64_t)k * B + b] = (m + logf(se)) - lg[(int64_t)y * ldb];
   const float inv = 1.f / se, invB = 1.f / (float)B;
-  TA* out = dz + r * ldc;
-  for (int c = lane; c < C; c += 32) {
-    const float p = expf(lg[c] - m) * inv;
-    out[c] = from_float<TA>((p - (c == y ? 1.f : 0.f)) * invB);
+  TA* out = dz + (int64_t)k * C * ldb + b;
+  for (int c = 0; c < C; ++c) {
+    const float p = expf(lg[(int64_t)c * ldb] - m) * inv;
+    out[(int64_t)c * ldb] = from_float<TA>((p - (c == y ? 1.f : 0.f)) * invB);
   }
 }
 
@@ -198,17 +221,19 @@ __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float
 }
 
 // ------------------------------------------------------------------------------------------------ bias gradient
-// g[z][b_off + o] = sum_b dz[z][b][o], samples in ascending order.  grid (ceil(out / 256), K).
+// g[z][b_off + o] = sum_b dz[z][o][b]: one warp per (replica, unit); lane l adds samples l, l + 32, ... in ascending
+// order, then the xor-shuffle tree (a fixed order).  grid (ceil(out / 8), K), block 256.
 template <typename TA>
 __global__ void __launch_bounds__(256)
-bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldz, float* __restrict__ g, int64_t ld_g, int64_t b_off) {
-  const int o = blockIdx.x * blockDim.x + threadIdx.x;
+bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off) {
+  const int o = blockIdx.x * 8 + (threadIdx.x >> 5);
   if (o >= out) return;
-  const int z = blockIdx.y;
-  const TA* p = dz + (int64_t)z * B * ldz + o;
+  const int z = blockIdx.y, lane = threadIdx.x & 31;
+  const TA* p = dz + ((int64_t)z * out + o) * ldb;
   float s = 0.f;
-  for (int b = 0; b < B; ++b) s += to_float(p[(int64_t)b * ldz]);
-  g[(int64_t)z * ld_g + b_off + o] = s;
+  for (int b = lane; b < B; b += 32) s += to_float(p[b]);
+  s = warp_sum(s);
+  if (lane == 0) g[(int64_t)z * ld_g + b_off + o] = s;
 }
 
 // ------------------------------------------------------------------------------------------------ least squares
