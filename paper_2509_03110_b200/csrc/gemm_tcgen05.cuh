@@ -77,6 +77,17 @@ __device__ inline void tma_load_3d(void* dst, const CUtensorMap* map, int c0, in
       : "memory");
 }
 
+// 3-D tiled TMA store from this CTA's shared memory (bulk async group); rows / columns outside the tensor are clipped.
+__device__ inline void tma_store_3d(const CUtensorMap* map, const void* src, int c0, int c1, int c2) {
+  asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+__device__ inline void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// wait until at most N of this thread's bulk groups are still READING shared memory / still pending at all
+template <int N> __device__ inline void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+template <int N> __device__ inline void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
+
 __device__ inline void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
   asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -156,7 +167,7 @@ template <int BLOCK_N>
 __host__ __device__ constexpr int tc_stages() { return BLOCK_N == 256 ? 4 : (BLOCK_N == 128 ? 6 : 8); }
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + BLOCK_N) * kTcBlockK * 2; }
-constexpr int kTcStageOutBytes = 4 * 32 * 33 * 4;  // epilogue staging: one 32 x 33 fp32 block per epilogue warp
+constexpr int kTcStageOutBytes = 4 * 2 * 4096;  // wgrad epilogue staging: two 32 x 32 fp32 blocks (128B-swizzled) per epilogue warp
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_smem_bytes() {
   return tc_stages<BLOCK_N>() * tc_stage_bytes<BLOCK_N>() + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTcStageOutBytes;
@@ -168,7 +179,8 @@ __host__ __device__ constexpr int tc_smem_bytes() {
 //   M/N-contiguous operand:         map dims {rows, Kd, Z}, box {64, 64, 1} (one box per 64 rows of the tile)
 template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(kTcThreads, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int M, int N, int Kd,
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                    const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
                     int Z, TcEpi ep, int* __restrict__ status) {
   constexpr int STAGES = tc_stages<BLOCK_N>();
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
@@ -177,15 +189,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   constexpr uint32_t IDESC = tc::instr_desc(kTcBlockM, BLOCK_N, A_MN, B_MN);
 
   extern __shared__ uint8_t smem_raw[];
-  uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles + STAGES * (A_BYTES + B_BYTES));
+  // round the tile area up to 1024 bytes by pointer arithmetic on the shared array itself (keeps the address space known)
+  uint8_t* tiles = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
+  uint8_t* stage = tiles + STAGES * (A_BYTES + B_BYTES);  // 1024-byte aligned: the tile area is a multiple of 1024
+  uint64_t* bars = reinterpret_cast<uint64_t*>(stage + kTcStageOutBytes);
   uint64_t* full = bars;                     // [STAGES]  TMA -> MMA
   uint64_t* empty = bars + STAGES;           // [STAGES]  MMA -> TMA
   uint64_t* acc_full = bars + 2 * STAGES;    // [2]       MMA -> epilogue
   uint64_t* acc_empty = acc_full + 2;        // [2]       epilogue -> MMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  float* stage = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(bars) + 256);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (M + kTcBlockM - 1) / kTcBlockM;
@@ -275,6 +288,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
     const int quad = warp & 3;
+    int sbuf_sel = 0;  // staging buffer of the next output block (wgrad)
     int as = 0;
     uint32_t aph = 0;
     bool ok = true;
@@ -294,21 +308,28 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         tc::tmem_ld_wait();
         const int nb = n0 + c * 32;
         if (EPI == TC_EPI_WGRAD) {
-          // Stage the warp's 32 x 32 block through shared memory (row stride 33: conflict-free both ways) so that
-          // every store instruction of the warp writes one full 128-byte line of a gradient row.
-          float* st = stage + (warp - 2) * (32 * 33);
-#pragma unroll
-          for (int j = 0; j < 32; ++j) st[lane * 33 + j] = __uint_as_float(r[j]);
-          __syncwarp();
+          // The warp's 32 x 32 fp32 block goes to shared memory in the 128-byte-swizzled layout of the output tensor
+          // map (row = lane, 16-byte chunk q stored at position q ^ (row % 8)), then one TMA store writes it to the
+          // gradient rows (clipped at the ragged edges).  Two buffers per warp: the store of a chunk overlaps the
+          // staging of the next one.
           const int mrow0 = mt * kTcBlockM + quad * 32;
-          const int col = nb + lane;
-          if (col < N) {
-            float* dst = ep.g + (int64_t)z * ep.ld_g + ep.w_off + (int64_t)mrow0 * ep.ldw + col;
-            const int rows = M - mrow0 < 32 ? M - mrow0 : 32;
-#pragma unroll 8
-            for (int i = 0; i < rows; ++i) dst[(int64_t)i * ep.ldw] = st[i * 33 + lane];
+          if (mrow0 < M && nb < N) {  // warp-uniform: blocks wholly outside the matrix are neither staged nor stored
+            uint8_t* sbuf = stage + (warp - 2) * 8192 + sbuf_sel * 4096;
+            sbuf_sel ^= 1;
+            // at most one store may still be reading shared memory: the previous one, which used the other buffer
+            if (lane == 0) tc::bulk_wait_read<1>();
+            __syncwarp();
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *reinterpret_cast<float4*>(sbuf + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                  make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+            tc::fence_proxy_async();
+            __syncwarp();
+            if (lane == 0) {
+              tc::tma_store_3d(&map_c, sbuf, nb, mrow0, z);
+              tc::bulk_commit();
+            }
           }
-          __syncwarp();
         } else if (m < M && nb < N) {
           // element (unit m, sample nb + j) of the feature-major buffers: 32 consecutive samples per thread
           const int64_t t0 = ((int64_t)z * M + m) * ep.ldb + nb;
@@ -412,6 +433,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (lane == 0) tc::mbar_arrive(&acc_empty[as]);
       if (++as == 2) { as = 0; aph ^= 1u; }
     }
+    if (EPI == TC_EPI_WGRAD && lane == 0) tc::bulk_wait_all<0>();  // every gradient block has reached global memory
     if (!ok && lane == 0) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
   }
 
@@ -439,7 +461,7 @@ struct TcBuffers {
 };
 
 struct TcGemm {
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_c;  // map_c: fp32 output of wgrad (a copy of map_a elsewhere, unused)
   int M = 0, N = 0, Kd = 0, block_n = 0;
   TcEpi ep{};
   bool valid = false;
@@ -468,16 +490,18 @@ inline PFN_encodeTiled tc_encode_fn() {
 }
 
 // bf16 tensor [Z][rows][cols] with element strides (row_stride, z_stride); dim 0 = cols (contiguous).
-inline bool tc_make_map(CUtensorMap* m, const bf16* base, uint64_t cols, uint64_t rows, uint64_t Z, uint64_t row_stride,
+template <typename T>
+inline bool tc_make_map(CUtensorMap* m, const T* base, uint64_t cols, uint64_t rows, uint64_t Z, uint64_t row_stride,
                         uint64_t z_stride, uint32_t box_cols, uint32_t box_rows) {
   PFN_encodeTiled enc = tc_encode_fn();
   if (!enc) return false;
-  if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride * 2) % 16 || (z_stride * 2) % 16) return false;
+  constexpr uint64_t ES = sizeof(T);
+  if ((reinterpret_cast<uintptr_t>(base) & 15) || (row_stride * ES) % 16 || (z_stride * ES) % 16 || box_cols * ES > 128) return false;
   cuuint64_t dims[3] = {cols, rows, Z};
-  cuuint64_t strides[2] = {row_stride * 2, z_stride * 2};
+  cuuint64_t strides[2] = {row_stride * ES, z_stride * ES};
   cuuint32_t box[3] = {box_cols, box_rows, 1};
   cuuint32_t estr[3] = {1, 1, 1};
-  return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<bf16*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+  return enc(m, sizeof(T) == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<T*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -515,6 +539,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       g.ep.bias = b.xop + ly.b_pad; g.ep.ld_p = b.ld; g.ep.ldb = b.ldb;
       if (head) g.ep.logits = b.logits;
       else { g.ep.out = b.act[l + 1]; g.ep.skip = ly.residual ? b.act[l] : nullptr; g.ep.mask = b.mask[l]; }
+      g.map_c = g.map_a;
       g.valid = ok;
     }
     {  // wgrad: A = dz_l [out][B] (samples contiguous = contraction), B = act_l [in][B]
@@ -522,6 +547,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in);
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.block_n);
+      ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.valid = ok;
     }
@@ -533,6 +559,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       g.ep.dh_next = ly.residual ? b.dh[(l + 1) & 1] : nullptr;
       g.ep.dh_out = layers[l - 1].residual ? b.dh[l & 1] : nullptr;
       g.ep.dz_prev = b.dz[cur ^ 1]; g.ep.mask_prev = b.mask[l - 1]; g.ep.ldb = b.ldb;
+      g.map_c = g.map_a;
       g.valid = ok;
     }
     if (!ok) { why = "tensor map creation failed"; return 1; }
@@ -550,7 +577,7 @@ inline int tc_launch_one(const TcPlan& P, const TcGemm& g, cudaStream_t stream) 
   }
   const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, kTcBlockM) * ceil_div(g.N, BLOCK_N);
   const int grid = (int)(tiles < P.sms ? tiles : P.sms);
-  kern<<<grid, kTcThreads, tc_smem_bytes<BLOCK_N>(), stream>>>(g.map_a, g.map_b, g.M, g.N, g.Kd, P.Z, g.ep, P.status);
+  kern<<<grid, kTcThreads, tc_smem_bytes<BLOCK_N>(), stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status);
   return cudaPeekAtLastError() == cudaSuccess ? 0 : 1;
 }
 
