@@ -156,6 +156,8 @@ struct TcEpi {
   const bf16* dh_next;  bf16* dh_out;  bf16* dz_prev;  const uint8_t* mask_prev;
   // wgrad: g[z * ld_g + w_off + m * ldw + n]
   float* g;  int64_t ld_g, w_off;  int ldw;
+  // wgrad: sum of squares of every 32-row block of the tile -> partial[z * ld_partial + slot0 + (mt * n_tiles + nt) * 4 + quad]
+  float* partial;  int64_t ld_partial;  int slot0;
   int ldb;  // sample stride of the feature-major buffers (multiple of 16)
 };
 
@@ -300,6 +302,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       tc::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BLOCK_N);
       float bias = 0.f;
+      float ssq = 0.f;  // wgrad: sum of squares of this thread's row of the tile
       if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) bias = to_float(ep.bias[(int64_t)z * ep.ld_p + m]);
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
@@ -314,6 +317,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           // staging of the next one.
           const int mrow0 = mt * kTcBlockM + quad * 32;
           if (mrow0 < M && nb < N) {  // warp-uniform: blocks wholly outside the matrix are neither staged nor stored
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ssq = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ssq);  // zero-filled edges add 0
             uint8_t* sbuf = stage + (warp - 2) * 8192 + sbuf_sel * 4096;
             sbuf_sel ^= 1;
             // at most one store may still be reading shared memory: the previous one, which used the other buffer
@@ -428,6 +433,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
         }
       }
+      if (EPI == TC_EPI_WGRAD && ep.partial != nullptr) {
+        // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows
+        const float tot = warp_sum(ssq);
+        if (lane == 0) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)mt * n_tiles + nt) * 4 + quad] = tot;
+      }
       tc::tc_fence_before();
       __syncwarp();
       if (lane == 0) tc::mbar_arrive(&acc_empty[as]);
@@ -458,6 +468,7 @@ struct TcBuffers {
   bf16* xop; float* g; int64_t ld;
   bf16* act[9]; uint8_t* mask[9]; float* logits; bf16* dz[2]; bf16* dh[2]; int* status;
   int ldb;
+  float* partial; int64_t ld_partial;  // per-replica slots for the fused sum of squares
 };
 
 struct TcGemm {
@@ -472,6 +483,8 @@ struct TcPlan {
   int* status = nullptr;
   int64_t* launches = nullptr;
   std::vector<TcGemm> fwd, dgrad, wgrad;
+  std::vector<int> bias_slot0;  // first partial slot of the bias-gradient blocks of each layer
+  int n_slots = 0;              // partial slots used per replica
 };
 
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -506,6 +519,16 @@ inline bool tc_make_map(CUtensorMap* m, const T* base, uint64_t cols, uint64_t r
 }
 
 inline int tc_pick_block_n(int n) { return n > 128 ? 256 : (n > 64 ? 128 : 64); }
+// Partial-sum slots one replica needs when the sum of squares is fused into the weight-gradient epilogue:
+// four per output tile (one per 32-row block) plus one per 8 bias units.
+inline int64_t tc_norm_slots(const lsam_config& c) {
+  int64_t n = 0;
+  for (int l = 0; l < c.n_layers; ++l) {
+    const int in = c.widths[l], out = c.widths[l + 1];
+    n += ceil_div(out, kTcBlockM) * ceil_div(in, tc_pick_block_n(in)) * 4 + ceil_div(out, 8);
+  }
+  return n;
+}
 
 // The tensor-core path needs every layer's input width to be a multiple of 8 (16-byte row strides of W and of
 // the activations); output widths are free (padded strides, TMA zero-fills the ragged edge).
@@ -525,6 +548,8 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   const int L = P.n_layers, B = c.batch, Z = c.K;
   P.fwd.assign(L, TcGemm()); P.dgrad.assign(L, TcGemm()); P.wgrad.assign(L, TcGemm());
   const uint64_t ldb = (uint64_t)b.ldb;
+  P.bias_slot0.assign(L, 0);
+  int slot = 0;
   for (int l = 0; l < L; ++l) {
     const TcLayer& ly = layers[l];
     const int cur = (L - 1 - l) & 1;  // dz buffer holding the pre-activation gradient of layer l
@@ -549,6 +574,10 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.block_n);
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
+      g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
+      slot += (int)(ceil_div(ly.out, kTcBlockM) * ceil_div(ly.in, g.block_n) * 4);
+      P.bias_slot0[l] = slot;
+      slot += (int)ceil_div(ly.out, 8);
       g.valid = ok;
     }
     if (l > 0) {  // dgrad: A = W [out][in] read as (m = in contiguous, kd = out), B = dz_l [out][B] (samples contiguous)
@@ -564,6 +593,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     }
     if (!ok) { why = "tensor map creation failed"; return 1; }
   }
+  P.n_slots = slot;
   return 0;
 }
 

@@ -91,6 +91,10 @@ bool plan(const lsam_config& c, Layout& L) {
   L.ring = c.stale_max + 2;
   // partial-sum slots per replica; FLAT may fall back to scalar chunks when the caller's gradient buffers are misaligned
   L.nchunks = ceil_div(L.ld, (c.model == LSAM_MODEL_FLAT) ? norm_chunk<1>() : norm_chunk<4>());
+  if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {  // room for the slots of the fused tensor-core norm
+    const int64_t slots = tc_norm_slots(c);
+    L.nchunks = slots > L.nchunks ? slots : L.nchunks;
+  }
 
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 256); return o; };
@@ -237,6 +241,12 @@ int prof_end(lsam_ctx* c) {
 int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float rho, float* norm_out, float* scale_out) {
   float* partial = c->at<float>(c->L.partial);
   const int64_t nch = c->L.nchunks;
+  if (c->use_tc) {
+    // tensor-core path: the weight- and bias-gradient kernels of the pass just run have left the sums of squares of
+    // all their blocks in the partial slots; only the fixed-order final sum remains
+    LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status()));
+    return LSAM_OK;
+  }
   dim3 grid((unsigned)ceil_div(n, vec4 ? norm_chunk<4>() : norm_chunk<1>()), c->cfg.K);
   if ((int64_t)grid.x > nch) return c->fail(LSAM_ERR_WORKSPACE, "norm: partial-sum buffer too small");
   if (vec4) LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<4><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch));
@@ -338,7 +348,8 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
     const LayerInfo& li = L.layers[l];
     const T* dz = c->at<T>(L.dz[cur]);
     const T* a_in = c->at<T>(L.act[l]);
-    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad));
+    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad,
+        c->use_tc ? c->at<float>(L.partial) : nullptr, L.nchunks, c->use_tc ? c->tc.bias_slot0[l] : 0));
     if (c->use_tc) {
       int trc = 0;
       LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream));
@@ -499,6 +510,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     for (int i = 0; i < 2; ++i) { b.dz[i] = c->at<bf16>(L.dz[i]); b.dh[i] = c->at<bf16>(L.dh[i]); }
     b.status = c->status();
     b.ldb = L.ldb;
+    b.partial = c->at<float>(L.partial); b.ld_partial = L.nchunks;
     std::vector<TcLayer> tl;
     for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
     std::string why;

@@ -223,17 +223,31 @@ __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float
 // ------------------------------------------------------------------------------------------------ bias gradient
 // g[z][b_off + o] = sum_b dz[z][o][b]: one warp per (replica, unit); lane l adds samples l, l + 32, ... in ascending
 // order, then the xor-shuffle tree (a fixed order).  grid (ceil(out / 8), K), block 256.
+// If partial != nullptr the block also writes the sum of squares of its 8 bias gradients (warps in ascending order)
+// to partial[z * ld_partial + slot0 + blockIdx.x], for the fused gradient norm.
 template <typename TA>
 __global__ void __launch_bounds__(256)
-bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off) {
-  const int o = blockIdx.x * 8 + (threadIdx.x >> 5);
-  if (o >= out) return;
+bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off,
+                 float* __restrict__ partial, int64_t ld_partial, int slot0) {
+  __shared__ float sq[8];
+  const int w = threadIdx.x >> 5, o = blockIdx.x * 8 + w;
   const int z = blockIdx.y, lane = threadIdx.x & 31;
-  const TA* p = dz + ((int64_t)z * out + o) * ldb;
   float s = 0.f;
-  for (int b = lane; b < B; b += 32) s += to_float(p[b]);
-  s = warp_sum(s);
-  if (lane == 0) g[(int64_t)z * ld_g + b_off + o] = s;
+  if (o < out) {
+    const TA* p = dz + ((int64_t)z * out + o) * ldb;
+    for (int b = lane; b < B; b += 32) s += to_float(p[b]);
+    s = warp_sum(s);
+    if (lane == 0) g[(int64_t)z * ld_g + b_off + o] = s;
+  }
+  if (partial != nullptr) {
+    if (lane == 0) sq[w] = s * s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+      for (int i = 0; i < 8; ++i) t += sq[i];
+      partial[(int64_t)z * ld_partial + slot0 + blockIdx.x] = t;
+    }
+  }
 }
 
 // ------------------------------------------------------------------------------------------------ least squares
