@@ -67,7 +67,7 @@ def work_model(w, tc):
     K, B, d = w["K"], w["B"], param_count(w)
     op = 2 if w["bf16"] else 4
     out = {}
-    out["norm"] = dict(bytes=4.0 * K * d)                                    # read g1
+    out["norm"] = dict(bytes=0.0 if tc else 4.0 * K * d)                     # read g1 (fused into the wgrad epilogue on the tensor-core path)
     out["perturb"] = dict(bytes=(4.0 + 4.0 + op) * K * d)                    # read x, g1; write x~
     out["update"] = dict(bytes=(4.0 + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2, x rw, v rw, operand copy; y, acc rw
     if w["model"] in (MLP, RESMLP):
@@ -424,8 +424,7 @@ def main():
     # the three streaming kernels of the fused update path, always reported
     stream_gbs = {}
     for k in ("norm", "perturb", "update"):
-        if prof[k][1] > 0:
-            n_main = prof[k][1] / (2 if k == "norm" else 1)  # the norm class counts its tiny finalize launch too
+        if prof[k][1] > 0 and work[k]["bytes"] > 0:
             stream_gbs[k] = round(work[k]["bytes"] * args.steps / (prof[k][0] * 1e-3) / 1e9, 1)
     roof["streaming_kernels_gbs"] = stream_gbs
 

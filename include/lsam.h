@@ -137,6 +137,8 @@ int lsam_read_step_info(lsam_ctx* ctx, float* h_loss, float* h_gnorm1, float* h_
  * (as stored: rounded to bf16 in BF16 mode, where it also needs LSAM_FLAG_KEEP_G1 because the operand buffer
  * is reused by the update).  h_dst [K, d] unpadded, host.  Synchronises. */
 int lsam_read_grads(lsam_ctx* ctx, int pass, float* h_dst);
+/* Same for the single replica k: h_dst [d]. */
+int lsam_read_grads_replica(lsam_ctx* ctx, int pass, int k, float* h_dst);
 /* FLAT only: device buffers [K, d] fp32 (row stride d) holding g1 and g2 for the following steps; borrowed. */
 int lsam_set_external_grads(lsam_ctx* ctx, const float* d_g1, const float* d_g2);
 /* Overwrite worker iterates x [K, d], momentum v [K, d] and the CURRENT centre y [d] (device pointers, any may be

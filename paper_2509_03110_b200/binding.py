@@ -21,7 +21,7 @@ PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "l
 
 EXPORTS = [
     "lsam_param_count", "lsam_workspace_bytes", "lsam_init", "lsam_step", "lsam_step_batch", "lsam_couple",
-    "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads",
+    "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads", "lsam_read_grads_replica",
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
     "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static",
@@ -74,6 +74,7 @@ def lib():
     L.lsam_read_schedule.argtypes = [vp, C.c_int64, vp, vp, vp]
     L.lsam_read_step_info.argtypes = [vp, vp, vp, vp]
     L.lsam_read_grads.argtypes = [vp, C.c_int, vp]
+    L.lsam_read_grads_replica.argtypes = [vp, C.c_int, C.c_int, vp]
     L.lsam_set_external_grads.argtypes = [vp, vp, vp]
     L.lsam_write_state.argtypes = [vp, vp, vp, vp]
     L.lsam_read_state.argtypes = [vp, vp, vp, vp]
@@ -241,6 +242,11 @@ class Lsam:
     def read_grads(self, which_pass):
         out = np.empty((self.K, self.d), dtype=np.float32)
         self._check(lib().lsam_read_grads(self._h, int(which_pass), _np_ptr(out)))
+        return out
+
+    def read_grads_replica(self, which_pass, k):
+        out = np.empty(self.d, dtype=np.float32)
+        self._check(lib().lsam_read_grads_replica(self._h, int(which_pass), int(k), _np_ptr(out)))
         return out
 
     def set_external_grads(self, g1, g2):

@@ -611,13 +611,14 @@ int lsam_read_step_info(lsam_ctx* c, float* h_loss, float* h_gnorm1, float* h_gn
   return LSAM_OK;
 }
 
-int lsam_read_grads(lsam_ctx* c, int pass, float* h_dst) {
+static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float* h_dst) {
   if (!c || !h_dst || pass < 1 || pass > 3) return LSAM_ERR_INVALID;
   const Layout& L = c->L;
   const int K = c->cfg.K;
   const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
   float* tmp = c->at<float>(L.tmp);
-  for (int k = 0; k < K; ++k) {
+  (void)K;
+  for (int k = k_begin; k < k_end; ++k) {
     int rc = LSAM_OK;
     if (pass == 3) {
       if (c->cfg.gemm_dtype == LSAM_GEMM_BF16) {
@@ -639,10 +640,20 @@ int lsam_read_grads(lsam_ctx* c, int pass, float* h_dst) {
       rc = seg_copy<false>(c, src + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
     }
     if (rc != LSAM_OK) return rc;
-    LSAM_CUDA(c, cudaMemcpyAsync(h_dst + (size_t)k * L.d, tmp, sizeof(float) * L.d, cudaMemcpyDeviceToHost, c->stream));
+    LSAM_CUDA(c, cudaMemcpyAsync(h_dst + (size_t)(k - k_begin) * L.d, tmp, sizeof(float) * L.d, cudaMemcpyDeviceToHost, c->stream));
     LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
   }
   return LSAM_OK;
+}
+
+int lsam_read_grads(lsam_ctx* c, int pass, float* h_dst) {
+  if (!c) return LSAM_ERR_INVALID;
+  return read_grads_range(c, pass, 0, c->cfg.K, h_dst);
+}
+
+int lsam_read_grads_replica(lsam_ctx* c, int pass, int k, float* h_dst) {
+  if (!c || k < 0 || k >= c->cfg.K) return LSAM_ERR_INVALID;
+  return read_grads_range(c, pass, k, k + 1, h_dst);
 }
 
 int lsam_set_external_grads(lsam_ctx* c, const float* d_g1, const float* d_g2) {
