@@ -42,6 +42,9 @@ WORKLOADS = {
 LAMBDA0, MU, BETA, ETA_PRIME, GAMMA = 0.9, 0.9, 0.9, 1.0, 1e-12
 NOMINAL_HBM_GBS, FALLBACK_HBM_GBS, FALLBACK_BF16_TF = 8000.0, 6650.0, 1590.0
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x max SM clock
+# ncu counters of one update_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) at the c4 shape with K = 4
+# replicas, see profiles/dram_traffic_c4_k4.md; traffic grows with (22 K + 12) d, so it is scaled to the K of the run.
+NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=6646099712.0)
 
 
 def param_count(w):
@@ -51,6 +54,10 @@ def param_count(w):
         return w["widths"][0]
     ws = w["widths"]
     return sum(ws[i] * ws[i + 1] + ws[i + 1] for i in range(len(ws) - 1))
+
+
+def wk_bytes(work, name):
+    return work[name]["bytes"]
 
 
 def peaks():
@@ -407,6 +414,9 @@ def main():
     wk = work.get(top, {})
     launches_per_step = tn / args.steps
     roof = dict(kernel=top, share_of_kernel_time=shares.get(top), traffic=None, kernel_time_shares=shares)
+    if top == "update" and args.workload == NCU_UPDATE_TRAFFIC["workload"] and w["bf16"]:
+        roof["traffic"] = NCU_UPDATE_TRAFFIC["bytes"] * (22.0 * w["K"] + 12.0) / (22.0 * NCU_UPDATE_TRAFFIC["K"] + 12.0)
+        roof["traffic_source"] = "ncu at K=4 scaled by (22K+12)/(22*4+12); algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
     if top in ("gemm_fwd", "gemm_dgrad") and ctx.uses_tcgen05():
         ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
         roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_sustained"], peak_source=f"{pk['src']} (sustained bf16)")
@@ -427,6 +437,13 @@ def main():
         if prof[k][1] > 0 and work[k]["bytes"] > 0:
             stream_gbs[k] = round(work[k]["bytes"] * args.steps / (prof[k][0] * 1e-3) / 1e9, 1)
     roof["streaming_kernels_gbs"] = stream_gbs
+    gemm = {}
+    for k in ("gemm_fwd", "gemm_dgrad", "gemm_wgrad"):
+        if k in work and prof[k][1] > 0:
+            sec = prof[k][0] * 1e-3
+            gemm[k] = dict(tflops=round(work[k]["flops"] * args.steps / sec / 1e12, 1), gbs=round(work[k]["bytes"] * args.steps / sec / 1e9, 1),
+                           frac_of_bf16_sustained=round(work[k]["flops"] * args.steps / sec / 1e12 / pk["bf16_sustained"], 3) if w["bf16"] else None)
+    roof["gemm_classes"] = gemm
 
     cpu = None
     if not args.no_cpu_baseline:

@@ -340,7 +340,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
   // loss and its gradient w.r.t. the logits
   const int C = L.layers[nl - 1].out;
   int cur = 0;
-  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 128), K), 128, 0, c->stream>>>(
+  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
       c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status()));
   if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out));
   // backward

@@ -181,30 +181,46 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi) {
 }
 
 // ------------------------------------------------------------------------------------------------ softmax cross-entropy
-// One thread per sample (consecutive threads = consecutive samples, so every access is coalesced); logits and dz are
-// feature-major [K, C, ldb].  rowloss[k][b] = logsumexp(l) - l[y];  dz[k][c][b] = TA((softmax(l)[c] - [c == y]) / B).
-// grid (ceil(B / 128), K), block 128.
+// logits and dz are feature-major [K, C, ldb].  A block handles 32 consecutive samples (threadIdx.x, so every access is
+// coalesced) with 8 class groups (threadIdx.y: classes cg, cg + 8, ...); the per-sample maximum and sum of exponentials
+// are combined across the groups in group order.
+//   rowloss[k][b] = logsumexp(l) - l[y];  dz[k][c][b] = TA((softmax(l)[c] - [c == y]) / B).
+// grid (ceil(B / 32), K), block (32, 8).
 template <typename TA>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(256)
 softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int B, int C, int ldb,
                   TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status) {
-  const int b = blockIdx.x * blockDim.x + threadIdx.x;
-  if (b >= B) return;
-  const int k = blockIdx.y;
-  const float* lg = logits + (int64_t)k * C * ldb + b;
+  __shared__ float red[8][33];
+  const int b = blockIdx.x * 32 + threadIdx.x, cg = threadIdx.y, k = blockIdx.y;
+  const bool live = b < B;
+  const float* lg = logits + (int64_t)k * C * ldb + (live ? b : 0);
   float m = -INFINITY;
-  for (int c = 0; c < C; ++c) m = fmaxf(m, lg[(int64_t)c * ldb]);
+  if (live)
+    for (int c = cg; c < C; c += 8) m = fmaxf(m, lg[(int64_t)c * ldb]);
+  red[cg][threadIdx.x] = m;
+  __syncthreads();
+  m = red[0][threadIdx.x];
+#pragma unroll
+  for (int i = 1; i < 8; ++i) m = fmaxf(m, red[i][threadIdx.x]);
+  __syncthreads();
   float se = 0.f;
-  for (int c = 0; c < C; ++c) se += expf(lg[(int64_t)c * ldb] - m);
+  if (live)
+    for (int c = cg; c < C; c += 8) se += expf(lg[(int64_t)c * ldb] - m);
+  red[cg][threadIdx.x] = se;
+  __syncthreads();
+  se = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) se += red[i][threadIdx.x];
+  if (!live) return;
   int y = labels[(int64_t)k * B + b];
   if (y < 0 || y >= C) {
-    atomicOr(status, STATUS_BAD_INDEX);
+    if (cg == 0) atomicOr(status, STATUS_BAD_INDEX);
     y = 0;
   }
-  rowloss[(int64_t)k * B + b] = (m + logf(se)) - lg[(int64_t)y * ldb];
+  if (cg == 0) rowloss[(int64_t)k * B + b] = (m + logf(se)) - lg[(int64_t)y * ldb];
   const float inv = 1.f / se, invB = 1.f / (float)B;
   TA* out = dz + (int64_t)k * C * ldb + b;
-  for (int c = 0; c < C; ++c) {
+  for (int c = cg; c < C; c += 8) {
     const float p = expf(lg[(int64_t)c * ldb] - m) * inv;
     out[(int64_t)c * ldb] = from_float<TA>((p - (c == y ? 1.f : 0.f)) * invB);
   }
