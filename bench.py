@@ -56,6 +56,23 @@ def param_count(w):
     return sum(ws[i] * ws[i + 1] + ws[i + 1] for i in range(len(ws) - 1))
 
 
+def max_over_ranks(ms, world, device=None):
+    """Time of the slowest rank (the job's time); a plain float when there is one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([float(ms)], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(world, units_per_rank_step, ms_per_step):
+    """Aggregate throughput of `world` independent replicas of the workload (weak scaling, no data-path collective)."""
+    return world * units_per_rank_step / (ms_per_step * 1e-3)
+
+
 def wk_bytes(work, name):
     return work[name]["bytes"]
 
@@ -336,13 +353,10 @@ def main():
     launches = ctx.launch_count() - launches0
     if ctx.status() != 0:
         raise SystemExit("device status word is not clean after the timed region")
-    if world > 1:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = max_over_ranks(ms, world, dev)
     ms_step = ms / args.steps
     units_step = (36.0 * w["K"] * d / 1e9) if flat else float(w["K"] * w["B"])
-    value = world * units_step / (ms_step * 1e-3)
+    value = whole_job_value(world, units_step, ms_step)
 
     # ---- end to end through the C ABI with host buffers (minibatch H2D and loss D2H inside the timed region)
     e2e = None
@@ -367,12 +381,8 @@ def main():
                 ctx.couple()
         e1.record(stream)
         barrier()
-        ems = e0.elapsed_time(e1)
-        if world > 1:
-            tmax = torch.tensor([ems], device=dev)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            ems = float(tmax.item())
-        e2e = dict(value=world * w["K"] * w["B"] / (ems / nst * 1e-3), unit=unit, h2d_bytes_per_step=int(xbs[0].numel() * 4 + ybs[0].numel() * 4),
+        ems = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        e2e = dict(value=whole_job_value(world, w["K"] * w["B"], ems / nst), unit=unit, h2d_bytes_per_step=int(xbs[0].numel() * 4 + ybs[0].numel() * 4),
                    d2h_bytes_per_step=int(4 * w["K"]), steps=nst)
     else:
         # optimiser-only: the gradients are the step's inputs; copy them from pinned host memory every step
@@ -392,8 +402,8 @@ def main():
                 ctx.read_step_info()
             e1.record(stream)
             barrier()
-            ems = e0.elapsed_time(e1)
-            e2e = dict(value=world * units_step / (ems / nst * 1e-3), unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K), steps=nst)
+            ems = max_over_ranks(e0.elapsed_time(e1), world, dev)
+            e2e = dict(value=whole_job_value(world, units_step, ems / nst), unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K), steps=nst)
         else:
             e2e = dict(value=None, unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K),
                        note="gradient buffers of this sweep point exceed the pinned-memory budget; run --flat-d <= 64000000")
