@@ -166,13 +166,22 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
   if (j >= a.n) return;
   if (VEC == 4) {
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll 2
+    // software pipeline over the replicas: the four loads of replica k + 1 are issued before the arithmetic and the
+    // stores of replica k, so that twice as many bytes are in flight per thread
+    float4 gv = __ldcs(reinterpret_cast<const float4*>(a.g + j));
+    float4 xv = *reinterpret_cast<const float4*>(a.x + j);
+    float4 vv = *reinterpret_cast<const float4*>(a.v + j);
+    float4 yv = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[0] * a.ld + j));
     for (int k = 0; k < a.K; ++k) {
       const int64_t o = (int64_t)k * a.ld + j;
-      const float4 gv = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)k * a.ldg + j));
-      float4 xv = *reinterpret_cast<const float4*>(a.x + o);
-      float4 vv = *reinterpret_cast<const float4*>(a.v + o);
-      const float4 yv = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[k] * a.ld + j));
+      float4 gn = gv, xn = xv, vn = vv, yn = yv;
+      if (k + 1 < a.K) {
+        const int64_t on = o + a.ld;
+        gn = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)(k + 1) * a.ldg + j));
+        xn = *reinterpret_cast<const float4*>(a.x + on);
+        vn = *reinterpret_cast<const float4*>(a.v + on);
+        yn = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[k + 1] * a.ld + j));
+      }
       float G;
 #define LSAM_UPD(c)                                                         \
   G = fmaf(a.lambda, xv.c - yv.c, gv.c);                                    \
@@ -192,6 +201,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
           *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(a.xop) + o) = pk;
         }
       }
+      gv = gn; xv = xn; vv = vn; yv = yn;
     }
     float4 av = *reinterpret_cast<const float4*>(a.acc + j);
     av.x += s.x; av.y += s.y; av.z += s.z; av.w += s.w;
