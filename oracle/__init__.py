@@ -33,7 +33,7 @@ class OracleConfig(C.Structure):
     _fields_ = [
         ("model", C.c_int32), ("n_layers", C.c_int32), ("widths", C.c_int32 * 9), ("K", C.c_int32),
         ("batch", C.c_int32), ("gemm_dtype", C.c_int32), ("nesterov", C.c_int32), ("tau", C.c_int32),
-        ("stale_max", C.c_int32), ("reserved", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
+        ("stale_max", C.c_int32), ("active_num", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_double), ("gamma", C.c_double), ("lam", C.c_double),
         ("beta", C.c_double), ("eta_prime", C.c_double),
     ]
@@ -66,6 +66,9 @@ def lib():
         L.oracle_read_grads.argtypes = [vp, vp, vp, vp]
         L.oracle_set_external_grads.argtypes = [vp, vp, vp]
         L.oracle_read_counters.argtypes = [vp, vp, vp, vp]
+        L.oracle_read_active.argtypes = [vp, vp]
+        L.oracle_tag_active.restype = C.c_uint64
+        L.oracle_tag_order.restype = C.c_uint64
         L.oracle_loss_grad.argtypes = [cfgp, vp, vp, vp, vp, C.c_int32, vp, vp]
         L.oracle_forward.argtypes = [cfgp, vp, vp, vp, C.c_int32, vp]
         L.oracle_mix64.restype = C.c_uint64
@@ -82,7 +85,7 @@ def lib():
 
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, nesterov=1, gamma=1e-12,
-                lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0):
+                lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, active_num=256):
     """Float hyper-parameters are taken at their fp32 value, the precision the C-ABI carries them in."""
     c = OracleConfig()
     c.model = model
@@ -92,6 +95,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, ne
         c.widths[i] = int(w)
     c.K, c.batch, c.gemm_dtype, c.nesterov, c.tau = int(K), int(batch), int(gemm_dtype), int(nesterov), int(tau)
     c.stale_max, c.n_samples, c.flat_d, c.seed = int(stale_max), int(n_samples), int(flat_d), int(seed)
+    c.active_num = int(active_num)
     f32 = lambda v: float(np.float32(v))
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = f32(mu), f32(gamma), f32(lam), f32(beta), f32(eta_prime)
     return c
@@ -227,6 +231,11 @@ class Oracle:
         g2 = np.ascontiguousarray(g2, dtype=np.float32).reshape(self.K, self.d)
         self._keep = [g1, g2]
         assert lib().oracle_set_external_grads(self._h, _ptr(g1), _ptr(g2)) == 0
+
+    def read_active(self):
+        a = np.zeros(self.K, dtype=np.int32)
+        assert lib().oracle_read_active(self._h, _ptr(a)) == 0
+        return a
 
     def counters(self):
         t = np.zeros(1, dtype=np.int64)

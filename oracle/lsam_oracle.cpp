@@ -28,6 +28,8 @@ inline uint64_t mix64(uint64_t z) {
 }
 const uint64_t TAG_IDX = 0x6c73616d5f696478ULL;    // ASCII "lsam_idx"
 const uint64_t TAG_STALE = 0x6c73616d5f73746cULL;  // ASCII "lsam_stl"
+const uint64_t TAG_ACT = 0x6c73616d5f616374ULL;    // ASCII "lsam_act"
+const uint64_t TAG_ORD = 0x6c73616d5f6f7264ULL;    // ASCII "lsam_ord"
 inline uint64_t hash5(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j) {
   return mix64(mix64(mix64(seed ^ tag) + t) + ((k << 20) + j));
 }
@@ -253,6 +255,7 @@ struct oracle_ctx {
   std::vector<int64_t> t_x;
   std::vector<int64_t> ver_at_step;  // ver_at_step[s] = centre version that was current when step s started
   std::vector<double> loss, gn1, gn2;
+  std::vector<int32_t> active;       // which workers stepped at the last tick
   const float* eg1 = nullptr;
   const float* eg2 = nullptr;
 };
@@ -263,6 +266,8 @@ uint64_t oracle_mix64(uint64_t z) { return mix64(z); }
 uint64_t oracle_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j) { return hash5(seed, tag, t, k, j); }
 uint64_t oracle_tag_idx(void) { return TAG_IDX; }
 uint64_t oracle_tag_stale(void) { return TAG_STALE; }
+uint64_t oracle_tag_active(void) { return TAG_ACT; }
+uint64_t oracle_tag_order(void) { return TAG_ORD; }
 float oracle_bf16_round(float v) { return bf16_round(v); }
 int oracle_num_threads(void) {
 #ifdef _OPENMP
@@ -311,6 +316,7 @@ oracle_ctx* oracle_create(const oracle_config* cfg, const float* X, const void* 
   o->loss.assign(K, 0.0);
   o->gn1.assign(K, 0.0);
   o->gn2.assign(K, 0.0);
+  o->active.assign(K, 1);
   return o;
 }
 
@@ -338,8 +344,36 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
   if (c.model == ORACLE_MODEL_FLAT && (!o->eg1 || !o->eg2)) return 2;
   o->ver_at_step.push_back(o->t_y);  // centre version current when this tick starts
   const int64_t t = o->t;
+  // Asynchronous progress (Algorithm 2: each worker advances its own counter; the sync fires when the total count of
+  // iterations reaches n tau).  A worker is ready at this tick with probability active_num/256; ready workers are served
+  // in the order of a seeded key, and only as many as are still missing to n tau: the others wait, like the workers that
+  // block on the shared request queue while the servers run the distributed step.
+  {
+    int64_t done = 0;
+    for (int64_t c_ : o->t_x) done += c_;
+    const int64_t budget = (int64_t)K * c.tau - done;
+    if (budget <= 0) {  // the sync is due: every worker waits until oracle_couple() has run
+      o->ver_at_step.pop_back();
+      return 4;
+    }
+    const bool always = (c.active_num <= 0 || c.active_num >= 256);
+    std::vector<int> ready(K);
+    std::vector<uint64_t> key(K);
+    for (int k = 0; k < K; ++k) {
+      const uint64_t kid = (uint64_t)o->rid[k];
+      ready[k] = always || (hash5(c.seed, TAG_ACT, (uint64_t)t, kid, 0) % 256ULL) < (uint64_t)c.active_num;
+      key[k] = hash5(c.seed, TAG_ORD, (uint64_t)t, kid, 0);
+    }
+    for (int k = 0; k < K; ++k) {
+      int64_t rank = 0;  // ready workers served before worker k
+      for (int j = 0; j < K; ++j)
+        if (ready[j] && (key[j] < key[k] || (key[j] == key[k] && j < k))) rank += 1;
+      o->active[k] = (ready[k] && rank < budget) ? 1 : 0;
+    }
+  }
 #pragma omp parallel for schedule(dynamic, 1)
   for (int k = 0; k < K; ++k) {
+    if (!o->active[k]) continue;
     double* x = o->x.data() + (size_t)k * d;
     double* v = o->v.data() + (size_t)k * d;
     double* acc = o->acc.data() + (size_t)k * d;
@@ -475,6 +509,12 @@ int oracle_set_external_grads(oracle_ctx* o, const float* g1, const float* g2) {
   if (!o || o->cfg.model != ORACLE_MODEL_FLAT) return 1;
   o->eg1 = g1;
   o->eg2 = g2;
+  return 0;
+}
+
+int oracle_read_active(const oracle_ctx* o, int32_t* active) {
+  if (!o || !active) return 1;
+  std::memcpy(active, o->active.data(), sizeof(int32_t) * (size_t)o->cfg.K);
   return 0;
 }
 

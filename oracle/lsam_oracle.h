@@ -40,7 +40,7 @@ typedef struct {
   int32_t nesterov;     /* 1: x <- x - eta (G + mu v); 0: x <- x - eta v                     */
   int32_t tau;          /* sync period of Algorithm 2                                        */
   int32_t stale_max;    /* staleness drawn uniformly from [0, stale_max]                     */
-  int32_t reserved;
+  int32_t active_num;   /* a worker is ready at a tick with probability active_num/256; 0 or 256: always  */
   int64_t n_samples;    /* rows of X                                                         */
   int64_t flat_d;       /* FLAT model only: length of a replica's vector                     */
   uint64_t seed;
@@ -64,7 +64,8 @@ oracle_ctx* oracle_create(const oracle_config* cfg, const float* X, const void* 
                           const double* x0, const double* y0, const int32_t* replica_ids);
 void oracle_destroy(oracle_ctx*);
 
-/* One tick of the sampling loop of Algorithm 2 for every replica (eta, rho per call). */
+/* One tick of the sampling loop of Algorithm 2 (eta, rho per call): every ready worker steps once, but no more workers
+ * than are missing to n tau iterations.  Returns 4 and does nothing while a sync is due (call oracle_couple first). */
 int oracle_step(oracle_ctx*, double eta, double rho);
 /* 1 when the sync condition of Algorithm 2 holds (and at least one iterate was collected). */
 int oracle_should_couple(const oracle_ctx*);
@@ -86,6 +87,8 @@ int oracle_read_step_info(const oracle_ctx*, double* loss, double* gnorm1, doubl
 int oracle_read_grads(const oracle_ctx*, double* g1, double* g2, double* x_pert);
 /* FLAT model: gradients used by the next steps, [K, d] fp32, borrowed. */
 int oracle_set_external_grads(oracle_ctx*, const float* g1, const float* g2);
+/* Which workers stepped at the LAST tick ([K], 1 = stepped). */
+int oracle_read_active(const oracle_ctx*, int32_t* active);
 /* Counters: t (steps), t_y (centre version), t_x [K]. */
 int oracle_read_counters(const oracle_ctx*, int64_t* t, int64_t* t_y, int64_t* t_x);
 
@@ -100,6 +103,8 @@ uint64_t oracle_mix64(uint64_t z);
 uint64_t oracle_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j);
 uint64_t oracle_tag_idx(void);
 uint64_t oracle_tag_stale(void);
+uint64_t oracle_tag_active(void);
+uint64_t oracle_tag_order(void);
 float oracle_bf16_round(float v);
 int oracle_num_threads(void);
 

@@ -291,7 +291,7 @@ def test_update_matches_torch_sgd_when_no_pull():
     # lambda = 0: the sampler is a plain (Nesterov or heavy-ball) momentum step on g2; torch.optim.SGD states the same rule
     for nesterov in (1, 0):
         K, d = 2, 7
-        o, x0, y0, g1, g2 = _flat_oracle(K=K, d=d, mu=0.9, nesterov=nesterov, lam=0.0)
+        o, x0, y0, g1, g2 = _flat_oracle(K=K, d=d, mu=0.9, nesterov=nesterov, lam=0.0, tau=100)
         p = torch.tensor(x0.astype(np.float64), requires_grad=True)
         opt = torch.optim.SGD([p], lr=float(np.float32(0.03)), momentum=float(np.float32(0.9)), nesterov=bool(nesterov))
         for _ in range(5):
@@ -489,3 +489,75 @@ def test_invalid_configs_rejected():
     assert O.param_count(O.make_config(O.MODEL_RESMLP, widths=(3072, 4096, 4096, 4096, 4096, 1000), K=1, batch=1)) == 67027944
     assert O.param_count(O.make_config(O.MODEL_MLP, widths=(3072, 2048, 2048, 2048, 100), K=1, batch=1)) == 14891108
     assert O.param_count(O.make_config(O.MODEL_MLP, widths=(784, 1024, 10), K=1, batch=1)) == 814090
+
+
+# ------------------------------------------------------------------------------------------- asynchronous progress
+def _expected_mask(seed, t, K, active_num, budget):
+    """The stated rule, written out: ready if H_act mod 256 < active_num; served in (H_ord, k) order up to the budget."""
+    ta, to = O.lib().oracle_tag_active(), O.lib().oracle_tag_order()
+    ready = [O.hash5(seed, ta, t, k, 0) % 256 < active_num for k in range(K)]
+    order = sorted((O.hash5(seed, to, t, k, 0), k) for k in range(K) if ready[k])
+    served = {k for _, k in order[:max(budget, 0)]}
+    return np.array([1 if k in served else 0 for k in range(K)], dtype=np.int32)
+
+
+def test_async_progress_mask_counters_and_exact_trigger():
+    # Algorithm 2: per-worker counters t_x^(i) advance independently and the sync fires when their sum reaches n tau
+    K, tau, d, num, seed = 5, 3, 4, 128, 77
+    o, x0, y0, g1, g2 = _flat_oracle(K=K, d=d, tau=tau, lam=0.2, seed=seed, active_num=num, beta=0.0, eta_prime=1.0)
+    ready_hits, ready_trials, syncs, unequal = 0, 0, 0, False
+    window = []
+    for t in range(300):
+        before = o.read_state()
+        _, _, t_x = o.counters()
+        budget = K * tau - int(t_x.sum())
+        o.step(0.05, 0.05)
+        act = o.read_active()
+        np.testing.assert_array_equal(act, _expected_mask(seed, t, K, num, budget))
+        after = o.read_state()
+        _, _, t_x2 = o.counters()
+        np.testing.assert_array_equal(t_x2 - t_x, act)
+        assert t_x2.sum() <= K * tau
+        for k in range(K):
+            if act[k]:
+                window.append(after["x"][k].copy())
+            else:  # a waiting worker is untouched
+                np.testing.assert_array_equal(after["x"][k], before["x"][k])
+                np.testing.assert_array_equal(after["v"][k], before["v"][k])
+        if budget >= K:  # the budget did not bind: activity is the plain Bernoulli(num/256) draw
+            ready_hits += int(act.sum())
+            ready_trials += K
+        if o.should_couple():
+            assert t_x2.sum() == K * tau and len(window) == K * tau
+            unequal |= len(set(t_x2.tolist())) > 1
+            assert o.couple() == 0
+            # beta = 0, eta' = 1: the centre is the mean of exactly the n tau iterates collected, whoever produced them
+            np.testing.assert_allclose(o.read_params(-1), np.mean(window, axis=0), rtol=1e-12, atol=1e-14)
+            window = []
+            syncs += 1
+        else:
+            assert t_x2.sum() < K * tau
+    assert syncs > 20 and unequal
+    p = ready_hits / ready_trials
+    assert abs(p - 0.5) < 4 * np.sqrt(0.25 / ready_trials)
+
+
+def test_always_ready_is_the_lock_step_schedule_and_waiting_for_sync_is_an_error():
+    a, *_ = _flat_oracle(K=3, d=4, tau=2, lam=0.2, seed=5)
+    b, *_ = _flat_oracle(K=3, d=4, tau=2, lam=0.2, seed=5, active_num=256)
+    c, *_ = _flat_oracle(K=3, d=4, tau=2, lam=0.2, seed=5, active_num=0)
+    for t in range(6):
+        for o in (a, b, c):
+            o.step(0.05, 0.05)
+            assert (o.read_active() == 1).all()
+            if o.should_couple():
+                assert o.couple() == 0
+    np.testing.assert_array_equal(a.read_state()["x"], b.read_state()["x"])
+    np.testing.assert_array_equal(a.read_state()["x"], c.read_state()["x"])
+    a.step(0.05, 0.05)
+    a.step(0.05, 0.05)
+    assert a.should_couple()
+    x = a.read_state()["x"].copy()
+    assert O.lib().oracle_step(a._h, 0.05, 0.05) == 4  # the sync is due: nobody may step
+    np.testing.assert_array_equal(a.read_state()["x"], x)
+    assert a.counters()[0] == 8
