@@ -197,7 +197,7 @@ def make_cfg(G, w, flags=0):
     return G.make_config(w["model"], widths=w["widths"], K=w["K"], batch=max(w["B"], 1) if w["model"] != FLAT else 0,
                          gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
                          beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
-                         flat_d=w.get("d", 0), flags=flags)
+                         flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256))
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
@@ -216,11 +216,16 @@ def oracle_baseline(w, X, Y, x0_row, budget_s=20.0):
         g1 = (0.1 * rng.standard_normal((Ks, ds))).astype(np.float32)
         o = O.Oracle(cfg, None, None, x0, x0.mean(0))
         o.set_external_grads(g1, g1)
-        o.step(w["eta"], w["rho"])
+        def tick():
+            o.step(w["eta"], w["rho"])
+            if o.should_couple():
+                o.couple()
+
+        tick()
         t0 = time.perf_counter()
         steps = 3
         for _ in range(steps):
-            o.step(w["eta"], w["rho"])
+            tick()
         dt = (time.perf_counter() - t0) / steps
         return dict(value=36.0 * Ks * ds / dt / 1e9, unit="GB/s (36 B per element-replica)", cores=min(cores, Ks), kind="oracle",
                     sample=f"K={Ks} replicas, d={ds} of {d} elements, {steps} steps"), dt
@@ -236,6 +241,8 @@ def oracle_baseline(w, X, Y, x0_row, budget_s=20.0):
     t0 = time.perf_counter()
     for _ in range(steps):
         o.step(w["eta"], w["rho"])
+        if o.should_couple():
+            o.couple()
     dt = (time.perf_counter() - t0) / steps
     o.close()
     return dict(value=Ks * Bs / dt, unit="worker-samples/s", cores=min(cores, Ks), kind="oracle",
@@ -279,6 +286,7 @@ def main():
     ap.add_argument("--flat-d", type=int, default=None, help="c5 only: vector length of the sweep point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
+    ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
     if args.flat_d and w["model"] == FLAT:
@@ -287,6 +295,9 @@ def main():
     if args.replicas:
         w["K"] = args.replicas
         w["name"] += f" [K overridden to {args.replicas}]"
+    if args.active_num != 256:
+        w["active_num"] = args.active_num
+        w["name"] += f" [workers ready with probability {args.active_num}/256 per tick]"
     flat = w["model"] == FLAT
     metric = "fused_update_hbm_gbs" if flat else "lsam_worker_samples_per_s"
     unit = "GB/s" if flat else "worker-samples/s"
@@ -343,7 +354,12 @@ def main():
     clocks = ClockSampler(local)
     barrier()
     clocks.start()
+    def iterations_done():  # worker iterations since the context was created: every sync closes exactly K tau of them
+        _, t_y, t_x = ctx.counters()
+        return w["K"] * w["tau"] * t_y + int(t_x.sum())
+
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    it0 = iterations_done()
     e0.record(stream)
     for _ in range(args.steps):
         one_step()
@@ -351,6 +367,7 @@ def main():
     barrier()
     clk = clocks.stop()
     ms = e0.elapsed_time(e1)
+    worker_iters_per_step = (iterations_done() - it0) / args.steps  # = K in lock-step mode
     if not events_in_timed:
         launches_timed = ctx.launch_count() - launches0
         ctx.profile_enable(True)
@@ -365,7 +382,7 @@ def main():
         raise SystemExit("device status word is not clean after the timed region")
     ms = max_over_ranks(ms, world, dev)
     ms_step = ms / args.steps
-    units_step = (36.0 * w["K"] * d / 1e9) if flat else float(w["K"] * w["B"])
+    units_step = (36.0 * worker_iters_per_step * d / 1e9) if flat else float(worker_iters_per_step * w["B"])
     value = whole_job_value(world, units_step, ms_step)
 
     # ---- end to end through the C ABI with host buffers (minibatch H2D and loss D2H inside the timed region)

@@ -84,7 +84,8 @@ typedef struct {
   float lambda;       /* pull strength lambda (the rule lambda0/(eta tau) of Appendix D is the caller's) */
   float beta;         /* centre look-ahead factor beta (Section 4.2)                                */
   float eta_prime;    /* centre step size eta'                                                      */
-  float reserved;
+  int32_t active_num; /* asynchronous progress: a worker is ready at a tick with probability active_num/256;
+                         0 or 256 = every worker steps at every tick (lock-step)                     */
 } lsam_config;
 
 /* Unpadded parameter count d of one replica, or -1 if the configuration is invalid. */
@@ -103,8 +104,11 @@ size_t lsam_workspace_bytes(const lsam_config* cfg);
 int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const void* d_Y, const float* d_x0,
               const float* d_y0, void* d_workspace, size_t workspace_bytes, void* cuda_stream);
 
-/* One worker tick for all K replicas (sampling loop of Algorithm 2; Eq. 3; Algorithm 1, first update), with
- * the minibatch drawn by the seeded schedule.  eta and rho are per call, so any schedule (eta0/sqrt(t+1),
+/* One worker tick (sampling loop of Algorithm 2; Eq. 3; Algorithm 1, first update).  Every ready worker steps once,
+ * but no more workers than are still missing to K tau iterations since the last sync: ready workers are served in the
+ * order of a seeded key and the rest wait, as the workers of the paper block on the request queue while the servers run
+ * the distributed step (Appendix C.1).  While a sync is due the call returns LSAM_ERR_STATE and does nothing.
+ * The minibatch is drawn by the seeded schedule.  eta and rho are per call, so any schedule (eta0/sqrt(t+1),
  * rho0/sqrt(t+1), step decay) is the caller's.  Asynchronous on the context's stream. */
 int lsam_step(lsam_ctx* ctx, float eta, float rho);
 
@@ -146,6 +150,8 @@ int lsam_set_external_grads(lsam_ctx* ctx, const float* d_g1, const float* d_g2)
 int lsam_write_state(lsam_ctx* ctx, const float* d_x, const float* d_v, const float* d_y);
 /* Read back momentum buffers and accumulator for checkpointing: h_v [K, d], h_acc [d], h_gprev [d] (nullable). Synchronises. */
 int lsam_read_state(lsam_ctx* ctx, float* h_v, float* h_acc, float* h_gprev);
+/* Which workers stepped at the last tick: h_active [K], 1 = stepped (computed by the device schedule kernel).  Synchronises. */
+int lsam_read_active(lsam_ctx* ctx, int32_t* h_active);
 /* Counters: steps taken t, centre version t_y, per-worker t_x [K] (host, nullable). */
 int lsam_read_counters(const lsam_ctx* ctx, int64_t* t, int64_t* t_y, int64_t* h_t_x);
 /* Synchronise the stream and map the device status word to LSAM_OK / LSAM_ERR_NONFINITE / LSAM_ERR_TIMEOUT. */

@@ -22,7 +22,7 @@ PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "l
 EXPORTS = [
     "lsam_param_count", "lsam_workspace_bytes", "lsam_init", "lsam_step", "lsam_step_batch", "lsam_couple",
     "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads", "lsam_read_grads_replica",
-    "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_status",
+    "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_read_active", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
     "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static",
 ]
@@ -34,7 +34,7 @@ class LsamConfig(C.Structure):
         ("gemm_dtype", C.c_int32), ("gemm_impl", C.c_int32), ("nesterov", C.c_int32), ("tau", C.c_int32),
         ("stale_max", C.c_int32), ("flags", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_float), ("gamma", C.c_float), ("lam", C.c_float), ("beta", C.c_float),
-        ("eta_prime", C.c_float), ("reserved", C.c_float),
+        ("eta_prime", C.c_float), ("active_num", C.c_int32),
     ]
 
 
@@ -79,6 +79,7 @@ def lib():
     L.lsam_write_state.argtypes = [vp, vp, vp, vp]
     L.lsam_read_state.argtypes = [vp, vp, vp, vp]
     L.lsam_read_counters.argtypes = [vp, vp, vp, vp]
+    L.lsam_read_active.argtypes = [vp, vp]
     L.lsam_status.argtypes = [vp]
     L.lsam_profile_enable.argtypes = [vp, C.c_int]
     L.lsam_profile_read.argtypes = [vp, vp, vp]
@@ -97,7 +98,8 @@ def lib():
 
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=IMPL_AUTO, mu=0.9, nesterov=1,
-                gamma=1e-12, lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, flags=0):
+                gamma=1e-12, lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, flags=0,
+                active_num=256):
     c = LsamConfig()
     c.model = model
     widths = list(widths)
@@ -107,6 +109,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=
     c.K, c.batch, c.gemm_dtype, c.gemm_impl, c.nesterov, c.tau = int(K), int(batch), int(gemm_dtype), int(gemm_impl), int(nesterov), int(tau)
     c.stale_max, c.flags, c.n_samples, c.flat_d, c.seed = int(stale_max), int(flags), int(n_samples), int(flat_d), int(seed)
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = mu, gamma, lam, beta, eta_prime
+    c.active_num = int(active_num)
     return c
 
 
@@ -265,6 +268,11 @@ class Lsam:
         gprev = np.empty(self.d, dtype=np.float32)
         self._check(lib().lsam_read_state(self._h, _np_ptr(v), _np_ptr(acc), _np_ptr(gprev)))
         return dict(v=v, acc=acc, gprev=gprev)
+
+    def read_active(self):
+        a = np.zeros(self.K, dtype=np.int32)
+        self._check(lib().lsam_read_active(self._h, _np_ptr(a)))
+        return a
 
     def counters(self):
         t = np.zeros(1, dtype=np.int64)

@@ -23,6 +23,8 @@ __host__ __device__ inline uint64_t mix64(uint64_t z) {
 }
 constexpr uint64_t kTagIdx = 0x6c73616d5f696478ULL;    // "lsam_idx"
 constexpr uint64_t kTagStale = 0x6c73616d5f73746cULL;  // "lsam_stl"
+constexpr uint64_t kTagAct = 0x6c73616d5f616374ULL;    // "lsam_act"
+constexpr uint64_t kTagOrd = 0x6c73616d5f6f7264ULL;    // "lsam_ord"
 __host__ __device__ inline uint64_t schedule_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j) {
   return mix64(mix64(mix64(seed ^ tag) + t) + ((k << 20) + j));
 }
@@ -41,6 +43,11 @@ __device__ inline float warp_sum(float v) {
   return v;
 }
 __device__ inline double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ inline int warp_sum(int v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;

@@ -183,7 +183,7 @@ template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
-                    int Z, TcEpi ep, int* __restrict__ status) {
+                    int Z, TcEpi ep, int* __restrict__ status, const int32_t* __restrict__ active) {
   constexpr int STAGES = tc_stages<BLOCK_N>();
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
   constexpr int B_BYTES = BLOCK_N * kTcBlockK * 2;
@@ -228,6 +228,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       bool ok = true;
       for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
         const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
+        if (active != nullptr && !active[z]) continue;  // waiting replica: all three roles skip the same tiles
         const int m0 = mt * kTcBlockM, n0 = nt * BLOCK_N;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -261,6 +262,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       uint32_t aph = 0;
       bool ok = true;
       for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+        if (active != nullptr && !active[(int)(t / ((int64_t)n_tiles * m_tiles))]) continue;
         if (!tc::mbar_wait(&acc_empty[as], aph ^ 1u, abort_flag)) { ok = false; break; }
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BLOCK_N);
@@ -296,6 +298,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     bool ok = true;
     for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
       const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
+      if (active != nullptr && !active[z]) continue;
       const int m = mt * kTcBlockM + quad * 32 + lane;
       const int n0 = nt * BLOCK_N;
       if (!tc::mbar_wait(&acc_full[as], aph, abort_flag)) { ok = false; break; }
@@ -479,6 +482,7 @@ struct TcGemm {
 };
 
 struct TcPlan {
+  const int32_t* active = nullptr;  // per-tick mask of the replicas that step (nullptr: all)
   int Z = 0, B = 0, n_layers = 0, sms = 148;
   int* status = nullptr;
   int64_t* launches = nullptr;
@@ -607,7 +611,7 @@ inline int tc_launch_one(const TcPlan& P, const TcGemm& g, cudaStream_t stream) 
   }
   const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, kTcBlockM) * ceil_div(g.N, BLOCK_N);
   const int grid = (int)(tiles < P.sms ? tiles : P.sms);
-  kern<<<grid, kTcThreads, tc_smem_bytes<BLOCK_N>(), stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status);
+  kern<<<grid, kTcThreads, tc_smem_bytes<BLOCK_N>(), stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status, P.active);
   return cudaPeekAtLastError() == cudaSuccess ? 0 : 1;
 }
 

@@ -4,10 +4,12 @@
 // buffer is carved from the caller's workspace.
 #include "lsam.h"
 
+#include <algorithm>
 #include <cstdio>
 #include <cstring>
 #include <mutex>
 #include <string>
+#include <utility>
 #include <vector>
 
 #include "common.cuh"
@@ -49,6 +51,7 @@ bool plan(const lsam_config& c, Layout& L) {
   if (c.gemm_dtype != LSAM_GEMM_FP32 && c.gemm_dtype != LSAM_GEMM_BF16) return false;
   if (c.gemm_impl < LSAM_IMPL_AUTO || c.gemm_impl > LSAM_IMPL_TCGEN05) return false;
   if (!(c.gamma > 0.f)) return false;
+  if (c.active_num < 0 || c.active_num > 256) return false;
   const bool bf = c.gemm_dtype == LSAM_GEMM_BF16;
   L.seg.n = 0;
   if (c.model == LSAM_MODEL_FLAT) {
@@ -171,6 +174,8 @@ struct lsam_ctx {
   std::vector<int> ver_at_step;
   bool have_prev = false;
   bool use_tc = false;
+  bool async_on = false;              // 0 < active_num < 256: unequal worker progress
+  std::vector<int32_t> active_host;   // host mirror of the last tick's mask (drives the counters t_x)
   int64_t launches = 0;
   Profiler prof;
   std::string err;
@@ -190,6 +195,9 @@ struct lsam_ctx {
   int32_t* stale() const { return at<int32_t>(L.sched); }
   int32_t* ver() const { return at<int32_t>(L.sched) + cfg.K; }
   int32_t* slot() const { return at<int32_t>(L.sched) + 2 * cfg.K; }
+  int32_t* active_buf() const { return at<int32_t>(L.sched) + 3 * cfg.K; }
+  // per-tick mask of the workers that step; nullptr in lock-step mode (every worker steps every tick)
+  const int32_t* act() const { return async_on ? active_buf() : nullptr; }
   int32_t* sched_scratch() const { return at<int32_t>(L.sched) + 4 * cfg.K; }
   float* yslot(int64_t version) const { return at<float>(L.yring) + (size_t)(version % L.ring) * L.ld; }
 
@@ -244,14 +252,14 @@ int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, 
   if (c->use_tc) {
     // tensor-core path: the weight- and bias-gradient kernels of the pass just run have left the sums of squares of
     // all their blocks in the partial slots; only the fixed-order final sum remains
-    LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status()));
+    LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act()));
     return LSAM_OK;
   }
   dim3 grid((unsigned)ceil_div(n, vec4 ? norm_chunk<4>() : norm_chunk<1>()), c->cfg.K);
   if ((int64_t)grid.x > nch) return c->fail(LSAM_ERR_WORKSPACE, "norm: partial-sum buffer too small");
-  if (vec4) LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<4><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch));
-  else LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<1><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch));
-  LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)grid.x, rho, c->cfg.gamma, norm_out, scale_out, c->status()));
+  if (vec4) LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<4><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch, c->act()));
+  else LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<1><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch, c->act()));
+  LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)grid.x, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act()));
   return LSAM_OK;
 }
 
@@ -260,13 +268,14 @@ int launch_perturb(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec
   TP* xt = c->at<TP>(c->L.xop);
   const int64_t per = (int64_t)kPertThreads * kPertIter * (vec4 ? 4 : 1);
   dim3 grid((unsigned)ceil_div(n, per), c->cfg.K);
-  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld));
-  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld));
+  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
+  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
   return LSAM_OK;
 }
 
 int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float eta) {
   UpdateArgs a;
+  a.active = c->act();
   a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
   a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
   a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
@@ -285,7 +294,7 @@ int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4
   return LSAM_OK;
 }
 
-int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot) {
+int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot, int64_t budget, int32_t* active) {
   VerHist h;
   for (int s = 0; s < 16; ++s) {
     const int64_t ts = t - s > 0 ? t - s : 0;
@@ -294,15 +303,28 @@ int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_
   const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
   LAUNCH(c, LSAM_PROF_SCHEDULE,
          schedule_kernel<<<c->cfg.K, 128, 0, c->stream>>>(c->cfg.seed, (uint64_t)t, flat ? 1 : c->cfg.n_samples, flat ? 0 : c->cfg.batch,
-                                                           c->cfg.stale_max, h, c->L.ring, flat ? nullptr : idx, stale, ver, slot));
+                                                           c->cfg.stale_max, h, c->L.ring, flat ? nullptr : idx, stale, ver, slot,
+                                                           c->cfg.K, c->cfg.active_num, budget, active));
   return LSAM_OK;
+}
+
+// Host statement of the same rule as schedule_kernel: which workers step at tick t given the remaining budget.
+void host_active_mask(const lsam_config& cfg, int64_t t, int64_t budget, std::vector<int32_t>& mask) {
+  const int K = cfg.K;
+  mask.assign(K, 0);
+  std::vector<std::pair<uint64_t, int>> ready;
+  for (int k = 0; k < K; ++k)
+    if ((schedule_hash(cfg.seed, kTagAct, (uint64_t)t, (uint64_t)k, 0) % 256ULL) < (uint64_t)cfg.active_num)
+      ready.push_back({schedule_hash(cfg.seed, kTagOrd, (uint64_t)t, (uint64_t)k, 0), k});
+  std::sort(ready.begin(), ready.end());
+  for (size_t r = 0; r < ready.size() && (int64_t)r < budget; ++r) mask[ready[r].second] = 1;
 }
 
 // ---- SIMT GEMM launches in logical coordinates
 template <typename TA, typename TB, class Epi>
 int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N, int Kd, const Epi& epi) {
   dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), c->cfg.K);
-  LAUNCH(c, cls, gemm_simt_kernel<TA, TB, Epi><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi));
+  LAUNCH(c, cls, gemm_simt_kernel<TA, TB, Epi><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));
   return LSAM_OK;
 }
 
@@ -341,15 +363,15 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
   const int C = L.layers[nl - 1].out;
   int cur = 0;
   LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
-      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status()));
-  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out));
+      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act()));
+  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
   // backward
   for (int l = nl - 1; l >= 0; --l) {
     const LayerInfo& li = L.layers[l];
     const T* dz = c->at<T>(L.dz[cur]);
     const T* a_in = c->at<T>(L.act[l]);
     LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad,
-        c->use_tc ? c->at<float>(L.partial) : nullptr, L.nchunks, c->use_tc ? c->tc.bias_slot0[l] : 0));
+        c->use_tc ? c->at<float>(L.partial) : nullptr, L.nchunks, c->use_tc ? c->tc.bias_slot0[l] : 0, c->act()));
     if (c->use_tc) {
       int trc = 0;
       LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream));
@@ -385,7 +407,7 @@ int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out) {
   if (cfg.model == LSAM_MODEL_LSQ) {
     const float* P = perturbed ? c->at<float>(c->L.xop) : c->x();
     LAUNCH(c, LSAM_PROF_LSQ_GRAD, lsq_grad_kernel<<<cfg.K, 256, sizeof(float) * cfg.batch, c->stream>>>(
-        c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, cfg.widths[0], c->g(), c->L.ld, loss_out));
+        c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, cfg.widths[0], c->g(), c->L.ld, loss_out, c->act()));
     return LSAM_OK;
   }
   if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out);
@@ -414,18 +436,23 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
   const bool flat = cfg.model == LSAM_MODEL_FLAT;
   if (flat && (!c->eg1 || !c->eg2)) return c->fail(LSAM_ERR_STATE, "FLAT model: call lsam_set_external_grads first");
   int rc;
+  int64_t done = 0;
+  for (int64_t v : c->t_x) done += v;
+  const int64_t budget = (int64_t)cfg.K * cfg.tau - done;  // iterations still missing to n tau (Algorithm 2, sync trigger)
+  if (budget <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
   c->ver_at_step.push_back((int)c->t_y);  // centre version current when this tick starts
-  if ((rc = launch_schedule(c, c->t, c->idx(), c->stale(), c->ver(), c->slot())) != LSAM_OK) return rc;
+  if (c->async_on) host_active_mask(cfg, c->t, budget, c->active_host);
+  if ((rc = launch_schedule(c, c->t, c->idx(), c->stale(), c->ver(), c->slot(), budget, c->async_on ? c->active_buf() : nullptr)) != LSAM_OK) return rc;
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   if (!flat && gather) {
     if (cfg.model == LSAM_MODEL_LSQ) {
-      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], cfg.widths[0], c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], cfg.widths[0], c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), cfg.batch, c->act()));
     } else {
       dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
       if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
       else
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status()));
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
     }
   }
   const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
@@ -447,7 +474,7 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
     if ((rc = launch_norm(c, g2, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
   // fused worker update
   if ((rc = launch_update(c, g2, ldg, n, vec4, eta)) != LSAM_OK) return rc;
-  for (auto& tx : c->t_x) tx += 1;
+  for (int k = 0; k < cfg.K; ++k) c->t_x[k] += c->async_on ? c->active_host[k] : 1;
   c->t += 1;
   return LSAM_OK;
 }
@@ -490,6 +517,8 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   c->X = reinterpret_cast<const float*>(d_X);
   c->Y = reinterpret_cast<const uint32_t*>(d_Y);
   c->t_x.assign(cfg->K, 0);
+  c->async_on = cfg->active_num > 0 && cfg->active_num < 256;
+  c->active_host.assign(cfg->K, 1);
   auto bail = [&](int code) { delete c; return code; };
   // tensor-core path: decided once per context
   const bool mlp = cfg->model == LSAM_MODEL_MLP || cfg->model == LSAM_MODEL_RESMLP;
@@ -511,6 +540,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     b.status = c->status();
     b.ldb = L.ldb;
     b.partial = c->at<float>(L.partial); b.ld_partial = L.nchunks;
+    c->tc.active = c->act();
     std::vector<TcLayer> tl;
     for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
     std::string why;
@@ -540,9 +570,9 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   if (!lsq) {
     dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
     if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status()));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
     else
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status()));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
   }
   int rc = step_common(c, eta, rho, false);
   if (rc != LSAM_OK) return rc;
@@ -591,7 +621,7 @@ int lsam_read_schedule(lsam_ctx* c, int64_t t, int32_t* h_idx, int32_t* h_stale,
   if (h_ver && t >= (int64_t)c->ver_at_step.size()) return c->fail(LSAM_ERR_STATE, "lsam_read_schedule: centre version of a future step");
   const int K = c->cfg.K;
   int32_t* s = c->sched_scratch();
-  int rc = launch_schedule(c, t, c->idx_scratch(), s, s + K, s + 2 * K);
+  int rc = launch_schedule(c, t, c->idx_scratch(), s, s + K, s + 2 * K, 0, nullptr);
   if (rc != LSAM_OK) return rc;
   if (h_idx && c->cfg.model != LSAM_MODEL_FLAT)
     LSAM_CUDA(c, cudaMemcpyAsync(h_idx, c->idx_scratch(), 4 * (size_t)K * c->cfg.batch, cudaMemcpyDeviceToHost, c->stream));
@@ -703,6 +733,17 @@ int lsam_read_counters(const lsam_ctx* c, int64_t* t, int64_t* t_y, int64_t* h_t
   return LSAM_OK;
 }
 
+int lsam_read_active(lsam_ctx* c, int32_t* h_active) {
+  if (!c || !h_active) return LSAM_ERR_INVALID;
+  if (!c->async_on) {
+    for (int k = 0; k < c->cfg.K; ++k) h_active[k] = 1;
+    return LSAM_OK;
+  }
+  LSAM_CUDA(c, cudaMemcpyAsync(h_active, c->active_buf(), sizeof(int32_t) * c->cfg.K, cudaMemcpyDeviceToHost, c->stream));
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LSAM_OK;
+}
+
 int lsam_status(lsam_ctx* c) {
   if (!c) return LSAM_ERR_INVALID;
   int h = 0;
@@ -802,9 +843,9 @@ extern "C" int lsam_row_norms_static(const float* d_g, int64_t ld, int64_t n, in
   // Every slot the second pass reads (k * nch + c, c < nch) is written by the first pass of this same call,
   // so the previous call's contents never need clearing.
   dim3 grid((unsigned)nch, (unsigned)K);
-  if (vec4) sumsq_partial_kernel<4><<<grid, kNormThreads, 0, stream>>>(d_g, ld, n, partial, nch);
-  else sumsq_partial_kernel<1><<<grid, kNormThreads, 0, stream>>>(d_g, ld, n, partial, nch);
-  norm_finalize_kernel<<<K, 256, 0, stream>>>(partial, nch, nch, 0.f, 1.f, d_norm, nullptr, nullptr);
+  if (vec4) sumsq_partial_kernel<4><<<grid, kNormThreads, 0, stream>>>(d_g, ld, n, partial, nch, nullptr);
+  else sumsq_partial_kernel<1><<<grid, kNormThreads, 0, stream>>>(d_g, ld, n, partial, nch, nullptr);
+  norm_finalize_kernel<<<K, 256, 0, stream>>>(partial, nch, nch, 0.f, 1.f, d_norm, nullptr, nullptr, nullptr);
   const cudaError_t e = cudaPeekAtLastError();
   if (e != cudaSuccess) {
     char msg[256];

@@ -11,8 +11,10 @@ namespace lsam {
 template <typename TA>
 __global__ void __launch_bounds__(128)
 gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx,
-              int64_t n_samples, int in, int ld, TA* __restrict__ xb, uint32_t* __restrict__ yb, int* __restrict__ status) {
+              int64_t n_samples, int in, int ld, TA* __restrict__ xb, uint32_t* __restrict__ yb, int* __restrict__ status,
+              int B, const int32_t* __restrict__ active) {
   const int64_t r = blockIdx.x;
+  if (active != nullptr && !active[r / B]) return;
   int64_t s = idx[r];
   if (s < 0 || s >= n_samples) {
     if (threadIdx.x == 0) atomicOr(status, STATUS_BAD_INDEX);
@@ -31,8 +33,10 @@ gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const
 template <typename TA>
 __global__ void __launch_bounds__(256)
 gather_t_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx, int64_t n_samples,
-                int B, int in, int ldb, TA* __restrict__ xt, uint32_t* __restrict__ yb, int* __restrict__ status) {
+                int B, int in, int ldb, TA* __restrict__ xt, uint32_t* __restrict__ yb, int* __restrict__ status,
+                const int32_t* __restrict__ active) {
   __shared__ float tile[32][33];
+  if (active != nullptr && !active[blockIdx.z]) return;
   const int k = blockIdx.z, i0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
   for (int r = threadIdx.y; r < 32; r += 8) {
     const int b = b0 + r, i = i0 + threadIdx.x;
@@ -123,8 +127,9 @@ struct GemmOperand { const void* p; int64_t sz, sr, sk; };  // element (z, r, kk
 
 template <typename TA_, typename TB_, class Epi>
 __global__ void __launch_bounds__(256)
-gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi) {
+gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, const int32_t* __restrict__ active) {
   constexpr int BM = 64, BN = 64, BK = 16;
+  if (active != nullptr && !active[blockIdx.z]) return;  // a waiting replica
   __shared__ float As[BK][BM + 4];
   __shared__ float Bs[BK][BN + 4];
   const int z = blockIdx.z;
@@ -189,8 +194,9 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi) {
 template <typename TA>
 __global__ void __launch_bounds__(256)
 softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int B, int C, int ldb,
-                  TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status) {
+                  TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status, const int32_t* __restrict__ active) {
   __shared__ float red[8][33];
+  if (active != nullptr && !active[blockIdx.y]) return;
   const int b = blockIdx.x * 32 + threadIdx.x, cg = threadIdx.y, k = blockIdx.y;
   const bool live = b < B;
   const float* lg = logits + (int64_t)k * C * ldb + (live ? b : 0);
@@ -227,8 +233,9 @@ softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ 
 }
 
 // loss[k] = mean over the minibatch of rowloss[k][b], samples added in ascending order.  grid K, block 32.
-__global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float* __restrict__ loss) {
+__global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float* __restrict__ loss, const int32_t* __restrict__ active) {
   const int k = blockIdx.x;
+  if (active != nullptr && !active[k]) return;
   if (threadIdx.x == 0) {
     double s = 0.0;
     for (int b = 0; b < B; ++b) s += (double)rowloss[(int64_t)k * B + b];
@@ -244,8 +251,9 @@ __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float
 template <typename TA>
 __global__ void __launch_bounds__(256)
 bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off,
-                 float* __restrict__ partial, int64_t ld_partial, int slot0) {
+                 float* __restrict__ partial, int64_t ld_partial, int slot0, const int32_t* __restrict__ active) {
   __shared__ float sq[8];
+  if (active != nullptr && !active[blockIdx.y]) return;
   const int w = threadIdx.x >> 5, o = blockIdx.x * 8 + w;
   const int z = blockIdx.y, lane = threadIdx.x & 31;
   float s = 0.f;
@@ -272,9 +280,11 @@ bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __re
 // xb [K, B, in] gathered minibatch, yb [K, B] targets, w = params (row stride ld_p).  Dynamic smem: B floats.
 __global__ void __launch_bounds__(256)
 lsq_grad_kernel(const float* __restrict__ xb, const float* __restrict__ yb, const float* __restrict__ params,
-                int64_t ld_p, int B, int in, float* __restrict__ g, int64_t ld_g, float* __restrict__ loss) {
+                int64_t ld_p, int B, int in, float* __restrict__ g, int64_t ld_g, float* __restrict__ loss,
+                const int32_t* __restrict__ active) {
   extern __shared__ float res[];
   const int k = blockIdx.x;
+  if (active != nullptr && !active[k]) return;
   const float* w = params + (int64_t)k * ld_p;
   const float* a = xb + (int64_t)k * B * in;
   const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;

@@ -10,10 +10,15 @@ namespace lsam {
 // hist.v[s] = centre version that was current when step t - s started (s = 0..15), clamped at step 0.
 struct VerHist { int v[16]; };
 
-// grid K, any block size.  idx [K, B]; stale, ver, slot [K].  slot = ring slot holding the version read.
-__global__ void schedule_kernel(uint64_t seed, uint64_t t, int64_t n_samples, int B, int stale_max, VerHist hist,
-                                int ring, int32_t* __restrict__ idx, int32_t* __restrict__ stale,
-                                int32_t* __restrict__ ver, int32_t* __restrict__ slot) {
+// grid K, block 128.  idx [K, B]; stale, ver, slot [K].  slot = ring slot holding the version read.
+// active (nullable) [K]: asynchronous progress.  Worker k is ready at this tick when H_act mod 256 < active_num; ready
+// workers are served in the order of (H_ord, k) and only the first `budget` of them step (budget = n tau minus the
+// iterations already counted since the last sync); active[k] = 1 for those.
+__global__ void __launch_bounds__(128)
+schedule_kernel(uint64_t seed, uint64_t t, int64_t n_samples, int B, int stale_max, VerHist hist, int ring,
+                int32_t* __restrict__ idx, int32_t* __restrict__ stale, int32_t* __restrict__ ver, int32_t* __restrict__ slot,
+                int K, int active_num, int64_t budget, int32_t* __restrict__ active) {
+  __shared__ int red[4];
   const uint64_t k = blockIdx.x;
   if (idx != nullptr)
     for (int j = threadIdx.x; j < B; j += blockDim.x)
@@ -24,6 +29,18 @@ __global__ void schedule_kernel(uint64_t seed, uint64_t t, int64_t n_samples, in
     if (stale) stale[k] = s;
     if (ver) ver[k] = u;
     if (slot) slot[k] = u >= 0 ? u % ring : 0;
+  }
+  if (active != nullptr) {
+    const bool ready_k = (schedule_hash(seed, kTagAct, t, k, 0) % 256ULL) < (uint64_t)active_num;
+    const uint64_t key_k = schedule_hash(seed, kTagOrd, t, k, 0);
+    int cnt = 0;  // ready workers served before worker k
+    for (int j = threadIdx.x; j < K; j += blockDim.x) {
+      const bool ready_j = (schedule_hash(seed, kTagAct, t, (uint64_t)j, 0) % 256ULL) < (uint64_t)active_num;
+      const uint64_t key_j = schedule_hash(seed, kTagOrd, t, (uint64_t)j, 0);
+      cnt += (ready_j && (key_j < key_k || (key_j == key_k && (uint64_t)j < k))) ? 1 : 0;
+    }
+    const int rank = block_sum<int>(cnt, red);
+    if (threadIdx.x == 0) active[k] = (ready_k && (int64_t)rank < budget) ? 1 : 0;
   }
 }
 
@@ -37,9 +54,11 @@ __host__ __device__ constexpr int64_t norm_chunk() { return (int64_t)kNormThread
 
 template <int VEC>
 __global__ void __launch_bounds__(kNormThreads)
-sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float* __restrict__ partial, int64_t nchunks) {
+sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float* __restrict__ partial, int64_t nchunks,
+                     const int32_t* __restrict__ active) {
   __shared__ float red[kNormThreads / 32];
   const int k = blockIdx.y;
+  if (active != nullptr && !active[k]) return;  // a waiting worker (block-uniform)
   const int64_t base = (int64_t)blockIdx.x * norm_chunk<VEC>();
   const float* row = g + (int64_t)k * ldg;
   float s = 0.f;
@@ -68,9 +87,11 @@ sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float*
 // grid K, block 256; partial has row stride nchunks, of which the first nused are summed.  A non-finite norm raises STATUS_NONFINITE and leaves scale = 0 (no perturbation).
 __global__ void __launch_bounds__(256)
 norm_finalize_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t nused, float rho, float gamma,
-                     float* __restrict__ norm_out, float* __restrict__ scale_out, int* __restrict__ status) {
+                     float* __restrict__ norm_out, float* __restrict__ scale_out, int* __restrict__ status,
+                     const int32_t* __restrict__ active) {
   __shared__ double red[8];
   const int k = blockIdx.x;
+  if (active != nullptr && !active[k]) return;
   double s = 0.0;
   for (int64_t c = threadIdx.x; c < nused; c += blockDim.x) s += (double)partial[(int64_t)k * nchunks + c];
   const double tot = block_sum<double>(s, red);
@@ -97,8 +118,9 @@ constexpr int kPertIter = 4;
 template <int VEC, typename TP>
 __global__ void __launch_bounds__(kPertThreads)
 perturb_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ g, int64_t ldg, int64_t n,
-               const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt) {
+               const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active) {
   const int k = blockIdx.y;
+  if (active != nullptr && !active[k]) return;
   const float sc = scale[k];
   const int64_t base = (int64_t)blockIdx.x * ((int64_t)kPertThreads * VEC * kPertIter);
   const float* xr = x + (int64_t)k * ldx;
@@ -151,6 +173,7 @@ struct UpdateArgs {
   const float* g;      // [K, ldg]
   const float* yring;  // [ring, ld]
   const int32_t* slot; // [K] ring slot of the centre version read by replica k
+  const int32_t* active;  // nullable [K]: replicas with 0 wait this tick and are left untouched
   float* acc;          // [ld]
   void* xop;           // [K, ld] operand copy (or nullptr)
   int64_t ld, ldg, n;
@@ -168,19 +191,28 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     // software pipeline over the replicas: the four loads of replica k + 1 are issued before the arithmetic and the
     // stores of replica k, so that twice as many bytes are in flight per thread
-    float4 gv = __ldcs(reinterpret_cast<const float4*>(a.g + j));
-    float4 xv = *reinterpret_cast<const float4*>(a.x + j);
-    float4 vv = *reinterpret_cast<const float4*>(a.v + j);
-    float4 yv = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[0] * a.ld + j));
-    for (int k = 0; k < a.K; ++k) {
+    int k = 0;
+    if (a.active != nullptr)
+      while (k < a.K && !a.active[k]) ++k;  // first replica that steps at this tick
+    float4 gv = make_float4(0.f, 0.f, 0.f, 0.f), xv = gv, vv = gv, yv = gv;
+    if (k < a.K) {
+      gv = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)k * a.ldg + j));
+      xv = *reinterpret_cast<const float4*>(a.x + (int64_t)k * a.ld + j);
+      vv = *reinterpret_cast<const float4*>(a.v + (int64_t)k * a.ld + j);
+      yv = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[k] * a.ld + j));
+    }
+    while (k < a.K) {
       const int64_t o = (int64_t)k * a.ld + j;
+      int kn = k + 1;
+      if (a.active != nullptr)
+        while (kn < a.K && !a.active[kn]) ++kn;
       float4 gn = gv, xn = xv, vn = vv, yn = yv;
-      if (k + 1 < a.K) {
-        const int64_t on = o + a.ld;
-        gn = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)(k + 1) * a.ldg + j));
+      if (kn < a.K) {
+        const int64_t on = (int64_t)kn * a.ld + j;
+        gn = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)kn * a.ldg + j));
         xn = *reinterpret_cast<const float4*>(a.x + on);
         vn = *reinterpret_cast<const float4*>(a.v + on);
-        yn = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[k + 1] * a.ld + j));
+        yn = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[kn] * a.ld + j));
       }
       float G;
 #define LSAM_UPD(c)                                                         \
@@ -202,6 +234,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
         }
       }
       gv = gn; xv = xn; vv = vn; yv = yn;
+      k = kn;
     }
     float4 av = *reinterpret_cast<const float4*>(a.acc + j);
     av.x += s.x; av.y += s.y; av.z += s.z; av.w += s.w;
@@ -209,6 +242,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
   } else {
     float s = 0.f;
     for (int k = 0; k < a.K; ++k) {
+      if (a.active != nullptr && !a.active[k]) continue;
       const int64_t o = (int64_t)k * a.ld + j;
       const float gv = a.g[(int64_t)k * a.ldg + j];
       float xv = a.x[o], vv = a.v[o];

@@ -276,6 +276,81 @@ def test_deterministic_repeat():
     np.testing.assert_array_equal(outs[0][1], outs[1][1])
 
 
+# ------------------------------------------------------------------------------------------------ asynchronous progress
+@pytest.mark.parametrize("kind", ["flat", "lsq", "mlp_fp32", "mlp_bf16_tcgen05"])
+def test_async_progress_masks_bit_exact_and_trajectory(kind):
+    # unequal worker progress (Algorithm 2): the per-tick mask and the counters are integers and must agree exactly;
+    # waiting replicas must be left untouched bit for bit; the trajectory stays within the usual tolerance
+    hp = dict(tau=3, lam=0.3, seed=31, stale_max=2, active_num=150)
+    if kind == "flat":
+        K, d = 8, 1000
+        x0, y0, g1, g2 = synth.flat_problem(K, d, seed=2)
+        p = Pair(G.MODEL_FLAT, K=K, flat_d=d, x0=x0, y0=y0, **hp)
+        p.set_external_grads(g1, g2)
+        tol = TOL_TRAJ_FP32
+    elif kind == "lsq":
+        K = 6
+        X, y, _ = synth.least_squares_data(300, 24, seed=3)
+        x0 = np.random.default_rng(4).standard_normal((K, 24)).astype(np.float32)
+        p = Pair(G.MODEL_LSQ, widths=(24,), K=K, batch=16, X=X, Y=y, x0=x0, y0=x0.mean(0), **hp)
+        tol = TOL_TRAJ_FP32
+    elif kind == "mlp_fp32":
+        K = 5
+        p = _mlp_pair(G.MODEL_MLP, (40, 64, 48, 6), K, 24, n=300, dtype=G.GEMM_FP32, jitter=0.01, **hp)
+        tol = TOL_TRAJ_FP32
+    else:
+        K = 5
+        p = _mlp_pair(G.MODEL_RESMLP, (64, 128, 128, 16), K, 48, n=300, dtype=G.GEMM_BF16, impl=G.IMPL_TCGEN05, jitter=0.01, **hp)
+        assert p.gpu.uses_tcgen05()
+        tol = TOL_TRAJ_BF16
+    waited = stepped = 0
+    for t in range(24):
+        before = p.gpu.read_all_params()
+        p.step(0.03, 0.05)
+        oa, ga = p.oracle.read_active(), p.gpu.read_active()
+        np.testing.assert_array_equal(ga, oa)
+        ot, oty, otx = p.oracle.counters()
+        gt, gty, gtx = p.gpu.counters()
+        assert (ot, oty) == (gt, gty) and (otx == gtx).all()
+        after = p.gpu.read_all_params()
+        for k in range(K):
+            if ga[k]:
+                stepped += 1
+                assert not np.array_equal(after[k], before[k])
+            else:
+                waited += 1
+                np.testing.assert_array_equal(after[k], before[k])
+        p.couple_if_due()
+    assert waited > 10 and stepped > 10
+    e = p.errors()
+    e.pop("acc")
+    ev = e.pop("v")
+    assert ev <= 10 * tol
+    _assert_all(e, tol, f"async {kind}")
+    assert p.gpu.status() == 0
+    # stepping while the sync is due is refused on both sides
+    p.close()
+
+
+def test_step_refused_while_sync_is_due():
+    import torch
+
+    cfg = G.make_config(G.MODEL_FLAT, K=2, flat_d=8, tau=1)
+    x0 = torch.zeros(2, 8, device="cuda")
+    g = torch.ones(2, 8, device="cuda")
+    gpu = G.Lsam(cfg, None, None, x0, torch.zeros(8, device="cuda"))
+    gpu.set_external_grads(g, g)
+    gpu.step(0.1, 0.1)
+    assert gpu.should_couple()
+    with pytest.raises(G.LsamError) as ei:
+        gpu.step(0.1, 0.1)
+    assert ei.value.code == G.LSAM_ERR_STATE
+    assert gpu.couple() == 0
+    gpu.step(0.1, 0.1)
+    assert gpu.counters()[0] == 2
+    gpu.close()
+
+
 # ------------------------------------------------------------------------------------------------ errors (host-side only)
 def test_error_paths():
     import torch
