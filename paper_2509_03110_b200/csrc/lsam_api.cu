@@ -323,8 +323,15 @@ void host_active_mask(const lsam_config& cfg, int64_t t, int64_t budget, std::ve
 // ---- SIMT GEMM launches in logical coordinates
 template <typename TA, typename TB, class Epi>
 int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N, int Kd, const Epi& epi) {
-  dim3 grid((unsigned)ceil_div(N, 64), (unsigned)ceil_div(M, 64), c->cfg.K);
-  LAUNCH(c, cls, gemm_simt_kernel<TA, TB, Epi><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));
+  dim3 grid((unsigned)ceil_div(N, kSimtBN), (unsigned)ceil_div(M, kSimtBM), c->cfg.K);
+  // every operand of the classifier is contiguous either along its rows or along the contraction index
+  const bool a_mc = (A.sr == 1), b_nc = (B.sr == 1);
+  if (!a_mc && A.sk != 1) return c->fail(LSAM_ERR_INVALID, "SIMT GEMM: operand A has no unit stride");
+  if (!b_nc && B.sk != 1) return c->fail(LSAM_ERR_INVALID, "SIMT GEMM: operand B has no unit stride");
+#define LSAM_SIMT(AM, BN_) LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()))
+  if (a_mc) { if (b_nc) LSAM_SIMT(true, true); else LSAM_SIMT(true, false); }
+  else      { if (b_nc) LSAM_SIMT(false, true); else LSAM_SIMT(false, false); }
+#undef LSAM_SIMT
   return LSAM_OK;
 }
 

@@ -122,60 +122,120 @@ struct EpiWgrad {
 
 // ------------------------------------------------------------------------------------------------ SIMT batched GEMM
 // C(z, m, n) = sum_kk A(z, m, kk) * B(z, n, kk), accumulated in fp32 in ascending kk; arbitrary element strides.
-// 64 x 64 tile, 16-deep slices, 256 threads, 4 x 4 outputs per thread.  SWAP_MN hands (z, n, m) to the epilogue.
+// 128 x 64 tile, 16-deep slices, 256 threads, 8 x 4 outputs per thread.  The next slice is fetched from global memory
+// into registers (128-bit loads along whichever direction of the operand is contiguous, when aligned) while the current
+// one is multiplied out of shared memory.
 struct GemmOperand { const void* p; int64_t sz, sr, sk; };  // element (z, r, kk) at p[z*sz + r*sr + kk*sk]
 
-template <typename TA_, typename TB_, class Epi>
+constexpr int kSimtBM = 128, kSimtBN = 64, kSimtBK = 16;
+
+// Four consecutive elements of an operand tile, along the rows (ROWS_CONTIG) or along the contraction index.
+// r, kk: first element; rmax, kmax: extents.  Out-of-range elements read as 0.
+template <typename T, bool ROWS_CONTIG>
+__device__ inline float4 simt_fetch4(const T* __restrict__ base, int64_t sr, int64_t sk, int r, int kk, int rmax, int kmax, bool vec_ok) {
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (ROWS_CONTIG) {
+    if (kk >= kmax || r >= rmax) return v;
+    const T* p = base + (int64_t)r * sr + (int64_t)kk * sk;
+    if (sizeof(T) == 4 && vec_ok && r + 3 < rmax) return *reinterpret_cast<const float4*>(p);
+    v.x = to_float(p[0]);
+    if (r + 1 < rmax) v.y = to_float(p[sr]);
+    if (r + 2 < rmax) v.z = to_float(p[2 * sr]);
+    if (r + 3 < rmax) v.w = to_float(p[3 * sr]);
+  } else {
+    if (r >= rmax || kk >= kmax) return v;
+    const T* p = base + (int64_t)r * sr + (int64_t)kk * sk;
+    if (sizeof(T) == 4 && vec_ok && kk + 3 < kmax) return *reinterpret_cast<const float4*>(p);
+    v.x = to_float(p[0]);
+    if (kk + 1 < kmax) v.y = to_float(p[sk]);
+    if (kk + 2 < kmax) v.z = to_float(p[2 * sk]);
+    if (kk + 3 < kmax) v.w = to_float(p[3 * sk]);
+  }
+  return v;
+}
+
+template <typename TA_, typename TB_, bool A_MC, bool B_NC, class Epi>
 __global__ void __launch_bounds__(256)
 gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, const int32_t* __restrict__ active) {
-  constexpr int BM = 64, BN = 64, BK = 16;
+  constexpr int BM = kSimtBM, BN = kSimtBN, BK = kSimtBK;
   if (active != nullptr && !active[blockIdx.z]) return;  // a waiting replica
-  __shared__ float As[BK][BM + 4];
-  __shared__ float Bs[BK][BN + 4];
+  __shared__ __align__(16) float As[BK][BM + 4];
+  __shared__ __align__(16) float Bs[BK][BN + 4];
   const int z = blockIdx.z;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const TA_* Ap = reinterpret_cast<const TA_*>(A.p) + (int64_t)z * A.sz;
   const TB_* Bp = reinterpret_cast<const TB_*>(Bo.p) + (int64_t)z * Bo.sz;
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;
-  // loader mapping: along the contiguous direction of each operand
-  const bool a_kc = (A.sk == 1), b_kc = (Bo.sk == 1);
-  float acc[4][4];
+  // 128-bit loads need the contiguous stride to be 1 (guaranteed by the template flag), the other stride a multiple
+  // of 4 elements and the replica's base 16-byte aligned
+  const bool vecA = sizeof(TA_) == 4 && (reinterpret_cast<uintptr_t>(Ap) & 15) == 0 && ((A_MC ? A.sk : A.sr) % 4) == 0;
+  const bool vecB = sizeof(TB_) == 4 && (reinterpret_cast<uintptr_t>(Bp) & 15) == 0 && ((B_NC ? Bo.sk : Bo.sr) % 4) == 0;
+  // this thread's slots in the tiles: A has 2 groups of 4 elements, B has 1
+  int a_r[2], a_k[2];
 #pragma unroll
-  for (int i = 0; i < 4; ++i)
+  for (int e = 0; e < 2; ++e) {
+    const int f = e * 256 + tid;
+    if (A_MC) { a_k[e] = f >> 5; a_r[e] = (f & 31) * 4; } else { a_r[e] = f >> 2; a_k[e] = (f & 3) * 4; }
+  }
+  int b_r, b_k;
+  if (B_NC) { b_k = tid >> 4; b_r = (tid & 15) * 4; } else { b_r = tid >> 2; b_k = (tid & 3) * 4; }
+
+  float acc[8][4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i)
 #pragma unroll
     for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
 
-  for (int k0 = 0; k0 < Kd; k0 += BK) {
+  float4 ra[2], rb;
+  auto fetch = [&](int k0) {
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const int lin = e * 256 + tid;
-      int r, kk;
-      if (a_kc) { kk = lin & 15; r = lin >> 4; } else { r = lin & 63; kk = lin >> 6; }
-      const int gm = m0 + r, gk = k0 + kk;
-      As[kk][r] = (gm < M && gk < Kd) ? to_float(Ap[(int64_t)gm * A.sr + (int64_t)gk * A.sk]) : 0.f;
-      if (b_kc) { kk = lin & 15; r = lin >> 4; } else { r = lin & 63; kk = lin >> 6; }
-      const int gn = n0 + r;
-      const int gk2 = k0 + kk;
-      Bs[kk][r] = (gn < N && gk2 < Kd) ? to_float(Bp[(int64_t)gn * Bo.sr + (int64_t)gk2 * Bo.sk]) : 0.f;
+    for (int e = 0; e < 2; ++e) ra[e] = simt_fetch4<TA_, A_MC>(Ap, A.sr, A.sk, m0 + a_r[e], k0 + a_k[e], M, Kd, vecA);
+    rb = simt_fetch4<TB_, B_NC>(Bp, Bo.sr, Bo.sk, n0 + b_r, k0 + b_k, N, Kd, vecB);
+  };
+  auto stash = [&]() {
+#pragma unroll
+    for (int e = 0; e < 2; ++e) {
+      if (A_MC) {
+        *reinterpret_cast<float4*>(&As[a_k[e]][a_r[e]]) = ra[e];
+      } else {
+        As[a_k[e]][a_r[e]] = ra[e].x; As[a_k[e] + 1][a_r[e]] = ra[e].y; As[a_k[e] + 2][a_r[e]] = ra[e].z; As[a_k[e] + 3][a_r[e]] = ra[e].w;
+      }
     }
-    __syncthreads();
+    if (B_NC) {
+      *reinterpret_cast<float4*>(&Bs[b_k][b_r]) = rb;
+    } else {
+      Bs[b_k][b_r] = rb.x; Bs[b_k + 1][b_r] = rb.y; Bs[b_k + 2][b_r] = rb.z; Bs[b_k + 3][b_r] = rb.w;
+    }
+  };
+
+  fetch(0);
+  stash();
+  __syncthreads();
+  for (int k0 = 0; k0 < Kd; k0 += BK) {
+    const bool more = k0 + BK < Kd;
+    if (more) fetch(k0 + BK);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
-      const float4 av = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
+      const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 8]);
+      const float4 a1 = *reinterpret_cast<const float4*>(&As[kk][ty * 8 + 4]);
       const float4 bv = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-      const float a_[4] = {av.x, av.y, av.z, av.w};
+      const float a_[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
       const float b_[4] = {bv.x, bv.y, bv.z, bv.w};
 #pragma unroll
-      for (int i = 0; i < 4; ++i)
+      for (int i = 0; i < 8; ++i)
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a_[i], b_[j], acc[i][j]);
     }
     __syncthreads();
+    if (more) {
+      stash();
+      __syncthreads();
+    }
   }
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const int gm = m0 + ty * 4 + i;
+  for (int i = 0; i < 8; ++i) {
+    const int gm = m0 + ty * 8 + i;
     if (gm >= M) continue;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
