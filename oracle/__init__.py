@@ -35,7 +35,7 @@ class OracleConfig(C.Structure):
         ("batch", C.c_int32), ("gemm_dtype", C.c_int32), ("nesterov", C.c_int32), ("tau", C.c_int32),
         ("stale_max", C.c_int32), ("active_num", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_double), ("gamma", C.c_double), ("lam", C.c_double),
-        ("beta", C.c_double), ("eta_prime", C.c_double),
+        ("beta", C.c_double), ("eta_prime", C.c_double), ("noise_temp", C.c_double),
     ]
 
 
@@ -71,6 +71,10 @@ def lib():
         L.oracle_tag_order.restype = C.c_uint64
         L.oracle_loss_grad.argtypes = [cfgp, vp, vp, vp, vp, C.c_int32, vp, vp]
         L.oracle_forward.argtypes = [cfgp, vp, vp, vp, C.c_int32, vp]
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        L.oracle_noise4.restype = None
+        L.oracle_noise4.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64, vp]
         L.oracle_mix64.restype = C.c_uint64
         L.oracle_mix64.argtypes = [C.c_uint64]
         L.oracle_hash.restype = C.c_uint64
@@ -85,7 +89,7 @@ def lib():
 
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, nesterov=1, gamma=1e-12,
-                lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, active_num=256):
+                lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, active_num=256, noise_temp=0.0):
     """Float hyper-parameters are taken at their fp32 value, the precision the C-ABI carries them in."""
     c = OracleConfig()
     c.model = model
@@ -98,6 +102,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, ne
     c.active_num = int(active_num)
     f32 = lambda v: float(np.float32(v))
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = f32(mu), f32(gamma), f32(lam), f32(beta), f32(eta_prime)
+    c.noise_temp = f32(noise_temp)
     return c
 
 
@@ -129,6 +134,20 @@ def forward(cfg, X, params, idx):
     out = np.zeros((len(idx), n_out), dtype=np.float64)
     rc = lib().oracle_forward(C.byref(cfg), _ptr(X), _ptr(params), _ptr(idx), len(idx), _ptr(out))
     assert rc == 0
+    return out
+
+
+def philox(counter, key):
+    c = np.asarray(counter, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().oracle_philox4x32_10(_ptr(c), _ptr(k), _ptr(out))
+    return [int(v) for v in out]
+
+
+def noise4(seed, t, k, seg, group):
+    out = np.zeros(4, dtype=np.float64)
+    lib().oracle_noise4(seed, t, k, seg, group, _ptr(out))
     return out
 
 

@@ -34,6 +34,38 @@ inline uint64_t hash5(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint6
   return mix64(mix64(mix64(seed ^ tag) + t) + ((k << 20) + j));
 }
 
+// ---- Langevin noise: Philox4x32-10 counter-based generator (Salmon, Moraes, Dror, Shaw, SC 2011) + Box-Muller.
+// One block gives the four normals of one group of four consecutive parameters of a segment (W_l: segment 2l,
+// b_l: segment 2l+1; least squares / flat vector: segment 0):
+//   counter = (group low 32 bits, segment, worker, tick low 32 bits), key = (seed low ^ "lang", seed high ^ tick high)
+//   u = ((r >> 8) + 0.5) 2^-24 from each 32-bit output r (exact in binary32, never 0 or 1)
+//   (z0, z1) = sqrt(-2 ln u0) (cos 2 pi u1, sin 2 pi u1), (z2, z3) likewise from (u2, u3)
+inline void philox4x32_10(const uint32_t c_in[4], const uint32_t k_in[2], uint32_t out[4]) {
+  uint32_t c[4] = {c_in[0], c_in[1], c_in[2], c_in[3]};
+  uint32_t k0 = k_in[0], k1 = k_in[1];
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    const uint64_t p0 = (uint64_t)0xD2511F53u * c[0], p1 = (uint64_t)0xCD9E8D57u * c[2];
+    const uint32_t hi0 = (uint32_t)(p0 >> 32), lo0 = (uint32_t)p0, hi1 = (uint32_t)(p1 >> 32), lo1 = (uint32_t)p1;
+    const uint32_t n0 = hi1 ^ c[1] ^ k0, n1 = lo1, n2 = hi0 ^ c[3] ^ k1, n3 = lo0;
+    c[0] = n0; c[1] = n1; c[2] = n2; c[3] = n3;
+  }
+  for (int i = 0; i < 4; ++i) out[i] = c[i];
+}
+inline void noise4(uint64_t seed, uint64_t t, uint64_t k, uint32_t seg, uint64_t group, double z[4]) {
+  const uint32_t ctr[4] = {(uint32_t)group, seg, (uint32_t)k, (uint32_t)t};
+  const uint32_t key[2] = {(uint32_t)seed ^ 0x6c616e67u, (uint32_t)(seed >> 32) ^ (uint32_t)(t >> 32)};
+  uint32_t r[4];
+  philox4x32_10(ctr, key, r);
+  const double two_pi = 6.283185307179586476925286766559;
+  for (int h = 0; h < 2; ++h) {
+    const double u0 = ((double)(r[2 * h] >> 8) + 0.5) / 16777216.0, u1 = ((double)(r[2 * h + 1] >> 8) + 0.5) / 16777216.0;
+    const double rad = std::sqrt(-2.0 * std::log(u0));
+    z[2 * h] = rad * std::cos(two_pi * u1);
+    z[2 * h + 1] = rad * std::sin(two_pi * u1);
+  }
+}
+
 // ---- bf16 round-to-nearest-even of an fp32 value (published format: 1-8-7, top half of binary32)
 inline float bf16_round(float v) {
   uint32_t u;
@@ -262,6 +294,8 @@ struct oracle_ctx {
 
 extern "C" {
 
+void oracle_philox4x32_10(const uint32_t* counter, const uint32_t* key, uint32_t* out) { philox4x32_10(counter, key, out); }
+void oracle_noise4(uint64_t seed, uint64_t t, uint64_t k, uint32_t seg, uint64_t group, double* out) { noise4(seed, t, k, seg, group, out); }
 uint64_t oracle_mix64(uint64_t z) { return mix64(z); }
 uint64_t oracle_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j) { return hash5(seed, tag, t, k, j); }
 uint64_t oracle_tag_idx(void) { return TAG_IDX; }
@@ -413,8 +447,28 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
       const double G = g2[j] + c.lambda * (x[j] - yk[j]);
       v[j] = c.mu * v[j] + G;
       x[j] = c.nesterov ? x[j] - eta * (G + c.mu * v[j]) : x[j] - eta * v[j];
-      acc[j] += x[j];  // running sum of post-update iterates since the last sync
     }
+    if (c.noise_temp > 0.0) {
+      // Langevin sampler: x <- x + sqrt(2 eta T) xi, xi ~ N(0, I) (Section 4.1; comment of Algorithm 1)
+      const double sigma = std::sqrt(2.0 * eta * c.noise_temp);
+      auto add_noise = [&](uint32_t seg, int64_t off, int64_t len) {
+        for (int64_t e = 0; e < len; e += 4) {
+          double z[4];
+          noise4(c.seed, (uint64_t)t, (uint64_t)o->rid[k], seg, (uint64_t)(e / 4), z);
+          for (int i = 0; i < 4 && e + i < len; ++i) x[off + e + i] += sigma * z[i];
+        }
+      };
+      if (o->net.layers.empty() || c.model == ORACLE_MODEL_LSQ) {
+        add_noise(0, 0, d);
+      } else {
+        for (size_t l = 0; l < o->net.layers.size(); ++l) {
+          const Layer& ly = o->net.layers[l];
+          add_noise((uint32_t)(2 * l), ly.w_off, (int64_t)ly.in * ly.out);
+          add_noise((uint32_t)(2 * l + 1), ly.b_off, ly.out);
+        }
+      }
+    }
+    for (int64_t j = 0; j < d; ++j) acc[j] += x[j];  // running sum of post-update iterates since the last sync
     o->t_x[k] += 1;
   }
   o->t += 1;

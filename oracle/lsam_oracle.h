@@ -49,6 +49,7 @@ typedef struct {
   double lambda;        /* pull strength of the Gaussian kernel                              */
   double beta;          /* centre look-ahead factor                                          */
   double eta_prime;     /* centre step size                                                  */
+  double noise_temp;    /* Langevin temperature T: x += sqrt(2 eta T) N(0, I) after the step; 0 = none */
 } oracle_config;
 
 typedef struct oracle_ctx oracle_ctx;
@@ -99,6 +100,10 @@ int oracle_loss_grad(const oracle_config* cfg, const float* X, const void* Y, co
 /* Logits (MLP/RESMLP: [n_idx, classes]) or predictions (LSQ: [n_idx]) at `params`. */
 int oracle_forward(const oracle_config* cfg, const float* X, const double* params,
                    const int32_t* idx, int32_t n_idx, double* out);
+/* Philox4x32-10 block (Salmon, Moraes, Dror, Shaw 2011): counter[4], key[2] -> out[4]. */
+void oracle_philox4x32_10(const uint32_t* counter, const uint32_t* key, uint32_t* out);
+/* The four standard normals of noise group `group` of parameter segment `seg` of worker k at tick t. */
+void oracle_noise4(uint64_t seed, uint64_t t, uint64_t k, uint32_t seg, uint64_t group, double* out);
 uint64_t oracle_mix64(uint64_t z);
 uint64_t oracle_hash(uint64_t seed, uint64_t tag, uint64_t t, uint64_t k, uint64_t j);
 uint64_t oracle_tag_idx(void);

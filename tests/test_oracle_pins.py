@@ -561,3 +561,90 @@ def test_always_ready_is_the_lock_step_schedule_and_waiting_for_sync_is_an_error
     assert O.lib().oracle_step(a._h, 0.05, 0.05) == 4  # the sync is due: nobody may step
     np.testing.assert_array_equal(a.read_state()["x"], x)
     assert a.counters()[0] == 8
+
+
+# ------------------------------------------------------------------------------------------- Langevin noise
+def test_philox_matches_published_known_answers():
+    for line in open(os.path.join(GOLD, "philox4x32_10_kat.txt")):
+        if not line.strip() or line.startswith("#"):
+            continue
+        v = [int(x, 16) for x in line.split()]
+        assert O.philox(v[0:4], v[4:6]) == v[6:10]
+
+
+def test_noise_is_standard_normal_and_keyed_by_all_of_its_arguments():
+    z = np.array([O.noise4(9, 3, 2, 1, g) for g in range(50000)])  # 200000 draws
+    flat = z.ravel()
+    n = flat.size
+    assert abs(flat.mean()) < 4 / np.sqrt(n)
+    assert abs(flat.var() - 1) < 4 * np.sqrt(2 / n)
+    assert abs(np.mean(flat**3)) < 4 * np.sqrt(15 / n)          # skewness 0
+    assert abs(np.mean(flat**4) - 3) < 4 * np.sqrt(96 / n)      # kurtosis 3
+    c = np.corrcoef(z.T)
+    assert np.abs(c - np.eye(4)).max() < 4 / np.sqrt(len(z))   # the four lanes are uncorrelated
+    # Kolmogorov distance to the normal CDF
+    from scipy import stats
+    assert stats.kstest(flat[:50000], "norm").pvalue > 1e-3
+    base = O.noise4(9, 3, 2, 1, 7)
+    for other in (O.noise4(10, 3, 2, 1, 7), O.noise4(9, 4, 2, 1, 7), O.noise4(9, 3, 3, 1, 7), O.noise4(9, 3, 2, 0, 7), O.noise4(9, 3, 2, 1, 8),
+                  O.noise4(9 + 2**32, 3, 2, 1, 7), O.noise4(9, 3 + 2**32, 2, 1, 7)):
+        assert not np.allclose(base, other)
+    np.testing.assert_array_equal(base, O.noise4(9, 3, 2, 1, 7))
+
+
+def test_langevin_step_adds_sqrt_2_eta_T_noise_and_samples_the_kernel_gibbs_density():
+    # zero gradients, mu = 0, fixed centre: x_{t+1} = (1 - eta lambda) x_t + eta lambda y + sqrt(2 eta T) xi is an AR(1) chain whose
+    # stationary law is N(y, 2 eta T / (1 - (1 - eta lambda)^2)) -> the Gibbs density exp(-(lambda/2)||x - y||^2 / T) as eta -> 0
+    K, d, eta, lam, T = 2, 4000, 0.05, 2.0, 0.3
+    cfg = O.make_config(O.MODEL_FLAT, K=K, flat_d=d, mu=0.0, lam=lam, tau=10**6, noise_temp=T, seed=4)
+    y0 = np.full(d, 1.5)
+    o = O.Oracle(cfg, None, None, np.tile(y0, (K, 1)), y0)
+    z = np.zeros((K, d), np.float32)
+    o.set_external_grads(z, z)
+    e, l, Tf = (float(np.float32(v)) for v in (eta, lam, T))
+    o.step(eta, 0.0)
+    x1 = o.read_state()["x"]
+    # first step from x = y: pure noise with variance 2 eta T, and exactly the tabulated normals
+    want = np.concatenate([O.noise4(4, 0, 1, 0, g) for g in range(d // 4)])
+    np.testing.assert_allclose(x1[1] - y0, np.sqrt(2 * e * Tf) * want, rtol=1e-12, atol=1e-15)
+    assert abs((x1 - y0).var() / (2 * e * Tf) - 1) < 0.05
+    for _ in range(150):
+        o.step(eta, 0.0)
+    var = (o.read_state()["x"] - y0).var()
+    stationary = 2 * e * Tf / (1 - (1 - e * l) ** 2)
+    assert abs(var / stationary - 1) < 0.05
+    assert abs(stationary / (Tf / l) - 1) < 0.06  # close to the continuous-time Gibbs variance T / lambda
+
+
+def test_zero_temperature_is_the_noise_free_step_and_noise_enters_the_iterate_sum():
+    a, x0, y0, g1, g2 = _flat_oracle(K=2, d=9, tau=3, lam=0.2, seed=5)
+    b, *_ = _flat_oracle(K=2, d=9, tau=3, lam=0.2, seed=5, noise_temp=0.0)
+    c, *_ = _flat_oracle(K=2, d=9, tau=3, lam=0.2, seed=5, noise_temp=0.5)
+    for o in (a, b, c):
+        o.step(0.05, 0.05)
+    np.testing.assert_array_equal(a.read_state()["x"], b.read_state()["x"])
+    sc = c.read_state()
+    assert not np.allclose(sc["x"], a.read_state()["x"])
+    np.testing.assert_array_equal(sc["acc"], sc["x"])  # the accumulated iterate is the noisy one
+    # d = 9: the last group is partial (one valid lane); segment 0, groups 0..2
+    sigma = np.sqrt(2 * float(np.float32(0.05)) * float(np.float32(0.5)))
+    z = np.concatenate([O.noise4(5, 0, 1, 0, g) for g in range(3)])[:9]
+    np.testing.assert_allclose(sc["x"][1] - a.read_state()["x"][1], sigma * z, rtol=1e-9, atol=1e-14)
+
+
+def test_noise_segments_follow_the_layers():
+    # W_l is segment 2l and b_l segment 2l + 1; the group index restarts in every segment
+    widths = (3, 5, 2)
+    X, labels = synth.gaussian_mixture(20, 3, 2, seed=1)
+    w0 = synth.mlp_init(widths, seed=1).astype(np.float64)
+    mk = lambda T: O.Oracle(O.make_config(O.MODEL_MLP, widths=widths, K=1, batch=4, n_samples=20, mu=0.0, tau=100, seed=8, noise_temp=T), X, labels, w0[None], w0)
+    a, b = mk(0.0), mk(1.0)
+    a.step(0.1, 0.0)
+    b.step(0.1, 0.0)
+    diff = (b.read_params(0) - a.read_params(0)) / np.sqrt(2 * float(np.float32(0.1)))
+    segs = [(0, 15), (1, 5), (2, 10), (3, 2)]
+    off = 0
+    for seg, ln in segs:
+        z = np.concatenate([O.noise4(8, 0, 0, seg, g) for g in range((ln + 3) // 4)])[:ln]
+        np.testing.assert_allclose(diff[off:off + ln], z, rtol=1e-9, atol=1e-12)
+        off += ln
