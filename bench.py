@@ -197,7 +197,8 @@ def make_cfg(G, w, flags=0):
     return G.make_config(w["model"], widths=w["widths"], K=w["K"], batch=max(w["B"], 1) if w["model"] != FLAT else 0,
                          gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
                          beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
-                         flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256))
+                         flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256),
+                         noise_temp=w.get("noise_temp", 0.0))
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
@@ -286,6 +287,7 @@ def main():
     ap.add_argument("--flat-d", type=int, default=None, help="c5 only: vector length of the sweep point")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
+    ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
     ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
@@ -295,6 +297,9 @@ def main():
     if args.replicas:
         w["K"] = args.replicas
         w["name"] += f" [K overridden to {args.replicas}]"
+    if args.noise_temp > 0.0:
+        w["noise_temp"] = args.noise_temp
+        w["name"] += f" [Langevin temperature {args.noise_temp}]"
     if args.active_num != 256:
         w["active_num"] = args.active_num
         w["name"] += f" [workers ready with probability {args.active_num}/256 per tick]"
@@ -443,6 +448,10 @@ def main():
     # ---- roofline of the dominant kernel class
     pk = peaks()
     work = work_model(w, ctx.uses_tcgen05())
+    frac_active = worker_iters_per_step / w["K"]  # waiting replicas are skipped by every kernel
+    for wk_ in work.values():
+        for key in wk_:
+            wk_[key] *= frac_active
     tot_ms = sum(v[0] for v in prof.values())
     top = max(prof, key=lambda k: prof[k][0])
     tms, tn = prof[top]

@@ -86,6 +86,8 @@ typedef struct {
   float eta_prime;    /* centre step size eta'                                                      */
   int32_t active_num; /* asynchronous progress: a worker is ready at a tick with probability active_num/256;
                          0 or 256 = every worker steps at every tick (lock-step)                     */
+  float noise_temp;   /* Langevin temperature T >= 0 (Section 4.1): x += sqrt(2 eta T) N(0, I) after the step,
+                         normals from Philox4x32-10 keyed by (seed, tick, worker, segment, offset); 0 = none */
 } lsam_config;
 
 /* Unpadded parameter count d of one replica, or -1 if the configuration is invalid. */

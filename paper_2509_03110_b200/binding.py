@@ -34,7 +34,7 @@ class LsamConfig(C.Structure):
         ("gemm_dtype", C.c_int32), ("gemm_impl", C.c_int32), ("nesterov", C.c_int32), ("tau", C.c_int32),
         ("stale_max", C.c_int32), ("flags", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_float), ("gamma", C.c_float), ("lam", C.c_float), ("beta", C.c_float),
-        ("eta_prime", C.c_float), ("active_num", C.c_int32),
+        ("eta_prime", C.c_float), ("active_num", C.c_int32), ("noise_temp", C.c_float),
     ]
 
 
@@ -99,7 +99,7 @@ def lib():
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=IMPL_AUTO, mu=0.9, nesterov=1,
                 gamma=1e-12, lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, flags=0,
-                active_num=256):
+                active_num=256, noise_temp=0.0):
     c = LsamConfig()
     c.model = model
     widths = list(widths)
@@ -110,6 +110,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=
     c.stale_max, c.flags, c.n_samples, c.flat_d, c.seed = int(stale_max), int(flags), int(n_samples), int(flat_d), int(seed)
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = mu, gamma, lam, beta, eta_prime
     c.active_num = int(active_num)
+    c.noise_temp = noise_temp
     return c
 
 

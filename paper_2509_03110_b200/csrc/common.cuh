@@ -29,6 +29,35 @@ __host__ __device__ inline uint64_t schedule_hash(uint64_t seed, uint64_t tag, u
   return mix64(mix64(mix64(seed ^ tag) + t) + ((k << 20) + j));
 }
 
+// ---- Langevin noise: Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC 2011) + Box-Muller, four normals per block.
+//   counter = (group low 32 bits, segment, worker, tick low 32 bits), key = (seed low ^ "lang", seed high ^ tick high)
+//   u = ((r >> 8) + 0.5) 2^-24 (exact in binary32), (z0, z1) = sqrt(-2 ln u0) (cos 2 pi u1, sin 2 pi u1), (z2, z3) from (u2, u3)
+__device__ inline void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0, uint32_t k1, uint32_t (&out)[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    if (r > 0) { k0 += 0x9E3779B9u; k1 += 0xBB67AE85u; }
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+__device__ inline void langevin_noise4(uint64_t seed, uint64_t t, uint32_t k, uint32_t seg, uint64_t group, float (&z)[4]) {
+  uint32_t r[4];
+  philox4x32_10((uint32_t)group, seg, k, (uint32_t)t, (uint32_t)seed ^ 0x6c616e67u, (uint32_t)(seed >> 32) ^ (uint32_t)(t >> 32), r);
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const float u0 = ((float)(r[2 * h] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    const float u1 = ((float)(r[2 * h + 1] >> 8) + 0.5f) * (1.0f / 16777216.0f);
+    const float rad = sqrtf(-2.0f * logf(u0));
+    float sn, cs;
+    sincospif(2.0f * u1, &sn, &cs);
+    z[2 * h] = rad * cs;
+    z[2 * h + 1] = rad * sn;
+  }
+}
+
 // ---- element conversion between the accumulator type (float) and a storage type
 template <typename T> __device__ inline T from_float(float v);
 template <> __device__ inline float from_float<float>(float v) { return v; }

@@ -52,6 +52,7 @@ bool plan(const lsam_config& c, Layout& L) {
   if (c.gemm_impl < LSAM_IMPL_AUTO || c.gemm_impl > LSAM_IMPL_TCGEN05) return false;
   if (!(c.gamma > 0.f)) return false;
   if (c.active_num < 0 || c.active_num > 256) return false;
+  if (!(c.noise_temp >= 0.f)) return false;
   const bool bf = c.gemm_dtype == LSAM_GEMM_BF16;
   L.seg.n = 0;
   if (c.model == LSAM_MODEL_FLAT) {
@@ -282,7 +283,14 @@ int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4
   const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16;
   const bool nes = c->cfg.nesterov != 0;
   const unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
-#define LSAM_UPD_LAUNCH(V, N, T, W) LAUNCH(c, LSAM_PROF_UPDATE, update_kernel<V, N, T, W><<<grid, kUpdThreads, 0, c->stream>>>(a))
+  const bool noise = c->cfg.noise_temp > 0.f;
+  a.sigma = noise ? sqrtf(2.0f * eta * c->cfg.noise_temp) : 0.f;
+  a.seed = c->cfg.seed; a.tick = (uint64_t)c->t; a.seg = c->L.seg;
+#define LSAM_UPD_LAUNCH(V, N, T, W)                                                                               \
+  do {                                                                                                            \
+    if (noise) LAUNCH(c, LSAM_PROF_UPDATE, update_kernel<V, N, T, W, true><<<grid, kUpdThreads, 0, c->stream>>>(a)); \
+    else LAUNCH(c, LSAM_PROF_UPDATE, update_kernel<V, N, T, W, false><<<grid, kUpdThreads, 0, c->stream>>>(a));     \
+  } while (0)
   if (vec4) {
     if (bf) { if (nes) LSAM_UPD_LAUNCH(4, true, bf16, true); else LSAM_UPD_LAUNCH(4, false, bf16, true); }
     else    { if (nes) LSAM_UPD_LAUNCH(4, true, float, false); else LSAM_UPD_LAUNCH(4, false, float, false); }

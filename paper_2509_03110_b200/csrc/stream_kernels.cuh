@@ -167,6 +167,11 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict
 // re-read from cache and the iterate accumulator is read and written once per column:
 //   G = g2 + lambda (x - y_slot[k]);  v <- mu v + G;  x <- x - eta (G + mu v)  [Nesterov]  or  x - eta v;
 //   acc += sum_k x_new;  optional operand copy xop = TP(x_new).
+// NOISE: the Langevin term sqrt(2 eta T) N(0, I) is added to x_new before it is stored and accumulated; the normals are
+// keyed by (tick, replica, segment, offset within the segment), so padding elements get none and stay zero.
+// Parameter segments of a replica's row: seg i = {offset in the unpadded vector, offset in the padded row, length}.
+struct SegMap { int n; int64_t src[18], dst[18], len[18]; };
+
 struct UpdateArgs {
   float* x;            // [K, ld]
   float* v;            // [K, ld]
@@ -179,14 +184,27 @@ struct UpdateArgs {
   int64_t ld, ldg, n;
   int K;
   float eta, mu, lambda;
+  // Langevin noise (NOISE variants): x_new += sigma * xi, xi from langevin_noise4(seed, tick, k, segment, offset / 4)
+  float sigma;
+  uint64_t seed, tick;
+  SegMap seg;
 };
 
 constexpr int kUpdThreads = 256;
 
-template <int VEC, bool NESTEROV, typename TP, bool WRITE_OP>
+template <int VEC, bool NESTEROV, typename TP, bool WRITE_OP, bool NOISE>
 __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a) {
   const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * VEC;
   if (j >= a.n) return;
+  // segment of this thread's elements (segments ascend; all VEC elements lie in one segment: starts are multiples of 64)
+  uint32_t nseg = 0;
+  int64_t noff = 0, nlen = 0;
+  if (NOISE) {
+    for (int s = 1; s < a.seg.n; ++s)
+      if (j >= a.seg.dst[s]) nseg = (uint32_t)s;
+    noff = j - a.seg.dst[nseg];
+    nlen = a.seg.len[nseg];
+  }
   if (VEC == 4) {
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     // software pipeline over the replicas: the four loads of replica k + 1 are issued before the arithmetic and the
@@ -218,10 +236,18 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
 #define LSAM_UPD(c)                                                         \
   G = fmaf(a.lambda, xv.c - yv.c, gv.c);                                    \
   vv.c = fmaf(a.mu, vv.c, G);                                               \
-  xv.c = NESTEROV ? xv.c - a.eta * fmaf(a.mu, vv.c, G) : xv.c - a.eta * vv.c; \
-  s.c += xv.c;
+  xv.c = NESTEROV ? xv.c - a.eta * fmaf(a.mu, vv.c, G) : xv.c - a.eta * vv.c;
       LSAM_UPD(x) LSAM_UPD(y) LSAM_UPD(z) LSAM_UPD(w)
 #undef LSAM_UPD
+      if (NOISE && noff < nlen) {
+        float z[4];
+        langevin_noise4(a.seed, a.tick, (uint32_t)k, nseg, (uint64_t)(noff >> 2), z);
+        xv.x = fmaf(a.sigma, z[0], xv.x);
+        if (noff + 1 < nlen) xv.y = fmaf(a.sigma, z[1], xv.y);
+        if (noff + 2 < nlen) xv.z = fmaf(a.sigma, z[2], xv.z);
+        if (noff + 3 < nlen) xv.w = fmaf(a.sigma, z[3], xv.w);
+      }
+      s.x += xv.x; s.y += xv.y; s.z += xv.z; s.w += xv.w;
       *reinterpret_cast<float4*>(a.x + o) = xv;
       __stcs(reinterpret_cast<float4*>(a.v + o), vv);
       if (WRITE_OP) {
@@ -250,6 +276,11 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       const float G = fmaf(a.lambda, xv - yv, gv);
       vv = fmaf(a.mu, vv, G);
       xv = NESTEROV ? xv - a.eta * fmaf(a.mu, vv, G) : xv - a.eta * vv;
+      if (NOISE && noff < nlen) {
+        float z[4];
+        langevin_noise4(a.seed, a.tick, (uint32_t)k, nseg, (uint64_t)(noff >> 2), z);
+        xv = fmaf(a.sigma, z[noff & 3], xv);
+      }
       s += xv;
       a.x[o] = xv;
       a.v[o] = vv;
@@ -286,8 +317,6 @@ cast_rows_kernel(const float* __restrict__ src, int64_t lds, TP* __restrict__ ds
   dst[(int64_t)k * ldd + j] = from_float<TP>(src[(int64_t)k * lds + j]);
 }
 
-// Copy between an unpadded vector and its padded layout.  seg[i] = {unpadded offset, padded offset, length}.
-struct SegMap { int n; int64_t src[18], dst[18], len[18]; };
 
 template <bool TO_PADDED, typename TS, typename TD>
 __global__ void __launch_bounds__(256)

@@ -332,6 +332,45 @@ def test_async_progress_masks_bit_exact_and_trajectory(kind):
     p.close()
 
 
+# ------------------------------------------------------------------------------------------------ Langevin noise
+@pytest.mark.parametrize("kind", ["flat_1000", "flat_1001", "flat_262147", "mlp_fp32", "resmlp_bf16_tcgen05"])
+def test_langevin_noise_matches_oracle(kind):
+    # the counter-based normals are the same numbers on both sides (integers from Philox, then fp32 vs double
+    # Box-Muller), so a noisy step must agree to the usual fp32 tolerance
+    hp = dict(tau=3, lam=0.3, seed=17, noise_temp=0.4)
+    if kind.startswith("flat"):
+        K, d = 4, int(kind.split("_")[1])
+        x0, y0, g1, g2 = synth.flat_problem(K, d, seed=6)
+        p = Pair(G.MODEL_FLAT, K=K, flat_d=d, x0=x0, y0=y0, **hp)
+        p.set_external_grads(g1, g2)
+        tol_step, tol = TOL_STEP_FP32, TOL_TRAJ_FP32
+    elif kind == "mlp_fp32":
+        p = _mlp_pair(G.MODEL_MLP, (20, 33, 7), 3, 10, n=200, dtype=G.GEMM_FP32, jitter=0.01, **hp)
+        tol_step, tol = TOL_STEP_FP32, TOL_TRAJ_FP32
+    else:
+        # a temperature at which the noise per step (sigma = 0.008) stays small against the weights: with sigma = 0.15 the
+        # network is shaken so hard that the ReLU decisions of the two sides drift apart within a dozen steps
+        hp["noise_temp"] = 1e-3
+        p = _mlp_pair(G.MODEL_RESMLP, (64, 128, 128, 16), 3, 48, n=300, dtype=G.GEMM_BF16, impl=G.IMPL_TCGEN05, jitter=0.01, **hp)
+        tol_step, tol = TOL_STEP_BF16, TOL_TRAJ_BF16
+    noiseless = p.oracle.read_state()["x"].copy()
+    p.teacher_force()
+    p.step(0.03, 0.05)
+    e = p.errors()
+    assert e["x"] <= tol_step and e["acc"] <= max(tol_step, 1e-5), e
+    assert not np.allclose(p.oracle.read_state()["x"], noiseless)
+    p.couple_if_due()
+    for t in range(12):
+        p.step(0.03, 0.05)
+        p.couple_if_due()
+    e = p.errors()
+    assert e["x"] <= tol and e["y"] <= tol, e
+    assert p.gpu.status() == 0
+    # padding of the device layout never receives noise: the unpadded read-back has exactly d finite entries and
+    # a second context with temperature 0 differs from this one
+    p.close()
+
+
 def test_step_refused_while_sync_is_due():
     import torch
 
