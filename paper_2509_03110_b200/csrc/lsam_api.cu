@@ -474,6 +474,19 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
   const int64_t n = flat ? L.d : L.ld;
   const int64_t ldg = flat ? L.d : L.ld;
   // ascent gradient, its norm, perturbation
+  if (rho == 0.f && !flat && !L.g1keep) {
+    // rho = 0: the perturbed point is x itself, so the two gradients coincide (entropy-/elastic-averaging SGD, the
+    // unperturbed case of Theorem 2): one gradient pass, no norm, no perturbation
+    if ((rc = grad_pass(c, false, c->loss())) != LSAM_OK) return rc;
+    if (cfg.flags & LSAM_FLAG_STEP_INFO) {
+      if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm1(), nullptr)) != LSAM_OK) return rc;
+      if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
+    }
+    if ((rc = launch_update(c, c->g(), ldg, n, vec4, eta)) != LSAM_OK) return rc;
+    for (int k = 0; k < cfg.K; ++k) c->t_x[k] += c->async_on ? c->active_host[k] : 1;
+    c->t += 1;
+    return LSAM_OK;
+  }
   const float* g1 = flat ? c->eg1 : c->g();
   if (!flat && (rc = grad_pass(c, false, c->loss())) != LSAM_OK) return rc;
   if (!flat && L.g1keep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));

@@ -371,6 +371,38 @@ def test_langevin_noise_matches_oracle(kind):
     p.close()
 
 
+@pytest.mark.parametrize("dtype,impl", [(G.GEMM_FP32, G.IMPL_AUTO), (G.GEMM_BF16, G.IMPL_TCGEN05)])
+def test_rho_zero_takes_the_single_pass_shortcut_and_matches_oracle(dtype, impl):
+    # rho = 0 (no perturbation): the library runs one gradient pass; the oracle still runs both and finds them equal
+    widths = (64, 128, 128, 16)
+    X, labels = synth.gaussian_mixture(300, widths[0], widths[-1], seed=2)
+    w0 = synth.mlp_init(widths, seed=2)
+    p = Pair(G.MODEL_RESMLP, widths=widths, K=3, batch=48, X=X, Y=labels, x0=synth.replicate(w0, 3, jitter=0.01), y0=w0,
+             gemm_dtype=dtype, gemm_impl=impl, tau=3, lam=0.3, seed=3, flags=G.FLAG_STEP_INFO)
+    launches = []
+    for t in range(9):
+        n0 = p.gpu.launch_count()
+        p.step(0.03, 0.0)
+        launches.append(p.gpu.launch_count() - n0)
+        ol, on1, on2 = p.oracle.read_step_info()
+        gl, gn1, gn2 = p.gpu.read_step_info()
+        if t == 0:
+            tol = TOL_STEP_BF16 if dtype == G.GEMM_BF16 else TOL_STEP_FP32
+            np.testing.assert_allclose(gl, ol, rtol=max(tol, 1e-5))
+            np.testing.assert_allclose(gn1, on1, rtol=tol)
+            np.testing.assert_allclose(gn2, on2, rtol=tol)
+            np.testing.assert_array_equal(on1, on2)
+        p.couple_if_due()
+    e = p.errors()
+    tol = TOL_TRAJ_BF16 if dtype == G.GEMM_BF16 else TOL_TRAJ_FP32
+    assert e["x"] <= tol and e["y"] <= tol, e
+    # and a step with rho > 0 launches about twice as many kernels
+    n0 = p.gpu.launch_count()
+    p.gpu.step(0.03, 0.05)
+    assert p.gpu.launch_count() - n0 > 1.5 * (launches[0] - 4)
+    p.close()
+
+
 def test_step_refused_while_sync_is_due():
     import torch
 
