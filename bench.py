@@ -326,8 +326,13 @@ def main():
     warm = max(args.warmup, 3)
 
     inp = make_inputs(w, dev, seed=rank)
-    cfg = make_cfg(G, w)
-    ctx = G.Lsam(cfg, inp["X"], inp["Y"], inp["x0"], inp["y0"])
+    # Latency-bound workloads (state resident in L2) replay each tick as one CUDA graph; that needs a capturable stream.
+    small = 4.0 * w["K"] * param_count(w) <= 126e6
+    cfg = make_cfg(G, w, flags=G.FLAG_CUDA_GRAPH if small else 0)
+    torch.cuda.synchronize()
+    work_stream = torch.cuda.Stream(device=dev)
+    torch.cuda.set_stream(work_stream)
+    ctx = G.Lsam(cfg, inp["X"], inp["Y"], inp["x0"], inp["y0"], stream=work_stream)
     d = ctx.d
     inp["x0"] = None
     torch.cuda.empty_cache()
@@ -499,7 +504,7 @@ def main():
 
     line = dict(metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=warm, ms_per_step=ms_step,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if w["bf16"] else "f32", data="synthetic",
-                config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt",
+                config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt", cuda_graph=bool(small),
                             l2="working set larger than L2" if events_in_timed else "L2-resident state (latency-bound workload); kernel shares from a separate profiled run",
                             parallelism="replicas only" if world > 1 else "1 GPU"),
                 clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)

@@ -54,7 +54,10 @@ enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
 enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2 };
 enum {
   LSAM_FLAG_KEEP_G1 = 1,   /* keep copies of the ascent gradient and (BF16 mode) of x~ for lsam_read_grads  */
-  LSAM_FLAG_STEP_INFO = 2  /* also reduce ||g2_k|| every step (one extra read of the gradient buffer)      */
+  LSAM_FLAG_STEP_INFO = 2, /* also reduce ||g2_k|| every step (one extra read of the gradient buffer)      */
+  LSAM_FLAG_CUDA_GRAPH = 4 /* replay each tick as one CUDA graph launch (recorded at the second tick of each variant;
+                              for launch-bound small models); needs a non-default stream (lsam_init fails with
+                              LSAM_ERR_INVALID otherwise); ignored while profiling is enabled               */
 };
 
 /* Models.

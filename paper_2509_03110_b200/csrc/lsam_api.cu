@@ -179,6 +179,15 @@ struct lsam_ctx {
   std::vector<int32_t> active_host;   // host mirror of the last tick's mask (drives the counters t_x)
   int64_t launches = 0;
   Profiler prof;
+  // CUDA-graph replay of the step (LSAM_FLAG_CUDA_GRAPH): one executable graph per launch sequence
+  struct GraphSlot {
+    bool warm = false;
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    cudaGraphNode_t n_sched = nullptr, n_fin = nullptr, n_upd = nullptr;
+    int64_t launches = 0;
+  } graphs[4];
+  void* upd_func = nullptr;  // the update_kernel instantiation this context launches
   std::string err;
   TcPlan tc;
 
@@ -246,6 +255,27 @@ int prof_end(lsam_ctx* c) {
     if (rc__ != LSAM_OK) return rc__;                          \
   } while (0)
 
+// Argument blocks of the three kernels whose parameters change from step to step (tick, centre-version history,
+// budget, rho, eta, noise scale).  They are launched through cudaLaunchKernel from these blocks, so that a captured
+// graph can be replayed with cudaGraphExecKernelNodeSetParams on the same blocks.
+struct SchedArgs {
+  uint64_t seed, t; int64_t n_samples; int B, stale_max; VerHist hist; int ring;
+  int32_t *idx, *stale, *ver, *slot; int K, active_num; int64_t budget; int32_t* active;
+  void* ptrs[15];
+  void bind() {
+    void* p[15] = {&seed, &t, &n_samples, &B, &stale_max, &hist, &ring, &idx, &stale, &ver, &slot, &K, &active_num, &budget, &active};
+    for (int i = 0; i < 15; ++i) ptrs[i] = p[i];
+  }
+};
+struct FinArgs {
+  const float* partial; int64_t nchunks, nused; float rho, gamma; float *norm_out, *scale_out; int* status; const int32_t* active;
+  void* ptrs[9];
+  void bind() {
+    void* p[9] = {&partial, &nchunks, &nused, &rho, &gamma, &norm_out, &scale_out, &status, &active};
+    for (int i = 0; i < 9; ++i) ptrs[i] = p[i];
+  }
+};
+
 // ---- norm of [K, n] rows -> norm_out[K] (and scale[K] = rho / (norm + gamma) if scale_out)
 int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float rho, float* norm_out, float* scale_out) {
   float* partial = c->at<float>(c->L.partial);
@@ -253,14 +283,18 @@ int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, 
   if (c->use_tc) {
     // tensor-core path: the weight- and bias-gradient kernels of the pass just run have left the sums of squares of
     // all their blocks in the partial slots; only the fixed-order final sum remains
-    LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act()));
+    FinArgs f{partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act(), {}};
+    f.bind();
+    LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(c->cfg.K), dim3(256), f.ptrs, 0, c->stream));
     return LSAM_OK;
   }
   dim3 grid((unsigned)ceil_div(n, vec4 ? norm_chunk<4>() : norm_chunk<1>()), c->cfg.K);
   if ((int64_t)grid.x > nch) return c->fail(LSAM_ERR_WORKSPACE, "norm: partial-sum buffer too small");
   if (vec4) LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<4><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch, c->act()));
   else LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<1><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch, c->act()));
-  LAUNCH(c, LSAM_PROF_NORM, norm_finalize_kernel<<<c->cfg.K, 256, 0, c->stream>>>(partial, nch, (int64_t)grid.x, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act()));
+  FinArgs f{partial, nch, (int64_t)grid.x, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act(), {}};
+  f.bind();
+  LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(c->cfg.K), dim3(256), f.ptrs, 0, c->stream));
   return LSAM_OK;
 }
 
@@ -274,45 +308,59 @@ int launch_perturb(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec
   return LSAM_OK;
 }
 
-int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float eta) {
+UpdateArgs make_update_args(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, float eta) {
   UpdateArgs a;
   a.active = c->act();
   a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
   a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
   a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
+  a.sigma = c->cfg.noise_temp > 0.f ? sqrtf(2.0f * eta * c->cfg.noise_temp) : 0.f;
+  a.seed = c->cfg.seed; a.tick = (uint64_t)c->t; a.seg = c->L.seg;
+  return a;
+}
+
+template <int V, bool N, typename T, bool W>
+void* update_func(bool noise) {
+  return noise ? (void*)update_kernel<V, N, T, W, true> : (void*)update_kernel<V, N, T, W, false>;
+}
+
+int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float eta) {
+  UpdateArgs a = make_update_args(c, g, ldg, n, eta);
   const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16;
   const bool nes = c->cfg.nesterov != 0;
-  const unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
   const bool noise = c->cfg.noise_temp > 0.f;
-  a.sigma = noise ? sqrtf(2.0f * eta * c->cfg.noise_temp) : 0.f;
-  a.seed = c->cfg.seed; a.tick = (uint64_t)c->t; a.seg = c->L.seg;
-#define LSAM_UPD_LAUNCH(V, N, T, W)                                                                               \
-  do {                                                                                                            \
-    if (noise) LAUNCH(c, LSAM_PROF_UPDATE, update_kernel<V, N, T, W, true><<<grid, kUpdThreads, 0, c->stream>>>(a)); \
-    else LAUNCH(c, LSAM_PROF_UPDATE, update_kernel<V, N, T, W, false><<<grid, kUpdThreads, 0, c->stream>>>(a));     \
-  } while (0)
+  const unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
+  void* f;
   if (vec4) {
-    if (bf) { if (nes) LSAM_UPD_LAUNCH(4, true, bf16, true); else LSAM_UPD_LAUNCH(4, false, bf16, true); }
-    else    { if (nes) LSAM_UPD_LAUNCH(4, true, float, false); else LSAM_UPD_LAUNCH(4, false, float, false); }
+    if (bf) f = nes ? update_func<4, true, bf16, true>(noise) : update_func<4, false, bf16, true>(noise);
+    else    f = nes ? update_func<4, true, float, false>(noise) : update_func<4, false, float, false>(noise);
   } else {
-    if (bf) { if (nes) LSAM_UPD_LAUNCH(1, true, bf16, true); else LSAM_UPD_LAUNCH(1, false, bf16, true); }
-    else    { if (nes) LSAM_UPD_LAUNCH(1, true, float, false); else LSAM_UPD_LAUNCH(1, false, float, false); }
+    if (bf) f = nes ? update_func<1, true, bf16, true>(noise) : update_func<1, false, bf16, true>(noise);
+    else    f = nes ? update_func<1, true, float, false>(noise) : update_func<1, false, float, false>(noise);
   }
-#undef LSAM_UPD_LAUNCH
+  c->upd_func = f;
+  void* ptrs[1] = {&a};
+  LAUNCH(c, LSAM_PROF_UPDATE, cudaLaunchKernel((const void*)f, dim3(grid), dim3(kUpdThreads), ptrs, 0, c->stream));
   return LSAM_OK;
 }
 
-int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot, int64_t budget, int32_t* active) {
-  VerHist h;
+SchedArgs make_sched_args(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot, int64_t budget, int32_t* active) {
+  SchedArgs a;
   for (int s = 0; s < 16; ++s) {
     const int64_t ts = t - s > 0 ? t - s : 0;
-    h.v[s] = ts < (int64_t)c->ver_at_step.size() ? c->ver_at_step[(size_t)ts] : -1;
+    a.hist.v[s] = ts < (int64_t)c->ver_at_step.size() ? c->ver_at_step[(size_t)ts] : -1;
   }
   const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
-  LAUNCH(c, LSAM_PROF_SCHEDULE,
-         schedule_kernel<<<c->cfg.K, 128, 0, c->stream>>>(c->cfg.seed, (uint64_t)t, flat ? 1 : c->cfg.n_samples, flat ? 0 : c->cfg.batch,
-                                                           c->cfg.stale_max, h, c->L.ring, flat ? nullptr : idx, stale, ver, slot,
-                                                           c->cfg.K, c->cfg.active_num, budget, active));
+  a.seed = c->cfg.seed; a.t = (uint64_t)t; a.n_samples = flat ? 1 : c->cfg.n_samples; a.B = flat ? 0 : c->cfg.batch;
+  a.stale_max = c->cfg.stale_max; a.ring = c->L.ring; a.idx = flat ? nullptr : idx; a.stale = stale; a.ver = ver; a.slot = slot;
+  a.K = c->cfg.K; a.active_num = c->cfg.active_num; a.budget = budget; a.active = active;
+  return a;
+}
+
+int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot, int64_t budget, int32_t* active) {
+  SchedArgs a = make_sched_args(c, t, idx, stale, ver, slot, budget, active);
+  a.bind();
+  LAUNCH(c, LSAM_PROF_SCHEDULE, cudaLaunchKernel((const void*)schedule_kernel, dim3(c->cfg.K), dim3(128), a.ptrs, 0, c->stream));
   return LSAM_OK;
 }
 
@@ -445,18 +493,12 @@ int seg_copy(lsam_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd
   return LSAM_OK;
 }
 
-int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
+// The launch sequence of one tick (no host state is changed here, so that it can also be recorded into a CUDA graph).
+int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget) {
   const lsam_config& cfg = c->cfg;
   const Layout& L = c->L;
   const bool flat = cfg.model == LSAM_MODEL_FLAT;
-  if (flat && (!c->eg1 || !c->eg2)) return c->fail(LSAM_ERR_STATE, "FLAT model: call lsam_set_external_grads first");
   int rc;
-  int64_t done = 0;
-  for (int64_t v : c->t_x) done += v;
-  const int64_t budget = (int64_t)cfg.K * cfg.tau - done;  // iterations still missing to n tau (Algorithm 2, sync trigger)
-  if (budget <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
-  c->ver_at_step.push_back((int)c->t_y);  // centre version current when this tick starts
-  if (c->async_on) host_active_mask(cfg, c->t, budget, c->active_host);
   if ((rc = launch_schedule(c, c->t, c->idx(), c->stale(), c->ver(), c->slot(), budget, c->async_on ? c->active_buf() : nullptr)) != LSAM_OK) return rc;
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   if (!flat && gather) {
@@ -483,8 +525,6 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
       if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
     }
     if ((rc = launch_update(c, c->g(), ldg, n, vec4, eta)) != LSAM_OK) return rc;
-    for (int k = 0; k < cfg.K; ++k) c->t_x[k] += c->async_on ? c->active_host[k] : 1;
-    c->t += 1;
     return LSAM_OK;
   }
   const float* g1 = flat ? c->eg1 : c->g();
@@ -502,6 +542,110 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
     if ((rc = launch_norm(c, g2, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
   // fused worker update
   if ((rc = launch_update(c, g2, ldg, n, vec4, eta)) != LSAM_OK) return rc;
+  return LSAM_OK;
+}
+
+
+// ---- CUDA-graph replay.  The sequence of a tick is recorded once per variant (gathered / supplied minibatch, rho = 0
+// shortcut or not) after one eager run; afterwards a tick is one graph launch, with the arguments of the three kernels
+// that change from tick to tick (schedule, norm finalisation, update) refreshed in the executable graph.
+int graph_capture(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, bool gather, int64_t budget) {
+  const int64_t l0 = c->launches;
+  LSAM_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+  const int rc = step_enqueue(c, eta, rho, gather, budget);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t e = cudaStreamEndCapture(c->stream, &graph);
+  if (rc != LSAM_OK || e != cudaSuccess || !graph) {
+    if (graph) cudaGraphDestroy(graph);
+    return rc != LSAM_OK ? rc : c->fail(LSAM_ERR_CUDA, std::string("cudaStreamEndCapture: ") + cudaGetErrorString(e));
+  }
+  gs.launches = c->launches - l0;
+  LSAM_CUDA(c, cudaGraphInstantiate(&gs.exec, graph, 0));
+  gs.graph = graph;
+  size_t n = 0;
+  LSAM_CUDA(c, cudaGraphGetNodes(graph, nullptr, &n));
+  std::vector<cudaGraphNode_t> nodes(n);
+  LSAM_CUDA(c, cudaGraphGetNodes(graph, nodes.data(), &n));
+  for (cudaGraphNode_t nd : nodes) {
+    cudaGraphNodeType ty;
+    LSAM_CUDA(c, cudaGraphNodeGetType(nd, &ty));
+    if (ty != cudaGraphNodeTypeKernel) continue;
+    cudaKernelNodeParams kp;
+    LSAM_CUDA(c, cudaGraphKernelNodeGetParams(nd, &kp));
+    if (kp.func == (void*)schedule_kernel) gs.n_sched = nd;
+    else if (kp.func == c->upd_func) gs.n_upd = nd;
+    else if (kp.func == (void*)norm_finalize_kernel && *reinterpret_cast<float**>(kp.kernelParams[6]) != nullptr) gs.n_fin = nd;  // the one that takes rho
+  }
+  if (!gs.n_sched || !gs.n_upd) return c->fail(LSAM_ERR_CUDA, "graph capture: step kernels not found in the captured graph");
+  LSAM_CUDA(c, cudaGraphLaunch(gs.exec, c->stream));  // the capture itself executed nothing: this is the tick
+  return LSAM_OK;
+}
+
+int graph_replay(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, int64_t budget) {
+  const lsam_config& cfg = c->cfg;
+  const bool flat = cfg.model == LSAM_MODEL_FLAT;
+  cudaKernelNodeParams kp;
+  SchedArgs sa = make_sched_args(c, c->t, c->idx(), c->stale(), c->ver(), c->slot(), budget, c->async_on ? c->active_buf() : nullptr);
+  sa.bind();
+  LSAM_CUDA(c, cudaGraphKernelNodeGetParams(gs.n_sched, &kp));
+  kp.kernelParams = sa.ptrs; kp.extra = nullptr;
+  LSAM_CUDA(c, cudaGraphExecKernelNodeSetParams(gs.exec, gs.n_sched, &kp));
+  if (gs.n_fin) {
+    LSAM_CUDA(c, cudaGraphKernelNodeGetParams(gs.n_fin, &kp));
+    FinArgs f;
+    f.partial = *reinterpret_cast<const float**>(kp.kernelParams[0]); f.nchunks = *reinterpret_cast<int64_t*>(kp.kernelParams[1]);
+    f.nused = *reinterpret_cast<int64_t*>(kp.kernelParams[2]); f.rho = rho; f.gamma = cfg.gamma;
+    f.norm_out = *reinterpret_cast<float**>(kp.kernelParams[5]); f.scale_out = *reinterpret_cast<float**>(kp.kernelParams[6]);
+    f.status = c->status(); f.active = c->act();
+    f.bind();
+    kp.kernelParams = f.ptrs; kp.extra = nullptr;
+    LSAM_CUDA(c, cudaGraphExecKernelNodeSetParams(gs.exec, gs.n_fin, &kp));
+  }
+  {
+    const bool vec_unused = false; (void)vec_unused;
+    LSAM_CUDA(c, cudaGraphKernelNodeGetParams(gs.n_upd, &kp));
+    UpdateArgs old = *reinterpret_cast<UpdateArgs*>(kp.kernelParams[0]);
+    UpdateArgs ua = make_update_args(c, old.g, old.ldg, old.n, eta);
+    void* ptrs[1] = {&ua};
+    kp.kernelParams = ptrs; kp.extra = nullptr;
+    LSAM_CUDA(c, cudaGraphExecKernelNodeSetParams(gs.exec, gs.n_upd, &kp));
+  }
+  (void)flat;
+  LSAM_CUDA(c, cudaGraphLaunch(gs.exec, c->stream));
+  c->launches += gs.launches;
+  return LSAM_OK;
+}
+
+void graphs_reset(lsam_ctx* c) {
+  for (auto& gs : c->graphs) {
+    if (gs.exec) cudaGraphExecDestroy(gs.exec);
+    if (gs.graph) cudaGraphDestroy(gs.graph);
+    gs = lsam_ctx::GraphSlot();
+  }
+}
+
+int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
+  const lsam_config& cfg = c->cfg;
+  const Layout& L = c->L;
+  const bool flat = cfg.model == LSAM_MODEL_FLAT;
+  if (flat && (!c->eg1 || !c->eg2)) return c->fail(LSAM_ERR_STATE, "FLAT model: call lsam_set_external_grads first");
+  int64_t done = 0;
+  for (int64_t v : c->t_x) done += v;
+  const int64_t budget = (int64_t)cfg.K * cfg.tau - done;  // iterations still missing to n tau (Algorithm 2, sync trigger)
+  if (budget <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
+  c->ver_at_step.push_back((int)c->t_y);  // centre version current when this tick starts
+  if (c->async_on) host_active_mask(cfg, c->t, budget, c->active_host);
+  int rc;
+  const bool shortcut = rho == 0.f && !flat && !L.g1keep;
+  if ((cfg.flags & LSAM_FLAG_CUDA_GRAPH) && !c->prof.on) {
+    lsam_ctx::GraphSlot& gs = c->graphs[(gather ? 1 : 0) + (shortcut ? 2 : 0)];
+    if (gs.exec) rc = graph_replay(c, gs, eta, rho, budget);
+    else if (gs.warm) rc = graph_capture(c, gs, eta, rho, gather, budget);
+    else { rc = step_enqueue(c, eta, rho, gather, budget); gs.warm = true; }
+  } else {
+    rc = step_enqueue(c, eta, rho, gather, budget);
+  }
+  if (rc != LSAM_OK) return rc;
   for (int k = 0; k < cfg.K; ++k) c->t_x[k] += c->async_on ? c->active_host[k] : 1;
   c->t += 1;
   return LSAM_OK;
@@ -537,6 +681,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   if (!plan(*cfg, L)) return LSAM_ERR_INVALID;
   if (cfg->model != LSAM_MODEL_FLAT && (!d_X || !d_Y)) return LSAM_ERR_INVALID;
   if (workspace_bytes < L.total || (reinterpret_cast<uintptr_t>(d_workspace) & 255) != 0) return LSAM_ERR_WORKSPACE;
+  if ((cfg->flags & LSAM_FLAG_CUDA_GRAPH) && cuda_stream == nullptr) return LSAM_ERR_INVALID;  // the default stream cannot be captured
   lsam_ctx* c = new lsam_ctx();
   c->cfg = *cfg;
   c->L = L;
@@ -717,6 +862,7 @@ int lsam_read_grads_replica(lsam_ctx* c, int pass, int k, float* h_dst) {
 int lsam_set_external_grads(lsam_ctx* c, const float* d_g1, const float* d_g2) {
   if (!c || !d_g1 || !d_g2) return LSAM_ERR_INVALID;
   if (c->cfg.model != LSAM_MODEL_FLAT) return c->fail(LSAM_ERR_INVALID, "external gradients are for the FLAT model only");
+  if (c->eg1 != d_g1 || c->eg2 != d_g2) graphs_reset(c);  // recorded graphs point at the old buffers
   c->eg1 = d_g1;
   c->eg2 = d_g2;
   c->ext_vec4 = ((reinterpret_cast<uintptr_t>(d_g1) | reinterpret_cast<uintptr_t>(d_g2)) & 15) == 0;
@@ -811,6 +957,7 @@ const char* lsam_last_error(const lsam_ctx* c) { return c ? c->err.c_str() : "nu
 void lsam_destroy(lsam_ctx* c) {
   if (!c) return;
   for (cudaEvent_t e : c->prof.pool) cudaEventDestroy(e);
+  graphs_reset(c);
   delete c;
 }
 

@@ -403,6 +403,58 @@ def test_rho_zero_takes_the_single_pass_shortcut_and_matches_oracle(dtype, impl)
     p.close()
 
 
+@pytest.mark.parametrize("kind", ["lsq", "mlp_fp32_async", "resmlp_bf16_tcgen05_noise", "flat"])
+def test_cuda_graph_replay_is_bitwise_identical_to_eager_launches(kind):
+    # LSAM_FLAG_CUDA_GRAPH replays each tick as one graph launch; step size, radius, tick, centre-version history and the
+    # async budget are refreshed in the executable graph, so the run must equal the eagerly launched one bit for bit
+    import torch
+
+    hp = dict(tau=3, lam=0.3, seed=23, stale_max=2)
+    if kind == "lsq":
+        X, y, _ = synth.least_squares_data(300, 24, seed=3)
+        x0 = np.random.default_rng(4).standard_normal((4, 24)).astype(np.float32)
+        mk = lambda fl: G.Lsam(G.make_config(G.MODEL_LSQ, widths=(24,), K=4, batch=16, n_samples=300, flags=fl, **hp),
+                               torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), torch.from_numpy(x0).cuda(), torch.from_numpy(x0.mean(0)).cuda())
+    elif kind == "flat":
+        x0, y0, g1, g2 = synth.flat_problem(4, 1001, seed=6)
+        dg1, dg2 = torch.from_numpy(g1).cuda(), torch.from_numpy(g2).cuda()
+
+        def mk(fl):
+            c = G.Lsam(G.make_config(G.MODEL_FLAT, K=4, flat_d=1001, flags=fl, noise_temp=0.1, **hp), None, None, torch.from_numpy(x0).cuda(), torch.from_numpy(y0).cuda())
+            c.set_external_grads(dg1, dg2)
+            return c
+    else:
+        bf = kind.startswith("resmlp")
+        widths = (64, 128, 128, 16)
+        X, labels = synth.gaussian_mixture(300, widths[0], widths[-1], seed=2)
+        w0 = synth.mlp_init(widths, seed=2)
+        x0 = synth.replicate(w0, 3, jitter=0.01)
+        extra = dict(noise_temp=1e-3) if bf else dict(active_num=170)
+        mk = lambda fl: G.Lsam(G.make_config(G.MODEL_RESMLP if bf else G.MODEL_MLP, widths=widths, K=3, batch=48, n_samples=300, flags=fl,
+                                             gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32, **extra, **hp),
+                               torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda(), torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()  # the default stream cannot be captured
+    with torch.cuda.stream(stream):
+        a, b = mk(0), mk(G.FLAG_CUDA_GRAPH)
+    assert b.stream.cuda_stream == stream.cuda_stream and stream.cuda_stream != 0
+    for t in range(14):
+        eta = 0.02 + 0.001 * t
+        rho = 0.0 if t in (4, 5, 9) else 0.03 + 0.002 * t
+        for c in (a, b):
+            c.step(eta, rho)
+            if c.should_couple():
+                assert c.couple() == 0
+    assert a.launch_count() == b.launch_count()
+    np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
+    np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
+    np.testing.assert_array_equal(a.read_state()["v"], b.read_state()["v"])
+    assert a.counters()[0] == b.counters()[0] and (a.counters()[2] == b.counters()[2]).all()
+    assert a.status() == 0 and b.status() == 0
+    a.close()
+    b.close()
+
+
 def test_step_refused_while_sync_is_due():
     import torch
 
