@@ -432,7 +432,9 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
     const double n1 = std::sqrt(ss);
     o->gn1[k] = n1;
     // look-back map: x~ = x + rho g1 / (||g1|| + gamma)
-    for (int64_t j = 0; j < d; ++j) xp[j] = x[j] + rho * g1[j] / (n1 + c.gamma);
+    // (bf16 mode: the ascent gradient is a stored backward quantity, so the perturbation uses its bf16 rounding;
+    //  its norm n1 is taken before rounding)
+    for (int64_t j = 0; j < d; ++j) xp[j] = x[j] + rho * o->net.q(g1[j]) / (n1 + c.gamma);
     // descent gradient at x~ on the same minibatch
     if (c.model == ORACLE_MODEL_FLAT) {
       for (int64_t j = 0; j < d; ++j) g2[j] = (double)o->eg2[(size_t)k * d + j];

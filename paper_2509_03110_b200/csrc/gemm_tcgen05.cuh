@@ -146,7 +146,9 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool a_mn, bool 
 }  // namespace tc
 
 // ------------------------------------------------------------------------------------------------ epilogue parameters
-enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3 };
+// TC_EPI_WGRAD_BF16: the weight gradient is stored rounded to bf16 (ascent pass: it only feeds the perturbation, whose
+// result is rounded to bf16 anyway; its norm is still taken from the fp32 accumulators).
+enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3, TC_EPI_WGRAD_BF16 = 4 };
 
 struct TcEpi {
   // forward: bias (operand copy), out / skip / mask [Z, M, ldb]; head: logits fp32 [Z, M, ldb]
@@ -293,6 +295,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // ------------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
     const int quad = warp & 3;
     int sbuf_sel = 0;  // staging buffer of the next output block (wgrad)
+    uint8_t* sbuf_cur = stage;
     int as = 0;
     uint32_t aph = 0;
     bool ok = true;
@@ -313,7 +316,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         tc::tmem_ld32(taddr + (uint32_t)(c * 32), r);
         tc::tmem_ld_wait();
         const int nb = n0 + c * 32;
-        if (EPI == TC_EPI_WGRAD) {
+        if (EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) {
           // The warp's 32 x 32 fp32 block goes to shared memory in the 128-byte-swizzled layout of the output tensor
           // map (row = lane, 16-byte chunk q stored at position q ^ (row % 8)), then one TMA store writes it to the
           // gradient rows (clipped at the ragged edges).  Two buffers per warp: the store of a chunk overlaps the
@@ -322,20 +325,43 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (mrow0 < M && nb < N) {  // warp-uniform: blocks wholly outside the matrix are neither staged nor stored
 #pragma unroll
             for (int j = 0; j < 32; ++j) ssq = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ssq);  // zero-filled edges add 0
-            uint8_t* sbuf = stage + (warp - 2) * 8192 + sbuf_sel * 4096;
-            sbuf_sel ^= 1;
-            // at most one store may still be reading shared memory: the previous one, which used the other buffer
-            if (lane == 0) tc::bulk_wait_read<1>();
-            __syncwarp();
+            // fp32: one 32-column block per store.  bf16: two consecutive blocks share one buffer (rows of 64 bf16 = 128
+            // bytes, the same swizzle) and are stored together after the second one, or after the last valid one.
+            const bool first_half = (EPI == TC_EPI_WGRAD) || ((c & 1) == 0);
+            const bool last_half = (EPI == TC_EPI_WGRAD) || ((c & 1) == 1) || (nb + 32 >= N);
+            if (first_half) {
+              sbuf_cur = stage + (warp - 2) * 8192 + sbuf_sel * 4096;
+              sbuf_sel ^= 1;
+              // at most one store may still be reading shared memory: the previous one, which used the other buffer
+              if (lane == 0) tc::bulk_wait_read<1>();
+              __syncwarp();
+            }
+            if (EPI == TC_EPI_WGRAD) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q)
-              *reinterpret_cast<float4*>(sbuf + lane * 128 + ((q ^ (lane & 7)) << 4)) =
-                  make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
-            tc::fence_proxy_async();
-            __syncwarp();
-            if (lane == 0) {
-              tc::tma_store_3d(&map_c, sbuf, nb, mrow0, z);
-              tc::bulk_commit();
+              for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<float4*>(sbuf_cur + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                    make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+            } else {
+#pragma unroll
+              for (int q = 0; q < 4; ++q) {
+                uint4 pk;
+                uint32_t* pw = reinterpret_cast<uint32_t*>(&pk);
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                  __nv_bfloat162 two = __floats2bfloat162_rn(__uint_as_float(r[8 * q + 2 * h]), __uint_as_float(r[8 * q + 2 * h + 1]));
+                  pw[h] = *reinterpret_cast<uint32_t*>(&two);
+                }
+                const int qq = (c & 1) * 4 + q;  // 16-byte chunk of the 128-byte row
+                *reinterpret_cast<uint4*>(sbuf_cur + lane * 128 + ((qq ^ (lane & 7)) << 4)) = pk;
+              }
+            }
+            if (last_half) {
+              tc::fence_proxy_async();
+              __syncwarp();
+              if (lane == 0) {
+                tc::tma_store_3d(&map_c, sbuf_cur, EPI == TC_EPI_WGRAD ? nb : nb - (c & 1) * 32, mrow0, z);
+                tc::bulk_commit();
+              }
             }
           }
         } else if (m < M && nb < N) {
@@ -436,7 +462,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
         }
       }
-      if (EPI == TC_EPI_WGRAD && ep.partial != nullptr) {
+      if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && ep.partial != nullptr) {
         // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows
         const float tot = warp_sum(ssq);
         if (lane == 0) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)mt * n_tiles + nt) * 4 + quad] = tot;
@@ -446,7 +472,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (lane == 0) tc::mbar_arrive(&acc_empty[as]);
       if (++as == 2) { as = 0; aph ^= 1u; }
     }
-    if (EPI == TC_EPI_WGRAD && lane == 0) tc::bulk_wait_all<0>();  // every gradient block has reached global memory
+    if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && lane == 0) tc::bulk_wait_all<0>();  // every gradient block has reached global memory
     if (!ok && lane == 0) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
   }
 
@@ -472,10 +498,12 @@ struct TcBuffers {
   bf16* act[9]; uint8_t* mask[9]; float* logits; bf16* dz[2]; bf16* dh[2]; int* status;
   int ldb;
   float* partial; int64_t ld_partial;  // per-replica slots for the fused sum of squares
+  bf16* g1b;                           // [Z, ld] bf16 copy of the ascent gradient
 };
 
 struct TcGemm {
   CUtensorMap map_a, map_b, map_c;  // map_c: fp32 output of wgrad (a copy of map_a elsewhere, unused)
+  CUtensorMap map_c16;              // wgrad only: the same output rows in the bf16 ascent-gradient buffer
   int M = 0, N = 0, Kd = 0, block_n = 0;
   TcEpi ep{};
   bool valid = false;
@@ -577,6 +605,8 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.block_n);
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
+      // the same rows of the bf16 ascent-gradient buffer
+      ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
       slot += (int)(ceil_div(ly.out, kTcBlockM) * ceil_div(ly.in, g.block_n) * 4);
@@ -629,7 +659,12 @@ inline int tc_forward(const TcPlan& P, int l, cudaStream_t stream) {
   return (l == P.n_layers - 1) ? tc_launch<false, true, TC_EPI_FWD_HEAD>(P, P.fwd[l], stream)
                                : tc_launch<false, true, TC_EPI_FWD_HIDDEN>(P, P.fwd[l], stream);
 }
-inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<false, false, TC_EPI_WGRAD>(P, P.wgrad[l], stream); }
+inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream, bool out_bf16) {
+  if (!out_bf16) return tc_launch<false, false, TC_EPI_WGRAD>(P, P.wgrad[l], stream);
+  TcGemm g = P.wgrad[l];
+  g.map_c = g.map_c16;
+  return tc_launch<false, false, TC_EPI_WGRAD_BF16>(P, g, stream);
+}
 inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, true, TC_EPI_DGRAD>(P, P.dgrad[l], stream); }
 
 }  // namespace lsam

@@ -38,7 +38,7 @@ struct Layout {
   int64_t nchunks = 0;
   bool vec4 = true;
   // byte offsets into the workspace
-  size_t x, v, g, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status;
+  size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status;
   size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage;
   size_t total = 0;
 };
@@ -110,6 +110,8 @@ bool plan(const lsam_config& c, Layout& L) {
   L.x = take(4 * K * ld);
   L.v = take(4 * K * ld);
   L.g = flat ? 0 : take(4 * K * ld);
+  // tensor-core path: the ascent gradient is kept in bf16 (it only feeds the perturbation, itself rounded to bf16)
+  L.g1b = (!flat && bf && c.model != LSAM_MODEL_LSQ) ? take(2 * K * ld) : 0;
   L.g1keep = (!flat && (c.flags & LSAM_FLAG_KEEP_G1)) ? take(4 * K * ld) : 0;
   L.xpkeep = (!flat && bf && (c.flags & LSAM_FLAG_KEEP_G1)) ? take(esz * K * ld) : 0;  // x~ survives the update
   L.xop = take(esz * K * ld);  // fp32: perturbed point x~;  bf16: operand copy of x, overwritten by x~
@@ -298,13 +300,13 @@ int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, 
   return LSAM_OK;
 }
 
-template <typename TP>
-int launch_perturb(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4) {
+template <typename TP, typename TG>
+int launch_perturb(lsam_ctx* c, const TG* g, int64_t ldg, int64_t n, bool vec4) {
   TP* xt = c->at<TP>(c->L.xop);
   const int64_t per = (int64_t)kPertThreads * kPertIter * (vec4 ? 4 : 1);
   dim3 grid((unsigned)ceil_div(n, per), c->cfg.K);
-  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
-  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
+  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP, TG, (sizeof(TP) == 2 && sizeof(TG) == 4)><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
+  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP, TG, (sizeof(TP) == 2 && sizeof(TG) == 4)><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
   return LSAM_OK;
 }
 
@@ -392,8 +394,9 @@ int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N
 }
 
 // One gradient pass of the classifier at the parameters P ([K, ld], type T); gradient -> g, loss -> loss_out (nullable).
+// g_bf16 (tensor-core path only): store the gradient rounded to bf16 in the g1b buffer instead of fp32 in g.
 template <typename T>
-int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
+int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
   const Layout& L = c->L;
   const int K = c->cfg.K, B = c->cfg.batch;
   const int nl = (int)L.layers.size();
@@ -433,11 +436,18 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
     const LayerInfo& li = L.layers[l];
     const T* dz = c->at<T>(L.dz[cur]);
     const T* a_in = c->at<T>(L.act[l]);
-    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad,
-        c->use_tc ? c->at<float>(L.partial) : nullptr, L.nchunks, c->use_tc ? c->tc.bias_slot0[l] : 0, c->act()));
+    {
+      float* part = c->use_tc ? c->at<float>(L.partial) : nullptr;
+      const int slot0 = c->use_tc ? c->tc.bias_slot0[l] : 0;
+      dim3 bgrid((unsigned)ceil_div(li.out, 8), K);
+      if (g_bf16)
+        LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, bf16><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->at<bf16>(L.g1b), ld, li.b_pad, part, L.nchunks, slot0, c->act()));
+      else
+        LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad, part, L.nchunks, slot0, c->act()));
+    }
     if (c->use_tc) {
       int trc = 0;
-      LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream));
+      LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream, g_bf16));
       if (trc == 0 && l > 0) LAUNCH(c, LSAM_PROF_GEMM_DGRAD, trc = tc_dgrad(c->tc, l, c->stream));
       if (trc != 0) return c->fail(LSAM_ERR_CUDA, "tcgen05 backward launch failed");
       cur ^= 1;
@@ -465,7 +475,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out) {
 }
 
 // Gradient of the minibatch loss at the parameters held in `params` (x master, or the operand buffer).
-int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out) {
+int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false) {
   const lsam_config& cfg = c->cfg;
   if (cfg.model == LSAM_MODEL_LSQ) {
     const float* P = perturbed ? c->at<float>(c->L.xop) : c->x();
@@ -473,8 +483,8 @@ int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out) {
         c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, cfg.widths[0], c->g(), c->L.ld, loss_out, c->act()));
     return LSAM_OK;
   }
-  if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out);
-  return mlp_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out);
+  if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out, g_bf16 && c->use_tc);
+  return mlp_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out, false);
 }
 
 int refresh_operand_copy(lsam_ctx* c) {
@@ -528,11 +538,16 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
     return LSAM_OK;
   }
   const float* g1 = flat ? c->eg1 : c->g();
-  if (!flat && (rc = grad_pass(c, false, c->loss())) != LSAM_OK) return rc;
-  if (!flat && L.g1keep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
+  const bool g1_bf16 = !flat && c->use_tc;  // tensor-core path: ascent gradient stored as bf16 in g1b
+  if (!flat && (rc = grad_pass(c, false, c->loss(), g1_bf16)) != LSAM_OK) return rc;
+  if (!flat && L.g1keep) {
+    if (g1_bf16) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.g1keep), c->at<bf16>(L.g1b), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
+    else LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
+  }
   if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
-  if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16>(c, g1, ldg, n, vec4);
-  else rc = launch_perturb<float>(c, g1, ldg, n, vec4);
+  if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
+  else if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
+  else rc = launch_perturb<float, float>(c, g1, ldg, n, vec4);
   if (rc != LSAM_OK) return rc;
   if (L.xpkeep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.xpkeep), c->at<bf16>(L.xop), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   // descent gradient at the perturbed point, same minibatch
@@ -713,6 +728,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     b.status = c->status();
     b.ldb = L.ldb;
     b.partial = c->at<float>(L.partial); b.ld_partial = L.nchunks;
+    b.g1b = c->at<bf16>(L.g1b);
     c->tc.active = c->act();
     std::vector<TcLayer> tl;
     for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
@@ -839,8 +855,15 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
       LSAM_CUDA(c, cudaMemcpyAsync(tmp, src + (size_t)k * L.d, sizeof(float) * L.d, cudaMemcpyDeviceToDevice, c->stream));
     } else {
       if (pass == 1 && !L.g1keep) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(1) needs LSAM_FLAG_KEEP_G1");
-      const float* src = pass == 1 ? c->at<float>(L.g1keep) : c->g();
-      rc = seg_copy<false>(c, src + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
+      if (pass == 1 && c->use_tc) {  // kept as stored: bf16
+        int64_t maxlen = 0;
+        for (int i = 0; i < L.seg.n; ++i) maxlen = L.seg.len[i] > maxlen ? L.seg.len[i] : maxlen;
+        dim3 grid((unsigned)ceil_div(maxlen, 256), L.seg.n, 1);
+        LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(c->at<bf16>(L.g1keep) + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
+      } else {
+        const float* src = pass == 1 ? c->at<float>(L.g1keep) : c->g();
+        rc = seg_copy<false>(c, src + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
+      }
     }
     if (rc != LSAM_OK) return rc;
     LSAM_CUDA(c, cudaMemcpyAsync(h_dst + (size_t)(k - k_begin) * L.d, tmp, sizeof(float) * L.d, cudaMemcpyDeviceToHost, c->stream));

@@ -308,9 +308,10 @@ __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float
 // order, then the xor-shuffle tree (a fixed order).  grid (ceil(out / 8), K), block 256.
 // If partial != nullptr the block also writes the sum of squares of its 8 bias gradients (warps in ascending order)
 // to partial[z * ld_partial + slot0 + blockIdx.x], for the fused gradient norm.
-template <typename TA>
+// TG = float, or bf16 for the ascent pass of the tensor-core path (same packed bf16 view as its weight gradients).
+template <typename TA, typename TG>
 __global__ void __launch_bounds__(256)
-bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off,
+bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, TG* __restrict__ g, int64_t ld_g, int64_t b_off,
                  float* __restrict__ partial, int64_t ld_partial, int slot0, const int32_t* __restrict__ active) {
   __shared__ float sq[8];
   if (active != nullptr && !active[blockIdx.y]) return;
@@ -321,7 +322,7 @@ bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, float* __re
     const TA* p = dz + ((int64_t)z * out + o) * ldb;
     for (int b = lane; b < B; b += 32) s += to_float(p[b]);
     s = warp_sum(s);
-    if (lane == 0) g[(int64_t)z * ld_g + b_off + o] = s;
+    if (lane == 0) g[(int64_t)z * ld_g + b_off + o] = from_float<TG>(s);
   }
   if (partial != nullptr) {
     if (lane == 0) sq[w] = s * s;

@@ -115,16 +115,18 @@ norm_finalize_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t
 constexpr int kPertThreads = 256;
 constexpr int kPertIter = 4;
 
-template <int VEC, typename TP>
+// TG = type of the stored gradient: float, or bf16 on the tensor-core path (packed bf16 rows of stride ldg).
+// ROUND_G: an fp32 gradient is rounded to bf16 before use, so that every path of the BF16 mode perturbs with the same value.
+template <int VEC, typename TP, typename TG, bool ROUND_G>
 __global__ void __launch_bounds__(kPertThreads)
-perturb_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ g, int64_t ldg, int64_t n,
+perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ g, int64_t ldg, int64_t n,
                const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active) {
   const int k = blockIdx.y;
   if (active != nullptr && !active[k]) return;
   const float sc = scale[k];
   const int64_t base = (int64_t)blockIdx.x * ((int64_t)kPertThreads * VEC * kPertIter);
   const float* xr = x + (int64_t)k * ldx;
-  const float* gr = g + (int64_t)k * ldg;
+  const TG* gr = g + (int64_t)k * ldg;
   TP* tr = xt + (int64_t)k * ldt;
   if (VEC == 4) {
     float4 xv[kPertIter], gv[kPertIter];
@@ -133,7 +135,18 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict
       const int64_t j = base + ((int64_t)i * kPertThreads + threadIdx.x) * 4;
       if (j < n) {
         xv[i] = *reinterpret_cast<const float4*>(xr + j);
-        gv[i] = __ldcs(reinterpret_cast<const float4*>(gr + j));
+        if (sizeof(TG) == 4) {
+          gv[i] = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(gr) + j));
+          if (ROUND_G) {
+            gv[i].x = to_float(__float2bfloat16_rn(gv[i].x)); gv[i].y = to_float(__float2bfloat16_rn(gv[i].y));
+            gv[i].z = to_float(__float2bfloat16_rn(gv[i].z)); gv[i].w = to_float(__float2bfloat16_rn(gv[i].w));
+          }
+        } else {
+          const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(gr) + j));
+          const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+          const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+          gv[i] = make_float4(lo.x, lo.y, hi.x, hi.y);
+        }
       }
     }
 #pragma unroll
@@ -157,7 +170,7 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict
 #pragma unroll
     for (int i = 0; i < kPertIter; ++i) {
       const int64_t j = base + (int64_t)i * kPertThreads + threadIdx.x;
-      if (j < n) tr[j] = from_float<TP>(fmaf(sc, gr[j], xr[j]));
+      if (j < n) tr[j] = from_float<TP>(fmaf(sc, ROUND_G ? to_float(__float2bfloat16_rn(to_float(gr[j]))) : to_float(gr[j]), xr[j]));
     }
   }
 }

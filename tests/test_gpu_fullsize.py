@@ -58,12 +58,15 @@ def test_full_shape_step_against_oracle_on_selected_replicas(name, both_passes):
     ocfg = _oracle_cfg(w, 1)
     rho, gam = float(np.float32(w["rho"])), float(np.float32(bench.GAMMA))
 
+    def q16(a):  # bf16 rounding (via fp32), as the BF16 mode applies to the stored ascent gradient
+        return torch.from_numpy(np.asarray(a, np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
+
     def one(k):
         l1, g1 = O.loss_grad(ocfg, X, Y, x0_rows[k], idx[k])
         out = dict(l1=l1, g1=g1)
         if both_passes:
             nrm = np.linalg.norm(g1)
-            xp = x0_rows[k] + rho * g1 / (nrm + gam)
+            xp = x0_rows[k] + rho * q16(g1) / (nrm + gam)
             out["g2"] = O.loss_grad(ocfg, X, Y, xp, idx[k])[1]
         return out
 
@@ -77,7 +80,7 @@ def test_full_shape_step_against_oracle_on_selected_replicas(name, both_passes):
         # perturbed point as stored (bf16 operand): sampled elements against Eq. 3 evaluated with the oracle's gradient
         xp_gpu = ctx.read_grads_replica(3, k)
         sel = np.random.default_rng(k).integers(0, ctx.d, 20000)
-        want = x0_rows[k][sel] + rho * r["g1"][sel] / (np.linalg.norm(r["g1"]) + gam)
+        want = x0_rows[k][sel] + rho * q16(r["g1"][sel]) / (np.linalg.norm(r["g1"]) + gam)
         want = torch.from_numpy(want.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
         assert rel_l2(xp_gpu[sel], want) <= 1e-3
         if both_passes:
