@@ -92,7 +92,7 @@ def work_model(w, tc):
     op = 2 if w["bf16"] else 4
     out = {}
     out["norm"] = dict(bytes=0.0 if tc else 4.0 * K * d)                     # read g1 (fused into the wgrad epilogue on the tensor-core path)
-    out["perturb"] = dict(bytes=(4.0 + 4.0 + op) * K * d)                    # read x, g1; write x~
+    out["perturb"] = dict(bytes=(4.0 + (2.0 if tc else 4.0) + op) * K * d)   # read x, g1 (bf16 on the tensor-core path); write x~
     out["update"] = dict(bytes=(4.0 + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2, x rw, v rw, operand copy; y, acc rw
     if w["model"] in (MLP, RESMLP):
         ws = w["widths"]
@@ -103,7 +103,7 @@ def work_model(w, tc):
             f_fwd += 2.0 * B * i * o
             b_fwd += op * (i * o + B * i + B * o)
             f_wg += 2.0 * B * i * o
-            b_wg += 4.0 * i * o + op * B * (i + o)
+            b_wg += (3.0 if tc else 4.0) * i * o + op * B * (i + o)         # tensor-core path: bf16 in the ascent pass, fp32 in the descent pass
             if l > 0:
                 f_dg += 2.0 * B * i * o
                 b_dg += op * (i * o + B * i + B * o)

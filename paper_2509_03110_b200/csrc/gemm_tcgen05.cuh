@@ -158,20 +158,24 @@ struct TcEpi {
   const bf16* dh_next;  bf16* dh_out;  bf16* dz_prev;  const uint8_t* mask_prev;
   // wgrad: g[z * ld_g + w_off + m * ldw + n]
   float* g;  int64_t ld_g, w_off;  int ldw;
-  // wgrad: sum of squares of every 32-row block of the tile -> partial[z * ld_partial + slot0 + (mt * n_tiles + nt) * 4 + quad]
+  // wgrad: sum of squares of every 32-row block of the tile -> partial[z * ld_partial + slot0 + (mt * n_tiles + nt) * 8 + epilogue warp]
   float* partial;  int64_t ld_partial;  int slot0;
   int ldb;  // sample stride of the feature-major buffers (multiple of 16)
 };
 
 constexpr int kTcBlockM = 128;
 constexpr int kTcBlockK = 64;
-constexpr int kTcThreads = 192;  // warp 0: TMA producer, warp 1: MMA issuer + tensor-memory owner, warps 2-5: epilogue
+// warp 0: TMA producer, warp 1: MMA issuer + tensor-memory owner, warps 2-9: epilogue.  Two epilogue warps share each
+// tensor-memory lane quadrant (warp % 4) and take alternate pairs of 32-column blocks, so that one drains while the other
+// converts and stores.
+constexpr int kTcThreads = 320;
+constexpr int kTcEpiWarps = 8;
 
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_stages() { return BLOCK_N == 256 ? 4 : (BLOCK_N == 128 ? 6 : 8); }
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + BLOCK_N) * kTcBlockK * 2; }
-constexpr int kTcStageOutBytes = 4 * 2 * 4096;  // wgrad epilogue staging: two 32 x 32 fp32 blocks (128B-swizzled) per epilogue warp
+constexpr int kTcStageOutBytes = 8 * 4096;  // wgrad epilogue staging: one 32-row x 128-byte block (128B-swizzled) per epilogue warp
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_smem_bytes() {
   return tc_stages<BLOCK_N>() * tc_stage_bytes<BLOCK_N>() + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTcStageOutBytes;
@@ -212,7 +216,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], 4); }
+    for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], kTcEpiWarps); }
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
@@ -294,7 +298,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else {
     // ------------------------------------------------------------------ epilogue (4 warps, one TMEM lane quadrant each)
     const int quad = warp & 3;
-    int sbuf_sel = 0;  // staging buffer of the next output block (wgrad)
+    const int ew = warp - 2;       // epilogue warp 0..7
+    const int half = ew >> 2;      // which of the two warps of this quadrant
     uint8_t* sbuf_cur = stage;
     int as = 0;
     uint32_t aph = 0;
@@ -312,6 +317,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) bias = to_float(ep.bias[(int64_t)z * ep.ld_p + m]);
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
+        if (((c >> 1) & 1) != half) continue;  // pairs of blocks alternate between the two warps of a quadrant
         uint32_t r[32];
         tc::tmem_ld32(taddr + (uint32_t)(c * 32), r);
         tc::tmem_ld_wait();
@@ -330,10 +336,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             const bool first_half = (EPI == TC_EPI_WGRAD) || ((c & 1) == 0);
             const bool last_half = (EPI == TC_EPI_WGRAD) || ((c & 1) == 1) || (nb + 32 >= N);
             if (first_half) {
-              sbuf_cur = stage + (warp - 2) * 8192 + sbuf_sel * 4096;
-              sbuf_sel ^= 1;
-              // at most one store may still be reading shared memory: the previous one, which used the other buffer
-              if (lane == 0) tc::bulk_wait_read<1>();
+              sbuf_cur = stage + ew * 4096;
+              // the previous store of this warp must have finished reading the buffer (the other warp of the quadrant
+              // keeps the SM busy meanwhile)
+              if (lane == 0) tc::bulk_wait_read<0>();
               __syncwarp();
             }
             if (EPI == TC_EPI_WGRAD) {
@@ -465,7 +471,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && ep.partial != nullptr) {
         // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows
         const float tot = warp_sum(ssq);
-        if (lane == 0) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)mt * n_tiles + nt) * 4 + quad] = tot;
+        if (lane == 0) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)mt * n_tiles + nt) * kTcEpiWarps + ew] = tot;
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -552,12 +558,12 @@ inline bool tc_make_map(CUtensorMap* m, const T* base, uint64_t cols, uint64_t r
 
 inline int tc_pick_block_n(int n) { return n > 128 ? 256 : (n > 64 ? 128 : 64); }
 // Partial-sum slots one replica needs when the sum of squares is fused into the weight-gradient epilogue:
-// four per output tile (one per 32-row block) plus one per 8 bias units.
+// eight per output tile (one per epilogue warp) plus one per 8 bias units.
 inline int64_t tc_norm_slots(const lsam_config& c) {
   int64_t n = 0;
   for (int l = 0; l < c.n_layers; ++l) {
     const int in = c.widths[l], out = c.widths[l + 1];
-    n += ceil_div(out, kTcBlockM) * ceil_div(in, tc_pick_block_n(in)) * 4 + ceil_div(out, 8);
+    n += ceil_div(out, kTcBlockM) * ceil_div(in, tc_pick_block_n(in)) * kTcEpiWarps + ceil_div(out, 8);
   }
   return n;
 }
@@ -609,7 +615,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
-      slot += (int)(ceil_div(ly.out, kTcBlockM) * ceil_div(ly.in, g.block_n) * 4);
+      slot += (int)(ceil_div(ly.out, kTcBlockM) * ceil_div(ly.in, g.block_n) * kTcEpiWarps);
       P.bias_slot0[l] = slot;
       slot += (int)ceil_div(ly.out, 8);
       g.valid = ok;

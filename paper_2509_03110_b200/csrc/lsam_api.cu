@@ -545,7 +545,11 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
     else LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   }
   if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
-  if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
+  if (g1_bf16 && vec4 && n % 8 == 0) {
+    dim3 pgrid((unsigned)ceil_div(n, (int64_t)kPertThreads * 8 * kPert8Iter), cfg.K);
+    LAUNCH(c, LSAM_PROF_PERTURB, perturb8_kernel<<<pgrid, kPertThreads, 0, c->stream>>>(c->x(), L.ld, c->at<bf16>(L.g1b), ldg, n, c->scale(), c->at<bf16>(L.xop), L.ld, c->act()));
+    rc = LSAM_OK;
+  } else if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
   else if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
   else rc = launch_perturb<float, float>(c, g1, ldg, n, vec4);
   if (rc != LSAM_OK) return rc;

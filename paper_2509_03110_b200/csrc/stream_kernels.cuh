@@ -175,6 +175,50 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ 
   }
 }
 
+// Tensor-core path: gradient and operand are both bf16, so a thread takes 8 elements per access (two 128-bit loads of x,
+// one of g, one 128-bit store).  Requires 16-byte aligned rows (ld multiples of 8).  grid (chunks, K).
+constexpr int kPert8Iter = 2;
+__global__ void __launch_bounds__(kPertThreads)
+perturb8_kernel(const float* __restrict__ x, int64_t ldx, const bf16* __restrict__ g, int64_t ldg, int64_t n,
+                const float* __restrict__ scale, bf16* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active) {
+  const int k = blockIdx.y;
+  if (active != nullptr && !active[k]) return;
+  const float sc = scale[k];
+  const int64_t base = (int64_t)blockIdx.x * ((int64_t)kPertThreads * 8 * kPert8Iter);
+  const float* xr = x + (int64_t)k * ldx;
+  const bf16* gr = g + (int64_t)k * ldg;
+  bf16* tr = xt + (int64_t)k * ldt;
+  float4 xa[kPert8Iter], xb[kPert8Iter];
+  uint4 gv[kPert8Iter];
+#pragma unroll
+  for (int i = 0; i < kPert8Iter; ++i) {
+    const int64_t j = base + ((int64_t)i * kPertThreads + threadIdx.x) * 8;
+    if (j < n) {
+      xa[i] = *reinterpret_cast<const float4*>(xr + j);
+      xb[i] = *reinterpret_cast<const float4*>(xr + j + 4);
+      gv[i] = __ldcs(reinterpret_cast<const uint4*>(gr + j));
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < kPert8Iter; ++i) {
+    const int64_t j = base + ((int64_t)i * kPertThreads + threadIdx.x) * 8;
+    if (j < n) {
+      const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv[i].x));
+      const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv[i].y));
+      const float2 g2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv[i].z));
+      const float2 g3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gv[i].w));
+      __nv_bfloat162 o0 = __floats2bfloat162_rn(fmaf(sc, g0.x, xa[i].x), fmaf(sc, g0.y, xa[i].y));
+      __nv_bfloat162 o1 = __floats2bfloat162_rn(fmaf(sc, g1.x, xa[i].z), fmaf(sc, g1.y, xa[i].w));
+      __nv_bfloat162 o2 = __floats2bfloat162_rn(fmaf(sc, g2.x, xb[i].x), fmaf(sc, g2.y, xb[i].y));
+      __nv_bfloat162 o3 = __floats2bfloat162_rn(fmaf(sc, g3.x, xb[i].z), fmaf(sc, g3.y, xb[i].w));
+      uint4 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&o0); pk.y = *reinterpret_cast<uint32_t*>(&o1);
+      pk.z = *reinterpret_cast<uint32_t*>(&o2); pk.w = *reinterpret_cast<uint32_t*>(&o3);
+      *reinterpret_cast<uint4*>(tr + j) = pk;
+    }
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ S6 fused update
 // One thread owns VEC consecutive columns for ALL replicas (k ascending), so that the centre versions are
 // re-read from cache and the iterate accumulator is read and written once per column:
