@@ -44,7 +44,7 @@ NOMINAL_HBM_GBS, FALLBACK_HBM_GBS, FALLBACK_BF16_TF = 8000.0, 6650.0, 1590.0
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x max SM clock
 # ncu counters of one update_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) at the c4 shape with K = 4
 # replicas, see profiles/dram_traffic_c4_k4.md; traffic grows with (22 K + 12) d, so it is scaled to the K of the run.
-NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=6647730688.0)
+NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=None)  # to be re-taken: the kernel changed (bf16 gradient input)
 
 
 def param_count(w):
@@ -93,7 +93,7 @@ def work_model(w, tc):
     out = {}
     out["norm"] = dict(bytes=0.0 if tc else 4.0 * K * d)                     # read g1 (fused into the wgrad epilogue on the tensor-core path)
     out["perturb"] = dict(bytes=(4.0 + (2.0 if tc else 4.0) + op) * K * d)   # read x, g1 (bf16 on the tensor-core path); write x~
-    out["update"] = dict(bytes=(4.0 + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2, x rw, v rw, operand copy; y, acc rw
+    out["update"] = dict(bytes=((2.0 if tc else 4.0) + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2 (bf16 on the tensor-core path), x rw, v rw, operand copy; y, acc rw
     if w["model"] in (MLP, RESMLP):
         ws = w["widths"]
         f_fwd = f_dg = f_wg = 0.0
@@ -103,7 +103,7 @@ def work_model(w, tc):
             f_fwd += 2.0 * B * i * o
             b_fwd += op * (i * o + B * i + B * o)
             f_wg += 2.0 * B * i * o
-            b_wg += (3.0 if tc else 4.0) * i * o + op * B * (i + o)         # tensor-core path: bf16 in the ascent pass, fp32 in the descent pass
+            b_wg += (2.0 if tc else 4.0) * i * o + op * B * (i + o)         # tensor-core path: the gradient is written as bf16
             if l > 0:
                 f_dg += 2.0 * B * i * o
                 b_dg += op * (i * o + B * i + B * o)
@@ -466,8 +466,8 @@ def main():
     launches_per_step = tn / args.steps
     roof = dict(kernel=top, share_of_kernel_time=shares.get(top), traffic=None, kernel_time_shares=shares)
     if top == "update" and args.workload == NCU_UPDATE_TRAFFIC["workload"] and w["bf16"]:
-        roof["traffic"] = NCU_UPDATE_TRAFFIC["bytes"] * (22.0 * w["K"] + 12.0) / (22.0 * NCU_UPDATE_TRAFFIC["K"] + 12.0)
-        roof["traffic_source"] = "ncu at K=4 scaled by (22K+12)/(22*4+12); algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
+        roof["traffic"] = NCU_UPDATE_TRAFFIC["bytes"] * (20.0 * w["K"] + 12.0) / (20.0 * NCU_UPDATE_TRAFFIC["K"] + 12.0) if NCU_UPDATE_TRAFFIC["bytes"] else None
+        roof["traffic_source"] = "ncu at K=4 scaled by (20K+12)/(20*4+12); algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
     if top in ("gemm_fwd", "gemm_dgrad") and ctx.uses_tcgen05():
         ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
         roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_sustained"], peak_source=f"{pk['src']} (sustained bf16)")

@@ -66,9 +66,9 @@ enum {
  *  RESMLP as MLP, but every hidden layer with equal input and output width is h_{l+1} = h_l + relu(W_l h_l + b_l).
  *  FLAT   no model: the two gradients of a step are buffers supplied with lsam_set_external_grads().
  * gemm_dtype BF16: matmul operands (weights, biases, inputs, stored activations and backward signals) are
- * rounded to bf16, products accumulate in fp32, the descent gradient and all optimiser state stay fp32.  On the
- * tensor-core path the ascent gradient g1, whose only uses are its norm (taken from the fp32 accumulators) and the
- * perturbation (rounded to bf16 anyway), is stored rounded to bf16.                                       */
+ * rounded to bf16, products accumulate in fp32, all optimiser state (x, v, centre, accumulator) stays fp32.  The
+ * weight-gradient matmul delivers g1 and g2 in the operand type: they are used rounded to bf16 (stored as bf16 on the
+ * tensor-core path), while their norms are taken from the fp32 accumulators.                               */
 typedef struct {
   int32_t model;      /* LSAM_MODEL_*                                                               */
   int32_t n_layers;   /* weight matrices (MLP/RESMLP: 1..8; LSQ: 1; FLAT: 0)                        */

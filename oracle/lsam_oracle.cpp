@@ -446,7 +446,8 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
     o->gn2[k] = std::sqrt(ss2);
     // sampler: momentum step on G = g2 + lambda (x - y); the pull is evaluated at x_k, not at x~
     for (int64_t j = 0; j < d; ++j) {
-      const double G = g2[j] + c.lambda * (x[j] - yk[j]);
+      // (bf16 mode: the weight-gradient matmul delivers its result in the operand type, so the sampler sees q(g2))
+      const double G = o->net.q(g2[j]) + c.lambda * (x[j] - yk[j]);
       v[j] = c.mu * v[j] + G;
       x[j] = c.nesterov ? x[j] - eta * (G + c.mu * v[j]) : x[j] - eta * v[j];
     }

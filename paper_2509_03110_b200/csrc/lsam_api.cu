@@ -310,8 +310,9 @@ int launch_perturb(lsam_ctx* c, const TG* g, int64_t ldg, int64_t n, bool vec4) 
   return LSAM_OK;
 }
 
-UpdateArgs make_update_args(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, float eta) {
+UpdateArgs make_update_args(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n, float eta) {
   UpdateArgs a;
+  a.g_mode = g_mode;
   a.active = c->act();
   a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
   a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
@@ -326,8 +327,8 @@ void* update_func(bool noise) {
   return noise ? (void*)update_kernel<V, N, T, W, true> : (void*)update_kernel<V, N, T, W, false>;
 }
 
-int launch_update(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float eta) {
-  UpdateArgs a = make_update_args(c, g, ldg, n, eta);
+int launch_update(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n, bool vec4, float eta) {
+  UpdateArgs a = make_update_args(c, g, g_mode, ldg, n, eta);
   const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16;
   const bool nes = c->cfg.nesterov != 0;
   const bool noise = c->cfg.noise_temp > 0.f;
@@ -525,20 +526,26 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
   const int64_t n = flat ? L.d : L.ld;
   const int64_t ldg = flat ? L.d : L.ld;
+  // Gradient storage: on the tensor-core path both gradients are written by the weight-gradient GEMM in bf16 (its output
+  // type, as in the usual bf16-GEMM / fp32-master pipeline) into the g1b buffer; every other path keeps fp32, and in
+  // BF16 mode rounds to bf16 on use so that all paths of the mode compute with the same values.
+  const bool gb = !flat && c->use_tc;
+  const int g_mode = gb ? 2 : ((!flat && cfg.gemm_dtype == LSAM_GEMM_BF16) ? 1 : 0);
+  const void* gptr = gb ? (const void*)c->at<bf16>(L.g1b) : (flat ? (const void*)c->eg2 : (const void*)c->g());
   // ascent gradient, its norm, perturbation
   if (rho == 0.f && !flat && !L.g1keep) {
     // rho = 0: the perturbed point is x itself, so the two gradients coincide (entropy-/elastic-averaging SGD, the
     // unperturbed case of Theorem 2): one gradient pass, no norm, no perturbation
-    if ((rc = grad_pass(c, false, c->loss())) != LSAM_OK) return rc;
+    if ((rc = grad_pass(c, false, c->loss(), gb)) != LSAM_OK) return rc;
     if (cfg.flags & LSAM_FLAG_STEP_INFO) {
       if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm1(), nullptr)) != LSAM_OK) return rc;
       if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
     }
-    if ((rc = launch_update(c, c->g(), ldg, n, vec4, eta)) != LSAM_OK) return rc;
+    if ((rc = launch_update(c, gptr, g_mode, ldg, n, vec4, eta)) != LSAM_OK) return rc;
     return LSAM_OK;
   }
   const float* g1 = flat ? c->eg1 : c->g();
-  const bool g1_bf16 = !flat && c->use_tc;  // tensor-core path: ascent gradient stored as bf16 in g1b
+  const bool g1_bf16 = gb;
   if (!flat && (rc = grad_pass(c, false, c->loss(), g1_bf16)) != LSAM_OK) return rc;
   if (!flat && L.g1keep) {
     if (g1_bf16) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.g1keep), c->at<bf16>(L.g1b), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
@@ -556,11 +563,11 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   if (L.xpkeep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.xpkeep), c->at<bf16>(L.xop), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   // descent gradient at the perturbed point, same minibatch
   const float* g2 = flat ? c->eg2 : c->g();
-  if (!flat && (rc = grad_pass(c, true, nullptr)) != LSAM_OK) return rc;
+  if (!flat && (rc = grad_pass(c, true, nullptr, gb)) != LSAM_OK) return rc;
   if (cfg.flags & LSAM_FLAG_STEP_INFO)
     if ((rc = launch_norm(c, g2, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
   // fused worker update
-  if ((rc = launch_update(c, g2, ldg, n, vec4, eta)) != LSAM_OK) return rc;
+  if ((rc = launch_update(c, gptr, g_mode, ldg, n, vec4, eta)) != LSAM_OK) return rc;
   return LSAM_OK;
 }
 
@@ -624,7 +631,7 @@ int graph_replay(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, int
     const bool vec_unused = false; (void)vec_unused;
     LSAM_CUDA(c, cudaGraphKernelNodeGetParams(gs.n_upd, &kp));
     UpdateArgs old = *reinterpret_cast<UpdateArgs*>(kp.kernelParams[0]);
-    UpdateArgs ua = make_update_args(c, old.g, old.ldg, old.n, eta);
+    UpdateArgs ua = make_update_args(c, old.g, old.g_mode, old.ldg, old.n, eta);
     void* ptrs[1] = {&ua};
     kp.kernelParams = ptrs; kp.extra = nullptr;
     LSAM_CUDA(c, cudaGraphExecKernelNodeSetParams(gs.exec, gs.n_upd, &kp));
@@ -859,11 +866,12 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
       LSAM_CUDA(c, cudaMemcpyAsync(tmp, src + (size_t)k * L.d, sizeof(float) * L.d, cudaMemcpyDeviceToDevice, c->stream));
     } else {
       if (pass == 1 && !L.g1keep) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(1) needs LSAM_FLAG_KEEP_G1");
-      if (pass == 1 && c->use_tc) {  // kept as stored: bf16
+      if (c->use_tc) {  // both gradients are stored as bf16 on the tensor-core path
+        const bf16* srcb = pass == 1 ? c->at<bf16>(L.g1keep) : c->at<bf16>(L.g1b);
         int64_t maxlen = 0;
         for (int i = 0; i < L.seg.n; ++i) maxlen = L.seg.len[i] > maxlen ? L.seg.len[i] : maxlen;
         dim3 grid((unsigned)ceil_div(maxlen, 256), L.seg.n, 1);
-        LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(c->at<bf16>(L.g1keep) + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
+        LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(srcb + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
       } else {
         const float* src = pass == 1 ? c->at<float>(L.g1keep) : c->g();
         rc = seg_copy<false>(c, src + (size_t)k * L.ld, L.ld, tmp, L.d, 1);

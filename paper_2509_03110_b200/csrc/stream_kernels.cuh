@@ -232,7 +232,8 @@ struct SegMap { int n; int64_t src[18], dst[18], len[18]; };
 struct UpdateArgs {
   float* x;            // [K, ld]
   float* v;            // [K, ld]
-  const float* g;      // [K, ldg]
+  const void* g;       // [K, ldg] descent gradient: fp32, or bf16 when g_mode == 2
+  int g_mode;          // 0: fp32 as is; 1: fp32, rounded to bf16 before use (BF16 mode on the SIMT path); 2: stored as bf16
   const float* yring;  // [ring, ld]
   const int32_t* slot; // [K] ring slot of the centre version read by replica k
   const int32_t* active;  // nullable [K]: replicas with 0 wait this tick and are left untouched
@@ -248,6 +249,26 @@ struct UpdateArgs {
 };
 
 constexpr int kUpdThreads = 256;
+
+__device__ inline float4 update_load_g4(const void* g, int64_t idx, int mode) {
+  if (mode == 2) {
+    const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(g) + idx));
+    const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+    const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+    return make_float4(lo.x, lo.y, hi.x, hi.y);
+  }
+  float4 v = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g) + idx));
+  if (mode == 1) {
+    v.x = to_float(__float2bfloat16_rn(v.x)); v.y = to_float(__float2bfloat16_rn(v.y));
+    v.z = to_float(__float2bfloat16_rn(v.z)); v.w = to_float(__float2bfloat16_rn(v.w));
+  }
+  return v;
+}
+__device__ inline float update_load_g1(const void* g, int64_t idx, int mode) {
+  if (mode == 2) return to_float(reinterpret_cast<const bf16*>(g)[idx]);
+  const float v = reinterpret_cast<const float*>(g)[idx];
+  return mode == 1 ? to_float(__float2bfloat16_rn(v)) : v;
+}
 
 template <int VEC, bool NESTEROV, typename TP, bool WRITE_OP, bool NOISE>
 __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a) {
@@ -271,7 +292,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       while (k < a.K && !a.active[k]) ++k;  // first replica that steps at this tick
     float4 gv = make_float4(0.f, 0.f, 0.f, 0.f), xv = gv, vv = gv, yv = gv;
     if (k < a.K) {
-      gv = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)k * a.ldg + j));
+      gv = update_load_g4(a.g, (int64_t)k * a.ldg + j, a.g_mode);
       xv = *reinterpret_cast<const float4*>(a.x + (int64_t)k * a.ld + j);
       vv = *reinterpret_cast<const float4*>(a.v + (int64_t)k * a.ld + j);
       yv = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[k] * a.ld + j));
@@ -284,7 +305,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       float4 gn = gv, xn = xv, vn = vv, yn = yv;
       if (kn < a.K) {
         const int64_t on = (int64_t)kn * a.ld + j;
-        gn = __ldcs(reinterpret_cast<const float4*>(a.g + (int64_t)kn * a.ldg + j));
+        gn = update_load_g4(a.g, (int64_t)kn * a.ldg + j, a.g_mode);
         xn = *reinterpret_cast<const float4*>(a.x + on);
         vn = *reinterpret_cast<const float4*>(a.v + on);
         yn = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[kn] * a.ld + j));
@@ -327,7 +348,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
     for (int k = 0; k < a.K; ++k) {
       if (a.active != nullptr && !a.active[k]) continue;
       const int64_t o = (int64_t)k * a.ld + j;
-      const float gv = a.g[(int64_t)k * a.ldg + j];
+      const float gv = update_load_g1(a.g, (int64_t)k * a.ldg + j, a.g_mode);
       float xv = a.x[o], vv = a.v[o];
       const float yv = a.yring[(int64_t)a.slot[k] * a.ld + j];
       const float G = fmaf(a.lambda, xv - yv, gv);

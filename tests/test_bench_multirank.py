@@ -49,7 +49,7 @@ def test_single_rank_helpers_need_no_process_group():
     w = bench.WORKLOADS["c4"]
     assert bench.param_count(w) == 67027944
     wm = bench.work_model(w, True)
-    assert wm["update"]["bytes"] == (22.0 * 32 + 12.0) * 67027944 and wm["norm"]["bytes"] == 0.0
+    assert wm["update"]["bytes"] == (20.0 * 32 + 12.0) * 67027944 and wm["norm"]["bytes"] == 0.0
 
 
 def test_reference_arm_prints_only_on_rank_zero():
