@@ -332,9 +332,13 @@ int launch_update(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n
   const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16;
   const bool nes = c->cfg.nesterov != 0;
   const bool noise = c->cfg.noise_temp > 0.f;
-  const unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
+  unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
   void* f;
-  if (vec4) {
+  if (g_mode == 2 && bf && vec4 && n % 8 == 0) {  // tensor-core path: 8 elements per thread
+    grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * 8);
+    if (nes) f = noise ? (void*)update8_kernel<true, true> : (void*)update8_kernel<true, false>;
+    else     f = noise ? (void*)update8_kernel<false, true> : (void*)update8_kernel<false, false>;
+  } else if (vec4) {
     if (bf) f = nes ? update_func<4, true, bf16, true>(noise) : update_func<4, false, bf16, true>(noise);
     else    f = nes ? update_func<4, true, float, false>(noise) : update_func<4, false, float, false>(noise);
   } else {
