@@ -43,8 +43,8 @@ LAMBDA0, MU, BETA, ETA_PRIME, GAMMA = 0.9, 0.9, 0.9, 1.0, 1e-12
 NOMINAL_HBM_GBS, FALLBACK_HBM_GBS, FALLBACK_BF16_TF = 8000.0, 6650.0, 1590.0
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x max SM clock
 # ncu counters of one update_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) at the c4 shape with K = 4
-# replicas, see profiles/dram_traffic_c4_k4.md; traffic grows with (22 K + 12) d, so it is scaled to the K of the run.
-NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=None)  # to be re-taken: the kernel changed (bf16 gradient input)
+# replicas, see profiles/dram_traffic_c4_k4.md; traffic grows with (20 K + 12) d, so it is scaled to the K of the run.
+NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=6111971328.0)
 
 
 def param_count(w):
