@@ -412,8 +412,13 @@ def main():
         ctx.step_batch(eta, rho, xbs[0], ybs[0], loss)
         barrier()
         e0.record(stream)
+        # every step's minibatch crosses PCIe inside the timed region; the copy of step i+1 is issued on the library's
+        # copy stream before step i is enqueued, so it overlaps that step's kernels
+        ctx.stage_batch(xbs[0], ybs[0])
         for i in range(nst):
-            ctx.step_batch(eta, rho, xbs[i % nb], ybs[i % nb], loss)
+            if i + 1 < nst:
+                ctx.stage_batch(xbs[(i + 1) % nb], ybs[(i + 1) % nb])
+            ctx.step_staged(eta, rho, loss)
             if ctx.should_couple():
                 ctx.couple()
         e1.record(stream)

@@ -126,6 +126,16 @@ int lsam_step(lsam_ctx* ctx, float eta, float rho);
  * The staleness part of the schedule is unchanged.  Not available for FLAT. */
 int lsam_step_batch(lsam_ctx* ctx, float eta, float rho, const float* xb, const void* yb, int on_host, float* h_loss);
 
+/* Prefetching variant of lsam_step_batch: lsam_stage_batch copies a minibatch (same layout) into one of two staging
+ * slots on a copy stream owned by the context, so that the transfer overlaps the tick in flight; lsam_step_staged then
+ * runs one tick on the oldest staged minibatch.  xb / yb must stay valid until the lsam_step_staged that consumes them
+ * has returned with h_loss != NULL, or the stream has been synchronised; a device source must be complete before
+ * lsam_stage_batch is called (the copy stream does not wait for the caller's streams).
+ * LSAM_ERR_STATE: both slots full / none staged.
+ * The copy stream and its events are host-side objects (no device memory is allocated). */
+int lsam_stage_batch(lsam_ctx* ctx, const float* xb, const void* yb, int on_host);
+int lsam_step_staged(lsam_ctx* ctx, float eta, float rho, float* h_loss);
+
 /* Sync branch of Algorithm 2 (centre update with look-ahead, counters reset).  Returns LSAM_ERR_STATE and does
  * nothing when the trigger (sum_k t_x[k] > 0 and sum_k t_x[k] mod K tau == 0) is false. */
 int lsam_couple(lsam_ctx* ctx);

@@ -20,7 +20,7 @@ PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "l
                 "perturb", "update", "couple", "copy"]
 
 EXPORTS = [
-    "lsam_param_count", "lsam_workspace_bytes", "lsam_init", "lsam_step", "lsam_step_batch", "lsam_couple",
+    "lsam_param_count", "lsam_workspace_bytes", "lsam_init", "lsam_step", "lsam_step_batch", "lsam_stage_batch", "lsam_step_staged", "lsam_couple",
     "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads", "lsam_read_grads_replica",
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_read_active", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
@@ -68,6 +68,8 @@ def lib():
     L.lsam_init.argtypes = [C.POINTER(vp), cfgp, vp, vp, vp, vp, vp, C.c_size_t, vp]
     L.lsam_step.argtypes = [vp, C.c_float, C.c_float]
     L.lsam_step_batch.argtypes = [vp, C.c_float, C.c_float, vp, vp, C.c_int, vp]
+    L.lsam_stage_batch.argtypes = [vp, vp, vp, C.c_int]
+    L.lsam_step_staged.argtypes = [vp, C.c_float, C.c_float, vp]
     L.lsam_couple.argtypes = [vp]
     L.lsam_should_couple.argtypes = [vp]
     L.lsam_read_params.argtypes = [vp, C.c_int, vp, C.c_int64, C.c_int]
@@ -210,6 +212,17 @@ class Lsam:
         px = C.c_void_p(xb.data_ptr()) if isinstance(xb, torch.Tensor) else _np_ptr(xb)
         py = C.c_void_p(yb.data_ptr()) if isinstance(yb, torch.Tensor) else _np_ptr(yb)
         self._check(lib().lsam_step_batch(self._h, eta, rho, px, py, 1 if on_host else 0, _np_ptr(h_loss)))
+
+    def stage_batch(self, xb, yb):
+        """Prefetch a minibatch (pinned host tensors / numpy arrays, or CUDA tensors) into the next staging slot."""
+        torch = self._torch
+        on_host = not (isinstance(xb, torch.Tensor) and xb.is_cuda)
+        px = C.c_void_p(xb.data_ptr()) if isinstance(xb, torch.Tensor) else _np_ptr(xb)
+        py = C.c_void_p(yb.data_ptr()) if isinstance(yb, torch.Tensor) else _np_ptr(yb)
+        self._check(lib().lsam_stage_batch(self._h, px, py, 1 if on_host else 0))
+
+    def step_staged(self, eta, rho, h_loss=None):
+        self._check(lib().lsam_step_staged(self._h, eta, rho, _np_ptr(h_loss)))
 
     def should_couple(self):
         return bool(lib().lsam_should_couple(self._h))

@@ -39,7 +39,7 @@ struct Layout {
   bool vec4 = true;
   // byte offsets into the workspace
   size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status;
-  size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage;
+  size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage, xstage2, ystage2;
   size_t total = 0;
 };
 
@@ -124,7 +124,7 @@ bool plan(const lsam_config& c, Layout& L) {
   L.partial = take(4 * K * (size_t)L.nchunks);
   L.ylab = take(4 * K * B);
   for (int i = 0; i < 9; ++i) L.act[i] = L.mask[i] = 0;
-  L.logits = L.rowloss = L.dz[0] = L.dz[1] = L.dh[0] = L.dh[1] = L.xstage = L.ystage = 0;
+  L.logits = L.rowloss = L.dz[0] = L.dz[1] = L.dh[0] = L.dh[1] = L.xstage = L.ystage = L.xstage2 = L.ystage2 = 0;
   if (!flat) {
     const size_t in0 = c.widths[0];
     const size_t ldb = L.ldb;
@@ -132,6 +132,8 @@ bool plan(const lsam_config& c, Layout& L) {
     L.act[0] = (c.model == LSAM_MODEL_LSQ) ? take(4 * K * B * in0) : take(esz * K * in0 * ldb);
     L.xstage = take(4 * K * B * in0);
     L.ystage = take(4 * K * B);
+    L.xstage2 = take(4 * K * B * in0);  // second slot of the prefetch queue (lsam_stage_batch)
+    L.ystage2 = take(4 * K * B);
     if (c.model != LSAM_MODEL_LSQ) {
       size_t maxw = 0;
       for (size_t l = 0; l < L.layers.size(); ++l) {
@@ -190,6 +192,11 @@ struct lsam_ctx {
     int64_t launches = 0;
   } graphs[4];
   void* upd_func = nullptr;  // the update_kernel instantiation this context launches
+  // prefetch queue of caller-supplied minibatches (lsam_stage_batch / lsam_step_staged): two slots, own copy stream
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t staged_done[2] = {nullptr, nullptr}, slot_free[2] = {nullptr, nullptr};
+  bool slot_used[2] = {false, false};
+  int stage_head = 0, stage_count = 0;
   std::string err;
   TcPlan tc;
 
@@ -787,6 +794,62 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   return LSAM_OK;
 }
 
+int lsam_stage_batch(lsam_ctx* c, const float* xb, const void* yb, int on_host) {
+  if (!c || !xb || !yb) return LSAM_ERR_INVALID;
+  const lsam_config& cfg = c->cfg;
+  if (cfg.model == LSAM_MODEL_FLAT) return c->fail(LSAM_ERR_INVALID, "lsam_stage_batch: not available for FLAT");
+  if (c->stage_count >= 2) return c->fail(LSAM_ERR_STATE, "lsam_stage_batch: both staging slots are full");
+  if (!c->copy_stream) {
+    LSAM_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i) {
+      LSAM_CUDA(c, cudaEventCreateWithFlags(&c->staged_done[i], cudaEventDisableTiming));
+      LSAM_CUDA(c, cudaEventCreateWithFlags(&c->slot_free[i], cudaEventDisableTiming));
+    }
+  }
+  const int slot = (c->stage_head + c->stage_count) & 1;
+  const int64_t rows = (int64_t)cfg.K * cfg.batch;
+  const cudaMemcpyKind kind = on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
+  // the slot may still be read by the tick that consumed it last
+  if (c->slot_used[slot]) LSAM_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->slot_free[slot], 0));
+  LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(slot ? c->L.xstage2 : c->L.xstage), xb, sizeof(float) * rows * cfg.widths[0], kind, c->copy_stream));
+  LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(slot ? c->L.ystage2 : c->L.ystage), yb, 4 * rows, kind, c->copy_stream));
+  LSAM_CUDA(c, cudaEventRecord(c->staged_done[slot], c->copy_stream));
+  c->stage_count += 1;
+  c->launches += 2;
+  return LSAM_OK;
+}
+
+int lsam_step_staged(lsam_ctx* c, float eta, float rho, float* h_loss) {
+  if (!c) return LSAM_ERR_INVALID;
+  if (c->stage_count <= 0) return c->fail(LSAM_ERR_STATE, "lsam_step_staged: no staged minibatch (call lsam_stage_batch first)");
+  const lsam_config& cfg = c->cfg;
+  const int slot = c->stage_head;
+  const int64_t rows = (int64_t)cfg.K * cfg.batch;
+  const float* xs = c->at<float>(slot ? c->L.xstage2 : c->L.xstage);
+  LSAM_CUDA(c, cudaStreamWaitEvent(c->stream, c->staged_done[slot], 0));
+  LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(c->L.ylab), c->at<uint32_t>(slot ? c->L.ystage2 : c->L.ystage), 4 * rows, cudaMemcpyDeviceToDevice, c->stream));
+  if (cfg.model == LSAM_MODEL_LSQ) {
+    LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(c->L.act[0]), xs, sizeof(float) * rows * cfg.widths[0], cudaMemcpyDeviceToDevice, c->stream));
+  } else {
+    dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16)
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
+    else
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
+  }
+  LSAM_CUDA(c, cudaEventRecord(c->slot_free[slot], c->stream));
+  c->slot_used[slot] = true;
+  c->stage_head ^= 1;
+  c->stage_count -= 1;
+  int rc = step_common(c, eta, rho, false);
+  if (rc != LSAM_OK) return rc;
+  if (h_loss) {
+    LSAM_CUDA(c, cudaMemcpyAsync(h_loss, c->loss(), sizeof(float) * cfg.K, cudaMemcpyDeviceToHost, c->stream));
+    LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  }
+  return LSAM_OK;
+}
+
 int lsam_should_couple(const lsam_ctx* c) {
   if (!c) return 0;
   int64_t s = 0;
@@ -997,6 +1060,11 @@ void lsam_destroy(lsam_ctx* c) {
   if (!c) return;
   for (cudaEvent_t e : c->prof.pool) cudaEventDestroy(e);
   graphs_reset(c);
+  for (int i = 0; i < 2; ++i) {
+    if (c->staged_done[i]) cudaEventDestroy(c->staged_done[i]);
+    if (c->slot_free[i]) cudaEventDestroy(c->slot_free[i]);
+  }
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
   delete c;
 }
 

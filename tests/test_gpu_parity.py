@@ -261,6 +261,57 @@ def test_step_batch_matches_gathered_step():
     b.close()
 
 
+@pytest.mark.parametrize("model", ["mlp", "lsq"])
+def test_staged_prefetch_matches_step_batch(model):
+    # the prefetch queue (copy stream, two slots) must reproduce the synchronous caller-supplied path bit for bit,
+    # with one minibatch always staged ahead of the tick that runs
+    import torch
+
+    K, B, T = 3, 16, 7
+    if model == "mlp":
+        widths = (32, 40, 6)
+        X, labels = synth.gaussian_mixture(200, 32, 6, seed=1)
+        w0 = synth.mlp_init(widths, seed=1)
+        x0 = synth.replicate(w0, K)
+        kw = dict(widths=widths, K=K, batch=B, n_samples=200, tau=2, lam=0.3, seed=9)
+        mk, fin, ytype = G.MODEL_MLP, 32, labels.dtype
+    else:
+        X, labels, _ = synth.least_squares_data(200, 24, seed=3)
+        w0 = np.zeros(24, np.float32)
+        x0 = np.random.default_rng(4).standard_normal((K, 24)).astype(np.float32)
+        kw = dict(widths=(24,), K=K, batch=B, n_samples=200, tau=2, lam=0.3, seed=9)
+        mk, fin, ytype = G.MODEL_LSQ, 24, labels.dtype
+    dX, dY = torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda()
+    s = torch.cuda.Stream()
+    with torch.cuda.stream(s):
+        a = G.Lsam(G.make_config(mk, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+        b = G.Lsam(G.make_config(mk, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+        with pytest.raises(G.LsamError):
+            b.step_staged(0.05, 0.05)  # nothing staged
+        batches = []
+        for t in range(T):
+            idx, _, _ = a.read_schedule(t, want_ver=False)
+            batches.append((torch.from_numpy(X[idx.ravel()].reshape(K, B, fin)).pin_memory(),
+                            torch.from_numpy(labels[idx.ravel()].reshape(K, B).astype(ytype)).pin_memory()))
+        la, lb = np.zeros(K, np.float32), np.zeros(K, np.float32)
+        b.stage_batch(*batches[0])
+        for t in range(T):
+            a.step_batch(0.05, 0.05, batches[t][0], batches[t][1], la)
+            if t + 1 < T:
+                b.stage_batch(*batches[t + 1])
+            if t == 2:
+                with pytest.raises(G.LsamError):
+                    b.stage_batch(*batches[t])  # both slots full
+            b.step_staged(0.05, 0.05, lb)
+            np.testing.assert_array_equal(la, lb)
+            if a.should_couple():
+                assert a.couple() == 0 and b.couple() == 0
+        np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
+        np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
+        a.close()
+        b.close()
+
+
 def test_deterministic_repeat():
     # same seed, same inputs: two runs agree bit for bit (fixed reduction orders, no float atomics)
     outs = []
