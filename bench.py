@@ -289,6 +289,7 @@ def main():
     ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
     ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
     ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
+    ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: when the state fits in L2)")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
     if args.flat_d and w["model"] == FLAT:
@@ -328,7 +329,11 @@ def main():
     inp = make_inputs(w, dev, seed=rank)
     # Latency-bound workloads (state resident in L2) replay each tick as one CUDA graph; that needs a capturable stream.
     small = 4.0 * w["K"] * param_count(w) <= 126e6
-    cfg = make_cfg(G, w, flags=G.FLAG_CUDA_GRAPH if small else 0)
+    # auto: also where the kernels of a step are short (tens of microseconds each), so that launch gaps and the
+    # per-launch events of the roofline pass would be a visible share of the step
+    short_kernels = 4.0 * w["K"] * param_count(w) <= 1.2e9
+    use_graph = (small or short_kernels) if args.cuda_graph == "auto" else args.cuda_graph == "on"
+    cfg = make_cfg(G, w, flags=G.FLAG_CUDA_GRAPH if use_graph else 0)
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(work_stream)
@@ -357,7 +362,7 @@ def main():
         one_step()
     # Per-kernel CUDA events ride inside the timed region when a step is long (working set beyond L2); for the
     # latency-bound workloads they would distort it, so there the shares come from a second, separate run of the same steps.
-    events_in_timed = 4.0 * w["K"] * d > 126e6
+    events_in_timed = 4.0 * w["K"] * d > 126e6 and not use_graph  # graph replay is off while per-launch events are recorded
     ctx.profile_enable(events_in_timed)
     ctx.profile_read()
     launches0 = ctx.launch_count()
@@ -509,7 +514,7 @@ def main():
 
     line = dict(metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=warm, ms_per_step=ms_step,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if w["bf16"] else "f32", data="synthetic",
-                config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt", cuda_graph=bool(small),
+                config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt", cuda_graph=bool(use_graph),
                             l2="working set larger than L2" if events_in_timed else "L2-resident state (latency-bound workload); kernel shares from a separate profiled run",
                             parallelism="replicas only" if world > 1 else "1 GPU"),
                 clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)

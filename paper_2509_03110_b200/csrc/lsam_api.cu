@@ -428,7 +428,11 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
     }
     GemmOperand A{a_in, (int64_t)li.in * ldb, 1, ldb};       // (z, b, i) in the feature-major buffer [z][i][b]
     GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, o, i)
-    if (head) {
+    if (head && li.out <= kHeadMaxOut) {
+      dim3 hgrid((unsigned)ceil_div(B, 32), K);
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, head_forward_kernel<T><<<hgrid, 256, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, P, ld, li.w_pad, li.b_pad, li.in, li.out, B, c->at<float>(L.logits), c->act()));
+      rc = LSAM_OK;
+    } else if (head) {
       EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), li.out, ldb};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
     } else {

@@ -95,6 +95,64 @@ struct EpiFwdHead {
   }
 };
 
+// Forward of a narrow head (out <= kHeadMaxOut classes) on the SIMT path: logits[z][f][b] = bias[f] + sum_i W[z][f][i] a[z][i][b].
+// A 128 x 64 GEMM tile would be almost empty here and leave one block per replica to walk the whole contraction.
+// Instead a block takes 32 samples and walks the inputs in chunks of 256: the chunk's weights are staged in shared
+// memory, then warp w multiplies inputs w, w + 8, ... of the chunk; a lane owns one sample, reads a[i][b] coalesced
+// (eight loads in flight) and the weights as shared-memory broadcasts, and keeps `out` accumulators.  The eight
+// per-warp sums are added in warp order at the end, so the result is deterministic.
+constexpr int kHeadMaxOut = 16;
+constexpr int kHeadChunk = 256;
+template <typename T>
+__global__ void __launch_bounds__(256)
+head_forward_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, const T* __restrict__ P, int64_t ld_p, int64_t w_off, int64_t b_off,
+                    int in, int out, int B, float* __restrict__ logits, const int32_t* __restrict__ active) {
+  const int z = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  __shared__ float wch[kHeadMaxOut][kHeadChunk];
+  __shared__ float part[8][kHeadMaxOut][32];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const int b = blockIdx.x * 32 + lane;
+  const bool bv = b < B;
+  const T* az = a + (int64_t)z * a_sz + (bv ? b : 0);
+  const T* W = P + (int64_t)z * ld_p + w_off;
+  float acc[kHeadMaxOut];
+#pragma unroll
+  for (int f = 0; f < kHeadMaxOut; ++f) acc[f] = 0.f;
+  for (int i0 = 0; i0 < in; i0 += kHeadChunk) {
+    const int len = min(kHeadChunk, in - i0);
+    __syncthreads();  // the previous chunk has been consumed
+    for (int e = threadIdx.x; e < kHeadMaxOut * kHeadChunk; e += 256) {
+      const int f = e / kHeadChunk, ii = e % kHeadChunk;
+      wch[f][ii] = (f < out && ii < len) ? to_float(W[(int64_t)f * in + i0 + ii]) : 0.f;
+    }
+    __syncthreads();
+    // inputs past the end of the last chunk have zero weights; their activations are not read
+    for (int ii = w; ii < len; ii += 64) {
+      float av[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) av[u] = (ii + 8 * u < len) ? to_float(az[(int64_t)(i0 + ii + 8 * u) * ldb]) : 0.f;
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int iu = min(ii + 8 * u, kHeadChunk - 1);
+#pragma unroll
+        for (int f = 0; f < kHeadMaxOut; ++f) acc[f] = fmaf(wch[f][iu], av[u], acc[f]);
+      }
+    }
+  }
+#pragma unroll
+  for (int f = 0; f < kHeadMaxOut; ++f) part[w][f][lane] = acc[f];
+  __syncthreads();
+  for (int e = threadIdx.x; e < out * 32; e += 256) {
+    const int f = e >> 5, l = e & 31, bb = blockIdx.x * 32 + l;
+    if (bb >= B) continue;
+    float s = to_float(P[(int64_t)z * ld_p + b_off + f]);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) s += part[q][f][l];
+    logits[((int64_t)z * out + f) * ldb + bb] = s;
+  }
+}
+
 // dgrad of layer l: dh = TA(acc + skip_grad);  dz_prev = mask_prev ? dh : 0;  optionally keep dh (residual nets)
 template <typename TA>
 struct EpiDgrad {
