@@ -5,8 +5,10 @@
 
 A step is one pass of the whole hot path (schedule, gather, ascent gradient, norm, perturbation, descent gradient,
 fused update) for all K replicas, plus the centre update whenever the sync trigger fires (every tau steps).
-With more than one GPU every rank runs an independent copy of the workload (replicas only: the path has no
-exchange step on one GPU and the cross-GPU accumulator all-reduce is not built), so scaling is weak.
+With more than one GPU every rank runs an independent copy of the workload (replicas only, the default: on one GPU
+the path has no exchange step), or, with --shard-workers, the ranks form ONE job of N*K workers around a single
+centre: K workers per GPU and one all-reduce of the iterate accumulator per sync (Algorithm 2, one worker per device).
+Either way the work per GPU is fixed, so scaling is weak.
 """
 import argparse
 import json
@@ -192,13 +194,13 @@ def make_inputs(w, dev, seed=0):
     return dict(X=X, Y=Y, x0=x0, y0=w0)
 
 
-def make_cfg(G, w, flags=0):
+def make_cfg(G, w, flags=0, K_total=0, k_offset=0):
     lam = w.get("lambda0", LAMBDA0) / (w["eta"] * w["tau"])
     return G.make_config(w["model"], widths=w["widths"], K=w["K"], batch=max(w["B"], 1) if w["model"] != FLAT else 0,
                          gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
                          beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
                          flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256),
-                         noise_temp=w.get("noise_temp", 0.0))
+                         noise_temp=w.get("noise_temp", 0.0), K_total=K_total, k_offset=k_offset)
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
@@ -289,6 +291,9 @@ def main():
     ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
     ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
     ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
+    ap.add_argument("--shard-workers", action="store_true",
+                    help="N > 1: one job of N*K workers with a single centre, K workers per GPU, accumulator all-reduce every tau steps "
+                         "(default: N independent copies of the workload)")
     ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: when the state fits in L2)")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
@@ -322,18 +327,23 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    shard = bool(args.shard_workers)
+    if world > 1 or shard:
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29541")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
     warm = max(args.warmup, 3)
 
-    inp = make_inputs(w, dev, seed=rank)
+    # sharded: every rank generates the same dataset and the same initial point (one job); else independent copies
+    inp = make_inputs(w, dev, seed=0 if shard else rank)
     # Latency-bound workloads (state resident in L2) replay each tick as one CUDA graph; that needs a capturable stream.
     small = 4.0 * w["K"] * param_count(w) <= 126e6
     # auto: also where the kernels of a step are short (tens of microseconds each), so that launch gaps and the
     # per-launch events of the roofline pass would be a visible share of the step
     short_kernels = 4.0 * w["K"] * param_count(w) <= 1.2e9
     use_graph = (small or short_kernels) if args.cuda_graph == "auto" else args.cuda_graph == "on"
-    cfg = make_cfg(G, w, flags=G.FLAG_CUDA_GRAPH if use_graph else 0)
+    cfg = make_cfg(G, w, flags=G.FLAG_CUDA_GRAPH if use_graph else 0, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0)
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(work_stream)
@@ -346,10 +356,19 @@ def main():
     stream = ctx.stream
     eta, rho = w["eta"], w["rho"]
 
+    if shard:
+        from paper_2509_03110_b200 import sharded
+
+    def couple():
+        if shard:
+            sharded.exchange_and_couple(ctx)  # all-reduce of the iterate accumulator over the ranks, then the centre update
+        else:
+            ctx.couple()
+
     def one_step():
         ctx.step(eta, rho)
         if ctx.should_couple():
-            ctx.couple()
+            couple()
 
     def barrier():
         torch.cuda.synchronize()
@@ -425,7 +444,7 @@ def main():
                 ctx.stage_batch(xbs[(i + 1) % nb], ybs[(i + 1) % nb])
             ctx.step_staged(eta, rho, loss)
             if ctx.should_couple():
-                ctx.couple()
+                couple()
         e1.record(stream)
         barrier()
         ems = max_over_ranks(e0.elapsed_time(e1), world, dev)
@@ -515,12 +534,14 @@ def main():
     line = dict(metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=warm, ms_per_step=ms_step,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if w["bf16"] else "f32", data="synthetic",
                 config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt", cuda_graph=bool(use_graph),
-                            l2="working set larger than L2" if events_in_timed else "L2-resident state (latency-bound workload); kernel shares from a separate profiled run",
-                            parallelism="replicas only" if world > 1 else "1 GPU"),
+                            l2=("working set larger than L2" if not small else "L2-resident state (latency-bound workload)") +
+                               ("" if events_in_timed else "; kernel shares and roofline from a separate pass over the same steps with per-launch events"),
+                            parallelism=(f"{world * w['K']} workers sharded over {world} GPU(s), one centre, accumulator all-reduce every tau steps" if shard
+                                         else ("replicas only" if world > 1 else "1 GPU"))),
                 clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)
     print(json.dumps(line))
     ctx.close()
-    if world > 1:
+    if world > 1 or shard:
         dist.destroy_process_group()
 
 

@@ -93,6 +93,9 @@ typedef struct {
                          0 or 256 = every worker steps at every tick (lock-step)                     */
   float noise_temp;   /* Langevin temperature T >= 0 (Section 4.1): x += sqrt(2 eta T) N(0, I) after the step,
                          normals from Philox4x32-10 keyed by (seed, tick, worker, segment, offset); 0 = none */
+  int32_t K_total;    /* workers of the whole job, n of Algorithm 2, when this context holds only a shard of them
+                         (one context per GPU); 0 = K, a single context holding every worker                  */
+  int32_t k_offset;   /* global index of this context's worker 0; workers k_offset .. k_offset + K - 1 live here */
 } lsam_config;
 
 /* Unpadded parameter count d of one replica, or -1 if the configuration is invalid. */
@@ -139,6 +142,19 @@ int lsam_step_staged(lsam_ctx* ctx, float eta, float rho, float* h_loss);
 /* Sync branch of Algorithm 2 (centre update with look-ahead, counters reset).  Returns LSAM_ERR_STATE and does
  * nothing when the trigger (sum_k t_x[k] > 0 and sum_k t_x[k] mod K tau == 0) is false. */
 int lsam_couple(lsam_ctx* ctx);
+
+/* Workers sharded over several contexts (K_total > K; Section 4 deploys one worker per GPU).  Between syncs the
+ * workers are independent; the sync branch of Algorithm 2 needs one exchange, the sum over ALL workers of their
+ * iterate accumulators.  Each context accumulates the iterates of its own workers; when the trigger holds the caller
+ * sums the accumulators of all contexts element by element into every one of them (an all-reduce over the GPUs,
+ * ordered with the context's stream) and then calls lsam_couple() on each: every context applies the same centre
+ * update, dividing by K_total tau, so the centres stay identical without a broadcast.
+ * The schedule (minibatch rows, staleness, noise keys) is keyed by the GLOBAL worker index k_offset + k, so a sharded
+ * run reproduces the run of one context with K_total workers up to the order of the floating-point sum.
+ * Lock-step schedule only (active_num 0 or 256): the serving order of unequal progress is a global decision.
+ *  *d_acc  receives the device address of the accumulator, *n the number of floats to sum (the padded row length;
+ *          padding elements are zero in every context).  The buffer lives in the caller's workspace. */
+int lsam_acc_buffer(lsam_ctx* ctx, float** d_acc, int64_t* n);
 /* 1 if the trigger of the sync branch holds, else 0.  Host-only. */
 int lsam_should_couple(const lsam_ctx* ctx);
 

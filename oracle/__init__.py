@@ -58,6 +58,7 @@ def lib():
         L.oracle_step.argtypes = [vp, C.c_double, C.c_double]
         L.oracle_should_couple.argtypes = [vp]
         L.oracle_couple.argtypes = [vp]
+        L.oracle_couple_sharded.argtypes = [vp, C.c_int32, vp]
         L.oracle_read_params.argtypes = [vp, C.c_int, vp]
         L.oracle_read_state.argtypes = [vp, vp, vp, vp, vp, vp]
         L.oracle_write_state.argtypes = [vp, vp, vp, vp]
@@ -209,6 +210,11 @@ class Oracle:
 
     def couple(self):
         return int(lib().oracle_couple(self._h))
+
+    def couple_sharded(self, n_total, total_acc=None):
+        """Sync branch for a shard: total_acc [d] is the summed accumulator of ALL workers of the job (this shard's included)."""
+        oa = None if total_acc is None else np.ascontiguousarray(total_acc, dtype=np.float64)
+        return int(lib().oracle_couple_sharded(self._h, int(n_total), _ptr(oa)))
 
     def read_params(self, which):
         out = np.zeros(self.d, dtype=np.float64)

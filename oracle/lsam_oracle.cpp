@@ -485,17 +485,23 @@ int oracle_should_couple(const oracle_ctx* o) {
   return (s > 0 && s % ((int64_t)o->cfg.K * o->cfg.tau) == 0) ? 1 : 0;
 }
 
-int oracle_couple(oracle_ctx* o) {
-  if (!o) return 1;
+int oracle_couple(oracle_ctx* o) { return o ? oracle_couple_sharded(o, o->cfg.K, nullptr) : 1; }
+
+// Sync branch of Algorithm 2 when the n workers of the job are spread over several contexts: the sum of iterates runs over
+// ALL workers (total_acc, the element-wise sum of every context's accumulators; NULL = the workers held here are all
+// there are) and the divisor is n tau.
+int oracle_couple_sharded(oracle_ctx* o, int32_t n_total, const double* total_acc) {
+  if (!o || n_total < o->cfg.K) return 1;
   if (!oracle_should_couple(o)) return 3;
   const oracle_config& c = o->cfg;
   const int64_t d = o->d;
   const std::vector<double>& y = o->y_hist.back();
   std::vector<double> yn(d);
-  const double ntau = (double)c.K * (double)c.tau;
+  const double ntau = (double)n_total * (double)c.tau;
   for (int64_t j = 0; j < d; ++j) {
     double s = 0.0;
-    for (int k = 0; k < c.K; ++k) s += o->acc[(size_t)k * d + j];
+    if (total_acc) s = total_acc[j];
+    else for (int k = 0; k < c.K; ++k) s += o->acc[(size_t)k * d + j];
     const double gp = s / ntau - y[j];                                        // g'
     const double g = o->have_prev ? gp + c.beta * (gp - o->gprev[j]) : gp;    // look-ahead direction
     yn[j] = y[j] + c.eta_prime * g;                                           // ascent on log pi_LSAM

@@ -72,6 +72,11 @@ int oracle_step(oracle_ctx*, double eta, double rho);
 int oracle_should_couple(const oracle_ctx*);
 /* The centre update of Algorithm 2; returns non-zero and does nothing if the trigger is false. */
 int oracle_couple(oracle_ctx*);
+/* The same update for a context that holds only K of the n_total workers of a job (Algorithm 2 runs one worker per
+ * device): total_acc [d] is the element-wise sum of the iterate accumulators of ALL n_total workers (this context's
+ * included; NULL = only those held here); the divisor is n_total * tau.  Lock-step schedule only (every shard reaches
+ * its trigger at the same tick). */
+int oracle_couple_sharded(oracle_ctx*, int32_t n_total, const double* total_acc);
 
 /* which in [0,K): replica; which = -1: current centre. dst [d]. */
 int oracle_read_params(const oracle_ctx*, int which, double* dst);

@@ -24,7 +24,7 @@ EXPORTS = [
     "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads", "lsam_read_grads_replica",
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_read_active", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
-    "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static",
+    "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static", "lsam_acc_buffer",
 ]
 
 
@@ -35,6 +35,7 @@ class LsamConfig(C.Structure):
         ("stale_max", C.c_int32), ("flags", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_float), ("gamma", C.c_float), ("lam", C.c_float), ("beta", C.c_float),
         ("eta_prime", C.c_float), ("active_num", C.c_int32), ("noise_temp", C.c_float),
+        ("K_total", C.c_int32), ("k_offset", C.c_int32),
     ]
 
 
@@ -71,6 +72,7 @@ def lib():
     L.lsam_stage_batch.argtypes = [vp, vp, vp, C.c_int]
     L.lsam_step_staged.argtypes = [vp, C.c_float, C.c_float, vp]
     L.lsam_couple.argtypes = [vp]
+    L.lsam_acc_buffer.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_int64)]
     L.lsam_should_couple.argtypes = [vp]
     L.lsam_read_params.argtypes = [vp, C.c_int, vp, C.c_int64, C.c_int]
     L.lsam_read_schedule.argtypes = [vp, C.c_int64, vp, vp, vp]
@@ -101,7 +103,7 @@ def lib():
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=IMPL_AUTO, mu=0.9, nesterov=1,
                 gamma=1e-12, lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, flags=0,
-                active_num=256, noise_temp=0.0):
+                active_num=256, noise_temp=0.0, K_total=0, k_offset=0):
     c = LsamConfig()
     c.model = model
     widths = list(widths)
@@ -113,6 +115,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = mu, gamma, lam, beta, eta_prime
     c.active_num = int(active_num)
     c.noise_temp = noise_temp
+    c.K_total, c.k_offset = int(K_total), int(k_offset)
     return c
 
 
@@ -229,6 +232,13 @@ class Lsam:
 
     def couple(self):
         return int(lib().lsam_couple(self._h))
+
+    def acc_tensor(self):
+        """The iterate accumulator as a CUDA fp32 tensor that aliases the workspace (sharded runs all-reduce it in place)."""
+        p, n = C.c_void_p(), C.c_int64()
+        self._check(lib().lsam_acc_buffer(self._h, C.byref(p), C.byref(n)))
+        off = int(p.value) - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * int(n.value)].view(self._torch.float32)
 
     def read_params(self, which, out=None):
         """Returns a numpy fp32 [d] (host copy) or fills the CUDA tensor `out`."""

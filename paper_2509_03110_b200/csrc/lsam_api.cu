@@ -53,6 +53,12 @@ bool plan(const lsam_config& c, Layout& L) {
   if (!(c.gamma > 0.f)) return false;
   if (c.active_num < 0 || c.active_num > 256) return false;
   if (!(c.noise_temp >= 0.f)) return false;
+  if (c.K_total != 0) {  // a shard of a larger job: lock-step schedule only
+    if (c.k_offset < 0 || c.K_total < c.K || c.k_offset > c.K_total - c.K) return false;
+    if (c.active_num != 0 && c.active_num != 256) return false;
+  } else if (c.k_offset != 0) {
+    return false;
+  }
   const bool bf = c.gemm_dtype == LSAM_GEMM_BF16;
   L.seg.n = 0;
   if (c.model == LSAM_MODEL_FLAT) {
@@ -269,11 +275,11 @@ int prof_end(lsam_ctx* c) {
 // graph can be replayed with cudaGraphExecKernelNodeSetParams on the same blocks.
 struct SchedArgs {
   uint64_t seed, t; int64_t n_samples; int B, stale_max; VerHist hist; int ring;
-  int32_t *idx, *stale, *ver, *slot; int K, active_num; int64_t budget; int32_t* active;
-  void* ptrs[15];
+  int32_t *idx, *stale, *ver, *slot; int K, active_num; int64_t budget; int32_t* active; int k_offset;
+  void* ptrs[16];
   void bind() {
-    void* p[15] = {&seed, &t, &n_samples, &B, &stale_max, &hist, &ring, &idx, &stale, &ver, &slot, &K, &active_num, &budget, &active};
-    for (int i = 0; i < 15; ++i) ptrs[i] = p[i];
+    void* p[16] = {&seed, &t, &n_samples, &B, &stale_max, &hist, &ring, &idx, &stale, &ver, &slot, &K, &active_num, &budget, &active, &k_offset};
+    for (int i = 0; i < 16; ++i) ptrs[i] = p[i];
   }
 };
 struct FinArgs {
@@ -323,7 +329,7 @@ UpdateArgs make_update_args(lsam_ctx* c, const void* g, int g_mode, int64_t ldg,
   a.active = c->act();
   a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
   a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
-  a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
+  a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.k_offset = c->cfg.k_offset; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
   a.sigma = c->cfg.noise_temp > 0.f ? sqrtf(2.0f * eta * c->cfg.noise_temp) : 0.f;
   a.seed = c->cfg.seed; a.tick = (uint64_t)c->t; a.seg = c->L.seg;
   return a;
@@ -367,7 +373,7 @@ SchedArgs make_sched_args(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, 
   const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
   a.seed = c->cfg.seed; a.t = (uint64_t)t; a.n_samples = flat ? 1 : c->cfg.n_samples; a.B = flat ? 0 : c->cfg.batch;
   a.stale_max = c->cfg.stale_max; a.ring = c->L.ring; a.idx = flat ? nullptr : idx; a.stale = stale; a.ver = ver; a.slot = slot;
-  a.K = c->cfg.K; a.active_num = c->cfg.active_num; a.budget = budget; a.active = active;
+  a.K = c->cfg.K; a.active_num = c->cfg.active_num; a.budget = budget; a.active = active; a.k_offset = c->cfg.k_offset;
   return a;
 }
 
@@ -865,12 +871,20 @@ int lsam_couple(lsam_ctx* c) {
   if (!c) return LSAM_ERR_INVALID;
   if (!lsam_should_couple(c)) return c->fail(LSAM_ERR_STATE, "lsam_couple: sync trigger is false");
   const Layout& L = c->L;
-  const float inv = 1.0f / ((float)c->cfg.K * (float)c->cfg.tau);
+  // divisor n tau of the sync branch: n counts the workers of the whole job (their accumulators have been summed into this one)
+  const float inv = 1.0f / ((float)(c->cfg.K_total > 0 ? c->cfg.K_total : c->cfg.K) * (float)c->cfg.tau);
   LAUNCH(c, LSAM_PROF_COUPLE, couple_kernel<<<(unsigned)ceil_div(L.ld, 256), 256, 0, c->stream>>>(
       c->at<float>(L.acc), c->yslot(c->t_y), c->yslot(c->t_y + 1), c->at<float>(L.gprev), L.ld, inv, c->cfg.beta, c->cfg.eta_prime, c->have_prev ? 1 : 0));
   c->have_prev = true;
   c->t_y += 1;
   for (auto& tx : c->t_x) tx = 0;
+  return LSAM_OK;
+}
+
+int lsam_acc_buffer(lsam_ctx* c, float** d_acc, int64_t* n) {
+  if (!c || !d_acc || !n) return LSAM_ERR_INVALID;
+  *d_acc = c->at<float>(c->L.acc);
+  *n = c->L.ld;
   return LSAM_OK;
 }
 

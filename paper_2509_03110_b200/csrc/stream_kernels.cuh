@@ -11,20 +11,21 @@ namespace lsam {
 struct VerHist { int v[16]; };
 
 // grid K, block 128.  idx [K, B]; stale, ver, slot [K].  slot = ring slot holding the version read.
-// active (nullable) [K]: asynchronous progress.  Worker k is ready at this tick when H_act mod 256 < active_num; ready
+// k_offset: global index of worker 0 (sharded contexts).  active (nullable) [K]: asynchronous progress (unsharded only).  Worker k is ready at this tick when H_act mod 256 < active_num; ready
 // workers are served in the order of (H_ord, k) and only the first `budget` of them step (budget = n tau minus the
 // iterations already counted since the last sync); active[k] = 1 for those.
 __global__ void __launch_bounds__(128)
 schedule_kernel(uint64_t seed, uint64_t t, int64_t n_samples, int B, int stale_max, VerHist hist, int ring,
                 int32_t* __restrict__ idx, int32_t* __restrict__ stale, int32_t* __restrict__ ver, int32_t* __restrict__ slot,
-                int K, int active_num, int64_t budget, int32_t* __restrict__ active) {
+                int K, int active_num, int64_t budget, int32_t* __restrict__ active, int k_offset) {
   __shared__ int red[4];
   const uint64_t k = blockIdx.x;
+  const uint64_t kg = k + (uint64_t)k_offset;  // global worker index: the key of the minibatch and staleness streams
   if (idx != nullptr)
     for (int j = threadIdx.x; j < B; j += blockDim.x)
-      idx[k * B + j] = (int32_t)(schedule_hash(seed, kTagIdx, t, k, (uint64_t)j) % (uint64_t)n_samples);
+      idx[k * B + j] = (int32_t)(schedule_hash(seed, kTagIdx, t, kg, (uint64_t)j) % (uint64_t)n_samples);
   if (threadIdx.x == 0) {
-    const int s = (int)(schedule_hash(seed, kTagStale, t, k, 0) % (uint64_t)(stale_max + 1));
+    const int s = (int)(schedule_hash(seed, kTagStale, t, kg, 0) % (uint64_t)(stale_max + 1));
     const int u = hist.v[s];
     if (stale) stale[k] = s;
     if (ver) ver[k] = u;
@@ -241,6 +242,7 @@ struct UpdateArgs {
   void* xop;           // [K, ld] operand copy (or nullptr)
   int64_t ld, ldg, n;
   int K;
+  int k_offset;        // global index of worker 0: the noise streams are keyed by the global worker index
   float eta, mu, lambda;
   // Langevin noise (NOISE variants): x_new += sigma * xi, xi from langevin_noise4(seed, tick, k, segment, offset / 4)
   float sigma;
@@ -319,7 +321,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
 #undef LSAM_UPD
       if (NOISE && noff < nlen) {
         float z[4];
-        langevin_noise4(a.seed, a.tick, (uint32_t)k, nseg, (uint64_t)(noff >> 2), z);
+        langevin_noise4(a.seed, a.tick, (uint32_t)(k + a.k_offset), nseg, (uint64_t)(noff >> 2), z);
         xv.x = fmaf(a.sigma, z[0], xv.x);
         if (noff + 1 < nlen) xv.y = fmaf(a.sigma, z[1], xv.y);
         if (noff + 2 < nlen) xv.z = fmaf(a.sigma, z[2], xv.z);
@@ -356,7 +358,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       xv = NESTEROV ? xv - a.eta * fmaf(a.mu, vv, G) : xv - a.eta * vv;
       if (NOISE && noff < nlen) {
         float z[4];
-        langevin_noise4(a.seed, a.tick, (uint32_t)k, nseg, (uint64_t)(noff >> 2), z);
+        langevin_noise4(a.seed, a.tick, (uint32_t)(k + a.k_offset), nseg, (uint64_t)(noff >> 2), z);
         xv = fmaf(a.sigma, z[noff & 3], xv);
       }
       s += xv;
@@ -437,7 +439,7 @@ __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a
       const int64_t no = noff + 4 * h;
       if (NOISE && no < nlen) {
         float z[4];
-        langevin_noise4(a.seed, a.tick, (uint32_t)k, nseg, (uint64_t)(no >> 2), z);
+        langevin_noise4(a.seed, a.tick, (uint32_t)(k + a.k_offset), nseg, (uint64_t)(no >> 2), z);
         xv[h].x = fmaf(a.sigma, z[0], xv[h].x);
         if (no + 1 < nlen) xv[h].y = fmaf(a.sigma, z[1], xv[h].y);
         if (no + 2 < nlen) xv[h].z = fmaf(a.sigma, z[2], xv[h].z);

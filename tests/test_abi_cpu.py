@@ -28,8 +28,8 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_config_struct_matches_header_size():
-    # 20 int32 + 2 int64 + 1 uint64 + 5 float + int32 + float = 80 + 24 + 28 = 132, rounded up to the 8-byte alignment
-    assert C.sizeof(G.LsamConfig) == 136
+    # 20 int32 + 2 int64 + 1 uint64 + 5 float + int32 + float + 2 int32 = 80 + 24 + 28 + 8 = 140, rounded up to the 8-byte alignment
+    assert C.sizeof(G.LsamConfig) == 144
 
 
 def test_param_counts_and_workspace_of_the_five_configs():
