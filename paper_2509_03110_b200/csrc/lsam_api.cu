@@ -630,7 +630,6 @@ int graph_capture(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, bo
 
 int graph_replay(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, int64_t budget) {
   const lsam_config& cfg = c->cfg;
-  const bool flat = cfg.model == LSAM_MODEL_FLAT;
   cudaKernelNodeParams kp;
   SchedArgs sa = make_sched_args(c, c->t, c->idx(), c->stale(), c->ver(), c->slot(), budget, c->async_on ? c->active_buf() : nullptr);
   sa.bind();
@@ -649,7 +648,6 @@ int graph_replay(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, int
     LSAM_CUDA(c, cudaGraphExecKernelNodeSetParams(gs.exec, gs.n_fin, &kp));
   }
   {
-    const bool vec_unused = false; (void)vec_unused;
     LSAM_CUDA(c, cudaGraphKernelNodeGetParams(gs.n_upd, &kp));
     UpdateArgs old = *reinterpret_cast<UpdateArgs*>(kp.kernelParams[0]);
     UpdateArgs ua = make_update_args(c, old.g, old.g_mode, old.ldg, old.n, eta);
@@ -657,7 +655,6 @@ int graph_replay(lsam_ctx* c, lsam_ctx::GraphSlot& gs, float eta, float rho, int
     kp.kernelParams = ptrs; kp.extra = nullptr;
     LSAM_CUDA(c, cudaGraphExecKernelNodeSetParams(gs.exec, gs.n_upd, &kp));
   }
-  (void)flat;
   LSAM_CUDA(c, cudaGraphLaunch(gs.exec, c->stream));
   c->launches += gs.launches;
   return LSAM_OK;

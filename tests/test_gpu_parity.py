@@ -194,6 +194,8 @@ def _per_step_then_trajectory(p, eta, rho, tol_step, tol_traj, steps=20, forced=
     (G.MODEL_MLP, (64, 128, 96, 10), 4, 64),      # several tiles
     (G.MODEL_RESMLP, (48, 80, 80, 80, 12), 2, 32),
     (G.MODEL_MLP, (30, 5), 2, 9),                 # linear softmax model
+    (G.MODEL_MLP, (300, 16), 2, 70),              # narrow-head kernel at its widest (16), two weight chunks, ragged sample blocks
+    (G.MODEL_MLP, (40, 300, 17), 2, 33),          # 17 classes: one more than the narrow-head kernel takes, GEMM tile path
 ])
 def test_classifier_fp32_small(model, widths, K, B):
     p = _mlp_pair(model, widths, K, B, n=300, dtype=G.GEMM_FP32, tau=4, lam=0.4, seed=3, jitter=0.01)
