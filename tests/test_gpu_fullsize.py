@@ -45,6 +45,7 @@ def test_full_shape_step_against_oracle_on_selected_replicas(name, both_passes):
     K = w["K"]
     picks = [0, K - 1]
     x0_rows = {k: inp["x0"][k].cpu().numpy().astype(np.float64) for k in picks}
+    y0_row = inp["y0"].cpu().numpy().astype(np.float64)
     cfg = bench.make_cfg(G, w, flags=G.FLAG_KEEP_G1 | G.FLAG_STEP_INFO)
     ctx = G.Lsam(cfg, inp["X"], inp["Y"], inp["x0"], inp["y0"])
     assert ctx.uses_tcgen05()
@@ -83,8 +84,16 @@ def test_full_shape_step_against_oracle_on_selected_replicas(name, both_passes):
         want = x0_rows[k][sel] + rho * q16(r["g1"][sel]) / (np.linalg.norm(r["g1"]) + gam)
         want = torch.from_numpy(want.astype(np.float32)).to(torch.bfloat16).to(torch.float64).numpy()
         assert rel_l2(xp_gpu[sel], want) <= 1e-3
+        g2 = ctx.read_grads_replica(2, k)
         if both_passes:
-            g2 = ctx.read_grads_replica(2, k)
             assert rel_l2(g2, r["g2"]) <= TOL_GRAD_BF16_FULL, (name, k, rel_l2(g2, r["g2"]))
             assert abs(n2[k] - np.linalg.norm(r["g2"])) <= 2e-3 * np.linalg.norm(r["g2"])
+        # fused update at full size, on sampled elements: first step, so v = G and the centre read is y0 whatever the
+        # staleness; x_new = x0 - eta (G + mu G) with G = q(g2) + lambda (x0 - y0), from the library's own g2
+        lam = float(np.float32(w.get("lambda0", bench.LAMBDA0) / (w["eta"] * w["tau"])))
+        eta, mu = float(np.float32(w["eta"])), float(np.float32(bench.MU))
+        Gs = q16(g2[sel]) + lam * (x0_rows[k][sel] - y0_row[sel])
+        want_x = x0_rows[k][sel] - eta * (Gs + mu * Gs)
+        got_x = ctx.read_params(k)[sel]
+        assert np.abs(got_x - want_x).max() <= 2e-7 * max(1.0, np.abs(want_x).max()), (name, k, np.abs(got_x - want_x).max())
     ctx.close()
