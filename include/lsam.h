@@ -189,6 +189,12 @@ int lsam_read_active(lsam_ctx* ctx, int32_t* h_active);
 int lsam_read_counters(const lsam_ctx* ctx, int64_t* t, int64_t* t_y, int64_t* h_t_x);
 /* Synchronise the stream and map the device status word to LSAM_OK / LSAM_ERR_NONFINITE / LSAM_ERR_TIMEOUT. */
 int lsam_status(lsam_ctx* ctx);
+/* Exercises the failure path of the device-side waits without a failure.  Every wait inside the tensor-core kernels (on a
+ * TMA load, an MMA completion, a drained accumulator) polls its barrier a bounded number of times; when the bound is hit the
+ * kernel sets a timeout bit in the status word and ends normally, and lsam_status() then returns LSAM_ERR_TIMEOUT.  This
+ * call enqueues a one-thread kernel that runs that same wait, `polls` times (1 .. 2^20), on a barrier that nothing completes.
+ * The status word is sticky: use a context you are about to destroy.  (No counterpart in the paper.) */
+int lsam_selftest_bounded_wait(lsam_ctx* ctx, uint32_t polls);
 /* Per-kernel-class device timing.  enable != 0: every launch of the following steps is bracketed by CUDA events
  * on the context's stream.  lsam_profile_read synchronises, adds the elapsed times to ms[c] and the launch counts
  * to launches[c] for c < LSAM_PROF_CLASSES (host arrays), and clears the record. */

@@ -24,7 +24,7 @@ EXPORTS = [
     "lsam_should_couple", "lsam_read_params", "lsam_read_schedule", "lsam_read_step_info", "lsam_read_grads", "lsam_read_grads_replica",
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_read_active", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
-    "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static", "lsam_acc_buffer",
+    "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static", "lsam_acc_buffer", "lsam_selftest_bounded_wait",
 ]
 
 
@@ -85,6 +85,7 @@ def lib():
     L.lsam_read_counters.argtypes = [vp, vp, vp, vp]
     L.lsam_read_active.argtypes = [vp, vp]
     L.lsam_status.argtypes = [vp]
+    L.lsam_selftest_bounded_wait.argtypes = [vp, C.c_uint32]
     L.lsam_profile_enable.argtypes = [vp, C.c_int]
     L.lsam_profile_read.argtypes = [vp, vp, vp]
     L.lsam_launch_count.restype = C.c_int64
@@ -307,6 +308,10 @@ class Lsam:
 
     def status(self):
         return int(lib().lsam_status(self._h))
+
+    def selftest_bounded_wait(self, polls=2048):
+        """Enqueue a wait that is bound to expire (see include/lsam.h); status() then reports LSAM_ERR_TIMEOUT."""
+        self._check(lib().lsam_selftest_bounded_wait(self._h, int(polls)))
 
     def profile_enable(self, on=True):
         self._check(lib().lsam_profile_enable(self._h, 1 if on else 0))

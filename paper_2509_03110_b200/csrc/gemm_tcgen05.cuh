@@ -56,12 +56,15 @@ __device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait: false when the limit expires or another role has already given up.
 constexpr uint32_t kSpinLimit = 1u << 22;
-__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i) {
+__device__ inline bool mbar_wait_limit(uint64_t* bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023u) == 1023u && *abort_flag) return false;
   }
   return false;
+}
+__device__ inline bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limit(bar, parity, abort_flag, kSpinLimit);
 }
 
 __device__ inline void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
@@ -494,6 +497,19 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (warp == 1) {
     tc::tc_fence_after();
     tc::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+// Self-test of the bounded wait: one thread waits, with the same routine the GEMM roles use, on a barrier that nothing
+// will ever complete.  After `limit` polls it gives up, raises STATUS_TIMEOUT and the kernel ends normally.
+__global__ void wait_selftest_kernel(uint32_t limit, int* __restrict__ status) {
+  __shared__ uint64_t bar;
+  __shared__ int abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0;
+    tc::mbar_init(&bar, 1);
+    tc::fence_barrier_init();
+    if (!tc::mbar_wait_limit(&bar, 0u, &abort_flag, limit)) atomicOr(status, STATUS_TIMEOUT);
   }
 }
 

@@ -1046,6 +1046,12 @@ int lsam_status(lsam_ctx* c) {
   return LSAM_OK;
 }
 
+int lsam_selftest_bounded_wait(lsam_ctx* c, uint32_t polls) {
+  if (!c || polls == 0 || polls > (1u << 20)) return LSAM_ERR_INVALID;
+  LAUNCH(c, LSAM_PROF_COPY, wait_selftest_kernel<<<1, 32, 0, c->stream>>>(polls, c->status()));
+  return LSAM_OK;
+}
+
 int lsam_profile_enable(lsam_ctx* c, int enable) {
   if (!c) return LSAM_ERR_INVALID;
   c->prof.on = enable != 0;

@@ -560,3 +560,26 @@ def test_error_paths():
     x = gpu.read_all_params()
     assert np.isfinite(x).all()  # scale = 0 for the bad replica, the update itself used the finite g2
     gpu.close()
+
+
+def test_expired_device_wait_is_reported_and_the_context_survives():
+    # the bounded wait of the tensor-core kernels, run on a barrier that nothing completes: it must give up, set the
+    # timeout bit and return, so that the host learns of it through lsam_status() and the GPU stays usable
+    import torch
+
+    x0, y0, g1, g2 = synth.flat_problem(2, 64, seed=1)
+    mk = lambda: G.Lsam(G.make_config(G.MODEL_FLAT, K=2, flat_d=64, tau=2), None, None, torch.from_numpy(x0).cuda(), torch.from_numpy(y0).cuda())
+    a = mk()
+    assert a.status() == 0
+    a.selftest_bounded_wait(2048)
+    assert a.status() == G.LSAM_ERR_TIMEOUT
+    assert a.status() == G.LSAM_ERR_TIMEOUT  # sticky
+    a.close()
+    b = mk()  # the CUDA context is intact: a fresh library context works and is clean
+    dg1, dg2 = torch.from_numpy(g1).cuda(), torch.from_numpy(g2).cuda()
+    b.set_external_grads(dg1, dg2)
+    b.step(0.1, 0.1)
+    assert b.status() == 0 and np.isfinite(b.read_all_params()).all()
+    with pytest.raises(G.LsamError):
+        b.selftest_bounded_wait(0)
+    b.close()
