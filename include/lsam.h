@@ -183,6 +183,18 @@ int lsam_set_external_grads(lsam_ctx* ctx, const float* d_g1, const float* d_g2)
 int lsam_write_state(lsam_ctx* ctx, const float* d_x, const float* d_v, const float* d_y);
 /* Read back momentum buffers and accumulator for checkpointing: h_v [K, d], h_acc [d], h_gprev [d] (nullable). Synchronises. */
 int lsam_read_state(lsam_ctx* ctx, float* h_v, float* h_acc, float* h_gprev);
+/* Checkpoint and resume.  lsam_save_checkpoint writes the whole state of the run -- worker iterates, momentum buffers, the
+ * iterate accumulator, g'_prev, every centre version a stale read can still reach, the counters t, t_y, t_x and the
+ * recent centre-version history -- into a host buffer of lsam_checkpoint_bytes() bytes (synchronises the stream).
+ * lsam_load_checkpoint restores it into a context created with the same model, K and stale_max (x0 / y0 given to that
+ * lsam_init are overwritten; hyper-parameters passed per call or held in the new configuration are the new context's).
+ * Because minibatch rows, staleness, worker readiness and noise are pure functions of (seed, tick, worker, ...), the
+ * resumed run continues bit for bit as the saved one would have, given the same seed and hyper-parameters.
+ * The blob holds the library's padded layout and is meant for the same library build; a blob of another shape is refused
+ * with LSAM_ERR_INVALID.  Minibatches staged with lsam_stage_batch are not part of the state.  (No counterpart in the paper.) */
+size_t lsam_checkpoint_bytes(const lsam_ctx* ctx);
+int lsam_save_checkpoint(lsam_ctx* ctx, void* h_buf, size_t bytes);
+int lsam_load_checkpoint(lsam_ctx* ctx, const void* h_buf, size_t bytes);
 /* Which workers stepped at the last tick: h_active [K], 1 = stepped (computed by the device schedule kernel).  Synchronises. */
 int lsam_read_active(lsam_ctx* ctx, int32_t* h_active);
 /* Counters: steps taken t, centre version t_y, per-worker t_x [K] (host, nullable). */

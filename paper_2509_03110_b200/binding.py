@@ -25,6 +25,7 @@ EXPORTS = [
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_read_active", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
     "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static", "lsam_acc_buffer", "lsam_selftest_bounded_wait",
+    "lsam_checkpoint_bytes", "lsam_save_checkpoint", "lsam_load_checkpoint",
 ]
 
 
@@ -85,6 +86,10 @@ def lib():
     L.lsam_read_counters.argtypes = [vp, vp, vp, vp]
     L.lsam_read_active.argtypes = [vp, vp]
     L.lsam_status.argtypes = [vp]
+    L.lsam_checkpoint_bytes.restype = C.c_size_t
+    L.lsam_checkpoint_bytes.argtypes = [vp]
+    L.lsam_save_checkpoint.argtypes = [vp, vp, C.c_size_t]
+    L.lsam_load_checkpoint.argtypes = [vp, vp, C.c_size_t]
     L.lsam_selftest_bounded_wait.argtypes = [vp, C.c_uint32]
     L.lsam_profile_enable.argtypes = [vp, C.c_int]
     L.lsam_profile_read.argtypes = [vp, vp, vp]
@@ -308,6 +313,17 @@ class Lsam:
 
     def status(self):
         return int(lib().lsam_status(self._h))
+
+    def save_checkpoint(self):
+        """The whole state of the run as a numpy byte array (host)."""
+        n = int(lib().lsam_checkpoint_bytes(self._h))
+        buf = np.empty(n, dtype=np.uint8)
+        self._check(lib().lsam_save_checkpoint(self._h, _np_ptr(buf), n))
+        return buf
+
+    def load_checkpoint(self, buf):
+        buf = np.ascontiguousarray(buf, dtype=np.uint8)
+        self._check(lib().lsam_load_checkpoint(self._h, _np_ptr(buf), buf.size))
 
     def selftest_bounded_wait(self, polls=2048):
         """Enqueue a wait that is bound to expire (see include/lsam.h); status() then reports LSAM_ERR_TIMEOUT."""

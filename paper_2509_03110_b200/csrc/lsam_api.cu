@@ -1016,6 +1016,80 @@ int lsam_read_state(lsam_ctx* c, float* h_v, float* h_acc, float* h_gprev) {
   return LSAM_OK;
 }
 
+// ---- checkpoint: a host blob = header, per-worker counters, then the raw (padded) state buffers
+namespace {
+struct CkptHeader {
+  char magic[8];
+  int64_t d, ld, K, ring, t, t_y, have_prev;
+  int32_t ver_hist[16];  // centre version current when step t - 1 - i started (-1: before step 0)
+};
+const char kCkptMagic[8] = {'L', 'S', 'A', 'M', 'C', 'K', 'P', '1'};
+size_t ckpt_floats(const lsam_ctx* c) { return (size_t)c->L.ld * (2 * (size_t)c->cfg.K + 2 + (size_t)c->L.ring); }
+}  // namespace
+
+size_t lsam_checkpoint_bytes(const lsam_ctx* c) {
+  return c ? sizeof(CkptHeader) + sizeof(int64_t) * (size_t)c->cfg.K + sizeof(float) * ckpt_floats(c) : 0;
+}
+
+int lsam_save_checkpoint(lsam_ctx* c, void* h_buf, size_t bytes) {
+  if (!c || !h_buf) return LSAM_ERR_INVALID;
+  if (bytes < lsam_checkpoint_bytes(c)) return c->fail(LSAM_ERR_INVALID, "lsam_save_checkpoint: buffer smaller than lsam_checkpoint_bytes()");
+  const Layout& L = c->L;
+  const size_t K = (size_t)c->cfg.K, ld = (size_t)L.ld;
+  CkptHeader h;
+  std::memset(&h, 0, sizeof(h));
+  std::memcpy(h.magic, kCkptMagic, 8);
+  h.d = L.d; h.ld = L.ld; h.K = c->cfg.K; h.ring = L.ring; h.t = c->t; h.t_y = c->t_y; h.have_prev = c->have_prev ? 1 : 0;
+  for (int i = 0; i < 16; ++i) {
+    const int64_t st = c->t - 1 - i;
+    h.ver_hist[i] = (st >= 0 && st < (int64_t)c->ver_at_step.size()) ? c->ver_at_step[(size_t)st] : -1;
+  }
+  char* p = reinterpret_cast<char*>(h_buf);
+  std::memcpy(p, &h, sizeof(h)); p += sizeof(h);
+  std::memcpy(p, c->t_x.data(), sizeof(int64_t) * K); p += sizeof(int64_t) * K;
+  const struct { const float* src; size_t n; } parts[5] = {
+      {c->x(), K * ld}, {c->v(), K * ld}, {c->at<float>(L.acc), ld}, {c->at<float>(L.gprev), ld}, {c->at<float>(L.yring), (size_t)L.ring * ld}};
+  for (const auto& q : parts) {
+    LSAM_CUDA(c, cudaMemcpyAsync(p, q.src, sizeof(float) * q.n, cudaMemcpyDeviceToHost, c->stream));
+    p += sizeof(float) * q.n;
+  }
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LSAM_OK;
+}
+
+int lsam_load_checkpoint(lsam_ctx* c, const void* h_buf, size_t bytes) {
+  if (!c || !h_buf) return LSAM_ERR_INVALID;
+  if (bytes < lsam_checkpoint_bytes(c)) return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: blob smaller than this context's checkpoint");
+  const Layout& L = c->L;
+  const size_t K = (size_t)c->cfg.K, ld = (size_t)L.ld;
+  CkptHeader h;
+  const char* p = reinterpret_cast<const char*>(h_buf);
+  std::memcpy(&h, p, sizeof(h)); p += sizeof(h);
+  if (std::memcmp(h.magic, kCkptMagic, 8) != 0) return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: not a checkpoint blob");
+  if (h.d != L.d || h.ld != L.ld || h.K != c->cfg.K || h.ring != L.ring || h.t < 0 || h.t_y < 0)
+    return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: the blob was written by a context of another shape");
+  // staged minibatches and recorded graphs belong to the run being replaced
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  graphs_reset(c);
+  c->t = h.t; c->t_y = h.t_y; c->have_prev = h.have_prev != 0;
+  std::memcpy(c->t_x.data(), p, sizeof(int64_t) * K); p += sizeof(int64_t) * K;
+  c->ver_at_step.assign((size_t)h.t, (int)h.t_y);  // only the last 16 entries are ever read again
+  for (int i = 0; i < 16; ++i) {
+    const int64_t st = h.t - 1 - i;
+    if (st >= 0) c->ver_at_step[(size_t)st] = h.ver_hist[i];
+  }
+  const struct { float* dst; size_t n; } parts[5] = {
+      {c->x(), K * ld}, {c->v(), K * ld}, {c->at<float>(L.acc), ld}, {c->at<float>(L.gprev), ld}, {c->at<float>(L.yring), (size_t)L.ring * ld}};
+  for (const auto& q : parts) {
+    LSAM_CUDA(c, cudaMemcpyAsync(q.dst, p, sizeof(float) * q.n, cudaMemcpyHostToDevice, c->stream));
+    p += sizeof(float) * q.n;
+  }
+  int rc = refresh_operand_copy(c);  // the bf16 operand copy is a function of x
+  if (rc != LSAM_OK) return rc;
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));  // the blob may be freed on return
+  return LSAM_OK;
+}
+
 int lsam_read_counters(const lsam_ctx* c, int64_t* t, int64_t* t_y, int64_t* h_t_x) {
   if (!c) return LSAM_ERR_INVALID;
   if (t) *t = c->t;

@@ -1,0 +1,74 @@
+"""Checkpoint and resume: a run saved in the middle of a sync period and loaded into a fresh context continues bit for bit."""
+import numpy as np
+import pytest
+
+from paper_2509_03110_b200 import binding as G
+from paper_2509_03110_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+HP = dict(tau=3, lam=0.3, seed=23, stale_max=2, mu=0.9, beta=0.9, eta_prime=1.0)
+
+
+def _make(kind):
+    import torch
+
+    if kind == "flat":
+        x0, y0, g1, g2 = synth.flat_problem(4, 1001, seed=6)
+        dg = [torch.from_numpy(g1).cuda(), torch.from_numpy(g2).cuda()]
+
+        def mk(x_init):
+            c = G.Lsam(G.make_config(G.MODEL_FLAT, K=4, flat_d=1001, noise_temp=0.05, **HP), None, None, torch.from_numpy(x_init).cuda(), torch.from_numpy(y0).cuda())
+            c.set_external_grads(*dg)  # borrowed buffers are the caller's to supply again after a resume
+            return c
+        return mk, x0
+    bf = kind == "resmlp_bf16_tcgen05"
+    widths = (64, 128, 128, 16)
+    X, labels = synth.gaussian_mixture(300, widths[0], widths[-1], seed=2)
+    w0 = synth.mlp_init(widths, seed=2)
+    x0 = synth.replicate(w0, 3, jitter=0.01)
+    extra = dict(noise_temp=1e-3) if bf else dict(active_num=170)
+    dX, dY = torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda()
+    mk = lambda x_init: G.Lsam(G.make_config(G.MODEL_RESMLP if bf else G.MODEL_MLP, widths=widths, K=3, batch=48, n_samples=300,
+                                             gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32, **extra, **HP),
+                               dX, dY, torch.from_numpy(x_init).cuda(), torch.from_numpy(w0).cuda())
+    return mk, x0
+
+
+def _run(c, t0, t1):
+    for t in range(t0, t1):
+        c.step(0.02 + 0.001 * t, 0.0 if t == 5 else 0.03 + 0.002 * t)
+        if c.should_couple():
+            assert c.couple() == 0
+
+
+@pytest.mark.parametrize("kind", ["flat", "mlp_fp32_async", "resmlp_bf16_tcgen05"])
+def test_resumed_run_continues_bit_for_bit(kind):
+    mk, x0 = _make(kind)
+    a = mk(x0)
+    _run(a, 0, 8)                      # 8 ticks: past two syncs, in the middle of a period, stale reads pending
+    blob = a.save_checkpoint()
+    _run(a, 8, 15)
+    b = mk(np.zeros_like(x0))          # a fresh context with another starting point: everything must come from the blob
+    b.load_checkpoint(blob)
+    assert b.counters()[0] == 8
+    _run(b, 8, 15)
+    np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
+    np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
+    sa, sb = a.read_state(), b.read_state()
+    for key in ("v", "acc", "gprev"):
+        np.testing.assert_array_equal(sa[key], sb[key])
+    ca, cb = a.counters(), b.counters()
+    assert ca[0] == cb[0] and ca[1] == cb[1] and (ca[2] == cb[2]).all()
+    for t in (13, 14):                 # centre versions read by the last ticks: the history survived the resume
+        np.testing.assert_array_equal(a.read_schedule(t)[2], b.read_schedule(t)[2])
+    assert a.status() == 0 and b.status() == 0
+    # a blob of another shape is refused, and so is a truncated one
+    with pytest.raises(G.LsamError):
+        b.load_checkpoint(blob[: blob.size // 2])
+    other_mk, other_x0 = _make("flat" if kind != "flat" else "mlp_fp32_async")
+    o = other_mk(other_x0)
+    with pytest.raises(G.LsamError):
+        o.load_checkpoint(np.concatenate([blob, np.zeros(1 << 22, np.uint8)]))
+    for c in (a, b, o):
+        c.close()
