@@ -20,7 +20,7 @@ def build(force=False, verbose=False):
     cmd = [
         "nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
         "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-        "-o", LIB, os.path.join(CSRC, "lsam_api.cu"),
+        "-o", LIB, os.path.join(CSRC, "lsam_api.cu"), "-ldl",
     ]
     if verbose:
         cmd.insert(1, "-Xptxas")

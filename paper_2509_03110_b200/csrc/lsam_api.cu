@@ -12,6 +12,8 @@
 #include <utility>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "common.cuh"
 #include "model_kernels.cuh"
 #include "stream_kernels.cuh"
@@ -525,8 +527,24 @@ int seg_copy(lsam_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd
   return LSAM_OK;
 }
 
+// NVTX ranges around the phases of a tick, so that a profiler can filter or colour them (host-side markers only: a few
+// tens of nanoseconds when no tool is attached).  next() closes the previous phase; the destructor closes the last one.
+struct PhaseRange {
+  bool open = false;
+  void next(const char* name) {
+    if (open) nvtxRangePop();
+    nvtxRangePushA(name);
+    open = true;
+  }
+  ~PhaseRange() {
+    if (open) nvtxRangePop();
+  }
+};
+
 // The launch sequence of one tick (no host state is changed here, so that it can also be recorded into a CUDA graph).
 int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget) {
+  PhaseRange phase;
+  phase.next("lsam S0-S1 schedule, gather");
   const lsam_config& cfg = c->cfg;
   const Layout& L = c->L;
   const bool flat = cfg.model == LSAM_MODEL_FLAT;
@@ -557,7 +575,9 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   if (rho == 0.f && !flat && !L.g1keep) {
     // rho = 0: the perturbed point is x itself, so the two gradients coincide (entropy-/elastic-averaging SGD, the
     // unperturbed case of Theorem 2): one gradient pass, no norm, no perturbation
+    phase.next("lsam S2 gradient (rho = 0: single pass)");
     if ((rc = grad_pass(c, false, c->loss(), gb)) != LSAM_OK) return rc;
+    phase.next("lsam S6 update");
     if (cfg.flags & LSAM_FLAG_STEP_INFO) {
       if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm1(), nullptr)) != LSAM_OK) return rc;
       if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
@@ -567,11 +587,13 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   }
   const float* g1 = flat ? c->eg1 : c->g();
   const bool g1_bf16 = gb;
+  phase.next("lsam S2 ascent gradient");
   if (!flat && (rc = grad_pass(c, false, c->loss(), g1_bf16)) != LSAM_OK) return rc;
   if (!flat && L.g1keep) {
     if (g1_bf16) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.g1keep), c->at<bf16>(L.g1b), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
     else LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   }
+  phase.next("lsam S3-S4 norm, perturbation");
   if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
   if (g1_bf16 && vec4 && n % 8 == 0) {
     dim3 pgrid((unsigned)ceil_div(n, (int64_t)kPertThreads * 8 * kPert8Iter), cfg.K);
@@ -584,7 +606,9 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   if (L.xpkeep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.xpkeep), c->at<bf16>(L.xop), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   // descent gradient at the perturbed point, same minibatch
   const float* g2 = flat ? c->eg2 : c->g();
+  phase.next("lsam S5 descent gradient");
   if (!flat && (rc = grad_pass(c, true, nullptr, gb)) != LSAM_OK) return rc;
+  phase.next("lsam S6 update");
   if (cfg.flags & LSAM_FLAG_STEP_INFO)
     if ((rc = launch_norm(c, g2, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
   // fused worker update
@@ -868,6 +892,8 @@ int lsam_couple(lsam_ctx* c) {
   if (!c) return LSAM_ERR_INVALID;
   if (!lsam_should_couple(c)) return c->fail(LSAM_ERR_STATE, "lsam_couple: sync trigger is false");
   const Layout& L = c->L;
+  PhaseRange phase;
+  phase.next("lsam S7 couple");
   // divisor n tau of the sync branch: n counts the workers of the whole job (their accumulators have been summed into this one)
   const float inv = 1.0f / ((float)(c->cfg.K_total > 0 ? c->cfg.K_total : c->cfg.K) * (float)c->cfg.tau);
   LAUNCH(c, LSAM_PROF_COUPLE, couple_kernel<<<(unsigned)ceil_div(L.ld, 256), 256, 0, c->stream>>>(
