@@ -170,6 +170,9 @@ int lsam_read_schedule(lsam_ctx* ctx, int64_t t, int32_t* h_idx, int32_t* h_stal
 /* Of the last step: minibatch loss at x_k, ||g1_k||, ||g2_k|| (host [K] each, nullable; ||g2|| needs
  * LSAM_FLAG_STEP_INFO, else it reads 0).  Synchronises. */
 int lsam_read_step_info(lsam_ctx* ctx, float* h_loss, float* h_gnorm1, float* h_gnorm2);
+/* Anchor gap of every worker, ||x_k - y|| with y the current centre (the quantity z_t = x_t - y_t that Lemma 5 bounds):
+ * h_gap [K], host.  Two-pass fixed-order reduction over one read of x; synchronises.  A monitoring call, not part of a tick. */
+int lsam_read_anchor_gap(lsam_ctx* ctx, float* h_gap);
 /* Of the last step: pass = 1 ascent gradient (needs LSAM_FLAG_KEEP_G1), 2 descent gradient, 3 perturbed point x~
  * (as stored: rounded to bf16 in BF16 mode, where it also needs LSAM_FLAG_KEEP_G1 because the operand buffer
  * is reused by the update).  h_dst [K, d] unpadded, host.  Synchronises. */

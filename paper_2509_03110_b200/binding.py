@@ -25,7 +25,7 @@ EXPORTS = [
     "lsam_set_external_grads", "lsam_write_state", "lsam_read_state", "lsam_read_counters", "lsam_read_active", "lsam_status",
     "lsam_profile_enable", "lsam_profile_read", "lsam_launch_count", "lsam_uses_tcgen05", "lsam_last_error",
     "lsam_destroy", "lsam_schedule_hash", "lsam_row_norms_static", "lsam_acc_buffer", "lsam_selftest_bounded_wait",
-    "lsam_checkpoint_bytes", "lsam_save_checkpoint", "lsam_load_checkpoint",
+    "lsam_checkpoint_bytes", "lsam_save_checkpoint", "lsam_load_checkpoint", "lsam_read_anchor_gap",
 ]
 
 
@@ -86,6 +86,7 @@ def lib():
     L.lsam_read_counters.argtypes = [vp, vp, vp, vp]
     L.lsam_read_active.argtypes = [vp, vp]
     L.lsam_status.argtypes = [vp]
+    L.lsam_read_anchor_gap.argtypes = [vp, vp]
     L.lsam_checkpoint_bytes.restype = C.c_size_t
     L.lsam_checkpoint_bytes.argtypes = [vp]
     L.lsam_save_checkpoint.argtypes = [vp, vp, C.c_size_t]
@@ -271,6 +272,12 @@ class Lsam:
         loss, n1, n2 = (np.zeros(self.K, dtype=np.float32) for _ in range(3))
         self._check(lib().lsam_read_step_info(self._h, _np_ptr(loss), _np_ptr(n1), _np_ptr(n2)))
         return loss, n1, n2
+
+    def read_anchor_gap(self):
+        """||x_k - y|| for every worker against the current centre (numpy fp32 [K])."""
+        out = np.zeros(self.K, dtype=np.float32)
+        self._check(lib().lsam_read_anchor_gap(self._h, _np_ptr(out)))
+        return out
 
     def read_grads(self, which_pass):
         out = np.empty((self.K, self.d), dtype=np.float32)

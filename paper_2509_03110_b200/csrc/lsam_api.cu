@@ -949,6 +949,24 @@ int lsam_read_step_info(lsam_ctx* c, float* h_loss, float* h_gnorm1, float* h_gn
   return LSAM_OK;
 }
 
+int lsam_read_anchor_gap(lsam_ctx* c, float* h_gap) {
+  if (!c || !h_gap) return LSAM_ERR_INVALID;
+  const Layout& L = c->L;
+  const int K = c->cfg.K;
+  const int64_t n = (c->cfg.model == LSAM_MODEL_FLAT) ? L.d : L.ld;  // padding elements are zero in x and in the centre
+  float* partial = c->at<float>(L.partial);
+  float* out = c->at<float>(L.scalars) + 4 * (size_t)K;
+  dim3 grid((unsigned)ceil_div(n, norm_chunk<4>()), K);
+  if ((int64_t)grid.x > L.nchunks) return c->fail(LSAM_ERR_WORKSPACE, "anchor gap: partial-sum buffer too small");
+  LAUNCH(c, LSAM_PROF_NORM, gap_sumsq_partial_kernel<<<grid, kNormThreads, 0, c->stream>>>(c->x(), L.ld, c->yslot(c->t_y), n, partial, L.nchunks));
+  FinArgs f{partial, L.nchunks, (int64_t)grid.x, 0.f, c->cfg.gamma, out, nullptr, c->status(), nullptr, {}};
+  f.bind();
+  LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(K), dim3(256), f.ptrs, 0, c->stream));
+  LSAM_CUDA(c, cudaMemcpyAsync(h_gap, out, sizeof(float) * K, cudaMemcpyDeviceToHost, c->stream));
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  return LSAM_OK;
+}
+
 static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float* h_dst) {
   if (!c || !h_dst || pass < 1 || pass > 3) return LSAM_ERR_INVALID;
   const Layout& L = c->L;

@@ -84,6 +84,29 @@ sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float*
   if (threadIdx.x == 0) partial[(int64_t)k * nchunks + blockIdx.x] = tot;
 }
 
+// Anchor gap (Lemma 5): partial sums of squares of x_k - y over fixed chunks of norm_chunk<4>() elements, same order as
+// above; the rows are 16-byte aligned, the tail of a row whose length is not a multiple of 4 is masked.  grid (chunks, K).
+__global__ void __launch_bounds__(kNormThreads)
+gap_sumsq_partial_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ y, int64_t n,
+                         float* __restrict__ partial, int64_t nchunks) {
+  __shared__ float red[kNormThreads / 32];
+  const int k = blockIdx.y;
+  const int64_t base = (int64_t)blockIdx.x * norm_chunk<4>();
+  const float* row = x + (int64_t)k * ldx;
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < kNormIter; ++i) {
+    const int64_t j = base + ((int64_t)i * kNormThreads + threadIdx.x) * 4;
+    if (j >= n) continue;
+    const float4 a = *reinterpret_cast<const float4*>(row + j);   // rows are padded to a multiple of 4 elements
+    const float4 b = __ldg(reinterpret_cast<const float4*>(y + j));
+    const float d0 = a.x - b.x, d1 = a.y - b.y, d2 = a.z - b.z, d3 = a.w - b.w;
+    s += (d0 * d0 + (j + 1 < n ? d1 * d1 : 0.f)) + ((j + 2 < n ? d2 * d2 : 0.f) + (j + 3 < n ? d3 * d3 : 0.f));
+  }
+  const float tot = block_sum<float>(s, red);
+  if (threadIdx.x == 0) partial[(int64_t)k * nchunks + blockIdx.x] = tot;
+}
+
 // Pass 2: norm[k] = sqrt(sum of partials) accumulated in double in a fixed order; scale[k] = rho / (norm + gamma).
 // grid K, block 256; partial has row stride nchunks, of which the first nused are summed.  A non-finite norm raises STATUS_NONFINITE and leaves scale = 0 (no perturbation).
 __global__ void __launch_bounds__(256)

@@ -583,3 +583,27 @@ def test_expired_device_wait_is_reported_and_the_context_survives():
     with pytest.raises(G.LsamError):
         b.selftest_bounded_wait(0)
     b.close()
+
+
+@pytest.mark.parametrize("kind", ["flat_1001", "mlp_bf16"])
+def test_anchor_gap_matches_its_definition(kind):
+    # ||x_k - y|| (the z_t of Lemma 5) from the library against the definition evaluated on the read-back iterates, and
+    # against the oracle's state after the same steps
+    if kind == "flat_1001":
+        x0, y0, g1, g2 = synth.flat_problem(5, 1001, seed=8)
+        p = Pair(G.MODEL_FLAT, K=5, x0=x0, y0=y0, flat_d=1001, tau=3, lam=0.4, stale_max=1, seed=5)
+        p.set_external_grads(g1, g2)
+        tol = TOL_TRAJ_FP32
+    else:
+        p = _mlp_pair(G.MODEL_MLP, (64, 128, 96, 10), 4, 64, n=300, dtype=G.GEMM_BF16, tau=3, lam=0.4, seed=4, jitter=0.01)
+        tol = TOL_TRAJ_BF16
+    for _ in range(5):
+        p.step(0.05, 0.05)
+        p.couple_if_due()
+    gap = p.gpu.read_anchor_gap()
+    xs, y = p.gpu.read_all_params().astype(np.float64), p.gpu.read_params(-1).astype(np.float64)
+    want = np.linalg.norm(xs - y[None, :], axis=1)
+    np.testing.assert_allclose(gap, want, rtol=2e-6)
+    st = p.oracle.read_state()
+    np.testing.assert_allclose(gap, np.linalg.norm(st["x"] - st["y"][None, :], axis=1), rtol=10 * tol)
+    p.close()
