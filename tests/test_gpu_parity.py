@@ -220,6 +220,7 @@ def test_classifier_bf16_simt_small(model, widths, K, B):
     (G.MODEL_MLP, (256, 256, 256, 128), 2, 128),     # N tile 128, several contraction blocks
     (G.MODEL_RESMLP, (128, 192, 192, 192, 100), 3, 200),  # N tile 256 with a ragged minibatch, skip connections
     (G.MODEL_MLP, (320, 520, 24), 2, 40),            # ragged M tiles (520 = 4 x 128 + 8), ragged contraction (320 = 5 x 64)
+    (G.MODEL_RESMLP, (128, 256, 256, 40), 2, 300),   # minibatch wider than one N tile (256 + 44), five contraction blocks in wgrad
 ])
 def test_classifier_bf16_tcgen05(model, widths, K, B):
     p = _mlp_pair(model, widths, K, B, n=400, dtype=G.GEMM_BF16, impl=G.IMPL_TCGEN05, tau=4, lam=0.4, seed=4, jitter=0.01)
