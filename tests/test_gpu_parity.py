@@ -608,3 +608,23 @@ def test_anchor_gap_matches_its_definition(kind):
     st = p.oracle.read_state()
     np.testing.assert_allclose(gap, np.linalg.norm(st["x"] - st["y"][None, :], axis=1), rtol=10 * tol)
     p.close()
+
+
+def test_degenerate_cases_match_oracle():
+    # zero ascent gradient (a stationary point: the stabiliser gamma of Eq. 3 keeps the perturbation at exactly zero),
+    # a single worker that syncs at every tick, the deepest staleness window, and a minibatch of one sample
+    K, d = 1, 37
+    x0, y0, g1, g2 = synth.flat_problem(K, d, seed=9)
+    p = Pair(G.MODEL_FLAT, K=K, x0=x0, y0=y0, flat_d=d, tau=1, lam=0.4, stale_max=15, seed=2)
+    p.set_external_grads(np.zeros_like(g1), g2)
+    for _ in range(20):
+        p.step(0.05, 0.05)
+        p.couple_if_due()
+    e = p.errors()
+    assert max(e["x"], e["y"]) <= TOL_TRAJ_FP32, e
+    _, n1, _ = p.gpu.read_step_info()
+    assert n1[0] == 0.0 and p.gpu.status() == 0 and p.gpu.counters()[1] == 20
+    p.close()
+    p = _mlp_pair(G.MODEL_MLP, (12, 9, 4), 2, 1, n=50, dtype=G.GEMM_FP32, tau=2, lam=0.4, seed=6, jitter=0.01)
+    _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, steps=8, forced=2, what="batch of one")
+    p.close()
