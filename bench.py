@@ -434,6 +434,8 @@ def main():
             ybs.append(inp["Y"][ii].reshape(w["K"], w["B"]).cpu().pin_memory())
         loss = np.zeros(w["K"], np.float32)
         ctx.step_batch(eta, rho, xbs[0], ybs[0], loss)
+        if ctx.should_couple():
+            couple()
         barrier()
         e0.record(stream)
         # every step's minibatch crosses PCIe inside the timed region; the copy of step i+1 is issued on the library's
