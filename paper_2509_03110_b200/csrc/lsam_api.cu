@@ -353,6 +353,11 @@ int launch_update(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n
     grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * 8);
     if (nes) f = noise ? (void*)update8_kernel<true, true> : (void*)update8_kernel<true, false>;
     else     f = noise ? (void*)update8_kernel<false, true> : (void*)update8_kernel<false, false>;
+  } else if (g_mode == 0 && !bf && vec4 && n % 8 == 0 && ldg % 4 == 0 && c->L.ld % 4 == 0 && n >= ((int64_t)1 << 22)) {
+    // fp32 gradients, long rows: 8 elements per thread (short rows keep 4, for twice as many blocks)
+    grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * 8);
+    if (nes) f = noise ? (void*)update8f_kernel<true, true> : (void*)update8f_kernel<true, false>;
+    else     f = noise ? (void*)update8f_kernel<false, true> : (void*)update8f_kernel<false, false>;
   } else if (vec4) {
     if (bf) f = nes ? update_func<4, true, bf16, true>(noise) : update_func<4, false, bf16, true>(noise);
     else    f = nes ? update_func<4, true, float, false>(noise) : update_func<4, false, float, false>(noise);

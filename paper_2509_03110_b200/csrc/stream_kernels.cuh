@@ -489,6 +489,90 @@ __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a
   }
 }
 
+// fp32 counterpart of update8_kernel (gradient fp32 used as is, no operand copy): 8 consecutive elements per thread, i.e.
+// two 128-bit accesses to each of g, x, v and the centre per replica, software-pipelined over the replicas.  Same arithmetic,
+// order and noise keys as update_kernel<4, ...>.  Needs n % 8 == 0, 16-byte aligned rows and g_mode == 0.
+template <bool NESTEROV, bool NOISE>
+__global__ void __launch_bounds__(kUpdThreads) update8f_kernel(const UpdateArgs a) {
+  const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * 8;
+  if (j >= a.n) return;
+  uint32_t nseg = 0;
+  int64_t noff = 0, nlen = 0;
+  if (NOISE) {
+    for (int s = 1; s < a.seg.n; ++s)
+      if (j >= a.seg.dst[s]) nseg = (uint32_t)s;
+    noff = j - a.seg.dst[nseg];
+    nlen = a.seg.len[nseg];
+  }
+  const float* gf = reinterpret_cast<const float*>(a.g);
+  float4 s[2] = {make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f)};
+  int k = 0;
+  if (a.active != nullptr)
+    while (k < a.K && !a.active[k]) ++k;
+  float4 gv[2], xv[2], vv[2], yv[2];
+  gv[0] = gv[1] = xv[0] = xv[1] = vv[0] = vv[1] = yv[0] = yv[1] = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (k < a.K) {
+    const int64_t o = (int64_t)k * a.ld + j;
+    const float* yp = a.yring + (int64_t)a.slot[k] * a.ld + j;
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      gv[h] = __ldcs(reinterpret_cast<const float4*>(gf + (int64_t)k * a.ldg + j + 4 * h));
+      xv[h] = *reinterpret_cast<const float4*>(a.x + o + 4 * h);
+      vv[h] = *reinterpret_cast<const float4*>(a.v + o + 4 * h);
+      yv[h] = __ldg(reinterpret_cast<const float4*>(yp + 4 * h));
+    }
+  }
+  while (k < a.K) {
+    const int64_t o = (int64_t)k * a.ld + j;
+    int kn = k + 1;
+    if (a.active != nullptr)
+      while (kn < a.K && !a.active[kn]) ++kn;
+    float4 gn[2] = {gv[0], gv[1]}, xn[2] = {xv[0], xv[1]}, vn[2] = {vv[0], vv[1]}, yn[2] = {yv[0], yv[1]};
+    if (kn < a.K) {
+      const int64_t on = (int64_t)kn * a.ld + j;
+      const float* yp = a.yring + (int64_t)a.slot[kn] * a.ld + j;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        gn[h] = __ldcs(reinterpret_cast<const float4*>(gf + (int64_t)kn * a.ldg + j + 4 * h));
+        xn[h] = *reinterpret_cast<const float4*>(a.x + on + 4 * h);
+        vn[h] = *reinterpret_cast<const float4*>(a.v + on + 4 * h);
+        yn[h] = __ldg(reinterpret_cast<const float4*>(yp + 4 * h));
+      }
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      float G;
+#define LSAM_UPD(c)                                                               \
+  G = fmaf(a.lambda, xv[h].c - yv[h].c, gv[h].c);                                 \
+  vv[h].c = fmaf(a.mu, vv[h].c, G);                                               \
+  xv[h].c = NESTEROV ? xv[h].c - a.eta * fmaf(a.mu, vv[h].c, G) : xv[h].c - a.eta * vv[h].c;
+      LSAM_UPD(x) LSAM_UPD(y) LSAM_UPD(z) LSAM_UPD(w)
+#undef LSAM_UPD
+      const int64_t no = noff + 4 * h;
+      if (NOISE && no < nlen) {
+        float z[4];
+        langevin_noise4(a.seed, a.tick, (uint32_t)(k + a.k_offset), nseg, (uint64_t)(no >> 2), z);
+        xv[h].x = fmaf(a.sigma, z[0], xv[h].x);
+        if (no + 1 < nlen) xv[h].y = fmaf(a.sigma, z[1], xv[h].y);
+        if (no + 2 < nlen) xv[h].z = fmaf(a.sigma, z[2], xv[h].z);
+        if (no + 3 < nlen) xv[h].w = fmaf(a.sigma, z[3], xv[h].w);
+      }
+      s[h].x += xv[h].x; s[h].y += xv[h].y; s[h].z += xv[h].z; s[h].w += xv[h].w;
+      *reinterpret_cast<float4*>(a.x + o + 4 * h) = xv[h];
+      __stcs(reinterpret_cast<float4*>(a.v + o + 4 * h), vv[h]);
+    }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) { gv[h] = gn[h]; xv[h] = xn[h]; vv[h] = vn[h]; yv[h] = yn[h]; }
+    k = kn;
+  }
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    float4 av = *reinterpret_cast<const float4*>(a.acc + j + 4 * h);
+    av.x += s[h].x; av.y += s[h].y; av.z += s[h].z; av.w += s[h].w;
+    *reinterpret_cast<float4*>(a.acc + j + 4 * h) = av;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ S7 centre update
 //   g' = acc / (K tau) - y;  g = have_prev ? g' + beta (g' - g'_prev) : g';  y_new = y + eta' g;
 //   g'_prev <- g';  acc <- 0.       (sync branch of Algorithm 2 with the look-ahead of Section 4.2)

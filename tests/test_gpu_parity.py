@@ -63,10 +63,11 @@ def test_schedule_bit_exact_with_staleness():
 
 
 # ------------------------------------------------------------------------------------------------ optimiser-only (FLAT)
-@pytest.mark.parametrize("K,d", [(1, 1), (8, 3), (1, 1000), (8, 1000), (3, 8191), (8, 1_000_000), (2, 1_048_577)])
+@pytest.mark.parametrize("K,d", [(1, 1), (8, 3), (1, 1000), (8, 1000), (3, 8191), (8, 1_000_000), (2, 1_048_577),
+                                 (3, 4_194_312)])  # the last one: long rows, the 8-elements-per-thread fp32 update
 @pytest.mark.parametrize("nesterov", [1, 0])
 def test_flat_streaming_kernels(K, d, nesterov):
-    if nesterov == 0 and d > 10000:
+    if nesterov == 0 and d > 10000 and d != 4_194_312:
         pytest.skip("heavy-ball form is covered at the small sizes")
     x0, y0, g1, g2 = synth.flat_problem(K, d, seed=d % 97)
     p = Pair(G.MODEL_FLAT, K=K, flat_d=d, x0=x0, y0=y0, tau=3, stale_max=2, seed=5, lam=0.3, beta=0.9, eta_prime=1.0, nesterov=nesterov)
@@ -387,7 +388,7 @@ def test_async_progress_masks_bit_exact_and_trajectory(kind):
 
 
 # ------------------------------------------------------------------------------------------------ Langevin noise
-@pytest.mark.parametrize("kind", ["flat_1000", "flat_1001", "flat_262147", "mlp_fp32", "resmlp_bf16_tcgen05"])
+@pytest.mark.parametrize("kind", ["flat_1000", "flat_1001", "flat_262147", "flat_4194312", "mlp_fp32", "resmlp_bf16_tcgen05"])
 def test_langevin_noise_matches_oracle(kind):
     # the counter-based normals are the same numbers on both sides (integers from Philox, then fp32 vs double
     # Box-Muller), so a noisy step must agree to the usual fp32 tolerance
