@@ -47,6 +47,9 @@ FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x m
 # ncu counters of one update_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) at the c4 shape with K = 4
 # replicas, see profiles/dram_traffic_c4_k4.md; traffic grows with (20 K + 12) d, so it is scaled to the K of the run.
 NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=6111971328.0)
+# the same for one update8f_kernel launch of the optimiser-only workload at K = 8, d = 25.6M (profiles/stream_kernels_c5_d25m.md);
+# traffic grows with (20 K + 12) d, so it is scaled to the d of the run (rows of at least 4 M elements: the same kernel)
+NCU_UPDATE_TRAFFIC_C5 = dict(K=8, d=25_600_000, bytes=4351901696.0)
 
 
 def param_count(w):
@@ -499,6 +502,9 @@ def main():
     if top == "update" and args.workload == NCU_UPDATE_TRAFFIC["workload"] and w["bf16"]:
         roof["traffic"] = NCU_UPDATE_TRAFFIC["bytes"] * (20.0 * w["K"] + 12.0) / (20.0 * NCU_UPDATE_TRAFFIC["K"] + 12.0) if NCU_UPDATE_TRAFFIC["bytes"] else None
         roof["traffic_source"] = "ncu at K=4 scaled by (20K+12)/(20*4+12); algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
+    if top == "update" and flat and w["K"] == NCU_UPDATE_TRAFFIC_C5["K"] and d >= (1 << 22) and d % 8 == 0:
+        roof["traffic"] = NCU_UPDATE_TRAFFIC_C5["bytes"] * d / NCU_UPDATE_TRAFFIC_C5["d"]
+        roof["traffic_source"] = "ncu at d=25.6M scaled by d; algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
     if top in ("gemm_fwd", "gemm_dgrad") and ctx.uses_tcgen05():
         ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
         roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_sustained"], peak_source=f"{pk['src']} (sustained bf16)")
