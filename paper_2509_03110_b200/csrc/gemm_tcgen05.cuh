@@ -164,6 +164,10 @@ struct TcEpi {
   // wgrad: sum of squares of every 32-row block of the tile -> partial[z * ld_partial + slot0 + (mt * n_tiles + nt) * 8 + epilogue warp]
   float* partial;  int64_t ld_partial;  int slot0;
   int ldb;  // sample stride of the feature-major buffers (multiple of 16)
+  // dgrad, optional (bias_g != nullptr; needs the whole minibatch in one N tile): the bias gradient of the layer below,
+  // db[m] = sum_b dz_prev[m][b], written to bias_g[z * bias_ld + bias_off + m] (bf16 if bias_bf16, else fp32), and the sum
+  // of squares of every 8 consecutive db to partial[z * ld_partial + bias_slot0 + m / 8]
+  void* bias_g;  int bias_bf16;  int64_t bias_ld, bias_off;  int bias_slot0;
 };
 
 constexpr int kTcBlockM = 128;
@@ -208,7 +212,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   uint64_t* empty = bars + STAGES;           // [STAGES]  MMA -> TMA
   uint64_t* acc_full = bars + 2 * STAGES;    // [2]       MMA -> epilogue
   uint64_t* acc_empty = acc_full + 2;        // [2]       epilogue -> MMA
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_empty + 2);
+  uint64_t* bias_bar = acc_empty + 2;        // [4 quadrants][2]  dgrad: the two epilogue warps of a quadrant have left their partial bias sums
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bias_bar + 8);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -220,6 +225,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
     for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], kTcEpiWarps); }
+    for (int s = 0; s < 8; ++s) tc::mbar_init(&bias_bar[s], 2);
+    static_assert((2 * STAGES + 4 + 8) * 8 + 8 <= 256, "barrier area");
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
@@ -317,6 +324,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BLOCK_N);
       float bias = 0.f;
       float ssq = 0.f;  // wgrad: sum of squares of this thread's row of the tile
+      float bsum = 0.f; // dgrad: this thread's share of the bias gradient of its row (samples of its chunks, ascending)
       if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) bias = to_float(ep.bias[(int64_t)z * ep.ld_p + m]);
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
@@ -453,6 +461,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               qb[j] = qq;
               zb[j] = mb[j] ? qq : __float2bfloat16_rn(0.f);
             }
+            if (ep.bias_g != nullptr) {  // masked entries and entries past the minibatch are zero
+#pragma unroll
+              for (int j = 0; j < 32; ++j) bsum += to_float(zb[j]);
+            }
             if (full) {
               if (ep.dh_out != nullptr) {
 #pragma unroll
@@ -475,6 +487,29 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows
         const float tot = warp_sum(ssq);
         if (lane == 0) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)mt * n_tiles + nt) * kTcEpiWarps + ew] = tot;
+      }
+      if (EPI == TC_EPI_DGRAD && ep.bias_g != nullptr) {
+        // the two warps of a quadrant hold the sums over their halves of the samples: exchange through shared memory (the
+        // staging area is unused in this kernel), first warp adds them in a fixed order, stores db and the sum of squares
+        // of each group of 8 (xor-shuffle tree over the 8 lanes)
+        float* bsm = reinterpret_cast<float*>(stage) + as * 256;
+        bsm[half * 128 + quad * 32 + lane] = bsum;
+        __syncwarp();
+        if (lane == 0) tc::mbar_arrive(&bias_bar[quad * 2 + as]);
+        if (half == 0) {
+          if (!tc::mbar_wait(&bias_bar[quad * 2 + as], aph, abort_flag)) { ok = false; break; }
+          const float db = bsm[quad * 32 + lane] + bsm[128 + quad * 32 + lane];
+          float sq = (m < M) ? db * db : 0.f;
+          sq += __shfl_xor_sync(0xffffffffu, sq, 1);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 2);
+          sq += __shfl_xor_sync(0xffffffffu, sq, 4);
+          if (m < M) {
+            const int64_t o = (int64_t)z * ep.bias_ld + ep.bias_off + m;
+            if (ep.bias_bf16) reinterpret_cast<bf16*>(ep.bias_g)[o] = __float2bfloat16_rn(db);
+            else reinterpret_cast<float*>(ep.bias_g)[o] = db;
+            if ((lane & 7) == 0 && ep.partial != nullptr) ep.partial[(int64_t)z * ep.ld_partial + ep.bias_slot0 + (m >> 3)] = sq;
+          }
+        }
       }
       tc::tc_fence_before();
       __syncwarp();
@@ -644,6 +679,8 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       g.ep.dh_next = ly.residual ? b.dh[(l + 1) & 1] : nullptr;
       g.ep.dh_out = layers[l - 1].residual ? b.dh[l & 1] : nullptr;
       g.ep.dz_prev = b.dz[cur ^ 1]; g.ep.mask_prev = b.mask[l - 1]; g.ep.ldb = b.ldb;
+      g.ep.bias_g = nullptr; g.ep.bias_ld = b.ld; g.ep.bias_off = layers[l - 1].b_pad;
+      g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.bias_slot0 = P.bias_slot0[l - 1];
       g.map_c = g.map_a;
       g.valid = ok;
     }
@@ -687,6 +724,14 @@ inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream, bool out_bf16) 
   g.map_c = g.map_c16;
   return tc_launch<false, false, TC_EPI_WGRAD_BF16>(P, g, stream);
 }
-inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream) { return tc_launch<true, true, TC_EPI_DGRAD>(P, P.dgrad[l], stream); }
+// The dgrad of layer l can also deliver the bias gradient of layer l - 1 (row sums of the backward signal it writes) when the
+// whole minibatch sits in one N tile; bias_g = destination buffer ([Z, ld] gradient rows, bf16 or fp32), nullptr = not fused.
+inline bool tc_dgrad_can_fuse_bias(const TcPlan& P, int l) { return l > 0 && P.dgrad[l].valid && P.dgrad[l].N <= P.dgrad[l].block_n; }
+inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream, void* bias_g = nullptr, bool bias_bf16 = false) {
+  if (bias_g == nullptr) return tc_launch<true, true, TC_EPI_DGRAD>(P, P.dgrad[l], stream);
+  TcGemm g = P.dgrad[l];
+  g.ep.bias_g = bias_g; g.ep.bias_bf16 = bias_bf16 ? 1 : 0;
+  return tc_launch<true, true, TC_EPI_DGRAD>(P, g, stream);
+}
 
 }  // namespace lsam

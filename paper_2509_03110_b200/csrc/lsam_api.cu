@@ -465,7 +465,9 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
     const LayerInfo& li = L.layers[l];
     const T* dz = c->at<T>(L.dz[cur]);
     const T* a_in = c->at<T>(L.act[l]);
-    {
+    // tensor-core path: the dgrad of the layer above has already left this layer's bias gradient (and its sum of squares)
+    const bool bias_done = c->use_tc && l < nl - 1 && tc_dgrad_can_fuse_bias(c->tc, l + 1);
+    if (!bias_done) {
       float* part = c->use_tc ? c->at<float>(L.partial) : nullptr;
       const int slot0 = c->use_tc ? c->tc.bias_slot0[l] : 0;
       dim3 bgrid((unsigned)ceil_div(li.out, 8), K);
@@ -477,7 +479,11 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
     if (c->use_tc) {
       int trc = 0;
       LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream, g_bf16));
-      if (trc == 0 && l > 0) LAUNCH(c, LSAM_PROF_GEMM_DGRAD, trc = tc_dgrad(c->tc, l, c->stream));
+      if (trc == 0 && l > 0) {
+        void* bias_g = nullptr;
+        if (tc_dgrad_can_fuse_bias(c->tc, l)) bias_g = g_bf16 ? (void*)c->at<bf16>(L.g1b) : (void*)c->g();
+        LAUNCH(c, LSAM_PROF_GEMM_DGRAD, trc = tc_dgrad(c->tc, l, c->stream, bias_g, g_bf16));
+      }
       if (trc != 0) return c->fail(LSAM_ERR_CUDA, "tcgen05 backward launch failed");
       cur ^= 1;
       continue;
