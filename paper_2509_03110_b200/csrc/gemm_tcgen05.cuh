@@ -72,7 +72,7 @@ __device__ inline void fence_proxy_async() { asm volatile("fence.proxy.async.sha
 __device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 3-D tiled TMA load into this CTA's shared memory (no multicast), completion counted on an mbarrier.
+// 3-D tiled TMA load into this CTA's shared memory (each CTA loads its own tiles), completion counted on an mbarrier.
 __device__ inline void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
   asm volatile(
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
