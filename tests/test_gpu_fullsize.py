@@ -32,7 +32,7 @@ def _oracle_cfg(w, K):
                          lam=lam, tau=w["tau"], beta=bench.BETA, eta_prime=bench.ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=w["n"])
 
 
-@pytest.mark.parametrize("name,both_passes", [("c3", True), ("c4", False)])
+@pytest.mark.parametrize("name,both_passes", [("c3", True), ("c4", True)])
 def test_full_shape_step_against_oracle_on_selected_replicas(name, both_passes):
     import torch
 
