@@ -55,9 +55,11 @@ enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2 };
 enum {
   LSAM_FLAG_KEEP_G1 = 1,   /* keep copies of the ascent gradient and (BF16 mode) of x~ for lsam_read_grads  */
   LSAM_FLAG_STEP_INFO = 2, /* also reduce ||g2_k|| every step (one extra read of the gradient buffer)      */
-  LSAM_FLAG_CUDA_GRAPH = 4 /* replay each tick as one CUDA graph launch (recorded at the second tick of each variant;
+  LSAM_FLAG_CUDA_GRAPH = 4, /* replay each tick as one CUDA graph launch (recorded at the second tick of each variant;
                               for launch-bound small models); needs a non-default stream (lsam_init fails with
                               LSAM_ERR_INVALID otherwise); ignored while profiling is enabled               */
+  LSAM_FLAG_GRAD_FP32 = 8   /* tensor-core path: store g1 and g2 in fp32 instead of bf16 (4 instead of 2 bytes per
+                              element written by the weight-gradient GEMM and read back by perturbation and update) */
 };
 
 /* Models.
@@ -66,9 +68,11 @@ enum {
  *  RESMLP as MLP, but every hidden layer with equal input and output width is h_{l+1} = h_l + relu(W_l h_l + b_l).
  *  FLAT   no model: the two gradients of a step are buffers supplied with lsam_set_external_grads().
  * gemm_dtype BF16: matmul operands (weights, biases, inputs, stored activations and backward signals) are
- * rounded to bf16, products accumulate in fp32, all optimiser state (x, v, centre, accumulator) stays fp32.  The
- * weight-gradient matmul delivers g1 and g2 in the operand type: they are used rounded to bf16 (stored as bf16 on the
- * tensor-core path), while their norms are taken from the fp32 accumulators.                               */
+ * rounded to bf16, products accumulate in fp32, all optimiser state (x, v, centre, accumulator) stays fp32.
+ * Eq. 3 and the worker update are defined on the gradients as computed.  The SIMT path keeps g1 and g2 in fp32.  The
+ * tensor-core path by default STORES them in bf16 (a storage format that saves 12 bytes of traffic per parameter and
+ * step; it adds a relative rounding of at most 2^-8 per element, inside the bf16 tolerances; the norms ||g1||, ||g2|| are
+ * taken from the fp32 accumulators before the rounding); LSAM_FLAG_GRAD_FP32 makes it store fp32 as well.   */
 typedef struct {
   int32_t model;      /* LSAM_MODEL_*                                                               */
   int32_t n_layers;   /* weight matrices (MLP/RESMLP: 1..8; LSQ: 1; FLAT: 0)                        */
@@ -164,7 +168,7 @@ int lsam_read_params(lsam_ctx* ctx, int which, float* dst, int64_t n, int dst_on
 
 /* ---- helpers (tests, checkpointing, measurement) ---- */
 /* Schedule of step t: h_idx [K, B] minibatch rows, h_stale [K], h_ver [K] centre version read (any may be NULL).
- * idx and stale are defined for every t >= 0; ver only for steps already taken (else LSAM_ERR_STATE).
+ * idx and stale are defined for every t >= 0; ver only for the last 16 steps taken (else LSAM_ERR_STATE).
  * Computed by the device kernel the step itself uses; synchronises. */
 int lsam_read_schedule(lsam_ctx* ctx, int64_t t, int32_t* h_idx, int32_t* h_stale, int32_t* h_ver);
 /* Of the last step: minibatch loss at x_k, ||g1_k||, ||g2_k|| (host [K] each, nullable; ||g2|| needs

@@ -431,10 +431,8 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
     for (int64_t j = 0; j < d; ++j) ss += g1[j] * g1[j];
     const double n1 = std::sqrt(ss);
     o->gn1[k] = n1;
-    // look-back map: x~ = x + rho g1 / (||g1|| + gamma)
-    // (bf16 mode: the ascent gradient is a stored backward quantity, so the perturbation uses its bf16 rounding;
-    //  its norm n1 is taken before rounding)
-    for (int64_t j = 0; j < d; ++j) xp[j] = x[j] + rho * o->net.q(g1[j]) / (n1 + c.gamma);
+    // look-back map: x~ = x + rho g1 / (||g1|| + gamma)   (Eq. 3 knows one gradient: no rounding in any mode)
+    for (int64_t j = 0; j < d; ++j) xp[j] = x[j] + rho * g1[j] / (n1 + c.gamma);
     // descent gradient at x~ on the same minibatch
     if (c.model == ORACLE_MODEL_FLAT) {
       for (int64_t j = 0; j < d; ++j) g2[j] = (double)o->eg2[(size_t)k * d + j];
@@ -446,8 +444,7 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
     o->gn2[k] = std::sqrt(ss2);
     // sampler: momentum step on G = g2 + lambda (x - y); the pull is evaluated at x_k, not at x~
     for (int64_t j = 0; j < d; ++j) {
-      // (bf16 mode: the weight-gradient matmul delivers its result in the operand type, so the sampler sees q(g2))
-      const double G = o->net.q(g2[j]) + c.lambda * (x[j] - yk[j]);
+      const double G = g2[j] + c.lambda * (x[j] - yk[j]);  // Algorithm 1, first update: the gradient as computed
       v[j] = c.mu * v[j] + G;
       x[j] = c.nesterov ? x[j] - eta * (G + c.mu * v[j]) : x[j] - eta * v[j];
     }

@@ -15,7 +15,7 @@ LSAM_OK, LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE, LSAM_ERR_STATE, LSAM_ERR_CUDA, LS
 MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT = 0, 1, 2, 3
 GEMM_FP32, GEMM_BF16 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
-FLAG_KEEP_G1, FLAG_STEP_INFO, FLAG_CUDA_GRAPH = 1, 2, 4
+FLAG_KEEP_G1, FLAG_STEP_INFO, FLAG_CUDA_GRAPH, FLAG_GRAD_FP32 = 1, 2, 4, 8
 PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "loss", "bias_grad", "lsq_grad", "norm",
                 "perturb", "update", "couple", "copy"]
 

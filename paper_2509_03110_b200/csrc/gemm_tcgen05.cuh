@@ -693,10 +693,13 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
 template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
 inline int tc_launch_one(const TcPlan& P, const TcGemm& g, cudaStream_t stream) {
   auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI>;
-  static bool attr_set = false;
-  if (!attr_set) {
+  // the shared-memory limit of a kernel is a per-device attribute: remember it per device ordinal
+  static bool attr_set[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
+  if (!attr_set[dev]) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes<BLOCK_N>()) != cudaSuccess) return 1;
-    attr_set = true;
+    attr_set[dev] = true;
   }
   const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, kTcBlockM) * ceil_div(g.N, BLOCK_N);
   const int grid = (int)(tiles < P.sms ? tiles : P.sms);

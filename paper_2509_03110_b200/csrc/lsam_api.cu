@@ -184,7 +184,12 @@ struct lsam_ctx {
   bool ext_vec4 = true;
   int64_t t = 0, t_y = 0;
   std::vector<int64_t> t_x;
-  std::vector<int> ver_at_step;
+  // centre version that was current when step s started, for the steps ver_lo <= s < ver_hi, kept in a ring keyed by
+  // s mod kVerRing (a tick reads at most the last 16 of them)
+  int ver_ring[32] = {};
+  int64_t ver_lo = 0, ver_hi = 0;
+  int device = 0;                     // ordinal of the GPU that holds the workspace
+  bool grads_bf16 = false;            // tensor-core path with its gradients stored in bf16
   bool have_prev = false;
   bool use_tc = false;
   bool async_on = false;              // 0 < active_num < 256: unequal worker progress
@@ -229,6 +234,20 @@ struct lsam_ctx {
   float* yslot(int64_t version) const { return at<float>(L.yring) + (size_t)(version % L.ring) * L.ld; }
 
   int fail(int code, const std::string& m) { err = m; return code; }
+  // version current when step s started, -1 when it is not (or no longer) on record
+  int ver_of_step(int64_t s) const { return (s >= ver_lo && s < ver_hi) ? ver_ring[s & 31] : -1; }
+  // the calls that touch the GPU want the context's device to be the current one
+  int check_device() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return fail(LSAM_ERR_CUDA, "cudaGetDevice failed");
+    if (dev != device) return fail(LSAM_ERR_INVALID, "the context lives on device " + std::to_string(device) + " but device " + std::to_string(dev) + " is current");
+    return LSAM_OK;
+  }
+  int64_t budget() const {  // iterations still missing to n tau (Algorithm 2, sync trigger)
+    int64_t done = 0;
+    for (int64_t v : t_x) done += v;
+    return (int64_t)cfg.K * cfg.tau - done;
+  }
 };
 
 namespace {
@@ -320,8 +339,8 @@ int launch_perturb(lsam_ctx* c, const TG* g, int64_t ldg, int64_t n, bool vec4) 
   TP* xt = c->at<TP>(c->L.xop);
   const int64_t per = (int64_t)kPertThreads * kPertIter * (vec4 ? 4 : 1);
   dim3 grid((unsigned)ceil_div(n, per), c->cfg.K);
-  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP, TG, (sizeof(TP) == 2 && sizeof(TG) == 4)><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
-  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP, TG, (sizeof(TP) == 2 && sizeof(TG) == 4)><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
+  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
+  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
   return LSAM_OK;
 }
 
@@ -375,7 +394,7 @@ SchedArgs make_sched_args(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, 
   SchedArgs a;
   for (int s = 0; s < 16; ++s) {
     const int64_t ts = t - s > 0 ? t - s : 0;
-    a.hist.v[s] = ts < (int64_t)c->ver_at_step.size() ? c->ver_at_step[(size_t)ts] : -1;
+    a.hist.v[s] = c->ver_of_step(ts);
   }
   const bool flat = c->cfg.model == LSAM_MODEL_FLAT;
   a.seed = c->cfg.seed; a.t = (uint64_t)t; a.n_samples = flat ? 1 : c->cfg.n_samples; a.B = flat ? 0 : c->cfg.batch;
@@ -576,11 +595,11 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
   const int64_t n = flat ? L.d : L.ld;
   const int64_t ldg = flat ? L.d : L.ld;
-  // Gradient storage: on the tensor-core path both gradients are written by the weight-gradient GEMM in bf16 (its output
-  // type, as in the usual bf16-GEMM / fp32-master pipeline) into the g1b buffer; every other path keeps fp32, and in
-  // BF16 mode rounds to bf16 on use so that all paths of the mode compute with the same values.
-  const bool gb = !flat && c->use_tc;
-  const int g_mode = gb ? 2 : ((!flat && cfg.gemm_dtype == LSAM_GEMM_BF16) ? 1 : 0);
+  // Gradient storage: the tensor-core path writes both gradients from the weight-gradient GEMM in bf16 into the g1b
+  // buffer (a storage format: 2 instead of 4 bytes per element written and read back; the norms come from the fp32
+  // accumulators) unless LSAM_FLAG_GRAD_FP32 asks for fp32; every other path keeps fp32 gradients and uses them as they are.
+  const bool gb = c->grads_bf16;
+  const int g_mode = gb ? 2 : 0;
   const void* gptr = gb ? (const void*)c->at<bf16>(L.g1b) : (flat ? (const void*)c->eg2 : (const void*)c->g());
   // ascent gradient, its norm, perturbation
   if (rho == 0.f && !flat && !L.g1keep) {
@@ -708,11 +727,12 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
   const Layout& L = c->L;
   const bool flat = cfg.model == LSAM_MODEL_FLAT;
   if (flat && (!c->eg1 || !c->eg2)) return c->fail(LSAM_ERR_STATE, "FLAT model: call lsam_set_external_grads first");
-  int64_t done = 0;
-  for (int64_t v : c->t_x) done += v;
-  const int64_t budget = (int64_t)cfg.K * cfg.tau - done;  // iterations still missing to n tau (Algorithm 2, sync trigger)
+  const int64_t budget = c->budget();
   if (budget <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
-  c->ver_at_step.push_back((int)c->t_y);  // centre version current when this tick starts
+  // centre version current when this tick starts; the entry only counts once the tick has been enqueued (ver_hi below)
+  c->ver_ring[c->t & 31] = (int)c->t_y;
+  c->ver_hi = c->t + 1;
+  if (c->ver_hi - c->ver_lo > 32) c->ver_lo = c->ver_hi - 32;
   if (c->async_on) host_active_mask(cfg, c->t, budget, c->active_host);
   int rc;
   const bool shortcut = rho == 0.f && !flat && !L.g1keep;
@@ -724,7 +744,10 @@ int step_common(lsam_ctx* c, float eta, float rho, bool gather) {
   } else {
     rc = step_enqueue(c, eta, rho, gather, budget);
   }
-  if (rc != LSAM_OK) return rc;
+  if (rc != LSAM_OK) {
+    c->ver_hi = c->t;  // the tick did not happen
+    return rc;
+  }
   for (int k = 0; k < cfg.K; ++k) c->t_x[k] += c->async_on ? c->active_host[k] : 1;
   c->t += 1;
   return LSAM_OK;
@@ -778,6 +801,16 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   if (mlp && cfg->gemm_dtype == LSAM_GEMM_BF16 && cfg->gemm_impl != LSAM_IMPL_SIMT) tc_ok = tc_supported(*cfg);
   if (cfg->gemm_impl == LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
   c->use_tc = tc_ok;
+  c->grads_bf16 = tc_ok && !(cfg->flags & LSAM_FLAG_GRAD_FP32);
+  {
+    // the device that holds the workspace is the context's device; it has to be the current one here and in every later call
+    cudaPointerAttributes pa;
+    int cur = -1;
+    if (cudaPointerGetAttributes(&pa, d_workspace) != cudaSuccess || cudaGetDevice(&cur) != cudaSuccess) return bail(LSAM_ERR_CUDA);
+    if (pa.type != cudaMemoryTypeDevice && pa.type != cudaMemoryTypeManaged) return bail(LSAM_ERR_INVALID);
+    if (pa.type == cudaMemoryTypeDevice && pa.device != cur) return bail(LSAM_ERR_INVALID);
+    c->device = cur;
+  }
   if (cudaMemsetAsync(c->ws, 0, L.total, c->stream) != cudaSuccess) return bail(LSAM_ERR_CUDA);
   int rc;
   if ((rc = seg_copy<true>(c, d_x0, L.d, c->x(), L.ld, cfg->K)) != LSAM_OK) return bail(rc);
@@ -805,6 +838,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
 
 int lsam_step(lsam_ctx* c, float eta, float rho) {
   if (!c) return LSAM_ERR_INVALID;
+  if (int rc = c->check_device()) return rc;
   return step_common(c, eta, rho, true);
 }
 
@@ -812,6 +846,9 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   if (!c || !xb || !yb) return LSAM_ERR_INVALID;
   const lsam_config& cfg = c->cfg;
   if (cfg.model == LSAM_MODEL_FLAT) return c->fail(LSAM_ERR_INVALID, "lsam_step_batch: not available for FLAT");
+  if (int rc = c->check_device()) return rc;
+  // refused before anything is copied: while the sync is due the call does nothing
+  if (c->budget() <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   const int64_t nx = rows * cfg.widths[0];
   const cudaMemcpyKind kind = on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
@@ -841,6 +878,7 @@ int lsam_stage_batch(lsam_ctx* c, const float* xb, const void* yb, int on_host) 
   const lsam_config& cfg = c->cfg;
   if (cfg.model == LSAM_MODEL_FLAT) return c->fail(LSAM_ERR_INVALID, "lsam_stage_batch: not available for FLAT");
   if (c->stage_count >= 2) return c->fail(LSAM_ERR_STATE, "lsam_stage_batch: both staging slots are full");
+  if (int rc = c->check_device()) return rc;
   if (!c->copy_stream) {
     LSAM_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
     for (int i = 0; i < 2; ++i) {
@@ -864,6 +902,9 @@ int lsam_stage_batch(lsam_ctx* c, const float* xb, const void* yb, int on_host) 
 int lsam_step_staged(lsam_ctx* c, float eta, float rho, float* h_loss) {
   if (!c) return LSAM_ERR_INVALID;
   if (c->stage_count <= 0) return c->fail(LSAM_ERR_STATE, "lsam_step_staged: no staged minibatch (call lsam_stage_batch first)");
+  if (int rc = c->check_device()) return rc;
+  // refused before the staged minibatch is taken off the queue: it stays staged for the call after lsam_couple
+  if (c->budget() <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
   const lsam_config& cfg = c->cfg;
   const int slot = c->stage_head;
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
@@ -902,6 +943,7 @@ int lsam_should_couple(const lsam_ctx* c) {
 int lsam_couple(lsam_ctx* c) {
   if (!c) return LSAM_ERR_INVALID;
   if (!lsam_should_couple(c)) return c->fail(LSAM_ERR_STATE, "lsam_couple: sync trigger is false");
+  if (int rc = c->check_device()) return rc;
   const Layout& L = c->L;
   PhaseRange phase;
   phase.next("lsam S7 couple");
@@ -925,6 +967,7 @@ int lsam_acc_buffer(lsam_ctx* c, float** d_acc, int64_t* n) {
 int lsam_read_params(lsam_ctx* c, int which, float* dst, int64_t n, int dst_on_device) {
   if (!c || !dst || which < -1 || which >= c->cfg.K) return LSAM_ERR_INVALID;
   if (n < c->L.d) return c->fail(LSAM_ERR_INVALID, "lsam_read_params: destination too small");
+  if (int drc = c->check_device()) return drc;
   const float* src = which < 0 ? c->yslot(c->t_y) : c->x() + (size_t)which * c->L.ld;
   int rc;
   if (dst_on_device) return seg_copy<false>(c, src, c->L.ld, dst, c->L.d, 1);
@@ -937,7 +980,8 @@ int lsam_read_params(lsam_ctx* c, int which, float* dst, int64_t n, int dst_on_d
 
 int lsam_read_schedule(lsam_ctx* c, int64_t t, int32_t* h_idx, int32_t* h_stale, int32_t* h_ver) {
   if (!c || t < 0) return LSAM_ERR_INVALID;
-  if (h_ver && t >= (int64_t)c->ver_at_step.size()) return c->fail(LSAM_ERR_STATE, "lsam_read_schedule: centre version of a future step");
+  if (h_ver && t >= c->ver_hi) return c->fail(LSAM_ERR_STATE, "lsam_read_schedule: centre version of a future step");
+  if (h_ver && (t > 15 ? t - 15 : 0) < c->ver_lo) return c->fail(LSAM_ERR_STATE, "lsam_read_schedule: the centre-version history of that step is no longer kept (last 16 steps only)");
   const int K = c->cfg.K;
   int32_t* s = c->sched_scratch();
   int rc = launch_schedule(c, t, c->idx_scratch(), s, s + K, s + 2 * K, 0, nullptr);
@@ -1003,7 +1047,7 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
       LSAM_CUDA(c, cudaMemcpyAsync(tmp, src + (size_t)k * L.d, sizeof(float) * L.d, cudaMemcpyDeviceToDevice, c->stream));
     } else {
       if (pass == 1 && !L.g1keep) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(1) needs LSAM_FLAG_KEEP_G1");
-      if (c->use_tc) {  // both gradients are stored as bf16 on the tensor-core path
+      if (c->grads_bf16) {  // both gradients are stored as bf16
         const bf16* srcb = pass == 1 ? c->at<bf16>(L.g1keep) : c->at<bf16>(L.g1b);
         int64_t maxlen = 0;
         for (int i = 0; i < L.seg.n; ++i) maxlen = L.seg.len[i] > maxlen ? L.seg.len[i] : maxlen;
@@ -1089,6 +1133,7 @@ size_t lsam_checkpoint_bytes(const lsam_ctx* c) {
 int lsam_save_checkpoint(lsam_ctx* c, void* h_buf, size_t bytes) {
   if (!c || !h_buf) return LSAM_ERR_INVALID;
   if (bytes < lsam_checkpoint_bytes(c)) return c->fail(LSAM_ERR_INVALID, "lsam_save_checkpoint: buffer smaller than lsam_checkpoint_bytes()");
+  if (int drc = c->check_device()) return drc;
   const Layout& L = c->L;
   const size_t K = (size_t)c->cfg.K, ld = (size_t)L.ld;
   CkptHeader h;
@@ -1097,7 +1142,7 @@ int lsam_save_checkpoint(lsam_ctx* c, void* h_buf, size_t bytes) {
   h.d = L.d; h.ld = L.ld; h.K = c->cfg.K; h.ring = L.ring; h.t = c->t; h.t_y = c->t_y; h.have_prev = c->have_prev ? 1 : 0;
   for (int i = 0; i < 16; ++i) {
     const int64_t st = c->t - 1 - i;
-    h.ver_hist[i] = (st >= 0 && st < (int64_t)c->ver_at_step.size()) ? c->ver_at_step[(size_t)st] : -1;
+    h.ver_hist[i] = st >= 0 ? c->ver_of_step(st) : -1;
   }
   char* p = reinterpret_cast<char*>(h_buf);
   std::memcpy(p, &h, sizeof(h)); p += sizeof(h);
@@ -1123,15 +1168,32 @@ int lsam_load_checkpoint(lsam_ctx* c, const void* h_buf, size_t bytes) {
   if (std::memcmp(h.magic, kCkptMagic, 8) != 0) return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: not a checkpoint blob");
   if (h.d != L.d || h.ld != L.ld || h.K != c->cfg.K || h.ring != L.ring || h.t < 0 || h.t_y < 0)
     return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: the blob was written by a context of another shape");
-  // staged minibatches and recorded graphs belong to the run being replaced
-  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
-  graphs_reset(c);
-  c->t = h.t; c->t_y = h.t_y; c->have_prev = h.have_prev != 0;
-  std::memcpy(c->t_x.data(), p, sizeof(int64_t) * K); p += sizeof(int64_t) * K;
-  c->ver_at_step.assign((size_t)h.t, (int)h.t_y);  // only the last 16 entries are ever read again
+  // the blob's counters must describe a state the run can continue from
+  std::vector<int64_t> tx(K);
+  std::memcpy(tx.data(), p, sizeof(int64_t) * K); p += sizeof(int64_t) * K;
+  int64_t done = 0;
+  for (int64_t v : tx) {
+    if (v < 0) return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: negative worker counter");
+    done += v;
+  }
+  if (done > (int64_t)c->cfg.K * c->cfg.tau) return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: worker counters exceed K tau");
   for (int i = 0; i < 16; ++i) {
     const int64_t st = h.t - 1 - i;
-    if (st >= 0) c->ver_at_step[(size_t)st] = h.ver_hist[i];
+    if (st >= 0 && (h.ver_hist[i] < 0 || h.ver_hist[i] > h.t_y)) return c->fail(LSAM_ERR_INVALID, "lsam_load_checkpoint: centre-version history out of range");
+  }
+  if (int drc = c->check_device()) return drc;
+  // staged minibatches and recorded graphs belong to the run being replaced
+  LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (c->copy_stream) LSAM_CUDA(c, cudaStreamSynchronize(c->copy_stream));
+  graphs_reset(c);
+  c->stage_head = 0; c->stage_count = 0; c->slot_used[0] = c->slot_used[1] = false;
+  c->t = h.t; c->t_y = h.t_y; c->have_prev = h.have_prev != 0;
+  c->t_x = tx;
+  c->ver_hi = h.t;
+  c->ver_lo = h.t > 16 ? h.t - 16 : 0;
+  for (int i = 0; i < 16; ++i) {
+    const int64_t st = h.t - 1 - i;
+    if (st >= 0) c->ver_ring[st & 31] = h.ver_hist[i];
   }
   const struct { float* dst; size_t n; } parts[5] = {
       {c->x(), K * ld}, {c->v(), K * ld}, {c->at<float>(L.acc), ld}, {c->at<float>(L.gprev), ld}, {c->at<float>(L.yring), (size_t)L.ring * ld}};
@@ -1242,7 +1304,8 @@ extern "C" int lsam_row_norms_static(const float* d_g, int64_t ld, int64_t n, in
   if (h_err && h_err_len > 0) h_err[0] = 0;
   if (!d_g || !d_norm || K < 1 || n < 1 || ld < n)
     return static_fail(LSAM_ERR_INVALID, "lsam_row_norms_static: need d_g, d_norm, K >= 1, n >= 1, ld >= n", h_err, h_err_len);
-  const bool vec4 = (reinterpret_cast<uintptr_t>(d_g) & 15) == 0 && (ld % 4) == 0;
+  // 128-bit loads only when every vector lies wholly inside the first n elements of its row
+  const bool vec4 = (reinterpret_cast<uintptr_t>(d_g) & 15) == 0 && (ld % 4) == 0 && (n % 4) == 0;
   const int64_t chunk = vec4 ? norm_chunk<4>() : norm_chunk<1>();
   const int64_t nch = ceil_div(n, chunk);
   if (nch > LSAM_STATIC_NORM_MAX_PARTIALS || (int64_t)K * nch > LSAM_STATIC_NORM_MAX_PARTIALS || K > 65535) {

@@ -139,9 +139,8 @@ norm_finalize_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t
 constexpr int kPertThreads = 256;
 constexpr int kPertIter = 4;
 
-// TG = type of the stored gradient: float, or bf16 on the tensor-core path (packed bf16 rows of stride ldg).
-// ROUND_G: an fp32 gradient is rounded to bf16 before use, so that every path of the BF16 mode perturbs with the same value.
-template <int VEC, typename TP, typename TG, bool ROUND_G>
+// TG = type of the stored gradient: float, or bf16 where the tensor-core path stores its gradients in bf16 (packed rows of stride ldg).
+template <int VEC, typename TP, typename TG>
 __global__ void __launch_bounds__(kPertThreads)
 perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ g, int64_t ldg, int64_t n,
                const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active) {
@@ -161,10 +160,6 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ 
         xv[i] = *reinterpret_cast<const float4*>(xr + j);
         if (sizeof(TG) == 4) {
           gv[i] = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(gr) + j));
-          if (ROUND_G) {
-            gv[i].x = to_float(__float2bfloat16_rn(gv[i].x)); gv[i].y = to_float(__float2bfloat16_rn(gv[i].y));
-            gv[i].z = to_float(__float2bfloat16_rn(gv[i].z)); gv[i].w = to_float(__float2bfloat16_rn(gv[i].w));
-          }
         } else {
           const uint2 raw = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(gr) + j));
           const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
@@ -194,7 +189,7 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ 
 #pragma unroll
     for (int i = 0; i < kPertIter; ++i) {
       const int64_t j = base + (int64_t)i * kPertThreads + threadIdx.x;
-      if (j < n) tr[j] = from_float<TP>(fmaf(sc, ROUND_G ? to_float(__float2bfloat16_rn(to_float(gr[j]))) : to_float(gr[j]), xr[j]));
+      if (j < n) tr[j] = from_float<TP>(fmaf(sc, to_float(gr[j]), xr[j]));
     }
   }
 }
@@ -257,7 +252,7 @@ struct UpdateArgs {
   float* x;            // [K, ld]
   float* v;            // [K, ld]
   const void* g;       // [K, ldg] descent gradient: fp32, or bf16 when g_mode == 2
-  int g_mode;          // 0: fp32 as is; 1: fp32, rounded to bf16 before use (BF16 mode on the SIMT path); 2: stored as bf16
+  int g_mode;          // 0: fp32; 2: stored as bf16 (gradient storage format of the tensor-core path)
   const float* yring;  // [ring, ld]
   const int32_t* slot; // [K] ring slot of the centre version read by replica k
   const int32_t* active;  // nullable [K]: replicas with 0 wait this tick and are left untouched
@@ -282,17 +277,11 @@ __device__ inline float4 update_load_g4(const void* g, int64_t idx, int mode) {
     const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
     return make_float4(lo.x, lo.y, hi.x, hi.y);
   }
-  float4 v = __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g) + idx));
-  if (mode == 1) {
-    v.x = to_float(__float2bfloat16_rn(v.x)); v.y = to_float(__float2bfloat16_rn(v.y));
-    v.z = to_float(__float2bfloat16_rn(v.z)); v.w = to_float(__float2bfloat16_rn(v.w));
-  }
-  return v;
+  return __ldcs(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g) + idx));
 }
 __device__ inline float update_load_g1(const void* g, int64_t idx, int mode) {
   if (mode == 2) return to_float(reinterpret_cast<const bf16*>(g)[idx]);
-  const float v = reinterpret_cast<const float*>(g)[idx];
-  return mode == 1 ? to_float(__float2bfloat16_rn(v)) : v;
+  return reinterpret_cast<const float*>(g)[idx];
 }
 
 template <int VEC, bool NESTEROV, typename TP, bool WRITE_OP, bool NOISE>

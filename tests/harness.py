@@ -17,6 +17,44 @@ def max_rel_rows(got, want):
     return max(rel_l2(g, w) for g, w in zip(np.atleast_2d(got), np.atleast_2d(want)))
 
 
+def max_abs_rows(got, want):
+    """Max over replicas of the largest element-wise error of a row, in units of that row's RMS."""
+    worst = 0.0
+    for g, w in zip(np.atleast_2d(got), np.atleast_2d(want)):
+        g = np.asarray(g, dtype=np.float64)
+        w = np.asarray(w, dtype=np.float64)
+        rms = float(np.sqrt(np.mean(w * w)))
+        worst = max(worst, float(np.abs(g - w).max()) / (rms if rms > 0 else 1.0))
+    return worst
+
+
+def median_abs_rows(got, want):
+    """Max over replicas of the MEDIAN element-wise error of a row, in units of that row's RMS."""
+    worst = 0.0
+    for g, w in zip(np.atleast_2d(got), np.atleast_2d(want)):
+        g = np.asarray(g, dtype=np.float64)
+        w = np.asarray(w, dtype=np.float64)
+        rms = float(np.sqrt(np.mean(w * w)))
+        worst = max(worst, float(np.median(np.abs(g - w))) / (rms if rms > 0 else 1.0))
+    return worst
+
+
+# Element-wise companion of every relative-L2 bound (a handful of wrong elements in a long row, or a small systematic
+# error, would pass an L2 bound unnoticed).
+#  fp32 paths: no single element may be off by more than ELEMENTWISE_FACTOR x the L2 tolerance x the RMS of its row.
+#  bf16 paths: the L2 error has a heavy tail of discrete decisions (a ReLU sign, a bf16 rounding boundary) that the fp32
+#  accumulation of the device and the double accumulation of the oracle take differently; each one moves a few elements
+#  by about their own size, so the largest element says nothing.  What a correct implementation keeps small is the bulk:
+#  the MEDIAN element error stays at the rounding level, BULK_DIVISOR times below the L2 tolerance.
+ELEMENTWISE_FACTOR = 50.0
+BULK_DIVISOR = 8.0
+
+
+def elem_stat(got, want, bf16):
+    """Element-wise statistic scaled so that it is compared with the same tolerance as the relative-L2 error."""
+    return median_abs_rows(got, want) * BULK_DIVISOR if bf16 else max_abs_rows(got, want) / ELEMENTWISE_FACTOR
+
+
 class Pair:
     """Same configuration and inputs on both sides.  Hyper-parameters are carried as fp32 values on both."""
 
@@ -29,6 +67,7 @@ class Pair:
         self.ocfg = O.make_config(model, widths=widths, K=K, batch=batch, n_samples=n_samples, flat_d=flat_d, **okw)
         self.gcfg = G.make_config(model, widths=widths, K=K, batch=batch, n_samples=n_samples, flat_d=flat_d, **hp)
         self.K = K
+        self.bf16 = self.gcfg.gemm_dtype == G.GEMM_BF16
         x0 = np.ascontiguousarray(x0, dtype=np.float32)
         y0 = np.ascontiguousarray(y0, dtype=np.float32)
         self.oracle = O.Oracle(self.ocfg, X, Y, x0.astype(np.float64), y0.astype(np.float64))
@@ -73,21 +112,44 @@ class Pair:
         s = self.oracle.read_state()
         gx = self.gpu.read_all_params()
         gs = self.gpu.read_state()
+        gy = self.gpu.read_params(-1)
         return dict(
             x=max_rel_rows(gx, s["x"]),
             v=max_rel_rows(gs["v"], s["v"]),
-            y=rel_l2(self.gpu.read_params(-1), s["y"]),
+            y=rel_l2(gy, s["y"]),
             acc=rel_l2(gs["acc"], s["acc"].sum(axis=0)) if np.any(s["acc"]) else float(np.abs(gs["acc"]).max()),
+            x_elem=elem_stat(gx, s["x"], self.bf16),
+            y_elem=elem_stat(gy, s["y"], self.bf16),
         )
+
+    def momentum_error(self):
+        """Worst ratio, over replicas, of the momentum buffer's absolute L2 error to (lambda ||x_k|| + ||g2_k||) / (1 - mu).
+
+        v is a geometric sum (ratio mu) of G = g2 + lambda (x - y); an error of relative size tol in x and g2 therefore moves
+        it by at most tol (lambda ||x|| + ||g2||) / (1 - mu), whatever the cancellation inside x - y.  The result is
+        compared with the same tolerance as x."""
+        s = self.oracle.read_state()
+        gv = self.gpu.read_state()["v"]
+        _, g2, _ = self.oracle.read_grads()
+        lam, mu = float(self.ocfg.lam), float(self.ocfg.mu)
+        worst = 0.0
+        for k in range(self.K):
+            scale = (lam * np.linalg.norm(s["x"][k]) + np.linalg.norm(g2[k])) / (1.0 - mu)
+            worst = max(worst, float(np.linalg.norm(gv[k].astype(np.float64) - s["v"][k])) / scale)
+        return worst
 
     def grad_errors(self):
         g1, g2, xp = self.oracle.read_grads()
         if self.gcfg.gemm_dtype == G.GEMM_BF16:  # the perturbed point is stored as the bf16 matmul operand
             t = self.torch
             xp = t.from_numpy(xp.astype(np.float32)).to(t.bfloat16).to(t.float64).numpy()
-        out = dict(g2=max_rel_rows(self.gpu.read_grads(2), g2), xp=max_rel_rows(self.gpu.read_grads(3), xp))
+        gg2, gxp = self.gpu.read_grads(2), self.gpu.read_grads(3)
+        out = dict(g2=max_rel_rows(gg2, g2), xp=max_rel_rows(gxp, xp),
+                   g2_elem=elem_stat(gg2, g2, self.bf16), xp_elem=elem_stat(gxp, xp, self.bf16))
         if self.gcfg.flags & G.FLAG_KEEP_G1 or self.gcfg.model == G.MODEL_FLAT:
-            out["g1"] = max_rel_rows(self.gpu.read_grads(1), g1)
+            gg1 = self.gpu.read_grads(1)
+            out["g1"] = max_rel_rows(gg1, g1)
+            out["g1_elem"] = elem_stat(gg1, g1, self.bf16)
         return out
 
     def close(self):

@@ -222,6 +222,67 @@ def test_bf16_mode_exact_on_representable_values_and_close_otherwise():
     assert np.linalg.norm(gq - gf) / np.linalg.norm(gf) < 2 ** -8
 
 
+def test_bf16_mode_step_keeps_gradients_and_optimiser_state_unrounded():
+    # BF16 mode rounds matmul OPERANDS only.  Eq. 3 and the first update of Algorithm 1 know one gradient, so the
+    # perturbation, the sampler and the centre update must be the FP32-mode arithmetic applied to that mode's gradients.
+    # (a) Least squares on bf16-representable inputs: the only operand the mode rounds is the minibatch, so a whole
+    #     trajectory (steps, stale centre reads, syncs) must be bit-equal to FP32 mode.  A rounding applied to g1, to its
+    #     norm, to the perturbed point, to g2 or to G would break the equality.
+    X, y, _ = synth.least_squares_data(64, 12, noise=0.01, seed=7)
+    Xq = torch.from_numpy(X).to(torch.bfloat16).to(torch.float32).numpy()
+    rng = np.random.default_rng(8)
+    x0, y0 = rng.standard_normal((3, 12)), rng.standard_normal(12)
+    runs = []
+    for dt in (O.GEMM_FP32, O.GEMM_BF16):
+        cfg = O.make_config(O.MODEL_LSQ, widths=(12,), K=3, batch=8, n_samples=64, gemm_dtype=dt, lam=0.3, tau=2, stale_max=2, seed=4)
+        o = O.Oracle(cfg, Xq, y, x0, y0)
+        for _ in range(7):
+            o.step(0.05, 0.1)
+            if o.should_couple():
+                assert o.couple() == 0
+        runs.append((o.read_state(), o.read_grads()))
+    for key in ("x", "v", "y", "acc", "gprev"):
+        np.testing.assert_array_equal(runs[0][0][key], runs[1][0][key])
+    for a, b in zip(runs[0][1], runs[1][1]):
+        np.testing.assert_array_equal(a, b)
+    # and the mode does act on operands: with inputs that are not bf16 values the two modes differ
+    o32 = O.Oracle(O.make_config(O.MODEL_LSQ, widths=(12,), K=3, batch=8, n_samples=64), X, y, x0, y0)
+    o16 = O.Oracle(O.make_config(O.MODEL_LSQ, widths=(12,), K=3, batch=8, n_samples=64, gemm_dtype=O.GEMM_BF16), X, y, x0, y0)
+    o32.step(0.05, 0.1)
+    o16.step(0.05, 0.1)
+    assert not np.array_equal(o32.read_state()["x"], o16.read_state()["x"])
+    # (b) A classifier in BF16 mode: one step equals the gradient-fed (FLAT) step, which has no modes, driven with
+    #     g1 = BF16-mode gradient at x and g2 = BF16-mode gradient at the UNROUNDED perturbed point x + rho g1/(|g1|+gamma)
+    #     (the matmul rounds its own operand copy).  The FLAT model carries gradients as fp32, hence 1e-6, not equality.
+    widths, K, B, n = (6, 8, 4), 2, 8, 40
+    Xc, labels = synth.gaussian_mixture(n, widths[0], widths[-1], seed=1)
+    w0 = synth.mlp_init(widths, seed=2).astype(np.float64)
+    xs = np.stack([w0, w0 + 0.01 * rng.standard_normal(w0.shape)])
+    yc = xs.mean(axis=0)
+    kw = dict(K=K, lam=0.7, tau=4, seed=9)
+    cfg = O.make_config(O.MODEL_MLP, widths=widths, batch=B, n_samples=n, gemm_dtype=O.GEMM_BF16, **kw)
+    o = O.Oracle(cfg, Xc, labels, xs, yc)
+    idx, _, _ = o.read_schedule(0)
+    rho, gam = float(np.float32(0.1)), float(np.float32(1e-12))
+    c1 = O.make_config(O.MODEL_MLP, widths=widths, K=1, batch=B, n_samples=n, gemm_dtype=O.GEMM_BF16)
+    g1 = np.stack([O.loss_grad(c1, Xc, labels, xs[k], idx[k])[1] for k in range(K)])
+    xp = np.stack([xs[k] + rho * g1[k] / (np.linalg.norm(g1[k]) + gam) for k in range(K)])
+    g2 = np.stack([O.loss_grad(c1, Xc, labels, xp[k], idx[k])[1] for k in range(K)])
+    o.step(0.05, 0.1)
+    og1, og2, oxp = o.read_grads()
+    np.testing.assert_allclose(og1, g1, rtol=1e-13, atol=1e-300)
+    np.testing.assert_allclose(oxp, xp, rtol=1e-13)
+    np.testing.assert_allclose(og2, g2, rtol=1e-12, atol=1e-300)
+    f = O.Oracle(O.make_config(O.MODEL_FLAT, flat_d=len(w0), **kw), None, None, xs, yc)
+    f.set_external_grads(g1, g2)
+    f.step(0.05, 0.1)
+    sf, so = f.read_state(), o.read_state()
+    for key in ("x", "v", "acc"):
+        assert np.linalg.norm(sf[key] - so[key]) <= 1e-6 * np.linalg.norm(so[key]), key
+    # the gradients really are unrounded: they are not bf16 values
+    assert np.mean([O.bf16_round(float(v)) == float(np.float32(v)) for v in og2[0][:200]]) < 0.2
+
+
 # ------------------------------------------------------------------------------------------- S4: perturbation
 def _lsq_oracle(K=2, B=8, n=64, f=12, noise=0.01, **kw):
     X, y, w_star = synth.least_squares_data(n, f, noise=noise, seed=7)

@@ -46,6 +46,26 @@ def test_static_row_norms_match_step_norms_twice_in_a_row(K, d):
     ctx.close()
 
 
+def test_static_row_norms_reduce_only_the_first_n_columns_of_padded_rows():
+    # rows whose stride is a multiple of 4 but whose length is not: the columns n .. ld-1 hold other data and must not count
+    import torch
+
+    K, ld, n = 5, 1004, 1001
+    rng = np.random.default_rng(3)
+    g = rng.standard_normal((K, ld)).astype(np.float32)
+    g[:, n:] = 100.0  # would dominate the norm if it were read
+    dg = torch.from_numpy(g).cuda()
+    out = torch.full((K,), -1.0, device="cuda")
+    for _ in range(2):
+        rc, msg = G.lsam_row_norms_static(dg, n, out, torch.cuda.current_stream())
+        assert rc == G.LSAM_OK, msg
+        np.testing.assert_allclose(out.cpu().numpy(), np.linalg.norm(g[:, :n].astype(np.float64), axis=1), rtol=1e-5)
+    # and a row length that IS a multiple of 4 inside a wider stride takes the 128-bit path
+    rc, msg = G.lsam_row_norms_static(dg, 1000, out, torch.cuda.current_stream())
+    assert rc == G.LSAM_OK, msg
+    np.testing.assert_allclose(out.cpu().numpy(), np.linalg.norm(g[:, :1000].astype(np.float64), axis=1), rtol=1e-5)
+
+
 def test_static_row_norms_reject_oversize_and_bad_arguments():
     import torch
 
