@@ -44,12 +44,22 @@ WORKLOADS = {
 LAMBDA0, MU, BETA, ETA_PRIME, GAMMA = 0.9, 0.9, 0.9, 1.0, 1e-12
 NOMINAL_HBM_GBS, FALLBACK_HBM_GBS, FALLBACK_BF16_TF = 8000.0, 6650.0, 1590.0
 FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x max SM clock
-# ncu counters of one update_kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) at the c4 shape with K = 4
-# replicas, see profiles/dram_traffic_c4_k4.md; traffic grows with (20 K + 12) d, so it is scaled to the K of the run.
-NCU_UPDATE_TRAFFIC = dict(workload="c4", K=4, bytes=6111971328.0)
-# the same for one update8f_kernel launch of the optimiser-only workload at K = 8, d = 25.6M (profiles/stream_kernels_c5_d25m.md);
-# traffic grows with (20 K + 12) d, so it is scaled to the d of the run (rows of at least 4 M elements: the same kernel)
-NCU_UPDATE_TRAFFIC_C5 = dict(K=8, d=25_600_000, bytes=4351901696.0)
+# ncu DRAM counters of one launch of the two update kernels live beside the summaries they were read from (profiles/);
+# they are scaled to the launch that is timed by its algorithmic bytes (20 K + 12) d.
+NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
+# The sample of each workload that the CPU oracle is timed on (fixed, so that the figure is a stable denominator):
+# replicas, samples per minibatch, steps.  The full model is always used.
+ORACLE_SAMPLE = {"c1": (4, 32, 20), "c2": (8, 16, 2), "c3": (2, 16, 1), "c4": (2, 8, 1)}
+
+
+def ncu_traffic(kernel, K, d):
+    """Measured DRAM bytes of one launch of `kernel`, scaled from the captured case to (K, d); None if not on record."""
+    try:
+        rec = json.load(open(NCU_TRAFFIC_FILE))[kernel]
+    except Exception:
+        return None, None
+    scale = (20.0 * K + 12.0) * d / ((20.0 * rec["K"] + 12.0) * rec["d"])
+    return rec["bytes"] * scale, f"ncu capture at K={rec['K']}, d={rec['d']} ({rec['source']}) scaled by (20K+12)d"
 
 
 def param_count(w):
@@ -91,14 +101,16 @@ def peaks():
 
 
 # ---------------------------------------------------------------------------------------------- algorithmic work per step
-def work_model(w, tc):
-    """Algorithmic bytes / flops per STEP of each kernel class (what the method must move or compute)."""
+def work_model(w, tc, grads_bf16=None):
+    """Algorithmic bytes / flops per STEP of each kernel class (what the launched kernels must move or compute).
+    grads_bf16: the tensor-core path stores both gradients in bf16 (its default), 2 instead of 4 bytes per element."""
     K, B, d = w["K"], w["B"], param_count(w)
     op = 2 if w["bf16"] else 4
+    gb = 2.0 if (tc if grads_bf16 is None else grads_bf16) else 4.0
     out = {}
     out["norm"] = dict(bytes=0.0 if tc else 4.0 * K * d)                     # read g1 (fused into the wgrad epilogue on the tensor-core path)
-    out["perturb"] = dict(bytes=(4.0 + (2.0 if tc else 4.0) + op) * K * d)   # read x, g1 (bf16 on the tensor-core path); write x~
-    out["update"] = dict(bytes=((2.0 if tc else 4.0) + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2 (bf16 on the tensor-core path), x rw, v rw, operand copy; y, acc rw
+    out["perturb"] = dict(bytes=(4.0 + gb + op) * K * d)                     # read x, g1; write x~
+    out["update"] = dict(bytes=(gb + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2, x rw, v rw, operand copy; y, acc rw
     if w["model"] in (MLP, RESMLP):
         ws = w["widths"]
         f_fwd = f_dg = f_wg = 0.0
@@ -108,7 +120,7 @@ def work_model(w, tc):
             f_fwd += 2.0 * B * i * o
             b_fwd += op * (i * o + B * i + B * o)
             f_wg += 2.0 * B * i * o
-            b_wg += (2.0 if tc else 4.0) * i * o + op * B * (i + o)         # tensor-core path: the gradient is written as bf16
+            b_wg += gb * i * o + op * B * (i + o)                           # the gradient is written in its storage type
             if l > 0:
                 f_dg += 2.0 * B * i * o
                 b_dg += op * (i * o + B * i + B * o)
@@ -207,56 +219,65 @@ def make_cfg(G, w, flags=0, K_total=0, k_offset=0):
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
-def oracle_baseline(w, X, Y, x0_row, budget_s=20.0):
-    """Time the oracle, as it stands, on a bounded sample of the workload: a subset of replicas and of each minibatch."""
-    import oracle as O
+class OracleSample:
+    """The oracle, as it stands, on a fixed bounded sample of the workload: a subset of the replicas and of each
+    minibatch, the full model.  timed_steps() runs `steps` ticks of it (centre updates included when due) and returns
+    the baseline record and the seconds per tick."""
 
-    cores = O.num_threads()
-    d = param_count(w)
-    lam = w.get("lambda0", LAMBDA0) / (w["eta"] * w["tau"])
-    if w["model"] == FLAT:
-        Ks, ds = w["K"], min(d, 4_000_000)
-        cfg = O.make_config(O.MODEL_FLAT, K=Ks, flat_d=ds, mu=MU, gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME)
-        rng = np.random.default_rng(0)
-        x0 = rng.standard_normal((Ks, ds))
-        g1 = (0.1 * rng.standard_normal((Ks, ds))).astype(np.float32)
-        o = O.Oracle(cfg, None, None, x0, x0.mean(0))
-        o.set_external_grads(g1, g1)
-        def tick():
+    def __init__(self, w, key, X, Y, x0_row):
+        import oracle as O
+
+        self.w, self.O = w, O
+        self.cores = O.num_threads()
+        d = param_count(w)
+        lam = w.get("lambda0", LAMBDA0) / (w["eta"] * w["tau"])
+        if w["model"] == FLAT:
+            self.Ks, self.ds, self.steps = w["K"], min(d, 4_000_000), 3
+            cfg = O.make_config(O.MODEL_FLAT, K=self.Ks, flat_d=self.ds, mu=MU, gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME)
+            rng = np.random.default_rng(0)
+            x0 = rng.standard_normal((self.Ks, self.ds))
+            g1 = (0.1 * rng.standard_normal((self.Ks, self.ds))).astype(np.float32)
+            self.o = O.Oracle(cfg, None, None, x0, x0.mean(0))
+            self.o.set_external_grads(g1, g1)
+            self.sample = f"K={self.Ks} replicas, d={self.ds} of {d} elements, {self.steps} steps per timing"
+        else:
+            Ks, Bs, self.steps = ORACLE_SAMPLE[key]
+            self.Ks, self.Bs = min(Ks, w["K"]), min(Bs, w["B"])
+            cfg = O.make_config(w["model"], widths=w["widths"], K=self.Ks, batch=self.Bs, gemm_dtype=O.GEMM_BF16 if w["bf16"] else O.GEMM_FP32, mu=MU,
+                                gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=w["n"])
+            x0 = np.repeat(x0_row[None, :].astype(np.float64), self.Ks, axis=0)
+            self.o = O.Oracle(cfg, X, Y, x0, x0_row.astype(np.float64))
+            self.sample = f"{self.Ks} of {w['K']} replicas x {self.Bs} of {w['B']} samples per minibatch, full model, {self.steps} step(s) per timing"
+
+    def timed_steps(self):
+        w, o = self.w, self.o
+        t0 = time.perf_counter()
+        for _ in range(self.steps):
             o.step(w["eta"], w["rho"])
             if o.should_couple():
                 o.couple()
+        dt = (time.perf_counter() - t0) / self.steps
+        if w["model"] == FLAT:
+            rec = dict(value=36.0 * self.Ks * self.ds / dt / 1e9, unit="GB/s (36 B per element-replica)")
+        else:
+            rec = dict(value=self.Ks * self.Bs / dt, unit="worker-samples/s")
+        rec.update(cores=min(self.cores, self.Ks), kind="oracle", sample=self.sample)
+        return rec, dt
 
-        tick()
-        t0 = time.perf_counter()
-        steps = 3
-        for _ in range(steps):
-            tick()
-        dt = (time.perf_counter() - t0) / steps
-        return dict(value=36.0 * Ks * ds / dt / 1e9, unit="GB/s (36 B per element-replica)", cores=min(cores, Ks), kind="oracle",
-                    sample=f"K={Ks} replicas, d={ds} of {d} elements, {steps} steps"), dt
-    # flops per worker-sample (12 per weight: two passes of fwd + dgrad + wgrad) and a measured-free guess of 1.5 GFLOP/s/core
-    flop_ws = 12.0 * d
-    Ks = min(w["K"], cores)
-    Bs = int(max(1, min(w["B"], budget_s * 1.5e9 / flop_ws)))
-    cfg = O.make_config(w["model"], widths=w["widths"], K=Ks, batch=Bs, gemm_dtype=O.GEMM_BF16 if w["bf16"] else O.GEMM_FP32, mu=MU,
-                        gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=w["n"])
-    x0 = np.repeat(x0_row[None, :].astype(np.float64), Ks, axis=0)
-    o = O.Oracle(cfg, X, Y, x0, x0_row.astype(np.float64))
-    steps = 1 if flop_ws * Bs > 2e9 else 5
-    t0 = time.perf_counter()
-    for _ in range(steps):
-        o.step(w["eta"], w["rho"])
-        if o.should_couple():
-            o.couple()
-    dt = (time.perf_counter() - t0) / steps
-    o.close()
-    return dict(value=Ks * Bs / dt, unit="worker-samples/s", cores=min(cores, Ks), kind="oracle",
-                sample=f"{Ks} of {w['K']} replicas x {Bs} of {w['B']} samples per minibatch, full model, {steps} step(s)"), dt
+    def close(self):
+        self.o.close()
+
+
+def oracle_baseline(w, key, X, Y, x0_row):
+    s = OracleSample(w, key, X, Y, x0_row)
+    out = s.timed_steps()
+    s.close()
+    return out
 
 
 def run_reference(args, w, metric, unit):
-    """--impl reference: the CPU oracle timed on bounded samples of the same workload (rank 0 only)."""
+    """--impl reference: the CPU oracle timed on the fixed bounded sample of the same workload (rank 0 only); every
+    warm-up or timed step of the run is one timing of that sample, on one oracle run that keeps going."""
     if int(os.environ.get("RANK", "0")) != 0:
         return
     import torch
@@ -264,80 +285,40 @@ def run_reference(args, w, metric, unit):
     inp = make_inputs(w, torch.device("cpu"), seed=0)
     X = None if inp["X"] is None else inp["X"].numpy()
     Y = None if inp["Y"] is None else inp["Y"].numpy()
-    x0_row = inp["y0"].numpy()
+    smp = OracleSample(w, args.workload, X, Y, inp["y0"].numpy())
     vals, dts = [], []
-    per = max(2.0, min(20.0, 120.0 / max(args.steps + args.warmup, 1)))
     for i in range(args.warmup + args.steps):
-        cb, dt = oracle_baseline(w, X, Y, x0_row, budget_s=per)
+        cb, dt = smp.timed_steps()
         if i >= args.warmup:
             vals.append(cb["value"])
             dts.append(dt)
+    smp.close()
     v = float(np.mean(vals))
     cb["value"] = v
     line = dict(impl="reference", metric=metric, value=v, unit=unit, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
                 ms_per_step=float(np.mean(dts) * 1e3), higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64",
-                data="synthetic", config=dict(workload=w["name"]), cpu_baseline=cb,
+                data="synthetic", config=workload_config(w), cpu_baseline=cb,
                 e2e=dict(value=v, unit=unit, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
 
 
-# ---------------------------------------------------------------------------------------------- main
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=4)
-    ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
-    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
-    ap.add_argument("--flat-d", type=int, default=None, help="c5 only: vector length of the sweep point")
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
-    ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
-    ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
-    ap.add_argument("--shard-workers", action="store_true",
-                    help="N > 1: one job of N*K workers with a single centre, K workers per GPU, accumulator all-reduce every tau steps "
-                         "(default: N independent copies of the workload)")
-    ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: when the state fits in L2)")
-    args = ap.parse_args()
-    w = dict(WORKLOADS[args.workload])
-    if args.flat_d and w["model"] == FLAT:
-        w["d"] = args.flat_d
-        w["name"] = f"optimiser-only sweep point d={args.flat_d}, K=8"
-    if args.replicas:
-        w["K"] = args.replicas
-        w["name"] += f" [K overridden to {args.replicas}]"
-    if args.noise_temp > 0.0:
-        w["noise_temp"] = args.noise_temp
-        w["name"] += f" [Langevin temperature {args.noise_temp}]"
-    if args.active_num != 256:
-        w["active_num"] = args.active_num
-        w["name"] += f" [workers ready with probability {args.active_num}/256 per tick]"
-    flat = w["model"] == FLAT
-    metric = "fused_update_hbm_gbs" if flat else "lsam_worker_samples_per_s"
-    unit = "GB/s" if flat else "worker-samples/s"
-    if args.impl == "reference":
-        return run_reference(args, w, metric, unit)
+def workload_config(w):
+    """The keys that name the workload; shared by both arms so that their records compare like with like."""
+    return dict(workload=w["name"], K=w["K"], batch=w["B"], d=param_count(w))
 
+
+# ---------------------------------------------------------------------------------------------- one workload on this rank's GPU
+def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True):
+    """Create the context, time `steps` steps after `warmup` untimed ones, and return the record of this workload
+    (rank 0; None on the other ranks).  A step is one pass of the whole hot path plus the centre update when it is due."""
     import torch
     import torch.distributed as dist
 
     from paper_2509_03110_b200 import binding as G
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    shard = bool(args.shard_workers)
-    if world > 1 or shard:
-        if world == 1:
-            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-            os.environ.setdefault("MASTER_PORT", "29541")
-        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
-    warm = max(args.warmup, 3)
-
+    flat = w["model"] == FLAT
+    unit = "GB/s" if flat else "worker-samples/s"
+    local = dev.index
     # sharded: every rank generates the same dataset and the same initial point (one job); else independent copies
     inp = make_inputs(w, dev, seed=0 if shard else rank)
     # Latency-bound workloads (state resident in L2) replay each tick as one CUDA graph; that needs a capturable stream.
@@ -345,8 +326,9 @@ def main():
     # auto: also where the kernels of a step are short (tens of microseconds each), so that launch gaps and the
     # per-launch events of the roofline pass would be a visible share of the step
     short_kernels = 4.0 * w["K"] * param_count(w) <= 1.2e9
-    use_graph = (small or short_kernels) if args.cuda_graph == "auto" else args.cuda_graph == "on"
-    cfg = make_cfg(G, w, flags=G.FLAG_CUDA_GRAPH if use_graph else 0, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0)
+    use_graph = (small or short_kernels) if cuda_graph == "auto" else cuda_graph == "on"
+    flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0)
+    cfg = make_cfg(G, w, flags=flags, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0)
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(work_stream)
@@ -380,7 +362,7 @@ def main():
             torch.cuda.synchronize()
 
     # ---- device-resident timing (value), with per-kernel-class events for the roofline
-    for _ in range(warm):
+    for _ in range(warmup):
         one_step()
     # Per-kernel CUDA events ride inside the timed region when a step is long (working set beyond L2); for the
     # latency-bound workloads they would distort it, so there the shares come from a second, separate run of the same steps.
@@ -391,6 +373,7 @@ def main():
     clocks = ClockSampler(local)
     barrier()
     clocks.start()
+
     def iterations_done():  # worker iterations since the context was created: every sync closes exactly K tau of them
         _, t_y, t_x = ctx.counters()
         return w["K"] * w["tau"] * t_y + int(t_x.sum())
@@ -398,34 +381,36 @@ def main():
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     it0 = iterations_done()
     e0.record(stream)
-    for _ in range(args.steps):
+    for _ in range(steps):
         one_step()
     e1.record(stream)
     barrier()
     clk = clocks.stop()
     ms = e0.elapsed_time(e1)
-    worker_iters_per_step = (iterations_done() - it0) / args.steps  # = K in lock-step mode
+    worker_iters_per_step = (iterations_done() - it0) / steps  # = K in lock-step mode
     if not events_in_timed:
         launches_timed = ctx.launch_count() - launches0
         ctx.profile_enable(True)
-        for _ in range(args.steps):
+        for _ in range(min(steps, 50)):
             one_step()
         barrier()
         launches0 = ctx.launch_count() - launches_timed
+    prof_steps = steps if events_in_timed else min(steps, 50)
     prof = ctx.profile_read()
     ctx.profile_enable(False)
     launches = ctx.launch_count() - launches0
-    if ctx.status() != 0:
-        raise SystemExit("device status word is not clean after the timed region")
+    st = ctx.status()
+    if st != 0:
+        raise SystemExit(f"{w['name']}: device status word is not clean after the timed region (lsam_status = {st}: {ctx.last_error()})")
     ms = max_over_ranks(ms, world, dev)
-    ms_step = ms / args.steps
+    ms_step = ms / steps
     units_step = (36.0 * worker_iters_per_step * d / 1e9) if flat else float(worker_iters_per_step * w["B"])
     value = whole_job_value(world, units_step, ms_step)
 
     # ---- end to end through the C ABI with host buffers (minibatch H2D and loss D2H inside the timed region)
     e2e = None
-    if not flat:
-        nst = min(args.steps, 8)
+    if with_e2e and not flat:
+        nst = min(steps, 8)
         nb = min(nst, 4)
         fin = w["widths"][0]
         t_now = ctx.counters()[0]
@@ -455,16 +440,15 @@ def main():
         ems = max_over_ranks(e0.elapsed_time(e1), world, dev)
         e2e = dict(value=whole_job_value(world, w["K"] * w["B"], ems / nst), unit=unit, h2d_bytes_per_step=int(xbs[0].numel() * 4 + ybs[0].numel() * 4),
                    d2h_bytes_per_step=int(4 * w["K"]), steps=nst)
-    else:
+    elif with_e2e:
         # optimiser-only: the gradients are the step's inputs; copy them from pinned host memory every step
         K = w["K"]
         hg = torch.empty(2, K, d, dtype=torch.float32).pin_memory() if d <= 64_000_000 else None
         if hg is not None:
             hg[0].copy_(inp["g1"].cpu())
             hg[1].copy_(inp["g2"].cpu())
-            out = np.zeros(d, np.float32)
             barrier()
-            nst = min(args.steps, 5)
+            nst = min(steps, 5)
             e0.record(stream)
             for _ in range(nst):
                 inp["g1"].copy_(hg[0], non_blocking=True)
@@ -479,36 +463,35 @@ def main():
             e2e = dict(value=None, unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K),
                        note="gradient buffers of this sweep point exceed the pinned-memory budget; run --flat-d <= 64000000")
 
+    uses_tc, grads_bf16 = ctx.uses_tcgen05(), ctx.uses_tcgen05() and not grad_fp32
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        ctx.close()
+        return None
 
     # ---- roofline of the dominant kernel class
     pk = peaks()
-    work = work_model(w, ctx.uses_tcgen05())
+    work = work_model(w, uses_tc, grads_bf16)
     frac_active = worker_iters_per_step / w["K"]  # waiting replicas are skipped by every kernel
     for wk_ in work.values():
-        for key in wk_:
-            wk_[key] *= frac_active
+        for k2 in wk_:
+            wk_[k2] *= frac_active
     tot_ms = sum(v[0] for v in prof.values())
     top = max(prof, key=lambda k: prof[k][0])
     tms, tn = prof[top]
     per_launch_s = tms / max(tn, 1) * 1e-3
     shares = {k: round(v[0] / tot_ms, 4) for k, v in prof.items() if v[1] > 0}
     wk = work.get(top, {})
-    launches_per_step = tn / args.steps
+    launches_per_step = tn / prof_steps
     roof = dict(kernel=top, share_of_kernel_time=shares.get(top), traffic=None, kernel_time_shares=shares)
-    if top == "update" and args.workload == NCU_UPDATE_TRAFFIC["workload"] and w["bf16"]:
-        roof["traffic"] = NCU_UPDATE_TRAFFIC["bytes"] * (20.0 * w["K"] + 12.0) / (20.0 * NCU_UPDATE_TRAFFIC["K"] + 12.0) if NCU_UPDATE_TRAFFIC["bytes"] else None
-        roof["traffic_source"] = "ncu at K=4 scaled by (20K+12)/(20*4+12); algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
-    if top == "update" and flat and w["K"] == NCU_UPDATE_TRAFFIC_C5["K"] and d >= (1 << 22) and d % 8 == 0:
-        roof["traffic"] = NCU_UPDATE_TRAFFIC_C5["bytes"] * d / NCU_UPDATE_TRAFFIC_C5["d"]
-        roof["traffic_source"] = "ncu at d=25.6M scaled by d; algorithmic bytes per launch %.4g" % wk_bytes(work, "update")
-    if top in ("gemm_fwd", "gemm_dgrad") and ctx.uses_tcgen05():
+    if top == "update" and frac_active == 1.0:
+        # which update kernel ran: bf16 gradients (padded rows, always multiples of 8) / long fp32 rows / the 4-per-thread form
+        kern = "update8_kernel" if grads_bf16 else ("update8f_kernel" if (flat and d >= (1 << 22) and d % 8 == 0) else None)
+        if kern:
+            roof["traffic"], roof["traffic_source"] = ncu_traffic(kern, w["K"], d)
+    if top in ("gemm_fwd", "gemm_dgrad") and uses_tc:
         ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
         roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_sustained"], peak_source=f"{pk['src']} (sustained bf16)")
-    elif top.startswith("gemm") and not ctx.uses_tcgen05() and not w["bf16"]:
+    elif top.startswith("gemm") and not uses_tc and not w["bf16"]:
         ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
         roof.update(bound="alu", achieved=ach, peak=FP32_ALU_TFLOPS, unit="TFLOP/s", frac=ach / FP32_ALU_TFLOPS, peak_source="148 SMs x 128 FMA lanes x 2 x 1.965 GHz")
     elif "bytes" in wk:
@@ -523,32 +506,131 @@ def main():
     stream_gbs = {}
     for k in ("norm", "perturb", "update"):
         if prof[k][1] > 0 and work[k]["bytes"] > 0:
-            stream_gbs[k] = round(work[k]["bytes"] * args.steps / (prof[k][0] * 1e-3) / 1e9, 1)
-    roof["streaming_kernels_gbs"] = stream_gbs
+            gbs = work[k]["bytes"] * prof_steps / (prof[k][0] * 1e-3) / 1e9
+            stream_gbs[k] = dict(gbs=round(gbs, 1), frac_of_measured_hbm=round(gbs / pk["hbm"], 3), frac_of_nominal_8TBs=round(gbs / NOMINAL_HBM_GBS, 3))
+    roof["streaming_kernels"] = stream_gbs
     gemm = {}
     for k in ("gemm_fwd", "gemm_dgrad", "gemm_wgrad"):
         if k in work and prof[k][1] > 0:
             sec = prof[k][0] * 1e-3
-            gemm[k] = dict(tflops=round(work[k]["flops"] * args.steps / sec / 1e12, 1), gbs=round(work[k]["bytes"] * args.steps / sec / 1e9, 1),
-                           frac_of_bf16_sustained=round(work[k]["flops"] * args.steps / sec / 1e12 / pk["bf16_sustained"], 3) if w["bf16"] else None)
+            tf = work[k]["flops"] * prof_steps / sec / 1e12
+            gemm[k] = dict(tflops=round(tf, 1), gbs=round(work[k]["bytes"] * prof_steps / sec / 1e9, 1),
+                           frac_of_bf16_sustained=round(tf / pk["bf16_sustained"], 3) if w["bf16"] else None,
+                           frac_of_bf16_burst=round(tf / pk["bf16"], 3) if w["bf16"] else None)
     roof["gemm_classes"] = gemm
 
     cpu = None
-    if not args.no_cpu_baseline:
+    if with_cpu:
         X = None if inp["X"] is None else inp["X"].cpu().numpy()
         Y = None if inp["Y"] is None else inp["Y"].cpu().numpy()
-        cpu, _ = oracle_baseline(w, X, Y, inp["y0"].cpu().numpy())
+        cpu, _ = oracle_baseline(w, key, X, Y, inp["y0"].cpu().numpy())
 
-    line = dict(metric=metric, value=value, unit=unit, n_gpus=world, steps=args.steps, warmup=warm, ms_per_step=ms_step,
-                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="bf16" if w["bf16"] else "f32", data="synthetic",
-                config=dict(workload=w["name"], K=w["K"], batch=w["B"], d=d, gemm="tcgen05" if ctx.uses_tcgen05() else "simt", cuda_graph=bool(use_graph),
-                            l2=("working set larger than L2" if not small else "L2-resident state (latency-bound workload)") +
-                               ("" if events_in_timed else "; kernel shares and roofline from a separate pass over the same steps with per-launch events"),
-                            parallelism=(f"{world * w['K']} workers sharded over {world} GPU(s), one centre, accumulator all-reduce every tau steps" if shard
-                                         else ("replicas only" if world > 1 else "1 GPU"))),
-                clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)
-    print(json.dumps(line))
+    cfgd = workload_config(w)
+    cfgd.update(gemm="tcgen05" if uses_tc else "simt", cuda_graph=bool(use_graph),
+                l2=("working set larger than L2" if not small else "L2-resident state (latency-bound workload)") +
+                   ("" if events_in_timed else "; kernel shares and roofline from a separate pass over the same steps with per-launch events"),
+                parallelism=(f"{world * w['K']} workers sharded over {world} GPU(s), one centre, accumulator all-reduce every tau steps" if shard
+                             else ("replicas only" if world > 1 else "1 GPU")))
+    if w["bf16"]:
+        cfgd["grad_storage"] = "bf16" if grads_bf16 else "fp32"
+    rec = dict(metric="fused_update_hbm_gbs" if flat else "lsam_worker_samples_per_s", value=value, unit=unit, ms_per_step=ms_step,
+               dtype="bf16" if w["bf16"] else "f32", config=cfgd, clocks=clk, e2e=e2e, gpu_launches=int(launches), roofline=roof, cpu_baseline=cpu)
     ctx.close()
+    return rec
+
+
+# What the default invocation measures after the headline workload, a few hundred milliseconds each, so that one run carries
+# the whole metric: the optimiser-only sweep at its five sizes and the three smaller model workloads.
+OTHER_WORKLOADS = [("c5", dict(d=1_000_000), 1000), ("c5", dict(d=11_200_000), 300), ("c5", dict(d=25_600_000), 150), ("c5", dict(d=86_000_000), 50),
+                   ("c5", dict(d=256_000_000), 20), ("c1", {}, 95), ("c2", {}, 400), ("c3", {}, 100)]
+
+
+# ---------------------------------------------------------------------------------------------- main
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=4)
+    ap.add_argument("--workload", default="c4", choices=sorted(WORKLOADS))
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--flat-d", type=int, default=None, help="c5 only: vector length of the sweep point")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--others", default="auto", choices=["auto", "on", "off"],
+                    help="also time the sweep sizes and the smaller workloads (auto: on one GPU with the default workload)")
+    ap.add_argument("--replicas", type=int, default=None, help="override K (small cases for profiler captures)")
+    ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
+    ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
+    ap.add_argument("--grad-fp32", action="store_true", help="tensor-core path: store the gradients in fp32 instead of bf16")
+    ap.add_argument("--shard-workers", action="store_true",
+                    help="N > 1: one job of N*K workers with a single centre, K workers per GPU, accumulator all-reduce every tau steps "
+                         "(default: N independent copies of the workload)")
+    ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: when the state fits in L2)")
+    args = ap.parse_args()
+    w = dict(WORKLOADS[args.workload])
+    modified = False
+    if args.flat_d and w["model"] == FLAT:
+        w["d"] = args.flat_d
+        w["name"] = f"optimiser-only sweep point d={args.flat_d}, K=8"
+    if args.replicas:
+        w["K"] = args.replicas
+        w["name"] += f" [K overridden to {args.replicas}]"
+        modified = True
+    if args.noise_temp > 0.0:
+        w["noise_temp"] = args.noise_temp
+        w["name"] += f" [Langevin temperature {args.noise_temp}]"
+        modified = True
+    if args.active_num != 256:
+        w["active_num"] = args.active_num
+        w["name"] += f" [workers ready with probability {args.active_num}/256 per tick]"
+        modified = True
+    flat = w["model"] == FLAT
+    metric = "fused_update_hbm_gbs" if flat else "lsam_worker_samples_per_s"
+    unit = "GB/s" if flat else "worker-samples/s"
+    if args.impl == "reference":
+        return run_reference(args, w, metric, unit)
+
+    import torch
+    import torch.distributed as dist
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    shard = bool(args.shard_workers)
+    if world > 1 or shard:
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29541")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+
+    rec = run_workload(args.workload, w, args.steps, args.warmup, dev, rank, world, shard=shard, cuda_graph=args.cuda_graph,
+                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline)
+    others = []
+    want_others = args.others == "on" or (args.others == "auto" and world == 1 and args.workload == "c4" and not modified and not shard)
+    if want_others and world == 1:
+        for key, over, nsteps in OTHER_WORKLOADS:
+            torch.cuda.empty_cache()
+            ow = dict(WORKLOADS[key])
+            ow.update(over)
+            if "d" in over:
+                ow["name"] = f"optimiser-only sweep point d={over['d']}, K={ow['K']}"
+            r = run_workload(key, ow, nsteps, 5, dev, rank, world, cuda_graph="auto", with_e2e=False, with_cpu=False)
+            ro = r["roofline"]
+            others.append(dict(workload=r["config"]["workload"], metric=r["metric"], value=r["value"], unit=r["unit"], ms_per_step=r["ms_per_step"], steps=nsteps, warmup=5,
+                               config=r["config"], clocks=r["clocks"], gpu_launches=r["gpu_launches"],
+                               roofline=dict(kernel=ro["kernel"], bound=ro.get("bound"), achieved=ro.get("achieved"), peak=ro.get("peak"), unit=ro.get("unit"),
+                                             frac=ro.get("frac"), traffic=ro.get("traffic"), share_of_kernel_time=ro.get("share_of_kernel_time"),
+                                             streaming_kernels=ro.get("streaming_kernels"), gemm_classes=ro.get("gemm_classes"))))
+    if rank == 0:
+        line = dict(metric=rec["metric"], value=rec["value"], unit=rec["unit"], n_gpus=world, steps=args.steps, warmup=args.warmup, ms_per_step=rec["ms_per_step"],
+                    higher_is_better=True, scaling="weak", vs_baseline=None, dtype=rec["dtype"], data="synthetic", config=rec["config"], clocks=rec["clocks"],
+                    e2e=rec["e2e"], gpu_launches=rec["gpu_launches"], roofline=rec["roofline"], cpu_baseline=rec["cpu_baseline"])
+        if others:
+            line["other_workloads"] = others
+        print(json.dumps(line))
     if world > 1 or shard:
         dist.destroy_process_group()
 

@@ -321,6 +321,9 @@ class Lsam:
     def status(self):
         return int(lib().lsam_status(self._h))
 
+    def last_error(self):
+        return (lib().lsam_last_error(self._h) or b"").decode()
+
     def save_checkpoint(self):
         """The whole state of the run as a numpy byte array (host)."""
         n = int(lib().lsam_checkpoint_bytes(self._h))

@@ -45,9 +45,10 @@ def median_abs_rows(got, want):
 #  bf16 paths: the L2 error has a heavy tail of discrete decisions (a ReLU sign, a bf16 rounding boundary) that the fp32
 #  accumulation of the device and the double accumulation of the oracle take differently; each one moves a few elements
 #  by about their own size, so the largest element says nothing.  What a correct implementation keeps small is the bulk:
-#  the MEDIAN element error stays at the rounding level, BULK_DIVISOR times below the L2 tolerance.
+#  the MEDIAN element error stays near the rounding level (bf16 gradient storage alone: about 1e-3 of the row RMS), and is
+#  held BULK_DIVISOR times below the L2 tolerance: 5e-3, which a systematic relative error of 0.75 % would already exceed.
 ELEMENTWISE_FACTOR = 50.0
-BULK_DIVISOR = 8.0
+BULK_DIVISOR = 4.0
 
 
 def elem_stat(got, want, bf16):

@@ -102,7 +102,6 @@ def test_c3_full_shape_sixteen_free_running_ticks_of_two_replicas():
                 for name, got, want in (("g1", first["g1"][i], og1[i]), ("g2", first["g2"][i], og2[i])):
                     e = rel_l2(got, want)
                     assert e <= TOL_GRAD_BF16_FULL, (name, k, e, _layer_errors(w["widths"], got, want))
-                    assert median_abs_rows(got, want) <= TOL_GRAD_BF16_FULL / BULK_DIVISOR, (name, k, median_abs_rows(got, want))
                 assert rel_l2(first["xp"][i], oxp16[i]) <= 1e-3
     assert o.should_couple()
     s = o.read_state()
