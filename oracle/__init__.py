@@ -17,6 +17,7 @@ _LIB = os.path.join(_HERE, "liblsam_oracle.so")
 
 MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT = 0, 1, 2, 3
 GEMM_FP32, GEMM_BF16 = 0, 1
+KERNEL_GAUSSIAN, KERNEL_EXP_POWER, KERNEL_CAUCHY, KERNEL_MATERN32 = 0, 1, 2, 3
 
 
 def build(force=False):
@@ -36,6 +37,7 @@ class OracleConfig(C.Structure):
         ("stale_max", C.c_int32), ("active_num", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_double), ("gamma", C.c_double), ("lam", C.c_double),
         ("beta", C.c_double), ("eta_prime", C.c_double), ("noise_temp", C.c_double),
+        ("kernel_kind", C.c_int32), ("dp_average", C.c_int32), ("kernel_param", C.c_double),
     ]
 
 
@@ -76,6 +78,11 @@ def lib():
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
         L.oracle_noise4.restype = None
         L.oracle_noise4.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64, C.c_uint32, C.c_uint64, vp]
+        L.oracle_kernel_phi.restype = C.c_double
+        L.oracle_kernel_phi.argtypes = [C.c_int32, C.c_double, C.c_double, C.c_double]
+        L.oracle_kernel_weight.restype = C.c_double
+        L.oracle_kernel_weight.argtypes = [C.c_int32, C.c_double, C.c_double, C.c_double]
+        L.oracle_read_pull_weights.argtypes = [vp, vp]
         L.oracle_mix64.restype = C.c_uint64
         L.oracle_mix64.argtypes = [C.c_uint64]
         L.oracle_hash.restype = C.c_uint64
@@ -90,7 +97,8 @@ def lib():
 
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, nesterov=1, gamma=1e-12,
-                lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, active_num=256, noise_temp=0.0):
+                lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, active_num=256, noise_temp=0.0,
+                kernel_kind=KERNEL_GAUSSIAN, kernel_param=0.0, dp_average=0):
     """Float hyper-parameters are taken at their fp32 value, the precision the C-ABI carries them in."""
     c = OracleConfig()
     c.model = model
@@ -104,6 +112,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, ne
     f32 = lambda v: float(np.float32(v))
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = f32(mu), f32(gamma), f32(lam), f32(beta), f32(eta_prime)
     c.noise_temp = f32(noise_temp)
+    c.kernel_kind, c.kernel_param, c.dp_average = int(kernel_kind), f32(kernel_param), int(dp_average)
     return c
 
 
@@ -150,6 +159,14 @@ def noise4(seed, t, k, seg, group):
     out = np.zeros(4, dtype=np.float64)
     lib().oracle_noise4(seed, t, k, seg, group, _ptr(out))
     return out
+
+
+def kernel_phi(kind, lam, param, r):
+    return float(lib().oracle_kernel_phi(int(kind), float(lam), float(param), float(r)))
+
+
+def kernel_weight(kind, lam, param, r):
+    return float(lib().oracle_kernel_weight(int(kind), float(lam), float(param), float(r)))
 
 
 def mix64(z):
@@ -256,6 +273,11 @@ class Oracle:
         g2 = np.ascontiguousarray(g2, dtype=np.float32).reshape(self.K, self.d)
         self._keep = [g1, g2]
         assert lib().oracle_set_external_grads(self._h, _ptr(g1), _ptr(g2)) == 0
+
+    def read_pull_weights(self):
+        w = np.zeros(self.K)
+        assert lib().oracle_read_pull_weights(self._h, _ptr(w)) == 0
+        return w
 
     def read_active(self):
         a = np.zeros(self.K, dtype=np.int32)

@@ -4,6 +4,7 @@
 //   * SAM perturbation  x~ = x + rho * grad f(x; xi) / (||grad f(x; xi)|| + gamma)      (Eq. 3, look-back map)
 //   * SAM gradient      g  = grad f(x~; xi), the SAME minibatch xi in both passes        (Theorems 3 and 4)
 //   * worker score      G  = g + lambda (x - y)                                          (Algorithm 1, first update)
+//                       (other stationary kernels phi(x - y): G = g + grad phi(x - y), Corollary 8 and its remark)
 //   * sampler           Nesterov-momentum step on G                                      (Section 4.3)
 //   * centre update     g' = (1/(n tau)) sum_i sum_s x_s^(i) - y ;  g = g' + beta (g' - g'_prev) ;
 //                       y <- y + eta' g ; counters reset                                 (Algorithm 2, sync branch)
@@ -77,6 +78,30 @@ inline float bf16_round(float v) {
   float r;
   std::memcpy(&r, &u, 4);
   return r;
+}
+
+// ---- stationary kernels k(x, y) = phi(x - y), radial: phi depends on r = ||x - y|| only (Corollary 8 and its remark).
+// kernel_phi is the kernel itself, kernel_weight the factor w(r) = phi'(r) / r of its gradient grad phi(z) = w(||z||) z.
+//   GAUSSIAN     phi = (lambda / 2) r^2                                   w = lambda          (Algorithm 1)
+//   EXP_POWER    phi = (lambda / a) r^a, a = param in [1, 2]              w = lambda r^(a-2)  (w(0) := 0 for a < 2)
+//   CAUCHY       phi = (lambda s^2 / 2) log(1 + r^2 / s^2), s = param     w = lambda / (1 + r^2 / s^2)
+//   MATERN32     exp(-phi) = (1 + c r) exp(-c r), c = sqrt(lambda)        w = lambda / (1 + c r)
+// Every one of them has w -> lambda for r -> 0 (a = 2 / s -> infinity / c r -> 0), the Gaussian pull.
+inline double kernel_phi(int kind, double lambda, double param, double r) {
+  switch (kind) {
+    case ORACLE_KERNEL_EXP_POWER: return lambda / param * std::pow(r, param);
+    case ORACLE_KERNEL_CAUCHY: return 0.5 * lambda * param * param * std::log1p(r * r / (param * param));
+    case ORACLE_KERNEL_MATERN32: { const double cr = std::sqrt(lambda) * r; return cr - std::log1p(cr); }
+    default: return 0.5 * lambda * r * r;
+  }
+}
+inline double kernel_weight(int kind, double lambda, double param, double r) {
+  switch (kind) {
+    case ORACLE_KERNEL_EXP_POWER: return (param == 2.0) ? lambda : (r > 0.0 ? lambda * std::pow(r, param - 2.0) : 0.0);
+    case ORACLE_KERNEL_CAUCHY: return lambda / (1.0 + r * r / (param * param));
+    case ORACLE_KERNEL_MATERN32: return lambda / (1.0 + std::sqrt(lambda) * r);
+    default: return lambda;
+  }
 }
 
 struct Layer {
@@ -286,7 +311,7 @@ struct oracle_ctx {
   int64_t t = 0, t_y = 0;
   std::vector<int64_t> t_x;
   std::vector<int64_t> ver_at_step;  // ver_at_step[s] = centre version that was current when step s started
-  std::vector<double> loss, gn1, gn2;
+  std::vector<double> loss, gn1, gn2, pullw;
   std::vector<int32_t> active;       // which workers stepped at the last tick
   const float* eg1 = nullptr;
   const float* eg2 = nullptr;
@@ -322,7 +347,11 @@ oracle_ctx* oracle_create(const oracle_config* cfg, const float* X, const void* 
   if (!cfg || !x0 || !y0) return nullptr;
   oracle_ctx* o = new oracle_ctx();
   o->cfg = *cfg;
-  if (!build_net(*cfg, o->net) || cfg->tau < 1 || cfg->stale_max < 0) {
+  const bool kernel_ok = cfg->kernel_kind == ORACLE_KERNEL_GAUSSIAN ||
+                         (cfg->kernel_kind == ORACLE_KERNEL_EXP_POWER && cfg->kernel_param >= 1.0 && cfg->kernel_param <= 2.0) ||
+                         (cfg->kernel_kind == ORACLE_KERNEL_CAUCHY && cfg->kernel_param > 0.0) || cfg->kernel_kind == ORACLE_KERNEL_MATERN32;
+  const bool dp_ok = !cfg->dp_average || cfg->active_num <= 0 || cfg->active_num >= 256;  // synchronous by definition
+  if (!build_net(*cfg, o->net) || cfg->tau < 1 || cfg->stale_max < 0 || !kernel_ok || !dp_ok) {
     delete o;
     return nullptr;
   }
@@ -350,6 +379,7 @@ oracle_ctx* oracle_create(const oracle_config* cfg, const float* X, const void* 
   o->loss.assign(K, 0.0);
   o->gn1.assign(K, 0.0);
   o->gn2.assign(K, 0.0);
+  o->pullw.assign(K, 0.0);
   o->active.assign(K, 1);
   return o;
 }
@@ -405,28 +435,44 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
       o->active[k] = (ready[k] && rank < budget) ? 1 : 0;
     }
   }
+  // ---- ascent gradient g1_k = grad of the minibatch loss at x_k (workers are independent: OpenMP over them only)
+  std::vector<std::vector<int32_t>> idx_of(K);
+  std::vector<std::vector<double>> a0_of(K);
+  std::vector<int32_t> ver_of(K, 0);
 #pragma omp parallel for schedule(dynamic, 1)
   for (int k = 0; k < K; ++k) {
     if (!o->active[k]) continue;
-    double* x = o->x.data() + (size_t)k * d;
-    double* v = o->v.data() + (size_t)k * d;
-    double* acc = o->acc.data() + (size_t)k * d;
     double* g1 = o->g1.data() + (size_t)k * d;
-    double* g2 = o->g2.data() + (size_t)k * d;
-    double* xp = o->xp.data() + (size_t)k * d;
-    std::vector<int32_t> idx(c.model == ORACLE_MODEL_FLAT ? 0 : c.batch);
-    int32_t s, ver;
-    schedule_of(o, t, k, idx.data(), &s, &ver);
-    const double* yk = o->y_hist[ver].data();  // possibly stale centre seen by this worker
-    std::vector<double> a0;
-    // ascent gradient g1 = grad of the minibatch loss at x_k
+    idx_of[k].resize(c.model == ORACLE_MODEL_FLAT ? 0 : c.batch);
+    int32_t s;
+    schedule_of(o, t, k, idx_of[k].data(), &s, &ver_of[k]);
     if (c.model == ORACLE_MODEL_FLAT) {
       for (int64_t j = 0; j < d; ++j) g1[j] = (double)o->eg1[(size_t)k * d + j];
       o->loss[k] = 0.0;
     } else {
-      gather_inputs(o->net, o->X, idx.data(), c.batch, a0);
-      o->loss[k] = net_loss_grad(o->net, x, a0, c.batch, o->Yf, o->Yi, idx.data(), g1, nullptr);
+      gather_inputs(o->net, o->X, idx_of[k].data(), c.batch, a0_of[k]);
+      o->loss[k] = net_loss_grad(o->net, o->x.data() + (size_t)k * d, a0_of[k], c.batch, o->Yf, o->Yi, idx_of[k].data(), g1, nullptr);
     }
+  }
+  // Synchronous data parallelism (the DP-SGD / DP-SAM baselines of Section 5.2: the workers' gradients are aggregated at
+  // every iteration): every worker continues with the mean over the workers, k ascending, of this pass's gradients.
+  auto average_over_workers = [&](std::vector<double>& g) {
+    std::vector<double> mean((size_t)d, 0.0);
+    for (int k = 0; k < K; ++k)
+      for (int64_t j = 0; j < d; ++j) mean[(size_t)j] += g[(size_t)k * d + j];
+    for (int64_t j = 0; j < d; ++j) mean[(size_t)j] /= (double)K;
+    for (int k = 0; k < K; ++k)
+      for (int64_t j = 0; j < d; ++j) g[(size_t)k * d + j] = mean[(size_t)j];
+  };
+  if (c.dp_average) average_over_workers(o->g1);
+  // ---- look-back map and descent gradient
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int k = 0; k < K; ++k) {
+    if (!o->active[k]) continue;
+    const double* x = o->x.data() + (size_t)k * d;
+    const double* g1 = o->g1.data() + (size_t)k * d;
+    double* g2 = o->g2.data() + (size_t)k * d;
+    double* xp = o->xp.data() + (size_t)k * d;
     double ss = 0.0;
     for (int64_t j = 0; j < d; ++j) ss += g1[j] * g1[j];
     const double n1 = std::sqrt(ss);
@@ -437,14 +483,31 @@ int oracle_step(oracle_ctx* o, double eta, double rho) {
     if (c.model == ORACLE_MODEL_FLAT) {
       for (int64_t j = 0; j < d; ++j) g2[j] = (double)o->eg2[(size_t)k * d + j];
     } else {
-      net_loss_grad(o->net, xp, a0, c.batch, o->Yf, o->Yi, idx.data(), g2, nullptr);
+      net_loss_grad(o->net, xp, a0_of[k], c.batch, o->Yf, o->Yi, idx_of[k].data(), g2, nullptr);
     }
+  }
+  if (c.dp_average) average_over_workers(o->g2);
+  // ---- sampler
+#pragma omp parallel for schedule(dynamic, 1)
+  for (int k = 0; k < K; ++k) {
+    if (!o->active[k]) continue;
+    double* x = o->x.data() + (size_t)k * d;
+    double* v = o->v.data() + (size_t)k * d;
+    double* acc = o->acc.data() + (size_t)k * d;
+    const double* g2 = o->g2.data() + (size_t)k * d;
+    const double* yk = o->y_hist[ver_of[k]].data();  // possibly stale centre seen by this worker
     double ss2 = 0.0;
     for (int64_t j = 0; j < d; ++j) ss2 += g2[j] * g2[j];
     o->gn2[k] = std::sqrt(ss2);
-    // sampler: momentum step on G = g2 + lambda (x - y); the pull is evaluated at x_k, not at x~
+    // pull of the stationary kernel k(x, y) = phi(x - y) (Corollary 8 and the remark after it): grad_x phi = w(r) (x - y)
+    // with r = ||x - y||; the Gaussian kernel of Algorithm 1 has the constant weight lambda
+    double r2 = 0.0;
+    for (int64_t j = 0; j < d; ++j) r2 += (x[j] - yk[j]) * (x[j] - yk[j]);
+    const double wk = kernel_weight(c.kernel_kind, c.lambda, c.kernel_param, std::sqrt(r2));
+    o->pullw[k] = wk;
+    // momentum step on G = g2 + grad_x phi(x - y); the pull is evaluated at x_k, not at x~
     for (int64_t j = 0; j < d; ++j) {
-      const double G = g2[j] + c.lambda * (x[j] - yk[j]);  // Algorithm 1, first update: the gradient as computed
+      const double G = g2[j] + wk * (x[j] - yk[j]);  // Algorithm 1, first update: the gradient as computed
       v[j] = c.mu * v[j] + G;
       x[j] = c.nesterov ? x[j] - eta * (G + c.mu * v[j]) : x[j] - eta * v[j];
     }
@@ -569,6 +632,14 @@ int oracle_set_external_grads(oracle_ctx* o, const float* g1, const float* g2) {
   if (!o || o->cfg.model != ORACLE_MODEL_FLAT) return 1;
   o->eg1 = g1;
   o->eg2 = g2;
+  return 0;
+}
+
+double oracle_kernel_phi(int32_t kind, double lambda, double param, double r) { return kernel_phi(kind, lambda, param, r); }
+double oracle_kernel_weight(int32_t kind, double lambda, double param, double r) { return kernel_weight(kind, lambda, param, r); }
+int oracle_read_pull_weights(const oracle_ctx* o, double* w) {
+  if (!o || !w) return 1;
+  std::memcpy(w, o->pullw.data(), sizeof(double) * (size_t)o->cfg.K);
   return 0;
 }
 

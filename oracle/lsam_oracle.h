@@ -3,7 +3,8 @@
  *
  * TEST INFRASTRUCTURE ONLY.  This is a plain, slow, double-precision restatement of
  * Algorithm 2 (asynchronous distributed LSAM) with the SAM perturbation of Eq. 3 and the
- * Gaussian-kernel pull of Algorithm 1 (first update line).  It shares no code with the CUDA
+ * Gaussian-kernel pull of Algorithm 1 (first update line); optionally the pull of another
+ * stationary kernel (Corollary 8), or the synchronous gradient averaging of the DP baselines.  It shares no code with the CUDA
  * library and must never be reached from the product path: only the test-suite, the smoke
  * check and the benchmark's CPU-baseline leg may load it.
  *
@@ -29,6 +30,8 @@ extern "C" {
 
 enum { ORACLE_MODEL_LSQ = 0, ORACLE_MODEL_MLP = 1, ORACLE_MODEL_RESMLP = 2, ORACLE_MODEL_FLAT = 3 };
 enum { ORACLE_GEMM_FP32 = 0, ORACLE_GEMM_BF16 = 1 };
+/* Stationary kernels k(x, y) = phi(x - y) of Corollary 8 and the remark after it; see kernel_phi in the source. */
+enum { ORACLE_KERNEL_GAUSSIAN = 0, ORACLE_KERNEL_EXP_POWER = 1, ORACLE_KERNEL_CAUCHY = 2, ORACLE_KERNEL_MATERN32 = 3 };
 
 typedef struct {
   int32_t model;        /* ORACLE_MODEL_*                                                    */
@@ -50,6 +53,10 @@ typedef struct {
   double beta;          /* centre look-ahead factor                                          */
   double eta_prime;     /* centre step size                                                  */
   double noise_temp;    /* Langevin temperature T: x += sqrt(2 eta T) N(0, I) after the step; 0 = none */
+  int32_t kernel_kind;  /* ORACLE_KERNEL_*: the worker's pull is grad phi(x - y) = w(||x - y||) (x - y)           */
+  int32_t dp_average;   /* 1: synchronous data parallelism (Section 5.2, DP-SGD / DP-SAM): both gradients of a tick
+                           are averaged over the K workers before they are used; lock-step schedule only          */
+  double kernel_param;  /* EXP_POWER: exponent a in [1, 2]; CAUCHY: scale s > 0; others: unused                   */
 } oracle_config;
 
 typedef struct oracle_ctx oracle_ctx;
@@ -93,6 +100,11 @@ int oracle_read_step_info(const oracle_ctx*, double* loss, double* gnorm1, doubl
 int oracle_read_grads(const oracle_ctx*, double* g1, double* g2, double* x_pert);
 /* FLAT model: gradients used by the next steps, [K, d] fp32, borrowed. */
 int oracle_set_external_grads(oracle_ctx*, const float* g1, const float* g2);
+/* The kernel phi(r) and the weight w(r) = phi'(r) / r of its gradient, exposed so that they can be pinned against each other. */
+double oracle_kernel_phi(int32_t kind, double lambda, double param, double r);
+double oracle_kernel_weight(int32_t kind, double lambda, double param, double r);
+/* Pull weights w(||x_k - y||) used at the LAST tick ([K]). */
+int oracle_read_pull_weights(const oracle_ctx*, double* w);
 /* Which workers stepped at the LAST tick ([K], 1 = stepped). */
 int oracle_read_active(const oracle_ctx*, int32_t* active);
 /* Counters: t (steps), t_y (centre version), t_x [K]. */

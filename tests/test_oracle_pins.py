@@ -709,3 +709,150 @@ def test_noise_segments_follow_the_layers():
         z = np.concatenate([O.noise4(8, 0, 0, seg, g) for g in range((ln + 3) // 4)])[:ln]
         np.testing.assert_allclose(diff[off:off + ln], z, rtol=1e-9, atol=1e-12)
         off += ln
+
+
+# ------------------------------------------------------------------------------------------- stationary kernels (Corollary 8)
+KERNELS = [(O.KERNEL_GAUSSIAN, 0.0), (O.KERNEL_EXP_POWER, 1.0), (O.KERNEL_EXP_POWER, 1.5), (O.KERNEL_EXP_POWER, 2.0), (O.KERNEL_CAUCHY, 0.7), (O.KERNEL_MATERN32, 0.0)]
+
+
+@pytest.mark.parametrize("kind,param", KERNELS)
+def test_kernel_pull_is_the_gradient_of_the_kernel(kind, param):
+    # grad_z phi(||z||) = w(||z||) z: central finite differences of the kernel itself against the weight the step uses
+    rng = np.random.default_rng(kind * 10 + int(param * 4))
+    lam = 0.8
+    for scale in (0.05, 1.0, 7.0):
+        z = scale * rng.standard_normal(6)
+        w = O.kernel_weight(kind, lam, param, np.linalg.norm(z))
+        for i in range(6):
+            h = 1e-6 * max(1.0, abs(z[i]))
+            zp, zm = z.copy(), z.copy()
+            zp[i] += h
+            zm[i] -= h
+            fd = (O.kernel_phi(kind, lam, param, np.linalg.norm(zp)) - O.kernel_phi(kind, lam, param, np.linalg.norm(zm))) / (2 * h)
+            assert abs(fd - w * z[i]) <= 1e-7 * max(1.0, abs(w * z[i])), (scale, i, fd, w * z[i])
+    # the kernel vanishes at the centre and grows with the distance (a pull, never a push)
+    assert O.kernel_phi(kind, lam, param, 0.0) == 0.0
+    rs = np.linspace(0.01, 20, 200)
+    assert all(O.kernel_weight(kind, lam, param, r) > 0 for r in rs)
+    assert np.all(np.diff([O.kernel_phi(kind, lam, param, r) for r in rs]) > 0)
+
+
+def test_kernel_family_members_and_their_gaussian_limits():
+    from scipy.special import gamma as Gamma, kv
+
+    lam = 1.7
+    for r in (0.0, 0.3, 2.0, 11.0):
+        # exponential-power family of the remark after Corollary 8, Gaussian when the exponent is 2
+        assert O.kernel_phi(O.KERNEL_EXP_POWER, lam, 2.0, r) == O.kernel_phi(O.KERNEL_GAUSSIAN, lam, 0.0, r) == 0.5 * lam * r * r
+        assert O.kernel_weight(O.KERNEL_EXP_POWER, lam, 2.0, r) == lam
+        assert np.isclose(O.kernel_phi(O.KERNEL_EXP_POWER, lam, 1.0, r), lam * r, rtol=1e-15)
+        # Cauchy: exp(-phi) is the Cauchy / Student profile (1 + r^2 / s^2)^(-lam s^2 / 2); wide scale -> Gaussian
+        s = 0.9
+        assert np.isclose(np.exp(-O.kernel_phi(O.KERNEL_CAUCHY, lam, s, r)), (1 + r * r / (s * s)) ** (-lam * s * s / 2), rtol=1e-13)
+        assert np.isclose(O.kernel_weight(O.KERNEL_CAUCHY, lam, 1e9, r), lam, rtol=1e-12)
+        # Matern class with smoothness 3/2 and length scale l: the textbook correlation 2^(1-nu)/Gamma(nu) u^nu K_nu(u), u = sqrt(2 nu) r / l
+        if r > 0:
+            nu, ell = 1.5, np.sqrt(3.0 / lam)
+            u = np.sqrt(2 * nu) * r / ell
+            assert np.isclose(np.exp(-O.kernel_phi(O.KERNEL_MATERN32, lam, 0.0, r)), 2 ** (1 - nu) / Gamma(nu) * u ** nu * kv(nu, u), rtol=1e-10)
+    assert np.isclose(O.kernel_weight(O.KERNEL_MATERN32, lam, 0.0, 1e-9), lam, rtol=1e-8)
+    # tail condition (i) of Corollary 8 (phi >= c r^a for large r) for the exponential-power and Matern members
+    assert O.kernel_phi(O.KERNEL_MATERN32, lam, 0.0, 50.0) >= 0.5 * np.sqrt(lam) * 50.0
+    # invalid parameters are refused
+    for kind, param in ((O.KERNEL_EXP_POWER, 0.5), (O.KERNEL_EXP_POWER, 2.5), (O.KERNEL_CAUCHY, 0.0), (7, 0.0)):
+        cfg = O.make_config(O.MODEL_FLAT, K=1, flat_d=3, kernel_kind=kind, kernel_param=param)
+        assert not O.lib().oracle_create(O.C.byref(cfg), None, None, O._ptr(np.zeros(3)), O._ptr(np.zeros(3)), None)
+
+
+@pytest.mark.parametrize("kind,param", KERNELS)
+def test_worker_step_with_a_stationary_kernel(kind, param):
+    K, d = 3, 9
+    x0, y0, g1, g2 = synth.flat_problem(K, d, seed=5)
+    lam = 0.6
+    hp = dict(K=K, flat_d=d, lam=lam, tau=2, stale_max=1, seed=3)
+    o = O.Oracle(O.make_config(O.MODEL_FLAT, kernel_kind=kind, kernel_param=param, **hp), None, None, x0, y0)
+    o.set_external_grads(g1, g2)
+    ref = O.Oracle(O.make_config(O.MODEL_FLAT, **hp), None, None, x0, y0)  # Gaussian kernel
+    ref.set_external_grads(g1, g2)
+    for t in range(5):
+        before = o.read_state()
+        _, _, ver = o.read_schedule(t) if t == 0 else (None, None, None)
+        o.step(0.05, 0.1)
+        w = o.read_pull_weights()
+        # the weight is w(||x_k - y||) at the state before the step and the centre version the worker read (the current
+        # one here except for stale reads, which the Gaussian run below covers through its identical schedule)
+        if t == 0:
+            r = np.linalg.norm(before["x"] - before["y"][None, :], axis=1)
+            np.testing.assert_allclose(w, [O.kernel_weight(kind, float(np.float32(lam)), float(np.float32(param)), ri) for ri in r], rtol=1e-13)
+        if o.should_couple():
+            assert o.couple() == 0
+        ref.step(0.05, 0.1)
+        if ref.should_couple():
+            assert ref.couple() == 0
+        if kind == O.KERNEL_GAUSSIAN or (kind == O.KERNEL_EXP_POWER and param == 2.0):
+            np.testing.assert_array_equal(o.read_state()["x"], ref.read_state()["x"])  # the Gaussian path, bit for bit
+            np.testing.assert_array_equal(o.read_state()["y"], ref.read_state()["y"])
+    if kind not in (O.KERNEL_GAUSSIAN,) and not (kind == O.KERNEL_EXP_POWER and param == 2.0):
+        assert not np.allclose(o.read_state()["x"], ref.read_state()["x"])
+    # one worker, one step: the step IS the Gaussian step with lambda replaced by this worker's weight (up to the fp32
+    # value the configuration carries lambda in)
+    a = O.Oracle(O.make_config(O.MODEL_FLAT, K=1, flat_d=d, lam=lam, kernel_kind=kind, kernel_param=param), None, None, x0[:1], y0)
+    a.set_external_grads(g1[:1], g2[:1])
+    a.step(0.05, 0.1)
+    wk = a.read_pull_weights()[0]
+    b = O.Oracle(O.make_config(O.MODEL_FLAT, K=1, flat_d=d, lam=wk), None, None, x0[:1], y0)
+    b.set_external_grads(g1[:1], g2[:1])
+    b.step(0.05, 0.1)
+    np.testing.assert_allclose(a.read_state()["x"], b.read_state()["x"], rtol=1e-6)
+    np.testing.assert_allclose(a.read_state()["v"], b.read_state()["v"], rtol=1e-6, atol=1e-9)
+
+
+# ------------------------------------------------------------------------------------------- synchronous data parallelism (Section 5.2)
+@pytest.mark.parametrize("model", ["lsq", "mlp"])
+def test_dp_average_is_sam_on_the_union_of_the_workers_minibatches(model):
+    # DP-SGD / DP-SAM aggregate the workers' gradients at every iteration: with equal minibatch sizes the mean of the K
+    # per-worker gradients is the gradient of the mean loss over the union of the K minibatches, at both points of the SAM step
+    K, B = 3, 8
+    if model == "lsq":
+        X, Y, _ = synth.least_squares_data(64, 12, noise=0.01, seed=7)
+        w0 = np.random.default_rng(1).standard_normal(12)
+        mk = dict(model=O.MODEL_LSQ, widths=(12,))
+    else:
+        widths = (6, 8, 4)
+        X, Y = synth.gaussian_mixture(64, 6, 4, seed=1)
+        w0 = synth.mlp_init(widths, seed=2).astype(np.float64)
+        mk = dict(model=O.MODEL_MLP, widths=widths)
+    d = len(w0)
+    x0 = np.repeat(w0[None, :], K, axis=0)
+    hp = dict(lam=0.0, tau=1, seed=11, mu=0.9)
+    o = O.Oracle(O.make_config(mk["model"], widths=mk["widths"], K=K, batch=B, n_samples=64, dp_average=1, **hp), X, Y, x0, w0)
+    idx, _, _ = o.read_schedule(0)
+    union = idx.reshape(-1)
+    cu = O.make_config(mk["model"], widths=mk["widths"], K=1, batch=K * B, n_samples=64)
+    rho, gam = float(np.float32(0.1)), float(np.float32(1e-12))
+    _, gb1 = O.loss_grad(cu, X, Y, w0, union)
+    xp = w0 + rho * gb1 / (np.linalg.norm(gb1) + gam)
+    _, gb2 = O.loss_grad(cu, X, Y, xp, union)
+    o.step(0.05, 0.1)
+    g1, g2, oxp = o.read_grads()
+    for k in range(K):
+        np.testing.assert_allclose(g1[k], gb1, rtol=1e-11, atol=1e-14)
+        np.testing.assert_allclose(oxp[k], xp, rtol=1e-12)
+        np.testing.assert_allclose(g2[k], gb2, rtol=1e-10, atol=1e-14)
+    _, n1, _ = o.read_step_info()
+    np.testing.assert_allclose(n1, np.linalg.norm(gb1), rtol=1e-12)
+    # the update is the single-worker step driven by the union-batch gradients (gradient-fed model, which has no modes)
+    f = O.Oracle(O.make_config(O.MODEL_FLAT, K=1, flat_d=d, **hp), None, None, w0[None, :], w0)
+    f.set_external_grads(gb1[None, :], gb2[None, :])
+    f.step(0.05, 0.1)
+    s = o.read_state()
+    for k in range(K):
+        np.testing.assert_allclose(s["x"][k], f.read_state()["x"][0], rtol=1e-6, atol=1e-9)
+        np.testing.assert_array_equal(s["x"][k], s["x"][0])  # the replicas of a data-parallel job stay identical
+    # without the flag the workers use their own gradients and drift apart
+    p = O.Oracle(O.make_config(mk["model"], widths=mk["widths"], K=K, batch=B, n_samples=64, **hp), X, Y, x0, w0)
+    p.step(0.05, 0.1)
+    assert not np.array_equal(p.read_state()["x"][1], p.read_state()["x"][0])
+    # asynchronous progress contradicts the synchronous aggregation
+    bad = O.make_config(O.MODEL_FLAT, K=2, flat_d=3, dp_average=1, active_num=100)
+    assert not O.lib().oracle_create(O.C.byref(bad), None, None, O._ptr(np.zeros((2, 3))), O._ptr(np.zeros(3)), None)
