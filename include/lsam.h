@@ -52,6 +52,15 @@ enum {
 enum { LSAM_MODEL_LSQ = 0, LSAM_MODEL_MLP = 1, LSAM_MODEL_RESMLP = 2, LSAM_MODEL_FLAT = 3 };
 enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
 enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2 };
+/* Stationary kernels k(x, y) = phi(x - y) (Corollary 8 and the remark after it).  The worker's pull is
+ * grad_x phi(x - y) = w(r) (x - y), r = ||x_k - y|| with y the centre version the worker reads; the centre update is
+ * the one Algorithm 2 states (mean of the iterates minus the centre) for every kernel.
+ *   GAUSSIAN   phi = (lambda / 2) r^2,                               w = lambda              (Algorithm 1)
+ *   EXP_POWER  phi = (lambda / a) r^a, a = kernel_param in [1, 2],   w = lambda r^(a-2)      (w = 0 at r = 0 for a < 2)
+ *   CAUCHY     phi = (lambda s^2 / 2) log(1 + r^2 / s^2), s = kernel_param > 0,  w = lambda / (1 + r^2 / s^2)
+ *   MATERN32   exp(-phi) = (1 + c r) exp(-c r), c = sqrt(lambda),    w = lambda / (1 + c r)
+ * A non-Gaussian kernel costs one more pass over x per tick (the distances r_k, fixed-order reduction).           */
+enum { LSAM_KERNEL_GAUSSIAN = 0, LSAM_KERNEL_EXP_POWER = 1, LSAM_KERNEL_CAUCHY = 2, LSAM_KERNEL_MATERN32 = 3 };
 enum {
   LSAM_FLAG_KEEP_G1 = 1,   /* keep copies of the ascent gradient and (BF16 mode) of x~ for lsam_read_grads  */
   LSAM_FLAG_STEP_INFO = 2, /* also reduce ||g2_k|| every step (one extra read of the gradient buffer)      */
@@ -100,6 +109,12 @@ typedef struct {
   int32_t K_total;    /* workers of the whole job, n of Algorithm 2, when this context holds only a shard of them
                          (one context per GPU); 0 = K, a single context holding every worker                  */
   int32_t k_offset;   /* global index of this context's worker 0; workers k_offset .. k_offset + K - 1 live here */
+  int32_t kernel_kind; /* LSAM_KERNEL_*: the stationary kernel k(x, y) = phi(x - y) that couples a worker to the centre       */
+  float kernel_param;  /* EXP_POWER: exponent a in [1, 2]; CAUCHY: scale s > 0; others: unused                                */
+  int32_t dp_average;  /* 1: synchronous data parallelism (the DP-SGD / DP-SAM baselines of Section 5.2): both gradients of a
+                          tick are averaged over the K workers before they are used (perturbation along the averaged gradient
+                          and its norm, update with the averaged descent gradient).  Workers that start equal stay equal;
+                          lock-step schedule only, one context holds the whole job.  rho = 0 gives DP-SGD.                   */
 } lsam_config;
 
 /* Unpadded parameter count d of one replica, or -1 if the configuration is invalid. */

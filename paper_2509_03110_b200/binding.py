@@ -15,6 +15,7 @@ LSAM_OK, LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE, LSAM_ERR_STATE, LSAM_ERR_CUDA, LS
 MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT = 0, 1, 2, 3
 GEMM_FP32, GEMM_BF16 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+KERNEL_GAUSSIAN, KERNEL_EXP_POWER, KERNEL_CAUCHY, KERNEL_MATERN32 = 0, 1, 2, 3
 FLAG_KEEP_G1, FLAG_STEP_INFO, FLAG_CUDA_GRAPH, FLAG_GRAD_FP32 = 1, 2, 4, 8
 PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "loss", "bias_grad", "lsq_grad", "norm",
                 "perturb", "update", "couple", "copy"]
@@ -36,7 +37,7 @@ class LsamConfig(C.Structure):
         ("stale_max", C.c_int32), ("flags", C.c_int32), ("n_samples", C.c_int64), ("flat_d", C.c_int64),
         ("seed", C.c_uint64), ("mu", C.c_float), ("gamma", C.c_float), ("lam", C.c_float), ("beta", C.c_float),
         ("eta_prime", C.c_float), ("active_num", C.c_int32), ("noise_temp", C.c_float),
-        ("K_total", C.c_int32), ("k_offset", C.c_int32),
+        ("K_total", C.c_int32), ("k_offset", C.c_int32), ("kernel_kind", C.c_int32), ("kernel_param", C.c_float), ("dp_average", C.c_int32),
     ]
 
 
@@ -110,7 +111,7 @@ def lib():
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=IMPL_AUTO, mu=0.9, nesterov=1,
                 gamma=1e-12, lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, flags=0,
-                active_num=256, noise_temp=0.0, K_total=0, k_offset=0):
+                active_num=256, noise_temp=0.0, K_total=0, k_offset=0, kernel_kind=KERNEL_GAUSSIAN, kernel_param=0.0, dp_average=0):
     c = LsamConfig()
     c.model = model
     widths = list(widths)
@@ -123,6 +124,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=
     c.active_num = int(active_num)
     c.noise_temp = noise_temp
     c.K_total, c.k_offset = int(K_total), int(k_offset)
+    c.kernel_kind, c.kernel_param, c.dp_average = int(kernel_kind), kernel_param, int(dp_average)
     return c
 
 

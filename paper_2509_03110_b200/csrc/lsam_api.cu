@@ -40,7 +40,7 @@ struct Layout {
   int64_t nchunks = 0;
   bool vec4 = true;
   // byte offsets into the workspace
-  size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status;
+  size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status, gbar1, gbar2;
   size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage, xstage2, ystage2;
   size_t total = 0;
 };
@@ -55,6 +55,11 @@ bool plan(const lsam_config& c, Layout& L) {
   if (!(c.gamma > 0.f)) return false;
   if (c.active_num < 0 || c.active_num > 256) return false;
   if (!(c.noise_temp >= 0.f)) return false;
+  if (c.kernel_kind < KERNEL_GAUSSIAN || c.kernel_kind > KERNEL_MATERN32) return false;
+  if (c.kernel_kind == KERNEL_EXP_POWER && !(c.kernel_param >= 1.f && c.kernel_param <= 2.f)) return false;
+  if (c.kernel_kind == KERNEL_CAUCHY && !(c.kernel_param > 0.f)) return false;
+  // synchronous gradient averaging: every worker steps at every tick, and all workers of the job live in this context
+  if (c.dp_average != 0 && ((c.active_num != 0 && c.active_num != 256) || c.K_total != 0)) return false;
   if (c.K_total != 0) {  // a shard of a larger job: lock-step schedule only
     if (c.k_offset < 0 || c.K_total < c.K || c.k_offset > c.K_total - c.K) return false;
     if (c.active_num != 0 && c.active_num != 256) return false;
@@ -127,6 +132,8 @@ bool plan(const lsam_config& c, Layout& L) {
   L.yring = take(4 * (size_t)L.ring * ld);
   L.gprev = take(4 * ld);
   L.tmp = take(4 * ld);
+  L.gbar1 = c.dp_average ? take(4 * ld) : 0;  // worker-averaged gradients of the two passes
+  L.gbar2 = c.dp_average ? take(4 * ld) : 0;
   L.idx = take(4 * K * B * 2);     // step indices + scratch for lsam_read_schedule
   L.sched = take(4 * K * 8);       // stale, ver, slot + scratch copies
   L.partial = take(4 * K * (size_t)L.nchunks);
@@ -221,6 +228,7 @@ struct lsam_ctx {
   float* norm2() const { return at<float>(L.scalars) + cfg.K; }
   float* scale() const { return at<float>(L.scalars) + 2 * cfg.K; }
   float* loss() const { return at<float>(L.scalars) + 3 * cfg.K; }
+  float* pull_weight() const { return at<float>(L.scalars) + 5 * cfg.K; }  // [K] w(||x_k - y||) of a non-Gaussian kernel
   int* status() const { return at<int>(L.status); }
   int32_t* idx() const { return at<int32_t>(L.idx); }
   int32_t* idx_scratch() const { return at<int32_t>(L.idx) + (size_t)cfg.K * (cfg.batch > 0 ? cfg.batch : 1); }
@@ -313,10 +321,11 @@ struct FinArgs {
 };
 
 // ---- norm of [K, n] rows -> norm_out[K] (and scale[K] = rho / (norm + gamma) if scale_out)
-int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float rho, float* norm_out, float* scale_out) {
+// fused_ok = false: reduce the rows of g even on the tensor-core path (g is not what the weight-gradient epilogues just summed)
+int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, float rho, float* norm_out, float* scale_out, bool fused_ok = true) {
   float* partial = c->at<float>(c->L.partial);
   const int64_t nch = c->L.nchunks;
-  if (c->use_tc) {
+  if (c->use_tc && fused_ok) {
     // tensor-core path: the weight- and bias-gradient kernels of the pass just run have left the sums of squares of
     // all their blocks in the partial slots; only the fixed-order final sum remains
     FinArgs f{partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act(), {}};
@@ -344,6 +353,34 @@ int launch_perturb(lsam_ctx* c, const TG* g, int64_t ldg, int64_t n, bool vec4) 
   return LSAM_OK;
 }
 
+// out[j] = mean over the K workers of g[k][j] (fp32 rows, or the bf16 rows of the tensor-core path)
+int launch_mean_rows(lsam_ctx* c, const void* g, bool g_is_bf16, int64_t ldg, int64_t n, bool vec4, float* out) {
+  const int K = c->cfg.K;
+  if (vec4) {
+    const unsigned grid = (unsigned)ceil_div(n, (int64_t)256 * 4);
+    if (g_is_bf16) LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<4, bf16><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const bf16*>(g), ldg, K, n, out));
+    else LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<4, float><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const float*>(g), ldg, K, n, out));
+  } else {
+    const unsigned grid = (unsigned)ceil_div(n, (int64_t)256);
+    if (g_is_bf16) LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<1, bf16><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const bf16*>(g), ldg, K, n, out));
+    else LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<1, float><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const float*>(g), ldg, K, n, out));
+  }
+  return LSAM_OK;
+}
+
+// Non-Gaussian stationary kernel: weight[k] = w(||x_k - y_read(k)||) from one pass over x (fixed-order two-pass reduction)
+int launch_pull_weights(lsam_ctx* c) {
+  const Layout& L = c->L;
+  const int K = c->cfg.K;
+  const int64_t n = (c->cfg.model == LSAM_MODEL_FLAT) ? L.d : L.ld;  // padding elements are zero in x and in every centre version
+  float* partial = c->at<float>(L.partial);
+  dim3 grid((unsigned)ceil_div(n, norm_chunk<4>()), K);
+  if ((int64_t)grid.x > L.nchunks) return c->fail(LSAM_ERR_WORKSPACE, "pull weights: partial-sum buffer too small");
+  LAUNCH(c, LSAM_PROF_NORM, gap_sumsq_partial_kernel<<<grid, kNormThreads, 0, c->stream>>>(c->x(), L.ld, c->at<float>(L.yring), n, partial, L.nchunks, c->slot(), c->act()));
+  LAUNCH(c, LSAM_PROF_NORM, pull_weight_kernel<<<K, 256, 0, c->stream>>>(partial, L.nchunks, (int64_t)grid.x, c->cfg.kernel_kind, c->cfg.lambda, c->cfg.kernel_param, c->pull_weight(), c->act()));
+  return LSAM_OK;
+}
+
 UpdateArgs make_update_args(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n, float eta) {
   UpdateArgs a;
   a.g_mode = g_mode;
@@ -351,6 +388,7 @@ UpdateArgs make_update_args(lsam_ctx* c, const void* g, int g_mode, int64_t ldg,
   a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
   a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
   a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.k_offset = c->cfg.k_offset; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
+  a.lam_k = c->cfg.kernel_kind != KERNEL_GAUSSIAN ? c->pull_weight() : nullptr;
   a.sigma = c->cfg.noise_temp > 0.f ? sqrtf(2.0f * eta * c->cfg.noise_temp) : 0.f;
   a.seed = c->cfg.seed; a.tick = (uint64_t)c->t; a.seg = c->L.seg;
   return a;
@@ -601,49 +639,71 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   const bool gb = c->grads_bf16;
   const int g_mode = gb ? 2 : 0;
   const void* gptr = gb ? (const void*)c->at<bf16>(L.g1b) : (flat ? (const void*)c->eg2 : (const void*)c->g());
+  const bool dp = cfg.dp_average != 0;        // synchronous data parallelism: both gradients are averaged over the workers
+  const bool other_kernel = cfg.kernel_kind != KERNEL_GAUSSIAN;
+  float* gbar1 = c->at<float>(L.gbar1);
+  float* gbar2 = c->at<float>(L.gbar2);
+  // the fused update on the descent gradient: per-worker rows, or (dp) the one averaged row read by every worker (row stride 0)
+  auto finish_tick = [&](const void* g2src) -> int {
+    int rc2;
+    if (dp) {
+      if ((rc2 = launch_mean_rows(c, g2src, gb, ldg, n, vec4, gbar2)) != LSAM_OK) return rc2;
+      if ((cfg.flags & LSAM_FLAG_STEP_INFO) && (rc2 = launch_norm(c, gbar2, 0, n, vec4, 0.f, c->norm2(), nullptr, false)) != LSAM_OK) return rc2;
+    } else if (cfg.flags & LSAM_FLAG_STEP_INFO) {
+      if ((rc2 = launch_norm(c, reinterpret_cast<const float*>(g2src), ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc2;
+    }
+    if (other_kernel && (rc2 = launch_pull_weights(c)) != LSAM_OK) return rc2;
+    if (dp) return launch_update(c, gbar2, 0, 0, n, vec4, eta);
+    return launch_update(c, gptr, g_mode, ldg, n, vec4, eta);
+  };
   // ascent gradient, its norm, perturbation
   if (rho == 0.f && !flat && !L.g1keep) {
     // rho = 0: the perturbed point is x itself, so the two gradients coincide (entropy-/elastic-averaging SGD, the
-    // unperturbed case of Theorem 2): one gradient pass, no norm, no perturbation
+    // unperturbed case of Theorem 2; with dp_average: DP-SGD): one gradient pass, no norm, no perturbation
     phase.next("lsam S2 gradient (rho = 0: single pass)");
     if ((rc = grad_pass(c, false, c->loss(), gb)) != LSAM_OK) return rc;
     phase.next("lsam S6 update");
     if (cfg.flags & LSAM_FLAG_STEP_INFO) {
-      if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm1(), nullptr)) != LSAM_OK) return rc;
-      if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
+      if (dp) {
+        if ((rc = launch_mean_rows(c, gptr, gb, ldg, n, vec4, gbar1)) != LSAM_OK) return rc;
+        if ((rc = launch_norm(c, gbar1, 0, n, vec4, 0.f, c->norm1(), nullptr, false)) != LSAM_OK) return rc;
+      } else if ((rc = launch_norm(c, c->g(), ldg, n, vec4, 0.f, c->norm1(), nullptr)) != LSAM_OK) return rc;
     }
-    if ((rc = launch_update(c, gptr, g_mode, ldg, n, vec4, eta)) != LSAM_OK) return rc;
-    return LSAM_OK;
+    return finish_tick(gptr);
   }
   const float* g1 = flat ? c->eg1 : c->g();
   const bool g1_bf16 = gb;
   phase.next("lsam S2 ascent gradient");
   if (!flat && (rc = grad_pass(c, false, c->loss(), g1_bf16)) != LSAM_OK) return rc;
-  if (!flat && L.g1keep) {
+  if (!flat && L.g1keep && !dp) {
     if (g1_bf16) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.g1keep), c->at<bf16>(L.g1b), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
     else LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(L.g1keep), c->g(), sizeof(float) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   }
   phase.next("lsam S3-S4 norm, perturbation");
-  if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
-  if (g1_bf16 && vec4 && n % 8 == 0) {
-    dim3 pgrid((unsigned)ceil_div(n, (int64_t)kPertThreads * 8 * kPert8Iter), cfg.K);
-    LAUNCH(c, LSAM_PROF_PERTURB, perturb8_kernel<<<pgrid, kPertThreads, 0, c->stream>>>(c->x(), L.ld, c->at<bf16>(L.g1b), ldg, n, c->scale(), c->at<bf16>(L.xop), L.ld, c->act()));
-    rc = LSAM_OK;
-  } else if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
-  else if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
-  else rc = launch_perturb<float, float>(c, g1, ldg, n, vec4);
+  if (dp) {
+    // the perturbation follows the averaged gradient and its norm (every worker's row of scale[] holds the same value)
+    const void* g1src = g1_bf16 ? (const void*)c->at<bf16>(L.g1b) : (const void*)g1;
+    if ((rc = launch_mean_rows(c, g1src, g1_bf16, ldg, n, vec4, gbar1)) != LSAM_OK) return rc;
+    if ((rc = launch_norm(c, gbar1, 0, n, vec4, rho, c->norm1(), c->scale(), false)) != LSAM_OK) return rc;
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, gbar1, 0, n, vec4);
+    else rc = launch_perturb<float, float>(c, gbar1, 0, n, vec4);
+  } else {
+    if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
+    if (g1_bf16 && vec4 && n % 8 == 0) {
+      dim3 pgrid((unsigned)ceil_div(n, (int64_t)kPertThreads * 8 * kPert8Iter), cfg.K);
+      LAUNCH(c, LSAM_PROF_PERTURB, perturb8_kernel<<<pgrid, kPertThreads, 0, c->stream>>>(c->x(), L.ld, c->at<bf16>(L.g1b), ldg, n, c->scale(), c->at<bf16>(L.xop), L.ld, c->act()));
+      rc = LSAM_OK;
+    } else if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
+    else if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
+    else rc = launch_perturb<float, float>(c, g1, ldg, n, vec4);
+  }
   if (rc != LSAM_OK) return rc;
   if (L.xpkeep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.xpkeep), c->at<bf16>(L.xop), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   // descent gradient at the perturbed point, same minibatch
-  const float* g2 = flat ? c->eg2 : c->g();
   phase.next("lsam S5 descent gradient");
   if (!flat && (rc = grad_pass(c, true, nullptr, gb)) != LSAM_OK) return rc;
   phase.next("lsam S6 update");
-  if (cfg.flags & LSAM_FLAG_STEP_INFO)
-    if ((rc = launch_norm(c, g2, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
-  // fused worker update
-  if ((rc = launch_update(c, gptr, g_mode, ldg, n, vec4, eta)) != LSAM_OK) return rc;
-  return LSAM_OK;
+  return finish_tick(gptr);
 }
 
 
@@ -1013,7 +1073,7 @@ int lsam_read_anchor_gap(lsam_ctx* c, float* h_gap) {
   float* out = c->at<float>(L.scalars) + 4 * (size_t)K;
   dim3 grid((unsigned)ceil_div(n, norm_chunk<4>()), K);
   if ((int64_t)grid.x > L.nchunks) return c->fail(LSAM_ERR_WORKSPACE, "anchor gap: partial-sum buffer too small");
-  LAUNCH(c, LSAM_PROF_NORM, gap_sumsq_partial_kernel<<<grid, kNormThreads, 0, c->stream>>>(c->x(), L.ld, c->yslot(c->t_y), n, partial, L.nchunks));
+  LAUNCH(c, LSAM_PROF_NORM, gap_sumsq_partial_kernel<<<grid, kNormThreads, 0, c->stream>>>(c->x(), L.ld, c->yslot(c->t_y), n, partial, L.nchunks, nullptr, nullptr));
   FinArgs f{partial, L.nchunks, (int64_t)grid.x, 0.f, c->cfg.gamma, out, nullptr, c->status(), nullptr, {}};
   f.bind();
   LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(K), dim3(256), f.ptrs, 0, c->stream));
@@ -1041,6 +1101,9 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
       } else {
         rc = seg_copy<false>(c, c->at<float>(L.xop) + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
       }
+    } else if (c->cfg.dp_average) {
+      // data-parallel mode: every worker used the gradient averaged over the workers
+      rc = seg_copy<false>(c, c->at<float>(pass == 1 ? L.gbar1 : L.gbar2), L.ld, tmp, L.d, 1);
     } else if (flat) {
       const float* src = pass == 1 ? c->eg1 : c->eg2;
       if (!src) return c->fail(LSAM_ERR_STATE, "no external gradients set");

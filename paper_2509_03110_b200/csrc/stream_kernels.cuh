@@ -86,13 +86,17 @@ sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float*
 
 // Anchor gap (Lemma 5): partial sums of squares of x_k - y over fixed chunks of norm_chunk<4>() elements, same order as
 // above; the rows are 16-byte aligned, the tail of a row whose length is not a multiple of 4 is masked.  grid (chunks, K).
+// slot (nullable) [K]: replica k is measured against row slot[k] of y (the centre version it reads, row stride ldx) instead of row 0.
 __global__ void __launch_bounds__(kNormThreads)
 gap_sumsq_partial_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ y, int64_t n,
-                         float* __restrict__ partial, int64_t nchunks) {
+                         float* __restrict__ partial, int64_t nchunks, const int32_t* __restrict__ slot,
+                         const int32_t* __restrict__ active) {
   __shared__ float red[kNormThreads / 32];
   const int k = blockIdx.y;
+  if (active != nullptr && !active[k]) return;
   const int64_t base = (int64_t)blockIdx.x * norm_chunk<4>();
   const float* row = x + (int64_t)k * ldx;
+  if (slot != nullptr) y += (int64_t)slot[k] * ldx;
   float s = 0.f;
 #pragma unroll
   for (int i = 0; i < kNormIter; ++i) {
@@ -130,6 +134,61 @@ norm_finalize_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t
         atomicOr(status, STATUS_NONFINITE);
       }
     }
+  }
+}
+
+// Pull weight of a stationary kernel phi(x - y) (Corollary 8 and the remark after it): the worker's pull is
+// grad phi(x - y) = w(r) (x - y) with r = ||x_k - y||.  partial holds the sums of squares of x_k - y per chunk (as above);
+// weight[k] = w(r_k).  kind: 0 Gaussian w = lambda; 1 exponential-power phi = (lambda / a) r^a, w = lambda r^(a-2), w(0) = 0 for
+// a < 2; 2 Cauchy phi = (lambda s^2 / 2) log(1 + r^2 / s^2), w = lambda / (1 + r^2 / s^2); 3 Matern-3/2, w = lambda / (1 + sqrt(lambda) r).
+// grid K, block 256.
+enum : int { KERNEL_GAUSSIAN = 0, KERNEL_EXP_POWER = 1, KERNEL_CAUCHY = 2, KERNEL_MATERN32 = 3 };
+__global__ void __launch_bounds__(256)
+pull_weight_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t nused, int kind, float lambda, float param,
+                   float* __restrict__ weight, const int32_t* __restrict__ active) {
+  __shared__ double red[8];
+  const int k = blockIdx.x;
+  if (active != nullptr && !active[k]) return;
+  double s = 0.0;
+  for (int64_t c = threadIdx.x; c < nused; c += blockDim.x) s += (double)partial[(int64_t)k * nchunks + c];
+  const double tot = block_sum<double>(s, red);
+  if (threadIdx.x == 0) {
+    const float r = (float)sqrt(tot);
+    float w = lambda;
+    if (kind == KERNEL_EXP_POWER) w = (param == 2.f) ? lambda : (r > 0.f ? lambda * powf(r, param - 2.f) : 0.f);
+    else if (kind == KERNEL_CAUCHY) w = lambda / (1.f + (r / param) * (r / param));
+    else if (kind == KERNEL_MATERN32) w = lambda / (1.f + sqrtf(lambda) * r);
+    weight[k] = w;
+  }
+}
+
+// Synchronous data parallelism (the DP-SGD / DP-SAM baselines aggregate the workers' gradients at every iteration):
+// out[j] = (1/K) sum_k g[k][j], k ascending, one thread per 4 consecutive columns (or per column when VEC == 1).
+// TG = float or bf16 (gradient storage of the tensor-core path).  out may alias row 0 of an fp32 g.
+template <int VEC, typename TG>
+__global__ void __launch_bounds__(256)
+mean_rows_kernel(const TG* g, int64_t ldg, int K, int64_t n, float* out) {
+  const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * VEC;
+  if (j >= n) return;
+  const float inv = 1.0f / (float)K;
+  if (VEC == 4) {
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int k = 0; k < K; ++k) {
+      if (sizeof(TG) == 4) {
+        const float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g) + (int64_t)k * ldg + j);
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      } else {
+        const uint2 raw = *reinterpret_cast<const uint2*>(reinterpret_cast<const bf16*>(g) + (int64_t)k * ldg + j);
+        const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.x));
+        const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&raw.y));
+        s.x += lo.x; s.y += lo.y; s.z += hi.x; s.w += hi.y;
+      }
+    }
+    *reinterpret_cast<float4*>(out + j) = make_float4(s.x * inv, s.y * inv, s.z * inv, s.w * inv);
+  } else {
+    float s = 0.f;
+    for (int k = 0; k < K; ++k) s += to_float(g[(int64_t)k * ldg + j]);
+    out[j] = s * inv;
   }
 }
 
@@ -262,6 +321,7 @@ struct UpdateArgs {
   int K;
   int k_offset;        // global index of worker 0: the noise streams are keyed by the global worker index
   float eta, mu, lambda;
+  const float* lam_k;  // nullable [K]: per-worker pull weight w(||x_k - y||) of a non-Gaussian stationary kernel, used instead of lambda
   // Langevin noise (NOISE variants): x_new += sigma * xi, xi from langevin_noise4(seed, tick, k, segment, offset / 4)
   float sigma;
   uint64_t seed, tick;
@@ -325,8 +385,9 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
         yn = __ldg(reinterpret_cast<const float4*>(a.yring + (int64_t)a.slot[kn] * a.ld + j));
       }
       float G;
+      const float lam = a.lam_k != nullptr ? a.lam_k[k] : a.lambda;
 #define LSAM_UPD(c)                                                         \
-  G = fmaf(a.lambda, xv.c - yv.c, gv.c);                                    \
+  G = fmaf(lam, xv.c - yv.c, gv.c);                                         \
   vv.c = fmaf(a.mu, vv.c, G);                                               \
   xv.c = NESTEROV ? xv.c - a.eta * fmaf(a.mu, vv.c, G) : xv.c - a.eta * vv.c;
       LSAM_UPD(x) LSAM_UPD(y) LSAM_UPD(z) LSAM_UPD(w)
@@ -365,7 +426,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       const float gv = update_load_g1(a.g, (int64_t)k * a.ldg + j, a.g_mode);
       float xv = a.x[o], vv = a.v[o];
       const float yv = a.yring[(int64_t)a.slot[k] * a.ld + j];
-      const float G = fmaf(a.lambda, xv - yv, gv);
+      const float G = fmaf(a.lam_k != nullptr ? a.lam_k[k] : a.lambda, xv - yv, gv);
       vv = fmaf(a.mu, vv, G);
       xv = NESTEROV ? xv - a.eta * fmaf(a.mu, vv, G) : xv - a.eta * vv;
       if (NOISE && noff < nlen) {
@@ -436,6 +497,7 @@ __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a
     }
     const uint32_t gw[4] = {gr.x, gr.y, gr.z, gr.w};
     uint32_t ow[4];
+    const float lam = a.lam_k != nullptr ? a.lam_k[k] : a.lambda;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       const float2 ga = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gw[2 * h]));
@@ -443,7 +505,7 @@ __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a
       const float4 gv = make_float4(ga.x, ga.y, gc.x, gc.y);
       float G;
 #define LSAM_UPD(c)                                                               \
-  G = fmaf(a.lambda, xv[h].c - yv[h].c, gv.c);                                    \
+  G = fmaf(lam, xv[h].c - yv[h].c, gv.c);                                         \
   vv[h].c = fmaf(a.mu, vv[h].c, G);                                               \
   xv[h].c = NESTEROV ? xv[h].c - a.eta * fmaf(a.mu, vv[h].c, G) : xv[h].c - a.eta * vv[h].c;
       LSAM_UPD(x) LSAM_UPD(y) LSAM_UPD(z) LSAM_UPD(w)
@@ -528,11 +590,12 @@ __global__ void __launch_bounds__(kUpdThreads) update8f_kernel(const UpdateArgs 
         yn[h] = __ldg(reinterpret_cast<const float4*>(yp + 4 * h));
       }
     }
+    const float lam = a.lam_k != nullptr ? a.lam_k[k] : a.lambda;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
       float G;
 #define LSAM_UPD(c)                                                               \
-  G = fmaf(a.lambda, xv[h].c - yv[h].c, gv[h].c);                                 \
+  G = fmaf(lam, xv[h].c - yv[h].c, gv[h].c);                                      \
   vv[h].c = fmaf(a.mu, vv[h].c, G);                                               \
   xv[h].c = NESTEROV ? xv[h].c - a.eta * fmaf(a.mu, vv[h].c, G) : xv[h].c - a.eta * vv[h].c;
       LSAM_UPD(x) LSAM_UPD(y) LSAM_UPD(z) LSAM_UPD(w)

@@ -27,9 +27,22 @@ def test_library_exports_every_declared_symbol():
     assert sorted(G.EXPORTS) == names
 
 
-def test_config_struct_matches_header_size():
-    # 20 int32 + 2 int64 + 1 uint64 + 5 float + int32 + float + 2 int32 = 80 + 24 + 28 + 8 = 140, rounded up to the 8-byte alignment
-    assert C.sizeof(G.LsamConfig) == 144
+def test_config_struct_matches_header_size(tmp_path):
+    # the ctypes mirror of lsam_config against the header itself, as the C compiler lays it out: size and field offsets
+    import subprocess
+
+    fields = [f[0] for f in G.LsamConfig._fields_]
+    cname = {"lam": "lambda"}
+    src = tmp_path / "layout.c"
+    lines = ['#include <stdio.h>', '#include <stddef.h>', '#include "lsam.h"', 'int main(void) {', '  printf("%zu\\n", sizeof(lsam_config));']
+    lines += [f'  printf("%zu\\n", offsetof(lsam_config, {cname.get(f, f)}));' for f in fields]
+    lines += ['  return 0;', '}']
+    src.write_text("\n".join(lines))
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    out = [int(v) for v in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    assert C.sizeof(G.LsamConfig) == out[0]
+    assert [getattr(G.LsamConfig, f).offset for f in fields] == out[1:]
 
 
 def test_param_counts_and_workspace_of_the_five_configs():
