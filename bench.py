@@ -209,12 +209,12 @@ def make_inputs(w, dev, seed=0):
     return dict(X=X, Y=Y, x0=x0, y0=w0)
 
 
-def make_cfg(G, w, flags=0, K_total=0, k_offset=0):
+def make_cfg(G, w, flags=0, K_total=0, k_offset=0, gemm_impl=0):
     lam = w.get("lambda0", LAMBDA0) / (w["eta"] * w["tau"])
     return G.make_config(w["model"], widths=w["widths"], K=w["K"], batch=max(w["B"], 1) if w["model"] != FLAT else 0,
                          gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
                          beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
-                         flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256),
+                         flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256), gemm_impl=gemm_impl,
                          noise_temp=w.get("noise_temp", 0.0), K_total=K_total, k_offset=k_offset)
 
 
@@ -308,7 +308,7 @@ def workload_config(w):
 
 
 # ---------------------------------------------------------------------------------------------- one workload on this rank's GPU
-def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True):
+def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True, gemm_impl=0):
     """Create the context, time `steps` steps after `warmup` untimed ones, and return the record of this workload
     (rank 0; None on the other ranks).  A step is one pass of the whole hot path plus the centre update when it is due."""
     import torch
@@ -328,7 +328,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
     short_kernels = 4.0 * w["K"] * param_count(w) <= 1.2e9
     use_graph = (small or short_kernels) if cuda_graph == "auto" else cuda_graph == "on"
     flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0)
-    cfg = make_cfg(G, w, flags=flags, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0)
+    cfg = make_cfg(G, w, flags=flags, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0, gemm_impl=gemm_impl)
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream(device=dev)
     torch.cuda.set_stream(work_stream)
@@ -526,7 +526,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
         cpu, _ = oracle_baseline(w, key, X, Y, inp["y0"].cpu().numpy())
 
     cfgd = workload_config(w)
-    cfgd.update(gemm="tcgen05" if uses_tc else "simt", cuda_graph=bool(use_graph),
+    cfgd.update(gemm=("tcgen05 (single-CTA kernels only)" if gemm_impl == G.IMPL_TCGEN05_1CTA else "tcgen05") if uses_tc else "simt", cuda_graph=bool(use_graph),
                 l2=("working set larger than L2" if not small else "L2-resident state (latency-bound workload)") +
                    ("" if events_in_timed else "; kernel shares and roofline from a separate pass over the same steps with per-launch events"),
                 parallelism=(f"{world * w['K']} workers sharded over {world} GPU(s), one centre, accumulator all-reduce every tau steps" if shard
@@ -561,6 +561,8 @@ def main():
     ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
     ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
     ap.add_argument("--grad-fp32", action="store_true", help="tensor-core path: store the gradients in fp32 instead of bf16")
+    ap.add_argument("--gemm-impl", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05-1cta", "tcgen05-pairs"],
+                    help="auto: tensor-core GEMMs for the bf16 workloads (CTA pairs where a GEMM is large enough); tcgen05-1cta: single-CTA kernels only")
     ap.add_argument("--shard-workers", action="store_true",
                     help="N > 1: one job of N*K workers with a single centre, K workers per GPU, accumulator all-reduce every tau steps "
                          "(default: N independent copies of the workload)")
@@ -607,8 +609,10 @@ def main():
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
     rec = run_workload(args.workload, w, args.steps, args.warmup, dev, rank, world, shard=shard, cuda_graph=args.cuda_graph,
-                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline)
+                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline,
+                       gemm_impl={"auto": 0, "simt": 1, "tcgen05": 2, "tcgen05-1cta": 3, "tcgen05-pairs": 4}[args.gemm_impl])
     others = []
+    modified = modified or args.gemm_impl != "auto" or args.grad_fp32
     want_others = args.others == "on" or (args.others == "auto" and world == 1 and args.workload == "c4" and not modified and not shard)
     if want_others and world == 1:
         for key, over, nsteps in OTHER_WORKLOADS:

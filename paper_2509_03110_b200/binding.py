@@ -14,7 +14,7 @@ _LIB_PATH = os.path.join(_HERE, "liblsam_b200.so")
 LSAM_OK, LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE, LSAM_ERR_STATE, LSAM_ERR_CUDA, LSAM_ERR_NONFINITE, LSAM_ERR_TIMEOUT = range(7)
 MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT = 0, 1, 2, 3
 GEMM_FP32, GEMM_BF16 = 0, 1
-IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05 = 0, 1, 2
+IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05, IMPL_TCGEN05_1CTA, IMPL_TCGEN05_PAIRS = 0, 1, 2, 3, 4
 KERNEL_GAUSSIAN, KERNEL_EXP_POWER, KERNEL_CAUCHY, KERNEL_MATERN32 = 0, 1, 2, 3
 FLAG_KEEP_G1, FLAG_STEP_INFO, FLAG_CUDA_GRAPH, FLAG_GRAD_FP32 = 1, 2, 4, 8
 PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "loss", "bias_grad", "lsq_grad", "norm",

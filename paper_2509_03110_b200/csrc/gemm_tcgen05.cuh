@@ -13,8 +13,16 @@
 // row a thread drains from tensor memory is then one feature x 32 consecutive samples, i.e. contiguous 16-byte
 // vectors in every buffer the epilogue touches.
 //
+// PAIR form (cta_group::2): two CTAs of a cluster share one 256-row M tile.  Each CTA stages its own 128 rows of A and
+// HALF of the N side of B; one thread of the leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2 with M = 256,
+// which reads the two halves of B from both CTAs' shared memory and leaves rows 0-127 of the tile in the leader's tensor
+// memory and rows 128-255 in the peer's.  A CTA so takes in a third fewer operand bytes per flop (the bound of the
+// single-CTA form is the rate at which an SM can fill its shared memory).  Each CTA issues its own TMA loads (no load is
+// multicast); the loads of both CTAs complete on the leader's `full` barrier, the leader's tcgen05.commit arrives on the
+// `empty` / `acc_full` barriers of both CTAs, and both CTAs' epilogue warps arrive on the leader's `acc_empty` barrier.
+//
 // All waits on mbarriers are bounded: when one expires the CTA raises STATUS_TIMEOUT, stops issuing work, lets the
-// copies in flight land, frees its tensor memory and returns.
+// copies in flight land, frees its tensor memory and returns (the peer of a pair then runs into its own bounds).
 #pragma once
 
 #include <cuda.h>
@@ -80,6 +88,34 @@ __device__ inline void tma_load_3d(void* dst, const CUtensorMap* map, int c0, in
       : "memory");
 }
 
+// The same load issued by a CTA of a pair: data into this CTA's shared memory, completion counted on a barrier given by its
+// shared::cluster address (the leader's `full` barrier, possibly in the peer CTA).  Not a multicast: one CTA, one destination.
+__device__ inline void tma_load_3d_pair(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster_addr)
+      : "memory");
+}
+__device__ inline uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// shared::cluster address of the location `local` (a shared::cta address of this CTA) in the CTA of rank `rank`
+__device__ inline uint32_t map_to_cta(uint32_t local, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+  return r;
+}
+__device__ inline void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// all threads of both CTAs of the cluster
+__device__ inline void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // 3-D tiled TMA store from this CTA's shared memory (bulk async group); rows / columns outside the tensor are clipped.
 __device__ inline void tma_store_3d(const CUtensorMap* map, const void* src, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
@@ -98,6 +134,14 @@ __device__ inline void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
 __device__ inline void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
   asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
 }
+// pair form: the same warp of BOTH CTAs executes these; the columns are allocated in both CTAs' tensor memory
+__device__ inline void tmem_alloc_pair(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ inline void tmem_dealloc_pair(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
 // D[tmem] (+)= A[smem desc] * B[smem desc], bf16 inputs, fp32 accumulate.
 __device__ inline void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
@@ -111,6 +155,22 @@ __device__ inline void umma_bf16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc
 // mbarrier arrives when all tcgen05.mma issued so far by this thread have completed.
 __device__ inline void umma_commit(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// pair form: M = 256 over the two CTAs (D rows 0-127 in the leader's tensor memory, 128-255 in the peer's; each CTA's shared
+// memory holds its 128 rows of A and half of the N side of B at the same offsets).  Issued by one thread of the leader.
+__device__ inline void umma_bf16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// the barrier at this offset in BOTH CTAs of the pair arrives when the pair's MMAs issued so far have completed
+__device__ inline void umma_commit_pair(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
 }
 // 32 lanes x 32 consecutive fp32 columns of tensor memory -> 32 registers per thread (thread = lane).
 __device__ inline void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
@@ -178,30 +238,36 @@ constexpr int kTcBlockK = 64;
 constexpr int kTcThreads = 320;
 constexpr int kTcEpiWarps = 8;
 
-template <int BLOCK_N>
-__host__ __device__ constexpr int tc_stages() { return BLOCK_N == 256 ? 4 : (BLOCK_N == 128 ? 6 : 8); }
-template <int BLOCK_N>
-__host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + BLOCK_N) * kTcBlockK * 2; }
+// PAIR: a CTA stages only BLOCK_N / 2 rows of B per k-block, so the ring is deeper
+template <int BLOCK_N, bool PAIR = false>
+__host__ __device__ constexpr int tc_stages() { return PAIR ? (BLOCK_N == 256 ? 6 : 8) : (BLOCK_N == 256 ? 4 : (BLOCK_N == 128 ? 6 : 8)); }
+template <int BLOCK_N, bool PAIR = false>
+__host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + (PAIR ? BLOCK_N / 2 : BLOCK_N)) * kTcBlockK * 2; }
 constexpr int kTcStageOutBytes = 8 * 4096;  // wgrad epilogue staging: one 32-row x 128-byte block (128B-swizzled) per epilogue warp
-template <int BLOCK_N>
+template <int BLOCK_N, bool PAIR = false>
 __host__ __device__ constexpr int tc_smem_bytes() {
-  return tc_stages<BLOCK_N>() * tc_stage_bytes<BLOCK_N>() + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTcStageOutBytes;
+  return tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>() + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTcStageOutBytes;
 }
 
 // ------------------------------------------------------------------------------------------------ the kernel
 // M, N, Kd: problem extents; Z replicas.  Operands are addressed through 3-D tensor maps (dim 2 = replica):
 //   contraction-contiguous operand: map dims {Kd, rows, Z}, box {64, tile rows, 1}
 //   M/N-contiguous operand:         map dims {rows, Kd, Z}, box {64, 64, 1} (one box per 64 rows of the tile)
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
+//   PAIR: the B box has BLOCK_N / 2 rows (contraction-contiguous) resp. the CTA loads BLOCK_N / 128 boxes (N-contiguous);
+//   the grid is a multiple of 2 and is launched with cluster dimension 2.
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
                     int Z, TcEpi ep, int* __restrict__ status, const int32_t* __restrict__ active) {
-  constexpr int STAGES = tc_stages<BLOCK_N>();
+  static_assert(!PAIR || BLOCK_N >= 128, "the pair form needs 64 rows of B per CTA");
+  constexpr int STAGES = tc_stages<BLOCK_N, PAIR>();
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
-  constexpr int B_BYTES = BLOCK_N * kTcBlockK * 2;
+  constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;  // rows of the N side staged by this CTA
+  constexpr int B_BYTES = B_ROWS * kTcBlockK * 2;
+  constexpr int TILE_M = PAIR ? 2 * kTcBlockM : kTcBlockM;  // rows of a tile of the work list
   constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;  // two accumulator stages (power of two >= 32)
-  constexpr uint32_t IDESC = tc::instr_desc(kTcBlockM, BLOCK_N, A_MN, B_MN);
+  constexpr uint32_t IDESC = tc::instr_desc(TILE_M, BLOCK_N, A_MN, B_MN);
 
   extern __shared__ uint8_t smem_raw[];
   // round the tile area up to 1024 bytes by pointer arithmetic on the shared array itself (keeps the address space known)
@@ -217,52 +283,93 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m_tiles = (M + kTcBlockM - 1) / kTcBlockM;
+  const int m_tiles = (M + TILE_M - 1) / TILE_M;
   const int n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_blocks = (Kd + kTcBlockK - 1) / kTcBlockK;
   const int64_t total = (int64_t)Z * m_tiles * n_tiles;
+  // a pair walks the work list together: unit = index of this CTA (or of its pair), units = how many walk the list
+  const uint32_t rank = PAIR ? tc::cluster_ctarank() : 0u;
+  const bool leader = rank == 0u;
+  const int64_t unit = PAIR ? blockIdx.x / 2 : blockIdx.x, units = PAIR ? gridDim.x / 2 : gridDim.x;
+  const int m_off = (int)rank * kTcBlockM;   // this CTA's rows inside a tile
+  const int n_off = (int)rank * B_ROWS;      // this CTA's share of the N side of B
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
-    for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], kTcEpiWarps); }
+    for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], PAIR ? 2 * kTcEpiWarps : kTcEpiWarps); }
     for (int s = 0; s < 8; ++s) tc::mbar_init(&bias_bar[s], 2);
     static_assert((2 * STAGES + 4 + 8) * 8 + 8 <= 256, "barrier area");
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
-  if (warp == 1) tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  if (warp == 1) {
+    if (PAIR) tc::tmem_alloc_pair(tmem_slot, TMEM_COLS);
+    else tc::tmem_alloc(tmem_slot, TMEM_COLS);
+  }
   tc::tc_fence_before();
   __syncthreads();
+  if (PAIR) tc::cluster_sync_all();  // the peer's barriers exist before anything arrives on them
   tc::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  if (PAIR) {
+    // one MMA addresses the accumulator columns of both CTAs with the same number, so the two allocations must agree
+    // (they do on SMs whose tensor memory was free); otherwise no role starts and the launch reports it
+    uint32_t peer_base;
+    asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(peer_base) : "r"(tc::map_to_cta(tc::smem_u32(tmem_slot), rank ^ 1u)) : "memory");
+    if (peer_base != tmem_base) {
+      if (threadIdx.x == 0) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
+      __syncthreads();
+    }
+  }
+  const bool run = !PAIR || (*abort_flag == 0);
 
-  if (warp == 0) {
+  if (!run) {
+    // nothing to do: fall through to the teardown
+  } else if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      for (int64_t t = unit; t < total && ok; t += units) {
         const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
         if (active != nullptr && !active[z]) continue;  // waiting replica: all three roles skip the same tiles
-        const int m0 = mt * kTcBlockM, n0 = nt * BLOCK_N;
+        const int m0 = mt * TILE_M + m_off, n0 = nt * BLOCK_N + n_off;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* a_dst = tiles + s * (A_BYTES + B_BYTES);
           uint8_t* b_dst = a_dst + A_BYTES;
-          tc::mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
           const int k0 = kb * kTcBlockK;
-          if (A_MN) {
+          if (PAIR) {
+            // both CTAs' loads of this stage complete on the leader's barrier, which the leader arms with the bytes of both
+            if (leader) tc::mbar_expect_tx(&full[s], 2 * (A_BYTES + B_BYTES));
+            const uint32_t bar = tc::map_to_cta(tc::smem_u32(&full[s]), 0u);
+            if (A_MN) {
 #pragma unroll
-            for (int i = 0; i < kTcBlockM / 64; ++i) tc::tma_load_3d(a_dst + i * 8192, &map_a, m0 + 64 * i, k0, z, &full[s]);
-          } else {
-            tc::tma_load_3d(a_dst, &map_a, k0, m0, z, &full[s]);
-          }
-          if (B_MN) {
+              for (int i = 0; i < kTcBlockM / 64; ++i) tc::tma_load_3d_pair(a_dst + i * 8192, &map_a, m0 + 64 * i, k0, z, bar);
+            } else {
+              tc::tma_load_3d_pair(a_dst, &map_a, k0, m0, z, bar);
+            }
+            if (B_MN) {
 #pragma unroll
-            for (int i = 0; i < BLOCK_N / 64; ++i) tc::tma_load_3d(b_dst + i * 8192, &map_b, n0 + 64 * i, k0, z, &full[s]);
+              for (int i = 0; i < B_ROWS / 64; ++i) tc::tma_load_3d_pair(b_dst + i * 8192, &map_b, n0 + 64 * i, k0, z, bar);
+            } else {
+              tc::tma_load_3d_pair(b_dst, &map_b, k0, n0, z, bar);
+            }
           } else {
-            tc::tma_load_3d(b_dst, &map_b, k0, n0, z, &full[s]);
+            tc::mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
+            if (A_MN) {
+#pragma unroll
+              for (int i = 0; i < kTcBlockM / 64; ++i) tc::tma_load_3d(a_dst + i * 8192, &map_a, m0 + 64 * i, k0, z, &full[s]);
+            } else {
+              tc::tma_load_3d(a_dst, &map_a, k0, m0, z, &full[s]);
+            }
+            if (B_MN) {
+#pragma unroll
+              for (int i = 0; i < BLOCK_N / 64; ++i) tc::tma_load_3d(b_dst + i * 8192, &map_b, n0 + 64 * i, k0, z, &full[s]);
+            } else {
+              tc::tma_load_3d(b_dst, &map_b, k0, n0, z, &full[s]);
+            }
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
@@ -271,13 +378,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    if (lane == 0 && leader) {  // pair form: the leader issues for both CTAs
       int s = 0;
       uint32_t ph = 0;
       int as = 0;
       uint32_t aph = 0;
       bool ok = true;
-      for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+      for (int64_t t = unit; t < total && ok; t += units) {
         if (active != nullptr && !active[(int)(t / ((int64_t)n_tiles * m_tiles))]) continue;
         if (!tc::mbar_wait(&acc_empty[as], aph ^ 1u, abort_flag)) { ok = false; break; }
         tc::tc_fence_after();
@@ -294,13 +401,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
             // a K = 16 slice is two such groups = 2048 B further.
             const uint64_t ad = A_MN ? tc::smem_desc(a_addr + k * 2048, 8192, 1024) : tc::smem_desc(a_addr + k * 32, 16, 1024);
             const uint64_t bd = B_MN ? tc::smem_desc(b_addr + k * 2048, 8192, 1024) : tc::smem_desc(b_addr + k * 32, 16, 1024);
-            tc::umma_bf16(d_tmem, ad, bd, IDESC, (kb | k) != 0 ? 1u : 0u);
+            if (PAIR) tc::umma_bf16_pair(d_tmem, ad, bd, IDESC, (kb | k) != 0 ? 1u : 0u);
+            else tc::umma_bf16(d_tmem, ad, bd, IDESC, (kb | k) != 0 ? 1u : 0u);
           }
-          tc::umma_commit(&empty[s]);  // frees the stage when these MMAs have read it
+          // frees the stage (in both CTAs of a pair) when these MMAs have read it
+          if (PAIR) tc::umma_commit_pair(&empty[s]);
+          else tc::umma_commit(&empty[s]);
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
-        tc::umma_commit(&acc_full[as]);
+        if (PAIR) tc::umma_commit_pair(&acc_full[as]);
+        else tc::umma_commit(&acc_full[as]);
         if (++as == 2) { as = 0; aph ^= 1u; }
       }
       if (!ok) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
@@ -314,10 +425,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     int as = 0;
     uint32_t aph = 0;
     bool ok = true;
-    for (int64_t t = blockIdx.x; t < total && ok; t += gridDim.x) {
+    const uint32_t acc_empty_leader[2] = {PAIR ? tc::map_to_cta(tc::smem_u32(&acc_empty[0]), 0u) : 0u, PAIR ? tc::map_to_cta(tc::smem_u32(&acc_empty[1]), 0u) : 0u};
+    for (int64_t t = unit; t < total && ok; t += units) {
       const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
       if (active != nullptr && !active[z]) continue;
-      const int m = mt * kTcBlockM + quad * 32 + lane;
+      const int m_base = mt * TILE_M + m_off;  // first row of the 128 rows this CTA drains
+      const int m = m_base + quad * 32 + lane;
       const int n0 = nt * BLOCK_N;
       if (!tc::mbar_wait(&acc_full[as], aph, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
@@ -338,7 +451,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           // map (row = lane, 16-byte chunk q stored at position q ^ (row % 8)), then one TMA store writes it to the
           // gradient rows (clipped at the ragged edges).  Two buffers per warp: the store of a chunk overlaps the
           // staging of the next one.
-          const int mrow0 = mt * kTcBlockM + quad * 32;
+          const int mrow0 = m_base + quad * 32;
           if (mrow0 < M && nb < N) {  // warp-uniform: blocks wholly outside the matrix are neither staged nor stored
 #pragma unroll
             for (int j = 0; j < 32; ++j) ssq = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ssq);  // zero-filled edges add 0
@@ -484,9 +597,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
       }
       if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && ep.partial != nullptr) {
-        // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows
+        // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows; the slots are
+        // laid out by 128-row block of the output (a CTA of a pair whose rows lie wholly outside the matrix has none)
         const float tot = warp_sum(ssq);
-        if (lane == 0) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)mt * n_tiles + nt) * kTcEpiWarps + ew] = tot;
+        if (lane == 0 && m_base < M) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)(m_base / kTcBlockM) * n_tiles + nt) * kTcEpiWarps + ew] = tot;
       }
       if (EPI == TC_EPI_DGRAD && ep.bias_g != nullptr) {
         // the two warps of a quadrant hold the sums over their halves of the samples: exchange through shared memory (the
@@ -513,7 +627,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       }
       tc::tc_fence_before();
       __syncwarp();
-      if (lane == 0) tc::mbar_arrive(&acc_empty[as]);
+      if (lane == 0) {
+        if (PAIR) tc::mbar_arrive_cluster(acc_empty_leader[as]);  // the issuing thread lives in the leader CTA
+        else tc::mbar_arrive(&acc_empty[as]);
+      }
       if (++as == 2) { as = 0; aph ^= 1u; }
     }
     if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && lane == 0) tc::bulk_wait_all<0>();  // every gradient block has reached global memory
@@ -529,9 +646,13 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     while (clock64() - t0 < 2000000LL) { }
     __syncthreads();
   }
+  // pair form: neither CTA may leave (or free its tensor memory) while the other can still read its shared memory, write
+  // its barriers or has MMAs in flight that fill its tensor memory; every role of both CTAs has ended here (all waits are bounded)
+  if (PAIR) tc::cluster_sync_all();
   if (warp == 1) {
     tc::tc_fence_after();
-    tc::tmem_dealloc(tmem_base, TMEM_COLS);
+    if (PAIR) tc::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    else tc::tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
 
@@ -564,6 +685,7 @@ struct TcGemm {
   int M = 0, N = 0, Kd = 0, block_n = 0;
   TcEpi ep{};
   bool valid = false;
+  bool pair = false;  // run by pairs of CTAs (cta_group::2) on 256-row tiles
 };
 
 struct TcPlan {
@@ -574,6 +696,9 @@ struct TcPlan {
   std::vector<TcGemm> fwd, dgrad, wgrad;
   std::vector<int> bias_slot0;  // first partial slot of the bias-gradient blocks of each layer
   int n_slots = 0;              // partial slots used per replica
+  bool allow_pair = true;       // false: every GEMM on the single-CTA kernels
+  bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
+  int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
 };
 
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -608,6 +733,11 @@ inline bool tc_make_map(CUtensorMap* m, const T* base, uint64_t cols, uint64_t r
 }
 
 inline int tc_pick_block_n(int n) { return n > 128 ? 256 : (n > 64 ? 128 : 64); }
+// Where the pair form is used: forward and dgrad with a 256-wide minibatch tile (measured at the 4096-wide layers with
+// B = 256: 985 -> 1100 and 945 -> 1030 TFLOP/s inside the step).  It loses with 128-wide minibatch tiles (short kernels: 415 -> 405,
+// 360 -> 335) and in the weight gradient (770 -> 650: with four k-blocks per tile the epilogue is the kernel, and in a pair
+// the slower of the two epilogues gates both CTAs), so those keep the single-CTA kernels; `force` (tests) pairs whatever can be.
+inline bool tc_pick_pair(int M, int block_n, bool wgrad, bool force) { return M >= 256 && (force ? block_n >= 128 : (block_n == 256 && !wgrad)); }
 // Partial-sum slots one replica needs when the sum of squares is fused into the weight-gradient epilogue:
 // eight per output tile (one per epilogue warp) plus one per 8 bias units.
 inline int64_t tc_norm_slots(const lsam_config& c) {
@@ -648,6 +778,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     {  // forward: A = W [out][in] (in contiguous), B = act_l [in][B] (samples contiguous)
       TcGemm& g = P.fwd[l];
       g.M = ly.out; g.N = B; g.Kd = ly.in; g.block_n = tc_pick_block_n(B);
+      g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, false, P.force_pair);
       ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, 64);
       g.ep.bias = b.xop + ly.b_pad; g.ep.ld_p = b.ld; g.ep.ldb = b.ldb;
@@ -659,8 +790,9 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     {  // wgrad: A = dz_l [out][B] (samples contiguous = contraction), B = act_l [in][B]
       TcGemm& g = P.wgrad[l];
       g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in);
+      g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, true, P.force_pair);
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
-      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.block_n);
+      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
       // the same rows of the bf16 ascent-gradient buffer
       ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
@@ -674,6 +806,7 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     if (l > 0) {  // dgrad: A = W [out][in] read as (m = in contiguous, kd = out), B = dz_l [out][B] (samples contiguous)
       TcGemm& g = P.dgrad[l];
       g.M = ly.in; g.N = B; g.Kd = ly.out; g.block_n = tc_pick_block_n(B);
+      g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, false, P.force_pair);
       ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, 64);
       ok &= tc_make_map(&g.map_b, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, 64);
       g.ep.dh_next = ly.residual ? b.dh[(l + 1) & 1] : nullptr;
@@ -690,38 +823,67 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   return 0;
 }
 
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI>
-inline int tc_launch_one(const TcPlan& P, const TcGemm& g, cudaStream_t stream) {
-  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI>;
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR>
+inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
+  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR>;
+  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR>();
   // the shared-memory limit of a kernel is a per-device attribute: remember it per device ordinal
   static bool attr_set[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 1;
   if (!attr_set[dev]) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc_smem_bytes<BLOCK_N>()) != cudaSuccess) return 1;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return 1;
     attr_set[dev] = true;
   }
-  const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, kTcBlockM) * ceil_div(g.N, BLOCK_N);
-  const int grid = (int)(tiles < P.sms ? tiles : P.sms);
-  kern<<<grid, kTcThreads, tc_smem_bytes<BLOCK_N>(), stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status, P.active);
-  return cudaPeekAtLastError() == cudaSuccess ? 0 : 1;
+  const int tile_m = PAIR ? 2 * kTcBlockM : kTcBlockM;
+  const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, tile_m) * ceil_div(g.N, BLOCK_N);
+  if (!PAIR) {
+    const int grid = (int)(tiles < P.sms ? tiles : P.sms);
+    kern<<<grid, kTcThreads, smem, stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status, P.active);
+    return cudaPeekAtLastError() == cudaSuccess ? 0 : 1;
+  }
+  // one persistent pair of CTAs (a cluster of two) per pair of SMs
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+  cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+  if (P.max_pairs == 0) {
+    cfg.gridDim = dim3((unsigned)(P.sms / 2 * 2));
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) return 1;
+    P.max_pairs = n < P.sms / 2 ? n : P.sms / 2;
+  }
+  const int pairs = (int)(tiles < P.max_pairs ? tiles : P.max_pairs);
+  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  int M = g.M, N = g.N, Kd = g.Kd, Z = P.Z;
+  int* status = P.status;
+  const int32_t* active = P.active;
+  void* args[] = {(void*)&g.map_a, (void*)&g.map_b, (void*)&g.map_c, &M, &N, &Kd, &Z, (void*)&g.ep, &status, &active};
+  return cudaLaunchKernelExC(&cfg, (const void*)kern, args) == cudaSuccess ? 0 : 1;
 }
 
 template <bool A_MN, bool B_MN, int EPI>
-inline int tc_launch(const TcPlan& P, const TcGemm& g, cudaStream_t stream) {
+inline int tc_launch(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
   if (!g.valid) return 1;
+  if (g.pair) {
+    switch (g.block_n) {
+      case 256: return tc_launch_one<256, A_MN, B_MN, EPI, true>(P, g, stream);
+      default: return tc_launch_one<128, A_MN, B_MN, EPI, true>(P, g, stream);
+    }
+  }
   switch (g.block_n) {
-    case 256: return tc_launch_one<256, A_MN, B_MN, EPI>(P, g, stream);
-    case 128: return tc_launch_one<128, A_MN, B_MN, EPI>(P, g, stream);
-    default: return tc_launch_one<64, A_MN, B_MN, EPI>(P, g, stream);
+    case 256: return tc_launch_one<256, A_MN, B_MN, EPI, false>(P, g, stream);
+    case 128: return tc_launch_one<128, A_MN, B_MN, EPI, false>(P, g, stream);
+    default: return tc_launch_one<64, A_MN, B_MN, EPI, false>(P, g, stream);
   }
 }
 
-inline int tc_forward(const TcPlan& P, int l, cudaStream_t stream) {
+inline int tc_forward(TcPlan& P, int l, cudaStream_t stream) {
   return (l == P.n_layers - 1) ? tc_launch<false, true, TC_EPI_FWD_HEAD>(P, P.fwd[l], stream)
                                : tc_launch<false, true, TC_EPI_FWD_HIDDEN>(P, P.fwd[l], stream);
 }
-inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream, bool out_bf16) {
+inline int tc_wgrad(TcPlan& P, int l, cudaStream_t stream, bool out_bf16) {
   if (!out_bf16) return tc_launch<false, false, TC_EPI_WGRAD>(P, P.wgrad[l], stream);
   TcGemm g = P.wgrad[l];
   g.map_c = g.map_c16;
@@ -730,7 +892,7 @@ inline int tc_wgrad(const TcPlan& P, int l, cudaStream_t stream, bool out_bf16) 
 // The dgrad of layer l can also deliver the bias gradient of layer l - 1 (row sums of the backward signal it writes) when the
 // whole minibatch sits in one N tile; bias_g = destination buffer ([Z, ld] gradient rows, bf16 or fp32), nullptr = not fused.
 inline bool tc_dgrad_can_fuse_bias(const TcPlan& P, int l) { return l > 0 && P.dgrad[l].valid && P.dgrad[l].N <= P.dgrad[l].block_n; }
-inline int tc_dgrad(const TcPlan& P, int l, cudaStream_t stream, void* bias_g = nullptr, bool bias_bf16 = false) {
+inline int tc_dgrad(TcPlan& P, int l, cudaStream_t stream, void* bias_g = nullptr, bool bias_bf16 = false) {
   if (bias_g == nullptr) return tc_launch<true, true, TC_EPI_DGRAD>(P, P.dgrad[l], stream);
   TcGemm g = P.dgrad[l];
   g.ep.bias_g = bias_g; g.ep.bias_bf16 = bias_bf16 ? 1 : 0;

@@ -51,7 +51,7 @@ bool plan(const lsam_config& c, Layout& L) {
   L = Layout();
   if (c.K < 1 || c.K > 4096 || c.tau < 1 || c.stale_max < 0 || c.stale_max > 15) return false;
   if (c.gemm_dtype != LSAM_GEMM_FP32 && c.gemm_dtype != LSAM_GEMM_BF16) return false;
-  if (c.gemm_impl < LSAM_IMPL_AUTO || c.gemm_impl > LSAM_IMPL_TCGEN05) return false;
+  if (c.gemm_impl < LSAM_IMPL_AUTO || c.gemm_impl > LSAM_IMPL_TCGEN05_PAIRS) return false;
   if (!(c.gamma > 0.f)) return false;
   if (c.active_num < 0 || c.active_num > 256) return false;
   if (!(c.noise_temp >= 0.f)) return false;
@@ -859,7 +859,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   const bool mlp = cfg->model == LSAM_MODEL_MLP || cfg->model == LSAM_MODEL_RESMLP;
   bool tc_ok = false;
   if (mlp && cfg->gemm_dtype == LSAM_GEMM_BF16 && cfg->gemm_impl != LSAM_IMPL_SIMT) tc_ok = tc_supported(*cfg);
-  if (cfg->gemm_impl == LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
+  if (cfg->gemm_impl >= LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
   c->use_tc = tc_ok;
   c->grads_bf16 = tc_ok && !(cfg->flags & LSAM_FLAG_GRAD_FP32);
   {
@@ -887,6 +887,8 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     b.partial = c->at<float>(L.partial); b.ld_partial = L.nchunks;
     b.g1b = c->at<bf16>(L.g1b);
     c->tc.active = c->act();
+    c->tc.allow_pair = cfg->gemm_impl != LSAM_IMPL_TCGEN05_1CTA;
+    c->tc.force_pair = cfg->gemm_impl == LSAM_IMPL_TCGEN05_PAIRS;
     std::vector<TcLayer> tl;
     for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
     std::string why;

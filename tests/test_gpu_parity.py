@@ -226,9 +226,11 @@ def test_classifier_bf16_simt_small(model, widths, K, B):
     (G.MODEL_RESMLP, (128, 192, 192, 192, 100), 3, 200),  # N tile 256 with a ragged minibatch, skip connections
     (G.MODEL_MLP, (320, 520, 24), 2, 40),            # ragged M tiles (520 = 4 x 128 + 8), ragged contraction (320 = 5 x 64)
     (G.MODEL_RESMLP, (128, 256, 256, 40), 2, 300),   # minibatch wider than one N tile (256 + 44), five contraction blocks in wgrad
+    (G.MODEL_RESMLP, (192, 640, 640, 300), 3, 256),  # pairs of CTAs: 2.5 tiles of 256 rows (the last pair's second CTA lies outside), ragged head
 ])
-def test_classifier_bf16_tcgen05(model, widths, K, B):
-    p = _mlp_pair(model, widths, K, B, n=400, dtype=G.GEMM_BF16, impl=G.IMPL_TCGEN05, tau=4, lam=0.4, seed=4, jitter=0.01)
+@pytest.mark.parametrize("impl", [G.IMPL_TCGEN05, G.IMPL_TCGEN05_1CTA, G.IMPL_TCGEN05_PAIRS])  # the library's choice / single CTAs only / CTA pairs wherever possible
+def test_classifier_bf16_tcgen05(model, widths, K, B, impl):
+    p = _mlp_pair(model, widths, K, B, n=400, dtype=G.GEMM_BF16, impl=impl, tau=4, lam=0.4, seed=4, jitter=0.01)
     assert p.gpu.uses_tcgen05()
     _per_step_then_trajectory(p, 0.05, 0.1, TOL_STEP_BF16, TOL_TRAJ_BF16, what=f"bf16 tcgen05 {widths}")
     p.close()
