@@ -52,7 +52,8 @@ enum {
 enum { LSAM_MODEL_LSQ = 0, LSAM_MODEL_MLP = 1, LSAM_MODEL_RESMLP = 2, LSAM_MODEL_FLAT = 3 };
 enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
 /* TCGEN05: tensor-core GEMMs; forward and dgrad with a minibatch tile of 256 samples are run by pairs of CTAs
- * (cta_group::2, 256-row tiles), everything else by single CTAs (128-row tiles).  TCGEN05_1CTA: single CTAs only;
+ * (cta_group::2, 256-row tiles), everything else by single CTAs (128-row tiles); the weight gradient of a minibatch of at
+ * most 256 samples keeps its dz block in shared memory over a run of tiles.  TCGEN05_1CTA: single CTAs walking single tiles only;
  * TCGEN05_PAIRS: pairs wherever the kernel supports them (at least 256 rows, minibatch tile of at least 128). */
 enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2, LSAM_IMPL_TCGEN05_1CTA = 3, LSAM_IMPL_TCGEN05_PAIRS = 4 };
 /* Stationary kernels k(x, y) = phi(x - y) (Corollary 8 and the remark after it).  The worker's pull is

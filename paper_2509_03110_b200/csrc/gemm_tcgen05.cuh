@@ -212,6 +212,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool a_mn, bool 
 // TC_EPI_WGRAD_BF16: the weight gradient is stored rounded to bf16 (ascent pass: it only feeds the perturbation, whose
 // result is rounded to bf16 anyway; its norm is still taken from the fp32 accumulators).
 enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3, TC_EPI_WGRAD_BF16 = 4 };
+__host__ __device__ constexpr bool tc_epi_is_wgrad(int e) { return e >= TC_EPI_WGRAD; }
 
 struct TcEpi {
   // forward: bias (operand copy), out / skip / mask [Z, M, ldb]; head: logits fp32 [Z, M, ldb]
@@ -224,6 +225,7 @@ struct TcEpi {
   // wgrad: sum of squares of every 32-row block of the tile -> partial[z * ld_partial + slot0 + (mt * n_tiles + nt) * 8 + epilogue warp]
   float* partial;  int64_t ld_partial;  int slot0;
   int ldb;  // sample stride of the feature-major buffers (multiple of 16)
+  int run_n;  // A-stationary weight gradient: consecutive n-tiles per unit of the work list (>= 1)
   // dgrad, optional (bias_g != nullptr; needs the whole minibatch in one N tile): the bias gradient of the layer below,
   // db[m] = sum_b dz_prev[m][b], written to bias_g[z * bias_ld + bias_off + m] (bf16 if bias_bf16, else fp32), and the sum
   // of squares of every 8 consecutive db to partial[z * ld_partial + bias_slot0 + m / 8]
@@ -244,9 +246,15 @@ __host__ __device__ constexpr int tc_stages() { return PAIR ? (BLOCK_N == 256 ? 
 template <int BLOCK_N, bool PAIR = false>
 __host__ __device__ constexpr int tc_stage_bytes() { return (kTcBlockM + (PAIR ? BLOCK_N / 2 : BLOCK_N)) * kTcBlockK * 2; }
 constexpr int kTcStageOutBytes = 8 * 4096;  // wgrad epilogue staging: one 32-row x 128-byte block (128B-swizzled) per epilogue warp
-template <int BLOCK_N, bool PAIR = false>
+// ASTAT (A-stationary, contraction of at most kTcAstatKBlocks k-blocks): the whole A block of a tile row stays in shared
+// memory for a run of n-tiles, the ring holds B tiles only
+constexpr int kTcAstatKBlocks = 4;
+template <int BLOCK_N>
+__host__ __device__ constexpr int tc_astat_stages() { return BLOCK_N == 256 ? 4 : 8; }
+template <int BLOCK_N, bool PAIR = false, bool ASTAT = false>
 __host__ __device__ constexpr int tc_smem_bytes() {
-  return tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>() + 1024 /*alignment slack*/ + 256 /*barriers*/ + kTcStageOutBytes;
+  return (ASTAT ? kTcAstatKBlocks * kTcBlockM * kTcBlockK * 2 + tc_astat_stages<BLOCK_N>() * BLOCK_N * kTcBlockK * 2
+                : tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>()) + 1024 /*alignment slack*/ + 512 /*barriers*/ + kTcStageOutBytes;
 }
 
 // ------------------------------------------------------------------------------------------------ the kernel
@@ -255,13 +263,19 @@ __host__ __device__ constexpr int tc_smem_bytes() {
 //   M/N-contiguous operand:         map dims {rows, Kd, Z}, box {64, 64, 1} (one box per 64 rows of the tile)
 //   PAIR: the B box has BLOCK_N / 2 rows (contraction-contiguous) resp. the CTA loads BLOCK_N / 128 boxes (N-contiguous);
 //   the grid is a multiple of 2 and is launched with cluster dimension 2.
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR>
+//   ASTAT (weight gradient, single CTA, at most 4 k-blocks): the work list is made of runs of ep.run_n consecutive n-tiles of
+//   one (replica, m-tile); the A block (dz rows, all k-blocks) is loaded once per run into its own slots and reused by every
+//   tile of the run, so a tile takes in BLOCK_N x Kd instead of (128 + BLOCK_N) x Kd operand elements (the weight gradient is
+//   bound by the rate at which TMA fills shared memory from L2).  A slot is handed back to the producer as soon as the last
+//   tile of the run has used it, so the next run's A block streams in behind the current run's last tile.
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
                     int Z, TcEpi ep, int* __restrict__ status, const int32_t* __restrict__ active) {
   static_assert(!PAIR || BLOCK_N >= 128, "the pair form needs 64 rows of B per CTA");
-  constexpr int STAGES = tc_stages<BLOCK_N, PAIR>();
+  static_assert(!ASTAT || (!PAIR && !A_MN && !B_MN), "A-stationary form: single CTA, both operands contraction-contiguous");
+  constexpr int STAGES = ASTAT ? tc_astat_stages<BLOCK_N>() : tc_stages<BLOCK_N, PAIR>();
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
   constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;  // rows of the N side staged by this CTA
   constexpr int B_BYTES = B_ROWS * kTcBlockK * 2;
@@ -272,21 +286,30 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   extern __shared__ uint8_t smem_raw[];
   // round the tile area up to 1024 bytes by pointer arithmetic on the shared array itself (keeps the address space known)
   uint8_t* tiles = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
-  uint8_t* stage = tiles + STAGES * (A_BYTES + B_BYTES);  // 1024-byte aligned: the tile area is a multiple of 1024
+  // ASTAT: [A slots: kTcAstatKBlocks x A_BYTES][B ring: STAGES x B_BYTES]; else a ring of STAGES x (A tile, B tile)
+  constexpr int RING_STRIDE = ASTAT ? B_BYTES : A_BYTES + B_BYTES;
+  constexpr int RING_B_OFF = ASTAT ? 0 : A_BYTES;
+  uint8_t* ring = tiles + (ASTAT ? kTcAstatKBlocks * A_BYTES : 0);
+  uint8_t* stage = ring + STAGES * RING_STRIDE;  // 1024-byte aligned: everything before it is a multiple of 1024
   uint64_t* bars = reinterpret_cast<uint64_t*>(stage + kTcStageOutBytes);
   uint64_t* full = bars;                     // [STAGES]  TMA -> MMA
   uint64_t* empty = bars + STAGES;           // [STAGES]  MMA -> TMA
   uint64_t* acc_full = bars + 2 * STAGES;    // [2]       MMA -> epilogue
   uint64_t* acc_empty = acc_full + 2;        // [2]       epilogue -> MMA
   uint64_t* bias_bar = acc_empty + 2;        // [4 quadrants][2]  dgrad: the two epilogue warps of a quadrant have left their partial bias sums
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bias_bar + 8);
+  uint64_t* a_full = bias_bar + 8;           // [4]  ASTAT: A slot kb loaded        TMA -> MMA
+  uint64_t* a_empty = a_full + 4;            // [4]  ASTAT: A slot kb free again    MMA -> TMA
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(a_empty + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int m_tiles = (M + TILE_M - 1) / TILE_M;
   const int n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_blocks = (Kd + kTcBlockK - 1) / kTcBlockK;
-  const int64_t total = (int64_t)Z * m_tiles * n_tiles;
+  // work list: units of (replica, m-tile, run of n-tiles); a run is one tile unless ASTAT
+  const int run_n = ASTAT ? (ep.run_n > 0 ? ep.run_n : 1) : 1;
+  const int runs = (n_tiles + run_n - 1) / run_n;
+  const int64_t total = (int64_t)Z * m_tiles * runs;
   // a pair walks the work list together: unit = index of this CTA (or of its pair), units = how many walk the list
   const uint32_t rank = PAIR ? tc::cluster_ctarank() : 0u;
   const bool leader = rank == 0u;
@@ -298,7 +321,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
     for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], PAIR ? 2 * kTcEpiWarps : kTcEpiWarps); }
     for (int s = 0; s < 8; ++s) tc::mbar_init(&bias_bar[s], 2);
-    static_assert((2 * STAGES + 4 + 8) * 8 + 8 <= 256, "barrier area");
+    for (int s = 0; s < 4; ++s) { tc::mbar_init(&a_full[s], 1); tc::mbar_init(&a_empty[s], 1); }
+    static_assert((2 * STAGES + 4 + 8 + 8) * 8 + 8 <= 512, "barrier area");
     *abort_flag = 0;
     tc::fence_barrier_init();
   }
@@ -331,16 +355,28 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
+      uint32_t run_ph = 0;  // ASTAT: phase of the A-slot barriers, one flip per run
       for (int64_t t = unit; t < total && ok; t += units) {
-        const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
+        const int r = (int)(t % runs), mt = (int)((t / runs) % m_tiles), z = (int)(t / ((int64_t)runs * m_tiles));
         if (active != nullptr && !active[z]) continue;  // waiting replica: all three roles skip the same tiles
+        const int nt_begin = r * run_n, nt_end = (nt_begin + run_n < n_tiles) ? nt_begin + run_n : n_tiles;
+        for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
         const int m0 = mt * TILE_M + m_off, n0 = nt * BLOCK_N + n_off;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
-          uint8_t* a_dst = tiles + s * (A_BYTES + B_BYTES);
-          uint8_t* b_dst = a_dst + A_BYTES;
           const int k0 = kb * kTcBlockK;
-          if (PAIR) {
+          if (ASTAT && nt == nt_begin) {
+            // first tile of a run: bring in A slot kb as soon as the previous run has released it
+            if (!tc::mbar_wait(&a_empty[kb], run_ph ^ 1u, abort_flag)) { ok = false; break; }
+            tc::mbar_expect_tx(&a_full[kb], A_BYTES);
+            tc::tma_load_3d(tiles + kb * A_BYTES, &map_a, k0, m0, z, &a_full[kb]);
+          }
+          if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
+          uint8_t* a_dst = ring + s * RING_STRIDE;
+          uint8_t* b_dst = a_dst + RING_B_OFF;
+          if (ASTAT) {
+            tc::mbar_expect_tx(&full[s], B_BYTES);
+            tc::tma_load_3d(b_dst, &map_b, k0, n0, z, &full[s]);
+          } else if (PAIR) {
             // both CTAs' loads of this stage complete on the leader's barrier, which the leader arms with the bytes of both
             if (leader) tc::mbar_expect_tx(&full[s], 2 * (A_BYTES + B_BYTES));
             const uint32_t bar = tc::map_to_cta(tc::smem_u32(&full[s]), 0u);
@@ -373,6 +409,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
+        }
+        run_ph ^= 1u;
       }
       if (!ok) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
     }
@@ -384,16 +422,20 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int as = 0;
       uint32_t aph = 0;
       bool ok = true;
+      uint32_t run_ph = 0;
       for (int64_t t = unit; t < total && ok; t += units) {
-        if (active != nullptr && !active[(int)(t / ((int64_t)n_tiles * m_tiles))]) continue;
+        if (active != nullptr && !active[(int)(t / ((int64_t)runs * m_tiles))]) continue;
+        const int nt_begin = (int)(t % runs) * run_n, nt_end = (nt_begin + run_n < n_tiles) ? nt_begin + run_n : n_tiles;
+        for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
         if (!tc::mbar_wait(&acc_empty[as], aph ^ 1u, abort_flag)) { ok = false; break; }
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(as * BLOCK_N);
         for (int kb = 0; kb < k_blocks; ++kb) {
+          if (ASTAT && nt == nt_begin && !tc::mbar_wait(&a_full[kb], run_ph, abort_flag)) { ok = false; break; }
           if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc::tc_fence_after();
-          const uint32_t a_addr = tc::smem_u32(tiles + s * (A_BYTES + B_BYTES));
-          const uint32_t b_addr = a_addr + A_BYTES;
+          const uint32_t a_addr = tc::smem_u32(ASTAT ? tiles + kb * A_BYTES : ring + s * RING_STRIDE);
+          const uint32_t b_addr = tc::smem_u32(ring + s * RING_STRIDE + RING_B_OFF);
 #pragma unroll
           for (int k = 0; k < kTcBlockK / 16; ++k) {
             // contraction-contiguous tile: rows of 128 B, 8-row groups 1024 B apart, a K = 16 slice is 32 B further along the row;
@@ -407,12 +449,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           // frees the stage (in both CTAs of a pair) when these MMAs have read it
           if (PAIR) tc::umma_commit_pair(&empty[s]);
           else tc::umma_commit(&empty[s]);
+          if (ASTAT && nt == nt_end - 1) tc::umma_commit(&a_empty[kb]);  // last tile of the run: the A slot is free once these MMAs are done
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
         if (PAIR) tc::umma_commit_pair(&acc_full[as]);
         else tc::umma_commit(&acc_full[as]);
         if (++as == 2) { as = 0; aph ^= 1u; }
+        }
+        run_ph ^= 1u;
       }
       if (!ok) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
     }
@@ -427,8 +472,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     bool ok = true;
     const uint32_t acc_empty_leader[2] = {PAIR ? tc::map_to_cta(tc::smem_u32(&acc_empty[0]), 0u) : 0u, PAIR ? tc::map_to_cta(tc::smem_u32(&acc_empty[1]), 0u) : 0u};
     for (int64_t t = unit; t < total && ok; t += units) {
-      const int nt = (int)(t % n_tiles), mt = (int)((t / n_tiles) % m_tiles), z = (int)(t / ((int64_t)n_tiles * m_tiles));
+      const int r_ = (int)(t % runs), mt = (int)((t / runs) % m_tiles), z = (int)(t / ((int64_t)runs * m_tiles));
       if (active != nullptr && !active[z]) continue;
+      const int nt_begin = r_ * run_n, nt_end = (nt_begin + run_n < n_tiles) ? nt_begin + run_n : n_tiles;
+      for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
       const int m_base = mt * TILE_M + m_off;  // first row of the 128 rows this CTA drains
       const int m = m_base + quad * 32 + lane;
       const int n0 = nt * BLOCK_N;
@@ -596,7 +643,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           }
         }
       }
-      if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && ep.partial != nullptr) {
+      if (tc_epi_is_wgrad(EPI) && ep.partial != nullptr) {
         // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows; the slots are
         // laid out by 128-row block of the output (a CTA of a pair whose rows lie wholly outside the matrix has none)
         const float tot = warp_sum(ssq);
@@ -632,6 +679,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         else tc::mbar_arrive(&acc_empty[as]);
       }
       if (++as == 2) { as = 0; aph ^= 1u; }
+      }
     }
     if ((EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) && lane == 0) tc::bulk_wait_all<0>();  // every gradient block has reached global memory
     if (!ok && lane == 0) { *abort_flag = 1; atomicOr(status, STATUS_TIMEOUT); }
@@ -686,6 +734,7 @@ struct TcGemm {
   TcEpi ep{};
   bool valid = false;
   bool pair = false;  // run by pairs of CTAs (cta_group::2) on 256-row tiles
+  bool astat = false; // weight gradient with the A block stationary over runs of n-tiles (ep.run_n)
 };
 
 struct TcPlan {
@@ -698,6 +747,7 @@ struct TcPlan {
   int n_slots = 0;              // partial slots used per replica
   bool allow_pair = true;       // false: every GEMM on the single-CTA kernels
   bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
+  bool allow_astat = true;      // false: the weight gradient walks single tiles
   int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
 };
 
@@ -794,11 +844,24 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
-      // the same rows of the bf16 ascent-gradient buffer
+      // the same rows of the bf16 gradient buffer
       ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
-      slot += (int)(ceil_div(ly.out, kTcBlockM) * ceil_div(ly.in, g.block_n) * kTcEpiWarps);
+      g.astat = P.allow_astat && !g.pair && B <= kTcAstatKBlocks * kTcBlockK;
+      g.ep.run_n = 1;
+      if (g.astat) {
+        // run length: a unit of the list costs run_n B tiles plus one A block (half a B tile at BLOCK_N = 256); the SMs work through
+        // ceil(units / SMs) rounds of units.  Pick the run length with the least bytes through the busiest SM.
+        const int64_t rows = (int64_t)Z * ceil_div(g.M, kTcBlockM), n_tiles = ceil_div(g.N, g.block_n);
+        double best = 0.0;
+        for (int rn = 1; rn <= n_tiles; ++rn) {
+          const int64_t units = rows * ceil_div(n_tiles, (int64_t)rn);
+          const double cost = (double)ceil_div(units, (int64_t)P.sms) * ((double)rn * g.block_n + kTcBlockM);
+          if (rn == 1 || cost < best) { best = cost; g.ep.run_n = rn; }
+        }
+      }
+      slot += (int)(ceil_div(g.M, kTcBlockM) * ceil_div(g.N, g.block_n) * kTcEpiWarps);
       P.bias_slot0[l] = slot;
       slot += (int)ceil_div(ly.out, 8);
       g.valid = ok;
@@ -823,10 +886,10 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   return 0;
 }
 
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR>
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false>
 inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
-  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR>;
-  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR>();
+  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR, ASTAT>;
+  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR, ASTAT>();
   // the shared-memory limit of a kernel is a per-device attribute: remember it per device ordinal
   static bool attr_set[64] = {};
   int dev = 0;
@@ -836,7 +899,8 @@ inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
     attr_set[dev] = true;
   }
   const int tile_m = PAIR ? 2 * kTcBlockM : kTcBlockM;
-  const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, tile_m) * ceil_div(g.N, BLOCK_N);
+  const int64_t n_tiles = ceil_div(g.N, BLOCK_N);
+  const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, tile_m) * (ASTAT ? ceil_div(n_tiles, (int64_t)(g.ep.run_n > 0 ? g.ep.run_n : 1)) : n_tiles);  // units of the work list
   if (!PAIR) {
     const int grid = (int)(tiles < P.sms ? tiles : P.sms);
     kern<<<grid, kTcThreads, smem, stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status, P.active);
@@ -870,6 +934,15 @@ inline int tc_launch(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
     switch (g.block_n) {
       case 256: return tc_launch_one<256, A_MN, B_MN, EPI, true>(P, g, stream);
       default: return tc_launch_one<128, A_MN, B_MN, EPI, true>(P, g, stream);
+    }
+  }
+  if constexpr (tc_epi_is_wgrad(EPI) && !A_MN && !B_MN) {
+    if (g.astat) {
+      switch (g.block_n) {
+        case 256: return tc_launch_one<256, A_MN, B_MN, EPI, false, true>(P, g, stream);
+        case 128: return tc_launch_one<128, A_MN, B_MN, EPI, false, true>(P, g, stream);
+        default: return tc_launch_one<64, A_MN, B_MN, EPI, false, true>(P, g, stream);
+      }
     }
   }
   switch (g.block_n) {

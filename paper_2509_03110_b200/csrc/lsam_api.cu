@@ -889,6 +889,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     c->tc.active = c->act();
     c->tc.allow_pair = cfg->gemm_impl != LSAM_IMPL_TCGEN05_1CTA;
     c->tc.force_pair = cfg->gemm_impl == LSAM_IMPL_TCGEN05_PAIRS;
+    c->tc.allow_astat = cfg->gemm_impl != LSAM_IMPL_TCGEN05_1CTA;  // the plain single-CTA kernels stay reachable (and tested) through this setting
     std::vector<TcLayer> tl;
     for (const LayerInfo& li : L.layers) tl.push_back({li.in, li.out, li.w_pad, li.b_pad, li.residual});
     std::string why;
