@@ -321,12 +321,11 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
     local = dev.index
     # sharded: every rank generates the same dataset and the same initial point (one job); else independent copies
     inp = make_inputs(w, dev, seed=0 if shard else rank)
-    # Latency-bound workloads (state resident in L2) replay each tick as one CUDA graph; that needs a capturable stream.
+    # Each tick is replayed as one CUDA graph (auto: always): the 30-40 launches of a tick leave gaps that are a visible share
+    # of the step for the latency-bound workloads (C1: 38.6 -> 25.8 us) and still 1 % at the largest one (16.45 -> 16.26 ms).
+    # That needs a capturable stream; the per-kernel shares then come from a second pass over the same steps with per-launch events.
     small = 4.0 * w["K"] * param_count(w) <= 126e6
-    # auto: also where the kernels of a step are short (tens of microseconds each), so that launch gaps and the
-    # per-launch events of the roofline pass would be a visible share of the step
-    short_kernels = 4.0 * w["K"] * param_count(w) <= 1.2e9
-    use_graph = (small or short_kernels) if cuda_graph == "auto" else cuda_graph == "on"
+    use_graph = True if cuda_graph == "auto" else cuda_graph == "on"
     flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0)
     cfg = make_cfg(G, w, flags=flags, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0, gemm_impl=gemm_impl)
     torch.cuda.synchronize()
@@ -566,7 +565,7 @@ def main():
     ap.add_argument("--shard-workers", action="store_true",
                     help="N > 1: one job of N*K workers with a single centre, K workers per GPU, accumulator all-reduce every tau steps "
                          "(default: N independent copies of the workload)")
-    ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: when the state fits in L2)")
+    ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: on)")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
     modified = False

@@ -112,13 +112,17 @@ def test_c3_full_shape_sixteen_free_running_ticks_of_two_replicas():
                 assert rel_l2(first["xp"][i], oxp16[i]) <= 1e-3
     assert o.should_couple()
     s = o.read_state()
+    lam = w.get("lambda0", bench.LAMBDA0) / (w["eta"] * w["tau"])
     for i, k in enumerate(picks):
         assert rel_l2(gx[i], s["x"][i]) <= TOL_TRAJ_BF16, (k, rel_l2(gx[i], s["x"][i]))
         assert median_abs_rows(gx[i], s["x"][i]) <= TOL_TRAJ_BF16 / BULK_DIVISOR
-        # the iterates barely move against their own norm in 16 ticks; the path travelled is the sharper quantity
+        # the iterates barely move against their own norm in 16 ticks; the path travelled is the sharper quantity.  It is a
+        # sum of gradient steps (and so is the momentum buffer), so it inherits the per-tick gradient bound
         moved = rel_l2(gx[i] - x0_rows[i], s["x"][i] - x0_rows[i])
-        assert moved <= TOL_TRAJ_BF16, (k, moved)
-        assert rel_l2(gv[i], s["v"][i]) <= TOL_TRAJ_BF16, (k, rel_l2(gv[i], s["v"][i]))
+        assert moved <= TOL_GRAD_BF16_FULL, (k, moved)
+        # momentum buffer: a geometric sum (ratio mu) of G = g2 + lambda (x - y), bounded on the scale of its inputs
+        scale = (lam * np.linalg.norm(s["x"][i]) + on2[i]) / (1.0 - bench.MU)
+        assert np.linalg.norm(gv[i] - s["v"][i]) <= TOL_TRAJ_BF16 * scale, (k, np.linalg.norm(gv[i] - s["v"][i]) / scale)
     ctx.close()
     o.close()
 
@@ -167,12 +171,12 @@ def test_c4_full_widths_two_replicas_sync_every_tick_with_stale_reads():
     s = o.read_state()
     gy = ctx.read_params(-1).astype(np.float64)
     assert rel_l2(gy, s["y"]) <= TOL_TRAJ_BF16
-    assert rel_l2(gy - y0, s["y"] - y0) <= TOL_TRAJ_BF16, rel_l2(gy - y0, s["y"] - y0)
+    assert rel_l2(gy - y0, s["y"] - y0) <= TOL_GRAD_BF16_FULL, rel_l2(gy - y0, s["y"] - y0)  # the path travelled: a sum of gradient steps
     assert median_abs_rows(gy, s["y"]) <= TOL_TRAJ_BF16 / BULK_DIVISOR
     for k in range(K):
         gx = ctx.read_params(k).astype(np.float64)
         assert rel_l2(gx, s["x"][k]) <= TOL_TRAJ_BF16
-        assert rel_l2(gx - x0[k], s["x"][k] - x0[k]) <= TOL_TRAJ_BF16, (k, rel_l2(gx - x0[k], s["x"][k] - x0[k]))
+        assert rel_l2(gx - x0[k], s["x"][k] - x0[k]) <= TOL_GRAD_BF16_FULL, (k, rel_l2(gx - x0[k], s["x"][k] - x0[k]))
         assert median_abs_rows(gx, s["x"][k]) <= TOL_TRAJ_BF16 / BULK_DIVISOR
     ctx.close()
     o.close()
