@@ -72,3 +72,51 @@ def test_resumed_run_continues_bit_for_bit(kind):
         o.load_checkpoint(np.concatenate([blob, np.zeros(1 << 22, np.uint8)]))
     for c in (a, b, o):
         c.close()
+
+
+def test_load_drops_staged_minibatches_and_refuses_inconsistent_counters():
+    # a minibatch staged before lsam_load_checkpoint belongs to the run being replaced: the resumed run must not consume it;
+    # a blob whose counters describe no reachable state (negative or more than K tau iterations since the last sync, a
+    # centre-version history beyond the current version) is refused and leaves the context as it was
+    import torch
+
+    widths, K, B = (32, 40, 6), 3, 16
+    X, labels = synth.gaussian_mixture(200, 32, 6, seed=1)
+    w0 = synth.mlp_init(widths, seed=1)
+    x0 = synth.replicate(w0, K)
+    dX, dY = torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda()
+    mk = lambda: G.Lsam(G.make_config(G.MODEL_MLP, widths=widths, K=K, batch=B, n_samples=200, tau=2, lam=0.3, seed=9), dX, dY,
+                        torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+    a = mk()
+    a.step(0.05, 0.05)
+    blob = a.save_checkpoint()
+    idx, _, _ = a.read_schedule(1, want_ver=False)
+    xb = torch.from_numpy(X[idx.ravel()].reshape(K, B, 32)).pin_memory()
+    yb = torch.from_numpy(labels[idx.ravel()].reshape(K, B)).pin_memory()
+    a.stage_batch(xb, yb)
+    a.load_checkpoint(blob)
+    with pytest.raises(G.LsamError) as ei:
+        a.step_staged(0.05, 0.05)  # nothing is staged any more
+    assert ei.value.code == G.LSAM_ERR_STATE
+    hdr = 8 + 8 * 7 + 4 * 16  # magic, seven int64 fields, sixteen int32 history entries
+    tx = blob[hdr:hdr + 8 * K].view(np.int64)
+    assert tx.tolist() == [1] * K
+    for mutate in ("negative", "too_many", "history"):
+        bad = blob.copy()
+        if mutate == "negative":
+            bad[hdr:hdr + 8].view(np.int64)[0] = -1
+        elif mutate == "too_many":
+            bad[hdr:hdr + 8].view(np.int64)[0] = 100
+        else:
+            bad[8 + 8 * 7:8 + 8 * 7 + 4].view(np.int32)[0] = 5  # step 0 started at centre version 5 of a run whose version is 0
+        with pytest.raises(G.LsamError) as ei:
+            a.load_checkpoint(bad)
+        assert ei.value.code == G.LSAM_ERR_INVALID
+        assert a.counters()[0] == 1 and a.counters()[2].tolist() == [1] * K  # untouched
+    b = mk()
+    b.load_checkpoint(blob)
+    for c in (a, b):
+        c.step(0.05, 0.05)
+    np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
+    a.close()
+    b.close()
