@@ -483,7 +483,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       tc::tc_fence_after();
       const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BLOCK_N);
       float bias = 0.f;
-      float ssq = 0.f;  // wgrad: sum of squares of this thread's row of the tile
+      float ssq4[4] = {0.f, 0.f, 0.f, 0.f};  // wgrad: sum of squares of this thread's row of the tile, four interleaved partial sums (column mod 4)
       float bsum = 0.f; // dgrad: this thread's share of the bias gradient of its row (samples of its chunks, ascending)
       if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) bias = to_float(ep.bias[(int64_t)z * ep.ld_p + m]);
 #pragma unroll 1
@@ -501,7 +501,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const int mrow0 = m_base + quad * 32;
           if (mrow0 < M && nb < N) {  // warp-uniform: blocks wholly outside the matrix are neither staged nor stored
 #pragma unroll
-            for (int j = 0; j < 32; ++j) ssq = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ssq);  // zero-filled edges add 0
+            for (int j = 0; j < 32; ++j) ssq4[j & 3] = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ssq4[j & 3]);  // zero-filled edges add 0
             // fp32: one 32-column block per store.  bf16: two consecutive blocks share one buffer (rows of 64 bf16 = 128
             // bytes, the same swizzle) and are stored together after the second one, or after the last valid one.
             const bool first_half = (EPI == TC_EPI_WGRAD) || ((c & 1) == 0);
@@ -646,7 +646,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       if (tc_epi_is_wgrad(EPI) && ep.partial != nullptr) {
         // fixed order: 32 columns x 8 chunks sequentially per thread, xor-shuffle tree over the 32 rows; the slots are
         // laid out by 128-row block of the output (a CTA of a pair whose rows lie wholly outside the matrix has none)
-        const float tot = warp_sum(ssq);
+        const float tot = warp_sum((ssq4[0] + ssq4[1]) + (ssq4[2] + ssq4[3]));
         if (lane == 0 && m_base < M) ep.partial[(int64_t)z * ep.ld_partial + ep.slot0 + ((int64_t)(m_base / kTcBlockM) * n_tiles + nt) * kTcEpiWarps + ew] = tot;
       }
       if (EPI == TC_EPI_DGRAD && ep.bias_g != nullptr) {
