@@ -468,7 +468,13 @@ int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N
   const bool a_mc = (A.sr == 1), b_nc = (B.sr == 1);
   if (!a_mc && A.sk != 1) return c->fail(LSAM_ERR_INVALID, "SIMT GEMM: operand A has no unit stride");
   if (!b_nc && B.sk != 1) return c->fail(LSAM_ERR_INVALID, "SIMT GEMM: operand B has no unit stride");
-#define LSAM_SIMT(AM, BN_) LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()))
+  // a tile list shorter than two blocks per SM with a long contraction: two thread groups per block split the contraction
+  const bool split = (int64_t)grid.x * grid.y * grid.z < 2 * 148 && Kd >= 8 * kSimtBK;
+#define LSAM_SIMT(AM, BN_)                                                                                                                        \
+  do {                                                                                                                                            \
+    if (split) LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 2><<<grid, 512, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));              \
+    else LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 1><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));                    \
+  } while (0)
   if (a_mc) { if (b_nc) LSAM_SIMT(true, true); else LSAM_SIMT(true, false); }
   else      { if (b_nc) LSAM_SIMT(false, true); else LSAM_SIMT(false, false); }
 #undef LSAM_SIMT
@@ -499,8 +505,13 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
     GemmOperand A{a_in, (int64_t)li.in * ldb, 1, ldb};       // (z, b, i) in the feature-major buffer [z][i][b]
     GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, o, i)
     if (head && li.out <= kHeadMaxOut) {
-      dim3 hgrid((unsigned)ceil_div(B, 32), K);
-      LAUNCH(c, LSAM_PROF_GEMM_FWD, head_forward_kernel<T><<<hgrid, 256, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, P, ld, li.w_pad, li.b_pad, li.in, li.out, B, c->at<float>(L.logits), c->act()));
+      if (ceil_div(B, 32) * K < 148) {  // too few blocks of 32 samples to fill the machine: 8 samples per block
+        dim3 hgrid((unsigned)ceil_div(B, 8), K);
+        LAUNCH(c, LSAM_PROF_GEMM_FWD, head_forward_kernel<T, 8><<<hgrid, 256, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, P, ld, li.w_pad, li.b_pad, li.in, li.out, B, c->at<float>(L.logits), c->act()));
+      } else {
+        dim3 hgrid((unsigned)ceil_div(B, 32), K);
+        LAUNCH(c, LSAM_PROF_GEMM_FWD, head_forward_kernel<T, 32><<<hgrid, 256, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, P, ld, li.w_pad, li.b_pad, li.in, li.out, B, c->at<float>(L.logits), c->act()));
+      }
       rc = LSAM_OK;
     } else if (head) {
       EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), li.out, ldb};

@@ -103,16 +103,20 @@ struct EpiFwdHead {
 // per-warp sums are added in warp order at the end, so the result is deterministic.
 constexpr int kHeadMaxOut = 16;
 constexpr int kHeadChunk = 256;
-template <typename T>
+// SPB = samples per block: 32 (a lane owns a sample) or 8 (a lane owns a sample and one of four interleaved input streams;
+// four times the blocks, for minibatches too small to fill the machine otherwise).
+template <typename T, int SPB>
 __global__ void __launch_bounds__(256)
 head_forward_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, const T* __restrict__ P, int64_t ld_p, int64_t w_off, int64_t b_off,
                     int in, int out, int B, float* __restrict__ logits, const int32_t* __restrict__ active) {
+  constexpr int QN = 32 / SPB;  // input streams per warp
   const int z = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   __shared__ float wch[kHeadMaxOut][kHeadChunk];
   __shared__ float part[8][kHeadMaxOut][32];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int b = blockIdx.x * 32 + lane;
+  const int sl = lane % SPB, q = lane / SPB;
+  const int b = blockIdx.x * SPB + sl;
   const bool bv = b < B;
   const T* az = a + (int64_t)z * a_sz + (bv ? b : 0);
   const T* W = P + (int64_t)z * ld_p + w_off;
@@ -128,13 +132,13 @@ head_forward_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, const T* __r
     }
     __syncthreads();
     // inputs past the end of the last chunk have zero weights; their activations are not read
-    for (int ii = w; ii < len; ii += 64) {
+    for (int ii = w * QN + q; ii < len; ii += 64 * QN) {
       float av[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) av[u] = (ii + 8 * u < len) ? to_float(az[(int64_t)(i0 + ii + 8 * u) * ldb]) : 0.f;
+      for (int u = 0; u < 8; ++u) av[u] = (ii + 8 * QN * u < len) ? to_float(az[(int64_t)(i0 + ii + 8 * QN * u) * ldb]) : 0.f;
 #pragma unroll
       for (int u = 0; u < 8; ++u) {
-        const int iu = min(ii + 8 * u, kHeadChunk - 1);
+        const int iu = min(ii + 8 * QN * u, kHeadChunk - 1);
 #pragma unroll
         for (int f = 0; f < kHeadMaxOut; ++f) acc[f] = fmaf(wch[f][iu], av[u], acc[f]);
       }
@@ -143,12 +147,15 @@ head_forward_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, const T* __r
 #pragma unroll
   for (int f = 0; f < kHeadMaxOut; ++f) part[w][f][lane] = acc[f];
   __syncthreads();
-  for (int e = threadIdx.x; e < out * 32; e += 256) {
-    const int f = e >> 5, l = e & 31, bb = blockIdx.x * 32 + l;
+  for (int e = threadIdx.x; e < out * SPB; e += 256) {
+    const int f = e / SPB, l = e % SPB, bb = blockIdx.x * SPB + l;
     if (bb >= B) continue;
     float s = to_float(P[(int64_t)z * ld_p + b_off + f]);
+    // fixed order: warps ascending, input streams ascending
 #pragma unroll
-    for (int q = 0; q < 8; ++q) s += part[q][f][l];
+    for (int qq = 0; qq < 8; ++qq)
+#pragma unroll
+      for (int k2 = 0; k2 < QN; ++k2) s += part[qq][f][k2 * SPB + l];
     logits[((int64_t)z * out + f) * ldb + bb] = s;
   }
 }
@@ -212,18 +219,29 @@ __device__ inline float4 simt_fetch4(const T* __restrict__ base, int64_t sr, int
   return v;
 }
 
-template <typename TA_, typename TB_, bool A_MC, bool B_NC, class Epi>
-__global__ void __launch_bounds__(256)
+// SPLITK = 2: the block has two groups of 256 threads that walk alternate BK-slabs of the contraction with their own
+// shared-memory tiles (twice the warps per SM for the GEMMs whose tile list is shorter than the machine); at the end group 1
+// hands its accumulators to group 0 through shared memory and group 0 adds them in a fixed order (own + other) and runs the
+// epilogue.  The groups synchronise on their own named barriers (their slab counts may differ by one).
+template <typename TA_, typename TB_, bool A_MC, bool B_NC, class Epi, int SPLITK = 1>
+__global__ void __launch_bounds__(256 * SPLITK)
 gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, const int32_t* __restrict__ active) {
   constexpr int BM = kSimtBM, BN = kSimtBN, BK = kSimtBK;
   if (active != nullptr && !active[blockIdx.z]) return;  // a waiting replica
-  __shared__ __align__(16) float As[BK][BM + 4];
-  __shared__ __align__(16) float Bs[BK][BN + 4];
+  constexpr int A_FLOATS = BK * (BM + 4), B_FLOATS = BK * (BN + 4);
+  __shared__ __align__(16) float smem[SPLITK * (A_FLOATS + B_FLOATS)];
+  const int grp = SPLITK == 1 ? 0 : (int)threadIdx.x / 256;
+  float (*As)[BM + 4] = reinterpret_cast<float (*)[BM + 4]>(smem + grp * (A_FLOATS + B_FLOATS));
+  float (*Bs)[BN + 4] = reinterpret_cast<float (*)[BN + 4]>(smem + grp * (A_FLOATS + B_FLOATS) + A_FLOATS);
+  auto group_sync = [&]() {
+    if (SPLITK == 1) __syncthreads();
+    else asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
+  };
   const int z = blockIdx.z;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const TA_* Ap = reinterpret_cast<const TA_*>(A.p) + (int64_t)z * A.sz;
   const TB_* Bp = reinterpret_cast<const TB_*>(Bo.p) + (int64_t)z * Bo.sz;
-  const int tid = threadIdx.x;
+  const int tid = threadIdx.x & 255;
   const int tx = tid & 15, ty = tid >> 4;
   // 128-bit loads need the contiguous stride to be 1 (guaranteed by the template flag), the other stride a multiple
   // of 4 elements and the replica's base 16-byte aligned
@@ -267,12 +285,15 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, c
     }
   };
 
-  fetch(0);
-  stash();
-  __syncthreads();
-  for (int k0 = 0; k0 < Kd; k0 += BK) {
-    const bool more = k0 + BK < Kd;
-    if (more) fetch(k0 + BK);
+  constexpr int KSTEP = SPLITK * BK;  // a group's slabs: grp * BK, grp * BK + KSTEP, ...
+  if (grp * BK < Kd) {
+    fetch(grp * BK);
+    stash();
+  }
+  group_sync();
+  for (int k0 = grp * BK; k0 < Kd; k0 += KSTEP) {
+    const bool more = k0 + KSTEP < Kd;
+    if (more) fetch(k0 + KSTEP);
 #pragma unroll
     for (int kk = 0; kk < BK; ++kk) {
       const float4 a0 = *reinterpret_cast<const float4*>(&As[kk][ty * 8]);
@@ -285,11 +306,32 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, c
 #pragma unroll
         for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a_[i], b_[j], acc[i][j]);
     }
-    __syncthreads();
+    group_sync();
     if (more) {
       stash();
-      __syncthreads();
+      group_sync();
     }
+  }
+  if (SPLITK == 2) {
+    // group 1 -> group 0, in two halves of 4 accumulator rows (16 KB each, in the tile memory both groups are done with)
+    float4* xch = reinterpret_cast<float4*>(smem);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      __syncthreads();
+      if (grp == 1) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) xch[i * 256 + tid] = make_float4(acc[4 * h + i][0], acc[4 * h + i][1], acc[4 * h + i][2], acc[4 * h + i][3]);
+      }
+      __syncthreads();
+      if (grp == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float4 o = xch[i * 256 + tid];
+          acc[4 * h + i][0] += o.x; acc[4 * h + i][1] += o.y; acc[4 * h + i][2] += o.z; acc[4 * h + i][3] += o.w;
+        }
+      }
+    }
+    if (grp == 1) return;
   }
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
