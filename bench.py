@@ -308,7 +308,7 @@ def workload_config(w):
 
 
 # ---------------------------------------------------------------------------------------------- one workload on this rank's GPU
-def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True, gemm_impl=0):
+def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True, gemm_impl=0, fused_update=False):
     """Create the context, time `steps` steps after `warmup` untimed ones, and return the record of this workload
     (rank 0; None on the other ranks).  A step is one pass of the whole hot path plus the centre update when it is due."""
     import torch
@@ -325,8 +325,8 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
     # of the step for the latency-bound workloads (C1: 38.6 -> 25.8 us) and still 1 % at the largest one (16.45 -> 16.26 ms).
     # That needs a capturable stream; the per-kernel shares then come from a second pass over the same steps with per-launch events.
     small = 4.0 * w["K"] * param_count(w) <= 126e6
-    use_graph = True if cuda_graph == "auto" else cuda_graph == "on"
-    flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0)
+    use_graph = (not fused_update) if cuda_graph == "auto" else cuda_graph == "on"
+    flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0) | (G.FLAG_FUSED_UPDATE if fused_update else 0)
     cfg = make_cfg(G, w, flags=flags, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0, gemm_impl=gemm_impl)
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream(device=dev)
@@ -560,6 +560,7 @@ def main():
     ap.add_argument("--noise-temp", type=float, default=0.0, help="Langevin temperature of the sampler (0 = none)")
     ap.add_argument("--active-num", type=int, default=256, help="asynchronous progress: a worker is ready at a tick with probability N/256")
     ap.add_argument("--grad-fp32", action="store_true", help="tensor-core path: store the gradients in fp32 instead of bf16")
+    ap.add_argument("--fused-update", action="store_true", help="tensor-core path: worker update of the weights inside the descent-pass weight-gradient epilogue")
     ap.add_argument("--gemm-impl", default="auto", choices=["auto", "simt", "tcgen05", "tcgen05-1cta", "tcgen05-pairs"],
                     help="auto: tensor-core GEMMs for the bf16 workloads (CTA pairs where a GEMM is large enough); tcgen05-1cta: single-CTA kernels only")
     ap.add_argument("--shard-workers", action="store_true",
@@ -608,10 +609,10 @@ def main():
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
     rec = run_workload(args.workload, w, args.steps, args.warmup, dev, rank, world, shard=shard, cuda_graph=args.cuda_graph,
-                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline,
+                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline, fused_update=args.fused_update,
                        gemm_impl={"auto": 0, "simt": 1, "tcgen05": 2, "tcgen05-1cta": 3, "tcgen05-pairs": 4}[args.gemm_impl])
     others = []
-    modified = modified or args.gemm_impl != "auto" or args.grad_fp32
+    modified = modified or args.gemm_impl != "auto" or args.grad_fp32 or args.fused_update
     want_others = args.others == "on" or (args.others == "auto" and world == 1 and args.workload == "c4" and not modified and not shard)
     if want_others and world == 1:
         for key, over, nsteps in OTHER_WORKLOADS:

@@ -71,8 +71,12 @@ enum {
   LSAM_FLAG_CUDA_GRAPH = 4, /* replay each tick as one CUDA graph launch (recorded at the second tick of each variant;
                               for launch-bound small models); needs a non-default stream (lsam_init fails with
                               LSAM_ERR_INVALID otherwise); ignored while profiling is enabled               */
-  LSAM_FLAG_GRAD_FP32 = 8   /* tensor-core path: store g1 and g2 in fp32 instead of bf16 (4 instead of 2 bytes per
+  LSAM_FLAG_GRAD_FP32 = 8,  /* tensor-core path: store g1 and g2 in fp32 instead of bf16 (4 instead of 2 bytes per
                               element written by the weight-gradient GEMM and read back by perturbation and update) */
+  LSAM_FLAG_FUSED_UPDATE = 16 /* tensor-core path: apply the worker update of the weights inside the epilogue of the descent-pass
+                              weight-gradient GEMM, so that the descent gradient of the weights never reaches memory (biases keep
+                              the streaming update kernel).  Needs the tensor-core path, noise_temp = 0, dp_average = 0 and no
+                              LSAM_FLAG_CUDA_GRAPH (lsam_init: LSAM_ERR_INVALID otherwise); lsam_read_grads(2) is then unavailable */
 };
 
 /* Models.

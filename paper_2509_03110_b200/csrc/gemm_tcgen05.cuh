@@ -17,8 +17,8 @@
 // HALF of the N side of B; one thread of the leader CTA (cluster rank 0) issues tcgen05.mma.cta_group::2 with M = 256,
 // which reads the two halves of B from both CTAs' shared memory and leaves rows 0-127 of the tile in the leader's tensor
 // memory and rows 128-255 in the peer's.  A CTA so takes in a third fewer operand bytes per flop (the bound of the
-// single-CTA form is the rate at which an SM can fill its shared memory).  Each CTA issues its own TMA loads (no load is
-// multicast); the loads of both CTAs complete on the leader's `full` barrier, the leader's tcgen05.commit arrives on the
+// single-CTA form is the rate at which an SM can fill its shared memory).  Each CTA issues its own TMA loads, each into
+// its own shared memory only; the loads of both CTAs complete on the leader's `full` barrier, the leader's tcgen05.commit arrives on the
 // `empty` / `acc_full` barriers of both CTAs, and both CTAs' epilogue warps arrive on the leader's `acc_empty` barrier.
 //
 // All waits on mbarriers are bounded: when one expires the CTA raises STATUS_TIMEOUT, stops issuing work, lets the
@@ -89,7 +89,7 @@ __device__ inline void tma_load_3d(void* dst, const CUtensorMap* map, int c0, in
 }
 
 // The same load issued by a CTA of a pair: data into this CTA's shared memory, completion counted on a barrier given by its
-// shared::cluster address (the leader's `full` barrier, possibly in the peer CTA).  Not a multicast: one CTA, one destination.
+// shared::cluster address (the leader's `full` barrier, possibly in the peer CTA).  The data go to the issuing CTA alone.
 __device__ inline void tma_load_3d_pair(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint32_t bar_cluster_addr) {
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
@@ -211,7 +211,10 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, bool a_mn, bool 
 // ------------------------------------------------------------------------------------------------ epilogue parameters
 // TC_EPI_WGRAD_BF16: the weight gradient is stored rounded to bf16 (ascent pass: it only feeds the perturbation, whose
 // result is rounded to bf16 anyway; its norm is still taken from the fp32 accumulators).
-enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3, TC_EPI_WGRAD_BF16 = 4 };
+// TC_EPI_WGRAD_UPD: the descent-pass weight gradient with the worker update (S6) applied in the epilogue: the gradient block
+// goes from tensor memory through the warp's staging buffer straight into G = g2 + lambda (x - y), v <- mu v + G,
+// x <- x - eta (G + mu v) on the weights of the tile, and never reaches global memory.
+enum : int { TC_EPI_FWD_HIDDEN = 0, TC_EPI_FWD_HEAD = 1, TC_EPI_DGRAD = 2, TC_EPI_WGRAD = 3, TC_EPI_WGRAD_BF16 = 4, TC_EPI_WGRAD_UPD = 5 };
 __host__ __device__ constexpr bool tc_epi_is_wgrad(int e) { return e >= TC_EPI_WGRAD; }
 
 struct TcEpi {
@@ -226,6 +229,10 @@ struct TcEpi {
   float* partial;  int64_t ld_partial;  int slot0;
   int ldb;  // sample stride of the feature-major buffers (multiple of 16)
   int run_n;  // A-stationary weight gradient: consecutive n-tiles per unit of the work list (>= 1)
+  // TC_EPI_WGRAD_UPD: worker state rows (same addressing as g: [z * ld_g + w_off + m * ldw + n]), centre ring and the ring slot
+  // each replica reads, the bf16 operand copy, and the step's scalars (lam_k nullable: per-replica pull weight instead of lambda)
+  float* upd_x;  float* upd_v;  const float* upd_yring;  const int32_t* upd_slot;  bf16* upd_xop;  const float* upd_lam_k;
+  float upd_eta, upd_mu, upd_lambda;  int upd_nesterov;
   // dgrad, optional (bias_g != nullptr; needs the whole minibatch in one N tile): the bias gradient of the layer below,
   // db[m] = sum_b dz_prev[m][b], written to bias_g[z * bias_ld + bias_off + m] (bf16 if bias_bf16, else fp32), and the sum
   // of squares of every 8 consecutive db to partial[z * ld_partial + bias_slot0 + m / 8]
@@ -493,7 +500,63 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         tc::tmem_ld32(taddr + (uint32_t)(c * 32), r);
         tc::tmem_ld_wait();
         const int nb = n0 + c * 32;
-        if (EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) {
+        if (EPI == TC_EPI_WGRAD_UPD) {
+          const int mrow0 = m_base + quad * 32;
+          if (mrow0 < M && nb < N) {  // warp-uniform
+#pragma unroll
+            for (int j = 0; j < 32; ++j) ssq4[j & 3] = fmaf(__uint_as_float(r[j]), __uint_as_float(r[j]), ssq4[j & 3]);  // zero-filled edges add 0
+            // transpose through the warp's staging buffer: written row = lane (swizzled 16-byte chunks), read back so that
+            // 8 lanes cover the 128 contiguous bytes of a row and every global access below is coalesced
+            uint8_t* sb = stage + ew * 4096;
+            __syncwarp();  // the reads of the previous block are done
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              *reinterpret_cast<float4*>(sb + lane * 128 + ((q ^ (lane & 7)) << 4)) =
+                  make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]), __uint_as_float(r[4 * q + 3]));
+            __syncwarp();
+            const int64_t base = (int64_t)z * ep.ld_g + ep.w_off;
+            const float* yb = ep.upd_yring + (int64_t)ep.upd_slot[z] * ep.ld_g + ep.w_off;
+            const float lam = ep.upd_lam_k != nullptr ? ep.upd_lam_k[z] : ep.upd_lambda;
+            const int cq = lane & 7, rsub = lane >> 3;
+#pragma unroll
+            for (int pass = 0; pass < 2; ++pass) {
+              float4 gv[4], xv[4], vv[4], yv[4];
+              int64_t off[4];
+              bool okv[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const int row = (pass * 4 + i) * 4 + rsub;
+                const int mm = mrow0 + row, nn = nb + 4 * cq;
+                okv[i] = mm < M && nn < N;  // rows are multiples of 8 elements long: a 4-element chunk is inside or outside as a whole
+                off[i] = (int64_t)mm * ep.ldw + nn;
+                gv[i] = *reinterpret_cast<const float4*>(sb + row * 128 + ((cq ^ (row & 7)) << 4));
+                if (okv[i]) {
+                  xv[i] = *reinterpret_cast<const float4*>(ep.upd_x + base + off[i]);
+                  vv[i] = *reinterpret_cast<const float4*>(ep.upd_v + base + off[i]);
+                  yv[i] = __ldg(reinterpret_cast<const float4*>(yb + off[i]));
+                }
+              }
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                if (!okv[i]) continue;
+                float G;
+#define LSAM_FUPD(c)                                                                  \
+  G = fmaf(lam, xv[i].c - yv[i].c, gv[i].c);                                          \
+  vv[i].c = fmaf(ep.upd_mu, vv[i].c, G);                                              \
+  xv[i].c = ep.upd_nesterov ? xv[i].c - ep.upd_eta * fmaf(ep.upd_mu, vv[i].c, G) : xv[i].c - ep.upd_eta * vv[i].c;
+                LSAM_FUPD(x) LSAM_FUPD(y) LSAM_FUPD(z) LSAM_FUPD(w)
+#undef LSAM_FUPD
+                *reinterpret_cast<float4*>(ep.upd_x + base + off[i]) = xv[i];
+                __stcs(reinterpret_cast<float4*>(ep.upd_v + base + off[i]), vv[i]);
+                __nv_bfloat162 lo = __floats2bfloat162_rn(xv[i].x, xv[i].y), hi = __floats2bfloat162_rn(xv[i].z, xv[i].w);
+                uint2 pk;
+                pk.x = *reinterpret_cast<uint32_t*>(&lo);
+                pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                *reinterpret_cast<uint2*>(ep.upd_xop + base + off[i]) = pk;
+              }
+            }
+          }
+        } else if (EPI == TC_EPI_WGRAD || EPI == TC_EPI_WGRAD_BF16) {
           // The warp's 32 x 32 fp32 block goes to shared memory in the 128-byte-swizzled layout of the output tensor
           // map (row = lane, 16-byte chunk q stored at position q ^ (row % 8)), then one TMA store writes it to the
           // gradient rows (clipped at the ragged edges).  Two buffers per warp: the store of a chunk overlaps the
@@ -961,6 +1024,17 @@ inline int tc_wgrad(TcPlan& P, int l, cudaStream_t stream, bool out_bf16) {
   TcGemm g = P.wgrad[l];
   g.map_c = g.map_c16;
   return tc_launch<false, false, TC_EPI_WGRAD_BF16>(P, g, stream);
+}
+// Descent-pass weight gradient of layer l with the worker update applied to the layer's weights in the epilogue.
+struct TcFusedUpdate {
+  float* x; float* v; const float* yring; const int32_t* slot; bf16* xop; const float* lam_k;
+  float eta, mu, lambda; int nesterov;
+};
+inline int tc_wgrad_update(TcPlan& P, int l, cudaStream_t stream, const TcFusedUpdate& u) {
+  TcGemm g = P.wgrad[l];
+  g.ep.upd_x = u.x; g.ep.upd_v = u.v; g.ep.upd_yring = u.yring; g.ep.upd_slot = u.slot; g.ep.upd_xop = u.xop; g.ep.upd_lam_k = u.lam_k;
+  g.ep.upd_eta = u.eta; g.ep.upd_mu = u.mu; g.ep.upd_lambda = u.lambda; g.ep.upd_nesterov = u.nesterov;
+  return tc_launch<false, false, TC_EPI_WGRAD_UPD>(P, g, stream);
 }
 // The dgrad of layer l can also deliver the bias gradient of layer l - 1 (row sums of the backward signal it writes) when the
 // whole minibatch sits in one N tile; bias_g = destination buffer ([Z, ld] gradient rows, bf16 or fp32), nullptr = not fused.

@@ -197,6 +197,7 @@ struct lsam_ctx {
   int64_t ver_lo = 0, ver_hi = 0;
   int device = 0;                     // ordinal of the GPU that holds the workspace
   bool grads_bf16 = false;            // tensor-core path with its gradients stored in bf16
+  bool fused_update = false;          // LSAM_FLAG_FUSED_UPDATE: weights updated inside the descent-pass weight-gradient epilogue
   bool have_prev = false;
   bool use_tc = false;
   bool async_on = false;              // 0 < active_num < 256: unequal worker progress
@@ -428,6 +429,28 @@ int launch_update(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n
   return LSAM_OK;
 }
 
+// The fused update on the parameters [off, off + n) of every row only (off and n multiples of 64: one padded segment)
+int launch_update_range(lsam_ctx* c, int64_t off, int64_t n, float eta) {
+  const bool bfg = c->grads_bf16;
+  const void* g = bfg ? (const void*)(c->at<bf16>(c->L.g1b) + off) : (const void*)(c->g() + off);
+  UpdateArgs a = make_update_args(c, g, bfg ? 2 : 0, c->L.ld, n, eta);
+  a.x += off; a.v += off; a.yring += off; a.acc += off;
+  a.xop = c->cfg.gemm_dtype == LSAM_GEMM_BF16 ? (void*)(c->at<bf16>(c->L.xop) + off) : (void*)(c->at<float>(c->L.xop) + off);
+  const bool nes = c->cfg.nesterov != 0;
+  void* f;
+  unsigned grid;
+  if (bfg) {
+    grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * 8);
+    f = nes ? (void*)update8_kernel<true, false> : (void*)update8_kernel<false, false>;
+  } else {
+    grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * 4);
+    f = nes ? update_func<4, true, bf16, true>(false) : update_func<4, false, bf16, true>(false);
+  }
+  void* ptrs[1] = {&a};
+  LAUNCH(c, LSAM_PROF_UPDATE, cudaLaunchKernel((const void*)f, dim3(grid), dim3(kUpdThreads), ptrs, 0, c->stream));
+  return LSAM_OK;
+}
+
 SchedArgs make_sched_args(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot, int64_t budget, int32_t* active) {
   SchedArgs a;
   for (int s = 0; s < 16; ++s) {
@@ -483,8 +506,10 @@ int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N
 
 // One gradient pass of the classifier at the parameters P ([K, ld], type T); gradient -> g, loss -> loss_out (nullable).
 // g_bf16 (tensor-core path only): store the gradient rounded to bf16 in the g1b buffer instead of fp32 in g.
+// fu != nullptr (tensor-core path, descent pass): the weight gradient of every layer is consumed by the worker update in its own
+// epilogue instead of being stored; the dgrad of a layer, which still reads the perturbed weights, then runs BEFORE that layer's wgrad.
 template <typename T>
-int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
+int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFusedUpdate* fu = nullptr) {
   const Layout& L = c->L;
   const int K = c->cfg.K, B = c->cfg.batch;
   const int nl = (int)L.layers.size();
@@ -546,11 +571,19 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
     }
     if (c->use_tc) {
       int trc = 0;
-      LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream, g_bf16));
-      if (trc == 0 && l > 0) {
+      auto dgrad = [&]() -> int {
+        if (l == 0) return LSAM_OK;
         void* bias_g = nullptr;
         if (tc_dgrad_can_fuse_bias(c->tc, l)) bias_g = g_bf16 ? (void*)c->at<bf16>(L.g1b) : (void*)c->g();
         LAUNCH(c, LSAM_PROF_GEMM_DGRAD, trc = tc_dgrad(c->tc, l, c->stream, bias_g, g_bf16));
+        return LSAM_OK;
+      };
+      if (fu != nullptr) {
+        if ((rc = dgrad()) != LSAM_OK) return rc;
+        if (trc == 0) LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad_update(c->tc, l, c->stream, *fu));
+      } else {
+        LAUNCH(c, LSAM_PROF_GEMM_WGRAD, trc = tc_wgrad(c->tc, l, c->stream, g_bf16));
+        if (trc == 0 && (rc = dgrad()) != LSAM_OK) return rc;
       }
       if (trc != 0) return c->fail(LSAM_ERR_CUDA, "tcgen05 backward launch failed");
       cur ^= 1;
@@ -578,7 +611,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16) {
 }
 
 // Gradient of the minibatch loss at the parameters held in `params` (x master, or the operand buffer).
-int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false) {
+int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false, const TcFusedUpdate* fu = nullptr) {
   const lsam_config& cfg = c->cfg;
   if (cfg.model == LSAM_MODEL_LSQ) {
     const float* P = perturbed ? c->at<float>(c->L.xop) : c->x();
@@ -586,7 +619,7 @@ int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false)
         c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, cfg.widths[0], c->g(), c->L.ld, loss_out, c->act()));
     return LSAM_OK;
   }
-  if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out, g_bf16 && c->use_tc);
+  if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out, g_bf16 && c->use_tc, c->use_tc ? fu : nullptr);
   return mlp_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out, false);
 }
 
@@ -712,6 +745,23 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   if (L.xpkeep) LSAM_CUDA(c, cudaMemcpyAsync(c->at<bf16>(L.xpkeep), c->at<bf16>(L.xop), sizeof(bf16) * cfg.K * L.ld, cudaMemcpyDeviceToDevice, c->stream));
   // descent gradient at the perturbed point, same minibatch
   phase.next("lsam S5 descent gradient");
+  if (c->fused_update) {
+    // weights: updated inside the weight-gradient epilogues of this pass; the pull weights of a non-Gaussian kernel are
+    // distances of the iterates BEFORE the update, so they are taken first
+    if (other_kernel && (rc = launch_pull_weights(c)) != LSAM_OK) return rc;
+    TcFusedUpdate fu{c->x(), c->v(), c->at<float>(L.yring), c->slot(), c->at<bf16>(L.xop), other_kernel ? c->pull_weight() : nullptr,
+                     eta, cfg.mu, cfg.lambda, cfg.nesterov != 0 ? 1 : 0};
+    if ((rc = grad_pass(c, true, nullptr, gb, &fu)) != LSAM_OK) return rc;
+    phase.next("lsam S6 update (biases, iterate sums)");
+    if (cfg.flags & LSAM_FLAG_STEP_INFO)
+      if ((rc = launch_norm(c, nullptr, ldg, n, vec4, 0.f, c->norm2(), nullptr)) != LSAM_OK) return rc;
+    for (const LayerInfo& li : L.layers) {
+      const int64_t wlen = round_up((int64_t)li.in * li.out, kSegAlign), blen = round_up((int64_t)li.out, kSegAlign);
+      if ((rc = launch_update_range(c, li.b_pad, blen, eta)) != LSAM_OK) return rc;  // bias gradients were stored as usual
+      LAUNCH(c, LSAM_PROF_UPDATE, acc_add_kernel<<<(unsigned)ceil_div(wlen, 1024), 256, 0, c->stream>>>(c->x(), L.ld, cfg.K, li.w_pad, wlen, c->at<float>(L.acc), c->act()));
+    }
+    return LSAM_OK;
+  }
   if (!flat && (rc = grad_pass(c, true, nullptr, gb)) != LSAM_OK) return rc;
   phase.next("lsam S6 update");
   return finish_tick(gptr);
@@ -873,6 +923,10 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   if (cfg->gemm_impl >= LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
   c->use_tc = tc_ok;
   c->grads_bf16 = tc_ok && !(cfg->flags & LSAM_FLAG_GRAD_FP32);
+  if (cfg->flags & LSAM_FLAG_FUSED_UPDATE) {
+    if (!tc_ok || cfg->noise_temp > 0.f || cfg->dp_average != 0 || (cfg->flags & LSAM_FLAG_CUDA_GRAPH)) return bail(LSAM_ERR_INVALID);
+    c->fused_update = true;
+  }
   {
     // the device that holds the workspace is the context's device; it has to be the current one here and in every later call
     cudaPointerAttributes pa;
@@ -1124,6 +1178,7 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
       LSAM_CUDA(c, cudaMemcpyAsync(tmp, src + (size_t)k * L.d, sizeof(float) * L.d, cudaMemcpyDeviceToDevice, c->stream));
     } else {
       if (pass == 1 && !L.g1keep) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(1) needs LSAM_FLAG_KEEP_G1");
+      if (pass == 2 && c->fused_update) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(2): with LSAM_FLAG_FUSED_UPDATE the descent gradient of the weights is never stored");
       if (c->grads_bf16) {  // both gradients are stored as bf16
         const bf16* srcb = pass == 1 ? c->at<bf16>(L.g1keep) : c->at<bf16>(L.g1b);
         int64_t maxlen = 0;

@@ -625,6 +625,24 @@ __global__ void __launch_bounds__(kUpdThreads) update8f_kernel(const UpdateArgs 
   }
 }
 
+// Iterate accumulation on its own (for the parameters whose update ran in a weight-gradient epilogue): acc[j] += sum over the
+// replicas that stepped, k ascending, of x[k][j], j in [off, off + n); one thread per 4 consecutive columns.
+__global__ void __launch_bounds__(256)
+acc_add_kernel(const float* __restrict__ x, int64_t ld, int K, int64_t off, int64_t n, float* __restrict__ acc,
+               const int32_t* __restrict__ active) {
+  const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
+  if (j >= n) return;
+  float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int k = 0; k < K; ++k) {
+    if (active != nullptr && !active[k]) continue;
+    const float4 v = *reinterpret_cast<const float4*>(x + (int64_t)k * ld + off + j);
+    s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+  }
+  float4 a = *reinterpret_cast<const float4*>(acc + off + j);
+  a.x += s.x; a.y += s.y; a.z += s.z; a.w += s.w;
+  *reinterpret_cast<float4*>(acc + off + j) = a;
+}
+
 // ------------------------------------------------------------------------------------------------ S7 centre update
 //   g' = acc / (K tau) - y;  g = have_prev ? g' + beta (g' - g'_prev) : g';  y_new = y + eta' g;
 //   g'_prev <- g';  acc <- 0.       (sync branch of Algorithm 2 with the look-ahead of Section 4.2)

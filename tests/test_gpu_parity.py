@@ -289,6 +289,54 @@ def test_gradient_storage_fp32_on_the_tensor_core_path_matches_oracle_and_bf16_s
     np.testing.assert_array_equal(runs["fp32"][2][1], runs["bf16"][2][1])
 
 
+@pytest.mark.parametrize("model,widths,K,B,extra", [
+    (G.MODEL_RESMLP, (128, 256, 256, 40), 2, 300, {}),                       # two N tiles in the forward pass, residual layers, ragged head
+    (G.MODEL_MLP, (320, 520, 24), 3, 40, dict(active_num=170)),              # ragged tiles, unequal worker progress
+    (G.MODEL_RESMLP, (192, 640, 640, 300), 3, 256, dict(kernel_kind=G.KERNEL_CAUCHY, kernel_param=0.7)),  # CTA pairs in forward / dgrad, non-Gaussian pull
+])
+def test_fused_update_in_the_weight_gradient_epilogue_matches_oracle(model, widths, K, B, extra):
+    # LSAM_FLAG_FUSED_UPDATE: the descent gradient of the weights goes from the accumulators straight into the worker update;
+    # same arithmetic as the oracle's (gradient unrounded), stale centre reads, syncs, iterate sums included
+    hp = dict(tau=3, lam=0.4, seed=4, stale_max=2, **extra)
+    X, labels = synth.gaussian_mixture(400, widths[0], widths[-1], seed=4)
+    w0 = synth.mlp_init(widths, seed=4)
+    p = Pair(model, widths=widths, K=K, batch=B, X=X, Y=labels, x0=synth.replicate(w0, K, jitter=0.01, seed=4), y0=w0, gemm_dtype=G.GEMM_BF16,
+             gemm_impl=G.IMPL_TCGEN05, flags=G.FLAG_FUSED_UPDATE | G.FLAG_STEP_INFO, **hp)
+    assert p.gpu.uses_tcgen05()
+    with pytest.raises(G.LsamError):
+        p.gpu.read_grads(2)
+    for t in range(3):
+        p.teacher_force()
+        p.step(0.05, 0.1)
+        e = p.errors()
+        acc = e.pop("acc")
+        _assert_all(e, TOL_STEP_BF16, f"fused update forced step {t}")
+        assert acc <= TOL_STEP_BF16
+        _, on1, on2 = p.oracle.read_step_info()
+        _, gn1, gn2 = p.gpu.read_step_info()
+        act = p.oracle.read_active().astype(bool)
+        np.testing.assert_allclose(gn2[act], on2[act], rtol=TOL_STEP_BF16)
+        p.couple_if_due()
+    p.teacher_force()
+    for t in range(14):
+        p.step(0.05, 0.1 if t != 5 else 0.0)  # one tick through the single-pass shortcut
+        p.couple_if_due()
+    e = p.errors()
+    e.pop("acc"), e.pop("v")
+    e["v_scaled"] = p.momentum_error()
+    _assert_all(e, TOL_TRAJ_BF16, "fused update trajectory")
+    assert p.gpu.status() == 0 and p.gpu.counters()[1] >= 3
+    p.close()
+    # not available off the tensor-core path, with noise, or with graph replay
+    for bad in (dict(gemm_impl=G.IMPL_SIMT), dict(noise_temp=0.1), dict(dp_average=1)):
+        import torch
+        kw = dict(widths=widths, K=K, batch=B, n_samples=400, gemm_dtype=G.GEMM_BF16, flags=G.FLAG_FUSED_UPDATE, tau=3)
+        kw.update(bad)
+        with pytest.raises(G.LsamError):
+            G.Lsam(G.make_config(model, **kw), torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda(),
+                   torch.from_numpy(synth.replicate(w0, K)).cuda(), torch.from_numpy(w0).cuda())
+
+
 def test_step_batch_matches_gathered_step():
     # the caller-supplied minibatch path (host buffers) must reproduce the resident-dataset path exactly
     import torch
