@@ -15,7 +15,7 @@ _SRC = os.path.join(_HERE, "lsam_oracle.cpp")
 _HDR = os.path.join(_HERE, "lsam_oracle.h")
 _LIB = os.path.join(_HERE, "liblsam_oracle.so")
 
-MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT = 0, 1, 2, 3
+MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT, MODEL_CNN = 0, 1, 2, 3, 4
 GEMM_FP32, GEMM_BF16 = 0, 1
 KERNEL_GAUSSIAN, KERNEL_EXP_POWER, KERNEL_CAUCHY, KERNEL_MATERN32 = 0, 1, 2, 3
 
@@ -38,6 +38,7 @@ class OracleConfig(C.Structure):
         ("seed", C.c_uint64), ("mu", C.c_double), ("gamma", C.c_double), ("lam", C.c_double),
         ("beta", C.c_double), ("eta_prime", C.c_double), ("noise_temp", C.c_double),
         ("kernel_kind", C.c_int32), ("dp_average", C.c_int32), ("kernel_param", C.c_double),
+        ("n_conv", C.c_int32), ("img_h", C.c_int32), ("img_w", C.c_int32),
     ]
 
 
@@ -98,12 +99,12 @@ def lib():
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, nesterov=1, gamma=1e-12,
                 lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, active_num=256, noise_temp=0.0,
-                kernel_kind=KERNEL_GAUSSIAN, kernel_param=0.0, dp_average=0):
+                kernel_kind=KERNEL_GAUSSIAN, kernel_param=0.0, dp_average=0, n_conv=0, img_h=0, img_w=0):
     """Float hyper-parameters are taken at their fp32 value, the precision the C-ABI carries them in."""
     c = OracleConfig()
     c.model = model
     widths = list(widths)
-    c.n_layers = max(len(widths) - 1, 0) if model in (MODEL_MLP, MODEL_RESMLP) else (1 if model == MODEL_LSQ else 0)
+    c.n_layers = max(len(widths) - 1, 0) if model in (MODEL_MLP, MODEL_RESMLP, MODEL_CNN) else (1 if model == MODEL_LSQ else 0)
     for i, w in enumerate(widths):
         c.widths[i] = int(w)
     c.K, c.batch, c.gemm_dtype, c.nesterov, c.tau = int(K), int(batch), int(gemm_dtype), int(nesterov), int(tau)
@@ -113,6 +114,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, mu=0.9, ne
     c.mu, c.gamma, c.lam, c.beta, c.eta_prime = f32(mu), f32(gamma), f32(lam), f32(beta), f32(eta_prime)
     c.noise_temp = f32(noise_temp)
     c.kernel_kind, c.kernel_param, c.dp_average = int(kernel_kind), f32(kernel_param), int(dp_average)
+    c.n_conv, c.img_h, c.img_w = int(n_conv), int(img_h), int(img_w)
     return c
 
 

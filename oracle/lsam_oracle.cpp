@@ -108,6 +108,9 @@ struct Layer {
   int in, out;
   int64_t w_off, b_off;  // offsets in the unpadded parameter vector; b_off = -1: no bias
   bool residual;         // h_next = h + relu(W h + b)
+  // convolution layer: 3x3, stride 1, zero padding 1, ReLU, then 2x2 max-pooling; in = Cin H W, out = Cout (H/2) (W/2)
+  bool conv = false;
+  int Cin = 0, Cout = 0, H = 0, W = 0;
 };
 
 struct Net {
@@ -138,14 +141,31 @@ bool build_net(const oracle_config& c, Net& net) {
     net.d = c.widths[0];
     return true;
   }
-  if (c.model != ORACLE_MODEL_MLP && c.model != ORACLE_MODEL_RESMLP) return false;
+  if (c.model != ORACLE_MODEL_MLP && c.model != ORACLE_MODEL_RESMLP && c.model != ORACLE_MODEL_CNN) return false;
   if (c.n_layers < 1 || c.n_layers > 8) return false;
+  const bool cnn = c.model == ORACLE_MODEL_CNN;
+  if (cnn && (c.n_conv < 1 || c.n_conv >= c.n_layers || c.img_h < 1 || c.img_w < 1 || c.img_h % (1 << c.n_conv) || c.img_w % (1 << c.n_conv))) return false;
   int64_t off = 0;
+  int H = c.img_h, W = c.img_w;
   for (int l = 0; l < c.n_layers; ++l) {
     Layer L;
-    L.in = c.widths[l];
+    if (c.widths[l] < 1 || c.widths[l + 1] < 1) return false;
+    if (cnn && l < c.n_conv) {
+      L.conv = true;
+      L.Cin = c.widths[l]; L.Cout = c.widths[l + 1]; L.H = H; L.W = W;
+      L.in = L.Cin * H * W;
+      H /= 2; W /= 2;
+      L.out = L.Cout * H * W;
+      L.w_off = off;
+      off += (int64_t)L.Cout * L.Cin * 9;
+      L.b_off = off;
+      off += L.Cout;
+      L.residual = false;
+      net.layers.push_back(L);
+      continue;
+    }
+    L.in = (cnn && l == c.n_conv) ? net.layers.back().out : c.widths[l];  // the first dense layer takes the flattened feature maps
     L.out = c.widths[l + 1];
-    if (L.in < 1 || L.out < 1) return false;
     L.w_off = off;
     off += (int64_t)L.in * L.out;
     L.b_off = off;
@@ -155,8 +175,32 @@ bool build_net(const oracle_config& c, Net& net) {
     net.layers.push_back(L);
   }
   net.d = off;
-  net.in0 = c.widths[0];
+  net.in0 = net.layers[0].in;
   return true;
+}
+
+// Gradient w.r.t. the pre-activation of a hidden layer from the gradient dh w.r.t. its output: dense layers pass it where the
+// ReLU was active; a convolution layer routes each pooled gradient to the element of its 2x2 window that was the maximum,
+// if that element's ReLU was active ([B][Cout][H][W] from [B][Cout][H/2][W/2]).
+std::vector<double> unpool_or_mask(const Layer& lp, const std::vector<double>& dh, const std::vector<unsigned char>& mask,
+                                   const std::vector<unsigned char>& arg, int B) {
+  if (!lp.conv) {
+    std::vector<double> dz((size_t)B * lp.out);
+    for (size_t e = 0; e < dz.size(); ++e) dz[e] = mask[e] ? dh[e] : 0.0;
+    return dz;
+  }
+  const int Hh = lp.H, Ww = lp.W, Ho = Hh / 2, Wo = Ww / 2;
+  std::vector<double> dz((size_t)B * lp.Cout * Hh * Ww, 0.0);
+  for (int b = 0; b < B; ++b)
+    for (int co = 0; co < lp.Cout; ++co)
+      for (int y = 0; y < Ho; ++y)
+        for (int x = 0; x < Wo; ++x) {
+          const size_t e = (size_t)b * lp.out + ((size_t)co * Ho + y) * Wo + x;
+          const int a = arg[e];
+          const size_t f = (size_t)b * lp.Cout * Hh * Ww + ((size_t)co * Hh + 2 * y + (a >> 1)) * Ww + 2 * x + (a & 1);
+          if (mask[f]) dz[f] = dh[e];
+        }
+  return dz;
 }
 
 // Mean loss over the minibatch and its gradient.  a0: [B, in0] inputs (already rounded in bf16 mode).
@@ -192,12 +236,56 @@ double net_loss_grad(const Net& net, const double* params, const std::vector<dou
 
   // ---- forward
   std::vector<std::vector<double>> h(L + 1);       // h[l]: input of layer l, [B, in_l]
-  std::vector<std::vector<unsigned char>> mask(L);  // mask[l][b*out+o] = (pre-activation > 0), hidden layers
+  std::vector<std::vector<unsigned char>> mask(L);  // mask[l][b*out+o] = (pre-activation > 0), hidden layers (convolutions: before pooling)
+  std::vector<std::vector<unsigned char>> pool_arg(L);  // convolutions: which element of its 2x2 window each pooled output took
   h[0] = a0;
   std::vector<double> logits;
   for (int l = 0; l < L; ++l) {
     const Layer& ly = net.layers[l];
     const bool head = (l == L - 1);
+    if (ly.conv) {
+      // z[b][co][y][x] = bias[co] + sum_{ci,kh,kw} W[co][ci*9 + kh*3 + kw] a[b][ci][y+kh-1][x+kw-1]  (zero outside the image);
+      // r = relu(z); pooled[b][co][y/2][x/2] = max of the 2x2 window (first maximum in row-major order)
+      const int Hh = ly.H, Ww = ly.W, Ho = Hh / 2, Wo = Ww / 2;
+      std::vector<double> r((size_t)B * ly.Cout * Hh * Ww);
+      mask[l].assign(r.size(), 0);
+      for (int b = 0; b < B; ++b)
+        for (int co = 0; co < ly.Cout; ++co)
+          for (int y = 0; y < Hh; ++y)
+            for (int x = 0; x < Ww; ++x) {
+              double s = 0.0;
+              for (int ci = 0; ci < ly.Cin; ++ci)
+                for (int kh = 0; kh < 3; ++kh)
+                  for (int kw = 0; kw < 3; ++kw) {
+                    const int yy = y + kh - 1, xx = x + kw - 1;
+                    if (yy < 0 || yy >= Hh || xx < 0 || xx >= Ww) continue;
+                    s += pq[(size_t)(ly.w_off + (int64_t)co * ly.Cin * 9 + ci * 9 + kh * 3 + kw)] *
+                         h[l][(size_t)b * ly.in + ((size_t)ci * Hh + yy) * Ww + xx];
+                  }
+              s += pq[(size_t)(ly.b_off + co)];
+              const size_t e = (size_t)b * ly.Cout * Hh * Ww + ((size_t)co * Hh + y) * Ww + x;
+              mask[l][e] = s > 0.0;
+              r[e] = s > 0.0 ? s : 0.0;
+            }
+      h[l + 1].resize((size_t)B * ly.out);
+      pool_arg[l].assign((size_t)B * ly.out, 0);
+      for (int b = 0; b < B; ++b)
+        for (int co = 0; co < ly.Cout; ++co)
+          for (int y = 0; y < Ho; ++y)
+            for (int x = 0; x < Wo; ++x) {
+              double best = -1.0;
+              int arg = 0;
+              for (int dy = 0; dy < 2; ++dy)
+                for (int dx = 0; dx < 2; ++dx) {
+                  const double v = r[(size_t)b * ly.Cout * Hh * Ww + ((size_t)co * Hh + 2 * y + dy) * Ww + 2 * x + dx];
+                  if (v > best) { best = v; arg = dy * 2 + dx; }
+                }
+              const size_t e = (size_t)b * ly.out + ((size_t)co * Ho + y) * Wo + x;
+              h[l + 1][e] = net.q(best);  // stored activation (bf16 mode: rounded)
+              pool_arg[l][e] = (unsigned char)arg;
+            }
+      continue;
+    }
     std::vector<double> z((size_t)B * ly.out);
     for (int b = 0; b < B; ++b)
       for (int o = 0; o < ly.out; ++o) {
@@ -248,6 +336,53 @@ double net_loss_grad(const Net& net, const double* params, const std::vector<dou
   std::vector<double> dh_next;  // gradient w.r.t. h[l+1] (needed by residual layers)
   for (int l = L - 1; l >= 0; --l) {
     const Layer& ly = net.layers[l];
+    if (ly.conv) {
+      // dz here: gradient w.r.t. the convolution's pre-activation, [B][Cout][H][W]
+      const int Hh = ly.H, Ww = ly.W;
+      const size_t plane = (size_t)Hh * Ww;
+      for (int co = 0; co < ly.Cout; ++co) {
+        double sb = 0.0;
+        for (int b = 0; b < B; ++b)
+          for (size_t e = 0; e < plane; ++e) sb += dz[((size_t)b * ly.Cout + co) * plane + e];
+        grad[ly.b_off + co] = sb;
+        for (int ci = 0; ci < ly.Cin; ++ci)
+          for (int kh = 0; kh < 3; ++kh)
+            for (int kw = 0; kw < 3; ++kw) {
+              double s = 0.0;  // samples, then rows, then columns, ascending
+              for (int b = 0; b < B; ++b)
+                for (int y = 0; y < Hh; ++y) {
+                  const int yy = y + kh - 1;
+                  if (yy < 0 || yy >= Hh) continue;
+                  for (int x = 0; x < Ww; ++x) {
+                    const int xx = x + kw - 1;
+                    if (xx < 0 || xx >= Ww) continue;
+                    s += dz[((size_t)b * ly.Cout + co) * plane + (size_t)y * Ww + x] * h[l][(size_t)b * ly.in + ((size_t)ci * Hh + yy) * Ww + xx];
+                  }
+                }
+              grad[ly.w_off + (int64_t)co * ly.Cin * 9 + ci * 9 + kh * 3 + kw] = s;
+            }
+      }
+      if (l == 0) break;
+      // gradient w.r.t. the layer's input: dh[b][ci][yy][xx] = sum_{co,kh,kw} dz[b][co][yy-kh+1][xx-kw+1] W[co][ci*9+kh*3+kw]
+      std::vector<double> dh((size_t)B * ly.in, 0.0);
+      for (int b = 0; b < B; ++b)
+        for (int ci = 0; ci < ly.Cin; ++ci)
+          for (int yy = 0; yy < Hh; ++yy)
+            for (int xx = 0; xx < Ww; ++xx) {
+              double s = 0.0;
+              for (int co = 0; co < ly.Cout; ++co)
+                for (int kh = 0; kh < 3; ++kh)
+                  for (int kw = 0; kw < 3; ++kw) {
+                    const int y = yy - kh + 1, x = xx - kw + 1;
+                    if (y < 0 || y >= Hh || x < 0 || x >= Ww) continue;
+                    s += dz[((size_t)b * ly.Cout + co) * plane + (size_t)y * Ww + x] * pq[(size_t)(ly.w_off + (int64_t)co * ly.Cin * 9 + ci * 9 + kh * 3 + kw)];
+                  }
+              dh[(size_t)b * ly.in + ((size_t)ci * Hh + yy) * Ww + xx] = net.q(s);
+            }
+      dz = unpool_or_mask(net.layers[l - 1], dh, mask[l - 1], pool_arg[l - 1], B);
+      dh_next.swap(dh);
+      continue;
+    }
     for (int o = 0; o < ly.out; ++o) {
       double sb = 0.0;
       for (int b = 0; b < B; ++b) sb += dz[(size_t)b * ly.out + o];
@@ -278,10 +413,7 @@ double net_loss_grad(const Net& net, const double* params, const std::vector<dou
       }
     }
     // pre-activation gradient of layer l-1 (always a hidden layer here)
-    const Layer& lp = net.layers[l - 1];
-    std::vector<double> dzp((size_t)B * lp.out);
-    for (size_t e = 0; e < dzp.size(); ++e) dzp[e] = mask[l - 1][e] ? dh[e] : 0.0;
-    dz.swap(dzp);
+    dz = unpool_or_mask(net.layers[l - 1], dh, mask[l - 1], pool_arg[l - 1], B);
     dh_next.swap(dh);
   }
   return loss;

@@ -28,7 +28,11 @@
 extern "C" {
 #endif
 
-enum { ORACLE_MODEL_LSQ = 0, ORACLE_MODEL_MLP = 1, ORACLE_MODEL_RESMLP = 2, ORACLE_MODEL_FLAT = 3 };
+/* CNN: n_conv layers of 3x3 convolution (stride 1, zero padding 1) + ReLU + 2x2 max-pooling, then dense layers as in MLP.
+ * widths = channels C0 .. C_nconv, then the dense widths (hidden..., classes); the input is img_h x img_w with C0 channels,
+ * a row of X holding it channel-major (feature = c * H * W + h * W + w, the flattening every later layer uses too).
+ * Parameters: conv W_l [Cout][Cin * 9] (column = ci * 9 + kh * 3 + kw) then b_l [Cout]; dense layers as in MLP. */
+enum { ORACLE_MODEL_LSQ = 0, ORACLE_MODEL_MLP = 1, ORACLE_MODEL_RESMLP = 2, ORACLE_MODEL_FLAT = 3, ORACLE_MODEL_CNN = 4 };
 enum { ORACLE_GEMM_FP32 = 0, ORACLE_GEMM_BF16 = 1 };
 /* Stationary kernels k(x, y) = phi(x - y) of Corollary 8 and the remark after it; see kernel_phi in the source. */
 enum { ORACLE_KERNEL_GAUSSIAN = 0, ORACLE_KERNEL_EXP_POWER = 1, ORACLE_KERNEL_CAUCHY = 2, ORACLE_KERNEL_MATERN32 = 3 };
@@ -57,6 +61,8 @@ typedef struct {
   int32_t dp_average;   /* 1: synchronous data parallelism (Section 5.2, DP-SGD / DP-SAM): both gradients of a tick
                            are averaged over the K workers before they are used; lock-step schedule only          */
   double kernel_param;  /* EXP_POWER: exponent a in [1, 2]; CAUCHY: scale s > 0; others: unused                   */
+  int32_t n_conv;       /* CNN: number of convolution layers (the first n_conv of the n_layers)                    */
+  int32_t img_h, img_w; /* CNN: input image size; both divisible by 2^n_conv                                       */
 } oracle_config;
 
 typedef struct oracle_ctx oracle_ctx;

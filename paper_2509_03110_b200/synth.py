@@ -47,6 +47,29 @@ def mlp_init(widths, seed=0):
     return np.concatenate(parts)
 
 
+def cnn_dense_in(channels, img_h, img_w):
+    """Features entering the first dense layer: the last channel count times the image size after one 2x2 pooling per convolution."""
+    n_conv = len(channels) - 1
+    return channels[-1] * (img_h >> n_conv) * (img_w >> n_conv)
+
+
+def cnn_param_count(channels, dense, img_h, img_w):
+    n = sum(channels[l + 1] * channels[l] * 9 + channels[l + 1] for l in range(len(channels) - 1))
+    return int(n + mlp_param_count([cnn_dense_in(channels, img_h, img_w)] + list(dense)))
+
+
+def cnn_init(channels, dense, img_h, img_w, seed=0):
+    """Flat vector of the convolutional model: per convolution W [Cout, Cin * 9] ~ N(0, 2 / (9 Cin)) then b = 0, then the dense layers as in mlp_init."""
+    rng = np.random.default_rng(seed + 15485863)
+    parts = []
+    for l in range(len(channels) - 1):
+        fan_in = channels[l] * 9
+        parts.append((rng.standard_normal((channels[l + 1], fan_in), dtype=np.float32) * np.float32(np.sqrt(2.0 / fan_in))).reshape(-1))
+        parts.append(np.zeros(channels[l + 1], dtype=np.float32))
+    parts.append(mlp_init([cnn_dense_in(channels, img_h, img_w)] + list(dense), seed=seed))
+    return np.concatenate(parts)
+
+
 def replicate(x, K, jitter=0.0, seed=0):
     """Stack one vector K times ([K, d]); jitter > 0 adds N(0, jitter^2) so that replicas start apart."""
     out = np.repeat(np.asarray(x, dtype=np.float32)[None, :], K, axis=0).copy()

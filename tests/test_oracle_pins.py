@@ -856,3 +856,92 @@ def test_dp_average_is_sam_on_the_union_of_the_workers_minibatches(model):
     # asynchronous progress contradicts the synchronous aggregation
     bad = O.make_config(O.MODEL_FLAT, K=2, flat_d=3, dp_average=1, active_num=100)
     assert not O.lib().oracle_create(O.C.byref(bad), None, None, O._ptr(np.zeros((2, 3))), O._ptr(np.zeros(3)), None)
+
+
+# ------------------------------------------------------------------------------------------- convolutional model
+def _torch_cnn_loss(channels, dense, H, W, params, Xb, yb):
+    """Independent statement of the convolutional model with torch's own conv2d / max_pool2d (double), loss and autograd gradient."""
+    import torch.nn.functional as F
+
+    p = torch.tensor(params, dtype=torch.float64, requires_grad=True)
+    x = torch.tensor(Xb, dtype=torch.float64).reshape(len(Xb), channels[0], H, W)
+    off = 0
+    for l in range(len(channels) - 1):
+        ci, co = channels[l], channels[l + 1]
+        Wt = p[off:off + co * ci * 9].reshape(co, ci, 3, 3)
+        off += co * ci * 9
+        b = p[off:off + co]
+        off += co
+        x = F.max_pool2d(F.relu(F.conv2d(x, Wt, b, stride=1, padding=1)), 2)
+    x = x.flatten(1)
+    widths = [x.shape[1]] + list(dense)
+    for l in range(len(widths) - 1):
+        Wl = p[off:off + widths[l] * widths[l + 1]].reshape(widths[l + 1], widths[l])
+        off += widths[l] * widths[l + 1]
+        b = p[off:off + widths[l + 1]]
+        off += widths[l + 1]
+        x = x @ Wl.T + b
+        if l < len(widths) - 2:
+            x = F.relu(x)
+    assert off == len(params)
+    loss = F.cross_entropy(x, torch.tensor(yb, dtype=torch.long))
+    loss.backward()
+    return float(loss.detach()), p.grad.numpy(), x.detach().numpy()
+
+
+@pytest.mark.parametrize("channels,dense,H,W", [((2, 3), (5, 4), 4, 6), ((3, 4, 5), (7, 3), 8, 8), ((1, 2, 2, 3), (3,), 8, 8)])
+def test_cnn_gradient_vs_torch_conv_autograd_and_finite_differences(channels, dense, H, W):
+    n, B = 30, 5
+    classes = dense[-1]
+    X, labels = synth.gaussian_mixture(n, channels[0] * H * W, classes, seed=3)
+    params = synth.cnn_init(channels, dense, H, W, seed=4).astype(np.float64)
+    params += 0.05 * np.random.default_rng(5).standard_normal(params.shape)  # nonzero biases
+    cfg = O.make_config(O.MODEL_CNN, widths=tuple(channels) + tuple(dense), K=1, batch=B, n_samples=n, n_conv=len(channels) - 1, img_h=H, img_w=W)
+    assert O.param_count(cfg) == synth.cnn_param_count(channels, dense, H, W) == len(params)
+    idx = np.array([3, 17, 0, 29, 11], dtype=np.int32)
+    loss, grad = O.loss_grad(cfg, X, labels, params, idx)
+    tl, tg, tlogits = _torch_cnn_loss(channels, dense, H, W, params, X[idx], labels[idx])
+    np.testing.assert_allclose(O.forward(cfg, X, params, idx), tlogits, rtol=1e-11, atol=1e-12)
+    assert abs(loss - tl) <= 1e-12 * abs(tl)
+    np.testing.assert_allclose(grad, tg, rtol=1e-9, atol=1e-13)
+    # central finite differences on a sample of coordinates of every parameter block
+    rng = np.random.default_rng(6)
+    for j in rng.choice(len(params), 25, replace=False):
+        h = 1e-6
+        pp, pm = params.copy(), params.copy()
+        pp[j] += h
+        pm[j] -= h
+        fd = (O.loss_grad(cfg, X, labels, pp, idx)[0] - O.loss_grad(cfg, X, labels, pm, idx)[0]) / (2 * h)
+        assert abs(fd - grad[j]) <= 1e-6 * max(1.0, abs(grad[j])), (j, fd, grad[j])
+    # bf16 mode: exact where every operand is representable (dyadic inputs and weights, one convolution), close otherwise
+    c16 = O.make_config(O.MODEL_CNN, widths=tuple(channels) + tuple(dense), K=1, batch=B, n_samples=n, n_conv=len(channels) - 1, img_h=H, img_w=W,
+                        gemm_dtype=O.GEMM_BF16)
+    l16, g16 = O.loss_grad(c16, X, labels, params, idx)
+    assert 0 < np.linalg.norm(g16 - grad) / np.linalg.norm(grad) < 5e-2 and abs(l16 - loss) < 5e-2 * abs(loss)
+    # invalid geometry is refused
+    assert O.param_count(O.make_config(O.MODEL_CNN, widths=(2, 3, 4), K=1, batch=1, n_conv=1, img_h=5, img_w=4)) == -1
+    assert O.param_count(O.make_config(O.MODEL_CNN, widths=(2, 3, 4), K=1, batch=1, n_conv=2, img_h=4, img_w=4)) == -1
+
+
+def test_cnn_step_runs_the_same_sam_step_as_the_other_models():
+    # the step itself is model-independent: with the convolutional model it equals the gradient-fed step driven by that model's gradients
+    channels, dense, H, W = (2, 3), (4, 3), 4, 4
+    n, B, K = 24, 6, 2
+    X, labels = synth.gaussian_mixture(n, channels[0] * H * W, 3, seed=8)
+    w0 = synth.cnn_init(channels, dense, H, W, seed=9).astype(np.float64)
+    xs = np.stack([w0, w0 + 0.01 * np.random.default_rng(1).standard_normal(w0.shape)])
+    kw = dict(K=K, lam=0.5, tau=2, seed=5)
+    geo = dict(widths=channels + dense, n_conv=1, img_h=H, img_w=W, batch=B, n_samples=n)
+    o = O.Oracle(O.make_config(O.MODEL_CNN, **geo, **kw), X, labels, xs, w0)
+    idx, _, _ = o.read_schedule(0)
+    c1 = O.make_config(O.MODEL_CNN, **dict(geo, batch=B), K=1)
+    rho, gam = float(np.float32(0.1)), float(np.float32(1e-12))
+    g1 = np.stack([O.loss_grad(c1, X, labels, xs[k], idx[k])[1] for k in range(K)])
+    xp = np.stack([xs[k] + rho * g1[k] / (np.linalg.norm(g1[k]) + gam) for k in range(K)])
+    g2 = np.stack([O.loss_grad(c1, X, labels, xp[k], idx[k])[1] for k in range(K)])
+    o.step(0.05, 0.1)
+    f = O.Oracle(O.make_config(O.MODEL_FLAT, flat_d=len(w0), **kw), None, None, xs, w0)
+    f.set_external_grads(g1, g2)
+    f.step(0.05, 0.1)
+    for key in ("x", "v", "acc"):
+        assert np.linalg.norm(f.read_state()[key] - o.read_state()[key]) <= 1e-6 * np.linalg.norm(o.read_state()[key]), key
