@@ -49,7 +49,7 @@ enum {
   LSAM_ERR_TIMEOUT = 6    /* a bounded device-side wait expired (reported by lsam_status)           */
 };
 
-enum { LSAM_MODEL_LSQ = 0, LSAM_MODEL_MLP = 1, LSAM_MODEL_RESMLP = 2, LSAM_MODEL_FLAT = 3 };
+enum { LSAM_MODEL_LSQ = 0, LSAM_MODEL_MLP = 1, LSAM_MODEL_RESMLP = 2, LSAM_MODEL_FLAT = 3, LSAM_MODEL_CNN = 4 };
 enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
 /* TCGEN05: tensor-core GEMMs; forward and dgrad with a minibatch tile of 256 samples are run by pairs of CTAs
  * (cta_group::2, 256-row tiles), everything else by single CTAs (128-row tiles); the weight gradient of a minibatch of at
@@ -84,6 +84,12 @@ enum {
  *  MLP    h_{l+1} = relu(W_l h_l + b_l), linear head, softmax cross-entropy averaged over the minibatch.
  *  RESMLP as MLP, but every hidden layer with equal input and output width is h_{l+1} = h_l + relu(W_l h_l + b_l).
  *  FLAT   no model: the two gradients of a step are buffers supplied with lsam_set_external_grads().
+ *  CNN    n_conv layers of 3x3 convolution (stride 1, zero padding 1) + ReLU + 2x2 max-pooling, then dense layers as in MLP (the paper's
+ *         experiments train small convolutional nets, Section 5.1).  widths = channels C0 .. C_nconv, then the dense widths (hidden..., classes);
+ *         a row of X is an img_h x img_w image with C0 channels, channel-major (feature = c H W + y W + x: the flattening every later layer uses
+ *         too); img_h and img_w divisible by 2^n_conv, batch a multiple of 16.  Parameters: conv W_l [Cout][Cin * 9] (column = ci * 9 + kh * 3 + kw)
+ *         then b_l [Cout]; dense layers as in MLP, the first one taking C_nconv (img_h / 2^n_conv) (img_w / 2^n_conv) inputs.  Runs on the SIMT
+ *         GEMMs (fp32, or bf16 operands with fp32 accumulation) through an explicit patch matrix.
  * gemm_dtype BF16: matmul operands (weights, biases, inputs, stored activations and backward signals) are
  * rounded to bf16, products accumulate in fp32, all optimiser state (x, v, centre, accumulator) stays fp32.
  * Eq. 3 and the worker update are defined on the gradients as computed.  The SIMT path keeps g1 and g2 in fp32.  The
@@ -123,6 +129,8 @@ typedef struct {
                           tick are averaged over the K workers before they are used (perturbation along the averaged gradient
                           and its norm, update with the averaged descent gradient).  Workers that start equal stay equal;
                           lock-step schedule only, one context holds the whole job.  rho = 0 gives DP-SGD.                   */
+  int32_t n_conv;      /* CNN: number of convolution layers (the first n_conv of the n_layers)                                */
+  int32_t img_h, img_w; /* CNN: input image size                                                                              */
 } lsam_config;
 
 /* Unpadded parameter count d of one replica, or -1 if the configuration is invalid. */

@@ -265,7 +265,9 @@ double net_loss_grad(const Net& net, const double* params, const std::vector<dou
               s += pq[(size_t)(ly.b_off + co)];
               const size_t e = (size_t)b * ly.Cout * Hh * Ww + ((size_t)co * Hh + y) * Ww + x;
               mask[l][e] = s > 0.0;
-              r[e] = s > 0.0 ? s : 0.0;
+              // the ReLU output is a stored activation (bf16 mode: rounded), and the pooling compares the stored values: its
+              // choice of the maximum is a discrete decision, taken on both sides in the precision the activations are kept in
+              r[e] = net.q(s > 0.0 ? s : 0.0);
             }
       h[l + 1].resize((size_t)B * ly.out);
       pool_arg[l].assign((size_t)B * ly.out, 0);
@@ -281,7 +283,7 @@ double net_loss_grad(const Net& net, const double* params, const std::vector<dou
                   if (v > best) { best = v; arg = dy * 2 + dx; }
                 }
               const size_t e = (size_t)b * ly.out + ((size_t)co * Ho + y) * Wo + x;
-              h[l + 1][e] = net.q(best);  // stored activation (bf16 mode: rounded)
+              h[l + 1][e] = best;  // the maximum of stored values
               pool_arg[l][e] = (unsigned char)arg;
             }
       continue;

@@ -12,7 +12,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "liblsam_b200.so")
 
 LSAM_OK, LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE, LSAM_ERR_STATE, LSAM_ERR_CUDA, LSAM_ERR_NONFINITE, LSAM_ERR_TIMEOUT = range(7)
-MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT = 0, 1, 2, 3
+MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT, MODEL_CNN = 0, 1, 2, 3, 4
 GEMM_FP32, GEMM_BF16 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05, IMPL_TCGEN05_1CTA, IMPL_TCGEN05_PAIRS = 0, 1, 2, 3, 4
 KERNEL_GAUSSIAN, KERNEL_EXP_POWER, KERNEL_CAUCHY, KERNEL_MATERN32 = 0, 1, 2, 3
@@ -38,6 +38,7 @@ class LsamConfig(C.Structure):
         ("seed", C.c_uint64), ("mu", C.c_float), ("gamma", C.c_float), ("lam", C.c_float), ("beta", C.c_float),
         ("eta_prime", C.c_float), ("active_num", C.c_int32), ("noise_temp", C.c_float),
         ("K_total", C.c_int32), ("k_offset", C.c_int32), ("kernel_kind", C.c_int32), ("kernel_param", C.c_float), ("dp_average", C.c_int32),
+        ("n_conv", C.c_int32), ("img_h", C.c_int32), ("img_w", C.c_int32),
     ]
 
 
@@ -111,11 +112,11 @@ def lib():
 
 def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=IMPL_AUTO, mu=0.9, nesterov=1,
                 gamma=1e-12, lam=0.0, tau=4, beta=0.9, eta_prime=1.0, stale_max=0, seed=0, n_samples=1, flat_d=0, flags=0,
-                active_num=256, noise_temp=0.0, K_total=0, k_offset=0, kernel_kind=KERNEL_GAUSSIAN, kernel_param=0.0, dp_average=0):
+                active_num=256, noise_temp=0.0, K_total=0, k_offset=0, kernel_kind=KERNEL_GAUSSIAN, kernel_param=0.0, dp_average=0, n_conv=0, img_h=0, img_w=0):
     c = LsamConfig()
     c.model = model
     widths = list(widths)
-    c.n_layers = max(len(widths) - 1, 0) if model in (MODEL_MLP, MODEL_RESMLP) else (1 if model == MODEL_LSQ else 0)
+    c.n_layers = max(len(widths) - 1, 0) if model in (MODEL_MLP, MODEL_RESMLP, MODEL_CNN) else (1 if model == MODEL_LSQ else 0)
     for i, w in enumerate(widths):
         c.widths[i] = int(w)
     c.K, c.batch, c.gemm_dtype, c.gemm_impl, c.nesterov, c.tau = int(K), int(batch), int(gemm_dtype), int(gemm_impl), int(nesterov), int(tau)
@@ -125,6 +126,7 @@ def make_config(model, widths=(), K=1, batch=1, gemm_dtype=GEMM_FP32, gemm_impl=
     c.noise_temp = noise_temp
     c.K_total, c.k_offset = int(K_total), int(k_offset)
     c.kernel_kind, c.kernel_param, c.dp_average = int(kernel_kind), kernel_param, int(dp_average)
+    c.n_conv, c.img_h, c.img_w = int(n_conv), int(img_h), int(img_w)
     return c
 
 

@@ -24,10 +24,14 @@ using namespace lsam;
 namespace {
 
 struct LayerInfo {
-  int in, out;
+  int in, out;           // shape of the weight matrix [out, in] (a convolution: [Cout, Cin * 9])
   int64_t w_unp, b_unp;  // offsets in the unpadded vector
   int64_t w_pad, b_pad;  // offsets in the padded row
   bool residual;
+  // convolution layer (3x3, stride 1, padding 1, ReLU, 2x2 max-pooling) on H x W feature maps
+  bool conv = false;
+  int Cin = 0, Cout = 0, H = 0, W = 0;
+  int64_t feat_in = 0, feat_out = 0;  // features per sample entering / leaving the layer (dense: in / out)
 };
 
 struct Layout {
@@ -35,6 +39,7 @@ struct Layout {
   int64_t d = 0, ld = 0;
   std::vector<LayerInfo> layers;
   int ldb = 0;  // sample stride of the feature-major activation-like buffers [K, width, ldb] (multiple of 16)
+  int in0 = 0;  // features of one minibatch row (widths[0]; convolutional model: C0 * H * W)
   SegMap seg{};
   int ring = 2;
   int64_t nchunks = 0;
@@ -42,6 +47,7 @@ struct Layout {
   // byte offsets into the workspace
   size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status, gbar1, gbar2;
   size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage, xstage2, ystage2;
+  size_t col[9], parg[9], zout, dzc, dcol;  // convolutional model: patch matrices, pooling choices, pre-pooling output, its gradient, patch-matrix gradient
   size_t total = 0;
 };
 
@@ -78,18 +84,33 @@ bool plan(const lsam_config& c, Layout& L) {
   } else if (c.model == LSAM_MODEL_LSQ) {
     if (c.widths[0] < 1 || c.batch < 1 || c.n_samples < 1 || bf) return false;
     L.d = c.widths[0];
+    L.in0 = c.widths[0];
     L.ld = round_up(L.d, kSegAlign);
     L.layers.push_back({c.widths[0], 1, 0, -1, 0, -1, false});
     L.seg.n = 1;
     L.seg.src[0] = 0; L.seg.dst[0] = 0; L.seg.len[0] = L.d;
-  } else if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {
+  } else if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP || c.model == LSAM_MODEL_CNN) {
     if (c.n_layers < 1 || c.n_layers > 8 || c.batch < 1 || c.n_samples < 1) return false;
+    const bool cnn = c.model == LSAM_MODEL_CNN;
+    // convolutional model: positions are indexed (y, x, sample) with the sample fastest, so the minibatch must fill its stride
+    if (cnn && (c.n_conv < 1 || c.n_conv >= c.n_layers || c.img_h < 1 || c.img_w < 1 || c.img_h % (1 << c.n_conv) || c.img_w % (1 << c.n_conv) || c.batch % 16)) return false;
     int64_t unp = 0, pad = 0;
+    int H = c.img_h, W = c.img_w;
     for (int l = 0; l < c.n_layers; ++l) {
       LayerInfo li;
-      li.in = c.widths[l];
-      li.out = c.widths[l + 1];
-      if (li.in < 1 || li.out < 1) return false;
+      if (c.widths[l] < 1 || c.widths[l + 1] < 1) return false;
+      if (cnn && l < c.n_conv) {
+        li.conv = true;
+        li.Cin = c.widths[l]; li.Cout = c.widths[l + 1]; li.H = H; li.W = W;
+        li.in = li.Cin * 9; li.out = li.Cout;
+        li.feat_in = (int64_t)li.Cin * H * W;
+        H /= 2; W /= 2;
+        li.feat_out = (int64_t)li.Cout * H * W;
+      } else {
+        li.in = (cnn && l == c.n_conv) ? (int)L.layers.back().feat_out : c.widths[l];  // the first dense layer takes the flattened feature maps
+        li.out = c.widths[l + 1];
+        li.feat_in = li.in; li.feat_out = li.out;
+      }
       li.w_unp = unp; unp += (int64_t)li.in * li.out;
       li.b_unp = unp; unp += li.out;
       li.w_pad = pad; pad = round_up(pad + (int64_t)li.in * li.out, kSegAlign);
@@ -99,6 +120,7 @@ bool plan(const lsam_config& c, Layout& L) {
       L.seg.src[L.seg.n] = li.w_unp; L.seg.dst[L.seg.n] = li.w_pad; L.seg.len[L.seg.n] = (int64_t)li.in * li.out; ++L.seg.n;
       L.seg.src[L.seg.n] = li.b_unp; L.seg.dst[L.seg.n] = li.b_pad; L.seg.len[L.seg.n] = li.out; ++L.seg.n;
     }
+    L.in0 = (int)L.layers[0].feat_in;
     L.ldb = (int)round_up(c.batch, 16);
     L.d = unp;
     L.ld = pad;
@@ -108,7 +130,7 @@ bool plan(const lsam_config& c, Layout& L) {
   L.ring = c.stale_max + 2;
   // partial-sum slots per replica; FLAT may fall back to scalar chunks when the caller's gradient buffers are misaligned
   L.nchunks = ceil_div(L.ld, (c.model == LSAM_MODEL_FLAT) ? norm_chunk<1>() : norm_chunk<4>());
-  if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {  // room for the slots of the fused tensor-core norm
+  if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {  // room for the slots of the fused tensor-core norm (the convolutional model runs on the SIMT GEMMs)
     const int64_t slots = tc_norm_slots(c);
     L.nchunks = slots > L.nchunks ? slots : L.nchunks;
   }
@@ -140,8 +162,10 @@ bool plan(const lsam_config& c, Layout& L) {
   L.ylab = take(4 * K * B);
   for (int i = 0; i < 9; ++i) L.act[i] = L.mask[i] = 0;
   L.logits = L.rowloss = L.dz[0] = L.dz[1] = L.dh[0] = L.dh[1] = L.xstage = L.ystage = L.xstage2 = L.ystage2 = 0;
+  for (int i = 0; i < 9; ++i) L.col[i] = L.parg[i] = 0;
+  L.zout = L.dzc = L.dcol = 0;
   if (!flat) {
-    const size_t in0 = c.widths[0];
+    const size_t in0 = L.in0;
     const size_t ldb = L.ldb;
     // least squares keeps its minibatch sample-major [K, B, in]; the classifiers store everything feature-major [K, width, ldb]
     L.act[0] = (c.model == LSAM_MODEL_LSQ) ? take(4 * K * B * in0) : take(esz * K * in0 * ldb);
@@ -150,15 +174,26 @@ bool plan(const lsam_config& c, Layout& L) {
     L.xstage2 = take(4 * K * B * in0);  // second slot of the prefetch queue (lsam_stage_batch)
     L.ystage2 = take(4 * K * B);
     if (c.model != LSAM_MODEL_LSQ) {
-      size_t maxw = 0;
+      size_t maxw = 0, max_full = 0, max_dcol = 0;
       for (size_t l = 0; l < L.layers.size(); ++l) {
-        const size_t w = L.layers[l].out;
+        const LayerInfo& li = L.layers[l];
+        const size_t w = (size_t)li.feat_out;
         maxw = w > maxw ? w : maxw;
         if (l + 1 < L.layers.size()) {
           L.act[l + 1] = take(esz * K * w * ldb);
-          L.mask[l] = take(K * w * ldb);
+          // ReLU mask: at the resolution before pooling for a convolution
+          L.mask[l] = take(K * (li.conv ? (size_t)li.Cout * li.H * li.W : w) * ldb);
+        }
+        if (li.conv) {
+          const size_t P = (size_t)li.H * li.W * ldb;
+          L.col[l] = take(esz * K * (size_t)li.in * P);
+          L.parg[l] = take(K * w * ldb);
+          max_full = std::max(max_full, (size_t)li.Cout * P);
+          if (l > 0) max_dcol = std::max(max_dcol, (size_t)li.in * P);
         }
       }
+      if (max_full) { L.zout = take(esz * K * max_full); L.dzc = take(esz * K * max_full); }
+      if (max_dcol) L.dcol = take(esz * K * max_dcol);
       L.logits = take(4 * K * (size_t)L.layers.back().out * ldb);
       L.rowloss = take(4 * K * B);
       for (int i = 0; i < 2; ++i) L.dz[i] = take(esz * K * maxw * ldb);
@@ -610,14 +645,113 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
   return LSAM_OK;
 }
 
+// One gradient pass of the convolutional model (SIMT GEMMs): convolution layers through an explicit patch matrix, then the
+// dense layers exactly as in mlp_pass.  Feature maps are [K, C, (y, x, sample)] with the sample fastest (see im2col_kernel).
+template <typename T>
+int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
+  const Layout& L = c->L;
+  const int K = c->cfg.K, B = c->cfg.batch;
+  const int nl = (int)L.layers.size(), nconv = c->cfg.n_conv;
+  const int64_t ld = L.ld;
+  const int ldb = L.ldb;  // = B for this model
+  int rc;
+  // forward
+  for (int l = 0; l < nl; ++l) {
+    const LayerInfo& li = L.layers[l];
+    const T* a_in = c->at<T>(L.act[l]);
+    const bool head = (l == nl - 1);
+    if (li.conv) {
+      const int64_t Pn = (int64_t)li.H * li.W * ldb;
+      T* col = c->at<T>(L.col[l]);
+      LAUNCH(c, LSAM_PROF_GATHER, im2col_kernel<T><<<dim3((unsigned)ceil_div(Pn, 256), li.in, K), 256, 0, c->stream>>>(a_in, li.Cin, li.H, li.W, ldb, col, c->act()));
+      GemmOperand A{col, (int64_t)li.in * Pn, 1, Pn};           // (z, position, patch element)
+      GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, output channel, patch element)
+      EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.zout), nullptr, c->at<uint8_t>(L.mask[l]), li.Cout, (int)Pn};
+      if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, (int)Pn, li.Cout, li.in, e)) != LSAM_OK) return rc;
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, maxpool_kernel<T><<<dim3((unsigned)ceil_div(Pn / 4, 256), li.Cout, K), 256, 0, c->stream>>>(
+          c->at<T>(L.zout), li.Cout, li.H, li.W, ldb, c->at<T>(L.act[l + 1]), c->at<uint8_t>(L.parg[l]), c->act()));
+      continue;
+    }
+    GemmOperand A{a_in, (int64_t)li.in * ldb, 1, ldb};
+    GemmOperand W{P + li.w_pad, ld, li.in, 1};
+    if (head) {
+      EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), li.out, ldb};
+      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
+    } else {
+      EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.act[l + 1]), nullptr, c->at<uint8_t>(L.mask[l]), li.out, ldb};
+      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
+    }
+    if (rc != LSAM_OK) return rc;
+  }
+  const int C = L.layers[nl - 1].out;
+  int cur = 0;
+  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
+      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act()));
+  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
+  // backward.  dz[cur] holds, for a dense layer, the gradient w.r.t. its pre-activation; for a convolution layer, the gradient
+  // w.r.t. its POOLED output (the pooling and the ReLU are undone by unpool_kernel)
+  for (int l = nl - 1; l >= 0; --l) {
+    const LayerInfo& li = L.layers[l];
+    const T* a_in = c->at<T>(L.act[l]);
+    if (li.conv) {
+      const int64_t Pn = (int64_t)li.H * li.W * ldb;
+      T* dzc = c->at<T>(L.dzc);
+      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, unpool_kernel<T><<<dim3((unsigned)ceil_div(Pn, 256), li.Cout, K), 256, 0, c->stream>>>(
+          c->at<T>(L.dz[cur]), c->at<uint8_t>(L.parg[l]), c->at<uint8_t>(L.mask[l]), li.Cout, li.H, li.W, ldb, dzc, c->act()));
+      LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<dim3((unsigned)ceil_div(li.Cout, 8), K), 256, 0, c->stream>>>(
+          dzc, (int)Pn, li.Cout, (int)Pn, c->g(), ld, li.b_pad, nullptr, L.nchunks, 0, c->act()));
+      {
+        GemmOperand A{dzc, (int64_t)li.Cout * Pn, Pn, 1};                 // (z, output channel, position)
+        GemmOperand Bm{c->at<T>(L.col[l]), (int64_t)li.in * Pn, Pn, 1};   // (z, patch element, position)
+        EpiWgrad e{c->g(), ld, li.w_pad, li.in};
+        if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.Cout, li.in, (int)Pn, e)) != LSAM_OK) return rc;
+      }
+      if (l > 0) {
+        T* dcol = c->at<T>(L.dcol);
+        GemmOperand A{dzc, (int64_t)li.Cout * Pn, 1, Pn};                  // (z, position, output channel)
+        GemmOperand W{P + li.w_pad, ld, 1, li.in};                         // (z, patch element, output channel)
+        EpiDgrad<T> e{nullptr, nullptr, dcol, nullptr, li.in, (int)Pn};    // the raw gradient of the patch matrix
+        if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_DGRAD, A, W, (int)Pn, li.in, li.Cout, e)) != LSAM_OK) return rc;
+        LAUNCH(c, LSAM_PROF_GEMM_DGRAD, col2im_kernel<T><<<dim3((unsigned)ceil_div(Pn, 256), li.Cin, K), 256, 0, c->stream>>>(
+            dcol, li.Cin, li.H, li.W, ldb, c->at<T>(L.dz[cur ^ 1]), c->act()));
+      }
+      cur ^= 1;
+      continue;
+    }
+    const T* dz = c->at<T>(L.dz[cur]);
+    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(
+        dz, B, li.out, ldb, c->g(), ld, li.b_pad, nullptr, L.nchunks, 0, c->act()));
+    {
+      GemmOperand A{dz, (int64_t)li.out * ldb, ldb, 1};
+      GemmOperand Bm{a_in, (int64_t)li.in * ldb, ldb, 1};
+      EpiWgrad e{c->g(), ld, li.w_pad, li.in};
+      if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.out, li.in, B, e)) != LSAM_OK) return rc;
+    }
+    {
+      GemmOperand A{dz, (int64_t)li.out * ldb, 1, ldb};
+      GemmOperand W{P + li.w_pad, ld, 1, li.in};
+      // the layer below is dense (its ReLU mask applies here) or the last convolution (the raw gradient of its pooled output)
+      const bool below_conv = (l - 1 < nconv);
+      EpiDgrad<T> e{nullptr, nullptr, c->at<T>(L.dz[cur ^ 1]), below_conv ? nullptr : c->at<uint8_t>(L.mask[l - 1]), li.in, ldb};
+      if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_DGRAD, A, W, B, li.in, li.out, e)) != LSAM_OK) return rc;
+    }
+    cur ^= 1;
+  }
+  return LSAM_OK;
+}
+
 // Gradient of the minibatch loss at the parameters held in `params` (x master, or the operand buffer).
 int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false, const TcFusedUpdate* fu = nullptr) {
   const lsam_config& cfg = c->cfg;
   if (cfg.model == LSAM_MODEL_LSQ) {
     const float* P = perturbed ? c->at<float>(c->L.xop) : c->x();
     LAUNCH(c, LSAM_PROF_LSQ_GRAD, lsq_grad_kernel<<<cfg.K, 256, sizeof(float) * cfg.batch, c->stream>>>(
-        c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, cfg.widths[0], c->g(), c->L.ld, loss_out, c->act()));
+        c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, c->L.in0, c->g(), c->L.ld, loss_out, c->act()));
     return LSAM_OK;
+  }
+  if (cfg.model == LSAM_MODEL_CNN) {
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16) return cnn_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out);
+    return cnn_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out);
   }
   if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out, g_bf16 && c->use_tc, c->use_tc ? fu : nullptr);
   return mlp_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out, false);
@@ -665,13 +799,13 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   if (!flat && gather) {
     if (cfg.model == LSAM_MODEL_LSQ) {
-      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.widths[0], cfg.widths[0], c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), cfg.batch, c->act()));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, c->L.in0, c->L.in0, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), cfg.batch, c->act()));
     } else {
-      dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
+      dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
       if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
       else
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, cfg.widths[0], L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
     }
   }
   const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
@@ -978,7 +1112,7 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   // refused before anything is copied: while the sync is due the call does nothing
   if (c->budget() <= 0) return c->fail(LSAM_ERR_STATE, "the sync is due: call lsam_couple before the next lsam_step");
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
-  const int64_t nx = rows * cfg.widths[0];
+  const int64_t nx = rows * c->L.in0;
   const cudaMemcpyKind kind = on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
   const bool lsq = cfg.model == LSAM_MODEL_LSQ;
   float* xdst = lsq ? c->at<float>(c->L.act[0]) : c->at<float>(c->L.xstage);  // classifiers: staged, then stored feature-major
@@ -986,11 +1120,11 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   LSAM_CUDA(c, cudaMemcpyAsync(xdst, xb, sizeof(float) * nx, kind, c->stream));
   LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(c->L.ylab), yb, 4 * rows, kind, c->stream));
   if (!lsq) {
-    dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
+    dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
     if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
     else
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
   }
   int rc = step_common(c, eta, rho, false);
   if (rc != LSAM_OK) return rc;
@@ -1019,7 +1153,7 @@ int lsam_stage_batch(lsam_ctx* c, const float* xb, const void* yb, int on_host) 
   const cudaMemcpyKind kind = on_host ? cudaMemcpyHostToDevice : cudaMemcpyDeviceToDevice;
   // the slot may still be read by the tick that consumed it last
   if (c->slot_used[slot]) LSAM_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->slot_free[slot], 0));
-  LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(slot ? c->L.xstage2 : c->L.xstage), xb, sizeof(float) * rows * cfg.widths[0], kind, c->copy_stream));
+  LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(slot ? c->L.xstage2 : c->L.xstage), xb, sizeof(float) * rows * c->L.in0, kind, c->copy_stream));
   LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(slot ? c->L.ystage2 : c->L.ystage), yb, 4 * rows, kind, c->copy_stream));
   LSAM_CUDA(c, cudaEventRecord(c->staged_done[slot], c->copy_stream));
   c->stage_count += 1;
@@ -1040,13 +1174,13 @@ int lsam_step_staged(lsam_ctx* c, float eta, float rho, float* h_loss) {
   LSAM_CUDA(c, cudaStreamWaitEvent(c->stream, c->staged_done[slot], 0));
   LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(c->L.ylab), c->at<uint32_t>(slot ? c->L.ystage2 : c->L.ystage), 4 * rows, cudaMemcpyDeviceToDevice, c->stream));
   if (cfg.model == LSAM_MODEL_LSQ) {
-    LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(c->L.act[0]), xs, sizeof(float) * rows * cfg.widths[0], cudaMemcpyDeviceToDevice, c->stream));
+    LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(c->L.act[0]), xs, sizeof(float) * rows * c->L.in0, cudaMemcpyDeviceToDevice, c->stream));
   } else {
-    dim3 grid((unsigned)ceil_div(cfg.widths[0], 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
+    dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
     if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
     else
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, cfg.widths[0], c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
   }
   LSAM_CUDA(c, cudaEventRecord(c->slot_free[slot], c->stream));
   c->slot_used[slot] = true;

@@ -173,7 +173,7 @@ struct EpiDgrad {
     const float s = dh_next ? acc + to_float(dh_next[e]) : acc;
     const TA q = from_float<TA>(s);
     if (dh_out) dh_out[e] = q;
-    dz_prev[e] = mask_prev[e] ? q : from_float<TA>(0.f);
+    dz_prev[e] = (mask_prev == nullptr || mask_prev[e]) ? q : from_float<TA>(0.f);  // no mask: the raw gradient (pooled layers apply theirs later)
   }
 };
 
@@ -433,6 +433,99 @@ bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, TG* __restr
       partial[(int64_t)z * ld_partial + slot0 + blockIdx.x] = t;
     }
   }
+}
+
+// ------------------------------------------------------------------------------------------------ convolution layers
+// A convolution layer (3x3, stride 1, zero padding 1, ReLU, 2x2 max-pooling) runs on the batched GEMMs through an explicit
+// patch matrix.  Feature maps are feature-major like every activation buffer, [K, C, P] with the position index
+// p = (y * W + x) * B + b (sample fastest), so that the gathered minibatch [K, C0 * H * W, B] already is the first layer's input and
+// the pooled output of the last convolution already is the dense layers' input [K, C * H' * W', B].
+//   col[z][ci * 9 + kh * 3 + kw][(y, x, b)] = a[z][ci][(y + kh - 1, x + kw - 1, b)]  (0 outside the image)
+// One thread per element of col, consecutive threads along p.  grid (ceil(P / 256), Cin * 9, K).
+template <typename T>
+__global__ void __launch_bounds__(256)
+im2col_kernel(const T* __restrict__ a, int Cin, int H, int W, int B, T* __restrict__ col, const int32_t* __restrict__ active) {
+  const int z = blockIdx.z;
+  if (active != nullptr && !active[z]) return;
+  const int64_t P = (int64_t)H * W * B;
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  const int r = blockIdx.y, ci = r / 9, kh = (r % 9) / 3, kw = r % 3;
+  const int b = (int)(p % B);
+  const int x = (int)((p / B) % W), y = (int)(p / ((int64_t)B * W));
+  const int yy = y + kh - 1, xx = x + kw - 1;
+  T v = from_float<T>(0.f);
+  if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = a[((int64_t)z * Cin + ci) * P + ((int64_t)yy * W + xx) * B + b];
+  col[((int64_t)z * Cin * 9 + r) * P + p] = v;
+}
+
+// 2x2 max-pooling of the ReLU output r [K, C, (H, W, B)] -> pooled [K, C, (H/2, W/2, B)]; arg = which element of the window
+// (dy * 2 + dx, the first maximum in that order).  One thread per pooled element.  grid (ceil(P4 / 256), C, K).
+template <typename T>
+__global__ void __launch_bounds__(256)
+maxpool_kernel(const T* __restrict__ r, int C, int H, int W, int B, T* __restrict__ pooled, uint8_t* __restrict__ arg,
+               const int32_t* __restrict__ active) {
+  const int z = blockIdx.z, c = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  const int Ho = H / 2, Wo = W / 2;
+  const int64_t P4 = (int64_t)Ho * Wo * B;
+  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (q >= P4) return;
+  const int b = (int)(q % B), xo = (int)((q / B) % Wo), yo = (int)(q / ((int64_t)B * Wo));
+  const T* src = r + ((int64_t)z * C + c) * (int64_t)H * W * B;
+  float best = -1.f;
+  int a = 0;
+#pragma unroll
+  for (int dy = 0; dy < 2; ++dy)
+#pragma unroll
+    for (int dx = 0; dx < 2; ++dx) {
+      const float v = to_float(src[((int64_t)(2 * yo + dy) * W + 2 * xo + dx) * B + b]);
+      if (v > best) { best = v; a = dy * 2 + dx; }
+    }
+  pooled[((int64_t)z * C + c) * P4 + q] = from_float<T>(best);
+  arg[((int64_t)z * C + c) * P4 + q] = (uint8_t)a;
+}
+
+// Backward of the pooling and the ReLU in one: dz[z][c][(y, x, b)] = dpool[z][c][(y/2, x/2, b)] if (y, x) was its window's
+// maximum and the ReLU was active there, else 0.  One thread per full-resolution element.  grid (ceil(P / 256), C, K).
+template <typename T>
+__global__ void __launch_bounds__(256)
+unpool_kernel(const T* __restrict__ dpool, const uint8_t* __restrict__ arg, const uint8_t* __restrict__ mask, int C, int H, int W, int B,
+              T* __restrict__ dz, const int32_t* __restrict__ active) {
+  const int z = blockIdx.z, c = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  const int64_t P = (int64_t)H * W * B;
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  const int b = (int)(p % B), x = (int)((p / B) % W), y = (int)(p / ((int64_t)B * W));
+  const int64_t q = ((int64_t)(y / 2) * (W / 2) + x / 2) * B + b;
+  const int64_t pc = ((int64_t)z * C + c);
+  const bool hit = arg[pc * (P / 4) + q] == (uint8_t)((y & 1) * 2 + (x & 1)) && mask[pc * P + p] != 0;
+  dz[pc * P + p] = hit ? dpool[pc * (P / 4) + q] : from_float<T>(0.f);
+}
+
+// Gradient w.r.t. a convolution's input from the gradient of its patch matrix:
+//   da[z][ci][(y, x, b)] = sum over (kh, kw) ascending of dcol[z][ci * 9 + kh * 3 + kw][(y - kh + 1, x - kw + 1, b)]  (terms outside the image dropped)
+// summed in fp32, stored as T.  One thread per element.  grid (ceil(P / 256), Cin, K).
+template <typename T>
+__global__ void __launch_bounds__(256)
+col2im_kernel(const T* __restrict__ dcol, int Cin, int H, int W, int B, T* __restrict__ da, const int32_t* __restrict__ active) {
+  const int z = blockIdx.z, ci = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  const int64_t P = (int64_t)H * W * B;
+  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (p >= P) return;
+  const int b = (int)(p % B), x = (int)((p / B) % W), y = (int)(p / ((int64_t)B * W));
+  float s = 0.f;
+#pragma unroll
+  for (int kh = 0; kh < 3; ++kh)
+#pragma unroll
+    for (int kw = 0; kw < 3; ++kw) {
+      const int yy = y - kh + 1, xx = x - kw + 1;
+      if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+      s += to_float(dcol[((int64_t)z * Cin * 9 + ci * 9 + kh * 3 + kw) * P + ((int64_t)yy * W + xx) * B + b]);
+    }
+  da[((int64_t)z * Cin + ci) * P + p] = from_float<T>(s);
 }
 
 // ------------------------------------------------------------------------------------------------ least squares

@@ -337,6 +337,36 @@ def test_fused_update_in_the_weight_gradient_epilogue_matches_oracle(model, widt
                    torch.from_numpy(synth.replicate(w0, K)).cuda(), torch.from_numpy(w0).cuda())
 
 
+# ------------------------------------------------------------------------------------------------ convolutional model
+@pytest.mark.parametrize("channels,dense,H,W,K,B", [
+    ((3, 8, 12), (32, 10), 8, 8, 3, 16),     # two convolutions, two dense layers
+    ((2, 5), (7,), 4, 8, 2, 16),             # one convolution straight into the head, non-square image
+    ((1, 4, 6, 9), (20, 5), 16, 16, 2, 32),  # three convolutions, positions spanning several GEMM tiles
+])
+@pytest.mark.parametrize("dtype", [G.GEMM_FP32, G.GEMM_BF16])
+def test_convolutional_model_matches_oracle(channels, dense, H, W, K, B, dtype):
+    # 3x3 convolution + ReLU + 2x2 max-pooling layers through an explicit patch matrix on the batched GEMMs, then dense layers
+    n = 200
+    X, labels = synth.gaussian_mixture(n, channels[0] * H * W, dense[-1], seed=5)
+    w0 = synth.cnn_init(channels, dense, H, W, seed=6)
+    p = Pair(G.MODEL_CNN, widths=tuple(channels) + tuple(dense), K=K, batch=B, X=X, Y=labels, x0=synth.replicate(w0, K, jitter=0.01, seed=6), y0=w0,
+             gemm_dtype=dtype, flags=G.FLAG_KEEP_G1 | G.FLAG_STEP_INFO, n_conv=len(channels) - 1, img_h=H, img_w=W, tau=4, lam=0.4, seed=3, stale_max=1)
+    assert p.d == synth.cnn_param_count(channels, dense, H, W) and not p.gpu.uses_tcgen05()
+    bf = dtype == G.GEMM_BF16
+    _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_BF16 if bf else TOL_STEP_FP32, TOL_TRAJ_BF16 if bf else TOL_TRAJ_FP32, steps=12, forced=2,
+                              what=f"cnn {channels} {dense}")
+    p.close()
+
+
+def test_convolutional_model_configuration_is_checked():
+    geo = dict(widths=(3, 8, 16, 10), K=2, n_samples=10, n_conv=2)
+    assert G.lsam_param_count(G.make_config(G.MODEL_CNN, batch=16, img_h=8, img_w=8, **geo)) == 8 * 27 + 8 + 16 * 72 + 16 + 16 * 4 * 10 + 10
+    assert G.lsam_workspace_bytes(G.make_config(G.MODEL_CNN, batch=16, img_h=6, img_w=8, **geo)) == 0    # 6 is not divisible by 4
+    assert G.lsam_workspace_bytes(G.make_config(G.MODEL_CNN, batch=10, img_h=8, img_w=8, **geo)) == 0    # the minibatch must be a multiple of 16
+    assert G.lsam_workspace_bytes(G.make_config(G.MODEL_CNN, batch=16, img_h=8, img_w=8, **dict(geo, n_conv=3))) == 0  # no dense layer left
+    assert G.lsam_workspace_bytes(G.make_config(G.MODEL_CNN, batch=16, img_h=8, img_w=8, **geo)) > 0
+
+
 def test_step_batch_matches_gathered_step():
     # the caller-supplied minibatch path (host buffers) must reproduce the resident-dataset path exactly
     import torch
