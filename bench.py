@@ -23,7 +23,7 @@ import numpy as np
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
-LSQ, MLP, RESMLP, FLAT = 0, 1, 2, 3
+LSQ, MLP, RESMLP, FLAT, CNN = 0, 1, 2, 3, 4
 
 # The five workloads (shapes, replica counts, batch sizes and radii as configured).  Where a workload leaves them open:
 # tau = 16 as in the paper's experiments, lambda = lambda0 / (eta tau) with lambda0 = 0.9 from the grid of Appendix D,
@@ -38,6 +38,10 @@ WORKLOADS = {
                eta=0.01, tau=16, stale_max=0, name="MLP 3072-2048x3-100 bf16 GEMM, K=16, B=128"),
     "c4": dict(model=RESMLP, widths=(3072, 4096, 4096, 4096, 4096, 1000), K=32, B=256, n=200000, classes=1000, bf16=True,
                rho=0.1, eta=0.002, tau=16, stale_max=3, head_scale=0.1, res_scale=0.25, name="residual MLP 3072-4096x4-1000 bf16 GEMM, K=32, B=256, staleness [0,3]"),
+    # a convolutional second workload with the image shape of the paper's CIFAR runs (its own conv nets are not reproduced):
+    # two 3x3 convolution + ReLU + 2x2 max-pooling layers (3 -> 32 -> 64 channels), then dense 4096 -> 256 -> 10
+    "cnn": dict(model=CNN, widths=(3, 32, 64, 256, 10), n_conv=2, img=(32, 32), K=4, B=64, n=50000, classes=10, bf16=False, rho=0.05, eta=0.002, tau=16, head_scale=0.1,
+                stale_max=0, name="CNN 3x32x32 conv32-conv64-256-10 fp32, K=4, B=64"),
     "c5": dict(model=FLAT, widths=(), K=8, B=0, n=0, classes=0, bf16=False, rho=0.1, eta=0.05, tau=16, stale_max=0, d=256_000_000,
                name="optimiser-only sweep point d=256M, K=8"),
 }
@@ -49,7 +53,7 @@ FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12  # SMs x FMA lanes x 2 flop x m
 NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
 # The sample of each workload that the CPU oracle is timed on (fixed, so that the figure is a stable denominator):
 # replicas, samples per minibatch, steps.  The full model is always used.
-ORACLE_SAMPLE = {"c1": (4, 32, 20), "c2": (8, 16, 2), "c3": (2, 16, 1), "c4": (2, 8, 1)}
+ORACLE_SAMPLE = {"c1": (4, 32, 20), "c2": (8, 16, 2), "c3": (2, 16, 1), "c4": (2, 8, 1), "cnn": (4, 16, 1)}
 
 
 def ncu_traffic(kernel, K, d):
@@ -62,13 +66,28 @@ def ncu_traffic(kernel, K, d):
     return rec["bytes"] * scale, f"ncu capture at K={rec['K']}, d={rec['d']} ({rec['source']}) scaled by (20K+12)d"
 
 
+def gemm_layers(w):
+    """(positions per sample, in, out) of every weight matrix: a dense layer has one position per sample, a 3x3 convolution H x W of them."""
+    ws = w["widths"]
+    if w["model"] != CNN:
+        return [(1, ws[i], ws[i + 1]) for i in range(len(ws) - 1)]
+    H, W = w["img"]
+    out = []
+    for l in range(w["n_conv"]):
+        out.append((H * W, ws[l] * 9, ws[l + 1]))
+        H, W = H // 2, W // 2
+    feat = ws[w["n_conv"]] * H * W
+    for l in range(w["n_conv"], len(ws) - 1):
+        out.append((1, feat if l == w["n_conv"] else ws[l], ws[l + 1]))
+    return out
+
+
 def param_count(w):
     if w["model"] == FLAT:
         return w["d"]
     if w["model"] == LSQ:
         return w["widths"][0]
-    ws = w["widths"]
-    return sum(ws[i] * ws[i + 1] + ws[i + 1] for i in range(len(ws) - 1))
+    return sum(i * o + o for _, i, o in gemm_layers(w))
 
 
 def max_over_ranks(ms, world, device=None):
@@ -111,19 +130,18 @@ def work_model(w, tc, grads_bf16=None):
     out["norm"] = dict(bytes=0.0 if tc else 4.0 * K * d)                     # read g1 (fused into the wgrad epilogue on the tensor-core path)
     out["perturb"] = dict(bytes=(4.0 + gb + op) * K * d)                     # read x, g1; write x~
     out["update"] = dict(bytes=(gb + 8.0 + 8.0 + (2.0 if w["bf16"] else 0.0)) * K * d + 12.0 * d)  # g2, x rw, v rw, operand copy; y, acc rw
-    if w["model"] in (MLP, RESMLP):
-        ws = w["widths"]
+    if w["model"] in (MLP, RESMLP, CNN):
         f_fwd = f_dg = f_wg = 0.0
         b_fwd = b_dg = b_wg = 0.0
-        for l in range(len(ws) - 1):
-            i, o = ws[l], ws[l + 1]
-            f_fwd += 2.0 * B * i * o
-            b_fwd += op * (i * o + B * i + B * o)
-            f_wg += 2.0 * B * i * o
-            b_wg += gb * i * o + op * B * (i + o)                           # the gradient is written in its storage type
+        for l, (pos, i, o) in enumerate(gemm_layers(w)):
+            Bp = B * pos                                                    # rows of the GEMM: samples x positions
+            f_fwd += 2.0 * Bp * i * o
+            b_fwd += op * (i * o + Bp * i + Bp * o)
+            f_wg += 2.0 * Bp * i * o
+            b_wg += gb * i * o + op * Bp * (i + o)                          # the gradient is written in its storage type
             if l > 0:
-                f_dg += 2.0 * B * i * o
-                b_dg += op * (i * o + B * i + B * o)
+                f_dg += 2.0 * Bp * i * o
+                b_dg += op * (i * o + Bp * i + Bp * o)
         for name, f, b in (("gemm_fwd", f_fwd, b_fwd), ("gemm_dgrad", f_dg, b_dg), ("gemm_wgrad", f_wg, b_wg)):
             out[name] = dict(flops=2.0 * K * f, bytes=2.0 * K * b)          # two gradient passes per step
     return out
@@ -182,7 +200,7 @@ def make_inputs(w, dev, seed=0):
         g1 = torch.randn(K, d, device=dev, generator=g) * 0.1
         g2 = torch.randn(K, d, device=dev, generator=g) * 0.1
         return dict(X=None, Y=None, x0=x0, y0=x0.mean(0), g1=g1, g2=g2)
-    n, fin = w["n"], w["widths"][0]
+    n, fin = w["n"], (w["widths"][0] * w["img"][0] * w["img"][1] if w["model"] == CNN else w["widths"][0])
     if w["model"] == LSQ:
         X = torch.randn(n, fin, device=dev, generator=g)
         wstar = torch.randn(fin, device=dev, generator=g)
@@ -196,14 +214,15 @@ def make_inputs(w, dev, seed=0):
         X += means[Y.long()]
         parts = []
         ws = w["widths"]
-        for l in range(len(ws) - 1):
-            scale = (2.0 / ws[l]) ** 0.5
-            if l == len(ws) - 2:
+        shapes = gemm_layers(w)
+        for l, (_, fan_in, fan_out) in enumerate(shapes):
+            scale = (2.0 / fan_in) ** 0.5
+            if l == len(shapes) - 1:
                 scale *= w.get("head_scale", 1.0)       # small head: the initial loss starts near log(classes)
             elif w["model"] == RESMLP and ws[l] == ws[l + 1]:
                 scale *= w.get("res_scale", 1.0)        # damped residual branches: no normalisation layers here
-            parts.append((torch.randn(ws[l + 1], ws[l], device=dev, generator=g) * scale).reshape(-1))
-            parts.append(torch.zeros(ws[l + 1], device=dev))
+            parts.append((torch.randn(fan_out, fan_in, device=dev, generator=g) * scale).reshape(-1))
+            parts.append(torch.zeros(fan_out, device=dev))
         w0 = torch.cat(parts)
     x0 = w0.unsqueeze(0).expand(K, -1).contiguous()
     return dict(X=X, Y=Y, x0=x0, y0=w0)
@@ -215,7 +234,8 @@ def make_cfg(G, w, flags=0, K_total=0, k_offset=0, gemm_impl=0):
                          gemm_dtype=G.GEMM_BF16 if w["bf16"] else G.GEMM_FP32, mu=MU, nesterov=1, gamma=GAMMA, lam=lam, tau=w["tau"],
                          beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=max(w["n"], 1),
                          flat_d=w.get("d", 0), flags=flags, active_num=w.get("active_num", 256), gemm_impl=gemm_impl,
-                         noise_temp=w.get("noise_temp", 0.0), K_total=K_total, k_offset=k_offset)
+                         noise_temp=w.get("noise_temp", 0.0), K_total=K_total, k_offset=k_offset,
+                         n_conv=w.get("n_conv", 0), img_h=w.get("img", (0, 0))[0], img_w=w.get("img", (0, 0))[1])
 
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
@@ -244,7 +264,8 @@ class OracleSample:
             Ks, Bs, self.steps = ORACLE_SAMPLE[key]
             self.Ks, self.Bs = min(Ks, w["K"]), min(Bs, w["B"])
             cfg = O.make_config(w["model"], widths=w["widths"], K=self.Ks, batch=self.Bs, gemm_dtype=O.GEMM_BF16 if w["bf16"] else O.GEMM_FP32, mu=MU,
-                                gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=w["n"])
+                                gamma=GAMMA, lam=lam, tau=w["tau"], beta=BETA, eta_prime=ETA_PRIME, stale_max=w["stale_max"], seed=0, n_samples=w["n"],
+                                n_conv=w.get("n_conv", 0), img_h=w.get("img", (0, 0))[0], img_w=w.get("img", (0, 0))[1])
             x0 = np.repeat(x0_row[None, :].astype(np.float64), self.Ks, axis=0)
             self.o = O.Oracle(cfg, X, Y, x0, x0_row.astype(np.float64))
             self.sample = f"{self.Ks} of {w['K']} replicas x {self.Bs} of {w['B']} samples per minibatch, full model, {self.steps} step(s) per timing"
@@ -411,7 +432,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
     if with_e2e and not flat:
         nst = min(steps, 8)
         nb = min(nst, 4)
-        fin = w["widths"][0]
+        fin = inp["X"].shape[1]
         t_now = ctx.counters()[0]
         xbs, ybs = [], []
         for i in range(nb):
@@ -541,7 +562,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
 # What the default invocation measures after the headline workload, a few hundred milliseconds each, so that one run carries
 # the whole metric: the optimiser-only sweep at its five sizes and the three smaller model workloads.
 OTHER_WORKLOADS = [("c5", dict(d=1_000_000), 1000), ("c5", dict(d=11_200_000), 300), ("c5", dict(d=25_600_000), 150), ("c5", dict(d=86_000_000), 50),
-                   ("c5", dict(d=256_000_000), 20), ("c1", {}, 95), ("c2", {}, 400), ("c3", {}, 100)]
+                   ("c5", dict(d=256_000_000), 20), ("c1", {}, 95), ("c2", {}, 400), ("c3", {}, 100), ("cnn", {}, 100)]
 
 
 # ---------------------------------------------------------------------------------------------- main

@@ -31,6 +31,7 @@ struct LayerInfo {
   // convolution layer (3x3, stride 1, padding 1, ReLU, 2x2 max-pooling) on H x W feature maps
   bool conv = false;
   int Cin = 0, Cout = 0, H = 0, W = 0;
+  int wg_parts = 1, wg_chunk = 0;     // convolution: the weight gradient's contraction (one term per position and sample) is split over blocks
   int64_t feat_in = 0, feat_out = 0;  // features per sample entering / leaving the layer (dense: in / out)
 };
 
@@ -47,7 +48,7 @@ struct Layout {
   // byte offsets into the workspace
   size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status, gbar1, gbar2;
   size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage, xstage2, ystage2;
-  size_t col[9], parg[9], zout, dzc, dcol;  // convolutional model: patch matrices, pooling choices, pre-pooling output, its gradient, patch-matrix gradient
+  size_t col[9], parg[9], zout, dzc, dcol, wpart;  // convolutional model: patch matrices, pooling choices, pre-pooling output, its gradient, patch-matrix gradient
   size_t total = 0;
 };
 
@@ -163,7 +164,7 @@ bool plan(const lsam_config& c, Layout& L) {
   for (int i = 0; i < 9; ++i) L.act[i] = L.mask[i] = 0;
   L.logits = L.rowloss = L.dz[0] = L.dz[1] = L.dh[0] = L.dh[1] = L.xstage = L.ystage = L.xstage2 = L.ystage2 = 0;
   for (int i = 0; i < 9; ++i) L.col[i] = L.parg[i] = 0;
-  L.zout = L.dzc = L.dcol = 0;
+  L.zout = L.dzc = L.dcol = L.wpart = 0;
   if (!flat) {
     const size_t in0 = L.in0;
     const size_t ldb = L.ldb;
@@ -174,9 +175,9 @@ bool plan(const lsam_config& c, Layout& L) {
     L.xstage2 = take(4 * K * B * in0);  // second slot of the prefetch queue (lsam_stage_batch)
     L.ystage2 = take(4 * K * B);
     if (c.model != LSAM_MODEL_LSQ) {
-      size_t maxw = 0, max_full = 0, max_dcol = 0;
+      size_t maxw = 0, max_full = 0, max_dcol = 0, max_part = 0;
       for (size_t l = 0; l < L.layers.size(); ++l) {
-        const LayerInfo& li = L.layers[l];
+        LayerInfo& li = L.layers[l];
         const size_t w = (size_t)li.feat_out;
         maxw = w > maxw ? w : maxw;
         if (l + 1 < L.layers.size()) {
@@ -190,10 +191,19 @@ bool plan(const lsam_config& c, Layout& L) {
           L.parg[l] = take(K * w * ldb);
           max_full = std::max(max_full, (size_t)li.Cout * P);
           if (l > 0) max_dcol = std::max(max_dcol, (size_t)li.in * P);
+          // weight gradient [Cout, 9 Cin] with P terms per element: enough parts of the contraction for two blocks per SM,
+          // each part at least 8 slabs long and a multiple of the slab
+          const int64_t tiles = ceil_div(li.Cout, kSimtBM) * ceil_div(li.in, kSimtBN) * (int64_t)K;
+          int64_t parts = std::max<int64_t>(1, std::min<int64_t>(ceil_div(2 * 148, tiles), (int64_t)P / (8 * kSimtBK)));
+          const int64_t chunk = round_up(ceil_div((int64_t)P, parts), kSimtBK);
+          parts = ceil_div((int64_t)P, chunk);
+          li.wg_parts = (int)parts; li.wg_chunk = (int)chunk;
+          if (parts > 1) max_part = std::max(max_part, (size_t)parts * li.Cout * li.in);
         }
       }
       if (max_full) { L.zout = take(esz * K * max_full); L.dzc = take(esz * K * max_full); }
       if (max_dcol) L.dcol = take(esz * K * max_dcol);
+      if (max_part) L.wpart = take(4 * K * max_part);
       L.logits = take(4 * K * (size_t)L.layers.back().out * ldb);
       L.rowloss = take(4 * K * B);
       for (int i = 0; i < 2; ++i) L.dz[i] = take(esz * K * maxw * ldb);
@@ -520,18 +530,18 @@ void host_active_mask(const lsam_config& cfg, int64_t t, int64_t budget, std::ve
 
 // ---- SIMT GEMM launches in logical coordinates
 template <typename TA, typename TB, class Epi>
-int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N, int Kd, const Epi& epi) {
-  dim3 grid((unsigned)ceil_div(N, kSimtBN), (unsigned)ceil_div(M, kSimtBM), c->cfg.K);
+int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N, int Kd, const Epi& epi, int parts = 1, int chunk = 0) {
+  dim3 grid((unsigned)ceil_div(N, kSimtBN), (unsigned)ceil_div(M, kSimtBM), c->cfg.K * parts);
   // every operand of the classifier is contiguous either along its rows or along the contraction index
   const bool a_mc = (A.sr == 1), b_nc = (B.sr == 1);
   if (!a_mc && A.sk != 1) return c->fail(LSAM_ERR_INVALID, "SIMT GEMM: operand A has no unit stride");
   if (!b_nc && B.sk != 1) return c->fail(LSAM_ERR_INVALID, "SIMT GEMM: operand B has no unit stride");
   // a tile list shorter than two blocks per SM with a long contraction: two thread groups per block split the contraction
-  const bool split = (int64_t)grid.x * grid.y * grid.z < 2 * 148 && Kd >= 8 * kSimtBK;
+  const bool split = parts == 1 && (int64_t)grid.x * grid.y * grid.z < 2 * 148 && Kd >= 8 * kSimtBK;
 #define LSAM_SIMT(AM, BN_)                                                                                                                        \
   do {                                                                                                                                            \
     if (split) LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 2><<<grid, 512, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));              \
-    else LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 1><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));                    \
+    else LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 1><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act(), parts, chunk));       \
   } while (0)
   if (a_mc) { if (b_nc) LSAM_SIMT(true, true); else LSAM_SIMT(true, false); }
   else      { if (b_nc) LSAM_SIMT(false, true); else LSAM_SIMT(false, false); }
@@ -703,8 +713,16 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
       {
         GemmOperand A{dzc, (int64_t)li.Cout * Pn, Pn, 1};                 // (z, output channel, position)
         GemmOperand Bm{c->at<T>(L.col[l]), (int64_t)li.in * Pn, Pn, 1};   // (z, patch element, position)
-        EpiWgrad e{c->g(), ld, li.w_pad, li.in};
-        if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.Cout, li.in, (int)Pn, e)) != LSAM_OK) return rc;
+        if (li.wg_parts > 1) {
+          // partial products per share of the positions, then their sum in a fixed order
+          EpiPartial e{c->at<float>(L.wpart), li.Cout, li.in};
+          if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.Cout, li.in, (int)Pn, e, li.wg_parts, li.wg_chunk)) != LSAM_OK) return rc;
+          LAUNCH(c, LSAM_PROF_GEMM_WGRAD, sum_parts_kernel<<<dim3((unsigned)ceil_div((int64_t)li.Cout * li.in, 256), K), 256, 0, c->stream>>>(
+              c->at<float>(L.wpart), li.wg_parts, li.Cout, li.in, c->g(), ld, li.w_pad, c->act()));
+        } else {
+          EpiWgrad e{c->g(), ld, li.w_pad, li.in};
+          if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.Cout, li.in, (int)Pn, e)) != LSAM_OK) return rc;
+        }
       }
       if (l > 0) {
         T* dcol = c->at<T>(L.dcol);

@@ -223,11 +223,18 @@ __device__ inline float4 simt_fetch4(const T* __restrict__ base, int64_t sr, int
 // shared-memory tiles (twice the warps per SM for the GEMMs whose tile list is shorter than the machine); at the end group 1
 // hands its accumulators to group 0 through shared memory and group 0 adds them in a fixed order (own + other) and runs the
 // epilogue.  The groups synchronise on their own named barriers (their slab counts may differ by one).
+// parts > 1: the contraction is also split over blocks, for products with a small output and a very long contraction (the weight
+// gradient of a convolution: Cout x 9 Cin outputs, one term per image position and sample).  blockIdx.z = replica * parts + part;
+// part s contracts kk in [s * chunk, (s + 1) * chunk) and hands its result to the epilogue under the index blockIdx.z, which stores
+// the partial products for a second, fixed-order pass (EpiPartial / sum_parts_kernel).
 template <typename TA_, typename TB_, bool A_MC, bool B_NC, class Epi, int SPLITK = 1>
 __global__ void __launch_bounds__(256 * SPLITK)
-gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, const int32_t* __restrict__ active) {
+gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd_all, Epi epi, const int32_t* __restrict__ active, int parts = 1, int chunk = 0) {
   constexpr int BM = kSimtBM, BN = kSimtBN, BK = kSimtBK;
-  if (active != nullptr && !active[blockIdx.z]) return;  // a waiting replica
+  const int z = parts > 1 ? (int)blockIdx.z / parts : (int)blockIdx.z;
+  if (active != nullptr && !active[z]) return;  // a waiting replica
+  const int k_begin = parts > 1 ? ((int)blockIdx.z % parts) * chunk : 0;
+  const int Kd = parts > 1 ? min(Kd_all, k_begin + chunk) : Kd_all;  // end of this block's share of the contraction
   constexpr int A_FLOATS = BK * (BM + 4), B_FLOATS = BK * (BN + 4);
   __shared__ __align__(16) float smem[SPLITK * (A_FLOATS + B_FLOATS)];
   const int grp = SPLITK == 1 ? 0 : (int)threadIdx.x / 256;
@@ -237,7 +244,6 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, c
     if (SPLITK == 1) __syncthreads();
     else asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
   };
-  const int z = blockIdx.z;
   const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
   const TA_* Ap = reinterpret_cast<const TA_*>(A.p) + (int64_t)z * A.sz;
   const TB_* Bp = reinterpret_cast<const TB_*>(Bo.p) + (int64_t)z * Bo.sz;
@@ -285,13 +291,13 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, c
     }
   };
 
-  constexpr int KSTEP = SPLITK * BK;  // a group's slabs: grp * BK, grp * BK + KSTEP, ...
-  if (grp * BK < Kd) {
-    fetch(grp * BK);
+  constexpr int KSTEP = SPLITK * BK;  // a group's slabs: k_begin + grp * BK, + KSTEP, ...
+  if (k_begin + grp * BK < Kd) {
+    fetch(k_begin + grp * BK);
     stash();
   }
   group_sync();
-  for (int k0 = grp * BK; k0 < Kd; k0 += KSTEP) {
+  for (int k0 = k_begin + grp * BK; k0 < Kd; k0 += KSTEP) {
     const bool more = k0 + KSTEP < Kd;
     if (more) fetch(k0 + KSTEP);
 #pragma unroll
@@ -340,9 +346,27 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd, Epi epi, c
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const int gn = n0 + tx * 4 + j;
-      if (gn < N) epi(z, gm, gn, acc[i][j]);
+      if (gn < N) epi((int)blockIdx.z, gm, gn, acc[i][j]);
     }
   }
+}
+
+// partial products of a contraction split over blocks: part[zz][m][n], zz = replica * parts + part
+struct EpiPartial {
+  float* part;  int M, N;
+  __device__ inline void operator()(int zz, int m, int n, float acc) const { part[((int64_t)zz * M + m) * N + n] = acc; }
+};
+// g[z][w_off + m * N + n] = sum over the parts, ascending, of part[z * parts + s][m][n].  grid (ceil(M N / 256), K).
+__global__ void __launch_bounds__(256)
+sum_parts_kernel(const float* __restrict__ part, int parts, int M, int N, float* __restrict__ g, int64_t ld_g, int64_t w_off,
+                 const int32_t* __restrict__ active) {
+  const int z = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (int64_t)M * N) return;
+  float s = 0.f;
+  for (int q = 0; q < parts; ++q) s += part[((int64_t)z * parts + q) * M * N + e];
+  g[(int64_t)z * ld_g + w_off + e] = s;
 }
 
 // ------------------------------------------------------------------------------------------------ softmax cross-entropy
