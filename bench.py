@@ -483,7 +483,9 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
             e2e = dict(value=None, unit=unit, h2d_bytes_per_step=int(8 * K * d), d2h_bytes_per_step=int(12 * K),
                        note="gradient buffers of this sweep point exceed the pinned-memory budget; run --flat-d <= 64000000")
 
-    uses_tc, grads_bf16 = ctx.uses_tcgen05(), ctx.uses_tcgen05() and not grad_fp32
+    uses_tc = ctx.uses_tcgen05()
+    x3 = uses_tc and not w.get("bf16", False)  # fp32 GEMMs as six bf16 plane-pair products on the tensor cores
+    grads_bf16 = uses_tc and not x3 and not grad_fp32
     if rank != 0:
         ctx.close()
         return None
@@ -508,7 +510,12 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
         kern = "update8_kernel" if grads_bf16 else ("update8f_kernel" if (flat and d >= (1 << 22) and d % 8 == 0) else None)
         if kern:
             roof["traffic"], roof["traffic_source"] = ncu_traffic(kern, w["K"], d)
-    if top in ("gemm_fwd", "gemm_dgrad") and uses_tc:
+    if top.startswith("gemm") and x3:
+        # the fp32-equivalent rate against the sustained bf16 rate divided by the six bf16 products each fp32 product costs
+        ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
+        roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"] / 6, unit="TFLOP/s", frac=ach / (pk["bf16_sustained"] / 6),
+                    peak_source=f"{pk['src']} (sustained bf16) / 6 plane-pair products per fp32 product")
+    elif top in ("gemm_fwd", "gemm_dgrad") and uses_tc:
         ach = wk["flops"] / launches_per_step / per_launch_s / 1e12
         roof.update(bound="tensor", achieved=ach, peak=pk["bf16_sustained"], unit="TFLOP/s", frac=ach / pk["bf16_sustained"], peak_source=f"{pk['src']} (sustained bf16)")
     elif top.startswith("gemm") and not uses_tc and not w["bf16"]:
@@ -546,7 +553,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
         cpu, _ = oracle_baseline(w, key, X, Y, inp["y0"].cpu().numpy())
 
     cfgd = workload_config(w)
-    cfgd.update(gemm=("tcgen05 (single-CTA kernels only)" if gemm_impl == G.IMPL_TCGEN05_1CTA else "tcgen05") if uses_tc else "simt", cuda_graph=bool(use_graph),
+    cfgd.update(gemm=("tcgen05, fp32 as three bf16 planes per operand" if x3 else "tcgen05 (single-CTA kernels only)" if gemm_impl == G.IMPL_TCGEN05_1CTA else "tcgen05") if uses_tc else "simt", cuda_graph=bool(use_graph),
                 l2=("working set larger than L2" if not small else "L2-resident state (latency-bound workload)") +
                    ("" if events_in_timed else "; kernel shares and roofline from a separate pass over the same steps with per-launch events"),
                 parallelism=(f"{world * w['K']} workers sharded over {world} GPU(s), one centre, accumulator all-reduce every tau steps" if shard

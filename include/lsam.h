@@ -54,7 +54,13 @@ enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
 /* TCGEN05: tensor-core GEMMs; forward and dgrad with a minibatch tile of 256 samples are run by pairs of CTAs
  * (cta_group::2, 256-row tiles), everything else by single CTAs (128-row tiles); the weight gradient of a minibatch of at
  * most 256 samples keeps its dz block in shared memory over a run of tiles.  TCGEN05_1CTA: single CTAs walking single tiles only;
- * TCGEN05_PAIRS: pairs wherever the kernel supports them (at least 256 rows, minibatch tile of at least 128). */
+ * TCGEN05_PAIRS: pairs wherever the kernel supports them (at least 256 rows, minibatch tile of at least 128).
+ * LSAM_GEMM_FP32 with LSAM_IMPL_TCGEN05 (LSAM_MODEL_MLP, widths multiples of 8): the fp32 GEMMs run on the bf16 tensor cores.
+ * Every GEMM operand a is held as three bf16 planes bf16(a), bf16(a - p0), bf16(a - p0 - p1), whose sum is a, and a product is
+ * the sum of the six plane pairs (i, j) with i + j <= 2 accumulated in fp32 (what is left out is below 2^-24 |a||b| per term):
+ * fp32 results to within the fp32 tolerances of this library, parameters, gradients and optimiser state in fp32 as in the
+ * SIMT path.  AUTO takes this form for an fp32 MLP whose widths allow it and whose largest layer has at least 2^27
+ * multiply-adds per GEMM (K * batch * in * out), and the SIMT kernels otherwise. */
 enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2, LSAM_IMPL_TCGEN05_1CTA = 3, LSAM_IMPL_TCGEN05_PAIRS = 4 };
 /* Stationary kernels k(x, y) = phi(x - y) (Corollary 8 and the remark after it).  The worker's pull is
  * grad_x phi(x - y) = w(r) (x - y), r = ||x_k - y|| with y the centre version the worker reads; the centre update is
@@ -103,7 +109,8 @@ typedef struct {
   int32_t K;          /* worker replicas, the paper's n (Algorithm 2 inputs)                        */
   int32_t batch;      /* per-worker minibatch size B                                                */
   int32_t gemm_dtype; /* LSAM_GEMM_*                                                                */
-  int32_t gemm_impl;  /* LSAM_IMPL_*: AUTO picks tcgen05 for bf16 shapes it supports, else SIMT       */
+  int32_t gemm_impl;  /* LSAM_IMPL_*: AUTO picks tcgen05 for bf16 shapes it supports, else SIMT; a TCGEN05* value
+                         the configuration cannot run on (see above) makes lsam_init return LSAM_ERR_INVALID */
   int32_t nesterov;   /* 1: Nesterov form (Section 4.3); 0: heavy-ball x <- x - eta v               */
   int32_t tau;        /* sync period tau                                                            */
   int32_t stale_max;  /* staleness uniform in [0, stale_max], 0 = every worker reads the current centre; <= 15 */

@@ -258,10 +258,15 @@ constexpr int kTcStageOutBytes = 8 * 4096;  // wgrad epilogue staging: one 32-ro
 constexpr int kTcAstatKBlocks = 4;
 template <int BLOCK_N>
 __host__ __device__ constexpr int tc_astat_stages() { return BLOCK_N == 256 ? 4 : 8; }
-template <int BLOCK_N, bool PAIR = false, bool ASTAT = false>
+// SPLIT (fp32 operands as three bf16 planes each): a stage holds the three planes of the A tile and the three planes of
+// the B tile of one k-block, and feeds six MMA groups (the plane pairs (i, j) with i + j <= 2)
+constexpr int kTcSplitStages = 2;
+constexpr int kTcSplitPairs = 6;
+template <int BLOCK_N, bool PAIR = false, bool ASTAT = false, bool SPLIT = false>
 __host__ __device__ constexpr int tc_smem_bytes() {
-  return (ASTAT ? kTcAstatKBlocks * kTcBlockM * kTcBlockK * 2 + tc_astat_stages<BLOCK_N>() * BLOCK_N * kTcBlockK * 2
-                : tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>()) + 1024 /*alignment slack*/ + 512 /*barriers*/ + kTcStageOutBytes;
+  return (SPLIT ? kTcSplitStages * 3 * tc_stage_bytes<BLOCK_N, false>()
+          : ASTAT ? kTcAstatKBlocks * kTcBlockM * kTcBlockK * 2 + tc_astat_stages<BLOCK_N>() * BLOCK_N * kTcBlockK * 2
+                  : tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>()) + 1024 /*alignment slack*/ + 512 /*barriers*/ + kTcStageOutBytes;
 }
 
 // ------------------------------------------------------------------------------------------------ the kernel
@@ -275,27 +280,40 @@ __host__ __device__ constexpr int tc_smem_bytes() {
 //   tile of the run, so a tile takes in BLOCK_N x Kd instead of (128 + BLOCK_N) x Kd operand elements (the weight gradient is
 //   bound by the rate at which TMA fills shared memory from L2).  A slot is handed back to the producer as soon as the last
 //   tile of the run has used it, so the next run's A block streams in behind the current run's last tile.
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false>
+//   SPLIT (fp32 GEMM on the bf16 tensor cores): every operand tensor is stored as three bf16 planes p0 = bf16(a),
+//   p1 = bf16(a - p0), p2 = bf16(a - p0 - p1), plane p of replica z being "replica" z + p Z of the tensor map.  A stage
+//   holds the three planes of both tiles; the product is the sum of the six plane pairs (i, j), i + j <= 2 (the pairs
+//   left out are below 2^-24 of |a||b|), smallest terms first, all into the same fp32 accumulator.  The epilogues write
+//   their bf16 outputs as three planes again (plane stride Z * M * ldb) and read the bias as the sum of its planes.
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false, bool SPLIT = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
                     int Z, TcEpi ep, int* __restrict__ status, const int32_t* __restrict__ active) {
   static_assert(!PAIR || BLOCK_N >= 128, "the pair form needs 64 rows of B per CTA");
   static_assert(!ASTAT || (!PAIR && !A_MN && !B_MN), "A-stationary form: single CTA, both operands contraction-contiguous");
-  constexpr int STAGES = ASTAT ? tc_astat_stages<BLOCK_N>() : tc_stages<BLOCK_N, PAIR>();
+  static_assert(!SPLIT || (!PAIR && !ASTAT && BLOCK_N <= 128 && EPI <= TC_EPI_WGRAD), "three-plane form: single CTAs, N tile of at most 128, fp32 gradient");
+  constexpr int STAGES = SPLIT ? kTcSplitStages : (ASTAT ? tc_astat_stages<BLOCK_N>() : tc_stages<BLOCK_N, PAIR>());
+  constexpr int NPL = SPLIT ? 3 : 1;  // planes per operand
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
   constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;  // rows of the N side staged by this CTA
   constexpr int B_BYTES = B_ROWS * kTcBlockK * 2;
   constexpr int TILE_M = PAIR ? 2 * kTcBlockM : kTcBlockM;  // rows of a tile of the work list
-  constexpr uint32_t TMEM_COLS = 2 * BLOCK_N;  // two accumulator stages (power of two >= 32)
+  // two accumulator stages (power of two >= 32).  SPLIT: a stage is two accumulators, [BLOCK_N columns: the product of the
+  // leading planes][BLOCK_N columns: the five small plane pairs]; the epilogue adds them.  The tensor core aligns every
+  // addend to the accumulator and drops the bits below its last place, so small terms added to a large running sum lose
+  // their low bits one-sidedly (measured: 9e-6 relative error at a contraction of 784 against 6e-7 with the small terms kept apart).
+  constexpr uint32_t ACC_COLS = SPLIT ? 2 * BLOCK_N : BLOCK_N;
+  constexpr uint32_t TMEM_COLS = 2 * ACC_COLS;
   constexpr uint32_t IDESC = tc::instr_desc(TILE_M, BLOCK_N, A_MN, B_MN);
 
   extern __shared__ uint8_t smem_raw[];
   // round the tile area up to 1024 bytes by pointer arithmetic on the shared array itself (keeps the address space known)
   uint8_t* tiles = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
   // ASTAT: [A slots: kTcAstatKBlocks x A_BYTES][B ring: STAGES x B_BYTES]; else a ring of STAGES x (A tile, B tile)
-  constexpr int RING_STRIDE = ASTAT ? B_BYTES : A_BYTES + B_BYTES;
-  constexpr int RING_B_OFF = ASTAT ? 0 : A_BYTES;
+  // SPLIT: a stage is [A plane 0, 1, 2][B plane 0, 1, 2]
+  constexpr int RING_STRIDE = ASTAT ? B_BYTES : NPL * (A_BYTES + B_BYTES);
+  constexpr int RING_B_OFF = ASTAT ? 0 : NPL * A_BYTES;
   uint8_t* ring = tiles + (ASTAT ? kTcAstatKBlocks * A_BYTES : 0);
   uint8_t* stage = ring + STAGES * RING_STRIDE;  // 1024-byte aligned: everything before it is a multiple of 1024
   uint64_t* bars = reinterpret_cast<uint64_t*>(stage + kTcStageOutBytes);
@@ -400,18 +418,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
               tc::tma_load_3d_pair(b_dst, &map_b, k0, n0, z, bar);
             }
           } else {
-            tc::mbar_expect_tx(&full[s], A_BYTES + B_BYTES);
-            if (A_MN) {
+            tc::mbar_expect_tx(&full[s], NPL * (A_BYTES + B_BYTES));
 #pragma unroll
-              for (int i = 0; i < kTcBlockM / 64; ++i) tc::tma_load_3d(a_dst + i * 8192, &map_a, m0 + 64 * i, k0, z, &full[s]);
-            } else {
-              tc::tma_load_3d(a_dst, &map_a, k0, m0, z, &full[s]);
-            }
-            if (B_MN) {
+            for (int p = 0; p < NPL; ++p) {
+              const int zp = z + p * Z;  // plane p of replica z
+              uint8_t* a_p = a_dst + p * A_BYTES;
+              uint8_t* b_p = b_dst + p * B_BYTES;
+              if (A_MN) {
 #pragma unroll
-              for (int i = 0; i < BLOCK_N / 64; ++i) tc::tma_load_3d(b_dst + i * 8192, &map_b, n0 + 64 * i, k0, z, &full[s]);
-            } else {
-              tc::tma_load_3d(b_dst, &map_b, k0, n0, z, &full[s]);
+                for (int i = 0; i < kTcBlockM / 64; ++i) tc::tma_load_3d(a_p + i * 8192, &map_a, m0 + 64 * i, k0, zp, &full[s]);
+              } else {
+                tc::tma_load_3d(a_p, &map_a, k0, m0, zp, &full[s]);
+              }
+              if (B_MN) {
+#pragma unroll
+                for (int i = 0; i < BLOCK_N / 64; ++i) tc::tma_load_3d(b_p + i * 8192, &map_b, n0 + 64 * i, k0, zp, &full[s]);
+              } else {
+                tc::tma_load_3d(b_p, &map_b, k0, n0, zp, &full[s]);
+              }
             }
           }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
@@ -436,7 +460,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
         if (!tc::mbar_wait(&acc_empty[as], aph ^ 1u, abort_flag)) { ok = false; break; }
         tc::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(as * BLOCK_N);
+        const uint32_t d_tmem = tmem_base + (uint32_t)as * ACC_COLS;
         for (int kb = 0; kb < k_blocks; ++kb) {
           if (ASTAT && nt == nt_begin && !tc::mbar_wait(&a_full[kb], run_ph, abort_flag)) { ok = false; break; }
           if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
@@ -444,14 +468,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const uint32_t a_addr = tc::smem_u32(ASTAT ? tiles + kb * A_BYTES : ring + s * RING_STRIDE);
           const uint32_t b_addr = tc::smem_u32(ring + s * RING_STRIDE + RING_B_OFF);
 #pragma unroll
-          for (int k = 0; k < kTcBlockK / 16; ++k) {
-            // contraction-contiguous tile: rows of 128 B, 8-row groups 1024 B apart, a K = 16 slice is 32 B further along the row;
-            // M/N-contiguous tile: 64-element blocks 8192 B apart (leading offset), 8 contraction rows = 1024 B (stride offset),
-            // a K = 16 slice is two such groups = 2048 B further.
-            const uint64_t ad = A_MN ? tc::smem_desc(a_addr + k * 2048, 8192, 1024) : tc::smem_desc(a_addr + k * 32, 16, 1024);
-            const uint64_t bd = B_MN ? tc::smem_desc(b_addr + k * 2048, 8192, 1024) : tc::smem_desc(b_addr + k * 32, 16, 1024);
-            if (PAIR) tc::umma_bf16_pair(d_tmem, ad, bd, IDESC, (kb | k) != 0 ? 1u : 0u);
-            else tc::umma_bf16(d_tmem, ad, bd, IDESC, (kb | k) != 0 ? 1u : 0u);
+          for (int pp = 0; pp < (SPLIT ? kTcSplitPairs : 1); ++pp) {
+            // SPLIT: plane pairs (A plane, B plane) in the order (0,2) (1,1) (2,0) (0,1) (1,0) into the second accumulator,
+            // then (0,0) into the first
+            const int pa = SPLIT ? (pp < 3 ? pp : (pp < 5 ? pp - 3 : 0)) : 0;
+            const int pb = SPLIT ? (pp < 3 ? 2 - pp : (pp < 5 ? 4 - pp : 0)) : 0;
+            const uint32_t a_pl = a_addr + (uint32_t)(pa * A_BYTES), b_pl = b_addr + (uint32_t)(pb * B_BYTES);
+            const uint32_t d_pp = (SPLIT && pp < 5) ? d_tmem + (uint32_t)BLOCK_N : d_tmem;
+            const int first = (SPLIT && pp == 5) ? 0 : pp;  // 0: this pair opens its accumulator at the first k-block
+#pragma unroll
+            for (int k = 0; k < kTcBlockK / 16; ++k) {
+              // contraction-contiguous tile: rows of 128 B, 8-row groups 1024 B apart, a K = 16 slice is 32 B further along the row;
+              // M/N-contiguous tile: 64-element blocks 8192 B apart (leading offset), 8 contraction rows = 1024 B (stride offset),
+              // a K = 16 slice is two such groups = 2048 B further.
+              const uint64_t ad = A_MN ? tc::smem_desc(a_pl + k * 2048, 8192, 1024) : tc::smem_desc(a_pl + k * 32, 16, 1024);
+              const uint64_t bd = B_MN ? tc::smem_desc(b_pl + k * 2048, 8192, 1024) : tc::smem_desc(b_pl + k * 32, 16, 1024);
+              if (PAIR) tc::umma_bf16_pair(d_pp, ad, bd, IDESC, (kb | k | first) != 0 ? 1u : 0u);
+              else tc::umma_bf16(d_pp, ad, bd, IDESC, (kb | k | first) != 0 ? 1u : 0u);
+            }
           }
           // frees the stage (in both CTAs of a pair) when these MMAs have read it
           if (PAIR) tc::umma_commit_pair(&empty[s]);
@@ -488,17 +522,28 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const int n0 = nt * BLOCK_N;
       if (!tc::mbar_wait(&acc_full[as], aph, abort_flag)) { ok = false; break; }
       tc::tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(as * BLOCK_N);
+      const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)as * ACC_COLS;
       float bias = 0.f;
       float ssq4[4] = {0.f, 0.f, 0.f, 0.f};  // wgrad: sum of squares of this thread's row of the tile, four interleaved partial sums (column mod 4)
       float bsum = 0.f; // dgrad: this thread's share of the bias gradient of its row (samples of its chunks, ascending)
-      if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) bias = to_float(ep.bias[(int64_t)z * ep.ld_p + m]);
+      if ((EPI == TC_EPI_FWD_HIDDEN || EPI == TC_EPI_FWD_HEAD) && m < M) {
+        const bf16* bp = ep.bias + (int64_t)z * ep.ld_p + m;
+        bias = to_float(bp[0]);
+        if (SPLIT) bias = (bias + to_float(bp[(int64_t)Z * ep.ld_p])) + to_float(bp[2 * (int64_t)Z * ep.ld_p]);  // exact: the planes of an fp32 value
+      }
 #pragma unroll 1
       for (int c = 0; c < BLOCK_N / 32; ++c) {
         if (((c >> 1) & 1) != half) continue;  // pairs of blocks alternate between the two warps of a quadrant
         uint32_t r[32];
         tc::tmem_ld32(taddr + (uint32_t)(c * 32), r);
         tc::tmem_ld_wait();
+        if (SPLIT) {
+          uint32_t r2[32];
+          tc::tmem_ld32(taddr + (uint32_t)(BLOCK_N + c * 32), r2);
+          tc::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + __uint_as_float(r2[j]));
+        }
         const int nb = n0 + c * 32;
         if (EPI == TC_EPI_WGRAD_UPD) {
           const int mrow0 = m_base + quad * 32;
@@ -609,7 +654,61 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const int64_t t0 = ((int64_t)z * M + m) * ep.ldb + nb;
           const bool full = nb + 32 <= N;
           const int nvalid = full ? 32 : N - nb;
-          if (EPI == TC_EPI_FWD_HIDDEN) {
+          if (SPLIT && EPI != TC_EPI_FWD_HEAD) {
+            // three-plane outputs: forward  a = relu(acc + bias) with its mask, dgrad  dz_prev = mask ? acc : 0  (no skip paths)
+            uint4 ov[4], mv[2];
+            bf16* ob = reinterpret_cast<bf16*>(ov);
+            uint8_t* mb = reinterpret_cast<uint8_t*>(mv);
+            bf16* dst = (EPI == TC_EPI_FWD_HIDDEN) ? ep.out : ep.dz_prev;
+            if (EPI == TC_EPI_FWD_HIDDEN) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                const float v = __uint_as_float(r[j]) + bias;
+                mb[j] = v > 0.f ? 1 : 0;
+                r[j] = __float_as_uint(v > 0.f ? v : 0.f);
+              }
+              if (full) {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) *reinterpret_cast<uint4*>(ep.mask + t0 + q * 16) = mv[q];
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (j < nvalid) ep.mask[t0 + j] = mb[j];
+              }
+            } else {
+              if (full) {
+#pragma unroll
+                for (int q = 0; q < 2; ++q) mv[q] = *reinterpret_cast<const uint4*>(ep.mask_prev + t0 + q * 16);
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) mb[j] = j < nvalid ? ep.mask_prev[t0 + j] : 0;
+              }
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (!mb[j]) r[j] = 0u;
+              if (ep.bias_g != nullptr) {  // masked entries and entries past the minibatch are zero
+#pragma unroll
+                for (int j = 0; j < 32; ++j) bsum += __uint_as_float(r[j]);
+              }
+            }
+            const int64_t plane = (int64_t)Z * M * ep.ldb;
+#pragma unroll
+            for (int p = 0; p < 3; ++p) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) {
+                ob[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
+                r[j] = __float_as_uint(__uint_as_float(r[j]) - to_float(ob[j]));  // exact: the part the planes so far leave out
+              }
+              if (full) {
+#pragma unroll
+                for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(dst + p * plane + t0 + q * 8) = ov[q];
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                  if (j < nvalid) dst[p * plane + t0 + j] = ob[j];
+              }
+            }
+          } else if (EPI == TC_EPI_FWD_HIDDEN) {
             uint4 skv[4], ov[4], mv[2];
             bf16* skb = reinterpret_cast<bf16*>(skv);
             bf16* ob = reinterpret_cast<bf16*>(ov);
@@ -788,6 +887,8 @@ struct TcBuffers {
   int ldb;
   float* partial; int64_t ld_partial;  // per-replica slots for the fused sum of squares
   bf16* g1b;                           // [Z, ld] bf16 copy of the ascent gradient
+  // fp32 GEMMs on three bf16 planes per operand: xop, act[], dz[] hold three planes each ([3][Z][...], plane-major), g is fp32
+  bool split = false;
 };
 
 struct TcGemm {
@@ -798,6 +899,7 @@ struct TcGemm {
   bool valid = false;
   bool pair = false;  // run by pairs of CTAs (cta_group::2) on 256-row tiles
   bool astat = false; // weight gradient with the A block stationary over runs of n-tiles (ep.run_n)
+  bool split = false; // operands stored as three bf16 planes (fp32 GEMM); single CTAs, N tile of at most 128
 };
 
 struct TcPlan {
@@ -845,7 +947,7 @@ inline bool tc_make_map(CUtensorMap* m, const T* base, uint64_t cols, uint64_t r
              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-inline int tc_pick_block_n(int n) { return n > 128 ? 256 : (n > 64 ? 128 : 64); }
+inline int tc_pick_block_n(int n, bool split = false) { return (n > 128 && !split) ? 256 : (n > 64 ? 128 : 64); }
 // Where the pair form is used: forward and dgrad with a 256-wide minibatch tile (measured at the 4096-wide layers with
 // B = 256: 985 -> 1100 and 945 -> 1030 TFLOP/s inside the step).  It loses with 128-wide minibatch tiles (short kernels: 415 -> 405,
 // 360 -> 335) and in the weight gradient (770 -> 650: with four k-blocks per tile the epilogue is the kernel, and in a pair
@@ -853,11 +955,11 @@ inline int tc_pick_block_n(int n) { return n > 128 ? 256 : (n > 64 ? 128 : 64); 
 inline bool tc_pick_pair(int M, int block_n, bool wgrad, bool force) { return M >= 256 && (force ? block_n >= 128 : (block_n == 256 && !wgrad)); }
 // Partial-sum slots one replica needs when the sum of squares is fused into the weight-gradient epilogue:
 // eight per output tile (one per epilogue warp) plus one per 8 bias units.
-inline int64_t tc_norm_slots(const lsam_config& c) {
+inline int64_t tc_norm_slots(const lsam_config& c, bool split = false) {
   int64_t n = 0;
   for (int l = 0; l < c.n_layers; ++l) {
     const int in = c.widths[l], out = c.widths[l + 1];
-    n += ceil_div(out, kTcBlockM) * ceil_div(in, tc_pick_block_n(in)) * kTcEpiWarps + ceil_div(out, 8);
+    n += ceil_div(out, kTcBlockM) * ceil_div(in, tc_pick_block_n(in, split)) * kTcEpiWarps + ceil_div(out, 8);
   }
   return n;
 }
@@ -878,6 +980,9 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&P.sms, cudaDevAttrMultiProcessorCount, dev);
   const int L = P.n_layers, B = c.batch, Z = c.K;
+  const bool sp = b.split;
+  const uint64_t ZM = sp ? 3 * (uint64_t)Z : (uint64_t)Z;  // "replicas" of an operand tensor map: plane p of replica z is z + p Z
+  if (sp) { P.allow_pair = false; P.allow_astat = false; }
   P.fwd.assign(L, TcGemm()); P.dgrad.assign(L, TcGemm()); P.wgrad.assign(L, TcGemm());
   const uint64_t ldb = (uint64_t)b.ldb;
   P.bias_slot0.assign(L, 0);
@@ -890,10 +995,12 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     bool ok = true;
     {  // forward: A = W [out][in] (in contiguous), B = act_l [in][B] (samples contiguous)
       TcGemm& g = P.fwd[l];
-      g.M = ly.out; g.N = B; g.Kd = ly.in; g.block_n = tc_pick_block_n(B);
+      g.M = ly.out; g.N = B; g.Kd = ly.in; g.block_n = tc_pick_block_n(B, sp); g.split = sp;
+      // three-plane form: a tile list shorter than the machine is cut into 64-sample tiles (twice as many CTAs, each taking in 3/4 of the bytes)
+      if (sp && g.block_n == 128 && (int64_t)Z * ceil_div(g.M, kTcBlockM) * ceil_div(B, 128) < P.sms) g.block_n = 64;
       g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, false, P.force_pair);
-      ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, kTcBlockM);
-      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, 64);
+      ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, ZM, ly.in, b.ld, 64, kTcBlockM);
+      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, ZM, ldb, (uint64_t)ly.in * ldb, 64, 64);
       g.ep.bias = b.xop + ly.b_pad; g.ep.ld_p = b.ld; g.ep.ldb = b.ldb;
       if (head) g.ep.logits = b.logits;
       else { g.ep.out = b.act[l + 1]; g.ep.skip = ly.residual ? b.act[l] : nullptr; g.ep.mask = b.mask[l]; }
@@ -902,13 +1009,13 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     }
     {  // wgrad: A = dz_l [out][B] (samples contiguous = contraction), B = act_l [in][B]
       TcGemm& g = P.wgrad[l];
-      g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in);
+      g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in, sp); g.split = sp;
       g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, true, P.force_pair);
-      ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
-      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, Z, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
+      ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, ZM, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
+      ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, ZM, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
       // the same rows of the bf16 gradient buffer
-      ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
+      if (!sp) ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
       g.astat = P.allow_astat && !g.pair && B <= kTcAstatKBlocks * kTcBlockK;
@@ -931,10 +1038,10 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
     }
     if (l > 0) {  // dgrad: A = W [out][in] read as (m = in contiguous, kd = out), B = dz_l [out][B] (samples contiguous)
       TcGemm& g = P.dgrad[l];
-      g.M = ly.in; g.N = B; g.Kd = ly.out; g.block_n = tc_pick_block_n(B);
+      g.M = ly.in; g.N = B; g.Kd = ly.out; g.block_n = tc_pick_block_n(B, sp); g.split = sp;
       g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, false, P.force_pair);
-      ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, Z, ly.in, b.ld, 64, 64);
-      ok &= tc_make_map(&g.map_b, b.dz[cur], B, ly.out, Z, ldb, (uint64_t)ly.out * ldb, 64, 64);
+      ok &= tc_make_map(&g.map_a, W, ly.in, ly.out, ZM, ly.in, b.ld, 64, 64);
+      ok &= tc_make_map(&g.map_b, b.dz[cur], B, ly.out, ZM, ldb, (uint64_t)ly.out * ldb, 64, 64);
       g.ep.dh_next = ly.residual ? b.dh[(l + 1) & 1] : nullptr;
       g.ep.dh_out = layers[l - 1].residual ? b.dh[l & 1] : nullptr;
       g.ep.dz_prev = b.dz[cur ^ 1]; g.ep.mask_prev = b.mask[l - 1]; g.ep.ldb = b.ldb;
@@ -949,10 +1056,10 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   return 0;
 }
 
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false>
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false, bool SPLIT = false>
 inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
-  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR, ASTAT>;
-  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR, ASTAT>();
+  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR, ASTAT, SPLIT>;
+  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR, ASTAT, SPLIT>();
   // the shared-memory limit of a kernel is a per-device attribute: remember it per device ordinal
   static bool attr_set[64] = {};
   int dev = 0;
@@ -993,6 +1100,14 @@ inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
 template <bool A_MN, bool B_MN, int EPI>
 inline int tc_launch(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
   if (!g.valid) return 1;
+  if constexpr (EPI <= TC_EPI_WGRAD) {
+    if (g.split) {
+      if (g.block_n > 128 || g.pair || g.astat) return 1;
+      return g.block_n == 128 ? tc_launch_one<128, A_MN, B_MN, EPI, false, false, true>(P, g, stream)
+                              : tc_launch_one<64, A_MN, B_MN, EPI, false, false, true>(P, g, stream);
+    }
+  }
+  if (g.split) return 1;
   if (g.pair) {
     switch (g.block_n) {
       case 256: return tc_launch_one<256, A_MN, B_MN, EPI, true>(P, g, stream);

@@ -48,6 +48,10 @@ struct Layout {
   // byte offsets into the workspace
   size_t x, v, g, g1b, g1keep, xpkeep, xop, acc, yring, gprev, tmp, idx, ylab, sched, partial, scalars, status, gbar1, gbar2;
   size_t act[9], mask[9], logits, rowloss, dz[2], dh[2], xstage, ystage, xstage2, ystage2;
+  // fp32 GEMMs on the bf16 tensor cores (LSAM_GEMM_FP32 with LSAM_IMPL_TCGEN05): the parameters the next gradient pass reads,
+  // activations and backward signals are stored as three bf16 planes each; xpl = planes of the parameters [3][K][ld]
+  bool x3 = false;
+  size_t xpl = 0;
   size_t col[9], parg[9], zout, dzc, dcol, wpart;  // convolutional model: patch matrices, pooling choices, pre-pooling output, its gradient, patch-matrix gradient
   size_t total = 0;
 };
@@ -74,6 +78,14 @@ bool plan(const lsam_config& c, Layout& L) {
     return false;
   }
   const bool bf = c.gemm_dtype == LSAM_GEMM_BF16;
+  // fp32 MLP on the tensor cores (three bf16 planes per operand): on request, or by AUTO where the shapes are supported and a layer is
+  // large enough for the tensor-core kernels to win (measured at 784-1024-10, K = 8, B = 128: 0.365 -> 0.238 ms per step)
+  L.x3 = false;
+  if (!bf && c.model == LSAM_MODEL_MLP && c.n_layers >= 1 && c.n_layers <= 8 && c.batch >= 1) {
+    int64_t macs = 0;
+    for (int l = 0; l < c.n_layers; ++l) macs = std::max<int64_t>(macs, (int64_t)c.K * c.batch * c.widths[l] * c.widths[l + 1]);
+    L.x3 = c.gemm_impl == LSAM_IMPL_TCGEN05 || (c.gemm_impl == LSAM_IMPL_AUTO && tc_supported(c) && macs >= ((int64_t)1 << 27));
+  }
   L.seg.n = 0;
   if (c.model == LSAM_MODEL_FLAT) {
     if (c.flat_d < 1 || bf) return false;
@@ -132,7 +144,7 @@ bool plan(const lsam_config& c, Layout& L) {
   // partial-sum slots per replica; FLAT may fall back to scalar chunks when the caller's gradient buffers are misaligned
   L.nchunks = ceil_div(L.ld, (c.model == LSAM_MODEL_FLAT) ? norm_chunk<1>() : norm_chunk<4>());
   if (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) {  // room for the slots of the fused tensor-core norm (the convolutional model runs on the SIMT GEMMs)
-    const int64_t slots = tc_norm_slots(c);
+    const int64_t slots = tc_norm_slots(c, L.x3);
     L.nchunks = slots > L.nchunks ? slots : L.nchunks;
   }
 
@@ -140,6 +152,7 @@ bool plan(const lsam_config& c, Layout& L) {
   auto take = [&](size_t bytes) { size_t o = off; off = (size_t)round_up((int64_t)(off + bytes), 256); return o; };
   const size_t K = c.K, ld = L.ld, B = c.batch > 0 ? c.batch : 1;
   const size_t esz = bf ? 2 : 4;
+  const size_t asz = L.x3 ? 6 : esz;  // activation-like operands: three bf16 planes in the x3 form
   const bool flat = c.model == LSAM_MODEL_FLAT;
   L.status = take(256);
   L.scalars = take(sizeof(float) * 8 * K);  // norm1, norm2, scale, loss (4 x [K], padded)
@@ -151,6 +164,7 @@ bool plan(const lsam_config& c, Layout& L) {
   L.g1keep = (!flat && (c.flags & LSAM_FLAG_KEEP_G1)) ? take(4 * K * ld) : 0;
   L.xpkeep = (!flat && bf && (c.flags & LSAM_FLAG_KEEP_G1)) ? take(esz * K * ld) : 0;  // x~ survives the update
   L.xop = take(esz * K * ld);  // fp32: perturbed point x~;  bf16: operand copy of x, overwritten by x~
+  L.xpl = L.x3 ? take(6 * K * ld) : 0;
   L.acc = take(4 * ld);
   L.yring = take(4 * (size_t)L.ring * ld);
   L.gprev = take(4 * ld);
@@ -169,7 +183,7 @@ bool plan(const lsam_config& c, Layout& L) {
     const size_t in0 = L.in0;
     const size_t ldb = L.ldb;
     // least squares keeps its minibatch sample-major [K, B, in]; the classifiers store everything feature-major [K, width, ldb]
-    L.act[0] = (c.model == LSAM_MODEL_LSQ) ? take(4 * K * B * in0) : take(esz * K * in0 * ldb);
+    L.act[0] = (c.model == LSAM_MODEL_LSQ) ? take(4 * K * B * in0) : take(asz * K * in0 * ldb);
     L.xstage = take(4 * K * B * in0);
     L.ystage = take(4 * K * B);
     L.xstage2 = take(4 * K * B * in0);  // second slot of the prefetch queue (lsam_stage_batch)
@@ -181,7 +195,7 @@ bool plan(const lsam_config& c, Layout& L) {
         const size_t w = (size_t)li.feat_out;
         maxw = w > maxw ? w : maxw;
         if (l + 1 < L.layers.size()) {
-          L.act[l + 1] = take(esz * K * w * ldb);
+          L.act[l + 1] = take(asz * K * w * ldb);
           // ReLU mask: at the resolution before pooling for a convolution
           L.mask[l] = take(K * (li.conv ? (size_t)li.Cout * li.H * li.W : w) * ldb);
         }
@@ -206,7 +220,7 @@ bool plan(const lsam_config& c, Layout& L) {
       if (max_part) L.wpart = take(4 * K * max_part);
       L.logits = take(4 * K * (size_t)L.layers.back().out * ldb);
       L.rowloss = take(4 * K * B);
-      for (int i = 0; i < 2; ++i) L.dz[i] = take(esz * K * maxw * ldb);
+      for (int i = 0; i < 2; ++i) L.dz[i] = take(asz * K * maxw * ldb);
       for (int i = 0; i < 2; ++i) L.dh[i] = take(esz * K * maxw * ldb);
     }
   }
@@ -285,6 +299,8 @@ struct lsam_ctx {
   // per-tick mask of the workers that step; nullptr in lock-step mode (every worker steps every tick)
   const int32_t* act() const { return async_on ? active_buf() : nullptr; }
   int32_t* sched_scratch() const { return at<int32_t>(L.sched) + 4 * cfg.K; }
+  // x3 form: distance between the planes of the gathered minibatch [K, in0, ldb]
+  int64_t in_plane() const { return L.x3 ? (int64_t)cfg.K * L.in0 * L.ldb : 0; }
   float* yslot(int64_t version) const { return at<float>(L.yring) + (size_t)(version % L.ring) * L.ld; }
 
   int fail(int code, const std::string& m) { err = m; return code; }
@@ -391,11 +407,16 @@ int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, 
 
 template <typename TP, typename TG>
 int launch_perturb(lsam_ctx* c, const TG* g, int64_t ldg, int64_t n, bool vec4) {
-  TP* xt = c->at<TP>(c->L.xop);
+  // x3 form (TP = bf16): the perturbed point goes straight into the three planes the descent pass reads; an fp32 copy is kept
+  // only where lsam_read_grads(3) can ask for it
+  const bool x3 = c->L.x3;
+  TP* xt = x3 ? c->at<TP>(c->L.xpl) : c->at<TP>(c->L.xop);
+  const int64_t plane = x3 ? (int64_t)c->cfg.K * c->L.ld : 0;
+  float* xt32 = (x3 && (c->cfg.flags & LSAM_FLAG_KEEP_G1)) ? c->at<float>(c->L.xop) : nullptr;
   const int64_t per = (int64_t)kPertThreads * kPertIter * (vec4 ? 4 : 1);
   dim3 grid((unsigned)ceil_div(n, per), c->cfg.K);
-  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
-  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act()));
+  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act(), plane, xt32));
+  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act(), plane, xt32));
   return LSAM_OK;
 }
 
@@ -432,7 +453,9 @@ UpdateArgs make_update_args(lsam_ctx* c, const void* g, int g_mode, int64_t ldg,
   a.g_mode = g_mode;
   a.active = c->act();
   a.x = c->x(); a.v = c->v(); a.g = g; a.yring = c->at<float>(c->L.yring); a.slot = c->slot();
-  a.acc = c->at<float>(c->L.acc); a.xop = c->at<void>(c->L.xop);
+  a.acc = c->at<float>(c->L.acc);
+  a.xop = c->L.x3 ? c->at<void>(c->L.xpl) : c->at<void>(c->L.xop);
+  a.xop_plane = c->L.x3 ? (int64_t)c->cfg.K * c->L.ld : 0;
   a.ld = c->L.ld; a.ldg = ldg; a.n = n; a.K = c->cfg.K; a.k_offset = c->cfg.k_offset; a.eta = eta; a.mu = c->cfg.mu; a.lambda = c->cfg.lambda;
   a.lam_k = c->cfg.kernel_kind != KERNEL_GAUSSIAN ? c->pull_weight() : nullptr;
   a.sigma = c->cfg.noise_temp > 0.f ? sqrtf(2.0f * eta * c->cfg.noise_temp) : 0.f;
@@ -447,7 +470,7 @@ void* update_func(bool noise) {
 
 int launch_update(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n, bool vec4, float eta) {
   UpdateArgs a = make_update_args(c, g, g_mode, ldg, n, eta);
-  const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16;
+  const bool bf = c->cfg.gemm_dtype == LSAM_GEMM_BF16 || c->L.x3;  // a bf16 operand copy (x3: its three planes) is written with x
   const bool nes = c->cfg.nesterov != 0;
   const bool noise = c->cfg.noise_temp > 0.f;
   unsigned grid = (unsigned)ceil_div(n, (int64_t)kUpdThreads * (vec4 ? 4 : 1));
@@ -595,13 +618,16 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
   // loss and its gradient w.r.t. the logits
   const int C = L.layers[nl - 1].out;
   int cur = 0;
+  // x3 form: backward signals are three planes, (K * width * ldb) elements apart
   LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
-      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act()));
+      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act(),
+      L.x3 ? (int64_t)K * C * ldb : 0));
   if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
   // backward
   for (int l = nl - 1; l >= 0; --l) {
     const LayerInfo& li = L.layers[l];
     const T* dz = c->at<T>(L.dz[cur]);
+    const int64_t dz_plane = L.x3 ? (int64_t)K * li.out * ldb : 0;
     const T* a_in = c->at<T>(L.act[l]);
     // tensor-core path: the dgrad of the layer above has already left this layer's bias gradient (and its sum of squares)
     const bool bias_done = c->use_tc && l < nl - 1 && tc_dgrad_can_fuse_bias(c->tc, l + 1);
@@ -612,7 +638,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
       if (g_bf16)
         LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, bf16><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->at<bf16>(L.g1b), ld, li.b_pad, part, L.nchunks, slot0, c->act()));
       else
-        LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad, part, L.nchunks, slot0, c->act()));
+        LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad, part, L.nchunks, slot0, c->act(), dz_plane));
     }
     if (c->use_tc) {
       int trc = 0;
@@ -772,10 +798,19 @@ int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false,
     return cnn_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out);
   }
   if (cfg.gemm_dtype == LSAM_GEMM_BF16) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xop), loss_out, g_bf16 && c->use_tc, c->use_tc ? fu : nullptr);
+  if (c->L.x3) return mlp_pass<bf16>(c, c->at<bf16>(c->L.xpl), loss_out, false);  // the planes hold x or x~, whichever was split last
   return mlp_pass<float>(c, perturbed ? c->at<float>(c->L.xop) : c->x(), loss_out, false);
 }
 
+// x3 form: the three bf16 planes of src [K, ld] (x, or the perturbed point) -> xpl
+int launch_split3(lsam_ctx* c, const float* src) {
+  dim3 grid((unsigned)ceil_div(c->L.ld, 1024), c->cfg.K);
+  LAUNCH(c, LSAM_PROF_COPY, split3_rows_kernel<<<grid, 256, 0, c->stream>>>(src, c->L.ld, c->L.ld, c->at<bf16>(c->L.xpl), c->L.ld, (int64_t)c->cfg.K * c->L.ld));
+  return LSAM_OK;
+}
+
 int refresh_operand_copy(lsam_ctx* c) {
+  if (c->L.x3) return launch_split3(c, c->x());
   if (c->cfg.gemm_dtype != LSAM_GEMM_BF16) return LSAM_OK;
   dim3 grid((unsigned)ceil_div(c->L.ld, 256), c->cfg.K);
   LAUNCH(c, LSAM_PROF_COPY, cast_rows_kernel<bf16><<<grid, 256, 0, c->stream>>>(c->x(), c->L.ld, c->at<bf16>(c->L.xop), c->L.ld, c->L.ld));
@@ -820,8 +855,8 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
       LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, c->L.in0, c->L.in0, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), cfg.batch, c->act()));
     } else {
       dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
-      if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
+      if (cfg.gemm_dtype == LSAM_GEMM_BF16 || L.x3)
+        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act(), c->in_plane()));
       else
         LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
     }
@@ -881,7 +916,7 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
     const void* g1src = g1_bf16 ? (const void*)c->at<bf16>(L.g1b) : (const void*)g1;
     if ((rc = launch_mean_rows(c, g1src, g1_bf16, ldg, n, vec4, gbar1)) != LSAM_OK) return rc;
     if ((rc = launch_norm(c, gbar1, 0, n, vec4, rho, c->norm1(), c->scale(), false)) != LSAM_OK) return rc;
-    if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, gbar1, 0, n, vec4);
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16 || L.x3) rc = launch_perturb<bf16, float>(c, gbar1, 0, n, vec4);
     else rc = launch_perturb<float, float>(c, gbar1, 0, n, vec4);
   } else {
     if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
@@ -890,7 +925,7 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
       LAUNCH(c, LSAM_PROF_PERTURB, perturb8_kernel<<<pgrid, kPertThreads, 0, c->stream>>>(c->x(), L.ld, c->at<bf16>(L.g1b), ldg, n, c->scale(), c->at<bf16>(L.xop), L.ld, c->act()));
       rc = LSAM_OK;
     } else if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
-    else if (cfg.gemm_dtype == LSAM_GEMM_BF16) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
+    else if (cfg.gemm_dtype == LSAM_GEMM_BF16 || L.x3) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
     else rc = launch_perturb<float, float>(c, g1, ldg, n, vec4);
   }
   if (rc != LSAM_OK) return rc;
@@ -1072,11 +1107,12 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   const bool mlp = cfg->model == LSAM_MODEL_MLP || cfg->model == LSAM_MODEL_RESMLP;
   bool tc_ok = false;
   if (mlp && cfg->gemm_dtype == LSAM_GEMM_BF16 && cfg->gemm_impl != LSAM_IMPL_SIMT) tc_ok = tc_supported(*cfg);
+  if (L.x3) tc_ok = tc_supported(*cfg);  // fp32 GEMMs as three bf16 planes per operand
   if (cfg->gemm_impl >= LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
   c->use_tc = tc_ok;
-  c->grads_bf16 = tc_ok && !(cfg->flags & LSAM_FLAG_GRAD_FP32);
+  c->grads_bf16 = tc_ok && !L.x3 && !(cfg->flags & LSAM_FLAG_GRAD_FP32);
   if (cfg->flags & LSAM_FLAG_FUSED_UPDATE) {
-    if (!tc_ok || cfg->noise_temp > 0.f || cfg->dp_average != 0 || (cfg->flags & LSAM_FLAG_CUDA_GRAPH)) return bail(LSAM_ERR_INVALID);
+    if (!tc_ok || L.x3 || cfg->noise_temp > 0.f || cfg->dp_average != 0 || (cfg->flags & LSAM_FLAG_CUDA_GRAPH)) return bail(LSAM_ERR_INVALID);
     c->fused_update = true;
   }
   {
@@ -1095,7 +1131,8 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   if ((rc = refresh_operand_copy(c)) != LSAM_OK) return bail(rc);
   if (c->use_tc) {
     TcBuffers b;
-    b.xop = c->at<bf16>(L.xop); b.g = c->g(); b.ld = L.ld;
+    b.xop = L.x3 ? c->at<bf16>(L.xpl) : c->at<bf16>(L.xop); b.g = c->g(); b.ld = L.ld;
+    b.split = L.x3;
     for (int i = 0; i < 9; ++i) { b.act[i] = c->at<bf16>(L.act[i]); b.mask[i] = c->at<uint8_t>(L.mask[i]); }
     b.logits = c->at<float>(L.logits);
     for (int i = 0; i < 2; ++i) { b.dz[i] = c->at<bf16>(L.dz[i]); b.dh[i] = c->at<bf16>(L.dh[i]); }
@@ -1139,8 +1176,8 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   LSAM_CUDA(c, cudaMemcpyAsync(c->at<uint32_t>(c->L.ylab), yb, 4 * rows, kind, c->stream));
   if (!lsq) {
     dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
-    if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16 || c->L.x3)
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr, c->in_plane()));
     else
       LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
   }
@@ -1195,8 +1232,8 @@ int lsam_step_staged(lsam_ctx* c, float eta, float rho, float* h_loss) {
     LSAM_CUDA(c, cudaMemcpyAsync(c->at<float>(c->L.act[0]), xs, sizeof(float) * rows * c->L.in0, cudaMemcpyDeviceToDevice, c->stream));
   } else {
     dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
-    if (cfg.gemm_dtype == LSAM_GEMM_BF16)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr));
+    if (cfg.gemm_dtype == LSAM_GEMM_BF16 || c->L.x3)
+      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr, c->in_plane()));
     else
       LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
   }

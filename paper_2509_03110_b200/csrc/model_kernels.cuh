@@ -30,11 +30,32 @@ gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const
 // sample index is the contiguous one (see the layout note above the epilogues).  32 x 32 tiles go through shared
 // memory: reads run along the features of a sample, writes along the samples of a feature.
 // grid (ceil(in / 32), ceil(B / 32), K), block (32, 8).  idx == nullptr: rows come from the dense minibatch src [K, B, in].
+// plane != 0 (TA = bf16): the value is stored as three bf16 planes p0 = bf16(v), p1 = bf16(v - p0), p2 = bf16(v - p0 - p1),
+// `plane` elements apart (fp32 GEMMs on the bf16 tensor cores read their operands in this form).
+template <typename TA>
+__device__ inline void store_planes(TA* p, int64_t plane, float v) {
+  const TA h = from_float<TA>(v);
+  p[0] = h;
+  if (sizeof(TA) == 2 && plane != 0) {
+    float r = v - to_float(h);
+    const TA m = from_float<TA>(r);
+    p[plane] = m;
+    r -= to_float(m);
+    p[2 * plane] = from_float<TA>(r);
+  }
+}
+template <typename TA>
+__device__ inline float load_planes(const TA* p, int64_t plane) {
+  float v = to_float(p[0]);
+  if (sizeof(TA) == 2 && plane != 0) v = (v + to_float(p[plane])) + to_float(p[2 * plane]);  // exact for the planes of an fp32 value
+  return v;
+}
+
 template <typename TA>
 __global__ void __launch_bounds__(256)
 gather_t_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx, int64_t n_samples,
                 int B, int in, int ldb, TA* __restrict__ xt, uint32_t* __restrict__ yb, int* __restrict__ status,
-                const int32_t* __restrict__ active) {
+                const int32_t* __restrict__ active, int64_t plane = 0) {
   __shared__ float tile[32][33];
   if (active != nullptr && !active[blockIdx.z]) return;
   const int k = blockIdx.z, i0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
@@ -55,7 +76,7 @@ gather_t_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, con
   __syncthreads();
   for (int r = threadIdx.y; r < 32; r += 8) {
     const int i = i0 + r, b = b0 + threadIdx.x;
-    if (i < in && b < B) xt[((int64_t)k * in + i) * ldb + b] = from_float<TA>(tile[threadIdx.x][r]);
+    if (i < in && b < B) store_planes(xt + ((int64_t)k * in + i) * ldb + b, plane, tile[threadIdx.x][r]);
   }
 }
 
@@ -378,7 +399,8 @@ sum_parts_kernel(const float* __restrict__ part, int parts, int M, int N, float*
 template <typename TA>
 __global__ void __launch_bounds__(256)
 softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int B, int C, int ldb,
-                  TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status, const int32_t* __restrict__ active) {
+                  TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status, const int32_t* __restrict__ active,
+                  int64_t plane = 0) {
   __shared__ float red[8][33];
   if (active != nullptr && !active[blockIdx.y]) return;
   const int b = blockIdx.x * 32 + threadIdx.x, cg = threadIdx.y, k = blockIdx.y;
@@ -412,7 +434,7 @@ softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ 
   TA* out = dz + (int64_t)k * C * ldb + b;
   for (int c = cg; c < C; c += 8) {
     const float p = expf(lg[(int64_t)c * ldb] - m) * inv;
-    out[(int64_t)c * ldb] = from_float<TA>((p - (c == y ? 1.f : 0.f)) * invB);
+    store_planes(out + (int64_t)c * ldb, plane, (p - (c == y ? 1.f : 0.f)) * invB);
   }
 }
 
@@ -436,7 +458,7 @@ __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float
 template <typename TA, typename TG>
 __global__ void __launch_bounds__(256)
 bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, TG* __restrict__ g, int64_t ld_g, int64_t b_off,
-                 float* __restrict__ partial, int64_t ld_partial, int slot0, const int32_t* __restrict__ active) {
+                 float* __restrict__ partial, int64_t ld_partial, int slot0, const int32_t* __restrict__ active, int64_t plane = 0) {
   __shared__ float sq[8];
   if (active != nullptr && !active[blockIdx.y]) return;
   const int w = threadIdx.x >> 5, o = blockIdx.x * 8 + w;
@@ -444,7 +466,7 @@ bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, TG* __restr
   float s = 0.f;
   if (o < out) {
     const TA* p = dz + ((int64_t)z * out + o) * ldb;
-    for (int b = lane; b < B; b += 32) s += to_float(p[b]);
+    for (int b = lane; b < B; b += 32) s += load_planes(p + b, plane);
     s = warp_sum(s);
     if (lane == 0) g[(int64_t)z * ld_g + b_off + o] = from_float<TG>(s);
   }

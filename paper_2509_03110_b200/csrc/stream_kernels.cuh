@@ -192,6 +192,42 @@ mean_rows_kernel(const TG* g, int64_t ldg, int K, int64_t n, float* out) {
   }
 }
 
+// ------------------------------------------------------------------------------------------------ three bf16 planes of fp32 rows
+// planes[p][k][j], p = 0, 1, 2:  p0 = bf16(a), p1 = bf16(a - p0), p2 = bf16(a - p0 - p1)  for a = src[k][j]  (the operand form of
+// the fp32 GEMMs on the bf16 tensor cores; p0 + p1 + p2 = a exactly unless a part underflows).  n a multiple of 4.
+// grid (ceil(n / 1024), K), block 256.
+// four consecutive values -> plane 0 at dst, and (plane != 0) planes 1 and 2 at dst + plane, dst + 2 plane
+__device__ inline void store_planes4(bf16* dst, int64_t plane, float a, float b, float c, float d) {
+  float r[4] = {a, b, c, d};
+  const int np = plane != 0 ? 3 : 1;
+  for (int p = 0; p < np; ++p) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(r[0], r[1]), hi = __floats2bfloat162_rn(r[2], r[3]);
+    const float2 flo = __bfloat1622float2(lo), fhi = __bfloat1622float2(hi);
+    r[0] -= flo.x; r[1] -= flo.y; r[2] -= fhi.x; r[3] -= fhi.y;
+    uint2 pk;
+    pk.x = *reinterpret_cast<uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(dst + p * plane) = pk;
+  }
+}
+__device__ inline void store_planes1(bf16* dst, int64_t plane, float a) {
+  const int np = plane != 0 ? 3 : 1;
+  for (int p = 0; p < np; ++p) {
+    const bf16 h = __float2bfloat16_rn(a);
+    dst[p * plane] = h;
+    a -= __bfloat162float(h);
+  }
+}
+
+__global__ void __launch_bounds__(256)
+split3_rows_kernel(const float* __restrict__ src, int64_t ld_src, int64_t n, bf16* __restrict__ planes, int64_t ld, int64_t plane) {
+  const int k = blockIdx.y;
+  const int64_t j = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
+  if (j >= n) return;
+  const float4 a = *reinterpret_cast<const float4*>(src + (int64_t)k * ld_src + j);
+  store_planes4(planes + (int64_t)k * ld + j, plane, a.x, a.y, a.z, a.w);
+}
+
 // ------------------------------------------------------------------------------------------------ S4 perturb
 // xt[k][j] = x[k][j] + scale[k] * g[k][j]  (Eq. 3 with scale = rho / (||g|| + gamma)); the master x is not modified.
 // TP = float (fp32 operand) or bf16 (tensor-core operand copy).  grid (chunks, K).
@@ -199,10 +235,13 @@ constexpr int kPertThreads = 256;
 constexpr int kPertIter = 4;
 
 // TG = type of the stored gradient: float, or bf16 where the tensor-core path stores its gradients in bf16 (packed rows of stride ldg).
+// plane != 0 (TP = bf16): the perturbed point is written as three bf16 planes, `plane` elements apart (fp32 GEMMs on the tensor
+// cores); xt32 != nullptr: an fp32 copy of it is kept as well (rows of stride ldt).
 template <int VEC, typename TP, typename TG>
 __global__ void __launch_bounds__(kPertThreads)
 perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ g, int64_t ldg, int64_t n,
-               const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active) {
+               const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active,
+               int64_t plane = 0, float* __restrict__ xt32 = nullptr) {
   const int k = blockIdx.y;
   if (active != nullptr && !active[k]) return;
   const float sc = scale[k];
@@ -236,11 +275,8 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ 
         if (sizeof(TP) == 4) {
           *reinterpret_cast<float4*>(reinterpret_cast<float*>(tr) + j) = make_float4(a, b, c, d);
         } else {
-          __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
-          uint2 pk;
-          pk.x = *reinterpret_cast<uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(tr) + j) = pk;
+          store_planes4(reinterpret_cast<bf16*>(tr) + j, plane, a, b, c, d);
+          if (xt32 != nullptr) *reinterpret_cast<float4*>(xt32 + (int64_t)k * ldt + j) = make_float4(a, b, c, d);
         }
       }
     }
@@ -248,7 +284,15 @@ perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ 
 #pragma unroll
     for (int i = 0; i < kPertIter; ++i) {
       const int64_t j = base + (int64_t)i * kPertThreads + threadIdx.x;
-      if (j < n) tr[j] = from_float<TP>(fmaf(sc, to_float(gr[j]), xr[j]));
+      if (j < n) {
+        const float a = fmaf(sc, to_float(gr[j]), xr[j]);
+        if (sizeof(TP) == 4) {
+          reinterpret_cast<float*>(tr)[j] = a;
+        } else {
+          store_planes1(reinterpret_cast<bf16*>(tr) + j, plane, a);
+          if (xt32 != nullptr) xt32[(int64_t)k * ldt + j] = a;
+        }
+      }
     }
   }
 }
@@ -317,6 +361,7 @@ struct UpdateArgs {
   const int32_t* active;  // nullable [K]: replicas with 0 wait this tick and are left untouched
   float* acc;          // [ld]
   void* xop;           // [K, ld] operand copy (or nullptr)
+  int64_t xop_plane;   // != 0 (bf16 operand copy): three bf16 planes of x, this many elements apart (fp32 GEMMs on the tensor cores)
   int64_t ld, ldg, n;
   int K;
   int k_offset;        // global index of worker 0: the noise streams are keyed by the global worker index
@@ -404,13 +449,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       *reinterpret_cast<float4*>(a.x + o) = xv;
       __stcs(reinterpret_cast<float4*>(a.v + o), vv);
       if (WRITE_OP) {
-        if (sizeof(TP) == 2) {
-          __nv_bfloat162 lo = __floats2bfloat162_rn(xv.x, xv.y), hi = __floats2bfloat162_rn(xv.z, xv.w);
-          uint2 pk;
-          pk.x = *reinterpret_cast<uint32_t*>(&lo);
-          pk.y = *reinterpret_cast<uint32_t*>(&hi);
-          *reinterpret_cast<uint2*>(reinterpret_cast<bf16*>(a.xop) + o) = pk;
-        }
+        if (sizeof(TP) == 2) store_planes4(reinterpret_cast<bf16*>(a.xop) + o, a.xop_plane, xv.x, xv.y, xv.z, xv.w);
       }
       gv = gn; xv = xn; vv = vn; yv = yn;
       k = kn;
@@ -437,7 +476,10 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
       s += xv;
       a.x[o] = xv;
       a.v[o] = vv;
-      if (WRITE_OP) reinterpret_cast<TP*>(a.xop)[o] = from_float<TP>(xv);
+      if (WRITE_OP) {
+        if (sizeof(TP) == 2) store_planes1(reinterpret_cast<bf16*>(a.xop) + o, a.xop_plane, xv);
+        else reinterpret_cast<TP*>(a.xop)[o] = from_float<TP>(xv);
+      }
     }
     a.acc[j] += s;
   }

@@ -236,9 +236,38 @@ def test_classifier_bf16_tcgen05(model, widths, K, B, impl):
     p.close()
 
 
-def test_config2_mlp_784_1024_10_full_shape():
+@pytest.mark.parametrize("widths,K,B", [
+    ((64, 128, 96, 10), 4, 64),        # N tile 64, ragged head (10 outputs), 96-wide layer
+    ((256, 256, 256, 128), 2, 128),    # N tile 128, several contraction blocks, bias gradient out of the dgrad epilogue
+    ((320, 520, 24), 2, 40),           # ragged M tiles, ragged contraction (320 = 5 x 64), ragged minibatch
+    ((128, 264, 40), 3, 300),          # minibatch wider than one N tile (128 + 128 + 44): bias gradient by its own kernel from the planes
+    ((784, 1024, 10), 8, 128),         # the C2 shape
+])
+def test_classifier_fp32_on_the_tensor_cores_with_three_bf16_planes_per_operand(widths, K, B):
+    # fp32 GEMMs as sums of six bf16 plane products: held to the same fp32 tolerances as the SIMT kernels, against the fp32 oracle
+    p = _mlp_pair(G.MODEL_MLP, widths, K, B, n=600, dtype=G.GEMM_FP32, impl=G.IMPL_TCGEN05, tau=4, lam=0.4, seed=5, jitter=0.01)
+    assert p.gpu.uses_tcgen05()
+    _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, what=f"fp32 on tcgen05 {widths}")
+    p.close()
+
+
+def test_fp32_on_the_tensor_cores_is_refused_where_it_is_not_built():
+    import torch
+    X, labels = synth.gaussian_mixture(64, 48, 12, seed=1)
+    for model, widths in [(G.MODEL_RESMLP, (48, 80, 80, 12)), (G.MODEL_MLP, (44, 80, 12))]:  # skip connections; a width that is no multiple of 8
+        w0 = synth.mlp_init(widths, seed=1)
+        Xm = X[:, :widths[0]].copy()
+        with pytest.raises(G.LsamError):
+            G.Lsam(G.make_config(model, widths=widths, K=2, batch=16, gemm_dtype=G.GEMM_FP32, gemm_impl=G.IMPL_TCGEN05, n_samples=64),
+                   torch.from_numpy(Xm).cuda(), torch.from_numpy(labels).cuda(), torch.from_numpy(synth.replicate(w0, 2)).cuda(), torch.from_numpy(w0).cuda())
+
+
+@pytest.mark.parametrize("impl", [G.IMPL_AUTO, G.IMPL_SIMT])
+def test_config2_mlp_784_1024_10_full_shape(impl):
+    # AUTO (what bench.py times): the fp32 GEMMs of this shape run on the tensor cores; SIMT: the fp32 FFMA kernels
     widths = (784, 1024, 10)
-    p = _mlp_pair(G.MODEL_MLP, widths, K=8, B=128, n=60000, dtype=G.GEMM_FP32, tau=4, lam=0.5 / (0.05 * 4), seed=0)
+    p = _mlp_pair(G.MODEL_MLP, widths, K=8, B=128, n=60000, dtype=G.GEMM_FP32, impl=impl, tau=4, lam=0.5 / (0.05 * 4), seed=0)
+    assert p.gpu.uses_tcgen05() == (impl == G.IMPL_AUTO)
     _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, steps=20, forced=2, what="C2")
     p.close()
 
@@ -498,7 +527,7 @@ def test_deterministic_repeat():
 
 
 # ------------------------------------------------------------------------------------------------ asynchronous progress
-@pytest.mark.parametrize("kind", ["flat", "lsq", "mlp_fp32", "mlp_bf16_tcgen05"])
+@pytest.mark.parametrize("kind", ["flat", "lsq", "mlp_fp32", "mlp_fp32_tcgen05", "mlp_bf16_tcgen05"])
 def test_async_progress_masks_bit_exact_and_trajectory(kind):
     # unequal worker progress (Algorithm 2): the per-tick mask and the counters are integers and must agree exactly;
     # waiting replicas must be left untouched bit for bit; the trajectory stays within the usual tolerance
@@ -518,6 +547,11 @@ def test_async_progress_masks_bit_exact_and_trajectory(kind):
     elif kind == "mlp_fp32":
         K = 5
         p = _mlp_pair(G.MODEL_MLP, (40, 64, 48, 6), K, 24, n=300, dtype=G.GEMM_FP32, jitter=0.01, **hp)
+        tol = TOL_TRAJ_FP32
+    elif kind == "mlp_fp32_tcgen05":  # fp32 GEMMs on the tensor cores: waiting replicas are skipped by the plane kernels too
+        K = 5
+        p = _mlp_pair(G.MODEL_MLP, (40, 64, 48, 6), K, 24, n=300, dtype=G.GEMM_FP32, impl=G.IMPL_TCGEN05, jitter=0.01, **hp)
+        assert p.gpu.uses_tcgen05()
         tol = TOL_TRAJ_FP32
     else:
         K = 5
@@ -625,7 +659,7 @@ def test_non_gaussian_kernel_pull_matches_oracle(case, kind, param):
     p.close()
 
 
-@pytest.mark.parametrize("case", ["flat_1001", "lsq", "mlp_fp32", "mlp_bf16_simt", "resmlp_bf16_tcgen05", "resmlp_bf16_tcgen05_gradfp32"])
+@pytest.mark.parametrize("case", ["flat_1001", "lsq", "mlp_fp32", "mlp_fp32_tcgen05", "mlp_bf16_simt", "resmlp_bf16_tcgen05", "resmlp_bf16_tcgen05_gradfp32"])
 @pytest.mark.parametrize("rho", [0.05, 0.0])
 def test_dp_average_matches_oracle_and_keeps_the_replicas_identical(case, rho):
     # synchronous data parallelism (DP-SAM; rho = 0: DP-SGD): both gradients averaged over the workers, workers that start
@@ -708,7 +742,7 @@ def test_rho_zero_takes_the_single_pass_shortcut_and_matches_oracle(dtype, impl)
     p.close()
 
 
-@pytest.mark.parametrize("kind", ["lsq", "mlp_fp32_async", "resmlp_bf16_tcgen05_noise", "flat"])
+@pytest.mark.parametrize("kind", ["lsq", "mlp_fp32_async", "mlp_fp32_tcgen05_async", "resmlp_bf16_tcgen05_noise", "flat"])
 def test_cuda_graph_replay_is_bitwise_identical_to_eager_launches(kind):
     # LSAM_FLAG_CUDA_GRAPH replays each tick as one graph launch; step size, radius, tick, centre-version history and the
     # async budget are refreshed in the executable graph, so the run must equal the eagerly launched one bit for bit
@@ -736,7 +770,7 @@ def test_cuda_graph_replay_is_bitwise_identical_to_eager_launches(kind):
         x0 = synth.replicate(w0, 3, jitter=0.01)
         extra = dict(noise_temp=1e-3) if bf else dict(active_num=170)
         mk = lambda fl: G.Lsam(G.make_config(G.MODEL_RESMLP if bf else G.MODEL_MLP, widths=widths, K=3, batch=48, n_samples=300, flags=fl,
-                                             gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32, **extra, **hp),
+                                             gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32, gemm_impl=G.IMPL_TCGEN05 if "tcgen05" in kind else G.IMPL_AUTO, **extra, **hp),
                                torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda(), torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
     torch.cuda.synchronize()
     stream = torch.cuda.Stream()  # the default stream cannot be captured
