@@ -52,6 +52,7 @@ struct Layout {
   // activations and backward signals are stored as three bf16 planes each; xpl = planes of the parameters [3][K][ld]
   bool x3 = false;
   size_t xpl = 0;
+  size_t hpart = 0;  // narrow head: partial logits [K, chunks, kHeadMaxOut, ldb]
   size_t col[9], parg[9], zout, dzc, dcol, wpart;  // convolutional model: patch matrices, pooling choices, pre-pooling output, its gradient, patch-matrix gradient
   size_t total = 0;
 };
@@ -219,6 +220,7 @@ bool plan(const lsam_config& c, Layout& L) {
       if (max_dcol) L.dcol = take(esz * K * max_dcol);
       if (max_part) L.wpart = take(4 * K * max_part);
       L.logits = take(4 * K * (size_t)L.layers.back().out * ldb);
+      if (L.layers.back().out <= kHeadMaxOut) L.hpart = take(4 * K * (size_t)ceil_div(L.layers.back().in, kHeadChunkIn) * kHeadMaxOut * ldb);
       L.rowloss = take(4 * K * B);
       for (int i = 0; i < 2; ++i) L.dz[i] = take(asz * K * maxw * ldb);
       for (int i = 0; i < 2; ++i) L.dh[i] = take(esz * K * maxw * ldb);
@@ -584,11 +586,21 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
   const int64_t ld = L.ld;
   const int ldb = L.ldb;
   int rc;
+  // a head of at most kHeadMaxOut classes: chunked forward + sum in the loss kernel (SIMT paths and the three-plane form; the
+  // bf16 tensor-core path keeps its GEMM)
+  const bool narrow = L.layers[nl - 1].out <= kHeadMaxOut && (!c->use_tc || L.x3);
+  const int64_t p_plane = L.x3 ? (int64_t)K * ld : 0;
   // forward
   for (int l = 0; l < nl; ++l) {
     const LayerInfo& li = L.layers[l];
     const T* a_in = c->at<T>(L.act[l]);
     const bool head = (l == nl - 1);
+    if (head && narrow) {
+      dim3 hgrid((unsigned)ceil_div(li.in, kHeadChunkIn), (unsigned)ceil_div(B, 128), K);
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, head_chunk_kernel<T><<<hgrid, 128, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, L.x3 ? (int64_t)K * li.in * ldb : 0, P, ld,
+                                                                                     li.w_pad, p_plane, li.in, li.out, B, c->at<float>(L.hpart), c->act()));
+      continue;
+    }
     if (c->use_tc) {
       int trc = 0;
       LAUNCH(c, LSAM_PROF_GEMM_FWD, trc = tc_forward(c->tc, l, c->stream));
@@ -597,16 +609,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
     }
     GemmOperand A{a_in, (int64_t)li.in * ldb, 1, ldb};       // (z, b, i) in the feature-major buffer [z][i][b]
     GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, o, i)
-    if (head && li.out <= kHeadMaxOut) {
-      if (ceil_div(B, 32) * K < 148) {  // too few blocks of 32 samples to fill the machine: 8 samples per block
-        dim3 hgrid((unsigned)ceil_div(B, 8), K);
-        LAUNCH(c, LSAM_PROF_GEMM_FWD, head_forward_kernel<T, 8><<<hgrid, 256, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, P, ld, li.w_pad, li.b_pad, li.in, li.out, B, c->at<float>(L.logits), c->act()));
-      } else {
-        dim3 hgrid((unsigned)ceil_div(B, 32), K);
-        LAUNCH(c, LSAM_PROF_GEMM_FWD, head_forward_kernel<T, 32><<<hgrid, 256, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, P, ld, li.w_pad, li.b_pad, li.in, li.out, B, c->at<float>(L.logits), c->act()));
-      }
-      rc = LSAM_OK;
-    } else if (head) {
+    if (head) {
       EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), li.out, ldb};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
     } else {
@@ -621,7 +624,8 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
   // x3 form: backward signals are three planes, (K * width * ldb) elements apart
   LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
       c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act(),
-      L.x3 ? (int64_t)K * C * ldb : 0));
+      L.x3 ? (int64_t)K * C * ldb : 0, narrow ? c->at<float>(L.hpart) : nullptr, (int)ceil_div(L.layers[nl - 1].in, kHeadChunkIn),
+      P + L.layers[nl - 1].b_pad, ld, p_plane));
   if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
   // backward
   for (int l = nl - 1; l >= 0; --l) {
@@ -690,6 +694,7 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
   const int nl = (int)L.layers.size(), nconv = c->cfg.n_conv;
   const int64_t ld = L.ld;
   const int ldb = L.ldb;  // = B for this model
+  const bool narrow = L.layers[nl - 1].out <= kHeadMaxOut;  // chunked head forward, summed by the loss kernel
   int rc;
   // forward
   for (int l = 0; l < nl; ++l) {
@@ -710,7 +715,12 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
     }
     GemmOperand A{a_in, (int64_t)li.in * ldb, 1, ldb};
     GemmOperand W{P + li.w_pad, ld, li.in, 1};
-    if (head) {
+    if (head && narrow) {
+      dim3 hgrid((unsigned)ceil_div(li.in, kHeadChunkIn), (unsigned)ceil_div(B, 128), K);
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, head_chunk_kernel<T><<<hgrid, 128, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, 0, P, ld, li.w_pad, 0, li.in, li.out, B,
+                                                                                     c->at<float>(L.hpart), c->act()));
+      rc = LSAM_OK;
+    } else if (head) {
       EpiFwdHead<T> e{P + li.b_pad, ld, c->at<float>(L.logits), li.out, ldb};
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
     } else {
@@ -722,7 +732,8 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
   const int C = L.layers[nl - 1].out;
   int cur = 0;
   LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
-      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act()));
+      c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act(),
+      0, narrow ? c->at<float>(L.hpart) : nullptr, (int)ceil_div(L.layers[nl - 1].in, kHeadChunkIn), P + L.layers[nl - 1].b_pad, ld, 0));
   if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
   // backward.  dz[cur] holds, for a dense layer, the gradient w.r.t. its pre-activation; for a convolution layer, the gradient
   // w.r.t. its POOLED output (the pooling and the ReLU are undone by unpool_kernel)

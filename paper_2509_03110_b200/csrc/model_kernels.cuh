@@ -116,69 +116,56 @@ struct EpiFwdHead {
   }
 };
 
-// Forward of a narrow head (out <= kHeadMaxOut classes) on the SIMT path: logits[z][f][b] = bias[f] + sum_i W[z][f][i] a[z][i][b].
-// A 128 x 64 GEMM tile would be almost empty here and leave one block per replica to walk the whole contraction.
-// Instead a block takes 32 samples and walks the inputs in chunks of 256: the chunk's weights are staged in shared
-// memory, then warp w multiplies inputs w, w + 8, ... of the chunk; a lane owns one sample, reads a[i][b] coalesced
-// (eight loads in flight) and the weights as shared-memory broadcasts, and keeps `out` accumulators.  The eight
-// per-warp sums are added in warp order at the end, so the result is deterministic.
+// Forward of a narrow head (out <= kHeadMaxOut classes): logits[z][f][b] = bias[f] + sum_i W[z][f][i] a[z][i][b].
+// A GEMM tile would be almost empty here and leave a handful of blocks to walk the whole contraction.  Instead the
+// contraction is cut into chunks of kHeadChunkIn inputs, one block per (chunk, 128 samples, replica): the chunk's weights
+// are staged in shared memory, a thread owns one sample, reads a[i][b] coalesced (all loads of the chunk in flight at once) and the weights as
+// shared-memory broadcasts, and leaves its `out` partial sums in part[z][chunk][f][b]; softmax_ce_kernel adds the chunks
+// in ascending order on top of the bias, so the result is deterministic.  a_plane / p_plane != 0: activations / parameters
+// are stored as three bf16 planes (their sum is the fp32 value).  grid (chunks, ceil(B / 128), K), block 128.
 constexpr int kHeadMaxOut = 16;
-constexpr int kHeadChunk = 256;
-// SPB = samples per block: 32 (a lane owns a sample) or 8 (a lane owns a sample and one of four interleaved input streams;
-// four times the blocks, for minibatches too small to fill the machine otherwise).
-template <typename T, int SPB>
-__global__ void __launch_bounds__(256)
-head_forward_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, const T* __restrict__ P, int64_t ld_p, int64_t w_off, int64_t b_off,
-                    int in, int out, int B, float* __restrict__ logits, const int32_t* __restrict__ active) {
-  constexpr int QN = 32 / SPB;  // input streams per warp
-  const int z = blockIdx.y;
+constexpr int kHeadChunkIn = 32;
+template <typename T>
+__global__ void __launch_bounds__(128)
+head_chunk_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, int64_t a_plane, const T* __restrict__ P, int64_t ld_p, int64_t w_off,
+                  int64_t p_plane, int in, int out, int B, float* __restrict__ part, const int32_t* __restrict__ active) {
+  const int z = blockIdx.z;
   if (active != nullptr && !active[z]) return;
-  __shared__ float wch[kHeadMaxOut][kHeadChunk];
-  __shared__ float part[8][kHeadMaxOut][32];
-  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  const int sl = lane % SPB, q = lane / SPB;
-  const int b = blockIdx.x * SPB + sl;
-  const bool bv = b < B;
-  const T* az = a + (int64_t)z * a_sz + (bv ? b : 0);
+  __shared__ __align__(16) float w[kHeadChunkIn][kHeadMaxOut];  // [input][class]: a thread reads the 16 weights of an input as four 128-bit broadcasts
+  const int i0 = blockIdx.x * kHeadChunkIn;
+  const int len = min(kHeadChunkIn, in - i0);
+  const int b = blockIdx.y * 128 + threadIdx.x;
+  const bool live = b < B;
+  // every load of the chunk is issued before the first use: one round trip to memory per thread
+  const T* az = a + (int64_t)z * a_sz + (int64_t)i0 * ldb + (live ? b : 0);
+  float av[kHeadChunkIn];
+#pragma unroll
+  for (int u = 0; u < kHeadChunkIn; ++u) av[u] = (live && u < len) ? load_planes(az + (int64_t)u * ldb, a_plane) : 0.f;
   const T* W = P + (int64_t)z * ld_p + w_off;
+  for (int e = threadIdx.x; e < kHeadMaxOut * kHeadChunkIn; e += 128) {
+    const int f = e / kHeadChunkIn, ii = e % kHeadChunkIn;
+    w[ii][f] = (f < out && ii < len) ? load_planes(W + (int64_t)f * in + i0 + ii, p_plane) : 0.f;
+  }
+  __syncthreads();
+  if (!live) return;
   float acc[kHeadMaxOut];
 #pragma unroll
   for (int f = 0; f < kHeadMaxOut; ++f) acc[f] = 0.f;
-  for (int i0 = 0; i0 < in; i0 += kHeadChunk) {
-    const int len = min(kHeadChunk, in - i0);
-    __syncthreads();  // the previous chunk has been consumed
-    for (int e = threadIdx.x; e < kHeadMaxOut * kHeadChunk; e += 256) {
-      const int f = e / kHeadChunk, ii = e % kHeadChunk;
-      wch[f][ii] = (f < out && ii < len) ? to_float(W[(int64_t)f * in + i0 + ii]) : 0.f;
-    }
-    __syncthreads();
-    // inputs past the end of the last chunk have zero weights; their activations are not read
-    for (int ii = w * QN + q; ii < len; ii += 64 * QN) {
-      float av[8];
 #pragma unroll
-      for (int u = 0; u < 8; ++u) av[u] = (ii + 8 * QN * u < len) ? to_float(az[(int64_t)(i0 + ii + 8 * QN * u) * ldb]) : 0.f;
+  for (int u = 0; u < kHeadChunkIn; ++u) {  // inputs past the end of the chunk have zero weights and zero activations
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        const int iu = min(ii + 8 * QN * u, kHeadChunk - 1);
-#pragma unroll
-        for (int f = 0; f < kHeadMaxOut; ++f) acc[f] = fmaf(wch[f][iu], av[u], acc[f]);
-      }
+    for (int q = 0; q < kHeadMaxOut / 4; ++q) {
+      const float4 wv = *reinterpret_cast<const float4*>(&w[u][4 * q]);
+      acc[4 * q] = fmaf(wv.x, av[u], acc[4 * q]);
+      acc[4 * q + 1] = fmaf(wv.y, av[u], acc[4 * q + 1]);
+      acc[4 * q + 2] = fmaf(wv.z, av[u], acc[4 * q + 2]);
+      acc[4 * q + 3] = fmaf(wv.w, av[u], acc[4 * q + 3]);
     }
   }
+  float* dst = part + (((int64_t)z * gridDim.x + blockIdx.x) * kHeadMaxOut) * ldb + b;
 #pragma unroll
-  for (int f = 0; f < kHeadMaxOut; ++f) part[w][f][lane] = acc[f];
-  __syncthreads();
-  for (int e = threadIdx.x; e < out * SPB; e += 256) {
-    const int f = e / SPB, l = e % SPB, bb = blockIdx.x * SPB + l;
-    if (bb >= B) continue;
-    float s = to_float(P[(int64_t)z * ld_p + b_off + f]);
-    // fixed order: warps ascending, input streams ascending
-#pragma unroll
-    for (int qq = 0; qq < 8; ++qq)
-#pragma unroll
-      for (int k2 = 0; k2 < QN; ++k2) s += part[qq][f][k2 * SPB + l];
-    logits[((int64_t)z * out + f) * ldb + bb] = s;
-  }
+  for (int f = 0; f < kHeadMaxOut; ++f)
+    if (f < out) dst[(int64_t)f * ldb] = acc[f];
 }
 
 // dgrad of layer l: dh = TA(acc + skip_grad);  dz_prev = mask_prev ? dh : 0;  optionally keep dh (residual nets)
@@ -398,13 +385,24 @@ sum_parts_kernel(const float* __restrict__ part, int parts, int M, int N, float*
 // grid (ceil(B / 32), K), block (32, 8).
 template <typename TA>
 __global__ void __launch_bounds__(256)
-softmax_ce_kernel(const float* __restrict__ logits, const int32_t* __restrict__ labels, int B, int C, int ldb,
+softmax_ce_kernel(float* logits, const int32_t* __restrict__ labels, int B, int C, int ldb,
                   TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status, const int32_t* __restrict__ active,
-                  int64_t plane = 0) {
+                  int64_t plane = 0, const float* __restrict__ part = nullptr, int nparts = 0, const TA* __restrict__ bias = nullptr,
+                  int64_t ld_p = 0, int64_t p_plane = 0) {
   __shared__ float red[8][33];
   if (active != nullptr && !active[blockIdx.y]) return;
   const int b = blockIdx.x * 32 + threadIdx.x, cg = threadIdx.y, k = blockIdx.y;
   const bool live = b < B;
+  if (part != nullptr) {
+    // narrow head (head_chunk_kernel): the logits are the bias plus the partial sums of the input chunks, in ascending order
+    if (live)
+      for (int c = cg; c < C; c += 8) {
+        float v = load_planes(bias + (int64_t)k * ld_p + c, p_plane);
+        for (int p = 0; p < nparts; ++p) v += part[(((int64_t)k * nparts + p) * kHeadMaxOut + c) * ldb + b];
+        logits[((int64_t)k * C + c) * ldb + b] = v;
+      }
+    __syncthreads();  // a sample's classes are spread over the eight thread rows of this block
+  }
   const float* lg = logits + (int64_t)k * C * ldb + (live ? b : 0);
   float m = -INFINITY;
   if (live)
