@@ -116,7 +116,7 @@ def _rank(rank, world, port, out):
 
 def test_exchange_helper_two_gloo_ranks(oracle_mod):
     port = _free_port()
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_rank, args=(2, port, out), nprocs=2, join=True)
         res = dict(out)
