@@ -256,8 +256,9 @@ constexpr int kTcStageOutBytes = 8 * 4096;  // wgrad epilogue staging: one 32-ro
 // ASTAT (A-stationary, contraction of at most kTcAstatKBlocks k-blocks): the whole A block of a tile row stays in shared
 // memory for a run of n-tiles, the ring holds B tiles only
 constexpr int kTcAstatKBlocks = 4;
-template <int BLOCK_N>
-__host__ __device__ constexpr int tc_astat_stages() { return BLOCK_N == 256 ? 4 : 8; }
+// PAIR: a CTA stages half the rows of a B tile, so the ring is twice as deep in the same space
+template <int BLOCK_N, bool PAIR = false>
+__host__ __device__ constexpr int tc_astat_stages() { return (BLOCK_N == 256 && !PAIR) ? 4 : 8; }
 // SPLIT (fp32 operands as three bf16 planes each): a stage holds the three planes of the A tile and the three planes of
 // the B tile of one k-block, and feeds six MMA groups (the plane pairs (i, j) with i + j <= 2)
 constexpr int kTcSplitStages = 2;
@@ -265,7 +266,7 @@ constexpr int kTcSplitPairs = 6;
 template <int BLOCK_N, bool PAIR = false, bool ASTAT = false, bool SPLIT = false>
 __host__ __device__ constexpr int tc_smem_bytes() {
   return (SPLIT ? kTcSplitStages * 3 * tc_stage_bytes<BLOCK_N, false>()
-          : ASTAT ? kTcAstatKBlocks * kTcBlockM * kTcBlockK * 2 + tc_astat_stages<BLOCK_N>() * BLOCK_N * kTcBlockK * 2
+          : ASTAT ? kTcAstatKBlocks * kTcBlockM * kTcBlockK * 2 + tc_astat_stages<BLOCK_N, PAIR>() * (PAIR ? BLOCK_N / 2 : BLOCK_N) * kTcBlockK * 2
                   : tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>()) + 1024 /*alignment slack*/ + 512 /*barriers*/ + kTcStageOutBytes;
 }
 
@@ -291,9 +292,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
                     int Z, TcEpi ep, int* __restrict__ status, const int32_t* __restrict__ active) {
   static_assert(!PAIR || BLOCK_N >= 128, "the pair form needs 64 rows of B per CTA");
-  static_assert(!ASTAT || (!PAIR && !A_MN && !B_MN), "A-stationary form: single CTA, both operands contraction-contiguous");
+  static_assert(!ASTAT || (!A_MN && !B_MN), "A-stationary form: both operands contraction-contiguous");
   static_assert(!SPLIT || (!PAIR && !ASTAT && BLOCK_N <= 128 && EPI <= TC_EPI_WGRAD), "three-plane form: single CTAs, N tile of at most 128, fp32 gradient");
-  constexpr int STAGES = SPLIT ? kTcSplitStages : (ASTAT ? tc_astat_stages<BLOCK_N>() : tc_stages<BLOCK_N, PAIR>());
+  constexpr int STAGES = SPLIT ? kTcSplitStages : (ASTAT ? tc_astat_stages<BLOCK_N, PAIR>() : tc_stages<BLOCK_N, PAIR>());
   constexpr int NPL = SPLIT ? 3 : 1;  // planes per operand
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
   constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;  // rows of the N side staged by this CTA
@@ -390,15 +391,24 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         for (int kb = 0; kb < k_blocks; ++kb) {
           const int k0 = kb * kTcBlockK;
           if (ASTAT && nt == nt_begin) {
-            // first tile of a run: bring in A slot kb as soon as the previous run has released it
+            // first tile of a run: bring in A slot kb as soon as the previous run has released it (pair form: each CTA its own
+            // 128 rows into its own slot, both loads completing on the leader's barrier, which the leader arms with the bytes of both)
             if (!tc::mbar_wait(&a_empty[kb], run_ph ^ 1u, abort_flag)) { ok = false; break; }
-            tc::mbar_expect_tx(&a_full[kb], A_BYTES);
-            tc::tma_load_3d(tiles + kb * A_BYTES, &map_a, k0, m0, z, &a_full[kb]);
+            if (PAIR) {
+              if (leader) tc::mbar_expect_tx(&a_full[kb], 2 * A_BYTES);
+              tc::tma_load_3d_pair(tiles + kb * A_BYTES, &map_a, k0, m0, z, tc::map_to_cta(tc::smem_u32(&a_full[kb]), 0u));
+            } else {
+              tc::mbar_expect_tx(&a_full[kb], A_BYTES);
+              tc::tma_load_3d(tiles + kb * A_BYTES, &map_a, k0, m0, z, &a_full[kb]);
+            }
           }
           if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* a_dst = ring + s * RING_STRIDE;
           uint8_t* b_dst = a_dst + RING_B_OFF;
-          if (ASTAT) {
+          if (ASTAT && PAIR) {
+            if (leader) tc::mbar_expect_tx(&full[s], 2 * B_BYTES);
+            tc::tma_load_3d_pair(b_dst, &map_b, k0, n0, z, tc::map_to_cta(tc::smem_u32(&full[s]), 0u));
+          } else if (ASTAT) {
             tc::mbar_expect_tx(&full[s], B_BYTES);
             tc::tma_load_3d(b_dst, &map_b, k0, n0, z, &full[s]);
           } else if (PAIR) {
@@ -490,7 +500,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           // frees the stage (in both CTAs of a pair) when these MMAs have read it
           if (PAIR) tc::umma_commit_pair(&empty[s]);
           else tc::umma_commit(&empty[s]);
-          if (ASTAT && nt == nt_end - 1) tc::umma_commit(&a_empty[kb]);  // last tile of the run: the A slot is free once these MMAs are done
+          if (ASTAT && nt == nt_end - 1) {  // last tile of the run: the A slot (of both CTAs of a pair) is free once these MMAs are done
+            if (PAIR) tc::umma_commit_pair(&a_empty[kb]);
+            else tc::umma_commit(&a_empty[kb]);
+          }
           if (++s == STAGES) { s = 0; ph ^= 1u; }
         }
         if (!ok) break;
@@ -913,6 +926,7 @@ struct TcPlan {
   bool allow_pair = true;       // false: every GEMM on the single-CTA kernels
   bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
   bool allow_astat = true;      // false: the weight gradient walks single tiles
+  bool pair_wgrad = false;      // true: the weight gradient of wide layers by pairs of CTAs with the dz block stationary (measured slower, see tc_pick_pair)
   int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
 };
 
@@ -951,7 +965,8 @@ inline int tc_pick_block_n(int n, bool split = false) { return (n > 128 && !spli
 // Where the pair form is used: forward and dgrad with a 256-wide minibatch tile (measured at the 4096-wide layers with
 // B = 256: 985 -> 1100 and 945 -> 1030 TFLOP/s inside the step).  It loses with 128-wide minibatch tiles (short kernels: 415 -> 405,
 // 360 -> 335) and in the weight gradient (770 -> 650: with four k-blocks per tile the epilogue is the kernel, and in a pair
-// the slower of the two epilogues gates both CTAs), so those keep the single-CTA kernels; `force` (tests) pairs whatever can be.
+// the slower of the two epilogues gates both CTAs; the same 650 with the dz block stationary on top, which halves what a CTA takes in:
+// the weight gradient is not bound by its operand loads), so those keep the single-CTA kernels; `force` (tests) pairs whatever can be.
 inline bool tc_pick_pair(int M, int block_n, bool wgrad, bool force) { return M >= 256 && (force ? block_n >= 128 : (block_n == 256 && !wgrad)); }
 // Partial-sum slots one replica needs when the sum of squares is fused into the weight-gradient epilogue:
 // eight per output tile (one per epilogue warp) plus one per 8 bias units.
@@ -1011,6 +1026,11 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       TcGemm& g = P.wgrad[l];
       g.M = ly.out; g.N = ly.in; g.Kd = B; g.block_n = tc_pick_block_n(ly.in, sp); g.split = sp;
       g.pair = P.allow_pair && tc_pick_pair(g.M, g.block_n, true, P.force_pair);
+      // a minibatch of at most 256 samples (four k-blocks): the dz block stays in shared memory over a run of tiles; with 256-wide
+      // tiles a pair of CTAs shares each activation tile on top of that (each CTA takes in half of it)
+      const bool astat_ok = P.allow_astat && B <= kTcAstatKBlocks * kTcBlockK;
+      if (P.allow_pair && P.pair_wgrad && astat_ok && g.M >= 256 && g.block_n == 256) g.pair = true;
+      g.astat = astat_ok && (!g.pair || g.block_n >= 128);
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, ZM, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, ZM, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
@@ -1018,16 +1038,17 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       if (!sp) ok &= tc_make_map(&g.map_c16, b.g1b + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 64, 32);
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
-      g.astat = P.allow_astat && !g.pair && B <= kTcAstatKBlocks * kTcBlockK;
       g.ep.run_n = 1;
       if (g.astat) {
-        // run length: a unit of the list costs run_n B tiles plus one A block (half a B tile at BLOCK_N = 256); the SMs work through
-        // ceil(units / SMs) rounds of units.  Pick the run length with the least bytes through the busiest SM.
-        const int64_t rows = (int64_t)Z * ceil_div(g.M, kTcBlockM), n_tiles = ceil_div(g.N, g.block_n);
+        // run length: a unit of the list costs a CTA run_n B tiles (half tiles in a pair) plus one A block of 128 rows; the SMs (pairs of SMs)
+        // work through ceil(units / SMs) rounds of units.  Pick the run length with the least bytes through the busiest SM.
+        const int64_t rows = (int64_t)Z * ceil_div(g.M, g.pair ? 2 * kTcBlockM : kTcBlockM), n_tiles = ceil_div(g.N, g.block_n);
+        const int64_t workers = g.pair ? P.sms / 2 : P.sms;
+        const double b_rows = g.pair ? g.block_n / 2 : g.block_n;
         double best = 0.0;
         for (int rn = 1; rn <= n_tiles; ++rn) {
           const int64_t units = rows * ceil_div(n_tiles, (int64_t)rn);
-          const double cost = (double)ceil_div(units, (int64_t)P.sms) * ((double)rn * g.block_n + kTcBlockM);
+          const double cost = (double)ceil_div(units, workers) * ((double)rn * b_rows + kTcBlockM);
           if (rn == 1 || cost < best) { best = cost; g.ep.run_n = rn; }
         }
       }
@@ -1109,6 +1130,14 @@ inline int tc_launch(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
   }
   if (g.split) return 1;
   if (g.pair) {
+    if constexpr (tc_epi_is_wgrad(EPI) && !A_MN && !B_MN) {
+      if (g.astat) {
+        switch (g.block_n) {
+          case 256: return tc_launch_one<256, A_MN, B_MN, EPI, true, true>(P, g, stream);
+          default: return tc_launch_one<128, A_MN, B_MN, EPI, true, true>(P, g, stream);
+        }
+      }
+    }
     switch (g.block_n) {
       case 256: return tc_launch_one<256, A_MN, B_MN, EPI, true>(P, g, stream);
       default: return tc_launch_one<128, A_MN, B_MN, EPI, true>(P, g, stream);
