@@ -55,7 +55,8 @@ enum { LSAM_GEMM_FP32 = 0, LSAM_GEMM_BF16 = 1 };
  * (cta_group::2, 256-row tiles), everything else by single CTAs (128-row tiles); the weight gradient of a minibatch of at
  * most 256 samples keeps its dz block in shared memory over a run of tiles.  TCGEN05_1CTA: single CTAs walking single tiles only;
  * TCGEN05_PAIRS: pairs wherever the kernel supports them (at least 256 rows, minibatch tile of at least 128).
- * LSAM_GEMM_FP32 with LSAM_IMPL_TCGEN05 (LSAM_MODEL_MLP, widths multiples of 8): the fp32 GEMMs run on the bf16 tensor cores.
+ * LSAM_GEMM_FP32 with LSAM_IMPL_TCGEN05 (LSAM_MODEL_MLP and LSAM_MODEL_RESMLP, every layer's input width a multiple of 8): the fp32 GEMMs
+ * run on the bf16 tensor cores.
  * Every GEMM operand a is held as three bf16 planes bf16(a), bf16(a - p0), bf16(a - p0 - p1), whose sum is a, and a product is
  * the sum of the six plane pairs (i, j) with i + j <= 2 accumulated in fp32 (what is left out is below 2^-24 |a||b| per term):
  * fp32 results to within the fp32 tolerances of this library, parameters, gradients and optimiser state in fp32 as in the
@@ -72,7 +73,7 @@ enum { LSAM_IMPL_AUTO = 0, LSAM_IMPL_SIMT = 1, LSAM_IMPL_TCGEN05 = 2, LSAM_IMPL_
  * A non-Gaussian kernel costs one more pass over x per tick (the distances r_k, fixed-order reduction).           */
 enum { LSAM_KERNEL_GAUSSIAN = 0, LSAM_KERNEL_EXP_POWER = 1, LSAM_KERNEL_CAUCHY = 2, LSAM_KERNEL_MATERN32 = 3 };
 enum {
-  LSAM_FLAG_KEEP_G1 = 1,   /* keep copies of the ascent gradient and (BF16 mode) of x~ for lsam_read_grads  */
+  LSAM_FLAG_KEEP_G1 = 1,   /* keep copies of the ascent gradient and (BF16 mode, fp32 GEMMs on the tensor cores) of x~ for lsam_read_grads */
   LSAM_FLAG_STEP_INFO = 2, /* also reduce ||g2_k|| every step (one extra read of the gradient buffer)      */
   LSAM_FLAG_CUDA_GRAPH = 4, /* replay each tick as one CUDA graph launch (recorded at the second tick of each variant;
                               for launch-bound small models); needs a non-default stream (lsam_init fails with
@@ -217,7 +218,8 @@ int lsam_read_step_info(lsam_ctx* ctx, float* h_loss, float* h_gnorm1, float* h_
 int lsam_read_anchor_gap(lsam_ctx* ctx, float* h_gap);
 /* Of the last step: pass = 1 ascent gradient (needs LSAM_FLAG_KEEP_G1), 2 descent gradient, 3 perturbed point x~
  * (as stored: rounded to bf16 in BF16 mode, where it also needs LSAM_FLAG_KEEP_G1 because the operand buffer
- * is reused by the update).  h_dst [K, d] unpadded, host.  Synchronises. */
+ * is reused by the update; the same holds for fp32 GEMMs on the tensor cores, whose operand planes are reused).
+ * h_dst [K, d] unpadded, host; LSAM_ERR_STATE where the flag is missing.  Synchronises. */
 int lsam_read_grads(lsam_ctx* ctx, int pass, float* h_dst);
 /* Same for the single replica k: h_dst [d]. */
 int lsam_read_grads_replica(lsam_ctx* ctx, int pass, int k, float* h_dst);

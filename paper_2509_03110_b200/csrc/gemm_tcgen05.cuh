@@ -668,11 +668,49 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           const bool full = nb + 32 <= N;
           const int nvalid = full ? 32 : N - nb;
           if (SPLIT && EPI != TC_EPI_FWD_HEAD) {
-            // three-plane outputs: forward  a = relu(acc + bias) with its mask, dgrad  dz_prev = mask ? acc : 0  (no skip paths)
+            // three-plane outputs: forward  a = skip + relu(acc + bias) with its mask; dgrad  dh = acc + dh_next,  dz_prev = mask ? dh : 0
             uint4 ov[4], mv[2];
             bf16* ob = reinterpret_cast<bf16*>(ov);
             uint8_t* mb = reinterpret_cast<uint8_t*>(mv);
-            bf16* dst = (EPI == TC_EPI_FWD_HIDDEN) ? ep.out : ep.dz_prev;
+            const int64_t plane = (int64_t)Z * M * ep.ldb;
+            float rr[32];
+            // r[j] += the fp32 value held in the three planes at src: the planes are summed first (exact), so the accumulator
+            // takes one fp32 addition of the stored value
+            auto add_planes = [&](const bf16* src) {
+#pragma unroll
+              for (int p = 0; p < 3; ++p) {
+                if (full) {
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) ov[q] = *reinterpret_cast<const uint4*>(src + p * plane + t0 + q * 8);
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j) ob[j] = j < nvalid ? src[p * plane + t0 + j] : __float2bfloat16_rn(0.f);
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) rr[j] = p == 0 ? to_float(ob[j]) : rr[j] + to_float(ob[j]);
+              }
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) + rr[j]);
+            };
+            // the three planes of rr[j] -> dst (rr is used up)
+            auto store_planes = [&](bf16* dst) {
+#pragma unroll
+              for (int p = 0; p < 3; ++p) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                  ob[j] = __float2bfloat16_rn(rr[j]);
+                  rr[j] -= to_float(ob[j]);  // exact: the part the planes so far leave out
+                }
+                if (full) {
+#pragma unroll
+                  for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(dst + p * plane + t0 + q * 8) = ov[q];
+                } else {
+#pragma unroll
+                  for (int j = 0; j < 32; ++j)
+                    if (j < nvalid) dst[p * plane + t0 + j] = ob[j];
+                }
+              }
+            };
             if (EPI == TC_EPI_FWD_HIDDEN) {
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
@@ -688,7 +726,17 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 for (int j = 0; j < 32; ++j)
                   if (j < nvalid) ep.mask[t0 + j] = mb[j];
               }
+              if (ep.skip != nullptr) add_planes(ep.skip);
+#pragma unroll
+              for (int j = 0; j < 32; ++j) rr[j] = __uint_as_float(r[j]);
+              store_planes(ep.out);
             } else {
+              if (ep.dh_next != nullptr) add_planes(ep.dh_next);
+              if (ep.dh_out != nullptr) {
+#pragma unroll
+                for (int j = 0; j < 32; ++j) rr[j] = __uint_as_float(r[j]);
+                store_planes(ep.dh_out);
+              }
               if (full) {
 #pragma unroll
                 for (int q = 0; q < 2; ++q) mv[q] = *reinterpret_cast<const uint4*>(ep.mask_prev + t0 + q * 16);
@@ -697,29 +745,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                 for (int j = 0; j < 32; ++j) mb[j] = j < nvalid ? ep.mask_prev[t0 + j] : 0;
               }
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (!mb[j]) r[j] = 0u;
+              for (int j = 0; j < 32; ++j) rr[j] = mb[j] ? __uint_as_float(r[j]) : 0.f;
               if (ep.bias_g != nullptr) {  // masked entries and entries past the minibatch are zero
 #pragma unroll
-                for (int j = 0; j < 32; ++j) bsum += __uint_as_float(r[j]);
+                for (int j = 0; j < 32; ++j) bsum += rr[j];
               }
-            }
-            const int64_t plane = (int64_t)Z * M * ep.ldb;
-#pragma unroll
-            for (int p = 0; p < 3; ++p) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) {
-                ob[j] = __float2bfloat16_rn(__uint_as_float(r[j]));
-                r[j] = __float_as_uint(__uint_as_float(r[j]) - to_float(ob[j]));  // exact: the part the planes so far leave out
-              }
-              if (full) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) *reinterpret_cast<uint4*>(dst + p * plane + t0 + q * 8) = ov[q];
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                  if (j < nvalid) dst[p * plane + t0 + j] = ob[j];
-              }
+              store_planes(ep.dz_prev);
             }
           } else if (EPI == TC_EPI_FWD_HIDDEN) {
             uint4 skv[4], ov[4], mv[2];

@@ -82,7 +82,7 @@ bool plan(const lsam_config& c, Layout& L) {
   // fp32 MLP on the tensor cores (three bf16 planes per operand): on request, or by AUTO where the shapes are supported and a layer is
   // large enough for the tensor-core kernels to win (measured at 784-1024-10, K = 8, B = 128: 0.365 -> 0.238 ms per step)
   L.x3 = false;
-  if (!bf && c.model == LSAM_MODEL_MLP && c.n_layers >= 1 && c.n_layers <= 8 && c.batch >= 1) {
+  if (!bf && (c.model == LSAM_MODEL_MLP || c.model == LSAM_MODEL_RESMLP) && c.n_layers >= 1 && c.n_layers <= 8 && c.batch >= 1) {
     int64_t macs = 0;
     for (int l = 0; l < c.n_layers; ++l) macs = std::max<int64_t>(macs, (int64_t)c.K * c.batch * c.widths[l] * c.widths[l + 1]);
     L.x3 = c.gemm_impl == LSAM_IMPL_TCGEN05 || (c.gemm_impl == LSAM_IMPL_AUTO && tc_supported(c) && macs >= ((int64_t)1 << 27));
@@ -223,7 +223,7 @@ bool plan(const lsam_config& c, Layout& L) {
       if (L.layers.back().out <= kHeadMaxOut) L.hpart = take(4 * K * (size_t)ceil_div(L.layers.back().in, kHeadChunkIn) * kHeadMaxOut * ldb);
       L.rowloss = take(4 * K * B);
       for (int i = 0; i < 2; ++i) L.dz[i] = take(asz * K * maxw * ldb);
-      for (int i = 0; i < 2; ++i) L.dh[i] = take(esz * K * maxw * ldb);
+      for (int i = 0; i < 2; ++i) L.dh[i] = take(asz * K * maxw * ldb);
     }
   }
   L.total = off;
@@ -1367,6 +1367,8 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
         dim3 grid((unsigned)ceil_div(maxlen, 256), L.seg.n, 1);
         LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(c->at<bf16>(L.xpkeep) + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
       } else {
+        // fp32 GEMMs on the tensor cores: the perturbed point lives in the three operand planes, which the update overwrites; an fp32 copy is kept on request
+        if (L.x3 && !(c->cfg.flags & LSAM_FLAG_KEEP_G1)) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(3) with fp32 GEMMs on the tensor cores needs LSAM_FLAG_KEEP_G1");
         rc = seg_copy<false>(c, c->at<float>(L.xop) + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
       }
     } else if (c->cfg.dp_average) {

@@ -236,16 +236,18 @@ def test_classifier_bf16_tcgen05(model, widths, K, B, impl):
     p.close()
 
 
-@pytest.mark.parametrize("widths,K,B", [
-    ((64, 128, 96, 10), 4, 64),        # N tile 64, ragged head (10 outputs), 96-wide layer
-    ((256, 256, 256, 128), 2, 128),    # N tile 128, several contraction blocks, bias gradient out of the dgrad epilogue
-    ((320, 520, 24), 2, 40),           # ragged M tiles, ragged contraction (320 = 5 x 64), ragged minibatch
-    ((128, 264, 40), 3, 300),          # minibatch wider than one N tile (128 + 128 + 44): bias gradient by its own kernel from the planes
-    ((784, 1024, 10), 8, 128),         # the C2 shape
+@pytest.mark.parametrize("model,widths,K,B", [
+    (G.MODEL_MLP, (64, 128, 96, 10), 4, 64),        # N tile 64, ragged head (10 outputs), 96-wide layer
+    (G.MODEL_MLP, (256, 256, 256, 128), 2, 128),    # N tile 128, several contraction blocks, bias gradient out of the dgrad epilogue
+    (G.MODEL_MLP, (320, 520, 24), 2, 40),           # ragged M tiles, ragged contraction (320 = 5 x 64), ragged minibatch
+    (G.MODEL_MLP, (128, 264, 40), 3, 300),          # minibatch wider than one N tile (128 + 128 + 44): bias gradient by its own kernel from the planes
+    (G.MODEL_MLP, (784, 1024, 10), 8, 128),         # the C2 shape
+    (G.MODEL_RESMLP, (128, 192, 192, 192, 100), 3, 200),  # skip connections: the planes of the skipped activation and of its gradient are read back and added
+    (G.MODEL_RESMLP, (48, 80, 80, 80, 12), 2, 32),        # the same with a narrow head and ragged tiles
 ])
-def test_classifier_fp32_on_the_tensor_cores_with_three_bf16_planes_per_operand(widths, K, B):
+def test_classifier_fp32_on_the_tensor_cores_with_three_bf16_planes_per_operand(model, widths, K, B):
     # fp32 GEMMs as sums of six bf16 plane products: held to the same fp32 tolerances as the SIMT kernels, against the fp32 oracle
-    p = _mlp_pair(G.MODEL_MLP, widths, K, B, n=600, dtype=G.GEMM_FP32, impl=G.IMPL_TCGEN05, tau=4, lam=0.4, seed=5, jitter=0.01)
+    p = _mlp_pair(model, widths, K, B, n=600, dtype=G.GEMM_FP32, impl=G.IMPL_TCGEN05, tau=4, lam=0.4, seed=5, jitter=0.01)
     assert p.gpu.uses_tcgen05()
     _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, what=f"fp32 on tcgen05 {widths}")
     p.close()
@@ -254,12 +256,24 @@ def test_classifier_fp32_on_the_tensor_cores_with_three_bf16_planes_per_operand(
 def test_fp32_on_the_tensor_cores_is_refused_where_it_is_not_built():
     import torch
     X, labels = synth.gaussian_mixture(64, 48, 12, seed=1)
-    for model, widths in [(G.MODEL_RESMLP, (48, 80, 80, 12)), (G.MODEL_MLP, (44, 80, 12))]:  # skip connections; a width that is no multiple of 8
+    for model, widths in [(G.MODEL_MLP, (44, 80, 12)), (G.MODEL_RESMLP, (48, 80, 80, 12, 12))]:  # input widths that are no multiples of 8
         w0 = synth.mlp_init(widths, seed=1)
         Xm = X[:, :widths[0]].copy()
         with pytest.raises(G.LsamError):
             G.Lsam(G.make_config(model, widths=widths, K=2, batch=16, gemm_dtype=G.GEMM_FP32, gemm_impl=G.IMPL_TCGEN05, n_samples=64),
                    torch.from_numpy(Xm).cuda(), torch.from_numpy(labels).cuda(), torch.from_numpy(synth.replicate(w0, 2)).cuda(), torch.from_numpy(w0).cuda())
+    # the perturbed point lives in the operand planes, which the update overwrites: reading it back needs the kept copy
+    widths = (48, 80, 12)
+    w0 = synth.mlp_init(widths, seed=1)
+    c = G.Lsam(G.make_config(G.MODEL_MLP, widths=widths, K=2, batch=16, gemm_dtype=G.GEMM_FP32, gemm_impl=G.IMPL_TCGEN05, n_samples=64),
+               torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda(), torch.from_numpy(synth.replicate(w0, 2)).cuda(), torch.from_numpy(w0).cuda())
+    assert c.uses_tcgen05()
+    c.step(0.05, 0.05)
+    assert np.isfinite(c.read_grads(2)).all()
+    with pytest.raises(G.LsamError) as ei:
+        c.read_grads(3)
+    assert ei.value.code == G.LSAM_ERR_STATE
+    c.close()
 
 
 @pytest.mark.parametrize("impl", [G.IMPL_AUTO, G.IMPL_SIMT])
