@@ -263,9 +263,13 @@ __host__ __device__ constexpr int tc_astat_stages() { return (BLOCK_N == 256 && 
 // the B tile of one k-block, and feeds six MMA groups (the plane pairs (i, j) with i + j <= 2)
 constexpr int kTcSplitStages = 2;
 constexpr int kTcSplitPairs = 6;
-template <int BLOCK_N, bool PAIR = false, bool ASTAT = false, bool SPLIT = false>
+// BSTAT (B-stationary): the B block of a tile column (all k-blocks) stays in shared memory over a run of m-tiles, the ring holds A tiles
+template <int BLOCK_N>
+__host__ __device__ constexpr int tc_bstat_stages() { return BLOCK_N == 256 ? 4 : 8; }
+template <int BLOCK_N, bool PAIR = false, bool ASTAT = false, bool SPLIT = false, bool BSTAT = false>
 __host__ __device__ constexpr int tc_smem_bytes() {
-  return (SPLIT ? kTcSplitStages * 3 * tc_stage_bytes<BLOCK_N, false>()
+  return (BSTAT ? kTcAstatKBlocks * BLOCK_N * kTcBlockK * 2 + tc_bstat_stages<BLOCK_N>() * kTcBlockM * kTcBlockK * 2
+          : SPLIT ? kTcSplitStages * 3 * tc_stage_bytes<BLOCK_N, false>()
           : ASTAT ? kTcAstatKBlocks * kTcBlockM * kTcBlockK * 2 + tc_astat_stages<BLOCK_N, PAIR>() * (PAIR ? BLOCK_N / 2 : BLOCK_N) * kTcBlockK * 2
                   : tc_stages<BLOCK_N, PAIR>() * tc_stage_bytes<BLOCK_N, PAIR>()) + 1024 /*alignment slack*/ + 512 /*barriers*/ + kTcStageOutBytes;
 }
@@ -286,7 +290,12 @@ __host__ __device__ constexpr int tc_smem_bytes() {
 //   holds the three planes of both tiles; the product is the sum of the six plane pairs (i, j), i + j <= 2 (the pairs
 //   left out are below 2^-24 of |a||b|), smallest terms first, all into the same fp32 accumulator.  The epilogues write
 //   their bf16 outputs as three planes again (plane stride Z * M * ldb) and read the bias as the sum of its planes.
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false, bool SPLIT = false>
+//   BSTAT (weight gradient, single CTA, at most 4 k-blocks): the mirror image of ASTAT.  The work list is made of runs of ep.run_n
+//   consecutive m-tiles of one (replica, n-tile); the B block (activation rows of the tile column, all k-blocks) is loaded once per run
+//   and the ring streams the A tiles (dz rows), so a tile takes in 128 x Kd instead of BLOCK_N x Kd operand elements: half the bytes of
+//   the A-stationary form at BLOCK_N = 256.  (Measured per tile, stand-alone: the A-stationary main loop waits for its loads, 128 KB per
+//   tile at about 30 B per clock and SM, while the epilogue is hidden.)
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false, bool SPLIT = false, bool BSTAT = false>
 __global__ void __launch_bounds__(kTcThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                     const __grid_constant__ CUtensorMap map_c, int M, int N, int Kd,
@@ -294,7 +303,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   static_assert(!PAIR || BLOCK_N >= 128, "the pair form needs 64 rows of B per CTA");
   static_assert(!ASTAT || (!A_MN && !B_MN), "A-stationary form: both operands contraction-contiguous");
   static_assert(!SPLIT || (!PAIR && !ASTAT && BLOCK_N <= 128 && EPI <= TC_EPI_WGRAD), "three-plane form: single CTAs, N tile of at most 128, fp32 gradient");
-  constexpr int STAGES = SPLIT ? kTcSplitStages : (ASTAT ? tc_astat_stages<BLOCK_N, PAIR>() : tc_stages<BLOCK_N, PAIR>());
+  static_assert(!BSTAT || (!PAIR && !ASTAT && !SPLIT && !A_MN && !B_MN), "B-stationary form: single CTA, both operands contraction-contiguous");
+  constexpr bool STAT = ASTAT || BSTAT;  // one operand block stays in shared memory over a run of tiles
+  constexpr int STAGES = BSTAT ? tc_bstat_stages<BLOCK_N>() : SPLIT ? kTcSplitStages : (ASTAT ? tc_astat_stages<BLOCK_N, PAIR>() : tc_stages<BLOCK_N, PAIR>());
   constexpr int NPL = SPLIT ? 3 : 1;  // planes per operand
   constexpr int A_BYTES = kTcBlockM * kTcBlockK * 2;
   constexpr int B_ROWS = PAIR ? BLOCK_N / 2 : BLOCK_N;  // rows of the N side staged by this CTA
@@ -311,11 +322,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   extern __shared__ uint8_t smem_raw[];
   // round the tile area up to 1024 bytes by pointer arithmetic on the shared array itself (keeps the address space known)
   uint8_t* tiles = smem_raw + ((1024u - (tc::smem_u32(smem_raw) & 1023u)) & 1023u);
-  // ASTAT: [A slots: kTcAstatKBlocks x A_BYTES][B ring: STAGES x B_BYTES]; else a ring of STAGES x (A tile, B tile)
-  // SPLIT: a stage is [A plane 0, 1, 2][B plane 0, 1, 2]
-  constexpr int RING_STRIDE = ASTAT ? B_BYTES : NPL * (A_BYTES + B_BYTES);
-  constexpr int RING_B_OFF = ASTAT ? 0 : NPL * A_BYTES;
-  uint8_t* ring = tiles + (ASTAT ? kTcAstatKBlocks * A_BYTES : 0);
+  // ASTAT: [A slots: kTcAstatKBlocks x A_BYTES][B ring: STAGES x B_BYTES]; BSTAT: [B slots: kTcAstatKBlocks x B_BYTES][A ring: STAGES x A_BYTES];
+  // else a ring of STAGES x (A tile, B tile).  SPLIT: a stage is [A plane 0, 1, 2][B plane 0, 1, 2]
+  constexpr int SLOT_BYTES = ASTAT ? A_BYTES : B_BYTES;  // a slot of the stationary block
+  constexpr int RING_STRIDE = ASTAT ? B_BYTES : (BSTAT ? A_BYTES : NPL * (A_BYTES + B_BYTES));
+  constexpr int RING_B_OFF = STAT ? 0 : NPL * A_BYTES;
+  uint8_t* ring = tiles + (STAT ? kTcAstatKBlocks * SLOT_BYTES : 0);
   uint8_t* stage = ring + STAGES * RING_STRIDE;  // 1024-byte aligned: everything before it is a multiple of 1024
   uint64_t* bars = reinterpret_cast<uint64_t*>(stage + kTcStageOutBytes);
   uint64_t* full = bars;                     // [STAGES]  TMA -> MMA
@@ -323,8 +335,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   uint64_t* acc_full = bars + 2 * STAGES;    // [2]       MMA -> epilogue
   uint64_t* acc_empty = acc_full + 2;        // [2]       epilogue -> MMA
   uint64_t* bias_bar = acc_empty + 2;        // [4 quadrants][2]  dgrad: the two epilogue warps of a quadrant have left their partial bias sums
-  uint64_t* a_full = bias_bar + 8;           // [4]  ASTAT: A slot kb loaded        TMA -> MMA
-  uint64_t* a_empty = a_full + 4;            // [4]  ASTAT: A slot kb free again    MMA -> TMA
+  uint64_t* a_full = bias_bar + 8;           // [4]  ASTAT / BSTAT: slot kb of the stationary block loaded        TMA -> MMA
+  uint64_t* a_empty = a_full + 4;            // [4]  ASTAT / BSTAT: slot kb free again                            MMA -> TMA
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(a_empty + 4);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
@@ -333,9 +345,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const int n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_blocks = (Kd + kTcBlockK - 1) / kTcBlockK;
   // work list: units of (replica, m-tile, run of n-tiles); a run is one tile unless ASTAT
-  const int run_n = ASTAT ? (ep.run_n > 0 ? ep.run_n : 1) : 1;
-  const int runs = (n_tiles + run_n - 1) / run_n;
-  const int64_t total = (int64_t)Z * m_tiles * runs;
+  // a run walks `inner` (n-tiles; m-tiles in the B-stationary form) with the other tile index (`outer`) fixed
+  const int run_n = STAT ? (ep.run_n > 0 ? ep.run_n : 1) : 1;
+  const int inner_tiles = BSTAT ? m_tiles : n_tiles, outer_tiles = BSTAT ? n_tiles : m_tiles;
+  const int runs = (inner_tiles + run_n - 1) / run_n;
+  const int64_t total = (int64_t)Z * outer_tiles * runs;
   // a pair walks the work list together: unit = index of this CTA (or of its pair), units = how many walk the list
   const uint32_t rank = PAIR ? tc::cluster_ctarank() : 0u;
   const bool leader = rank == 0u;
@@ -383,14 +397,21 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       bool ok = true;
       uint32_t run_ph = 0;  // ASTAT: phase of the A-slot barriers, one flip per run
       for (int64_t t = unit; t < total && ok; t += units) {
-        const int r = (int)(t % runs), mt = (int)((t / runs) % m_tiles), z = (int)(t / ((int64_t)runs * m_tiles));
+        const int r = (int)(t % runs), fixed = (int)((t / runs) % outer_tiles), z = (int)(t / ((int64_t)runs * outer_tiles));
         if (active != nullptr && !active[z]) continue;  // waiting replica: all three roles skip the same tiles
-        const int nt_begin = r * run_n, nt_end = (nt_begin + run_n < n_tiles) ? nt_begin + run_n : n_tiles;
-        for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
+        const int nt_begin = r * run_n, nt_end = (nt_begin + run_n < inner_tiles) ? nt_begin + run_n : inner_tiles;
+        for (int it = nt_begin; it < nt_end && ok; ++it) {
+        const int mt = BSTAT ? it : fixed, nt = BSTAT ? fixed : it;
         const int m0 = mt * TILE_M + m_off, n0 = nt * BLOCK_N + n_off;
         for (int kb = 0; kb < k_blocks; ++kb) {
           const int k0 = kb * kTcBlockK;
-          if (ASTAT && nt == nt_begin) {
+          if (BSTAT && it == nt_begin) {
+            // first tile of a run: bring in B slot kb as soon as the previous run has released it
+            if (!tc::mbar_wait(&a_empty[kb], run_ph ^ 1u, abort_flag)) { ok = false; break; }
+            tc::mbar_expect_tx(&a_full[kb], B_BYTES);
+            tc::tma_load_3d(tiles + kb * B_BYTES, &map_b, k0, n0, z, &a_full[kb]);
+          }
+          if (ASTAT && it == nt_begin) {
             // first tile of a run: bring in A slot kb as soon as the previous run has released it (pair form: each CTA its own
             // 128 rows into its own slot, both loads completing on the leader's barrier, which the leader arms with the bytes of both)
             if (!tc::mbar_wait(&a_empty[kb], run_ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -405,7 +426,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           if (!tc::mbar_wait(&empty[s], ph ^ 1u, abort_flag)) { ok = false; break; }
           uint8_t* a_dst = ring + s * RING_STRIDE;
           uint8_t* b_dst = a_dst + RING_B_OFF;
-          if (ASTAT && PAIR) {
+          if (BSTAT) {
+            tc::mbar_expect_tx(&full[s], A_BYTES);
+            tc::tma_load_3d(a_dst, &map_a, k0, m0, z, &full[s]);
+          } else if (ASTAT && PAIR) {
             if (leader) tc::mbar_expect_tx(&full[s], 2 * B_BYTES);
             tc::tma_load_3d_pair(b_dst, &map_b, k0, n0, z, tc::map_to_cta(tc::smem_u32(&full[s]), 0u));
           } else if (ASTAT) {
@@ -465,18 +489,18 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       bool ok = true;
       uint32_t run_ph = 0;
       for (int64_t t = unit; t < total && ok; t += units) {
-        if (active != nullptr && !active[(int)(t / ((int64_t)runs * m_tiles))]) continue;
-        const int nt_begin = (int)(t % runs) * run_n, nt_end = (nt_begin + run_n < n_tiles) ? nt_begin + run_n : n_tiles;
+        if (active != nullptr && !active[(int)(t / ((int64_t)runs * outer_tiles))]) continue;
+        const int nt_begin = (int)(t % runs) * run_n, nt_end = (nt_begin + run_n < inner_tiles) ? nt_begin + run_n : inner_tiles;
         for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
         if (!tc::mbar_wait(&acc_empty[as], aph ^ 1u, abort_flag)) { ok = false; break; }
         tc::tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)as * ACC_COLS;
         for (int kb = 0; kb < k_blocks; ++kb) {
-          if (ASTAT && nt == nt_begin && !tc::mbar_wait(&a_full[kb], run_ph, abort_flag)) { ok = false; break; }
+          if (STAT && nt == nt_begin && !tc::mbar_wait(&a_full[kb], run_ph, abort_flag)) { ok = false; break; }
           if (!tc::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           tc::tc_fence_after();
           const uint32_t a_addr = tc::smem_u32(ASTAT ? tiles + kb * A_BYTES : ring + s * RING_STRIDE);
-          const uint32_t b_addr = tc::smem_u32(ring + s * RING_STRIDE + RING_B_OFF);
+          const uint32_t b_addr = tc::smem_u32(BSTAT ? tiles + kb * B_BYTES : ring + s * RING_STRIDE + RING_B_OFF);
 #pragma unroll
           for (int pp = 0; pp < (SPLIT ? kTcSplitPairs : 1); ++pp) {
             // SPLIT: plane pairs (A plane, B plane) in the order (0,2) (1,1) (2,0) (0,1) (1,0) into the second accumulator,
@@ -500,7 +524,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           // frees the stage (in both CTAs of a pair) when these MMAs have read it
           if (PAIR) tc::umma_commit_pair(&empty[s]);
           else tc::umma_commit(&empty[s]);
-          if (ASTAT && nt == nt_end - 1) {  // last tile of the run: the A slot (of both CTAs of a pair) is free once these MMAs are done
+          if (STAT && nt == nt_end - 1) {  // last tile of the run: the slot (of both CTAs of a pair) is free once these MMAs are done
             if (PAIR) tc::umma_commit_pair(&a_empty[kb]);
             else tc::umma_commit(&a_empty[kb]);
           }
@@ -526,10 +550,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     bool ok = true;
     const uint32_t acc_empty_leader[2] = {PAIR ? tc::map_to_cta(tc::smem_u32(&acc_empty[0]), 0u) : 0u, PAIR ? tc::map_to_cta(tc::smem_u32(&acc_empty[1]), 0u) : 0u};
     for (int64_t t = unit; t < total && ok; t += units) {
-      const int r_ = (int)(t % runs), mt = (int)((t / runs) % m_tiles), z = (int)(t / ((int64_t)runs * m_tiles));
+      const int r_ = (int)(t % runs), fixed = (int)((t / runs) % outer_tiles), z = (int)(t / ((int64_t)runs * outer_tiles));
       if (active != nullptr && !active[z]) continue;
-      const int nt_begin = r_ * run_n, nt_end = (nt_begin + run_n < n_tiles) ? nt_begin + run_n : n_tiles;
-      for (int nt = nt_begin; nt < nt_end && ok; ++nt) {
+      const int nt_begin = r_ * run_n, nt_end = (nt_begin + run_n < inner_tiles) ? nt_begin + run_n : inner_tiles;
+      for (int it = nt_begin; it < nt_end && ok; ++it) {
+      const int mt = BSTAT ? it : fixed, nt = BSTAT ? fixed : it;
       const int m_base = mt * TILE_M + m_off;  // first row of the 128 rows this CTA drains
       const int m = m_base + quad * 32 + lane;
       const int n0 = nt * BLOCK_N;
@@ -943,6 +968,7 @@ struct TcGemm {
   bool valid = false;
   bool pair = false;  // run by pairs of CTAs (cta_group::2) on 256-row tiles
   bool astat = false; // weight gradient with the A block stationary over runs of n-tiles (ep.run_n)
+  bool bstat = false; // weight gradient with the B block stationary over runs of m-tiles (ep.run_n); single CTAs
   bool split = false; // operands stored as three bf16 planes (fp32 GEMM); single CTAs, N tile of at most 128
 };
 
@@ -957,6 +983,7 @@ struct TcPlan {
   bool allow_pair = true;       // false: every GEMM on the single-CTA kernels
   bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
   bool allow_astat = true;      // false: the weight gradient walks single tiles
+  bool allow_bstat = true;      // false: no B-stationary weight gradient (the A-stationary form instead)
   bool pair_wgrad = false;      // true: the weight gradient of wide layers by pairs of CTAs with the dz block stationary (measured slower, see tc_pick_pair)
   int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
 };
@@ -1062,6 +1089,11 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       const bool astat_ok = P.allow_astat && B <= kTcAstatKBlocks * kTcBlockK;
       if (P.allow_pair && P.pair_wgrad && astat_ok && g.M >= 256 && g.block_n == 256) g.pair = true;
       g.astat = astat_ok && (!g.pair || g.block_n >= 128);
+      // single CTAs with 256-wide tiles: the activation block (256 rows) is the larger operand, so it is the one to keep in shared
+      // memory: a tile then takes in 128 instead of 256 rows (measured inside the step at B = 256, 4096-wide layers: 783-798 -> 823-837
+      // TFLOP/s; no gain with two k-blocks, B = 128, where the stores of the tile are what takes the time)
+      g.bstat = g.astat && !g.pair && P.allow_bstat && g.block_n == 256 && B > 2 * kTcBlockK;
+      if (g.bstat) g.astat = false;
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, ZM, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, ZM, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
       ok &= tc_make_map(&g.map_c, b.g + ly.w_pad, ly.in, ly.out, Z, ly.in, b.ld, 32, 32);
@@ -1070,6 +1102,15 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       g.ep.g = b.g; g.ep.ld_g = b.ld; g.ep.w_off = ly.w_pad; g.ep.ldw = ly.in; g.ep.ldb = b.ldb;
       g.ep.partial = b.partial; g.ep.ld_partial = b.ld_partial; g.ep.slot0 = slot;
       g.ep.run_n = 1;
+      if (g.bstat) {
+        const int64_t cols = (int64_t)Z * ceil_div(g.N, g.block_n), m_tiles = ceil_div(g.M, kTcBlockM);
+        double best = 0.0;
+        for (int rn = 1; rn <= m_tiles; ++rn) {
+          const int64_t units = cols * ceil_div(m_tiles, (int64_t)rn);
+          const double cost = (double)ceil_div(units, (int64_t)P.sms) * ((double)rn * kTcBlockM + g.block_n);
+          if (rn == 1 || cost < best) { best = cost; g.ep.run_n = rn; }
+        }
+      }
       if (g.astat) {
         // run length: a unit of the list costs a CTA run_n B tiles (half tiles in a pair) plus one A block of 128 rows; the SMs (pairs of SMs)
         // work through ceil(units / SMs) rounds of units.  Pick the run length with the least bytes through the busiest SM.
@@ -1108,10 +1149,10 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
   return 0;
 }
 
-template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false, bool SPLIT = false>
+template <int BLOCK_N, bool A_MN, bool B_MN, int EPI, bool PAIR, bool ASTAT = false, bool SPLIT = false, bool BSTAT = false>
 inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
-  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR, ASTAT, SPLIT>;
-  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR, ASTAT, SPLIT>();
+  auto kern = gemm_tcgen05_kernel<BLOCK_N, A_MN, B_MN, EPI, PAIR, ASTAT, SPLIT, BSTAT>;
+  constexpr int smem = tc_smem_bytes<BLOCK_N, PAIR, ASTAT, SPLIT, BSTAT>();
   // the shared-memory limit of a kernel is a per-device attribute: remember it per device ordinal
   static bool attr_set[64] = {};
   int dev = 0;
@@ -1122,7 +1163,9 @@ inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
   }
   const int tile_m = PAIR ? 2 * kTcBlockM : kTcBlockM;
   const int64_t n_tiles = ceil_div(g.N, BLOCK_N);
-  const int64_t tiles = (int64_t)P.Z * ceil_div(g.M, tile_m) * (ASTAT ? ceil_div(n_tiles, (int64_t)(g.ep.run_n > 0 ? g.ep.run_n : 1)) : n_tiles);  // units of the work list
+  const int64_t rn = g.ep.run_n > 0 ? g.ep.run_n : 1;
+  const int64_t tiles = BSTAT ? (int64_t)P.Z * n_tiles * ceil_div(ceil_div(g.M, tile_m), rn)
+                              : (int64_t)P.Z * ceil_div(g.M, tile_m) * (ASTAT ? ceil_div(n_tiles, rn) : n_tiles);  // units of the work list
   if (!PAIR) {
     const int grid = (int)(tiles < P.sms ? tiles : P.sms);
     kern<<<grid, kTcThreads, smem, stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status, P.active);
@@ -1175,6 +1218,7 @@ inline int tc_launch(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
     }
   }
   if constexpr (tc_epi_is_wgrad(EPI) && !A_MN && !B_MN) {
+    if (g.bstat && g.block_n == 256) return tc_launch_one<256, A_MN, B_MN, EPI, false, false, false, true>(P, g, stream);
     if (g.astat) {
       switch (g.block_n) {
         case 256: return tc_launch_one<256, A_MN, B_MN, EPI, false, true>(P, g, stream);
