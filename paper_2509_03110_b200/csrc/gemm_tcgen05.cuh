@@ -107,8 +107,11 @@ __device__ inline uint32_t map_to_cta(uint32_t local, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
   return r;
 }
+// Arrive on a barrier of another CTA of the cluster.  Default semantics (release at CTA scope): what the barrier orders here are
+// tensor-memory reads, which tcgen05.wait::ld and the tcgen05 fences have already completed.  A release at cluster scope would make the
+// warp wait for every global store it has issued before (the outputs of the tile): measured 2000-3000 clocks per tile.
 __device__ inline void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 // all threads of both CTAs of the cluster
 __device__ inline void cluster_sync_all() {
@@ -984,7 +987,7 @@ struct TcPlan {
   bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
   bool allow_astat = true;      // false: the weight gradient walks single tiles
   bool allow_bstat = true;      // false: no B-stationary weight gradient (the A-stationary form instead)
-  bool pair_wgrad = false;      // true: the weight gradient of wide layers by pairs of CTAs with the dz block stationary (measured slower, see tc_pick_pair)
+  bool pair_wgrad = true;       // the weight gradient of wide layers by pairs of CTAs with the dz block stationary
   int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
 };
 
@@ -1021,10 +1024,9 @@ inline bool tc_make_map(CUtensorMap* m, const T* base, uint64_t cols, uint64_t r
 
 inline int tc_pick_block_n(int n, bool split = false) { return (n > 128 && !split) ? 256 : (n > 64 ? 128 : 64); }
 // Where the pair form is used: forward and dgrad with a 256-wide minibatch tile (measured at the 4096-wide layers with
-// B = 256: 985 -> 1100 and 945 -> 1030 TFLOP/s inside the step).  It loses with 128-wide minibatch tiles (short kernels: 415 -> 405,
-// 360 -> 335) and in the weight gradient (770 -> 650: with four k-blocks per tile the epilogue is the kernel, and in a pair
-// the slower of the two epilogues gates both CTAs; the same 650 with the dz block stationary on top, which halves what a CTA takes in:
-// the weight gradient is not bound by its operand loads), so those keep the single-CTA kernels; `force` (tests) pairs whatever can be.
+// B = 256: 985 -> 1100 and 945 -> 1030 TFLOP/s inside the step), and the weight gradient with 256-wide tiles and a minibatch of at
+// most 256 samples, where the pair also keeps its dz blocks in shared memory (tc_plan; 850 -> 980).  It loses with 128-wide
+// minibatch tiles (short kernels: 415 -> 405, 360 -> 335), which keep the single-CTA kernels; `force` (tests) pairs whatever can be.
 inline bool tc_pick_pair(int M, int block_n, bool wgrad, bool force) { return M >= 256 && (force ? block_n >= 128 : (block_n == 256 && !wgrad)); }
 // Partial-sum slots one replica needs when the sum of squares is fused into the weight-gradient epilogue:
 // eight per output tile (one per epilogue warp) plus one per 8 bias units.
