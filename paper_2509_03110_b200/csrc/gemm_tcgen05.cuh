@@ -1,7 +1,7 @@
 // gemm_tcgen05.cuh -- batched-over-replicas bf16 GEMMs of the classifier path on the 5th-generation tensor cores:
 // TMA (cp.async.bulk.tensor) stages 128B-swizzled operand tiles in shared memory, one elected thread issues
-// tcgen05.mma with fp32 accumulators in tensor memory, four warps drain the accumulators with tcgen05.ld and apply
-// the fused epilogue.  One persistent CTA per SM walks the (replica, m-tile, n-tile) list; the accumulator is
+// tcgen05.mma with fp32 accumulators in tensor memory, eight warps (two per lane quadrant) drain the accumulators with
+// tcgen05.ld and apply the fused epilogue.  One persistent CTA per SM walks the (replica, m-tile, n-tile) list; the accumulator is
 // double-buffered in tensor memory so that the epilogue of a tile overlaps the main loop of the next one.
 //
 // Every GEMM is D(z, m, n) = sum_kd A(z, m, kd) * B(z, n, kd) with the 128-row M side on the weights:
@@ -231,7 +231,7 @@ struct TcEpi {
   // wgrad: sum of squares of every 32-row block of the tile -> partial[z * ld_partial + slot0 + (mt * n_tiles + nt) * 8 + epilogue warp]
   float* partial;  int64_t ld_partial;  int slot0;
   int ldb;  // sample stride of the feature-major buffers (multiple of 16)
-  int run_n;  // A-stationary weight gradient: consecutive n-tiles per unit of the work list (>= 1)
+  int run_n;  // stationary weight gradient: consecutive n-tiles (B-stationary: m-tiles) per unit of the work list (>= 1)
   // TC_EPI_WGRAD_UPD: worker state rows (same addressing as g: [z * ld_g + w_off + m * ldw + n]), centre ring and the ring slot
   // each replica reads, the bf16 operand copy, and the step's scalars (lam_k nullable: per-replica pull weight instead of lambda)
   float* upd_x;  float* upd_v;  const float* upd_yring;  const int32_t* upd_slot;  bf16* upd_xop;  const float* upd_lam_k;
@@ -283,11 +283,13 @@ __host__ __device__ constexpr int tc_smem_bytes() {
 //   M/N-contiguous operand:         map dims {rows, Kd, Z}, box {64, 64, 1} (one box per 64 rows of the tile)
 //   PAIR: the B box has BLOCK_N / 2 rows (contraction-contiguous) resp. the CTA loads BLOCK_N / 128 boxes (N-contiguous);
 //   the grid is a multiple of 2 and is launched with cluster dimension 2.
-//   ASTAT (weight gradient, single CTA, at most 4 k-blocks): the work list is made of runs of ep.run_n consecutive n-tiles of
+//   ASTAT (weight gradient, single CTA or pair, at most 4 k-blocks): the work list is made of runs of ep.run_n consecutive n-tiles of
 //   one (replica, m-tile); the A block (dz rows, all k-blocks) is loaded once per run into its own slots and reused by every
 //   tile of the run, so a tile takes in BLOCK_N x Kd instead of (128 + BLOCK_N) x Kd operand elements (the weight gradient is
 //   bound by the rate at which TMA fills shared memory from L2).  A slot is handed back to the producer as soon as the last
-//   tile of the run has used it, so the next run's A block streams in behind the current run's last tile.
+//   tile of the run has used it, so the next run's A block streams in behind the current run's last tile.  In a pair each CTA keeps
+//   the block of its own 128 rows and stages half of every B tile; the slot barriers work like the ring's (loads of both CTAs complete
+//   on the leader's barrier, the leader's commit frees the slot in both).
 //   SPLIT (fp32 GEMM on the bf16 tensor cores): every operand tensor is stored as three bf16 planes p0 = bf16(a),
 //   p1 = bf16(a - p0), p2 = bf16(a - p0 - p1), plane p of replica z being "replica" z + p Z of the tensor map.  A stage
 //   holds the three planes of both tiles; the product is the sum of the six plane pairs (i, j), i + j <= 2 (the pairs
@@ -347,7 +349,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const int m_tiles = (M + TILE_M - 1) / TILE_M;
   const int n_tiles = (N + BLOCK_N - 1) / BLOCK_N;
   const int k_blocks = (Kd + kTcBlockK - 1) / kTcBlockK;
-  // work list: units of (replica, m-tile, run of n-tiles); a run is one tile unless ASTAT
+  // work list: units of (replica, m-tile, run of n-tiles), B-stationary: (replica, n-tile, run of m-tiles); a run is one tile unless a block is stationary
   // a run walks `inner` (n-tiles; m-tiles in the B-stationary form) with the other tile index (`outer`) fixed
   const int run_n = STAT ? (ep.run_n > 0 ? ep.run_n : 1) : 1;
   const int inner_tiles = BSTAT ? m_tiles : n_tiles, outer_tiles = BSTAT ? n_tiles : m_tiles;
@@ -398,7 +400,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       int s = 0;
       uint32_t ph = 0;
       bool ok = true;
-      uint32_t run_ph = 0;  // ASTAT: phase of the A-slot barriers, one flip per run
+      uint32_t run_ph = 0;  // phase of the barriers of the stationary slots, one flip per run
       for (int64_t t = unit; t < total && ok; t += units) {
         const int r = (int)(t % runs), fixed = (int)((t / runs) % outer_tiles), z = (int)(t / ((int64_t)runs * outer_tiles));
         if (active != nullptr && !active[z]) continue;  // waiting replica: all three roles skip the same tiles
