@@ -32,6 +32,7 @@ struct LayerInfo {
   bool conv = false;
   int Cin = 0, Cout = 0, H = 0, W = 0;
   int wg_parts = 1, wg_chunk = 0;     // convolution: the weight gradient's contraction (one term per position and sample) is split over blocks
+  int fw_parts = 1, fw_chunk = 0;     // dense layer of the convolutional model with few tiles and a long contraction: forward split over blocks
   int64_t feat_in = 0, feat_out = 0;  // features per sample entering / leaving the layer (dense: in / out)
 };
 
@@ -108,6 +109,7 @@ bool plan(const lsam_config& c, Layout& L) {
     const bool cnn = c.model == LSAM_MODEL_CNN;
     // convolutional model: positions are indexed (y, x, sample) with the sample fastest, so the minibatch must fill its stride
     if (cnn && (c.n_conv < 1 || c.n_conv >= c.n_layers || c.img_h < 1 || c.img_w < 1 || c.img_h % (1 << c.n_conv) || c.img_w % (1 << c.n_conv) || c.batch % 16)) return false;
+    if (cnn && (int64_t)c.img_h * c.img_w * c.batch >= ((int64_t)1 << 31)) return false;  // the helper kernels index positions with 32 bits
     int64_t unp = 0, pad = 0;
     int H = c.img_h, W = c.img_w;
     for (int l = 0; l < c.n_layers; ++l) {
@@ -214,6 +216,15 @@ bool plan(const lsam_config& c, Layout& L) {
           parts = ceil_div((int64_t)P, chunk);
           li.wg_parts = (int)parts; li.wg_chunk = (int)chunk;
           if (parts > 1) max_part = std::max(max_part, (size_t)parts * li.Cout * li.in);
+        } else if (c.model == LSAM_MODEL_CNN && l + 1 < L.layers.size()) {
+          // dense hidden layer behind the convolutions (flattened feature maps in, a few hundred units out): a handful of tiles walking
+          // thousands of inputs; split the inputs over blocks the same way
+          const int64_t tiles = ceil_div((int64_t)B, kSimtBM) * ceil_div(li.out, kSimtBN) * (int64_t)K;
+          int64_t parts = std::max<int64_t>(1, std::min<int64_t>(ceil_div(2 * 148, tiles), (int64_t)li.in / (8 * kSimtBK)));
+          const int64_t chunk = round_up(ceil_div((int64_t)li.in, parts), kSimtBK);
+          parts = ceil_div((int64_t)li.in, chunk);
+          li.fw_parts = (int)parts; li.fw_chunk = (int)chunk;
+          if (parts > 1) max_part = std::max(max_part, (size_t)parts * B * li.out);
         }
       }
       if (max_full) { L.zout = take(esz * K * max_full); L.dzc = take(esz * K * max_full); }
@@ -704,12 +715,12 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
     if (li.conv) {
       const int64_t Pn = (int64_t)li.H * li.W * ldb;
       T* col = c->at<T>(L.col[l]);
-      LAUNCH(c, LSAM_PROF_GATHER, im2col_kernel<T><<<dim3((unsigned)ceil_div(Pn, 256), li.in, K), 256, 0, c->stream>>>(a_in, li.Cin, li.H, li.W, ldb, col, c->act()));
+      LAUNCH(c, LSAM_PROF_GATHER, im2col_kernel<T><<<dim3((unsigned)ceil_div(Pn, 1024), li.in, K), 256, 0, c->stream>>>(a_in, li.Cin, li.H, li.W, ldb, col, c->act()));
       GemmOperand A{col, (int64_t)li.in * Pn, 1, Pn};           // (z, position, patch element)
       GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, output channel, patch element)
       EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.zout), nullptr, c->at<uint8_t>(L.mask[l]), li.Cout, (int)Pn};
       if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, (int)Pn, li.Cout, li.in, e)) != LSAM_OK) return rc;
-      LAUNCH(c, LSAM_PROF_GEMM_FWD, maxpool_kernel<T><<<dim3((unsigned)ceil_div(Pn / 4, 256), li.Cout, K), 256, 0, c->stream>>>(
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, maxpool_kernel<T><<<dim3((unsigned)ceil_div(Pn / 4, 1024), li.Cout, K), 256, 0, c->stream>>>(
           c->at<T>(L.zout), li.Cout, li.H, li.W, ldb, c->at<T>(L.act[l + 1]), c->at<uint8_t>(L.parg[l]), c->act()));
       continue;
     }
@@ -725,7 +736,16 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
     } else {
       EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.act[l + 1]), nullptr, c->at<uint8_t>(L.mask[l]), li.out, ldb};
-      rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
+      if (li.fw_parts > 1) {
+        // partial products per share of the inputs, then their sum in a fixed order handed to the layer's epilogue
+        EpiPartial ep{c->at<float>(L.wpart), B, li.out};
+        if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, ep, li.fw_parts, li.fw_chunk)) != LSAM_OK) return rc;
+        LAUNCH(c, LSAM_PROF_GEMM_FWD, sum_parts_epi_kernel<EpiFwdHidden<T, T>><<<dim3((unsigned)ceil_div((int64_t)B * li.out, 256), K), 256, 0, c->stream>>>(
+            c->at<float>(L.wpart), li.fw_parts, B, li.out, e, c->act()));
+        rc = LSAM_OK;
+      } else {
+        rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, e);
+      }
     }
     if (rc != LSAM_OK) return rc;
   }
@@ -743,10 +763,9 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
     if (li.conv) {
       const int64_t Pn = (int64_t)li.H * li.W * ldb;
       T* dzc = c->at<T>(L.dzc);
-      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, unpool_kernel<T><<<dim3((unsigned)ceil_div(Pn, 256), li.Cout, K), 256, 0, c->stream>>>(
+      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, unpool_kernel<T><<<dim3((unsigned)ceil_div(Pn, 1024), li.Cout, K), 256, 0, c->stream>>>(
           c->at<T>(L.dz[cur]), c->at<uint8_t>(L.parg[l]), c->at<uint8_t>(L.mask[l]), li.Cout, li.H, li.W, ldb, dzc, c->act()));
-      LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<dim3((unsigned)ceil_div(li.Cout, 8), K), 256, 0, c->stream>>>(
-          dzc, (int)Pn, li.Cout, (int)Pn, c->g(), ld, li.b_pad, nullptr, L.nchunks, 0, c->act()));
+      LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_long_kernel<T><<<dim3((unsigned)li.Cout, K), 256, 0, c->stream>>>(dzc, Pn, li.Cout, Pn, c->g(), ld, li.b_pad, c->act()));
       {
         GemmOperand A{dzc, (int64_t)li.Cout * Pn, Pn, 1};                 // (z, output channel, position)
         GemmOperand Bm{c->at<T>(L.col[l]), (int64_t)li.in * Pn, Pn, 1};   // (z, patch element, position)
@@ -767,7 +786,7 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
         GemmOperand W{P + li.w_pad, ld, 1, li.in};                         // (z, patch element, output channel)
         EpiDgrad<T> e{nullptr, nullptr, dcol, nullptr, li.in, (int)Pn};    // the raw gradient of the patch matrix
         if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_DGRAD, A, W, (int)Pn, li.in, li.Cout, e)) != LSAM_OK) return rc;
-        LAUNCH(c, LSAM_PROF_GEMM_DGRAD, col2im_kernel<T><<<dim3((unsigned)ceil_div(Pn, 256), li.Cin, K), 256, 0, c->stream>>>(
+        LAUNCH(c, LSAM_PROF_GEMM_DGRAD, col2im_kernel<T><<<dim3((unsigned)ceil_div(Pn, 1024), li.Cin, K), 256, 0, c->stream>>>(
             dcol, li.Cin, li.H, li.W, ldb, c->at<T>(L.dz[cur ^ 1]), c->act()));
       }
       cur ^= 1;

@@ -377,6 +377,22 @@ sum_parts_kernel(const float* __restrict__ part, int parts, int M, int N, float*
   g[(int64_t)z * ld_g + w_off + e] = s;
 }
 
+// The same sum handed to an epilogue functor instead (a forward or dgrad product whose contraction was split over blocks):
+// epi(z, m, n, sum over the parts, ascending).  Consecutive threads walk m (the sample index of the feature-major buffers).
+// grid (ceil(M N / 256), K).
+template <class Epi>
+__global__ void __launch_bounds__(256)
+sum_parts_epi_kernel(const float* __restrict__ part, int parts, int M, int N, Epi epi, const int32_t* __restrict__ active) {
+  const int z = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= (int64_t)M * N) return;
+  const int n = (int)(e / M), m = (int)(e % M);
+  float s = 0.f;
+  for (int q = 0; q < parts; ++q) s += part[(((int64_t)z * parts + q) * M + m) * N + n];
+  epi(z, m, n, s);
+}
+
 // ------------------------------------------------------------------------------------------------ softmax cross-entropy
 // logits and dz are feature-major [K, C, ldb].  A block handles 32 consecutive samples (threadIdx.x, so every access is
 // coalesced) with 8 class groups (threadIdx.y: classes cg, cg + 8, ...); the per-sample maximum and sum of exponentials
@@ -479,32 +495,63 @@ bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, TG* __restr
   }
 }
 
+// The same for long rows (a convolution's bias gradient sums over every position and sample): one block per (replica, unit);
+// thread t adds elements t, t + 256, ... in ascending order, then the xor-shuffle tree, then the eight warp sums in warp order.
+// grid (out, K), block 256.
+template <typename TA>
+__global__ void __launch_bounds__(256)
+bias_grad_long_kernel(const TA* __restrict__ dz, int64_t B, int out, int64_t ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off,
+                      const int32_t* __restrict__ active) {
+  __shared__ float ws[8];
+  const int o = blockIdx.x, z = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  const TA* p = dz + ((int64_t)z * out + o) * ldb;
+  float s = 0.f;
+  for (int64_t b = threadIdx.x; b < B; b += 256) s += to_float(p[b]);
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) ws[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int i = 0; i < 8; ++i) t += ws[i];
+    g[(int64_t)z * ld_g + b_off + o] = t;
+  }
+}
+
 // ------------------------------------------------------------------------------------------------ convolution layers
 // A convolution layer (3x3, stride 1, zero padding 1, ReLU, 2x2 max-pooling) runs on the batched GEMMs through an explicit
 // patch matrix.  Feature maps are feature-major like every activation buffer, [K, C, P] with the position index
 // p = (y * W + x) * B + b (sample fastest), so that the gathered minibatch [K, C0 * H * W, B] already is the first layer's input and
 // the pooled output of the last convolution already is the dense layers' input [K, C * H' * W', B].
 //   col[z][ci * 9 + kh * 3 + kw][(y, x, b)] = a[z][ci][(y + kh - 1, x + kw - 1, b)]  (0 outside the image)
-// One thread per element of col, consecutive threads along p.  grid (ceil(P / 256), Cin * 9, K).
+// The four helpers below give a thread FOUR consecutive positions p (the same pixel, four consecutive samples: B is a multiple of
+// 16) moved as one 16- or 8-byte vector, with 32-bit index arithmetic (H W B < 2^31).
+template <typename T>
+struct alignas(sizeof(T) * 4) Vec4 { T v[4]; };
+struct alignas(4) Byte4 { uint8_t v[4]; };
+
+// One thread per four elements of col, consecutive threads along p.  grid (ceil(P / 1024), Cin * 9, K).
 template <typename T>
 __global__ void __launch_bounds__(256)
 im2col_kernel(const T* __restrict__ a, int Cin, int H, int W, int B, T* __restrict__ col, const int32_t* __restrict__ active) {
   const int z = blockIdx.z;
   if (active != nullptr && !active[z]) return;
-  const int64_t P = (int64_t)H * W * B;
-  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int P = H * W * B;
+  const int p = ((int)blockIdx.x * (int)blockDim.x + (int)threadIdx.x) * 4;
   if (p >= P) return;
   const int r = blockIdx.y, ci = r / 9, kh = (r % 9) / 3, kw = r % 3;
-  const int b = (int)(p % B);
-  const int x = (int)((p / B) % W), y = (int)(p / ((int64_t)B * W));
+  const int b = p % B, pix = p / B;
+  const int x = pix % W, y = pix / W;
   const int yy = y + kh - 1, xx = x + kw - 1;
-  T v = from_float<T>(0.f);
-  if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = a[((int64_t)z * Cin + ci) * P + ((int64_t)yy * W + xx) * B + b];
-  col[((int64_t)z * Cin * 9 + r) * P + p] = v;
+  Vec4<T> v;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) v.v[i] = from_float<T>(0.f);
+  if (yy >= 0 && yy < H && xx >= 0 && xx < W) v = *reinterpret_cast<const Vec4<T>*>(a + ((int64_t)z * Cin + ci) * P + (yy * W + xx) * B + b);
+  *reinterpret_cast<Vec4<T>*>(col + ((int64_t)z * Cin * 9 + r) * P + p) = v;
 }
 
 // 2x2 max-pooling of the ReLU output r [K, C, (H, W, B)] -> pooled [K, C, (H/2, W/2, B)]; arg = which element of the window
-// (dy * 2 + dx, the first maximum in that order).  One thread per pooled element.  grid (ceil(P4 / 256), C, K).
+// (dy * 2 + dx, the first maximum in that order).  One thread per four pooled elements.  grid (ceil(P4 / 1024), C, K).
 template <typename T>
 __global__ void __launch_bounds__(256)
 maxpool_kernel(const T* __restrict__ r, int C, int H, int W, int B, T* __restrict__ pooled, uint8_t* __restrict__ arg,
@@ -512,64 +559,87 @@ maxpool_kernel(const T* __restrict__ r, int C, int H, int W, int B, T* __restric
   const int z = blockIdx.z, c = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   const int Ho = H / 2, Wo = W / 2;
-  const int64_t P4 = (int64_t)Ho * Wo * B;
-  const int64_t q = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int P4 = Ho * Wo * B;
+  const int q = ((int)blockIdx.x * (int)blockDim.x + (int)threadIdx.x) * 4;
   if (q >= P4) return;
-  const int b = (int)(q % B), xo = (int)((q / B) % Wo), yo = (int)(q / ((int64_t)B * Wo));
+  const int b = q % B, pix = q / B;
+  const int xo = pix % Wo, yo = pix / Wo;
   const T* src = r + ((int64_t)z * C + c) * (int64_t)H * W * B;
-  float best = -1.f;
-  int a = 0;
+  float best[4] = {-1.f, -1.f, -1.f, -1.f};
+  Byte4 a;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) a.v[i] = 0;
 #pragma unroll
   for (int dy = 0; dy < 2; ++dy)
 #pragma unroll
     for (int dx = 0; dx < 2; ++dx) {
-      const float v = to_float(src[((int64_t)(2 * yo + dy) * W + 2 * xo + dx) * B + b]);
-      if (v > best) { best = v; a = dy * 2 + dx; }
+      const Vec4<T> v = *reinterpret_cast<const Vec4<T>*>(src + ((2 * yo + dy) * W + 2 * xo + dx) * B + b);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float f = to_float(v.v[i]);
+        if (f > best[i]) { best[i] = f; a.v[i] = (uint8_t)(dy * 2 + dx); }
+      }
     }
-  pooled[((int64_t)z * C + c) * P4 + q] = from_float<T>(best);
-  arg[((int64_t)z * C + c) * P4 + q] = (uint8_t)a;
+  Vec4<T> o;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o.v[i] = from_float<T>(best[i]);
+  *reinterpret_cast<Vec4<T>*>(pooled + ((int64_t)z * C + c) * P4 + q) = o;
+  *reinterpret_cast<Byte4*>(arg + ((int64_t)z * C + c) * P4 + q) = a;
 }
 
 // Backward of the pooling and the ReLU in one: dz[z][c][(y, x, b)] = dpool[z][c][(y/2, x/2, b)] if (y, x) was its window's
-// maximum and the ReLU was active there, else 0.  One thread per full-resolution element.  grid (ceil(P / 256), C, K).
+// maximum and the ReLU was active there, else 0.  One thread per four full-resolution elements.  grid (ceil(P / 1024), C, K).
 template <typename T>
 __global__ void __launch_bounds__(256)
 unpool_kernel(const T* __restrict__ dpool, const uint8_t* __restrict__ arg, const uint8_t* __restrict__ mask, int C, int H, int W, int B,
               T* __restrict__ dz, const int32_t* __restrict__ active) {
   const int z = blockIdx.z, c = blockIdx.y;
   if (active != nullptr && !active[z]) return;
-  const int64_t P = (int64_t)H * W * B;
-  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int P = H * W * B;
+  const int p = ((int)blockIdx.x * (int)blockDim.x + (int)threadIdx.x) * 4;
   if (p >= P) return;
-  const int b = (int)(p % B), x = (int)((p / B) % W), y = (int)(p / ((int64_t)B * W));
-  const int64_t q = ((int64_t)(y / 2) * (W / 2) + x / 2) * B + b;
+  const int b = p % B, pix = p / B;
+  const int x = pix % W, y = pix / W;
+  const int q = ((y / 2) * (W / 2) + x / 2) * B + b;
   const int64_t pc = ((int64_t)z * C + c);
-  const bool hit = arg[pc * (P / 4) + q] == (uint8_t)((y & 1) * 2 + (x & 1)) && mask[pc * P + p] != 0;
-  dz[pc * P + p] = hit ? dpool[pc * (P / 4) + q] : from_float<T>(0.f);
+  const Byte4 ar = *reinterpret_cast<const Byte4*>(arg + pc * (P / 4) + q);
+  const Byte4 mk = *reinterpret_cast<const Byte4*>(mask + pc * P + p);
+  const Vec4<T> dp = *reinterpret_cast<const Vec4<T>*>(dpool + pc * (P / 4) + q);
+  const uint8_t me = (uint8_t)((y & 1) * 2 + (x & 1));
+  Vec4<T> o;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o.v[i] = (ar.v[i] == me && mk.v[i] != 0) ? dp.v[i] : from_float<T>(0.f);
+  *reinterpret_cast<Vec4<T>*>(dz + pc * P + p) = o;
 }
 
 // Gradient w.r.t. a convolution's input from the gradient of its patch matrix:
 //   da[z][ci][(y, x, b)] = sum over (kh, kw) ascending of dcol[z][ci * 9 + kh * 3 + kw][(y - kh + 1, x - kw + 1, b)]  (terms outside the image dropped)
-// summed in fp32, stored as T.  One thread per element.  grid (ceil(P / 256), Cin, K).
+// summed in fp32, stored as T.  One thread per four elements.  grid (ceil(P / 1024), Cin, K).
 template <typename T>
 __global__ void __launch_bounds__(256)
 col2im_kernel(const T* __restrict__ dcol, int Cin, int H, int W, int B, T* __restrict__ da, const int32_t* __restrict__ active) {
   const int z = blockIdx.z, ci = blockIdx.y;
   if (active != nullptr && !active[z]) return;
-  const int64_t P = (int64_t)H * W * B;
-  const int64_t p = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  const int P = H * W * B;
+  const int p = ((int)blockIdx.x * (int)blockDim.x + (int)threadIdx.x) * 4;
   if (p >= P) return;
-  const int b = (int)(p % B), x = (int)((p / B) % W), y = (int)(p / ((int64_t)B * W));
-  float s = 0.f;
+  const int b = p % B, pix = p / B;
+  const int x = pix % W, y = pix / W;
+  float s[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
   for (int kh = 0; kh < 3; ++kh)
 #pragma unroll
     for (int kw = 0; kw < 3; ++kw) {
       const int yy = y - kh + 1, xx = x - kw + 1;
       if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
-      s += to_float(dcol[((int64_t)z * Cin * 9 + ci * 9 + kh * 3 + kw) * P + ((int64_t)yy * W + xx) * B + b]);
+      const Vec4<T> v = *reinterpret_cast<const Vec4<T>*>(dcol + ((int64_t)z * Cin * 9 + ci * 9 + kh * 3 + kw) * P + (yy * W + xx) * B + b);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) s[i] += to_float(v.v[i]);
     }
-  da[((int64_t)z * Cin + ci) * P + p] = from_float<T>(s);
+  Vec4<T> o;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) o.v[i] = from_float<T>(s[i]);
+  *reinterpret_cast<Vec4<T>*>(da + ((int64_t)z * Cin + ci) * P + p) = o;
 }
 
 // ------------------------------------------------------------------------------------------------ least squares
