@@ -92,6 +92,7 @@ gather_t_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, con
 // hidden layer: v = acc + bias[f]; r = relu(v); mask = v > 0; out = TA(skip + r)
 template <typename TP, typename TA>
 struct EpiFwdHidden {
+  static constexpr bool kRowsContiguous = true;  // what it writes is contiguous along the GEMM's M index (the sample)
   const TP* bias;  int64_t ld_p;           // bias[z * ld_p + f]
   TA* out;  const TA* skip;  uint8_t* mask;  // [K, width, ldb]
   int width, ldb;
@@ -108,6 +109,7 @@ struct EpiFwdHidden {
 // head: logits = acc + bias[f]  (fp32, not rounded)
 template <typename TP>
 struct EpiFwdHead {
+  static constexpr bool kRowsContiguous = true;
   const TP* bias;  int64_t ld_p;
   float* logits;  // [K, width, ldb]
   int width, ldb;
@@ -171,6 +173,7 @@ head_chunk_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, int64_t a_plan
 // dgrad of layer l: dh = TA(acc + skip_grad);  dz_prev = mask_prev ? dh : 0;  optionally keep dh (residual nets)
 template <typename TA>
 struct EpiDgrad {
+  static constexpr bool kRowsContiguous = true;
   const TA* dh_next;      // gradient w.r.t. the output of a residual layer (nullptr otherwise) [K, width, ldb]
   TA* dh_out;             // nullable
   TA* dz_prev;            // [K, width, ldb]
@@ -187,6 +190,7 @@ struct EpiDgrad {
 
 // wgrad: g[z][w_off + o * in + i] = acc
 struct EpiWgrad {
+  static constexpr bool kRowsContiguous = false;  // g[o][i]: contiguous along the GEMM's N index
   float* g;  int64_t ld_g, w_off;  int in;
   __device__ inline void operator()(int z, int o, int i, float acc) const {
     g[(int64_t)z * ld_g + w_off + (int64_t)o * in + i] = acc;
@@ -347,20 +351,51 @@ gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd_all, Epi ep
     }
     if (grp == 1) return;
   }
+  if constexpr (Epi::kRowsContiguous) {
+    // the epilogue writes buffers that are contiguous along M (the sample index), while a thread holds 8 x 4 outputs with its
+    // lanes spread along N: turn the tile through shared memory, 16 columns at a time, so that a warp hands the functor 32
+    // consecutive rows of one column and every access it makes is coalesced
+    constexpr int TC = 16;  // columns per turn
+    float (*tr)[BM + 1] = reinterpret_cast<float (*)[BM + 1]>(smem);  // [TC][BM + 1] floats, in the tile memory the main loop is done with
+    static_assert(TC * (BM + 1) <= A_FLOATS + B_FLOATS && BN % TC == 0 && TC % 4 == 0, "transpose buffer");
+    const int warp = tid >> 5, lane = tid & 31;
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int gm = m0 + ty * 8 + i;
-    if (gm >= M) continue;
+    for (int h = 0; h < BN / TC; ++h) {
+      group_sync();  // the main loop (or the previous turn) has been read
+      if (tx / (TC / 4) == h) {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int gn = n0 + tx * 4 + j;
-      if (gn < N) epi((int)blockIdx.z, gm, gn, acc[i][j]);
+        for (int i = 0; i < 8; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) tr[(tx % (TC / 4)) * 4 + j][ty * 8 + i] = acc[i][j];
+      }
+      group_sync();
+      for (int nl = warp; nl < TC; nl += 8) {
+        const int gn = n0 + h * TC + nl;
+        if (gn >= N) break;  // rows of a warp ascend: nothing further is inside
+#pragma unroll
+        for (int q = 0; q < BM / 32; ++q) {
+          const int gm = m0 + q * 32 + lane;
+          if (gm < M) epi((int)blockIdx.z, gm, gn, tr[nl][q * 32 + lane]);
+        }
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int gm = m0 + ty * 8 + i;
+      if (gm >= M) continue;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int gn = n0 + tx * 4 + j;
+        if (gn < N) epi((int)blockIdx.z, gm, gn, acc[i][j]);
+      }
     }
   }
 }
 
 // partial products of a contraction split over blocks: part[zz][m][n], zz = replica * parts + part
 struct EpiPartial {
+  static constexpr bool kRowsContiguous = false;
   float* part;  int M, N;
   __device__ inline void operator()(int zz, int m, int n, float acc) const { part[((int64_t)zz * M + m) * N + n] = acc; }
 };
