@@ -385,6 +385,7 @@ def test_fused_update_in_the_weight_gradient_epilogue_matches_oracle(model, widt
     ((3, 8, 12), (32, 10), 8, 8, 3, 16),     # two convolutions, two dense layers
     ((2, 5), (7,), 4, 8, 2, 16),             # one convolution straight into the head, non-square image
     ((1, 4, 6, 9), (20, 5), 16, 16, 2, 32),  # three convolutions, positions spanning several GEMM tiles
+    ((3, 16), (24, 10), 8, 8, 2, 16),        # 256 flattened inputs into the first dense layer: its forward is split over blocks
 ])
 @pytest.mark.parametrize("dtype", [G.GEMM_FP32, G.GEMM_BF16])
 def test_convolutional_model_matches_oracle(channels, dense, H, W, K, B, dtype):
@@ -398,6 +399,18 @@ def test_convolutional_model_matches_oracle(channels, dense, H, W, K, B, dtype):
     bf = dtype == G.GEMM_BF16
     _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_BF16 if bf else TOL_STEP_FP32, TOL_TRAJ_BF16 if bf else TOL_TRAJ_FP32, steps=12, forced=2,
                               what=f"cnn {channels} {dense}")
+    p.close()
+
+
+def test_convolutional_workload_of_the_bench_at_full_shape():
+    # what bench.py --workload cnn times: 3x32x32 inputs, conv 32 - conv 64 - 256 - 10, K = 4, B = 64, fp32 (weight gradients of the
+    # convolutions and the forward of the 4096 -> 256 layer split over blocks, block-wide bias gradients, four-sample helpers)
+    channels, dense, H, W, K, B = (3, 32, 64), (256, 10), 32, 32, 4, 64
+    X, labels = synth.gaussian_mixture(400, channels[0] * H * W, dense[-1], seed=5)
+    w0 = synth.cnn_init(channels, dense, H, W, seed=6)
+    p = Pair(G.MODEL_CNN, widths=tuple(channels) + tuple(dense), K=K, batch=B, X=X, Y=labels, x0=synth.replicate(w0, K, jitter=0.01, seed=6), y0=w0,
+             gemm_dtype=G.GEMM_FP32, flags=G.FLAG_KEEP_G1 | G.FLAG_STEP_INFO, n_conv=2, img_h=H, img_w=W, tau=2, lam=0.4, seed=3)
+    _per_step_then_trajectory(p, 0.002, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, steps=4, forced=1, what="cnn bench shape")
     p.close()
 
 
