@@ -96,6 +96,10 @@ __device__ inline void tma_load_3d_pair(void* dst, const CUtensorMap* map, int c
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster_addr)
       : "memory");
 }
+// Bring a tensor map (a kernel parameter) into the descriptor cache before the first copy that uses it.
+__device__ inline void prefetch_tensormap(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
 __device__ inline uint32_t cluster_ctarank() {
   uint32_t r;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
@@ -363,6 +367,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const int n_off = (int)rank * B_ROWS;      // this CTA's share of the N side of B
 
   if (threadIdx.x == 0) {
+    tc::prefetch_tensormap(&map_a);
+    tc::prefetch_tensormap(&map_b);
+    if (tc_epi_is_wgrad(EPI)) tc::prefetch_tensormap(&map_c);
     for (int s = 0; s < STAGES; ++s) { tc::mbar_init(&full[s], 1); tc::mbar_init(&empty[s], 1); }
     for (int s = 0; s < 2; ++s) { tc::mbar_init(&acc_full[s], 1); tc::mbar_init(&acc_empty[s], PAIR ? 2 * kTcEpiWarps : kTcEpiWarps); }
     for (int s = 0; s < 8; ++s) tc::mbar_init(&bias_bar[s], 2);
@@ -988,8 +995,6 @@ struct TcPlan {
   bool allow_pair = true;       // false: every GEMM on the single-CTA kernels
   bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
   bool allow_astat = true;      // false: the weight gradient walks single tiles
-  bool allow_bstat = true;      // false: no B-stationary weight gradient (the A-stationary form instead)
-  bool pair_wgrad = true;       // the weight gradient of wide layers by pairs of CTAs with the dz block stationary
   int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
 };
 
@@ -1091,12 +1096,12 @@ inline int tc_plan(TcPlan& P, const lsam_config& c, const std::vector<TcLayer>& 
       // a minibatch of at most 256 samples (four k-blocks): the dz block stays in shared memory over a run of tiles; with 256-wide
       // tiles a pair of CTAs shares each activation tile on top of that (each CTA takes in half of it)
       const bool astat_ok = P.allow_astat && B <= kTcAstatKBlocks * kTcBlockK;
-      if (P.allow_pair && P.pair_wgrad && astat_ok && g.M >= 256 && g.block_n == 256) g.pair = true;
+      if (P.allow_pair && astat_ok && g.M >= 256 && g.block_n == 256) g.pair = true;
       g.astat = astat_ok && (!g.pair || g.block_n >= 128);
       // single CTAs with 256-wide tiles: the activation block (256 rows) is the larger operand, so it is the one to keep in shared
       // memory: a tile then takes in 128 instead of 256 rows (measured inside the step at B = 256, 4096-wide layers: 783-798 -> 823-837
       // TFLOP/s; no gain with two k-blocks, B = 128, where the stores of the tile are what takes the time)
-      g.bstat = g.astat && !g.pair && P.allow_bstat && g.block_n == 256 && B > 2 * kTcBlockK;
+      g.bstat = g.astat && !g.pair && g.block_n == 256 && B > 2 * kTcBlockK;
       if (g.bstat) g.astat = false;
       ok &= tc_make_map(&g.map_a, b.dz[cur], B, ly.out, ZM, ldb, (uint64_t)ly.out * ldb, 64, kTcBlockM);
       ok &= tc_make_map(&g.map_b, b.act[l], B, ly.in, ZM, ldb, (uint64_t)ly.in * ldb, 64, g.pair ? g.block_n / 2 : g.block_n);  // a CTA of a pair loads half the rows
