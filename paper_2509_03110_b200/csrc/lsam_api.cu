@@ -601,6 +601,8 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
   // bf16 tensor-core path keeps its GEMM)
   const bool narrow = L.layers[nl - 1].out <= kHeadMaxOut && (!c->use_tc || L.x3);
   const int64_t p_plane = L.x3 ? (int64_t)K * ld : 0;
+  // on the SIMT paths the same heads go backward through head_dgrad_kernel (the three-plane form keeps its GEMM, which measured the same)
+  const bool head_bwd = narrow && nl >= 2 && !c->use_tc;
   // forward
   for (int l = 0; l < nl; ++l) {
     const LayerInfo& li = L.layers[l];
@@ -645,7 +647,18 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
     const int64_t dz_plane = L.x3 ? (int64_t)K * li.out * ldb : 0;
     const T* a_in = c->at<T>(L.act[l]);
     // tensor-core path: the dgrad of the layer above has already left this layer's bias gradient (and its sum of squares)
-    const bool bias_done = c->use_tc && l < nl - 1 && tc_dgrad_can_fuse_bias(c->tc, l + 1);
+    // (and so has the backward kernel of a narrow head, on every path that uses it)
+    const bool bias_done = (c->use_tc && l < nl - 1 && tc_dgrad_can_fuse_bias(c->tc, l + 1)) || (head_bwd && l == nl - 2);
+    // backward through a narrow head into the layer below, with that layer's bias gradient
+    auto head_dgrad = [&]() -> int {
+      const LayerInfo& lp = L.layers[l - 1];
+      const int64_t out_plane = L.x3 ? (int64_t)K * li.in * ldb : 0;
+      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, head_dgrad_kernel<T><<<dim3((unsigned)ceil_div(li.in, 8), K), 256, 0, c->stream>>>(
+          dz, dz_plane, P, ld, li.w_pad, p_plane, li.in, li.out, B, ldb, c->at<uint8_t>(L.mask[l - 1]), c->at<T>(L.dz[cur ^ 1]),
+          lp.residual ? c->at<T>(L.dh[l & 1]) : nullptr, out_plane, c->g(), ld, lp.b_pad, c->use_tc ? c->at<float>(L.partial) : nullptr, L.nchunks,
+          c->use_tc ? c->tc.bias_slot0[l - 1] : 0, c->act()));
+      return LSAM_OK;
+    };
     if (!bias_done) {
       float* part = c->use_tc ? c->at<float>(L.partial) : nullptr;
       const int slot0 = c->use_tc ? c->tc.bias_slot0[l] : 0;
@@ -659,6 +672,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
       int trc = 0;
       auto dgrad = [&]() -> int {
         if (l == 0) return LSAM_OK;
+        if (head_bwd && l == nl - 1) return head_dgrad();
         void* bias_g = nullptr;
         if (tc_dgrad_can_fuse_bias(c->tc, l)) bias_g = g_bf16 ? (void*)c->at<bf16>(L.g1b) : (void*)c->g();
         LAUNCH(c, LSAM_PROF_GEMM_DGRAD, trc = tc_dgrad(c->tc, l, c->stream, bias_g, g_bf16));
@@ -682,7 +696,9 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
       rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.out, li.in, B, e);
       if (rc != LSAM_OK) return rc;
     }
-    if (l > 0) {
+    if (l > 0 && head_bwd && l == nl - 1) {
+      if ((rc = head_dgrad()) != LSAM_OK) return rc;
+    } else if (l > 0) {
       GemmOperand A{dz, (int64_t)li.out * ldb, 1, ldb};      // (z, b, o)
       GemmOperand W{P + li.w_pad, ld, 1, li.in};             // (z, i, o)
       EpiDgrad<T> e{li.residual ? c->at<T>(L.dh[(l + 1) & 1]) : nullptr,

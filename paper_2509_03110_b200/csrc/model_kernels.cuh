@@ -170,6 +170,61 @@ head_chunk_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, int64_t a_plan
     if (f < out) dst[(int64_t)f * ldb] = acc[f];
 }
 
+// Backward through a narrow head (out <= kHeadMaxOut classes) into the layer below, with that layer's bias gradient:
+//   dh[i][b] = sum_c W[c][i] dz[c][b] (classes ascending);  dz_prev[i][b] = mask[i][b] ? T(dh) : 0;  dh_out = T(dh) (skip connections, nullable);
+//   db[i] = sum_b dz_prev[i][b] as stored -> g[z][b_off + i];  sum of squares of the block's 8 db -> partial[z][slot0 + blockIdx.x] (nullable).
+// A GEMM would contract over at most 16 classes.  Warp w owns input unit i = 8 blockIdx.x + w, its lanes stride the samples (coalesced).
+// dz_plane / p_plane / out_plane != 0: backward signals / parameters / outputs are three bf16 planes.  grid (ceil(in / 8), K), block 256.
+template <typename T>
+__global__ void __launch_bounds__(256)
+head_dgrad_kernel(const T* __restrict__ dz, int64_t dz_plane, const T* __restrict__ P, int64_t ld_p, int64_t w_off, int64_t p_plane, int in, int out,
+                  int B, int ldb, const uint8_t* __restrict__ mask_prev, T* __restrict__ dz_prev, T* __restrict__ dh_out, int64_t out_plane,
+                  float* __restrict__ g, int64_t ld_g, int64_t b_off, float* __restrict__ partial, int64_t ld_partial, int slot0,
+                  const int32_t* __restrict__ active) {
+  const int z = blockIdx.y;
+  if (active != nullptr && !active[z]) return;
+  __shared__ float wv[8][kHeadMaxOut];
+  __shared__ float sq[8];
+  __shared__ float dzs[kHeadMaxOut][256];  // the backward signal of 256 samples, planes already summed: read once per block, used by its 8 warps
+  const int w = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int i0 = blockIdx.x * 8, i = i0 + w;
+  if (threadIdx.x < 8 * kHeadMaxOut) {
+    const int u = threadIdx.x / kHeadMaxOut, c = threadIdx.x % kHeadMaxOut;
+    wv[u][c] = (c < out && i0 + u < in) ? load_planes(P + (int64_t)z * ld_p + w_off + (int64_t)c * in + i0 + u, p_plane) : 0.f;
+  }
+  float bs = 0.f;
+  for (int b0 = 0; b0 < B; b0 += 256) {
+    __syncthreads();  // the weights are in place / the previous chunk has been used
+    const int nb = min(256, B - b0);
+    for (int c = 0; c < out; ++c) dzs[c][threadIdx.x] = (int)threadIdx.x < nb ? load_planes(dz + ((int64_t)z * out + c) * ldb + b0 + threadIdx.x, dz_plane) : 0.f;
+    __syncthreads();
+    if (i < in) {
+      for (int bl = lane; bl < nb; bl += 32) {
+        float s = 0.f;
+        for (int c = 0; c < out; ++c) s = fmaf(wv[w][c], dzs[c][bl], s);
+        const int64_t e = ((int64_t)z * in + i) * ldb + b0 + bl;
+        if (dh_out != nullptr) store_planes(dh_out + e, out_plane, s);
+        const float v = mask_prev[e] ? s : 0.f;
+        store_planes(dz_prev + e, out_plane, v);
+        bs += (sizeof(T) == 2 && out_plane == 0) ? to_float(from_float<T>(v)) : v;  // the value as stored (three planes hold it exactly)
+      }
+    }
+  }
+  bs = warp_sum(bs);
+  if (lane == 0) {
+    if (i < in) g[(int64_t)z * ld_g + b_off + i] = bs;
+    sq[w] = i < in ? bs * bs : 0.f;
+  }
+  if (partial != nullptr) {
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+      for (int q = 0; q < 8; ++q) t += sq[q];
+      partial[(int64_t)z * ld_partial + slot0 + blockIdx.x] = t;
+    }
+  }
+}
+
 // dgrad of layer l: dh = TA(acc + skip_grad);  dz_prev = mask_prev ? dh : 0;  optionally keep dh (residual nets)
 template <typename TA>
 struct EpiDgrad {
