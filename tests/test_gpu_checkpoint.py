@@ -30,7 +30,8 @@ def _make(kind):
     extra = dict(noise_temp=1e-3) if bf else dict(active_num=170)
     dX, dY = torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda()
     mk = lambda x_init: G.Lsam(G.make_config(G.MODEL_RESMLP if bf else G.MODEL_MLP, widths=widths, K=3, batch=48, n_samples=300,
-                                             gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32, **extra, **HP),
+                                             gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32,
+                                             gemm_impl=G.IMPL_TCGEN05 if kind == "mlp_fp32_tcgen05_async" else G.IMPL_AUTO, **extra, **HP),
                                dX, dY, torch.from_numpy(x_init).cuda(), torch.from_numpy(w0).cuda())
     return mk, x0
 
@@ -42,7 +43,7 @@ def _run(c, t0, t1):
             assert c.couple() == 0
 
 
-@pytest.mark.parametrize("kind", ["flat", "mlp_fp32_async", "resmlp_bf16_tcgen05"])
+@pytest.mark.parametrize("kind", ["flat", "mlp_fp32_async", "mlp_fp32_tcgen05_async", "resmlp_bf16_tcgen05"])  # the third: operand planes rebuilt from the loaded x
 def test_resumed_run_continues_bit_for_bit(kind):
     mk, x0 = _make(kind)
     a = mk(x0)
