@@ -329,7 +329,7 @@ def workload_config(w):
 
 
 # ---------------------------------------------------------------------------------------------- one workload on this rank's GPU
-def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True, gemm_impl=0, fused_update=False):
+def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_graph="auto", grad_fp32=False, with_e2e=True, with_cpu=True, gemm_impl=0, fused_update=False, pdl=False):
     """Create the context, time `steps` steps after `warmup` untimed ones, and return the record of this workload
     (rank 0; None on the other ranks).  A step is one pass of the whole hot path plus the centre update when it is due."""
     import torch
@@ -347,7 +347,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
     # That needs a capturable stream; the per-kernel shares then come from a second pass over the same steps with per-launch events.
     small = 4.0 * w["K"] * param_count(w) <= 126e6
     use_graph = (not fused_update) if cuda_graph == "auto" else cuda_graph == "on"
-    flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0) | (G.FLAG_FUSED_UPDATE if fused_update else 0)
+    flags = (G.FLAG_CUDA_GRAPH if use_graph else 0) | (G.FLAG_GRAD_FP32 if grad_fp32 else 0) | (G.FLAG_FUSED_UPDATE if fused_update else 0) | (G.FLAG_PDL if pdl else 0)
     cfg = make_cfg(G, w, flags=flags, K_total=world * w["K"] if shard else 0, k_offset=rank * w["K"] if shard else 0, gemm_impl=gemm_impl)
     torch.cuda.synchronize()
     work_stream = torch.cuda.Stream(device=dev)
@@ -553,7 +553,7 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
         cpu, _ = oracle_baseline(w, key, X, Y, inp["y0"].cpu().numpy())
 
     cfgd = workload_config(w)
-    cfgd.update(gemm=("tcgen05, fp32 as three bf16 planes per operand" if x3 else "tcgen05 (single-CTA kernels only)" if gemm_impl == G.IMPL_TCGEN05_1CTA else "tcgen05") if uses_tc else "simt", cuda_graph=bool(use_graph),
+    cfgd.update(gemm=("tcgen05, fp32 as three bf16 planes per operand" if x3 else "tcgen05 (single-CTA kernels only)" if gemm_impl == G.IMPL_TCGEN05_1CTA else "tcgen05") if uses_tc else "simt", cuda_graph=bool(use_graph), pdl=bool(pdl),
                 l2=("working set larger than L2" if not small else "L2-resident state (latency-bound workload)") +
                    ("" if events_in_timed else "; kernel shares and roofline from a separate pass over the same steps with per-launch events"),
                 parallelism=(f"{world * w['K']} workers sharded over {world} GPU(s), one centre, accumulator all-reduce every tau steps" if shard
@@ -595,6 +595,7 @@ def main():
                     help="N > 1: one job of N*K workers with a single centre, K workers per GPU, accumulator all-reduce every tau steps "
                          "(default: N independent copies of the workload)")
     ap.add_argument("--cuda-graph", default="auto", choices=["auto", "on", "off"], help="replay each tick as one CUDA graph (auto: on)")
+    ap.add_argument("--pdl", default="on", choices=["on", "off"], help="launch the kernels of a tick with programmatic stream serialization (LSAM_FLAG_PDL)")
     args = ap.parse_args()
     w = dict(WORKLOADS[args.workload])
     modified = False
@@ -637,10 +638,10 @@ def main():
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
     rec = run_workload(args.workload, w, args.steps, args.warmup, dev, rank, world, shard=shard, cuda_graph=args.cuda_graph,
-                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline, fused_update=args.fused_update,
+                       grad_fp32=args.grad_fp32, with_e2e=True, with_cpu=not args.no_cpu_baseline, fused_update=args.fused_update, pdl=args.pdl == "on",
                        gemm_impl={"auto": 0, "simt": 1, "tcgen05": 2, "tcgen05-1cta": 3, "tcgen05-pairs": 4}[args.gemm_impl])
     others = []
-    modified = modified or args.gemm_impl != "auto" or args.grad_fp32 or args.fused_update
+    modified = modified or args.gemm_impl != "auto" or args.grad_fp32 or args.fused_update or args.pdl != "on"
     want_others = args.others == "on" or (args.others == "auto" and world == 1 and args.workload == "c4" and not modified and not shard)
     if want_others and world == 1:
         for key, over, nsteps in OTHER_WORKLOADS:
@@ -649,7 +650,7 @@ def main():
             ow.update(over)
             if "d" in over:
                 ow["name"] = f"optimiser-only sweep point d={over['d']}, K={ow['K']}"
-            r = run_workload(key, ow, nsteps, 5, dev, rank, world, cuda_graph="auto", with_e2e=False, with_cpu=False)
+            r = run_workload(key, ow, nsteps, 5, dev, rank, world, cuda_graph="auto", with_e2e=False, with_cpu=False, pdl=args.pdl == "on")
             ro = r["roofline"]
             others.append(dict(workload=r["config"]["workload"], metric=r["metric"], value=r["value"], unit=r["unit"], ms_per_step=r["ms_per_step"], steps=nsteps, warmup=5,
                                config=r["config"], clocks=r["clocks"], gpu_launches=r["gpu_launches"],

@@ -80,10 +80,16 @@ enum {
                               LSAM_ERR_INVALID otherwise); ignored while profiling is enabled               */
   LSAM_FLAG_GRAD_FP32 = 8,  /* tensor-core path: store g1 and g2 in fp32 instead of bf16 (4 instead of 2 bytes per
                               element written by the weight-gradient GEMM and read back by perturbation and update) */
-  LSAM_FLAG_FUSED_UPDATE = 16 /* tensor-core path: apply the worker update of the weights inside the epilogue of the descent-pass
+  LSAM_FLAG_FUSED_UPDATE = 16, /* tensor-core path: apply the worker update of the weights inside the epilogue of the descent-pass
                               weight-gradient GEMM, so that the descent gradient of the weights never reaches memory (biases keep
                               the streaming update kernel).  Needs the tensor-core path, noise_temp = 0, dp_average = 0 and no
                               LSAM_FLAG_CUDA_GRAPH (lsam_init: LSAM_ERR_INVALID otherwise); lsam_read_grads(2) is then unavailable */
+  LSAM_FLAG_PDL = 32        /* programmatic dependent launch: kernels of a tick are launched with programmatic stream serialization, so
+                              that a kernel's blocks may become resident, and run their set-up, while the kernel before it drains; each
+                              kernel waits for all earlier ones before its first access to global memory, so results are those of
+                              plain in-order launches, bit for bit.  Taken by the tensor-core GEMMs, and, in contexts without them,
+                              by the kernels with small grids (where it was measured to pay); works with and without
+                              LSAM_FLAG_CUDA_GRAPH (the edges are recorded into the graph); inert while profiling is enabled    */
 };
 
 /* Models.

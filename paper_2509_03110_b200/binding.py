@@ -16,7 +16,7 @@ MODEL_LSQ, MODEL_MLP, MODEL_RESMLP, MODEL_FLAT, MODEL_CNN = 0, 1, 2, 3, 4
 GEMM_FP32, GEMM_BF16 = 0, 1
 IMPL_AUTO, IMPL_SIMT, IMPL_TCGEN05, IMPL_TCGEN05_1CTA, IMPL_TCGEN05_PAIRS = 0, 1, 2, 3, 4
 KERNEL_GAUSSIAN, KERNEL_EXP_POWER, KERNEL_CAUCHY, KERNEL_MATERN32 = 0, 1, 2, 3
-FLAG_KEEP_G1, FLAG_STEP_INFO, FLAG_CUDA_GRAPH, FLAG_GRAD_FP32, FLAG_FUSED_UPDATE = 1, 2, 4, 8, 16
+FLAG_KEEP_G1, FLAG_STEP_INFO, FLAG_CUDA_GRAPH, FLAG_GRAD_FP32, FLAG_FUSED_UPDATE, FLAG_PDL = 1, 2, 4, 8, 16, 32
 PROF_CLASSES = ["schedule", "gather", "gemm_fwd", "gemm_dgrad", "gemm_wgrad", "loss", "bias_grad", "lsq_grad", "norm",
                 "perturb", "update", "couple", "copy"]
 

@@ -12,6 +12,16 @@ typedef __nv_bfloat16 bf16;
 // Device status word: kernels OR these bits in, the host maps them to error codes.
 enum : int { STATUS_NONFINITE = 1, STATUS_TIMEOUT = 2, STATUS_BAD_INDEX = 4 };
 
+// Programmatic dependent launch.  Every kernel of the library opens with this pair: `launch_dependents` lets the next
+// kernel of the stream, if it was launched with programmatic stream serialization, make its blocks resident as soon as
+// every block of this grid has started (so its launch latency and set-up overlap this grid's tail); `wait` then holds
+// this block until the grids before it have completed and their writes are visible.  No global memory is touched before
+// the wait, so a kernel never reads what a predecessor has yet to write nor overwrites what it still reads; the chain is
+// transitive because a grid completes only after its own wait has returned.  Both are no-ops in a plain launch.
+__device__ inline void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ inline void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ inline void grid_dep_sync() { grid_dep_launch(); grid_dep_wait(); }
+
 __host__ __device__ inline int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
 __host__ __device__ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 

@@ -366,6 +366,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   const int m_off = (int)rank * kTcBlockM;   // this CTA's rows inside a tile
   const int n_off = (int)rank * B_ROWS;      // this CTA's share of the N side of B
 
+  // the next kernel's blocks may take the SMs this grid leaves free; this grid's own set-up (barriers, tensor memory, tensor
+  // maps: nothing a predecessor writes) runs before it waits for the grids before it
+  grid_dep_launch();
   if (threadIdx.x == 0) {
     tc::prefetch_tensormap(&map_a);
     tc::prefetch_tensormap(&map_b);
@@ -386,6 +389,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   __syncthreads();
   if (PAIR) tc::cluster_sync_all();  // the peer's barriers exist before anything arrives on them
   tc::tc_fence_after();
+  grid_dep_wait();  // every thread: from here on the roles read and write what earlier kernels produced
   const uint32_t tmem_base = *tmem_slot;
   if (PAIR) {
     // one MMA addresses the accumulator columns of both CTAs with the same number, so the two allocations must agree
@@ -952,6 +956,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 __global__ void wait_selftest_kernel(uint32_t limit, int* __restrict__ status) {
   __shared__ uint64_t bar;
   __shared__ int abort_flag;
+  grid_dep_sync();
   if (threadIdx.x == 0) {
     abort_flag = 0;
     tc::mbar_init(&bar, 1);
@@ -996,6 +1001,7 @@ struct TcPlan {
   bool force_pair = false;      // true: CTA pairs wherever the kernel supports them (test coverage of every pair instantiation)
   bool allow_astat = true;      // false: the weight gradient walks single tiles
   int max_pairs = 0;            // CTA pairs that can be resident at once (0: not yet asked)
+  bool pdl = false;             // launches carry the programmatic-stream-serialization attribute
 };
 
 typedef CUresult (*PFN_encodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -1175,25 +1181,33 @@ inline int tc_launch_one(TcPlan& P, const TcGemm& g, cudaStream_t stream) {
   const int64_t rn = g.ep.run_n > 0 ? g.ep.run_n : 1;
   const int64_t tiles = BSTAT ? (int64_t)P.Z * n_tiles * ceil_div(ceil_div(g.M, tile_m), rn)
                               : (int64_t)P.Z * ceil_div(g.M, tile_m) * (ASTAT ? ceil_div(n_tiles, rn) : n_tiles);  // units of the work list
-  if (!PAIR) {
-    const int grid = (int)(tiles < P.sms ? tiles : P.sms);
-    kern<<<grid, kTcThreads, smem, stream>>>(g.map_a, g.map_b, g.map_c, g.M, g.N, g.Kd, P.Z, g.ep, P.status, P.active);
-    return cudaPeekAtLastError() == cudaSuccess ? 0 : 1;
-  }
-  // one persistent pair of CTAs (a cluster of two) per pair of SMs
+  // one persistent CTA per SM, or one persistent pair of CTAs (a cluster of two) per pair of SMs
   cudaLaunchConfig_t cfg = {};
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-  cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
-  if (P.max_pairs == 0) {
+  cudaLaunchAttribute attr[2];
+  unsigned na = 0;
+  if (PAIR) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = 2; attr[na].val.clusterDim.y = 1; attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.blockDim = dim3(kTcThreads); cfg.dynamicSmemBytes = smem; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = na;
+  if (PAIR && P.max_pairs == 0) {
     cfg.gridDim = dim3((unsigned)(P.sms / 2 * 2));
     int n = 0;
     if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess || n < 1) return 1;
     P.max_pairs = n < P.sms / 2 ? n : P.sms / 2;
   }
-  const int pairs = (int)(tiles < P.max_pairs ? tiles : P.max_pairs);
-  cfg.gridDim = dim3((unsigned)(2 * pairs));
+  if (P.pdl) {
+    attr[na].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[na].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = ++na;
+  }
+  if (PAIR) {
+    const int pairs = (int)(tiles < P.max_pairs ? tiles : P.max_pairs);
+    cfg.gridDim = dim3((unsigned)(2 * pairs));
+  } else {
+    cfg.gridDim = dim3((unsigned)(tiles < P.sms ? tiles : P.sms));
+  }
   int M = g.M, N = g.N, Kd = g.Kd, Z = P.Z;
   int* status = P.status;
   const int32_t* active = P.active;

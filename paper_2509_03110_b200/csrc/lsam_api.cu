@@ -270,6 +270,7 @@ struct lsam_ctx {
   int device = 0;                     // ordinal of the GPU that holds the workspace
   bool grads_bf16 = false;            // tensor-core path with its gradients stored in bf16
   bool fused_update = false;          // LSAM_FLAG_FUSED_UPDATE: weights updated inside the descent-pass weight-gradient epilogue
+  bool pdl = false;                   // LSAM_FLAG_PDL: kernels launched with programmatic stream serialization
   bool have_prev = false;
   bool use_tc = false;
   bool async_on = false;              // 0 < active_num < 256: unequal worker progress
@@ -374,6 +375,36 @@ int prof_end(lsam_ctx* c) {
     if (rc__ != LSAM_OK) return rc__;                          \
   } while (0)
 
+// One kernel launch on the context's stream.  With LSAM_FLAG_PDL a launch may carry the programmatic-stream-serialization
+// attribute: the blocks of the kernel may become resident while the kernel before it in the stream is still draining; every
+// kernel of the library waits for its predecessors (grid_dep_sync) before its first global access, so the results are those
+// of a plain in-order stream.  Which launches take it is a measured choice: the tensor-core GEMMs always (their set-up of
+// barriers, tensor memory and tensor maps then overlaps the tail of the kernel before); the other kernels only in a context
+// without tensor-core GEMMs and only with grids of at most kPdlMaxBlocks blocks (a least-squares tick of 26.5 us took 22.3 us),
+// because beside tensor-core kernels they ran slower with it (perturb8_kernel at 58000 blocks took twice its time, the small
+// kernels of a 784-1024-10 MLP cost 2-9 us more per tick).  A failed launch is picked up by prof_end (cudaPeekAtLastError).
+constexpr int64_t kPdlMaxBlocks = 1024;
+inline void launch_attrs(const lsam_ctx* c, cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, dim3 grid, dim3 block, size_t smem) {
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = c->stream;
+  cfg.attrs = attr; cfg.numAttrs = (c->pdl && (int64_t)grid.x * grid.y * grid.z <= kPdlMaxBlocks) ? 1u : 0u;
+}
+template <typename... KArgs, typename... Args>
+inline void launch_k(lsam_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  launch_attrs(c, cfg, attr, grid, block, smem);
+  cudaLaunchKernelEx(&cfg, kern, std::forward<Args>(args)...);
+}
+// The same for a kernel whose arguments sit in a block of pointers (the kernels of a replayed graph whose arguments change per tick).
+inline cudaError_t launch_p(lsam_ctx* c, const void* kern, dim3 grid, dim3 block, void** ptrs) {
+  cudaLaunchConfig_t cfg = {};
+  cudaLaunchAttribute attr[1];
+  launch_attrs(c, cfg, attr, grid, block, 0);
+  return cudaLaunchKernelExC(&cfg, kern, ptrs);
+}
+
 // Argument blocks of the three kernels whose parameters change from step to step (tick, centre-version history,
 // budget, rho, eta, noise scale).  They are launched through cudaLaunchKernel from these blocks, so that a captured
 // graph can be replayed with cudaGraphExecKernelNodeSetParams on the same blocks.
@@ -405,16 +436,16 @@ int launch_norm(lsam_ctx* c, const float* g, int64_t ldg, int64_t n, bool vec4, 
     // all their blocks in the partial slots; only the fixed-order final sum remains
     FinArgs f{partial, nch, (int64_t)c->tc.n_slots, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act(), {}};
     f.bind();
-    LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(c->cfg.K), dim3(256), f.ptrs, 0, c->stream));
+    LAUNCH(c, LSAM_PROF_NORM, launch_p(c, (const void*)norm_finalize_kernel, dim3(c->cfg.K), dim3(256), f.ptrs));
     return LSAM_OK;
   }
   dim3 grid((unsigned)ceil_div(n, vec4 ? norm_chunk<4>() : norm_chunk<1>()), c->cfg.K);
   if ((int64_t)grid.x > nch) return c->fail(LSAM_ERR_WORKSPACE, "norm: partial-sum buffer too small");
-  if (vec4) LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<4><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch, c->act()));
-  else LAUNCH(c, LSAM_PROF_NORM, sumsq_partial_kernel<1><<<grid, kNormThreads, 0, c->stream>>>(g, ldg, n, partial, nch, c->act()));
+  if (vec4) LAUNCH(c, LSAM_PROF_NORM, launch_k(c, sumsq_partial_kernel<4>, grid, kNormThreads, 0, g, ldg, n, partial, nch, c->act()));
+  else LAUNCH(c, LSAM_PROF_NORM, launch_k(c, sumsq_partial_kernel<1>, grid, kNormThreads, 0, g, ldg, n, partial, nch, c->act()));
   FinArgs f{partial, nch, (int64_t)grid.x, rho, c->cfg.gamma, norm_out, scale_out, c->status(), c->act(), {}};
   f.bind();
-  LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(c->cfg.K), dim3(256), f.ptrs, 0, c->stream));
+  LAUNCH(c, LSAM_PROF_NORM, launch_p(c, (const void*)norm_finalize_kernel, dim3(c->cfg.K), dim3(256), f.ptrs));
   return LSAM_OK;
 }
 
@@ -428,8 +459,8 @@ int launch_perturb(lsam_ctx* c, const TG* g, int64_t ldg, int64_t n, bool vec4) 
   float* xt32 = (x3 && (c->cfg.flags & LSAM_FLAG_KEEP_G1)) ? c->at<float>(c->L.xop) : nullptr;
   const int64_t per = (int64_t)kPertThreads * kPertIter * (vec4 ? 4 : 1);
   dim3 grid((unsigned)ceil_div(n, per), c->cfg.K);
-  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<4, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act(), plane, xt32));
-  else LAUNCH(c, LSAM_PROF_PERTURB, perturb_kernel<1, TP, TG><<<grid, kPertThreads, 0, c->stream>>>(c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act(), plane, xt32));
+  if (vec4) LAUNCH(c, LSAM_PROF_PERTURB, launch_k(c, perturb_kernel<4, TP, TG>, grid, kPertThreads, 0, c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act(), plane, xt32));
+  else LAUNCH(c, LSAM_PROF_PERTURB, launch_k(c, perturb_kernel<1, TP, TG>, grid, kPertThreads, 0, c->x(), c->L.ld, g, ldg, n, c->scale(), xt, c->L.ld, c->act(), plane, xt32));
   return LSAM_OK;
 }
 
@@ -438,12 +469,12 @@ int launch_mean_rows(lsam_ctx* c, const void* g, bool g_is_bf16, int64_t ldg, in
   const int K = c->cfg.K;
   if (vec4) {
     const unsigned grid = (unsigned)ceil_div(n, (int64_t)256 * 4);
-    if (g_is_bf16) LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<4, bf16><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const bf16*>(g), ldg, K, n, out));
-    else LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<4, float><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const float*>(g), ldg, K, n, out));
+    if (g_is_bf16) LAUNCH(c, LSAM_PROF_NORM, launch_k(c, mean_rows_kernel<4, bf16>, grid, 256, 0, reinterpret_cast<const bf16*>(g), ldg, K, n, out));
+    else LAUNCH(c, LSAM_PROF_NORM, launch_k(c, mean_rows_kernel<4, float>, grid, 256, 0, reinterpret_cast<const float*>(g), ldg, K, n, out));
   } else {
     const unsigned grid = (unsigned)ceil_div(n, (int64_t)256);
-    if (g_is_bf16) LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<1, bf16><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const bf16*>(g), ldg, K, n, out));
-    else LAUNCH(c, LSAM_PROF_NORM, mean_rows_kernel<1, float><<<grid, 256, 0, c->stream>>>(reinterpret_cast<const float*>(g), ldg, K, n, out));
+    if (g_is_bf16) LAUNCH(c, LSAM_PROF_NORM, launch_k(c, mean_rows_kernel<1, bf16>, grid, 256, 0, reinterpret_cast<const bf16*>(g), ldg, K, n, out));
+    else LAUNCH(c, LSAM_PROF_NORM, launch_k(c, mean_rows_kernel<1, float>, grid, 256, 0, reinterpret_cast<const float*>(g), ldg, K, n, out));
   }
   return LSAM_OK;
 }
@@ -456,8 +487,8 @@ int launch_pull_weights(lsam_ctx* c) {
   float* partial = c->at<float>(L.partial);
   dim3 grid((unsigned)ceil_div(n, norm_chunk<4>()), K);
   if ((int64_t)grid.x > L.nchunks) return c->fail(LSAM_ERR_WORKSPACE, "pull weights: partial-sum buffer too small");
-  LAUNCH(c, LSAM_PROF_NORM, gap_sumsq_partial_kernel<<<grid, kNormThreads, 0, c->stream>>>(c->x(), L.ld, c->at<float>(L.yring), n, partial, L.nchunks, c->slot(), c->act()));
-  LAUNCH(c, LSAM_PROF_NORM, pull_weight_kernel<<<K, 256, 0, c->stream>>>(partial, L.nchunks, (int64_t)grid.x, c->cfg.kernel_kind, c->cfg.lambda, c->cfg.kernel_param, c->pull_weight(), c->act()));
+  LAUNCH(c, LSAM_PROF_NORM, launch_k(c, gap_sumsq_partial_kernel, grid, kNormThreads, 0, c->x(), L.ld, c->at<float>(L.yring), n, partial, L.nchunks, c->slot(), c->act()));
+  LAUNCH(c, LSAM_PROF_NORM, launch_k(c, pull_weight_kernel, K, 256, 0, partial, L.nchunks, (int64_t)grid.x, c->cfg.kernel_kind, c->cfg.lambda, c->cfg.kernel_param, c->pull_weight(), c->act()));
   return LSAM_OK;
 }
 
@@ -506,7 +537,7 @@ int launch_update(lsam_ctx* c, const void* g, int g_mode, int64_t ldg, int64_t n
   }
   c->upd_func = f;
   void* ptrs[1] = {&a};
-  LAUNCH(c, LSAM_PROF_UPDATE, cudaLaunchKernel((const void*)f, dim3(grid), dim3(kUpdThreads), ptrs, 0, c->stream));
+  LAUNCH(c, LSAM_PROF_UPDATE, launch_p(c, (const void*)f, dim3(grid), dim3(kUpdThreads), ptrs));
   return LSAM_OK;
 }
 
@@ -528,7 +559,7 @@ int launch_update_range(lsam_ctx* c, int64_t off, int64_t n, float eta) {
     f = nes ? update_func<4, true, bf16, true>(false) : update_func<4, false, bf16, true>(false);
   }
   void* ptrs[1] = {&a};
-  LAUNCH(c, LSAM_PROF_UPDATE, cudaLaunchKernel((const void*)f, dim3(grid), dim3(kUpdThreads), ptrs, 0, c->stream));
+  LAUNCH(c, LSAM_PROF_UPDATE, launch_p(c, (const void*)f, dim3(grid), dim3(kUpdThreads), ptrs));
   return LSAM_OK;
 }
 
@@ -548,7 +579,7 @@ SchedArgs make_sched_args(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, 
 int launch_schedule(lsam_ctx* c, int64_t t, int32_t* idx, int32_t* stale, int32_t* ver, int32_t* slot, int64_t budget, int32_t* active) {
   SchedArgs a = make_sched_args(c, t, idx, stale, ver, slot, budget, active);
   a.bind();
-  LAUNCH(c, LSAM_PROF_SCHEDULE, cudaLaunchKernel((const void*)schedule_kernel, dim3(c->cfg.K), dim3(128), a.ptrs, 0, c->stream));
+  LAUNCH(c, LSAM_PROF_SCHEDULE, launch_p(c, (const void*)schedule_kernel, dim3(c->cfg.K), dim3(128), a.ptrs));
   return LSAM_OK;
 }
 
@@ -576,8 +607,8 @@ int launch_simt(lsam_ctx* c, int cls, GemmOperand A, GemmOperand B, int M, int N
   const bool split = parts == 1 && (int64_t)grid.x * grid.y * grid.z < 2 * 148 && Kd >= 8 * kSimtBK;
 #define LSAM_SIMT(AM, BN_)                                                                                                                        \
   do {                                                                                                                                            \
-    if (split) LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 2><<<grid, 512, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act()));              \
-    else LAUNCH(c, cls, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 1><<<grid, 256, 0, c->stream>>>(A, B, M, N, Kd, epi, c->act(), parts, chunk));       \
+    if (split) LAUNCH(c, cls, launch_k(c, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 2>, grid, 512, 0, A, B, M, N, Kd, epi, c->act(), 1, 0));              \
+    else LAUNCH(c, cls, launch_k(c, gemm_simt_kernel<TA, TB, AM, BN_, Epi, 1>, grid, 256, 0, A, B, M, N, Kd, epi, c->act(), parts, chunk));       \
   } while (0)
   if (a_mc) { if (b_nc) LSAM_SIMT(true, true); else LSAM_SIMT(true, false); }
   else      { if (b_nc) LSAM_SIMT(false, true); else LSAM_SIMT(false, false); }
@@ -610,7 +641,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
     const bool head = (l == nl - 1);
     if (head && narrow) {
       dim3 hgrid((unsigned)ceil_div(li.in, kHeadChunkIn), (unsigned)ceil_div(B, 128), K);
-      LAUNCH(c, LSAM_PROF_GEMM_FWD, head_chunk_kernel<T><<<hgrid, 128, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, L.x3 ? (int64_t)K * li.in * ldb : 0, P, ld,
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, launch_k(c, head_chunk_kernel<T>, hgrid, 128, 0, a_in, (int64_t)li.in * ldb, ldb, L.x3 ? (int64_t)K * li.in * ldb : 0, P, ld,
                                                                                      li.w_pad, p_plane, li.in, li.out, B, c->at<float>(L.hpart), c->act()));
       continue;
     }
@@ -635,11 +666,11 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
   const int C = L.layers[nl - 1].out;
   int cur = 0;
   // x3 form: backward signals are three planes, (K * width * ldb) elements apart
-  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
+  LAUNCH(c, LSAM_PROF_LOSS, launch_k(c, softmax_ce_kernel<T>, dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, 
       c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act(),
       L.x3 ? (int64_t)K * C * ldb : 0, narrow ? c->at<float>(L.hpart) : nullptr, (int)ceil_div(L.layers[nl - 1].in, kHeadChunkIn),
       P + L.layers[nl - 1].b_pad, ld, p_plane));
-  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
+  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, launch_k(c, mean_loss_kernel, K, 32, 0, c->at<float>(L.rowloss), B, loss_out, c->act()));
   // backward
   for (int l = nl - 1; l >= 0; --l) {
     const LayerInfo& li = L.layers[l];
@@ -653,7 +684,7 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
     auto head_dgrad = [&]() -> int {
       const LayerInfo& lp = L.layers[l - 1];
       const int64_t out_plane = L.x3 ? (int64_t)K * li.in * ldb : 0;
-      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, head_dgrad_kernel<T><<<dim3((unsigned)ceil_div(li.in, 8), K), 256, 0, c->stream>>>(
+      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, launch_k(c, head_dgrad_kernel<T>, dim3((unsigned)ceil_div(li.in, 8), K), 256, 0, 
           dz, dz_plane, P, ld, li.w_pad, p_plane, li.in, li.out, B, ldb, c->at<uint8_t>(L.mask[l - 1]), c->at<T>(L.dz[cur ^ 1]),
           lp.residual ? c->at<T>(L.dh[l & 1]) : nullptr, out_plane, c->g(), ld, lp.b_pad, c->use_tc ? c->at<float>(L.partial) : nullptr, L.nchunks,
           c->use_tc ? c->tc.bias_slot0[l - 1] : 0, c->act()));
@@ -664,9 +695,9 @@ int mlp_pass(lsam_ctx* c, const T* P, float* loss_out, bool g_bf16, const TcFuse
       const int slot0 = c->use_tc ? c->tc.bias_slot0[l] : 0;
       dim3 bgrid((unsigned)ceil_div(li.out, 8), K);
       if (g_bf16)
-        LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, bf16><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->at<bf16>(L.g1b), ld, li.b_pad, part, L.nchunks, slot0, c->act()));
+        LAUNCH(c, LSAM_PROF_BIAS_GRAD, launch_k(c, bias_grad_kernel<T, bf16>, bgrid, 256, 0, dz, B, li.out, ldb, c->at<bf16>(L.g1b), ld, li.b_pad, part, L.nchunks, slot0, c->act(), (int64_t)0));
       else
-        LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<bgrid, 256, 0, c->stream>>>(dz, B, li.out, ldb, c->g(), ld, li.b_pad, part, L.nchunks, slot0, c->act(), dz_plane));
+        LAUNCH(c, LSAM_PROF_BIAS_GRAD, launch_k(c, bias_grad_kernel<T, float>, bgrid, 256, 0, dz, B, li.out, ldb, c->g(), ld, li.b_pad, part, L.nchunks, slot0, c->act(), dz_plane));
     }
     if (c->use_tc) {
       int trc = 0;
@@ -731,12 +762,12 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
     if (li.conv) {
       const int64_t Pn = (int64_t)li.H * li.W * ldb;
       T* col = c->at<T>(L.col[l]);
-      LAUNCH(c, LSAM_PROF_GATHER, im2col_kernel<T><<<dim3((unsigned)ceil_div(Pn, 1024), li.in, K), 256, 0, c->stream>>>(a_in, li.Cin, li.H, li.W, ldb, col, c->act()));
+      LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, im2col_kernel<T>, dim3((unsigned)ceil_div(Pn, 1024), li.in, K), 256, 0, a_in, li.Cin, li.H, li.W, ldb, col, c->act()));
       GemmOperand A{col, (int64_t)li.in * Pn, 1, Pn};           // (z, position, patch element)
       GemmOperand W{P + li.w_pad, ld, li.in, 1};               // (z, output channel, patch element)
       EpiFwdHidden<T, T> e{P + li.b_pad, ld, c->at<T>(L.zout), nullptr, c->at<uint8_t>(L.mask[l]), li.Cout, (int)Pn};
       if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, (int)Pn, li.Cout, li.in, e)) != LSAM_OK) return rc;
-      LAUNCH(c, LSAM_PROF_GEMM_FWD, maxpool_kernel<T><<<dim3((unsigned)ceil_div(Pn / 4, 1024), li.Cout, K), 256, 0, c->stream>>>(
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, launch_k(c, maxpool_kernel<T>, dim3((unsigned)ceil_div(Pn / 4, 1024), li.Cout, K), 256, 0, 
           c->at<T>(L.zout), li.Cout, li.H, li.W, ldb, c->at<T>(L.act[l + 1]), c->at<uint8_t>(L.parg[l]), c->act()));
       continue;
     }
@@ -744,7 +775,7 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
     GemmOperand W{P + li.w_pad, ld, li.in, 1};
     if (head && narrow) {
       dim3 hgrid((unsigned)ceil_div(li.in, kHeadChunkIn), (unsigned)ceil_div(B, 128), K);
-      LAUNCH(c, LSAM_PROF_GEMM_FWD, head_chunk_kernel<T><<<hgrid, 128, 0, c->stream>>>(a_in, (int64_t)li.in * ldb, ldb, 0, P, ld, li.w_pad, 0, li.in, li.out, B,
+      LAUNCH(c, LSAM_PROF_GEMM_FWD, launch_k(c, head_chunk_kernel<T>, hgrid, 128, 0, a_in, (int64_t)li.in * ldb, ldb, 0, P, ld, li.w_pad, 0, li.in, li.out, B,
                                                                                      c->at<float>(L.hpart), c->act()));
       rc = LSAM_OK;
     } else if (head) {
@@ -756,7 +787,7 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
         // partial products per share of the inputs, then their sum in a fixed order handed to the layer's epilogue
         EpiPartial ep{c->at<float>(L.wpart), B, li.out};
         if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_FWD, A, W, B, li.out, li.in, ep, li.fw_parts, li.fw_chunk)) != LSAM_OK) return rc;
-        LAUNCH(c, LSAM_PROF_GEMM_FWD, sum_parts_epi_kernel<EpiFwdHidden<T, T>><<<dim3((unsigned)ceil_div((int64_t)B * li.out, 256), K), 256, 0, c->stream>>>(
+        LAUNCH(c, LSAM_PROF_GEMM_FWD, launch_k(c, sum_parts_epi_kernel<EpiFwdHidden<T, T>>, dim3((unsigned)ceil_div((int64_t)B * li.out, 256), K), 256, 0, 
             c->at<float>(L.wpart), li.fw_parts, B, li.out, e, c->act()));
         rc = LSAM_OK;
       } else {
@@ -767,10 +798,10 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
   }
   const int C = L.layers[nl - 1].out;
   int cur = 0;
-  LAUNCH(c, LSAM_PROF_LOSS, softmax_ce_kernel<T><<<dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, c->stream>>>(
+  LAUNCH(c, LSAM_PROF_LOSS, launch_k(c, softmax_ce_kernel<T>, dim3((unsigned)ceil_div(B, 32), K), dim3(32, 8), 0, 
       c->at<float>(L.logits), c->at<int32_t>(L.ylab), B, C, ldb, c->at<T>(L.dz[cur]), c->at<float>(L.rowloss), c->status(), c->act(),
       0, narrow ? c->at<float>(L.hpart) : nullptr, (int)ceil_div(L.layers[nl - 1].in, kHeadChunkIn), P + L.layers[nl - 1].b_pad, ld, 0));
-  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, mean_loss_kernel<<<K, 32, 0, c->stream>>>(c->at<float>(L.rowloss), B, loss_out, c->act()));
+  if (loss_out) LAUNCH(c, LSAM_PROF_LOSS, launch_k(c, mean_loss_kernel, K, 32, 0, c->at<float>(L.rowloss), B, loss_out, c->act()));
   // backward.  dz[cur] holds, for a dense layer, the gradient w.r.t. its pre-activation; for a convolution layer, the gradient
   // w.r.t. its POOLED output (the pooling and the ReLU are undone by unpool_kernel)
   for (int l = nl - 1; l >= 0; --l) {
@@ -779,9 +810,9 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
     if (li.conv) {
       const int64_t Pn = (int64_t)li.H * li.W * ldb;
       T* dzc = c->at<T>(L.dzc);
-      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, unpool_kernel<T><<<dim3((unsigned)ceil_div(Pn, 1024), li.Cout, K), 256, 0, c->stream>>>(
+      LAUNCH(c, LSAM_PROF_GEMM_DGRAD, launch_k(c, unpool_kernel<T>, dim3((unsigned)ceil_div(Pn, 1024), li.Cout, K), 256, 0, 
           c->at<T>(L.dz[cur]), c->at<uint8_t>(L.parg[l]), c->at<uint8_t>(L.mask[l]), li.Cout, li.H, li.W, ldb, dzc, c->act()));
-      LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_long_kernel<T><<<dim3((unsigned)li.Cout, K), 256, 0, c->stream>>>(dzc, Pn, li.Cout, Pn, c->g(), ld, li.b_pad, c->act()));
+      LAUNCH(c, LSAM_PROF_BIAS_GRAD, launch_k(c, bias_grad_long_kernel<T>, dim3((unsigned)li.Cout, K), 256, 0, dzc, Pn, li.Cout, Pn, c->g(), ld, li.b_pad, c->act()));
       {
         GemmOperand A{dzc, (int64_t)li.Cout * Pn, Pn, 1};                 // (z, output channel, position)
         GemmOperand Bm{c->at<T>(L.col[l]), (int64_t)li.in * Pn, Pn, 1};   // (z, patch element, position)
@@ -789,7 +820,7 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
           // partial products per share of the positions, then their sum in a fixed order
           EpiPartial e{c->at<float>(L.wpart), li.Cout, li.in};
           if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_WGRAD, A, Bm, li.Cout, li.in, (int)Pn, e, li.wg_parts, li.wg_chunk)) != LSAM_OK) return rc;
-          LAUNCH(c, LSAM_PROF_GEMM_WGRAD, sum_parts_kernel<<<dim3((unsigned)ceil_div((int64_t)li.Cout * li.in, 256), K), 256, 0, c->stream>>>(
+          LAUNCH(c, LSAM_PROF_GEMM_WGRAD, launch_k(c, sum_parts_kernel, dim3((unsigned)ceil_div((int64_t)li.Cout * li.in, 256), K), 256, 0, 
               c->at<float>(L.wpart), li.wg_parts, li.Cout, li.in, c->g(), ld, li.w_pad, c->act()));
         } else {
           EpiWgrad e{c->g(), ld, li.w_pad, li.in};
@@ -802,15 +833,15 @@ int cnn_pass(lsam_ctx* c, const T* P, float* loss_out) {
         GemmOperand W{P + li.w_pad, ld, 1, li.in};                         // (z, patch element, output channel)
         EpiDgrad<T> e{nullptr, nullptr, dcol, nullptr, li.in, (int)Pn};    // the raw gradient of the patch matrix
         if ((rc = launch_simt<T, T>(c, LSAM_PROF_GEMM_DGRAD, A, W, (int)Pn, li.in, li.Cout, e)) != LSAM_OK) return rc;
-        LAUNCH(c, LSAM_PROF_GEMM_DGRAD, col2im_kernel<T><<<dim3((unsigned)ceil_div(Pn, 1024), li.Cin, K), 256, 0, c->stream>>>(
+        LAUNCH(c, LSAM_PROF_GEMM_DGRAD, launch_k(c, col2im_kernel<T>, dim3((unsigned)ceil_div(Pn, 1024), li.Cin, K), 256, 0, 
             dcol, li.Cin, li.H, li.W, ldb, c->at<T>(L.dz[cur ^ 1]), c->act()));
       }
       cur ^= 1;
       continue;
     }
     const T* dz = c->at<T>(L.dz[cur]);
-    LAUNCH(c, LSAM_PROF_BIAS_GRAD, bias_grad_kernel<T, float><<<dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, c->stream>>>(
-        dz, B, li.out, ldb, c->g(), ld, li.b_pad, nullptr, L.nchunks, 0, c->act()));
+    LAUNCH(c, LSAM_PROF_BIAS_GRAD, launch_k(c, bias_grad_kernel<T, float>, dim3((unsigned)ceil_div(li.out, 8), K), 256, 0, 
+        dz, B, li.out, ldb, c->g(), ld, li.b_pad, nullptr, L.nchunks, 0, c->act(), (int64_t)0));
     {
       GemmOperand A{dz, (int64_t)li.out * ldb, ldb, 1};
       GemmOperand Bm{a_in, (int64_t)li.in * ldb, ldb, 1};
@@ -835,7 +866,7 @@ int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false,
   const lsam_config& cfg = c->cfg;
   if (cfg.model == LSAM_MODEL_LSQ) {
     const float* P = perturbed ? c->at<float>(c->L.xop) : c->x();
-    LAUNCH(c, LSAM_PROF_LSQ_GRAD, lsq_grad_kernel<<<cfg.K, 256, sizeof(float) * cfg.batch, c->stream>>>(
+    LAUNCH(c, LSAM_PROF_LSQ_GRAD, launch_k(c, lsq_grad_kernel, cfg.K, 256, sizeof(float) * cfg.batch, 
         c->at<float>(c->L.act[0]), c->at<float>(c->L.ylab), P, c->L.ld, cfg.batch, c->L.in0, c->g(), c->L.ld, loss_out, c->act()));
     return LSAM_OK;
   }
@@ -851,7 +882,7 @@ int grad_pass(lsam_ctx* c, bool perturbed, float* loss_out, bool g_bf16 = false,
 // x3 form: the three bf16 planes of src [K, ld] (x, or the perturbed point) -> xpl
 int launch_split3(lsam_ctx* c, const float* src) {
   dim3 grid((unsigned)ceil_div(c->L.ld, 1024), c->cfg.K);
-  LAUNCH(c, LSAM_PROF_COPY, split3_rows_kernel<<<grid, 256, 0, c->stream>>>(src, c->L.ld, c->L.ld, c->at<bf16>(c->L.xpl), c->L.ld, (int64_t)c->cfg.K * c->L.ld));
+  LAUNCH(c, LSAM_PROF_COPY, launch_k(c, split3_rows_kernel, grid, 256, 0, src, c->L.ld, c->L.ld, c->at<bf16>(c->L.xpl), c->L.ld, (int64_t)c->cfg.K * c->L.ld));
   return LSAM_OK;
 }
 
@@ -859,7 +890,7 @@ int refresh_operand_copy(lsam_ctx* c) {
   if (c->L.x3) return launch_split3(c, c->x());
   if (c->cfg.gemm_dtype != LSAM_GEMM_BF16) return LSAM_OK;
   dim3 grid((unsigned)ceil_div(c->L.ld, 256), c->cfg.K);
-  LAUNCH(c, LSAM_PROF_COPY, cast_rows_kernel<bf16><<<grid, 256, 0, c->stream>>>(c->x(), c->L.ld, c->at<bf16>(c->L.xop), c->L.ld, c->L.ld));
+  LAUNCH(c, LSAM_PROF_COPY, launch_k(c, cast_rows_kernel<bf16>, grid, 256, 0, c->x(), c->L.ld, c->at<bf16>(c->L.xop), c->L.ld, c->L.ld));
   return LSAM_OK;
 }
 
@@ -868,7 +899,7 @@ int seg_copy(lsam_ctx* c, const float* src, int64_t lds, float* dst, int64_t ldd
   int64_t maxlen = 0;
   for (int i = 0; i < c->L.seg.n; ++i) maxlen = c->L.seg.len[i] > maxlen ? c->L.seg.len[i] : maxlen;
   dim3 grid((unsigned)ceil_div(maxlen, 256), c->L.seg.n, rows);
-  LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<TO_PADDED, float, float><<<grid, 256, 0, c->stream>>>(src, lds, dst, ldd, c->L.seg));
+  LAUNCH(c, LSAM_PROF_COPY, launch_k(c, seg_copy_kernel<TO_PADDED, float, float>, grid, 256, 0, src, lds, dst, ldd, c->L.seg));
   return LSAM_OK;
 }
 
@@ -898,13 +929,13 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
   const int64_t rows = (int64_t)cfg.K * cfg.batch;
   if (!flat && gather) {
     if (cfg.model == LSAM_MODEL_LSQ) {
-      LAUNCH(c, LSAM_PROF_GATHER, gather_kernel<float><<<(unsigned)rows, 128, 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, c->L.in0, c->L.in0, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), cfg.batch, c->act()));
+      LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_kernel<float>, (unsigned)rows, 128, 0, c->X, c->Y, c->idx(), cfg.n_samples, c->L.in0, c->L.in0, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), cfg.batch, c->act()));
     } else {
       dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
       if (cfg.gemm_dtype == LSAM_GEMM_BF16 || L.x3)
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act(), c->in_plane()));
+        LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_t_kernel<bf16>, grid, dim3(32, 8), 0, c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<bf16>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act(), c->in_plane()));
       else
-        LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act()));
+        LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_t_kernel<float>, grid, dim3(32, 8), 0, c->X, c->Y, c->idx(), cfg.n_samples, cfg.batch, c->L.in0, L.ldb, c->at<float>(L.act[0]), c->at<uint32_t>(L.ylab), c->status(), c->act(), (int64_t)0));
     }
   }
   const bool vec4 = L.vec4 && (!flat || c->ext_vec4);
@@ -968,7 +999,7 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
     if ((rc = launch_norm(c, g1, ldg, n, vec4, rho, c->norm1(), c->scale())) != LSAM_OK) return rc;
     if (g1_bf16 && vec4 && n % 8 == 0) {
       dim3 pgrid((unsigned)ceil_div(n, (int64_t)kPertThreads * 8 * kPert8Iter), cfg.K);
-      LAUNCH(c, LSAM_PROF_PERTURB, perturb8_kernel<<<pgrid, kPertThreads, 0, c->stream>>>(c->x(), L.ld, c->at<bf16>(L.g1b), ldg, n, c->scale(), c->at<bf16>(L.xop), L.ld, c->act()));
+      LAUNCH(c, LSAM_PROF_PERTURB, launch_k(c, perturb8_kernel, pgrid, kPertThreads, 0, c->x(), L.ld, c->at<bf16>(L.g1b), ldg, n, c->scale(), c->at<bf16>(L.xop), L.ld, c->act()));
       rc = LSAM_OK;
     } else if (g1_bf16) rc = launch_perturb<bf16, bf16>(c, c->at<bf16>(L.g1b), ldg, n, vec4);
     else if (cfg.gemm_dtype == LSAM_GEMM_BF16 || L.x3) rc = launch_perturb<bf16, float>(c, g1, ldg, n, vec4);
@@ -991,7 +1022,7 @@ int step_enqueue(lsam_ctx* c, float eta, float rho, bool gather, int64_t budget)
     for (const LayerInfo& li : L.layers) {
       const int64_t wlen = round_up((int64_t)li.in * li.out, kSegAlign), blen = round_up((int64_t)li.out, kSegAlign);
       if ((rc = launch_update_range(c, li.b_pad, blen, eta)) != LSAM_OK) return rc;  // bias gradients were stored as usual
-      LAUNCH(c, LSAM_PROF_UPDATE, acc_add_kernel<<<(unsigned)ceil_div(wlen, 1024), 256, 0, c->stream>>>(c->x(), L.ld, cfg.K, li.w_pad, wlen, c->at<float>(L.acc), c->act()));
+      LAUNCH(c, LSAM_PROF_UPDATE, launch_k(c, acc_add_kernel, (unsigned)ceil_div(wlen, 1024), 256, 0, c->x(), L.ld, cfg.K, li.w_pad, wlen, c->at<float>(L.acc), c->act()));
     }
     return LSAM_OK;
   }
@@ -1157,6 +1188,7 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
   if (cfg->gemm_impl >= LSAM_IMPL_TCGEN05 && !tc_ok) return bail(LSAM_ERR_INVALID);
   c->use_tc = tc_ok;
   c->grads_bf16 = tc_ok && !L.x3 && !(cfg->flags & LSAM_FLAG_GRAD_FP32);
+  c->pdl = (cfg->flags & LSAM_FLAG_PDL) != 0;
   if (cfg->flags & LSAM_FLAG_FUSED_UPDATE) {
     if (!tc_ok || L.x3 || cfg->noise_temp > 0.f || cfg->dp_average != 0 || (cfg->flags & LSAM_FLAG_CUDA_GRAPH)) return bail(LSAM_ERR_INVALID);
     c->fused_update = true;
@@ -1188,6 +1220,8 @@ int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const voi
     b.g1b = c->at<bf16>(L.g1b);
     c->tc.active = c->act();
     c->tc.allow_pair = cfg->gemm_impl != LSAM_IMPL_TCGEN05_1CTA;
+    c->tc.pdl = c->pdl;
+    c->pdl = false;  // beside tensor-core GEMMs only the GEMMs take the attribute (see launch_k)
     c->tc.force_pair = cfg->gemm_impl == LSAM_IMPL_TCGEN05_PAIRS;
     c->tc.allow_astat = cfg->gemm_impl != LSAM_IMPL_TCGEN05_1CTA;  // the plain single-CTA kernels stay reachable (and tested) through this setting
     std::vector<TcLayer> tl;
@@ -1223,9 +1257,9 @@ int lsam_step_batch(lsam_ctx* c, float eta, float rho, const float* xb, const vo
   if (!lsq) {
     dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
     if (cfg.gemm_dtype == LSAM_GEMM_BF16 || c->L.x3)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr, c->in_plane()));
+      LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_t_kernel<bf16>, grid, dim3(32, 8), 0, xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr, c->in_plane()));
     else
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
+      LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_t_kernel<float>, grid, dim3(32, 8), 0, xdst, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr, (int64_t)0));
   }
   int rc = step_common(c, eta, rho, false);
   if (rc != LSAM_OK) return rc;
@@ -1279,9 +1313,9 @@ int lsam_step_staged(lsam_ctx* c, float eta, float rho, float* h_loss) {
   } else {
     dim3 grid((unsigned)ceil_div(c->L.in0, 32), (unsigned)ceil_div(cfg.batch, 32), cfg.K);
     if (cfg.gemm_dtype == LSAM_GEMM_BF16 || c->L.x3)
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<bf16><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr, c->in_plane()));
+      LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_t_kernel<bf16>, grid, dim3(32, 8), 0, xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<bf16>(c->L.act[0]), nullptr, c->status(), nullptr, c->in_plane()));
     else
-      LAUNCH(c, LSAM_PROF_GATHER, gather_t_kernel<float><<<grid, dim3(32, 8), 0, c->stream>>>(xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr));
+      LAUNCH(c, LSAM_PROF_GATHER, launch_k(c, gather_t_kernel<float>, grid, dim3(32, 8), 0, xs, nullptr, nullptr, rows, cfg.batch, c->L.in0, c->L.ldb, c->at<float>(c->L.act[0]), nullptr, c->status(), nullptr, (int64_t)0));
   }
   LSAM_CUDA(c, cudaEventRecord(c->slot_free[slot], c->stream));
   c->slot_used[slot] = true;
@@ -1312,7 +1346,7 @@ int lsam_couple(lsam_ctx* c) {
   phase.next("lsam S7 couple");
   // divisor n tau of the sync branch: n counts the workers of the whole job (their accumulators have been summed into this one)
   const float inv = 1.0f / ((float)(c->cfg.K_total > 0 ? c->cfg.K_total : c->cfg.K) * (float)c->cfg.tau);
-  LAUNCH(c, LSAM_PROF_COUPLE, couple_kernel<<<(unsigned)ceil_div(L.ld, 256), 256, 0, c->stream>>>(
+  LAUNCH(c, LSAM_PROF_COUPLE, launch_k(c, couple_kernel, (unsigned)ceil_div(L.ld, 256), 256, 0, 
       c->at<float>(L.acc), c->yslot(c->t_y), c->yslot(c->t_y + 1), c->at<float>(L.gprev), L.ld, inv, c->cfg.beta, c->cfg.eta_prime, c->have_prev ? 1 : 0));
   c->have_prev = true;
   c->t_y += 1;
@@ -1376,10 +1410,10 @@ int lsam_read_anchor_gap(lsam_ctx* c, float* h_gap) {
   float* out = c->at<float>(L.scalars) + 4 * (size_t)K;
   dim3 grid((unsigned)ceil_div(n, norm_chunk<4>()), K);
   if ((int64_t)grid.x > L.nchunks) return c->fail(LSAM_ERR_WORKSPACE, "anchor gap: partial-sum buffer too small");
-  LAUNCH(c, LSAM_PROF_NORM, gap_sumsq_partial_kernel<<<grid, kNormThreads, 0, c->stream>>>(c->x(), L.ld, c->yslot(c->t_y), n, partial, L.nchunks, nullptr, nullptr));
+  LAUNCH(c, LSAM_PROF_NORM, launch_k(c, gap_sumsq_partial_kernel, grid, kNormThreads, 0, c->x(), L.ld, c->yslot(c->t_y), n, partial, L.nchunks, nullptr, nullptr));
   FinArgs f{partial, L.nchunks, (int64_t)grid.x, 0.f, c->cfg.gamma, out, nullptr, c->status(), nullptr, {}};
   f.bind();
-  LAUNCH(c, LSAM_PROF_NORM, cudaLaunchKernel((const void*)norm_finalize_kernel, dim3(K), dim3(256), f.ptrs, 0, c->stream));
+  LAUNCH(c, LSAM_PROF_NORM, launch_p(c, (const void*)norm_finalize_kernel, dim3(K), dim3(256), f.ptrs));
   LSAM_CUDA(c, cudaMemcpyAsync(h_gap, out, sizeof(float) * K, cudaMemcpyDeviceToHost, c->stream));
   LSAM_CUDA(c, cudaStreamSynchronize(c->stream));
   return LSAM_OK;
@@ -1400,7 +1434,7 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
         int64_t maxlen = 0;
         for (int i = 0; i < L.seg.n; ++i) maxlen = L.seg.len[i] > maxlen ? L.seg.len[i] : maxlen;
         dim3 grid((unsigned)ceil_div(maxlen, 256), L.seg.n, 1);
-        LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(c->at<bf16>(L.xpkeep) + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
+        LAUNCH(c, LSAM_PROF_COPY, launch_k(c, seg_copy_kernel<false, bf16, float>, grid, 256, 0, c->at<bf16>(L.xpkeep) + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
       } else {
         // fp32 GEMMs on the tensor cores: the perturbed point lives in the three operand planes, which the update overwrites; an fp32 copy is kept on request
         if (L.x3 && !(c->cfg.flags & LSAM_FLAG_KEEP_G1)) return c->fail(LSAM_ERR_STATE, "lsam_read_grads(3) with fp32 GEMMs on the tensor cores needs LSAM_FLAG_KEEP_G1");
@@ -1421,7 +1455,7 @@ static int read_grads_range(lsam_ctx* c, int pass, int k_begin, int k_end, float
         int64_t maxlen = 0;
         for (int i = 0; i < L.seg.n; ++i) maxlen = L.seg.len[i] > maxlen ? L.seg.len[i] : maxlen;
         dim3 grid((unsigned)ceil_div(maxlen, 256), L.seg.n, 1);
-        LAUNCH(c, LSAM_PROF_COPY, seg_copy_kernel<false, bf16, float><<<grid, 256, 0, c->stream>>>(srcb + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
+        LAUNCH(c, LSAM_PROF_COPY, launch_k(c, seg_copy_kernel<false, bf16, float>, grid, 256, 0, srcb + (size_t)k * L.ld, L.ld, tmp, L.d, L.seg));
       } else {
         const float* src = pass == 1 ? c->at<float>(L.g1keep) : c->g();
         rc = seg_copy<false>(c, src + (size_t)k * L.ld, L.ld, tmp, L.d, 1);
@@ -1608,7 +1642,7 @@ int lsam_status(lsam_ctx* c) {
 
 int lsam_selftest_bounded_wait(lsam_ctx* c, uint32_t polls) {
   if (!c || polls == 0 || polls > (1u << 20)) return LSAM_ERR_INVALID;
-  LAUNCH(c, LSAM_PROF_COPY, wait_selftest_kernel<<<1, 32, 0, c->stream>>>(polls, c->status()));
+  LAUNCH(c, LSAM_PROF_COPY, launch_k(c, wait_selftest_kernel, 1, 32, 0, polls, c->status()));
   return LSAM_OK;
 }
 

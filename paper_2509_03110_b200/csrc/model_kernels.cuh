@@ -13,6 +13,7 @@ __global__ void __launch_bounds__(128)
 gather_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx,
               int64_t n_samples, int in, int ld, TA* __restrict__ xb, uint32_t* __restrict__ yb, int* __restrict__ status,
               int B, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int64_t r = blockIdx.x;
   if (active != nullptr && !active[r / B]) return;
   int64_t s = idx[r];
@@ -56,6 +57,7 @@ __global__ void __launch_bounds__(256)
 gather_t_kernel(const float* __restrict__ X, const uint32_t* __restrict__ Y, const int32_t* __restrict__ idx, int64_t n_samples,
                 int B, int in, int ldb, TA* __restrict__ xt, uint32_t* __restrict__ yb, int* __restrict__ status,
                 const int32_t* __restrict__ active, int64_t plane = 0) {
+  grid_dep_sync();
   __shared__ float tile[32][33];
   if (active != nullptr && !active[blockIdx.z]) return;
   const int k = blockIdx.z, i0 = blockIdx.x * 32, b0 = blockIdx.y * 32;
@@ -131,6 +133,7 @@ template <typename T>
 __global__ void __launch_bounds__(128)
 head_chunk_kernel(const T* __restrict__ a, int64_t a_sz, int ldb, int64_t a_plane, const T* __restrict__ P, int64_t ld_p, int64_t w_off,
                   int64_t p_plane, int in, int out, int B, float* __restrict__ part, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.z;
   if (active != nullptr && !active[z]) return;
   __shared__ __align__(16) float w[kHeadChunkIn][kHeadMaxOut];  // [input][class]: a thread reads the 16 weights of an input as four 128-bit broadcasts
@@ -181,6 +184,7 @@ head_dgrad_kernel(const T* __restrict__ dz, int64_t dz_plane, const T* __restric
                   int B, int ldb, const uint8_t* __restrict__ mask_prev, T* __restrict__ dz_prev, T* __restrict__ dh_out, int64_t out_plane,
                   float* __restrict__ g, int64_t ld_g, int64_t b_off, float* __restrict__ partial, int64_t ld_partial, int slot0,
                   const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   __shared__ float wv[8][kHeadMaxOut];
@@ -297,6 +301,7 @@ __device__ inline float4 simt_fetch4(const T* __restrict__ base, int64_t sr, int
 template <typename TA_, typename TB_, bool A_MC, bool B_NC, class Epi, int SPLITK = 1>
 __global__ void __launch_bounds__(256 * SPLITK)
 gemm_simt_kernel(GemmOperand A, GemmOperand Bo, int M, int N, int Kd_all, Epi epi, const int32_t* __restrict__ active, int parts = 1, int chunk = 0) {
+  grid_dep_sync();
   constexpr int BM = kSimtBM, BN = kSimtBN, BK = kSimtBK;
   const int z = parts > 1 ? (int)blockIdx.z / parts : (int)blockIdx.z;
   if (active != nullptr && !active[z]) return;  // a waiting replica
@@ -458,6 +463,7 @@ struct EpiPartial {
 __global__ void __launch_bounds__(256)
 sum_parts_kernel(const float* __restrict__ part, int parts, int M, int N, float* __restrict__ g, int64_t ld_g, int64_t w_off,
                  const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -473,6 +479,7 @@ sum_parts_kernel(const float* __restrict__ part, int parts, int M, int N, float*
 template <class Epi>
 __global__ void __launch_bounds__(256)
 sum_parts_epi_kernel(const float* __restrict__ part, int parts, int M, int N, Epi epi, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -495,6 +502,7 @@ softmax_ce_kernel(float* logits, const int32_t* __restrict__ labels, int B, int 
                   TA* __restrict__ dz, float* __restrict__ rowloss, int* __restrict__ status, const int32_t* __restrict__ active,
                   int64_t plane = 0, const float* __restrict__ part = nullptr, int nparts = 0, const TA* __restrict__ bias = nullptr,
                   int64_t ld_p = 0, int64_t p_plane = 0) {
+  grid_dep_sync();
   __shared__ float red[8][33];
   if (active != nullptr && !active[blockIdx.y]) return;
   const int b = blockIdx.x * 32 + threadIdx.x, cg = threadIdx.y, k = blockIdx.y;
@@ -544,6 +552,7 @@ softmax_ce_kernel(float* logits, const int32_t* __restrict__ labels, int B, int 
 
 // loss[k] = mean over the minibatch of rowloss[k][b], samples added in ascending order.  grid K, block 32.
 __global__ void mean_loss_kernel(const float* __restrict__ rowloss, int B, float* __restrict__ loss, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int k = blockIdx.x;
   if (active != nullptr && !active[k]) return;
   if (threadIdx.x == 0) {
@@ -563,6 +572,7 @@ template <typename TA, typename TG>
 __global__ void __launch_bounds__(256)
 bias_grad_kernel(const TA* __restrict__ dz, int B, int out, int ldb, TG* __restrict__ g, int64_t ld_g, int64_t b_off,
                  float* __restrict__ partial, int64_t ld_partial, int slot0, const int32_t* __restrict__ active, int64_t plane = 0) {
+  grid_dep_sync();
   __shared__ float sq[8];
   if (active != nullptr && !active[blockIdx.y]) return;
   const int w = threadIdx.x >> 5, o = blockIdx.x * 8 + w;
@@ -592,6 +602,7 @@ template <typename TA>
 __global__ void __launch_bounds__(256)
 bias_grad_long_kernel(const TA* __restrict__ dz, int64_t B, int out, int64_t ldb, float* __restrict__ g, int64_t ld_g, int64_t b_off,
                       const int32_t* __restrict__ active) {
+  grid_dep_sync();
   __shared__ float ws[8];
   const int o = blockIdx.x, z = blockIdx.y;
   if (active != nullptr && !active[z]) return;
@@ -624,6 +635,7 @@ struct alignas(4) Byte4 { uint8_t v[4]; };
 template <typename T>
 __global__ void __launch_bounds__(256)
 im2col_kernel(const T* __restrict__ a, int Cin, int H, int W, int B, T* __restrict__ col, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.z;
   if (active != nullptr && !active[z]) return;
   const int P = H * W * B;
@@ -646,6 +658,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 maxpool_kernel(const T* __restrict__ r, int C, int H, int W, int B, T* __restrict__ pooled, uint8_t* __restrict__ arg,
                const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.z, c = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   const int Ho = H / 2, Wo = W / 2;
@@ -683,6 +696,7 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 unpool_kernel(const T* __restrict__ dpool, const uint8_t* __restrict__ arg, const uint8_t* __restrict__ mask, int C, int H, int W, int B,
               T* __restrict__ dz, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.z, c = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   const int P = H * W * B;
@@ -708,6 +722,7 @@ unpool_kernel(const T* __restrict__ dpool, const uint8_t* __restrict__ arg, cons
 template <typename T>
 __global__ void __launch_bounds__(256)
 col2im_kernel(const T* __restrict__ dcol, int Cin, int H, int W, int B, T* __restrict__ da, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int z = blockIdx.z, ci = blockIdx.y;
   if (active != nullptr && !active[z]) return;
   const int P = H * W * B;
@@ -740,6 +755,7 @@ __global__ void __launch_bounds__(256)
 lsq_grad_kernel(const float* __restrict__ xb, const float* __restrict__ yb, const float* __restrict__ params,
                 int64_t ld_p, int B, int in, float* __restrict__ g, int64_t ld_g, float* __restrict__ loss,
                 const int32_t* __restrict__ active) {
+  grid_dep_sync();
   extern __shared__ float res[];
   const int k = blockIdx.x;
   if (active != nullptr && !active[k]) return;

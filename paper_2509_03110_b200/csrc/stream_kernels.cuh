@@ -18,6 +18,7 @@ __global__ void __launch_bounds__(128)
 schedule_kernel(uint64_t seed, uint64_t t, int64_t n_samples, int B, int stale_max, VerHist hist, int ring,
                 int32_t* __restrict__ idx, int32_t* __restrict__ stale, int32_t* __restrict__ ver, int32_t* __restrict__ slot,
                 int K, int active_num, int64_t budget, int32_t* __restrict__ active, int k_offset) {
+  grid_dep_sync();
   __shared__ int red[4];
   const uint64_t k = blockIdx.x;
   const uint64_t kg = k + (uint64_t)k_offset;  // global worker index: the key of the minibatch and staleness streams
@@ -57,6 +58,7 @@ template <int VEC>
 __global__ void __launch_bounds__(kNormThreads)
 sumsq_partial_kernel(const float* __restrict__ g, int64_t ldg, int64_t n, float* __restrict__ partial, int64_t nchunks,
                      const int32_t* __restrict__ active) {
+  grid_dep_sync();
   __shared__ float red[kNormThreads / 32];
   const int k = blockIdx.y;
   if (active != nullptr && !active[k]) return;  // a waiting worker (block-uniform)
@@ -91,6 +93,7 @@ __global__ void __launch_bounds__(kNormThreads)
 gap_sumsq_partial_kernel(const float* __restrict__ x, int64_t ldx, const float* __restrict__ y, int64_t n,
                          float* __restrict__ partial, int64_t nchunks, const int32_t* __restrict__ slot,
                          const int32_t* __restrict__ active) {
+  grid_dep_sync();
   __shared__ float red[kNormThreads / 32];
   const int k = blockIdx.y;
   if (active != nullptr && !active[k]) return;
@@ -117,6 +120,7 @@ __global__ void __launch_bounds__(256)
 norm_finalize_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t nused, float rho, float gamma,
                      float* __restrict__ norm_out, float* __restrict__ scale_out, int* __restrict__ status,
                      const int32_t* __restrict__ active) {
+  grid_dep_sync();
   __shared__ double red[8];
   const int k = blockIdx.x;
   if (active != nullptr && !active[k]) return;
@@ -146,6 +150,7 @@ enum : int { KERNEL_GAUSSIAN = 0, KERNEL_EXP_POWER = 1, KERNEL_CAUCHY = 2, KERNE
 __global__ void __launch_bounds__(256)
 pull_weight_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t nused, int kind, float lambda, float param,
                    float* __restrict__ weight, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   __shared__ double red[8];
   const int k = blockIdx.x;
   if (active != nullptr && !active[k]) return;
@@ -168,6 +173,7 @@ pull_weight_kernel(const float* __restrict__ partial, int64_t nchunks, int64_t n
 template <int VEC, typename TG>
 __global__ void __launch_bounds__(256)
 mean_rows_kernel(const TG* g, int64_t ldg, int K, int64_t n, float* out) {
+  grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * VEC;
   if (j >= n) return;
   const float inv = 1.0f / (float)K;
@@ -221,6 +227,7 @@ __device__ inline void store_planes1(bf16* dst, int64_t plane, float a) {
 
 __global__ void __launch_bounds__(256)
 split3_rows_kernel(const float* __restrict__ src, int64_t ld_src, int64_t n, bf16* __restrict__ planes, int64_t ld, int64_t plane) {
+  grid_dep_sync();
   const int k = blockIdx.y;
   const int64_t j = ((int64_t)blockIdx.x * 256 + threadIdx.x) * 4;
   if (j >= n) return;
@@ -242,6 +249,7 @@ __global__ void __launch_bounds__(kPertThreads)
 perturb_kernel(const float* __restrict__ x, int64_t ldx, const TG* __restrict__ g, int64_t ldg, int64_t n,
                const float* __restrict__ scale, TP* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active,
                int64_t plane = 0, float* __restrict__ xt32 = nullptr) {
+  grid_dep_sync();
   const int k = blockIdx.y;
   if (active != nullptr && !active[k]) return;
   const float sc = scale[k];
@@ -303,6 +311,7 @@ constexpr int kPert8Iter = 2;
 __global__ void __launch_bounds__(kPertThreads)
 perturb8_kernel(const float* __restrict__ x, int64_t ldx, const bf16* __restrict__ g, int64_t ldg, int64_t n,
                 const float* __restrict__ scale, bf16* __restrict__ xt, int64_t ldt, const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int k = blockIdx.y;
   if (active != nullptr && !active[k]) return;
   const float sc = scale[k];
@@ -391,6 +400,7 @@ __device__ inline float update_load_g1(const void* g, int64_t idx, int mode) {
 
 template <int VEC, bool NESTEROV, typename TP, bool WRITE_OP, bool NOISE>
 __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a) {
+  grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * VEC;
   if (j >= a.n) return;
   // segment of this thread's elements (segments ascend; all VEC elements lie in one segment: starts are multiples of 64)
@@ -490,6 +500,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
 // Same arithmetic, order and noise keys as update_kernel<4, ...>.  Needs n % 8 == 0 and g_mode == 2.
 template <bool NESTEROV, bool NOISE>
 __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a) {
+  grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * 8;
   if (j >= a.n) return;
   uint32_t nseg = 0;
@@ -587,6 +598,7 @@ __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a
 // order and noise keys as update_kernel<4, ...>.  Needs n % 8 == 0, 16-byte aligned rows and g_mode == 0.
 template <bool NESTEROV, bool NOISE>
 __global__ void __launch_bounds__(kUpdThreads) update8f_kernel(const UpdateArgs a) {
+  grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * 8;
   if (j >= a.n) return;
   uint32_t nseg = 0;
@@ -672,6 +684,7 @@ __global__ void __launch_bounds__(kUpdThreads) update8f_kernel(const UpdateArgs 
 __global__ void __launch_bounds__(256)
 acc_add_kernel(const float* __restrict__ x, int64_t ld, int K, int64_t off, int64_t n, float* __restrict__ acc,
                const int32_t* __restrict__ active) {
+  grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) * 4;
   if (j >= n) return;
   float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -691,6 +704,7 @@ acc_add_kernel(const float* __restrict__ x, int64_t ld, int K, int64_t off, int6
 __global__ void __launch_bounds__(256)
 couple_kernel(float* __restrict__ acc, const float* __restrict__ y_cur, float* __restrict__ y_new,
               float* __restrict__ gprev, int64_t n, float inv_ktau, float beta, float eta_prime, int have_prev) {
+  grid_dep_sync();
   const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n) return;
   const float y = y_cur[j];
@@ -706,6 +720,7 @@ couple_kernel(float* __restrict__ acc, const float* __restrict__ y_cur, float* _
 template <typename TP>
 __global__ void __launch_bounds__(256)
 cast_rows_kernel(const float* __restrict__ src, int64_t lds, TP* __restrict__ dst, int64_t ldd, int64_t n) {
+  grid_dep_sync();
   const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (j >= n) return;
   const int k = blockIdx.y;
@@ -716,6 +731,7 @@ cast_rows_kernel(const float* __restrict__ src, int64_t lds, TP* __restrict__ ds
 template <bool TO_PADDED, typename TS, typename TD>
 __global__ void __launch_bounds__(256)
 seg_copy_kernel(const TS* __restrict__ src, int64_t lds, TD* __restrict__ dst, int64_t ldd, SegMap m) {
+  grid_dep_sync();
   const int k = blockIdx.z, sgi = blockIdx.y;
   const int64_t j = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (sgi >= m.n || j >= m.len[sgi]) return;

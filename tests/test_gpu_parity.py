@@ -801,24 +801,30 @@ def test_cuda_graph_replay_is_bitwise_identical_to_eager_launches(kind):
                                torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda(), torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
     torch.cuda.synchronize()
     stream = torch.cuda.Stream()  # the default stream cannot be captured
+    # LSAM_FLAG_PDL (kernels launched with programmatic stream serialization, each waiting for its predecessors before its
+    # first global access) must not change a bit either, launched eagerly or replayed from a graph
     with torch.cuda.stream(stream):
-        a, b = mk(0), mk(G.FLAG_CUDA_GRAPH)
-    assert b.stream.cuda_stream == stream.cuda_stream and stream.cuda_stream != 0
+        a = mk(0)
+        others = [mk(G.FLAG_CUDA_GRAPH), mk(G.FLAG_PDL), mk(G.FLAG_PDL | G.FLAG_CUDA_GRAPH)]
+    assert others[0].stream.cuda_stream == stream.cuda_stream and stream.cuda_stream != 0
     for t in range(14):
         eta = 0.02 + 0.001 * t
         rho = 0.0 if t in (4, 5, 9) else 0.03 + 0.002 * t
-        for c in (a, b):
+        for c in [a] + others:
             c.step(eta, rho)
             if c.should_couple():
                 assert c.couple() == 0
-    assert a.launch_count() == b.launch_count()
-    np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
-    np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
-    np.testing.assert_array_equal(a.read_state()["v"], b.read_state()["v"])
-    assert a.counters()[0] == b.counters()[0] and (a.counters()[2] == b.counters()[2]).all()
-    assert a.status() == 0 and b.status() == 0
+    n_a = a.launch_count()  # before the reads below, which launch copy kernels of their own
+    xa, ya, va = a.read_all_params(), a.read_params(-1), a.read_state()["v"]
+    for b in others:
+        assert n_a == b.launch_count()
+        np.testing.assert_array_equal(xa, b.read_all_params())
+        np.testing.assert_array_equal(ya, b.read_params(-1))
+        np.testing.assert_array_equal(va, b.read_state()["v"])
+        assert a.counters()[0] == b.counters()[0] and (a.counters()[2] == b.counters()[2]).all()
+        assert a.status() == 0 and b.status() == 0
+        b.close()
     a.close()
-    b.close()
 
 
 def test_step_refused_while_sync_is_due():
