@@ -541,9 +541,16 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
         if k in work and prof[k][1] > 0:
             sec = prof[k][0] * 1e-3
             tf = work[k]["flops"] * prof_steps / sec / 1e12
-            gemm[k] = dict(tflops=round(tf, 1), gbs=round(work[k]["bytes"] * prof_steps / sec / 1e9, 1),
+            gbs = work[k]["bytes"] * prof_steps / sec / 1e9
+            gemm[k] = dict(tflops=round(tf, 1), gbs=round(gbs, 1),
                            frac_of_bf16_sustained=round(tf / pk["bf16_sustained"], 3) if w["bf16"] else None,
-                           frac_of_bf16_burst=round(tf / pk["bf16"], 3) if w["bf16"] else None)
+                           frac_of_bf16_burst=round(tf / pk["bf16"], 3) if w["bf16"] else None,
+                           frac_of_measured_hbm=round(gbs / pk["hbm"], 3))
+            if w["bf16"]:
+                # which roof the shape sits under (flop per algorithmic byte against the ridge of the two measured peaks), and the
+                # fraction of that roof: time at the roof / measured time
+                t_tensor, t_hbm = tf / pk["bf16_sustained"], gbs / pk["hbm"]
+                gemm[k].update(bound="tensor" if t_tensor >= t_hbm else "hbm", frac_of_roofline=round(max(t_tensor, t_hbm), 3))
     roof["gemm_classes"] = gemm
 
     cpu = None
