@@ -30,7 +30,7 @@ LSQ, MLP, RESMLP, FLAT, CNN = 0, 1, 2, 3, 4
 # beta = 0.9, eta' = 1.  (With the look-ahead beta = 0.9 and worker momentum 0.9 the worker/centre recursion alone is
 # linearly unstable for short sync periods and weak pulls; tau = 16 with lambda0 = 0.9 is in its stable region.)
 WORKLOADS = {
-    "c1": dict(model=LSQ, widths=(256,), K=4, B=32, n=4096, classes=0, bf16=False, rho=0.05, eta=0.01, tau=4, stale_max=0, lambda0=0.5,
+    "c1": dict(model=LSQ, widths=(256,), K=4, B=32, n=4096, classes=0, bf16=False, rho=0.05, eta=0.01, tau=4, stale_max=0,
                name="least squares 4096x256, K=4, B=32"),
     "c2": dict(model=MLP, widths=(784, 1024, 10), K=8, B=128, n=60000, classes=10, bf16=False, rho=0.05, eta=0.05, tau=16,
                stale_max=0, name="MLP 784-1024-10 fp32, K=8, B=128"),
