@@ -45,6 +45,28 @@ def test_config_struct_matches_header_size(tmp_path):
     assert [getattr(G.LsamConfig, f).offset for f in fields] == out[1:]
 
 
+def test_binding_enumerators_match_the_header(tmp_path):
+    # every constant the binding mirrors, printed by a C program that includes the header
+    import subprocess
+
+    names = {"LSAM_OK": G.LSAM_OK, "LSAM_ERR_INVALID": G.LSAM_ERR_INVALID, "LSAM_ERR_WORKSPACE": G.LSAM_ERR_WORKSPACE, "LSAM_ERR_STATE": G.LSAM_ERR_STATE,
+             "LSAM_ERR_CUDA": G.LSAM_ERR_CUDA, "LSAM_ERR_NONFINITE": G.LSAM_ERR_NONFINITE, "LSAM_ERR_TIMEOUT": G.LSAM_ERR_TIMEOUT}
+    for group in ("MODEL_LSQ MODEL_MLP MODEL_RESMLP MODEL_FLAT MODEL_CNN GEMM_FP32 GEMM_BF16 IMPL_AUTO IMPL_SIMT IMPL_TCGEN05 IMPL_TCGEN05_1CTA "
+                  "IMPL_TCGEN05_PAIRS KERNEL_GAUSSIAN KERNEL_EXP_POWER KERNEL_CAUCHY KERNEL_MATERN32 FLAG_KEEP_G1 FLAG_STEP_INFO FLAG_CUDA_GRAPH "
+                  "FLAG_GRAD_FP32 FLAG_FUSED_UPDATE FLAG_PDL").split():
+        names["LSAM_" + group] = getattr(G, group)
+    names["LSAM_PROF_CLASSES"] = len(G.PROF_CLASSES)
+    for i, cls in enumerate(G.PROF_CLASSES):
+        names["LSAM_PROF_" + cls.upper()] = i
+    src = tmp_path / "enums.c"
+    keys = sorted(names)
+    src.write_text("\n".join(['#include <stdio.h>', '#include "lsam.h"', 'int main(void) {'] + [f'  printf("%d\\n", (int){k});' for k in keys] + ['  return 0;', '}']))
+    exe = tmp_path / "enums"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), "-o", str(exe), str(src)], check=True)
+    out = [int(v) for v in subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split()]
+    assert dict(zip(keys, out)) == names
+
+
 def test_param_counts_and_workspace_of_the_five_configs():
     cases = [
         (G.make_config(G.MODEL_LSQ, widths=(256,), K=4, batch=32, n_samples=4096), 256),
