@@ -499,7 +499,7 @@ __global__ void __launch_bounds__(kUpdThreads) update_kernel(const UpdateArgs a)
 // (one 128-bit load of g, two of x, v and the centre; one 128-bit store of the operand copy, two of x and v).
 // Same arithmetic, order and noise keys as update_kernel<4, ...>.  Needs n % 8 == 0 and g_mode == 2.
 template <bool NESTEROV, bool NOISE>
-__global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a) {
+__global__ void __launch_bounds__(kUpdThreads, NOISE ? 1 : 3) update8_kernel(const UpdateArgs a) {
   grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * 8;
   if (j >= a.n) return;
@@ -596,8 +596,9 @@ __global__ void __launch_bounds__(kUpdThreads) update8_kernel(const UpdateArgs a
 // fp32 counterpart of update8_kernel (gradient fp32 used as is, no operand copy): 8 consecutive elements per thread, i.e.
 // two 128-bit accesses to each of g, x, v and the centre per replica, software-pipelined over the replicas.  Same arithmetic,
 // order and noise keys as update_kernel<4, ...>.  Needs n % 8 == 0, 16-byte aligned rows and g_mode == 0.
+// Compiled for three blocks per SM (80 registers): at 90 registers only two fit and the kernel streamed 5 % slower.
 template <bool NESTEROV, bool NOISE>
-__global__ void __launch_bounds__(kUpdThreads) update8f_kernel(const UpdateArgs a) {
+__global__ void __launch_bounds__(kUpdThreads, NOISE ? 1 : 3) update8f_kernel(const UpdateArgs a) {
   grid_dep_sync();
   const int64_t j = ((int64_t)blockIdx.x * kUpdThreads + threadIdx.x) * 8;
   if (j >= a.n) return;
