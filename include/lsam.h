@@ -159,6 +159,8 @@ size_t lsam_workspace_bytes(const lsam_config* cfg);
  *  d_x0 [K, d] fp32 device, d_y0 [d] fp32 device: copied into the workspace.
  *  d_workspace: >= lsam_workspace_bytes() bytes, 256-byte aligned, owned by the caller, must outlive the context.
  *  cuda_stream: a cudaStream_t (NULL = default stream).
+ * d_x0 and d_y0 are read, and d_X / d_Y are read by every later tick, ON cuda_stream: whatever produced them must be ordered before
+ * this call on that stream (a non-blocking side stream does not wait for the default stream: synchronise or use an event first).
  * Errors: LSAM_ERR_INVALID, LSAM_ERR_WORKSPACE, LSAM_ERR_CUDA; *out is NULL on failure. */
 int lsam_init(lsam_ctx** out, const lsam_config* cfg, const void* d_X, const void* d_Y, const float* d_x0,
               const float* d_y0, void* d_workspace, size_t workspace_bytes, void* cuda_stream);

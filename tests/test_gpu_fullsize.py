@@ -234,3 +234,33 @@ def test_c4_full_shape_one_tick_of_all_32_replicas_against_oracle_on_two():
         assert rel_l2(got_x - x0_rows[k], want_x - x0_rows[k]) <= TOL_GRAD_BF16_FULL, (k, rel_l2(got_x - x0_rows[k], want_x - x0_rows[k]))
         assert median_abs_rows(got_x, want_x) <= TOL_TRAJ_BF16 / BULK_DIVISOR
     ctx.close()
+
+
+@pytest.mark.parametrize("key,K", [("c3", 16), ("c4", 4)])
+def test_bench_launch_configuration_is_bitwise_identical_to_plain_launches_at_full_shapes(key, K):
+    # bench.py replays each tick as a CUDA graph whose tensor-core GEMMs carry the programmatic-stream-serialization
+    # attribute (their blocks become resident while the kernel before drains, and wait for it before touching memory).  At
+    # the full layer shapes (several tiles per CTA, CTA pairs, weight-gradient runs) that must not change a bit against
+    # plain in-order launches of the same kernels, which the tests above hold against the oracle.
+    import torch
+
+    dev = torch.device("cuda", 0)
+    w, inp = _inputs(bench.WORKLOADS[key], dev, K=K)
+    w["tau"] = 2  # a sync every second tick: the update's stale reads and the centre update are inside the compared run
+    torch.cuda.synchronize()  # the inputs were generated on torch's default stream, which a side stream does not wait for
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        ctxs = [G.Lsam(bench.make_cfg(G, w, flags=fl), inp["X"], inp["Y"], inp["x0"], inp["y0"]) for fl in (0, G.FLAG_CUDA_GRAPH | G.FLAG_PDL)]
+    assert all(c.uses_tcgen05() for c in ctxs)
+    for t in range(5):
+        for c in ctxs:
+            c.step(w["eta"], w["rho"])
+            if c.should_couple():
+                assert c.couple() == 0
+    a, b = ctxs
+    assert a.status() == 0 and b.status() == 0 and a.launch_count() == b.launch_count()
+    for k in (0, K - 1):
+        np.testing.assert_array_equal(a.read_params(k), b.read_params(k))
+    np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
+    for c in ctxs:
+        c.close()
