@@ -552,6 +552,17 @@ def run_workload(key, w, steps, warmup, dev, rank, world, shard=False, cuda_grap
                 t_tensor, t_hbm = tf / pk["bf16_sustained"], gbs / pk["hbm"]
                 gemm[k].update(bound="tensor" if t_tensor >= t_hbm else "hbm", frac_of_roofline=round(max(t_tensor, t_hbm), 3))
     roof["gemm_classes"] = gemm
+    # the whole step against both roofs: algorithmic bytes and flops of every kernel class over the device-timed step
+    # (the kernels run one after another, so the sum of the per-kernel floors, not their maximum, bounds the step)
+    step_bytes = sum(v.get("bytes", 0.0) for v in work.values())
+    step_flops = sum(v.get("flops", 0.0) for v in work.values())
+    if step_bytes > 0 and not small:
+        floor_s = sum(max(v.get("bytes", 0.0) / (pk["hbm"] * 1e9), (v.get("flops", 0.0) / (pk["bf16_sustained"] * 1e12)) if (uses_tc and not x3) else 0.0)
+                      for v in work.values())
+        roof["whole_step"] = dict(bytes=step_bytes, flops=step_flops, gbs=round(step_bytes / (ms_step * 1e-3) / 1e9, 1),
+                                  frac_of_measured_hbm=round(step_bytes / (ms_step * 1e-3) / 1e9 / pk["hbm"], 3),
+                                  floor_ms=round(floor_s * 1e3, 3), frac_of_floor=round(floor_s * 1e3 / ms_step, 3),
+                                  floor="sum over the kernel classes of max(bytes / measured HBM rate, flops / sustained bf16 rate)")
 
     cpu = None
     if with_cpu:
