@@ -1013,3 +1013,40 @@ def test_random_shapes_every_gemm_form_against_oracle(seed):
         with pytest.raises(G.LsamError):
             Pair(G.MODEL_RESMLP if res else G.MODEL_MLP, widths=widths, K=K, batch=B, X=X, Y=labels, x0=x0, y0=w0, gemm_dtype=G.GEMM_BF16,
                  gemm_impl=G.IMPL_TCGEN05, tau=2, lam=0.4, seed=seed)
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 5, 8, 12, 17])
+def test_random_combinations_of_variants_against_oracle(seed):
+    # the variants are tested one at a time above; here a seeded draw combines them (sync period, pull, staleness window,
+    # heavy-ball / Nesterov, unequal progress, Langevin noise, non-Gaussian kernels, synchronous gradient averaging) on a
+    # drawn classifier shape, eight free-running ticks with one tick of radius zero, on three GEMM forms
+    rng = np.random.default_rng(9000 + seed)
+    nl = int(rng.integers(2, 4))
+    widths = tuple([int(rng.integers(2, 40)) * 8 for _ in range(nl)] + [int(rng.integers(2, 120))])
+    K = int(rng.integers(2, 6))
+    B = int(rng.choice([16, 32, 48, 64, 128, 200, 256]))
+    dp = int(rng.integers(0, 4) == 0)
+    hp = dict(tau=1 if dp else int(rng.integers(1, 5)), lam=float(rng.uniform(0.1, 0.6)), seed=seed, stale_max=0 if dp else int(rng.integers(0, 4)),
+              nesterov=int(rng.integers(0, 2)), dp_average=dp)
+    if not dp and rng.integers(0, 2):
+        hp["active_num"] = int(rng.integers(100, 250))
+    if not dp and rng.integers(0, 3) == 0:
+        hp["noise_temp"] = 1e-4
+    kk = int(rng.integers(0, 4))
+    if kk:
+        hp["kernel_kind"] = kk
+        hp["kernel_param"] = float(rng.uniform(1.2, 1.9)) if kk == G.KERNEL_EXP_POWER else float(rng.uniform(0.5, 2.0))
+    X, labels = synth.gaussian_mixture(400, widths[0], widths[-1], seed=seed)
+    w0 = synth.mlp_init(widths, seed=seed)
+    x0 = synth.replicate(w0, K, jitter=0.02, seed=seed)
+    for name, dt, impl, tol in (("bf16 tcgen05", G.GEMM_BF16, G.IMPL_TCGEN05, TOL_TRAJ_BF16), ("fp32 simt", G.GEMM_FP32, G.IMPL_SIMT, TOL_TRAJ_FP32),
+                                ("fp32 on tcgen05", G.GEMM_FP32, G.IMPL_TCGEN05, TOL_TRAJ_FP32)):
+        p = Pair(G.MODEL_MLP, widths=widths, K=K, batch=B, X=X, Y=labels, x0=x0, y0=w0, gemm_dtype=dt, gemm_impl=impl, flags=G.FLAG_STEP_INFO, **hp)
+        for t in range(8):
+            p.step(0.03, 0.05 if t != 3 else 0.0)
+            p.couple_if_due()
+        e = p.errors()
+        what = (name, widths, K, B, hp)
+        assert e["x"] <= tol and e["y"] <= tol and p.gpu.status() == 0, (what, e)
+        assert p.gpu.counters()[:2] == p.oracle.counters()[:2] and (p.gpu.counters()[2] == p.oracle.counters()[2]).all(), what
+        p.close()
