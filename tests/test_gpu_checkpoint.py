@@ -17,8 +17,8 @@ def _make(kind):
         x0, y0, g1, g2 = synth.flat_problem(4, 1001, seed=6)
         dg = [torch.from_numpy(g1).cuda(), torch.from_numpy(g2).cuda()]
 
-        def mk(x_init):
-            c = G.Lsam(G.make_config(G.MODEL_FLAT, K=4, flat_d=1001, noise_temp=0.05, **HP), None, None, torch.from_numpy(x_init).cuda(), torch.from_numpy(y0).cuda())
+        def mk(x_init, flags=0):
+            c = G.Lsam(G.make_config(G.MODEL_FLAT, K=4, flat_d=1001, noise_temp=0.05, flags=flags, **HP), None, None, torch.from_numpy(x_init).cuda(), torch.from_numpy(y0).cuda())
             c.set_external_grads(*dg)  # borrowed buffers are the caller's to supply again after a resume
             return c
         return mk, x0
@@ -29,7 +29,7 @@ def _make(kind):
     x0 = synth.replicate(w0, 3, jitter=0.01)
     extra = dict(noise_temp=1e-3) if bf else dict(active_num=170)
     dX, dY = torch.from_numpy(X).cuda(), torch.from_numpy(labels).cuda()
-    mk = lambda x_init: G.Lsam(G.make_config(G.MODEL_RESMLP if bf else G.MODEL_MLP, widths=widths, K=3, batch=48, n_samples=300,
+    mk = lambda x_init, flags=0: G.Lsam(G.make_config(G.MODEL_RESMLP if bf else G.MODEL_MLP, widths=widths, K=3, batch=48, n_samples=300, flags=flags,
                                              gemm_dtype=G.GEMM_BF16 if bf else G.GEMM_FP32,
                                              gemm_impl=G.IMPL_TCGEN05 if kind == "mlp_fp32_tcgen05_async" else G.IMPL_AUTO, **extra, **HP),
                                dX, dY, torch.from_numpy(x_init).cuda(), torch.from_numpy(w0).cuda())
@@ -73,6 +73,35 @@ def test_resumed_run_continues_bit_for_bit(kind):
         o.load_checkpoint(np.concatenate([blob, np.zeros(1 << 22, np.uint8)]))
     for c in (a, b, o):
         c.close()
+
+
+@pytest.mark.parametrize("kind", ["flat", "mlp_fp32_tcgen05_async", "resmlp_bf16_tcgen05"])
+def test_resume_into_a_graph_replaying_context(kind):
+    # saved by a context that launches its kernels plainly, resumed by one that replays each tick as a CUDA graph with
+    # programmatic dependent launch and has already recorded its graphs on another trajectory: tick, centre-version history
+    # and budget of the resumed run must reach the recorded graphs, so the two runs end bit for bit equal
+    import torch
+
+    mk, x0 = _make(kind)
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()  # the default stream cannot be captured
+    with torch.cuda.stream(stream):
+        a = mk(x0)
+        b = mk(x0 * 0.5, G.FLAG_CUDA_GRAPH | G.FLAG_PDL)
+    _run(a, 0, 8)
+    _run(b, 0, 5)                      # graphs of every tick variant are recorded here
+    blob = a.save_checkpoint()
+    b.load_checkpoint(blob)
+    _run(a, 8, 15)
+    _run(b, 8, 15)
+    np.testing.assert_array_equal(a.read_all_params(), b.read_all_params())
+    np.testing.assert_array_equal(a.read_params(-1), b.read_params(-1))
+    np.testing.assert_array_equal(a.read_state()["v"], b.read_state()["v"])
+    ca, cb = a.counters(), b.counters()
+    assert ca[0] == cb[0] and ca[1] == cb[1] and (ca[2] == cb[2]).all()
+    assert a.status() == 0 and b.status() == 0
+    a.close()
+    b.close()
 
 
 def test_load_drops_staged_minibatches_and_refuses_inconsistent_counters():
