@@ -477,7 +477,8 @@ def test_staged_prefetch_matches_step_batch(model):
     s = torch.cuda.Stream()
     with torch.cuda.stream(s):
         a = G.Lsam(G.make_config(mk, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
-        b = G.Lsam(G.make_config(mk, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
+        # the staged run in the launch configuration of bench.py's end-to-end figure: graph replay, programmatic dependent launch
+        b = G.Lsam(G.make_config(mk, flags=G.FLAG_CUDA_GRAPH | G.FLAG_PDL, **kw), dX, dY, torch.from_numpy(x0).cuda(), torch.from_numpy(w0).cuda())
         with pytest.raises(G.LsamError):
             b.step_staged(0.05, 0.05)  # nothing staged
         batches = []
